@@ -1,0 +1,372 @@
+"""Pins for the CPU oracle: every function is checked against something other than itself --
+hand-worked values (tests/golden), closed forms, invariants, special cases that reduce to a
+numpy/torch library routine, and brute force on tiny inputs.  No GPU needed."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_05168_b200 import inputs
+
+
+def _read_golden(path):
+    out = {}
+    with open(path) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = [float(v) for v in vals]
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# Hand-worked example: Eq. 1-3 order, layout, and the negative control (mask-then-quant).
+# ------------------------------------------------------------------------------------------------
+def test_worked_example_quant_then_mask(golden_dir):
+    g = _read_golden(os.path.join(golden_dir, "quant_then_mask_worked_example.txt"))
+    W = np.array([g["W"]], np.float32)
+    r = oracle.quantize_mask_pack(W)
+    assert r["scale"] == np.float32(g["gamma"][0])
+    assert r["dense_q"].tolist() == [[int(v) for v in g["dense_q"]]]
+    assert r["mask"].tolist() == [[int(v) for v in g["mask"]]]
+    assert r["vals"].tolist() == [[int(v) for v in g["vals"]]]
+    assert r["meta"].tolist() == [[int(v) for v in g["meta"]]]
+    weff, mask = oracle.unpack24(r["vals"], r["meta"])
+    assert weff.tolist() == [[int(v) for v in g["weff"]]]
+    # negative control: quantising the masked weights with the masked-subset gamma gives another
+    # answer; the oracle must NOT produce it.
+    Wm = (W * r["mask"]).astype(np.float32)
+    gam_c, scale_c, _ = oracle.absmean_scale(Wm)
+    assert gam_c == np.float32(g["control_gamma"][0])
+    control = oracle.ternarize(Wm, scale_c)
+    assert control.tolist() == [[int(v) for v in g["control_weff"]]]
+    assert control.tolist() != weff.tolist()
+
+
+def test_order_matters_on_gaussian():
+    # With gamma fixed, mask(.)Q(w) == Q(mask(.)w); only gamma differs.  For Gaussian W the
+    # masked-subset mean is ~0.7446 of the dense mean and ~1.4 % of W_eff entries change.
+    W = inputs.latent_weights(512, 1024, seed=11)
+    r = oracle.quantize_mask_pack(W)
+    weff, mask = oracle.unpack24(r["vals"], r["meta"])
+    assert np.array_equal(oracle.ternarize((W * mask).astype(np.float32), r["scale"]), weff)
+    Wm = (W * mask).astype(np.float32)
+    gm, sm, _ = oracle.absmean_scale(Wm)
+    # E|w| over the two largest of four iid half-normals, halved by the mask: closed form is
+    # awkward, so only a bracket is asserted here; the ratio is far from 1 either way.
+    assert 0.72 < gm / r["scale"] < 0.77
+    control = oracle.ternarize(Wm, sm)
+    frac = np.mean(control != weff)
+    assert 0.008 < frac < 0.02
+
+
+# ------------------------------------------------------------------------------------------------
+# Eq. 1 scale: closed forms.
+# ------------------------------------------------------------------------------------------------
+def test_gamma_closed_forms():
+    # |W| == c (power of two) -> gamma == c exactly, all q = sign
+    rng = np.random.default_rng(0)
+    sign = rng.choice([-1.0, 1.0], size=(32, 64)).astype(np.float32)
+    W = sign * np.float32(0.25)
+    g, s, _ = oracle.absmean_scale(W)
+    assert g == np.float32(0.25) and s == np.float32(0.25)
+    assert np.array_equal(oracle.ternarize(W, s), sign.astype(np.int8))
+    # W == 0 -> scale is the clamp 1e-5, all q = 0
+    Z = np.zeros((8, 16), np.float32)
+    g, s, _ = oracle.absmean_scale(Z)
+    assert g == 0.0 and s == np.float32(1e-5)
+    assert not oracle.ternarize(Z, s).any()
+    # tiny weights below the clamp: gamma < 1e-5 but scale = 1e-5
+    Tn = np.full((8, 16), 1e-7, np.float32)
+    g, s, _ = oracle.absmean_scale(Tn)
+    assert s == np.float32(1e-5) and g < s
+    # mean of 1..8 in a known arrangement
+    A = np.array([[1, -2, 3, -4, 5, -6, 7, -8]], np.float32)
+    g, s, _ = oracle.absmean_scale(A)
+    assert g == np.float32(4.5)
+
+
+def test_ternary_inputs_are_a_fixed_point():
+    # W = c * t with t ternary and non-zero fraction f: gamma = f*c, |w|/gamma = 1/f >= 1 > 0.5
+    rng = np.random.default_rng(1)
+    t = rng.choice([-1, 0, 1], size=(64, 128), p=[0.3, 0.4, 0.3]).astype(np.int8)
+    W = t.astype(np.float32) * np.float32(0.037)
+    _, s, _ = oracle.absmean_scale(W)
+    assert np.array_equal(oracle.ternarize(W, s), t)
+
+
+def test_ternarize_matches_numpy_rint_division():
+    # special case that reduces to library routines: fp32 division, rint (half-even), clip
+    W = inputs.latent_weights(128, 256, seed=2)
+    _, s, _ = oracle.absmean_scale(W)
+    ref = np.clip(np.rint(W / np.float32(s)), -1, 1).astype(np.int8)
+    assert np.array_equal(oracle.ternarize(W, s), ref)
+    # exact halves: 0.5 -> 0, 1.5 -> 2 -> clamp 1, -0.5 -> 0, 2.5 -> 1
+    H = np.array([[0.5, -0.5, 1.5, -1.5, 2.5, 0.49999997, 0.50000006, -0.50000006]], np.float32)
+    assert oracle.ternarize(H, 1.0).tolist() == [[0, 0, 1, -1, 1, 0, 1, -1]]
+
+
+def test_scale_uses_max_not_sum_for_epsilon():
+    # gamma + 1e-5 and max(gamma, 1e-5) disagree visibly when gamma ~ 1e-5
+    W = np.full((4, 8), 1.6e-5, np.float32)
+    _, s, _ = oracle.absmean_scale(W)
+    assert s == np.float32(1.6e-5)
+    assert (oracle.ternarize(W, s) == 1).all()
+
+
+def test_power_of_two_and_sign_invariance():
+    W = inputs.latent_weights(64, 256, seed=3)
+    r = oracle.quantize_mask_pack(W)
+    for j in (-3, 5):
+        r2 = oracle.quantize_mask_pack((W * np.float32(2.0 ** j)).astype(np.float32))
+        assert np.array_equal(r2["vals"], r["vals"]) and np.array_equal(r2["meta"], r["meta"])
+        assert r2["scale"] == np.float32(r["scale"] * np.float32(2.0 ** j))
+    rn = oracle.quantize_mask_pack(-W)
+    assert np.array_equal(rn["vals"], -r["vals"]) and np.array_equal(rn["meta"], r["meta"])
+
+
+# ------------------------------------------------------------------------------------------------
+# Eq. 2 mask: invariants and brute force.
+# ------------------------------------------------------------------------------------------------
+LEGAL_NIBBLES = {4, 8, 12, 9, 13, 14}
+
+
+def _brute_mask(W, n_keep, m_group):
+    N, K = W.shape
+    out = np.zeros((N, K), np.uint8)
+    for n in range(N):
+        for g in range(K // m_group):
+            a = [abs(float(W[n, g * m_group + j])) for j in range(m_group)]
+            order = sorted(range(m_group), key=lambda j: (-a[j], j))
+            for j in order[:n_keep]:
+                out[n, g * m_group + j] = 1
+    return out
+
+
+@pytest.mark.parametrize("n_keep,m_group", [(2, 4), (6, 8), (1, 4), (4, 8)])
+def test_mask_brute_force_and_invariants(n_keep, m_group):
+    rng = np.random.default_rng(4)
+    W = rng.standard_normal((16, 64)).astype(np.float32)
+    # inject ties, zeros and sign-mirrored duplicates
+    W[0, :8] = 0.0
+    W[1, :8] = [1, -1, 1, -1, 2, 2, -2, 2]
+    W[2, :8] = [0.5, 0.25, 0.5, 0.25, 0, 0, 1, 0]
+    mask = oracle.nm_mask(W, n_keep, m_group)
+    assert np.array_equal(mask, _brute_mask(W, n_keep, m_group))
+    grp = mask.reshape(16, -1, m_group)
+    assert (grp.sum(-1) == n_keep).all()
+    a = np.abs(W).reshape(16, -1, m_group)
+    kept_min = np.where(grp == 1, a, np.inf).min(-1)
+    drop_max = np.where(grp == 0, a, -np.inf).max(-1)
+    assert (kept_min >= drop_max).all()
+
+
+def test_mask_ties_keep_lower_columns():
+    W = np.zeros((1, 8), np.float32)
+    W[0, 4:] = 3.0
+    assert oracle.nm_mask(W).tolist() == [[1, 1, 0, 0, 1, 1, 0, 0]]
+
+
+def test_mask_comes_from_master_weights_not_from_ternary():
+    # group whose ternary image is all ones: only the fp32 magnitudes can rank it
+    W = np.array([[0.9, 1.3, 1.1, 1.2, 5, 5, 5, 5]], np.float32)
+    mask = oracle.nm_mask(W)
+    assert mask[0, :4].tolist() == [0, 1, 0, 1]
+
+
+def test_pack_layout_and_roundtrip():
+    W = inputs.latent_weights(32, 128, seed=5)
+    r = oracle.quantize_mask_pack(W)
+    assert set(np.unique(r["vals"]).tolist()) <= {-1, 0, 1}
+    nibs = np.concatenate([(r["meta"] & 15).ravel(), (r["meta"] >> 4).ravel()])
+    assert set(np.unique(nibs).tolist()) <= LEGAL_NIBBLES
+    weff, mask = oracle.unpack24(r["vals"], r["meta"])
+    assert np.array_equal(mask, r["mask"])
+    assert np.array_equal(weff, r["dense_q"] * r["mask"].astype(np.int8))
+    # explicit layout on one group: columns 1 and 3 kept -> nibble 1 | 3<<2 = 13
+    q = np.array([[0, 1, 0, -1, 1, 0, 0, 1]], np.int8)
+    m = np.array([[0, 1, 0, 1, 1, 0, 0, 1]], np.uint8)
+    vals, meta = oracle.pack24(q, m)
+    assert vals.tolist() == [[1, -1, 1, 1]]
+    assert meta.tolist() == [[13 | (12 << 4)]]
+    with pytest.raises(ValueError):
+        oracle.pack24(q, np.array([[1, 1, 1, 0, 1, 0, 0, 1]], np.uint8))
+
+
+def test_gaussian_closed_forms(golden_dir):
+    g = _read_golden(os.path.join(golden_dir, "gaussian_closed_forms.txt"))
+    sigma = 0.02
+    N, K = 1024, 2048
+    W = inputs.latent_weights(N, K, seed=6, sigma=sigma)
+    r = oracle.quantize_mask_pack(W)
+    tol = 4.0 / math.sqrt(N * K)
+    assert abs(r["scale"] / sigma - g["gamma_over_sigma"][0]) < 2e-3
+    assert abs(np.mean(r["dense_q"] == 0) - g["p_zero"][0]) < tol * 2
+    assert abs(np.mean(r["vals"] == 0) - g["kept_zero_fraction"][0]) < tol * 2
+    weff, _ = oracle.unpack24(r["vals"], r["meta"])
+    assert abs(np.mean(weff != 0) - g["weff_density"][0]) < tol * 2
+
+
+# ------------------------------------------------------------------------------------------------
+# Activation quantiser: closed forms.
+# ------------------------------------------------------------------------------------------------
+def _bf16(a):
+    return inputs.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def test_quant_act_integer_rows_are_identity():
+    rng = np.random.default_rng(7)
+    x = rng.integers(-127, 128, size=(16, 64)).astype(np.float32)
+    x[:, 0] = 127.0 * rng.choice([-1, 1], size=16)
+    xq, s = oracle.quant_act(_bf16(x))
+    assert np.array_equal(xq, x.astype(np.int8))
+    assert (s == np.float32(1.0)).all()
+
+
+def test_quant_act_half_to_even_and_zero_row():
+    x = np.zeros((3, 8), np.float32)
+    x[0] = [127, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5]
+    x[2] = [-127, 126.5, 125.5, 0, 0, 0, 0, 0]
+    xq, s = oracle.quant_act(_bf16(x))
+    assert xq[0].tolist() == [127, 0, 2, 2, 0, -2, -2, 4]
+    assert not xq[1].any() and s[1] == np.float32(np.float32(1e-5) / np.float32(127.0))
+    assert xq[2].tolist()[:3] == [-127, 126, 126]   # 126.5 -> 126 (even); 125.5 -> 126 (bf16: 125.5 exact)
+
+
+def test_quant_act_properties():
+    x = inputs.activations_bf16(64, 512, seed=8)
+    xq, s = oracle.quant_act(x)
+    xf = inputs.bf16_bits_to_f32(x)
+    am = np.abs(xf).argmax(1)
+    assert (np.abs(xq[np.arange(64), am].astype(np.int32)) == 127).all()
+    assert xq.min() >= -127 and xq.max() <= 127
+    assert np.array_equal(s, (np.abs(xf).max(1) / np.float32(127.0)).astype(np.float32))
+    # scaling by a power of two leaves the codes unchanged and scales a_scale exactly
+    xq2, s2 = oracle.quant_act(_bf16(xf * np.float32(8.0)))
+    assert np.array_equal(xq2, xq) and np.array_equal(s2, s * np.float32(8.0))
+    # the multiply-by-s_x form, as numpy does it in fp32
+    sx = (np.float32(127.0) / np.maximum(np.abs(xf).max(1, keepdims=True), np.float32(1e-5))).astype(np.float32)
+    ref = np.clip(np.rint(xf * sx), -128, 127).astype(np.int8)
+    assert np.array_equal(xq, ref)
+
+
+# ------------------------------------------------------------------------------------------------
+# Eq. 4: integer accumulation and scaling.
+# ------------------------------------------------------------------------------------------------
+def test_acc_brute_force_tiny():
+    rng = np.random.default_rng(9)
+    T, N, K = 5, 6, 16
+    xq = rng.integers(-127, 128, size=(T, K)).astype(np.int8)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    r = oracle.quantize_mask_pack(W)
+    weff, _ = oracle.unpack24(r["vals"], r["meta"])
+    brute = [[sum(int(xq[t, k]) * int(weff[n, k]) for k in range(K)) for n in range(N)] for t in range(T)]
+    assert oracle.acc_packed(xq, r["vals"], r["meta"]).tolist() == brute
+    assert oracle.acc_dense(xq, weff).tolist() == brute
+    brute_d = [[sum(int(xq[t, k]) * int(r["dense_q"][n, k]) for k in range(K)) for n in range(N)] for t in range(T)]
+    assert oracle.acc_dense(xq, r["dense_q"]).tolist() == brute_d
+
+
+def test_acc_routes_agree_with_int64_matmul():
+    W = inputs.latent_weights(96, 256, seed=10)
+    x = inputs.activations_bf16(40, 256, seed=11)
+    r = oracle.quantize_mask_pack(W)
+    xq, s = oracle.quant_act(x)
+    weff, mask = oracle.unpack24(r["vals"], r["meta"])
+    ref = xq.astype(np.int64) @ weff.astype(np.int64).T
+    a1 = oracle.acc_dense(xq, weff)
+    a2 = oracle.acc_packed(xq, r["vals"], r["meta"])
+    assert np.array_equal(a1, ref) and np.array_equal(a2, ref)
+    assert np.abs(ref).max() <= 127 * 256 // 2
+    # dense minus sparse is exactly the pruned part
+    ad = oracle.acc_dense(xq, r["dense_q"])
+    pruned = xq.astype(np.int64) @ (r["dense_q"].astype(np.int64) * (1 - mask.astype(np.int64))).T
+    assert np.array_equal(ad - a1, pruned)
+    # sampled variants agree with the full ones
+    t_idx, n_idx = inputs.sample_positions(40, 96, 50, seed=1)
+    assert np.array_equal(oracle.acc_packed_sampled(xq, r["vals"], r["meta"], t_idx, n_idx), ref[t_idx, n_idx])
+    assert np.array_equal(oracle.acc_dense_sampled(xq, r["dense_q"], t_idx, n_idx), ad[t_idx, n_idx])
+
+
+def test_exact_integer_layer():
+    # integer activations (s_x = 1) and ternary weights (fixed point): no quantisation error at
+    # all, so y equals gamma * (X @ (W (.) mask)^T) with an exact integer product
+    rng = np.random.default_rng(12)
+    T, N, K = 8, 16, 64
+    X = rng.integers(-127, 128, size=(T, K)).astype(np.float32)
+    X[:, 0] = 127
+    tern = rng.choice([-1, 0, 1], size=(N, K)).astype(np.int8)
+    tern[0, :4] = [1, 1, 1, 1]     # forces a pruning decision among equal magnitudes
+    c = np.float32(0.5)
+    W = tern.astype(np.float32) * c
+    r = oracle.quantize_mask_pack(W)
+    xq, s = oracle.quant_act(_bf16(X))
+    y, acc = oracle.sparse_bitlinear(xq, s, r["vals"], r["meta"], r["scale"])
+    mask = oracle.nm_mask(W)
+    ref = X.astype(np.int64) @ (tern.astype(np.int64) * mask).T
+    assert np.array_equal(acc, ref)
+    assert np.allclose(y, np.float64(r["scale"]) * ref, rtol=1e-6)
+
+
+def test_dequant_association_and_bias():
+    acc = np.array([[3, -5], [70000, 1]], np.int32)
+    a_scale = np.array([0.5, 0.25], np.float32)
+    y = oracle.dequant(acc, 2.0, a_scale)
+    assert y.tolist() == [[3.0, -5.0], [35000.0, 0.5]]
+    yb = oracle.dequant(acc, 2.0, a_scale, np.array([1.0, -1.0], np.float32))
+    assert yb.tolist() == [[4.0, -6.0], [35001.0, -0.5]]
+    # generic scales: float(acc) * fl(scale * a_scale), each product rounded once
+    rng = np.random.default_rng(13)
+    acc = rng.integers(-300000, 300000, size=(7, 9)).astype(np.int32)
+    a_scale = rng.random(7).astype(np.float32)
+    sc = np.float32(0.0159)
+    s = (sc * a_scale).astype(np.float32)
+    ref = (acc.astype(np.float32) * s[:, None]).astype(np.float32)
+    assert np.array_equal(oracle.dequant(acc, sc, a_scale), ref)
+    rel = np.abs(ref.astype(np.float64) / (np.float64(sc) * a_scale.astype(np.float64))[:, None] - acc)
+    assert (rel <= 2 * np.abs(acc) * 2.0 ** -23 + 1e-9).all()
+
+
+def test_bf16_rounding_matches_torch():
+    rng = np.random.default_rng(14)
+    y = rng.standard_normal(4096).astype(np.float32) * np.float32(37.0)
+    y[:4] = [1.00390625, 1.01171875, -1.00390625, 3.0]    # exact halves between bf16 neighbours
+    ref = torch.from_numpy(y).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(oracle.f32_to_bf16_bits(y), ref)
+    assert np.array_equal(inputs.f32_to_bf16_bits(y), ref)
+
+
+# ------------------------------------------------------------------------------------------------
+# Flip rate.
+# ------------------------------------------------------------------------------------------------
+def test_flip_count_cases():
+    W = inputs.latent_weights(64, 256, seed=15)
+    m0 = oracle.nm_mask(W)
+    assert oracle.flip_count(m0, m0) == 0
+    # swap the 2nd and 3rd magnitudes of one group -> exactly two positions change
+    W2 = W.copy()
+    grp = np.abs(W2[3, 8:12])
+    order = np.argsort(-grp)
+    j2, j3 = 8 + order[1], 8 + order[2]
+    W2[3, j2], W2[3, j3] = W2[3, j3], W2[3, j2]
+    m1 = oracle.nm_mask(W2)
+    assert oracle.flip_count(m0, m1) == 2
+    # per group the count is 0, 2 or 4
+    Wp = inputs.perturb_weights(W, seed=16, sigma=5e-3)
+    mp = oracle.nm_mask(Wp)
+    per_group = (m0 != mp).reshape(64, -1, 4).sum(-1)
+    assert set(np.unique(per_group).tolist()) <= {0, 2, 4}
+    assert oracle.flip_count(m0, mp) == int(per_group.sum())
+
+
+def test_flip_rate_of_the_dynamic_mask_workload():
+    # W ~ N(0, 0.02), one step W += N(0, 1e-4): the flip rate of the 2:4 mask is a few 1e-3
+    W = inputs.latent_weights(1024, 2560, seed=17)
+    Wp = inputs.perturb_weights(W, seed=18, sigma=1e-4)
+    r = oracle.flip_count(oracle.nm_mask(W), oracle.nm_mask(Wp)) / W.size
+    assert 2.5e-3 < r < 4.5e-3
