@@ -1,0 +1,171 @@
+/*
+ * sbn.h -- C ABI of libsbn: the 2:4-sparse ternary BitLinear layer of Sparse-BitNet on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the forward hot path of the Sparse-BitLinear layer (Sec. 2.2, Eq. 2-4,
+ * Algorithm 2) and of the dense BitLinear it is compared with (Sec. 2.1, Eq. 1):
+ *
+ *   part 1  sbn_quantize_mask_pack   W (fp32 master weights) -> ternary W_q (Eq. 1), 2:4 mask from
+ *                                    |W| of the pre-quantised weights (Eq. 2), W_eff = W_q (.) M
+ *                                    (Eq. 3), stored as compressed values + 2-bit index metadata
+ *   part 2  sbn_quant_act            x (bf16) -> per-token absmax int8 x~ and its scale (Sec. 2.1)
+ *   part 3  sbn_sparse_bitlinear     y = s * (W_eff x~) (Eq. 4): sparse int8 tensor-core GEMM,
+ *                                    int32 accumulation, scales applied in the epilogue
+ *   base    sbn_bitlinear            y = gamma * matmul(W_q, x~) (Sec. 2.1), dense int8 GEMM
+ *
+ * Notation: T = tokens, K = d_in, N = d_out.  All matrices are row-major.
+ *
+ * General rules
+ *   - Every pointer marked "device" is a CUDA device pointer owned by the caller.  The library
+ *     never allocates or frees device memory and keeps no reference after the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *     work on it; nothing here synchronises except sbn_check_status.
+ *   - Errors are return codes.  Argument errors are detected on the host before anything is
+ *     launched.  Device-side waits are bounded; a wait that runs out records SBN_ERR_TIMEOUT in a
+ *     device status word that sbn_check_status reads back.
+ *   - Inputs must be finite.  NaN/Inf give unspecified results.
+ *   - Shape limits of the GPU path: N % 128 == 0, K % 128 == 0, T >= 1, K <= 2^20, pointers
+ *     16-byte aligned (cudaMalloc alignment is always enough).
+ *
+ * Compressed 2:4 layout (the paper leaves the layout to the kernel; this is the library's):
+ *   groups are 4 consecutive columns of a row, aligned to column 0; group g of row n keeps the
+ *   columns 4g+i0 < 4g+i1;
+ *     vals[n][2g]   = W_q[n][4g+i0],  vals[n][2g+1] = W_q[n][4g+i1]          int8  [N][K/2]
+ *     nibble(g)     = i0 | (i1 << 2)
+ *     meta[n][b]    = nibble(2b) | (nibble(2b+1) << 4)                       uint8 [N][K/8]
+ */
+#ifndef SBN_H_
+#define SBN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SBN_OK = 0,
+    SBN_ERR_NULL = 1,        /* a required pointer is NULL */
+    SBN_ERR_SHAPE = 2,       /* a dimension is <= 0 or breaks the divisibility rules above */
+    SBN_ERR_ALIGN = 3,       /* a pointer is not 16-byte aligned */
+    SBN_ERR_UNSUPPORTED = 4, /* pattern other than 2:4, unknown dtype or op */
+    SBN_ERR_WORKSPACE = 5,   /* workspace missing or smaller than sbn_workspace_bytes() */
+    SBN_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, tensor map, ...) */
+    SBN_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (see sbn_check_status) */
+} sbn_status;
+
+typedef enum { SBN_OUT_F32 = 0, SBN_OUT_BF16 = 1 } sbn_out_dtype;
+
+typedef enum {
+    SBN_OP_QUANTIZE_MASK_PACK = 0,
+    SBN_OP_QUANT_ACT = 1,
+    SBN_OP_SPARSE_BITLINEAR = 2,
+    SBN_OP_BITLINEAR = 3
+} sbn_op;
+
+/* Host, pure.  Bytes of device workspace the given call needs for these sizes (0 if none).
+ * T is ignored by SBN_OP_QUANTIZE_MASK_PACK. */
+size_t sbn_workspace_bytes(int op, int T, int N, int K);
+
+/*
+ * Part 1 -- Eq. 1 (absmean ternary quantiser), Eq. 2 (magnitude N:M mask from the master
+ * weights), Eq. 3 (W_eff = W_q (.) M), in that order, then the compressed layout above.
+ *   gamma  = sum|W| / (N*K), accumulated in fp64, rounded to fp32 once, over the whole dense W
+ *   scale  = max(gamma, 1e-5)                            (Algorithm 2's clamp)
+ *   W_q    = clamp(round_half_even(W / scale), -1, +1)   (fp32 division)
+ *   mask   = the two largest |W| of every group of four; equal magnitudes -> lower column kept
+ * Arguments
+ *   W          device, fp32 [N][K], read only
+ *   n_keep, m_group  the N:M pattern; only 2:4 is implemented (else SBN_ERR_UNSUPPORTED)
+ *   vals       device out, int8 [N][K/2]
+ *   meta       device out, uint8 [N][K/8]; may be the same buffer as prev_meta
+ *   w_scale    device out, one fp32: `scale`
+ *   dense_q    device out or NULL, int8 [N][K]: the unmasked W_q (operand of sbn_bitlinear)
+ *   prev_meta  device or NULL, uint8 [N][K/8]: metadata of the previous step's mask
+ *   flip_bits  device out or NULL (required iff prev_meta != NULL), one uint64: number of
+ *              positions whose mask bit differs from prev_meta's, i.e. the numerator of the flip
+ *              rate r_t = ||m(w_t) - m(w_{t-1})||_1 / D (Sec. 4); overwritten, not accumulated
+ *   ws         device workspace of sbn_workspace_bytes(SBN_OP_QUANTIZE_MASK_PACK, 0, N, K)
+ *              bytes; contents need no initialisation; must not be shared by calls that may run
+ *              concurrently
+ */
+sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int m_group,
+                                  int8_t *vals, uint8_t *meta, float *w_scale, int8_t *dense_q,
+                                  const uint8_t *prev_meta, unsigned long long *flip_bits,
+                                  void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Part 2 -- per-token absmax int8 activation quantiser (Sec. 2.1; Algorithm 2, forward step 1):
+ *   a = max_k |x[t][k]|, d = max(a, 1e-5), s_x = 127 / d,
+ *   xq[t][k] = clamp(round_half_even(x[t][k] * s_x), -128, 127),  a_scale[t] = d / 127.
+ *   x_bf16   device, bf16 [T][K]
+ *   xq       device out, int8 [T][K]
+ *   a_scale  device out, fp32 [T]
+ * Here K only needs K % 8 == 0.
+ */
+sbn_status sbn_quant_act(const void *x_bf16, int T, int K, int8_t *xq, float *a_scale,
+                         void *stream);
+
+/*
+ * Part 3 -- Eq. 4: acc[t][n] = sum_k xq[t][k] * W_eff[n][k] in int32 (exact), then
+ *   y[t][n] = float(acc[t][n]) * (w_scale * a_scale[t]) (+ bias[n]),
+ * written as fp32 or as bf16 (round-to-nearest-even of the fp32 value).
+ *   xq, a_scale   device, outputs of sbn_quant_act
+ *   vals, meta, w_scale  device, outputs of sbn_quantize_mask_pack (w_scale stays on the device)
+ *   bias          device fp32 [N] or NULL
+ *   y             device out, [T][N] of `dt`
+ *   acc_out       device out or NULL, int32 [T][N]: the raw accumulators (for parity checks)
+ *   ws, ws_bytes  device workspace of sbn_workspace_bytes(SBN_OP_SPARSE_BITLINEAR, T, N, K)
+ *                 bytes (may be NULL when that is 0)
+ */
+sbn_status sbn_sparse_bitlinear(const int8_t *xq, const float *a_scale, int T,
+                                const int8_t *vals, const uint8_t *meta, const float *w_scale,
+                                int N, int K, const float *bias, void *y, sbn_out_dtype dt,
+                                int32_t *acc_out, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Baseline -- dense BitLinear (Sec. 2.1): same as above with the unmasked ternary
+ * dense_q int8 [N][K] in place of vals/meta.
+ */
+sbn_status sbn_bitlinear(const int8_t *xq, const float *a_scale, int T,
+                         const int8_t *dense_q, const float *w_scale,
+                         int N, int K, const float *bias, void *y, sbn_out_dtype dt,
+                         int32_t *acc_out, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Whole forward of one layer from HOST activations (Algorithm 2's forward with pre-packed
+ * weights): copies x (bf16 [T][K], host, ideally pinned) to `x_dev`, runs sbn_quant_act and
+ * sbn_sparse_bitlinear (or sbn_bitlinear when vals == NULL and dense_q != NULL), and copies
+ * y ([T][N] of `dt`) back to `y_host`.  All on `stream`; returns after enqueueing.
+ *   x_dev   device staging, T*K*2 bytes;  xq_dev  device, T*K bytes;  a_scale_dev device, T*4
+ *   y_dev   device staging for y
+ * Weights (vals/meta or dense_q, w_scale, bias) are device pointers as above.
+ */
+sbn_status sbn_layer_forward_host(const void *x_bf16_host, int T, int K,
+                                  void *x_dev, int8_t *xq_dev, float *a_scale_dev,
+                                  const int8_t *vals, const uint8_t *meta, const int8_t *dense_q,
+                                  const float *w_scale, int N, const float *bias,
+                                  void *y_dev, void *y_host, sbn_out_dtype dt,
+                                  void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, returns SBN_ERR_TIMEOUT if any kernel since the last call gave up on a
+ * bounded wait (and clears that record), SBN_ERR_CUDA if the stream reports an error, else
+ * SBN_OK. */
+sbn_status sbn_check_status(void *stream);
+
+/* Static string for a status code. */
+const char *sbn_status_string(sbn_status s);
+
+/* Tuning/diagnostic knob (host state, not thread-safe): force the token-tile width of the GEMM
+ * kernels to 64, 128 or 256 (0 = automatic), and the split-K factor (0 = automatic).  Results
+ * do not depend on it. */
+void sbn_set_gemm_tuning(int token_tile, int split_k);
+
+/* Number of kernels the library has launched since it was loaded (all calls, all streams). */
+unsigned long long sbn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBN_H_ */

@@ -1,0 +1,174 @@
+"""Thin ctypes binding over libsbn.so -- argument marshalling only.
+
+Function names match the C ABI in ``include/sbn.h``.  Tensors are torch CUDA tensors used purely
+as device buffers (``data_ptr()``), the stream is torch's current stream.  Nothing here computes:
+every step of the path runs inside the library's kernels.  If the library cannot be loaded the
+import of this module's functions fails loudly -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsbn.so")
+
+SBN_OK = 0
+OUT_F32, OUT_BF16 = 0, 1
+OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
+
+EXPORTS = [
+    "sbn_workspace_bytes", "sbn_quantize_mask_pack", "sbn_quant_act", "sbn_sparse_bitlinear",
+    "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
+    "sbn_set_gemm_tuning", "sbn_launch_count",
+]
+
+_lib = None
+
+
+class SbnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: sbn status {code} ({status_string(code)})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libsbn.so (built in-tree by paper_2603_05168_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2603_05168_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.sbn_workspace_bytes.restype = sz
+        L.sbn_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.sbn_quantize_mask_pack.restype = i32
+        L.sbn_quantize_mask_pack.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.sbn_quant_act.restype = i32
+        L.sbn_quant_act.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.sbn_sparse_bitlinear.restype = i32
+        L.sbn_sparse_bitlinear.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+        L.sbn_bitlinear.restype = i32
+        L.sbn_bitlinear.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+        L.sbn_layer_forward_host.restype = i32
+        L.sbn_layer_forward_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, sz, vp]
+        L.sbn_check_status.restype = i32
+        L.sbn_check_status.argtypes = [vp]
+        L.sbn_status_string.restype = ctypes.c_char_p
+        L.sbn_status_string.argtypes = [i32]
+        L.sbn_set_gemm_tuning.restype = None
+        L.sbn_set_gemm_tuning.argtypes = [i32, i32]
+        L.sbn_launch_count.restype = ctypes.c_ulonglong
+        L.sbn_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().sbn_status_string(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != SBN_OK:
+        raise SbnError(code, where)
+
+
+def sbn_workspace_bytes(op: int, T: int, N: int, K: int) -> int:
+    return int(lib().sbn_workspace_bytes(op, T, N, K))
+
+
+def sbn_quantize_mask_pack(W, vals, meta, w_scale, ws, dense_q=None, prev_meta=None, flip_bits=None,
+                           n_keep: int = 2, m_group: int = 4):
+    N, K = W.shape
+    _check(lib().sbn_quantize_mask_pack(_ptr(W), N, K, n_keep, m_group, _ptr(vals), _ptr(meta),
+                                        _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta), _ptr(flip_bits),
+                                        _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "sbn_quantize_mask_pack")
+
+
+def sbn_quant_act(x_bf16, xq, a_scale):
+    T, K = x_bf16.shape
+    _check(lib().sbn_quant_act(_ptr(x_bf16), T, K, _ptr(xq), _ptr(a_scale), _stream()), "sbn_quant_act")
+
+
+def _ws_args(ws):
+    if ws is None:
+        return None, 0
+    return _ptr(ws), ws.numel() * ws.element_size()
+
+
+def sbn_sparse_bitlinear(xq, a_scale, vals, meta, w_scale, y, bias=None, acc_out=None, ws=None):
+    T, K = xq.shape
+    N = vals.shape[0]
+    dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
+    wp, wb = _ws_args(ws)
+    _check(lib().sbn_sparse_bitlinear(_ptr(xq), _ptr(a_scale), T, _ptr(vals), _ptr(meta), _ptr(w_scale),
+                                      N, K, _ptr(bias), _ptr(y), dt, _ptr(acc_out), wp, wb, _stream()),
+           "sbn_sparse_bitlinear")
+
+
+def sbn_bitlinear(xq, a_scale, dense_q, w_scale, y, bias=None, acc_out=None, ws=None):
+    T, K = xq.shape
+    N = dense_q.shape[0]
+    dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
+    wp, wb = _ws_args(ws)
+    _check(lib().sbn_bitlinear(_ptr(xq), _ptr(a_scale), T, _ptr(dense_q), _ptr(w_scale), N, K,
+                               _ptr(bias), _ptr(y), dt, _ptr(acc_out), wp, wb, _stream()),
+           "sbn_bitlinear")
+
+
+def sbn_layer_forward_host(x_host, x_dev, xq_dev, a_scale_dev, w_scale, y_dev, y_host, vals=None,
+                           meta=None, dense_q=None, bias=None, ws=None):
+    """x_host / y_host are (pinned) CPU tensors; everything else lives on the device."""
+    T, K = x_host.shape
+    N = y_host.shape[1]
+    dt = OUT_BF16 if y_host.dtype == torch.bfloat16 else OUT_F32
+    wp, wb = _ws_args(ws)
+    _check(lib().sbn_layer_forward_host(_ptr(x_host), T, K, _ptr(x_dev), _ptr(xq_dev), _ptr(a_scale_dev),
+                                        _ptr(vals), _ptr(meta), _ptr(dense_q), _ptr(w_scale), N,
+                                        _ptr(bias), _ptr(y_dev), _ptr(y_host), dt, wp, wb, _stream()),
+           "sbn_layer_forward_host")
+
+
+def sbn_check_status():
+    _check(lib().sbn_check_status(_stream()), "sbn_check_status")
+
+
+def sbn_set_gemm_tuning(token_tile: int = 0, split_k: int = 0):
+    lib().sbn_set_gemm_tuning(int(token_tile), int(split_k))
+
+
+def sbn_launch_count() -> int:
+    return int(lib().sbn_launch_count())
+
+
+# -- small conveniences for callers (allocation only) ---------------------------------------------
+def alloc_packed(N: int, K: int, device="cuda", with_dense: bool = False):
+    """Device buffers for one packed weight matrix."""
+    out = dict(
+        vals=torch.empty((N, K // 2), dtype=torch.int8, device=device),
+        meta=torch.empty((N, K // 8), dtype=torch.uint8, device=device),
+        w_scale=torch.empty(1, dtype=torch.float32, device=device),
+        ws=torch.empty(sbn_workspace_bytes(OP_QUANTIZE_MASK_PACK, 0, N, K), dtype=torch.uint8, device=device),
+    )
+    if with_dense:
+        out["dense_q"] = torch.empty((N, K), dtype=torch.int8, device=device)
+    return out
+
+
+def alloc_gemm_ws(op: int, T: int, N: int, K: int, device="cuda"):
+    n = sbn_workspace_bytes(op, T, N, K)
+    return torch.empty(max(n, 16), dtype=torch.uint8, device=device)

@@ -1,0 +1,428 @@
+// Eq. 4 on the 5th-generation tensor cores: acc[t][n] = sum_k xq[t][k] * W[n][k] (int8 x int8 ->
+// int32), then y = float(acc) * (w_scale * a_scale[t]) (+ bias[n]) in the epilogue.
+//
+// One kernel template serves both layers:
+//   SPARSE = true   W = W_eff in the compressed 2:4 layout; tcgen05.mma.sp kind::i8, logical
+//                   K = 64 per instruction, metadata copied SMEM -> TMEM with tcgen05.cp
+//   SPARSE = false  W = dense ternary W_q; tcgen05.mma kind::i8, K = 32 per instruction
+//
+// Only operand A of the MMA may be sparse, so the weights are A (M dimension = output features)
+// and the activations are B (N dimension = tokens): D[n_out][token] lives in TMEM with the
+// output feature on the lane axis.  The epilogue thread that owns lane n writes y[t][n] for the
+// tokens in its registers; across a warp that is 32 consecutive n, i.e. one contiguous 128 B
+// (fp32) or 64 B (bf16) segment per store instruction, so no transpose through shared memory is
+// needed.
+//
+// CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (also owns the TMEM allocation),
+// warps 2-5 epilogue (one TMEM lane quarter each).  Persistent over output tiles
+// (128 features x BN tokens), static round-robin tile order, K-blocks of 128 logical columns:
+//   A stage   128 rows x 64 B (sparse, SWIZZLE_64B)  or 128 rows x 128 B (dense, SWIZZLE_128B)
+//   B stage   BN rows x 128 B (SWIZZLE_128B)
+//   E stage   128 rows x 16 B metadata (sparse only), plain row-major = the canonical layout
+// TMEM: ACC_STAGES accumulators of BN columns, then one 4-column metadata slot per smem stage.
+//
+// Every wait is bounded (wall-clock limit); a wait that runs out records SBN_ERR_TIMEOUT in the
+// device status word, raises a CTA-wide abort flag and every role leaves its loop.
+#pragma once
+
+#include <cuda.h>
+
+#include "sbn_common.cuh"
+
+namespace sbn {
+
+constexpr int kGemmThreads = 192;
+constexpr int kBM = 128;                 // output features per tile (MMA M)
+constexpr int kBK = 128;                 // logical K per pipeline stage
+constexpr uint32_t kTmemCols = 512;
+constexpr int kSmemBudget = 220 * 1024;  // of the 227 KB a CTA may use
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+struct GemmParams {
+    int T, N, K;
+    int k_blocks_total;          // K / 128
+    int k_splits;                // split-K factor (1 = none)
+    const float* a_scale;        // [T]
+    const float* w_scale;        // [1]
+    const float* bias;           // [N] or null
+    void* y;                     // [T][N] fp32 or bf16
+    int out_bf16;
+    int32_t* acc_out;            // [T][N] or null
+    int32_t* split_acc;          // [T][N] int32 zero-initialised scratch when k_splits > 1
+    unsigned int* split_counters;   // per output tile, zero-initialised, when k_splits > 1
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: false if the barrier did not flip within the limit or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    unsigned int spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_cp_128x128b(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void mma_i8_dense(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                             uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_i8_sparse(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                              uint32_t e_tmem, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.sp.cta_group::1.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(e_tmem), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (base + i).
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (K-major operand): start address, leading/stride byte offsets
+// in 16 B units, descriptor version 1, swizzle mode in the top three bits.
+constexpr uint64_t kSwzNone = 0, kSwz128 = 2, kSwz64 = 4;
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes,
+                                                   uint32_t sbo_bytes, uint64_t swizzle) {
+    return static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4) |
+           (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+           (static_cast<uint64_t>(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (swizzle << 61);
+}
+
+// Instruction descriptor for kind::i8: D = s32, A = B = signed 8 bit, both K-major.
+__host__ __device__ constexpr uint32_t make_idesc_i8(int mma_m, int mma_n, bool sparse) {
+    return (sparse ? (1u << 2) : 0u) | (2u << 4) | (1u << 7) | (1u << 10) |
+           (static_cast<uint32_t>(mma_n >> 3) << 17) | (static_cast<uint32_t>(mma_m >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Compile-time configuration
+// ---------------------------------------------------------------------------------------------
+template <bool SPARSE, int BN>
+struct GemmConfig {
+    static constexpr int A_BYTES = SPARSE ? kBM * (kBK / 2) : kBM * kBK;
+    static constexpr int B_BYTES = BN * kBK;
+    static constexpr int E_BYTES = SPARSE ? kBM * (kBK / 8) : 0;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+    static constexpr int STAGES_RAW = kSmemBudget / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+    static constexpr int META_COLS = SPARSE ? 4 * STAGES : 0;
+    static constexpr int ACC_STAGES = (2 * BN + META_COLS <= static_cast<int>(kTmemCols)) ? 2 : 1;
+    static constexpr int META_COL0 = ACC_STAGES * BN;
+    static constexpr uint32_t TX_BYTES = STAGE_BYTES;
+    // dynamic smem: 1 KB alignment slack + stages + barriers
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
+    static_assert(STAGES >= 2, "tile too large for shared memory");
+    static_assert(ACC_STAGES * BN + META_COLS <= static_cast<int>(kTmemCols), "TMEM overflow");
+};
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+template <bool SPARSE, int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                      const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_e,
+                      const GemmParams p) {
+    using Cfg = GemmConfig<SPARSE, BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr int ACC_STAGES = Cfg::ACC_STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    // 1 KB alignment: required by the 128 B swizzle atoms (8 rows x 128 B)
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_a = smem_base;
+    const uint32_t smem_b = smem_a + STAGES * Cfg::A_BYTES;
+    const uint32_t smem_e = smem_b + STAGES * Cfg::B_BYTES;
+    const uint32_t bar_base = smem_base + STAGES * Cfg::STAGE_BYTES;     // 8 B aligned
+    const uint32_t bar_full = bar_base;                       // [STAGES]   TMA -> MMA
+    const uint32_t bar_empty = bar_full + 8 * STAGES;         // [STAGES]   MMA -> TMA
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;     // [ACC]      MMA -> epilogue
+    const uint32_t bar_acc_empty = bar_acc_full + 8 * ACC_STAGES;   // [ACC] epilogue -> MMA
+    const uint32_t tmem_slot = bar_acc_empty + 8 * ACC_STAGES;      // 4 B: TMEM base address
+
+    __shared__ int s_abort;
+    volatile int* abort_flag = &s_abort;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    const int tiles_m = p.N / kBM;
+    const int tiles_t = (p.T + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_t * p.k_splits;
+    const int kb_per_split = p.k_blocks_total / p.k_splits;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < ACC_STAGES; ++a) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, 4);          // one arrival per epilogue warp
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tcgen05_fence_before();
+    }
+    __syncthreads();
+    tcgen05_fence_after();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_a);
+            tma_prefetch_desc(&tmap_b);
+            if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int split = tile % p.k_splits;
+                const int mt = (tile / p.k_splits) % tiles_m;
+                const int tt = (tile / p.k_splits) / tiles_m;
+                const int m0 = mt * kBM, t0 = tt * BN;
+                const int kb0 = split * kb_per_split;
+                for (int kb = kb0; kb < kb0 + kb_per_split; ++kb) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t full = bar_full + 8 * stage;
+                    mbar_expect_tx(full, Cfg::TX_BYTES);
+                    if constexpr (SPARSE) {
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, kb * (kBK / 2), m0, full);
+                        tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, kb * (kBK / 8), m0, full);
+                    } else {
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, kb * kBK, m0, full);
+                    }
+                    tma_load_2d(smem_b + stage * Cfg::B_BYTES, &tmap_b, kb * kBK, t0, full);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(kBM, BN, SPARSE);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+                for (int kb = 0; kb < kb_per_split; ++kb) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_a + stage * Cfg::A_BYTES;
+                    const uint32_t b_addr = smem_b + stage * Cfg::B_BYTES;
+                    if constexpr (SPARSE) {
+                        const uint32_t e_tmem = tmem_base + static_cast<uint32_t>(Cfg::META_COL0 + 4 * stage);
+                        const uint64_t e_desc = make_smem_desc(smem_e + stage * Cfg::E_BYTES, 128, 128, kSwzNone);
+                        tcgen05_cp_128x128b(e_tmem, e_desc);
+                        const uint64_t a_desc = make_smem_desc(a_addr, 16, 512, kSwz64);
+                        const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
+#pragma unroll
+                        for (int j = 0; j < kBK / 64; ++j) {
+                            // per instruction: 32 B of compressed A, 64 B of B, 2 metadata columns
+                            mma_i8_sparse(d_tmem, a_desc + static_cast<uint64_t>(2 * j),
+                                          b_desc + static_cast<uint64_t>(4 * j), e_tmem + 2 * j, idesc,
+                                          (kb | j) != 0 ? 1u : 0u);
+                        }
+                    } else {
+                        const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024, kSwz128);
+                        const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
+#pragma unroll
+                        for (int j = 0; j < kBK / 32; ++j) {
+                            mma_i8_dense(d_tmem, a_desc + static_cast<uint64_t>(2 * j),
+                                         b_desc + static_cast<uint64_t>(2 * j), idesc,
+                                         (kb | j) != 0 ? 1u : 0u);
+                        }
+                    }
+                    tcgen05_commit(bar_empty + 8 * stage);        // smem stage free once read
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tcgen05_commit(bar_acc_full + 8 * acc);           // accumulator complete
+                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (4 warps)
+        const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
+        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+        const float w_scale = __ldg(p.w_scale);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const int mt = (tile / p.k_splits) % tiles_m;
+            const int tt = (tile / p.k_splits) / tiles_m;
+            const int n = mt * kBM + quarter * 32 + lane;         // output feature of this thread
+            const int t0 = tt * BN;
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after();
+            const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(acc * BN + c * 32), r);
+                tmem_ld_wait();
+                if (c == BN / 32 - 1) {
+                    // all of this warp's reads of the accumulator are done: hand it back
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+                }
+                const int tc = t0 + c * 32;
+                if (p.k_splits > 1) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int t = tc + j;
+                        if (t < p.T) atomicAdd(p.split_acc + static_cast<size_t>(t) * p.N + n, static_cast<int>(r[j]));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int t = tc + j;
+                        if (t < p.T) {
+                            const size_t o = static_cast<size_t>(t) * p.N + n;
+                            const int a = static_cast<int>(r[j]);
+                            if (p.acc_out) p.acc_out[o] = a;
+                            const float s = __fmul_rn(w_scale, __ldg(p.a_scale + t));
+                            float v = __fmul_rn(static_cast<float>(a), s);
+                            if (p.bias) v = __fadd_rn(v, bias);
+                            if (p.out_bf16) {
+                                static_cast<uint16_t*>(p.y)[o] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+                            } else {
+                                static_cast<float*>(p.y)[o] = v;
+                            }
+                        }
+                    }
+                }
+            }
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // teardown: everyone meets here (also on the abort path), then the allocating warp frees TMEM
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// Split-K finish: y = dequant(split_acc), and clear split_acc for the next call.
+__global__ void __launch_bounds__(256)
+splitk_finish_kernel(int32_t* __restrict__ split_acc, int T, int N, const float* __restrict__ a_scale,
+                     const float* __restrict__ w_scale, const float* __restrict__ bias,
+                     void* __restrict__ y, int out_bf16, int32_t* __restrict__ acc_out) {
+    const size_t total = static_cast<size_t>(T) * N;
+    const float ws = __ldg(w_scale);
+    for (size_t i = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * 256) {
+        const int t = static_cast<int>(i / N);
+        const int n = static_cast<int>(i - static_cast<size_t>(t) * N);
+        const int a = split_acc[i];
+        split_acc[i] = 0;
+        if (acc_out) acc_out[i] = a;
+        const float s = __fmul_rn(ws, __ldg(a_scale + t));
+        float v = __fmul_rn(static_cast<float>(a), s);
+        if (bias) v = __fadd_rn(v, __ldg(bias + n));
+        if (out_bf16) static_cast<uint16_t*>(y)[i] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+        else static_cast<float*>(y)[i] = v;
+    }
+}
+
+}  // namespace sbn

@@ -1,0 +1,292 @@
+// libsbn: the C ABI declared in include/sbn.h.  Host side only validates arguments, encodes TMA
+// tensor maps and enqueues kernels on the caller's stream; every step of the path runs in the
+// kernels of this translation unit.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "sbn.h"
+#include "sbn_common.cuh"
+#include "quant_act.cuh"
+#include "quantize_mask_pack.cuh"
+#include "gemm_tcgen05.cuh"
+
+namespace sbn {
+
+// ------------------------------------------------------------------------------------------------
+// host state
+// ------------------------------------------------------------------------------------------------
+static int g_force_token_tile = 0;
+static int g_force_split_k = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess) {
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        }
+    });
+    return fn;
+}
+
+// 2-D uint8 row-major tensor [rows][cols_bytes] with a [box_rows][box_cols] box.
+static bool encode_2d_u8(CUtensorMap* map, const void* base, uint64_t cols_bytes, uint64_t rows,
+                         uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols_bytes, rows};
+    cuuint64_t strides[1] = {cols_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+static inline bool misaligned(const void* p, size_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
+}
+
+static inline int pick_token_tile(int T) {
+    if (g_force_token_tile == 64 || g_force_token_tile == 128 || g_force_token_tile == 256)
+        return g_force_token_tile;
+    if (T <= 64) return 64;
+    return 128;
+}
+
+static inline int pick_split_k(int T, int N, int K, int bn) {
+    const int kblocks = K / kBK;
+    int want = 1;
+    if (g_force_split_k > 0) {
+        want = g_force_split_k;
+    } else {
+        const int tiles = (N / kBM) * ((T + bn - 1) / bn);
+        // weight-streaming regime: too few tiles to cover the SMs -> split K
+        if (tiles * 2 <= kNumSMs) {
+            want = kNumSMs / tiles;
+        }
+    }
+    if (want > kblocks) want = kblocks;
+    while (want > 1 && kblocks % want != 0) --want;
+    return want < 1 ? 1 : want;
+}
+
+static size_t gemm_workspace_bytes(int T, int N, int K) {
+    // split-K scratch: int32 [T][N]; only the small-T regime ever splits
+    const int bn = pick_token_tile(T);
+    if (pick_split_k(T, N, K, bn) > 1) return static_cast<size_t>(T) * N * sizeof(int32_t);
+    return 0;
+}
+
+template <bool SPARSE, int BN>
+static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
+                                  const GemmParams& p, cudaStream_t stream) {
+    using Cfg = GemmConfig<SPARSE, BN>;
+    static bool configured = false;
+    auto kernel = bitlinear_gemm_kernel<SPARSE, BN>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        configured = true;
+    }
+    const int tiles = (p.N / kBM) * ((p.T + BN - 1) / BN) * p.k_splits;
+    const int grid = tiles < kNumSMs ? tiles : kNumSMs;
+    kernel<<<grid, kGemmThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, p);
+    ++g_launch_count;
+    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
+static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, int T,
+                           const int8_t* wvals, const uint8_t* meta, const float* w_scale,
+                           int N, int K, const float* bias, void* y, sbn_out_dtype dt,
+                           int32_t* acc_out, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    if (!xq || !a_scale || !wvals || !w_scale || !y || (sparse && !meta)) return SBN_ERR_NULL;
+    if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (dt != SBN_OUT_F32 && dt != SBN_OUT_BF16) return SBN_ERR_UNSUPPORTED;
+    if (misaligned(xq, 16) || misaligned(wvals, 16) || (sparse && misaligned(meta, 16)) ||
+        misaligned(y, 16) || misaligned(a_scale, 4) || misaligned(w_scale, 4) ||
+        (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)))
+        return SBN_ERR_ALIGN;
+
+    const int bn = pick_token_tile(T);
+    const int splits = pick_split_k(T, N, K, bn);
+    if (splits > 1) {
+        const size_t need = static_cast<size_t>(T) * N * sizeof(int32_t);
+        if (!ws || ws_bytes < need) return SBN_ERR_WORKSPACE;
+        if (misaligned(ws, 16)) return SBN_ERR_ALIGN;
+        if (cudaMemsetAsync(ws, 0, need, stream) != cudaSuccess) return SBN_ERR_CUDA;
+    }
+
+    CUtensorMap ta, tb, te;
+    bool ok;
+    if (sparse) {
+        ok = encode_2d_u8(&ta, wvals, static_cast<uint64_t>(K) / 2, N, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B) &&
+             encode_2d_u8(&te, meta, static_cast<uint64_t>(K) / 8, N, kBK / 8, kBM, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else {
+        ok = encode_2d_u8(&ta, wvals, K, N, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+        te = ta;
+    }
+    ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return SBN_ERR_CUDA;
+
+    GemmParams p;
+    p.T = T; p.N = N; p.K = K;
+    p.k_blocks_total = K / kBK;
+    p.k_splits = splits;
+    p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias;
+    p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
+    p.acc_out = acc_out;
+    p.split_acc = splits > 1 ? static_cast<int32_t*>(ws) : nullptr;
+    p.split_counters = nullptr;
+
+    sbn_status st;
+#define SBN_GEMM_CASE(S, B) st = launch_gemm_cfg<S, B>(ta, tb, te, p, stream)
+    if (sparse) {
+        if (bn == 64) SBN_GEMM_CASE(true, 64); else if (bn == 128) SBN_GEMM_CASE(true, 128); else SBN_GEMM_CASE(true, 256);
+    } else {
+        if (bn == 64) SBN_GEMM_CASE(false, 64); else if (bn == 128) SBN_GEMM_CASE(false, 128); else SBN_GEMM_CASE(false, 256);
+    }
+#undef SBN_GEMM_CASE
+    if (st != SBN_OK) return st;
+    if (splits > 1) {
+        const size_t total = static_cast<size_t>(T) * N;
+        size_t blocks = (total + 255) / 256;
+        if (blocks > static_cast<size_t>(kNumSMs * 8)) blocks = kNumSMs * 8;
+        splitk_finish_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+            p.split_acc, T, N, a_scale, w_scale, bias, y, p.out_bf16, acc_out);
+        ++g_launch_count;
+        if (cudaGetLastError() != cudaSuccess) return SBN_ERR_CUDA;
+    }
+    return SBN_OK;
+}
+
+}  // namespace sbn
+
+// ------------------------------------------------------------------------------------------------
+// extern "C"
+// ------------------------------------------------------------------------------------------------
+using namespace sbn;
+
+extern "C" {
+
+size_t sbn_workspace_bytes(int op, int T, int N, int K) {
+    switch (op) {
+        case SBN_OP_QUANTIZE_MASK_PACK: return sizeof(QmpWorkspace);
+        case SBN_OP_QUANT_ACT: return 0;
+        case SBN_OP_SPARSE_BITLINEAR:
+        case SBN_OP_BITLINEAR:
+            if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return 0;
+            return gemm_workspace_bytes(T, N, K);
+        default: return 0;
+    }
+}
+
+sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int m_group,
+                                  int8_t* vals, uint8_t* meta, float* w_scale, int8_t* dense_q,
+                                  const uint8_t* prev_meta, unsigned long long* flip_bits,
+                                  void* ws, size_t ws_bytes, void* stream) {
+    if (!W || !vals || !meta || !w_scale) return SBN_ERR_NULL;
+    if (prev_meta && !flip_bits) return SBN_ERR_NULL;
+    if (n_keep != 2 || m_group != 4) return SBN_ERR_UNSUPPORTED;
+    if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (!ws || ws_bytes < sizeof(QmpWorkspace)) return SBN_ERR_WORKSPACE;
+    if (misaligned(W, 16) || misaligned(vals, 16) || misaligned(meta, 16) || misaligned(ws, 16) ||
+        misaligned(w_scale, 4) || (dense_q && misaligned(dense_q, 16)) ||
+        (prev_meta && misaligned(prev_meta, 16)) || (flip_bits && misaligned(flip_bits, 8)))
+        return SBN_ERR_ALIGN;
+    return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+                                     static_cast<QmpWorkspace*>(ws)->partial,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale, void* stream) {
+    if (!x_bf16 || !xq || !a_scale) return SBN_ERR_NULL;
+    if (T <= 0 || K <= 0 || K % 8 != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(x_bf16, 16) || misaligned(xq, 8) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
+    return launch_quant_act(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_sparse_bitlinear(const int8_t* xq, const float* a_scale, int T, const int8_t* vals,
+                                const uint8_t* meta, const float* w_scale, int N, int K,
+                                const float* bias, void* y, sbn_out_dtype dt, int32_t* acc_out,
+                                void* ws, size_t ws_bytes, void* stream) {
+    return run_gemm(true, xq, a_scale, T, vals, meta, w_scale, N, K, bias, y, dt, acc_out, ws, ws_bytes,
+                    static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_bitlinear(const int8_t* xq, const float* a_scale, int T, const int8_t* dense_q,
+                         const float* w_scale, int N, int K, const float* bias, void* y,
+                         sbn_out_dtype dt, int32_t* acc_out, void* ws, size_t ws_bytes, void* stream) {
+    return run_gemm(false, xq, a_scale, T, dense_q, nullptr, w_scale, N, K, bias, y, dt, acc_out, ws,
+                    ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_layer_forward_host(const void* x_bf16_host, int T, int K, void* x_dev, int8_t* xq_dev,
+                                  float* a_scale_dev, const int8_t* vals, const uint8_t* meta,
+                                  const int8_t* dense_q, const float* w_scale, int N,
+                                  const float* bias, void* y_dev, void* y_host, sbn_out_dtype dt,
+                                  void* ws, size_t ws_bytes, void* stream) {
+    if (!x_bf16_host || !x_dev || !xq_dev || !a_scale_dev || !y_dev || !y_host) return SBN_ERR_NULL;
+    if (T <= 0 || K <= 0 || N <= 0) return SBN_ERR_SHAPE;
+    if (!vals && !dense_q) return SBN_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t x_bytes = static_cast<size_t>(T) * K * 2;
+    if (cudaMemcpyAsync(x_dev, x_bf16_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SBN_ERR_CUDA;
+    sbn_status st = sbn_quant_act(x_dev, T, K, xq_dev, a_scale_dev, stream);
+    if (st != SBN_OK) return st;
+    if (vals) {
+        st = sbn_sparse_bitlinear(xq_dev, a_scale_dev, T, vals, meta, w_scale, N, K, bias, y_dev, dt, nullptr, ws, ws_bytes, stream);
+    } else {
+        st = sbn_bitlinear(xq_dev, a_scale_dev, T, dense_q, w_scale, N, K, bias, y_dev, dt, nullptr, ws, ws_bytes, stream);
+    }
+    if (st != SBN_OK) return st;
+    const size_t y_bytes = static_cast<size_t>(T) * N * (dt == SBN_OUT_BF16 ? 2 : 4);
+    if (cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SBN_ERR_CUDA;
+    return SBN_OK;
+}
+
+sbn_status sbn_check_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SBN_ERR_CUDA;
+    int h = 0;
+    if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return SBN_ERR_CUDA;
+    if (h != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+        return static_cast<sbn_status>(h);
+    }
+    return SBN_OK;
+}
+
+const char* sbn_status_string(sbn_status s) {
+    switch (s) {
+        case SBN_OK: return "ok";
+        case SBN_ERR_NULL: return "a required pointer is NULL";
+        case SBN_ERR_SHAPE: return "bad shape (need T >= 1, N % 128 == 0, K % 128 == 0)";
+        case SBN_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case SBN_ERR_UNSUPPORTED: return "unsupported pattern, dtype or op";
+        case SBN_ERR_WORKSPACE: return "workspace missing or too small";
+        case SBN_ERR_CUDA: return "CUDA call failed";
+        case SBN_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+void sbn_set_gemm_tuning(int token_tile, int split_k) {
+    g_force_token_tile = token_tile;
+    g_force_split_k = split_k;
+}
+
+unsigned long long sbn_launch_count(void) { return g_launch_count; }
+
+}  // extern "C"

@@ -1,0 +1,146 @@
+// Per-token absmax int8 activation quantiser (Sec. 2.1; Algorithm 2, forward step 1).
+//
+//   a = max_k |x|, d = max(a, 1e-5), s_x = 127 / d,
+//   xq = clamp(rint(x * s_x), -128, 127),  a_scale = d / 127
+//
+// HBM-bound: 2 B read + 1 B written per element.  A group of G threads owns one token row and
+// keeps it in registers between the max and the rounding, so x is read from memory once.
+// Loads are 16 B (8 bf16) per lane, stores 8 B (8 int8) per lane, both fully coalesced.
+#pragma once
+
+#include "sbn_common.cuh"
+
+namespace sbn {
+
+constexpr int kActThreads = 256;
+constexpr int kActVecPerThread = 8;   // up to 8 x 16 B of one row per thread
+
+__device__ __forceinline__ float absmax8(const uint4& v) {
+    float m = fmaxf(fabsf(bf16lo_to_f32(v.x)), fabsf(bf16hi_to_f32(v.x)));
+    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.y)), fabsf(bf16hi_to_f32(v.y))));
+    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.z)), fabsf(bf16hi_to_f32(v.z))));
+    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.w)), fabsf(bf16hi_to_f32(v.w))));
+    return m;
+}
+
+__device__ __forceinline__ uint32_t quant1(float x, float s_x) {
+    int q = __float2int_rn(__fmul_rn(x, s_x));     // one fp32 multiply, then half-to-even
+    q = max(-128, min(127, q));
+    return static_cast<uint32_t>(q) & 0xFFu;
+}
+
+__device__ __forceinline__ uint32_t quant_pair2(uint32_t a, uint32_t b, float s_x) {
+    return quant1(bf16lo_to_f32(a), s_x) | (quant1(bf16hi_to_f32(a), s_x) << 8) |
+           (quant1(bf16lo_to_f32(b), s_x) << 16) | (quant1(bf16hi_to_f32(b), s_x) << 24);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kActThreads)
+quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
+                 float* __restrict__ a_scale) {
+    constexpr int ROWS = kActThreads / G;
+    constexpr int WARPS_PER_ROW = (G + 31) / 32;
+    __shared__ float s_max[kActThreads / 32];
+
+    const int r = threadIdx.x / G;
+    const int g = threadIdx.x % G;
+    const int row = blockIdx.x * ROWS + r;
+    const bool active = row < T;
+    const uint4* xr = x + static_cast<size_t>(active ? row : 0) * nvec;
+
+    uint4 v[kActVecPerThread];
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kActVecPerThread; ++i) {
+        const int idx = g + i * G;
+        if (active && idx < nvec) {
+            v[i] = __ldg(xr + idx);
+        } else {
+            v[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kActVecPerThread; ++i) amax = fmaxf(amax, absmax8(v[i]));
+
+    amax = warp_max(amax);
+    if constexpr (WARPS_PER_ROW > 1) {
+        const int warp = threadIdx.x >> 5;
+        if ((threadIdx.x & 31) == 0) s_max[warp] = amax;
+        __syncthreads();
+        const int w0 = (r * G) >> 5;
+        float m = s_max[w0];
+#pragma unroll
+        for (int w = 1; w < WARPS_PER_ROW; ++w) m = fmaxf(m, s_max[w0 + w]);
+        amax = m;
+    }
+    if (!active) return;
+
+    const float d = fmaxf(amax, kEps);
+    const float s_x = __fdiv_rn(127.0f, d);
+    if (g == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
+
+    uint2* qr = xq + static_cast<size_t>(row) * nvec;
+#pragma unroll
+    for (int i = 0; i < kActVecPerThread; ++i) {
+        const int idx = g + i * G;
+        if (idx < nvec) {
+            uint2 o;
+            o.x = quant_pair2(v[i].x, v[i].y, s_x);
+            o.y = quant_pair2(v[i].z, v[i].w, s_x);
+            qr[idx] = o;
+        }
+    }
+}
+
+// Rows too long for the register-resident kernel (K > 16384): one CTA per row, two passes over
+// the row (the second one served by L1/L2).
+__global__ void __launch_bounds__(kActThreads)
+quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
+                          float* __restrict__ a_scale) {
+    __shared__ float s_max[kActThreads / 32];
+    const int row = blockIdx.x;
+    if (row >= T) return;
+    const uint4* xr = x + static_cast<size_t>(row) * nvec;
+    float amax = 0.0f;
+    for (int idx = threadIdx.x; idx < nvec; idx += kActThreads) amax = fmaxf(amax, absmax8(__ldg(xr + idx)));
+    amax = warp_max(amax);
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    float m = s_max[0];
+#pragma unroll
+    for (int w = 1; w < kActThreads / 32; ++w) m = fmaxf(m, s_max[w]);
+    const float d = fmaxf(m, kEps);
+    const float s_x = __fdiv_rn(127.0f, d);
+    if (threadIdx.x == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
+    uint2* qr = xq + static_cast<size_t>(row) * nvec;
+    for (int idx = threadIdx.x; idx < nvec; idx += kActThreads) {
+        const uint4 v = __ldg(xr + idx);
+        uint2 o;
+        o.x = quant_pair2(v.x, v.y, s_x);
+        o.y = quant_pair2(v.z, v.w, s_x);
+        qr[idx] = o;
+    }
+}
+
+inline sbn_status launch_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale,
+                                   cudaStream_t stream) {
+    const int nvec = K / 8;
+    const uint4* x = static_cast<const uint4*>(x_bf16);
+    uint2* q = reinterpret_cast<uint2*>(xq);
+    const int per_thread_cap = kActVecPerThread;
+    if (nvec <= 32 * per_thread_cap) {
+        quant_act_kernel<32><<<(T + 7) / 8, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    } else if (nvec <= 64 * per_thread_cap) {
+        quant_act_kernel<64><<<(T + 3) / 4, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    } else if (nvec <= 128 * per_thread_cap) {
+        quant_act_kernel<128><<<(T + 1) / 2, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    } else if (nvec <= 256 * per_thread_cap) {
+        quant_act_kernel<256><<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    } else {
+        quant_act_long_row_kernel<<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    }
+    ++g_launch_count;
+    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
+}  // namespace sbn

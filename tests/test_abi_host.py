@@ -1,0 +1,94 @@
+"""CPU-only checks of the boundary: the library builds, loads, exports every symbol that
+include/sbn.h declares, and rejects bad arguments on the host before touching the GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2603_05168_b200 import build as sbn_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    sbn_build.build()
+    from paper_2603_05168_b200 import binding
+    return binding.lib()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "sbn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sbn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(L):
+    names = _declared_functions()
+    assert {"sbn_quantize_mask_pack", "sbn_quant_act", "sbn_sparse_bitlinear", "sbn_bitlinear"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in sbn.h but not exported"
+    from paper_2603_05168_b200 import binding
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_status_strings(L):
+    from paper_2603_05168_b200 import binding
+    seen = {binding.status_string(i) for i in range(8)}
+    assert len(seen) == 8
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_workspace_query(L):
+    from paper_2603_05168_b200 import binding as b
+    assert b.sbn_workspace_bytes(b.OP_QUANTIZE_MASK_PACK, 0, 256, 256) >= 8 * 148
+    assert b.sbn_workspace_bytes(b.OP_QUANT_ACT, 64, 0, 256) == 0
+    # large T: no split-K scratch; decode-sized T: int32 [T][N] scratch
+    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4096, 2560, 2560) == 0
+    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 4 * 2560 * 4
+    assert b.sbn_workspace_bytes(b.OP_BITLINEAR, 4, 2560, 100) == 0      # illegal shape -> 0
+    assert b.sbn_workspace_bytes(77, 4, 2560, 2560) == 0
+
+
+def test_argument_validation_on_host(L):
+    # fake, never dereferenced, 16-byte aligned "device pointers": every call below must return
+    # an error code from the host-side checks before any CUDA call is made
+    p = ctypes.c_void_p(0x1000)
+    odd = ctypes.c_void_p(0x1004)
+    NULL, SHAPE, ALIGN, UNSUP, WS = 1, 2, 3, 4, 5
+    assert L.sbn_quant_act(None, 4, 256, p, p, None) == NULL
+    assert L.sbn_quant_act(p, 0, 256, p, p, None) == SHAPE
+    assert L.sbn_quant_act(p, 4, 100, p, p, None) == SHAPE
+    assert L.sbn_quant_act(odd, 4, 256, p, p, None) == ALIGN
+    qmp = lambda **k: L.sbn_quantize_mask_pack(k.get("W", p), k.get("N", 256), k.get("K", 256), k.get("n", 2),
+                                               k.get("m", 4), p, p, p, None, k.get("prev"), k.get("flip"),
+                                               k.get("ws", p), k.get("wsb", 1 << 20), None)
+    assert qmp(W=None) == NULL
+    assert qmp(n=6, m=8) == UNSUP
+    assert qmp(N=100) == SHAPE
+    assert qmp(K=64) == SHAPE
+    assert qmp(wsb=8) == WS
+    assert qmp(ws=None) == WS
+    assert qmp(prev=p) == NULL           # prev_meta without flip_bits
+    assert qmp(W=odd) == ALIGN
+    gemm = lambda **k: L.sbn_sparse_bitlinear(k.get("xq", p), p, k.get("T", 64), p, k.get("meta", p), p,
+                                              k.get("N", 256), k.get("K", 256), None, p, k.get("dt", 0), None,
+                                              k.get("ws"), k.get("wsb", 0), None)
+    assert gemm(xq=None) == NULL
+    assert gemm(meta=None) == NULL
+    assert gemm(T=0) == SHAPE
+    assert gemm(N=130) == SHAPE
+    assert gemm(K=192) == SHAPE
+    assert gemm(dt=5) == UNSUP
+    assert gemm(xq=odd) == ALIGN
+    assert gemm(T=4, N=2560, K=2560) == WS          # decode shape needs split-K scratch
+    assert L.sbn_bitlinear(p, p, 64, None, p, 256, 256, None, p, 0, None, None, 0, None) == NULL
+
+
+def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
+    from paper_2603_05168_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError):
+        binding.lib()
