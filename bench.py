@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the 2:4-sparse ternary BitLinear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" = one pass of the whole path over the four BitNet-2B-shaped BitLinears at T = 4096
+tokens: for every layer  quantize/mask/pack(W fp32)  ->  quant_act(x bf16)  ->  sparse BitLinear
+(bf16 output).  Rank 0 prints ONE JSON line.  `value` is dense-equivalent tera-ops per second of
+the whole step (2*T*N*K summed over the four GEMMs, divided by the step time, summed over GPUs);
+the per-kernel and per-shape numbers that explain it ride along in the same line.
+
+Multi-GPU: the path has no exchange step, so N GPUs run N independent replicas ("replicas only",
+weak scaling); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_05168_b200 import inputs  # noqa: E402
+
+# NVIDIA's HGX B200 datasheet figures per GPU (dense; the sparse figure is twice that).
+DATASHEET_INT8_DENSE_TOPS = 4500.0
+DATASHEET_INT8_SPARSE_TOPS = 9000.0
+NOMINAL_BF16_DENSE_TFLOPS = 2250.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+T_TOKENS = 4096
+METRIC = "2:4 sparse ternary BitLinear TOPS, % sparse-INT8 peak, speedup vs dense ternary"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS,
+                bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def step_ops(T):
+    return sum(2.0 * T * N * K for _, K, N in inputs.SHAPES_2B)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampled during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.thread = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._reader, daemon=True)
+        self.thread.start()
+
+    def _reader(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for (ts, r) in self.rows if t0 - 0.05 <= ts <= t1 + 0.15] or [r for (_, r) in self.rows]
+        for r in rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_step(sample_tokens: int, cache: dict):
+    """One pass of the path through the CPU oracle on `sample_tokens` tokens of every layer.
+    Returns seconds."""
+    import oracle
+    if "data" not in cache:
+        cache["data"] = [(inputs.latent_weights(N, K, seed=1 + i),
+                          inputs.activations_bf16(sample_tokens, K, seed=11 + i))
+                         for i, (_, K, N) in enumerate(inputs.SHAPES_2B)]
+    t0 = time.perf_counter()
+    for W, x in cache["data"]:
+        r = oracle.quantize_mask_pack(W)
+        xq, s = oracle.quant_act(x)
+        y, _ = oracle.sparse_bitlinear(xq, s, r["vals"], r["meta"], r["scale"])
+        oracle.f32_to_bf16_bits(y)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    sample = 256
+    cache = {}
+    for _ in range(args.warmup):
+        oracle_step(sample, cache)
+    times = [oracle_step(sample, cache) for _ in range(args.steps)]
+    total = sum(times)
+    value = step_ops(sample) * args.steps / total / 1e12
+    cores = oracle.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic",
+        "config": {"workload": f"BitNet-2B-shaped BitLinears (qkv, o, gate_up, down), {sample}-token sample of the T={T_TOKENS} batch",
+                   "l2": "n/a (host)"},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} of {T_TOKENS} tokens per layer, all four weight matrices in full"},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+class Layer:
+    """Device (and pinned host) buffers of one BitLinear of the workload."""
+
+    def __init__(self, name, K, N, T, seed, torch, b):
+        self.name, self.K, self.N, self.T = name, K, N, T
+        W = inputs.latent_weights(N, K, seed=seed)
+        x = inputs.activations_bf16(T, K, seed=seed + 10)
+        self.W_host = torch.from_numpy(W).pin_memory()
+        self.x_host = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
+        self.W = self.W_host.cuda()
+        self.x = self.x_host.cuda()
+        self.W_stage = torch.empty_like(self.W)
+        self.x_stage = torch.empty_like(self.x)
+        self.packed = b.alloc_packed(N, K, with_dense=True)
+        self.xq = torch.empty((T, K), dtype=torch.int8, device="cuda")
+        self.a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+        self.y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+        self.y32 = torch.empty((T, N), dtype=torch.float32, device="cuda")
+        self.y_host = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
+        self.ws = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, K)
+        self.ops = 2.0 * T * N * K
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2603_05168_b200 import binding as b
+    from paper_2603_05168_b200 import build as sbn_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        sbn_build.build()
+    if world > 1:
+        dist.barrier()
+    b.lib()
+    peaks = load_peaks()
+    T = T_TOKENS
+    layers = [Layer(n, K, N, T, seed=1 + i, torch=torch, b=b) for i, (n, K, N) in enumerate(inputs.SHAPES_2B)]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    KERNELS = ("quantize_mask_pack", "quant_act", "sparse_bitlinear")
+
+    def step(evs=None):
+        for L in layers:
+            p = L.packed
+            if evs is not None:
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                e[0].record(stream)
+            b.sbn_quantize_mask_pack(L.W, p["vals"], p["meta"], p["w_scale"], p["ws"])
+            if evs is not None:
+                e[1].record(stream)
+            b.sbn_quant_act(L.x, L.xq, L.a_scale)
+            if evs is not None:
+                e[2].record(stream)
+            b.sbn_sparse_bitlinear(L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], L.y, ws=L.ws)
+            if evs is not None:
+                e[3].record(stream)
+                evs.append((L.name, e))
+
+    # ---- device-resident timing -----------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    b.sbn_check_status()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    evs = []
+    barrier()
+    launches0 = b.sbn_launch_count()
+    t_wall0 = time.time()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record(stream)
+    for _ in range(args.steps):
+        step(evs)
+    stop.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = b.sbn_launch_count() - launches0
+    b.sbn_check_status()
+    ms_total = start.elapsed_time(stop)
+    if world > 1:
+        tt = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_per_step = ms_total / args.steps
+    value = step_ops(T) * world / (ms_per_step * 1e-3) / 1e12
+
+    per_kernel = {k: {} for k in KERNELS}
+    for name, e in evs:
+        for i, k in enumerate(KERNELS):
+            per_kernel[k].setdefault(name, []).append(e[i].elapsed_time(e[i + 1]) * 1e3)   # us
+    kernel_us = {k: {n: statistics.mean(v) for n, v in d.items()} for k, d in per_kernel.items()}
+
+    # ---- end-to-end: host buffers, copies inside the timed region ----------------------------------
+    def e2e_step():
+        for L in layers:
+            p = L.packed
+            L.W_stage.copy_(L.W_host, non_blocking=True)
+            b.sbn_quantize_mask_pack(L.W_stage, p["vals"], p["meta"], p["w_scale"], p["ws"])
+            b.sbn_layer_forward_host(L.x_host, L.x_stage, L.xq, L.a_scale, p["w_scale"], L.y, L.y_host,
+                                     vals=p["vals"], meta=p["meta"], ws=L.ws)
+    e2e_steps = max(2, min(args.steps, 5))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    s2 = torch.cuda.Event(enable_timing=True)
+    e2 = torch.cuda.Event(enable_timing=True)
+    s2.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2.record(stream)
+    barrier()
+    b.sbn_check_status()
+    e2e_ms = s2.elapsed_time(e2)
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_ms /= e2e_steps
+    e2e_value = step_ops(T) * world / (e2e_ms * 1e-3) / 1e12
+    h2d = sum(L.W_host.numel() * 4 + L.x_host.numel() * 2 for L in layers)
+    d2h = sum(L.y_host.numel() * 2 for L in layers)
+
+    # ---- isolated kernels, cold L2 (a 512 MB buffer is overwritten before every launch) --------
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def time_cold(fn, iters):
+        ts = []
+        for _ in range(iters):
+            flush.zero_()
+            a = torch.cuda.Event(enable_timing=True)
+            c = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            c.record(stream)
+            c.synchronize()
+            ts.append(a.elapsed_time(c) * 1e3)
+        ts.sort()
+        return statistics.median(ts)
+
+    iters = 12
+    gemm = {}
+    for L in layers:
+        p = L.packed
+        b.sbn_quantize_mask_pack(L.W, p["vals"], p["meta"], p["w_scale"], p["ws"], dense_q=p["dense_q"])
+        b.sbn_quant_act(L.x, L.xq, L.a_scale)
+        row = {}
+        for tag, y in (("bf16", L.y), ("f32", L.y32)):
+            for _ in range(3):
+                b.sbn_sparse_bitlinear(L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=L.ws)
+                b.sbn_bitlinear(L.xq, L.a_scale, p["dense_q"], p["w_scale"], y, ws=L.ws)
+            sp = time_cold(lambda: b.sbn_sparse_bitlinear(L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=L.ws), iters)
+            de = time_cold(lambda: b.sbn_bitlinear(L.xq, L.a_scale, p["dense_q"], p["w_scale"], y, ws=L.ws), iters)
+            row[tag] = {"sparse_us": round(sp, 2), "dense_us": round(de, 2),
+                        "sparse_tops": round(L.ops / sp / 1e6, 1), "dense_tops": round(L.ops / de / 1e6, 1),
+                        "pct_sparse_int8_datasheet": round(100 * L.ops / sp / 1e6 / DATASHEET_INT8_SPARSE_TOPS, 1),
+                        "speedup_vs_dense": round(de / sp, 3)}
+        qmp = time_cold(lambda: b.sbn_quantize_mask_pack(L.W, p["vals"], p["meta"], p["w_scale"], p["ws"]), iters)
+        act = time_cold(lambda: b.sbn_quant_act(L.x, L.xq, L.a_scale), iters)
+        row["quantize_mask_pack_us"] = round(qmp, 2)
+        row["quantize_mask_pack_gbs"] = round(L.N * L.K * 4.625 / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
+        row["quant_act_us"] = round(act, 2)
+        row["quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act / 1e3, 1)
+        gemm[L.name] = row
+    b.sbn_check_status()
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+
+    # ---- roofline of the dominant kernel of the step -------------------------------------------------
+    tot = {k: sum(v.values()) for k, v in kernel_us.items()}
+    dominant = max(tot, key=tot.get)
+    if dominant == "sparse_bitlinear":
+        # a real contraction: sparse int8 tensor pipe.  Peak = measured bf16 burst x the nominal
+        # sparse-int8 : dense-bf16 ratio (4x).
+        ratio = DATASHEET_INT8_SPARSE_TOPS / NOMINAL_BF16_DENSE_TFLOPS
+        peak = peaks["bf16_tflops"] * ratio
+        achieved = sum(L.ops for L in layers) / (tot[dominant] * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "kernel": "bitlinear_gemm_kernel<sparse>", "achieved": round(achieved, 1),
+                    "peak": round(peak, 1), "unit": "TOP/s", "frac": round(achieved / peak, 4), "traffic": None,
+                    "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {ratio:g} (nominal sparse-int8 : bf16)",
+                    "frac_of_datasheet_sparse_int8": round(achieved / DATASHEET_INT8_SPARSE_TOPS, 4)}
+    else:
+        per_param = 4.625 if dominant == "quantize_mask_pack" else None
+        if dominant == "quantize_mask_pack":
+            bytes_ = sum(L.N * L.K * per_param for L in layers)
+        else:
+            bytes_ = sum(L.T * L.K * 3 + L.T * 4 for L in layers)
+        achieved = bytes_ / (tot[dominant] * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                    "peak_source": peaks["source"]}
+
+    # ---- CPU oracle baseline (rank 0, single GPU runs only) --------------------------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        sample = 1024
+        secs = oracle_step(sample, {})
+        cpu_baseline = {"value": step_ops(sample) / secs / 1e12, "unit": "TOPS", "cores": oracle.num_threads(),
+                        "kind": "oracle", "seconds": round(secs, 2),
+                        "sample": f"{sample} of {T} tokens per layer, all four weight matrices in full, one pass"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": f"BitNet-2B-shaped BitLinears at T={T}: qkv 2560->3840, o 2560->2560, gate_up 2560->6912, down 6912->2560; "
+                                   "step = quantize_mask_pack + quant_act + sparse_bitlinear (bf16 out) per layer",
+                       "tokens": T, "parallelism": "replicas" if world > 1 else "single",
+                       "l2": "step streams 327 MB of inputs (> 126 MB L2); isolated-kernel numbers flush L2 before every launch"},
+            "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roofline,
+            "cpu_baseline": cpu_baseline,
+            "kernel_us_in_step": {k: {n: round(v, 2) for n, v in d.items()} for k, d in kernel_us.items()},
+            "isolated": gemm,
+            "datasheet_int8_tops": {"dense": DATASHEET_INT8_DENSE_TOPS, "sparse": DATASHEET_INT8_SPARSE_TOPS},
+            "measured_peaks": peaks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -35,7 +35,11 @@ constexpr int kGemmThreads = 192;
 constexpr int kBM = 128;                 // output features per tile (MMA M)
 constexpr int kBK = 128;                 // logical K per pipeline stage
 constexpr uint32_t kTmemCols = 512;
-constexpr int kSmemBudget = 220 * 1024;  // of the 227 KB a CTA may use
+constexpr int kSmemBudget = 224 * 1024;  // of the 227 KB a CTA may use
+constexpr int kEpiWarpBufBytes = 32 * 32 * 4;                 // one 32-token x 32-feature fp32 slab
+constexpr int kEpiBytes = 4 * 2 * kEpiWarpBufBytes;           // 4 epilogue warps, double buffered
+constexpr int kScaleBytes = 4 * 256 * 4;                      // per-token scales, one copy per epilogue warp
+constexpr int kBarrierBytes = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 struct GemmParams {
@@ -108,6 +112,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         " [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
         : "memory");
+}
+// Tile store smem -> global (rows beyond the tensor's extent are clipped by the hardware).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(src) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
@@ -185,14 +195,14 @@ struct GemmConfig {
     static constexpr int B_BYTES = BN * kBK;
     static constexpr int E_BYTES = SPARSE ? kBM * (kBK / 8) : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-    static constexpr int STAGES_RAW = kSmemBudget / STAGE_BYTES;
+    static constexpr int STAGES_RAW = (kSmemBudget - 1024 - kEpiBytes - kScaleBytes - kBarrierBytes) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
     static constexpr int META_COLS = SPARSE ? 4 * STAGES : 0;
     static constexpr int ACC_STAGES = (2 * BN + META_COLS <= static_cast<int>(kTmemCols)) ? 2 : 1;
     static constexpr int META_COL0 = ACC_STAGES * BN;
     static constexpr uint32_t TX_BYTES = STAGE_BYTES;
     // dynamic smem: 1 KB alignment slack + stages + barriers
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + kEpiBytes + kScaleBytes + kBarrierBytes;
     static_assert(STAGES >= 2, "tile too large for shared memory");
     static_assert(ACC_STAGES * BN + META_COLS <= static_cast<int>(kTmemCols), "TMEM overflow");
 };
@@ -205,6 +215,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                       const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_e,
+                      const __grid_constant__ CUtensorMap tmap_y,
                       const GemmParams p) {
     using Cfg = GemmConfig<SPARSE, BN>;
     constexpr int STAGES = Cfg::STAGES;
@@ -216,7 +227,9 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t smem_a = smem_base;
     const uint32_t smem_b = smem_a + STAGES * Cfg::A_BYTES;
     const uint32_t smem_e = smem_b + STAGES * Cfg::B_BYTES;
-    const uint32_t bar_base = smem_base + STAGES * Cfg::STAGE_BYTES;     // 8 B aligned
+    const uint32_t smem_epi = smem_base + STAGES * Cfg::STAGE_BYTES;     // 1 KB aligned
+    const uint32_t smem_scale = smem_epi + kEpiBytes;                    // float [4][256]
+    const uint32_t bar_base = smem_scale + kScaleBytes;                  // 8 B aligned
     const uint32_t bar_full = bar_base;                       // [STAGES]   TMA -> MMA
     const uint32_t bar_empty = bar_full + 8 * STAGES;         // [STAGES]   MMA -> TMA
     const uint32_t bar_acc_full = bar_empty + 8 * STAGES;     // [ACC]      MMA -> epilogue
@@ -337,20 +350,37 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else {
         // ------------------------------------------------------------------ epilogue (4 warps)
+        // Each warp owns one TMEM lane quarter (32 output features) and works on its own:
+        // private scale staging, private double-buffered 32x32 output slab, private TMA stores.
         const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
+        const int ew = warp - 2;                          // 0..3: index of this epilogue warp
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const float w_scale = __ldg(p.w_scale);
+        uint8_t* const smem_generic = smem_raw + (smem_base - smem_u32(smem_raw));
+        const uint32_t slab_u32 = smem_epi + static_cast<uint32_t>(ew * 2 * kEpiWarpBufBytes);
+        uint8_t* const slab_ptr = smem_generic + (slab_u32 - smem_base);
+        float* const scale_s = reinterpret_cast<float*>(smem_generic + (smem_scale - smem_base)) + ew * 256;
         int acc = 0;
         uint32_t acc_phase = 0;
+        int buf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             const int mt = (tile / p.k_splits) % tiles_m;
             const int tt = (tile / p.k_splits) / tiles_m;
-            const int n = mt * kBM + quarter * 32 + lane;         // output feature of this thread
+            const int n0 = mt * kBM + quarter * 32;
+            const int n = n0 + lane;                              // output feature of this thread
             const int t0 = tt * BN;
+            // s absorbs both scales (Eq. 4): stage w_scale * a_scale[t] for the tile's tokens
+            __syncwarp();
+#pragma unroll
+            for (int i = lane; i < BN; i += 32) {
+                const int t = t0 + i;
+                scale_s[i] = t < p.T ? __fmul_rn(w_scale, __ldg(p.a_scale + t)) : 0.0f;
+            }
+            const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
+            __syncwarp();
             if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
-            const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
@@ -363,34 +393,72 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
                 }
                 const int tc = t0 + c * 32;
+                if (tc >= p.T) continue;                          // whole chunk beyond the last token
                 if (p.k_splits > 1) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int t = tc + j;
                         if (t < p.T) atomicAdd(p.split_acc + static_cast<size_t>(t) * p.N + n, static_cast<int>(r[j]));
                     }
-                } else {
+                    continue;
+                }
+                if (p.acc_out) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int t = tc + j;
-                        if (t < p.T) {
-                            const size_t o = static_cast<size_t>(t) * p.N + n;
-                            const int a = static_cast<int>(r[j]);
-                            if (p.acc_out) p.acc_out[o] = a;
-                            const float s = __fmul_rn(w_scale, __ldg(p.a_scale + t));
-                            float v = __fmul_rn(static_cast<float>(a), s);
-                            if (p.bias) v = __fadd_rn(v, bias);
-                            if (p.out_bf16) {
-                                static_cast<uint16_t*>(p.y)[o] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-                            } else {
-                                static_cast<float*>(p.y)[o] = v;
-                            }
-                        }
+                        if (t < p.T) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(r[j]);
                     }
                 }
+                // the slab written two chunks ago must have been read by its TMA store
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                uint8_t* const slab = slab_ptr + buf * kEpiWarpBufBytes;
+                const float4* sc4 = reinterpret_cast<const float4*>(scale_s + c * 32);
+                if (p.out_bf16) {
+                    uint16_t* o = reinterpret_cast<uint16_t*>(slab) + lane;
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 sc = sc4[j4];
+                        float v0 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 0])), sc.x);
+                        float v1 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 1])), sc.y);
+                        float v2 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 2])), sc.z);
+                        float v3 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 3])), sc.w);
+                        if (p.bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); v2 = __fadd_rn(v2, bias); v3 = __fadd_rn(v3, bias); }
+                        o[(4 * j4 + 0) * 32] = static_cast<uint16_t>(f32_to_bf16_rne(v0));
+                        o[(4 * j4 + 1) * 32] = static_cast<uint16_t>(f32_to_bf16_rne(v1));
+                        o[(4 * j4 + 2) * 32] = static_cast<uint16_t>(f32_to_bf16_rne(v2));
+                        o[(4 * j4 + 3) * 32] = static_cast<uint16_t>(f32_to_bf16_rne(v3));
+                    }
+                } else {
+                    float* o = reinterpret_cast<float*>(slab) + lane;
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 sc = sc4[j4];
+                        float v0 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 0])), sc.x);
+                        float v1 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 1])), sc.y);
+                        float v2 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 2])), sc.z);
+                        float v3 = __fmul_rn(static_cast<float>(static_cast<int>(r[4 * j4 + 3])), sc.w);
+                        if (p.bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); v2 = __fadd_rn(v2, bias); v3 = __fadd_rn(v3, bias); }
+                        o[(4 * j4 + 0) * 32] = v0;
+                        o[(4 * j4 + 1) * 32] = v1;
+                        o[(4 * j4 + 2) * 32] = v2;
+                        o[(4 * j4 + 3) * 32] = v3;
+                    }
+                }
+                // generic-proxy writes -> visible to the async proxy, then one lane issues the store
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmap_y, n0, tc, slab_u32 + static_cast<uint32_t>(buf * kEpiWarpBufBytes));
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                buf ^= 1;
             }
             if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
         }
+        // the slabs must stay valid until the stores have read them, and the writes must be done
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __syncwarp();
     }
 
     // teardown: everyone meets here (also on the abort path), then the allocating warp frees TMEM

@@ -39,6 +39,22 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// 2-D row-major output tensor y [T][N] (fp32 or bf16) with a 32 x 32 element box.
+static bool encode_2d_out(CUtensorMap* map, const void* base, uint64_t N, uint64_t T, bool bf16) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const uint64_t es = bf16 ? 2 : 4;
+    cuuint64_t dims[2] = {N, T};
+    cuuint64_t strides[1] = {N * es};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // 2-D uint8 row-major tensor [rows][cols_bytes] with a [box_rows][box_cols] box.
 static bool encode_2d_u8(CUtensorMap* map, const void* base, uint64_t cols_bytes, uint64_t rows,
                          uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle swz) {
@@ -91,7 +107,7 @@ static size_t gemm_workspace_bytes(int T, int N, int K) {
 
 template <bool SPARSE, int BN>
 static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
-                                  const GemmParams& p, cudaStream_t stream) {
+                                  const CUtensorMap& ty, const GemmParams& p, cudaStream_t stream) {
     using Cfg = GemmConfig<SPARSE, BN>;
     static bool configured = false;
     auto kernel = bitlinear_gemm_kernel<SPARSE, BN>;
@@ -102,7 +118,7 @@ static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, 
     }
     const int tiles = (p.N / kBM) * ((p.T + BN - 1) / BN) * p.k_splits;
     const int grid = tiles < kNumSMs ? tiles : kNumSMs;
-    kernel<<<grid, kGemmThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, p);
+    kernel<<<grid, kGemmThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, p);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -128,7 +144,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
         if (cudaMemsetAsync(ws, 0, need, stream) != cudaSuccess) return SBN_ERR_CUDA;
     }
 
-    CUtensorMap ta, tb, te;
+    CUtensorMap ta, tb, te, ty;
     bool ok;
     if (sparse) {
         ok = encode_2d_u8(&ta, wvals, static_cast<uint64_t>(K) / 2, N, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B) &&
@@ -138,6 +154,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
         te = ta;
     }
     ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16);
     if (!ok) return SBN_ERR_CUDA;
 
     GemmParams p;
@@ -151,7 +168,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     p.split_counters = nullptr;
 
     sbn_status st;
-#define SBN_GEMM_CASE(S, B) st = launch_gemm_cfg<S, B>(ta, tb, te, p, stream)
+#define SBN_GEMM_CASE(S, B) st = launch_gemm_cfg<S, B>(ta, tb, te, ty, p, stream)
     if (sparse) {
         if (bn == 64) SBN_GEMM_CASE(true, 64); else if (bn == 128) SBN_GEMM_CASE(true, 128); else SBN_GEMM_CASE(true, 256);
     } else {
