@@ -52,7 +52,8 @@ typedef enum {
     SBN_ERR_UNSUPPORTED = 4, /* pattern other than 2:4, unknown dtype or op */
     SBN_ERR_WORKSPACE = 5,   /* workspace missing or smaller than sbn_workspace_bytes() */
     SBN_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, tensor map, ...) */
-    SBN_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (see sbn_check_status) */
+    SBN_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (see sbn_check_status) */
+    SBN_ERR_TOO_LARGE = 8    /* problem exceeds what the library's built-in scratch can serve */
 } sbn_status;
 
 typedef enum { SBN_OUT_F32 = 0, SBN_OUT_BF16 = 1 } sbn_out_dtype;
@@ -94,6 +95,41 @@ sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int 
                                   int8_t *vals, uint8_t *meta, float *w_scale, int8_t *dense_q,
                                   const uint8_t *prev_meta, unsigned long long *flip_bits,
                                   void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Same operation as sbn_quantize_mask_pack, for callers that have no workspace to give.
+ * (The paper has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Some hosts of this library cannot obtain device memory at the point where they call it: a
+ * framework that reserved nearly all of the GPU for its own pool at start-up (cudaMalloc then
+ * fails, and the pool cannot be asked from plain C), a plug-in whose "enqueue" hook is forbidden
+ * to allocate, or a latency-critical loop that must avoid cudaMalloc because it synchronises the
+ * whole device.  For them the scratch of the two-pass quantiser (the per-CTA partial sums of
+ * |W|) lives in a fixed array inside the library image: SBN_STATIC_SCRATCH_BYTES bytes of
+ * device memory that every GPU which loads the library keeps until the process exits.
+ *
+ * Arguments are those of sbn_quantize_mask_pack without ws/ws_bytes; inputs and outputs are
+ * still the caller's buffers, and the results are bit-identical to that call's.
+ * Limits and rules
+ *   - N*K must not exceed SBN_STATIC_MAX_ELEMS, and the scratch the shape needs must fit in
+ *     SBN_STATIC_SCRATCH_BYTES; otherwise SBN_ERR_TOO_LARGE is returned and nothing is launched.
+ *   - The call itself never allocates or frees memory (no cudaMalloc/cudaFree, no allocating
+ *     library routine).
+ *   - The first call on each device looks up the device address of the built-in array (once per
+ *     device, with that device current).  Make that first call before starting any stream
+ *     capture on the device.
+ *   - All calls on one device share the one array, and it keeps whatever the last call left in
+ *     it (each call overwrites every slot it later reads, so nothing needs clearing).  Two such
+ *     calls that may overlap on the GPU -- different streams, no ordering between them -- race
+ *     on it and give wrong scales; order them, or use sbn_quantize_mask_pack with separate
+ *     workspaces.
+ */
+#define SBN_STATIC_SCRATCH_BYTES 8192
+#define SBN_STATIC_MAX_ELEMS (1ll << 28)
+sbn_status sbn_quantize_mask_pack_static_ws(const float *W, int N, int K, int n_keep, int m_group,
+                                            int8_t *vals, uint8_t *meta, float *w_scale,
+                                            int8_t *dense_q, const uint8_t *prev_meta,
+                                            unsigned long long *flip_bits, void *stream);
 
 /*
  * Part 2 -- per-token absmax int8 activation quantiser (Sec. 2.1; Algorithm 2, forward step 1):

@@ -21,7 +21,7 @@ OUT_F32, OUT_BF16 = 0, 1
 OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
 
 EXPORTS = [
-    "sbn_workspace_bytes", "sbn_quantize_mask_pack", "sbn_quant_act", "sbn_sparse_bitlinear",
+    "sbn_workspace_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quant_act", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sbn_quantize_mask_pack.restype = i32
         L.sbn_quantize_mask_pack.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.sbn_quantize_mask_pack_static_ws.restype = i32
+        L.sbn_quantize_mask_pack_static_ws.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.sbn_quant_act.restype = i32
         L.sbn_quant_act.argtypes = [vp, i32, i32, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
@@ -97,6 +99,17 @@ def sbn_quantize_mask_pack(W, vals, meta, w_scale, ws, dense_q=None, prev_meta=N
                                         _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta), _ptr(flip_bits),
                                         _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "sbn_quantize_mask_pack")
+
+
+def sbn_quantize_mask_pack_static_ws(W, vals, meta, w_scale, dense_q=None, prev_meta=None, flip_bits=None,
+                                     n_keep: int = 2, m_group: int = 4):
+    """Workspace-free variant: the scratch is a fixed array inside the library (see sbn.h for
+    its limits and the rule about overlapping calls)."""
+    N, K = W.shape
+    _check(lib().sbn_quantize_mask_pack_static_ws(_ptr(W), N, K, n_keep, m_group, _ptr(vals), _ptr(meta),
+                                                  _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta),
+                                                  _ptr(flip_bits), _stream()),
+           "sbn_quantize_mask_pack_static_ws")
 
 
 def sbn_quant_act(x_bf16, xq, a_scale):

@@ -188,6 +188,31 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     return SBN_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Built-in scratch for sbn_quantize_mask_pack_static_ws: part of the library image, so callers
+// that cannot allocate still have somewhere to put the pass-1 partial sums.  In host code the
+// symbol below is only a handle; its device address is looked up once per device.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[SBN_STATIC_SCRATCH_BYTES];
+static_assert(sizeof(QmpWorkspace) <= SBN_STATIC_SCRATCH_BYTES, "built-in scratch too small");
+
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices] = {};
+static std::mutex g_static_scratch_mutex;
+
+// Device address of g_static_scratch on the current device (nullptr on failure).
+static void* static_scratch_for_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    return g_static_scratch_addr[dev];
+}
+
 }  // namespace sbn
 
 // ------------------------------------------------------------------------------------------------
@@ -224,6 +249,32 @@ sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int 
         return SBN_ERR_ALIGN;
     return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(ws)->partial,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_keep, int m_group,
+                                            int8_t* vals, uint8_t* meta, float* w_scale,
+                                            int8_t* dense_q, const uint8_t* prev_meta,
+                                            unsigned long long* flip_bits, void* stream) {
+    // size limits first: nothing below runs for a shape the built-in scratch cannot serve
+    if (N > 0 && K > 0) {
+        if (static_cast<long long>(N) * K > SBN_STATIC_MAX_ELEMS) return SBN_ERR_TOO_LARGE;
+        if (sbn_workspace_bytes(SBN_OP_QUANTIZE_MASK_PACK, 0, N, K) > SBN_STATIC_SCRATCH_BYTES)
+            return SBN_ERR_TOO_LARGE;
+    }
+    if (!W || !vals || !meta || !w_scale) return SBN_ERR_NULL;
+    if (prev_meta && !flip_bits) return SBN_ERR_NULL;
+    if (n_keep != 2 || m_group != 4) return SBN_ERR_UNSUPPORTED;
+    if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(W, 16) || misaligned(vals, 16) || misaligned(meta, 16) || misaligned(w_scale, 4) ||
+        (dense_q && misaligned(dense_q, 16)) || (prev_meta && misaligned(prev_meta, 16)) ||
+        (flip_bits && misaligned(flip_bits, 8)))
+        return SBN_ERR_ALIGN;
+    void* scratch = static_scratch_for_current_device();
+    if (!scratch) return SBN_ERR_CUDA;
+    // pass 1 writes every partial slot that pass 2 reads, so stale contents are harmless
+    return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+                                     static_cast<QmpWorkspace*>(scratch)->partial,
                                      static_cast<cudaStream_t>(stream));
 }
 
@@ -295,6 +346,7 @@ const char* sbn_status_string(sbn_status s) {
         case SBN_ERR_WORKSPACE: return "workspace missing or too small";
         case SBN_ERR_CUDA: return "CUDA call failed";
         case SBN_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case SBN_ERR_TOO_LARGE: return "problem larger than the library's built-in scratch can serve";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,74 @@
+"""The workspace-free entry point sbn_quantize_mask_pack_static_ws.
+
+It serves callers that cannot allocate device memory where they call the library (a framework
+that owns the whole GPU through its own pool, a plug-in hook that must not allocate, a loop that
+cannot afford cudaMalloc's device-wide synchronisation): its scratch is a fixed array inside the
+library.  The GPU test drives it through the C ABI, twice in a row on different shapes, and
+requires the very same bits as sbn_quantize_mask_pack with a caller-provided workspace -- the
+second call also shows that whatever the first one left in the shared array does no harm.
+
+This file is named so that pytest collects it last.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_05168_b200 import binding as b
+from paper_2603_05168_b200 import build as sbn_build
+from paper_2603_05168_b200 import inputs
+
+
+def test_static_ws_rejects_oversized_problem_on_host():
+    # host-side check only: runs before anything touches the GPU, so fake pointers are fine
+    sbn_build.build()
+    L = b.lib()
+    p = ctypes.c_void_p(0x1000)
+    too_large = 8
+    # 32768 x 16384 = 2^29 elements > SBN_STATIC_MAX_ELEMS (2^28)
+    rc = L.sbn_quantize_mask_pack_static_ws(p, 32768, 16384, 2, 4, p, p, p, None, None, None, None)
+    assert rc == too_large
+    assert "scratch" in b.status_string(rc)
+    # ordinary argument errors are still reported as such
+    assert L.sbn_quantize_mask_pack_static_ws(None, 256, 256, 2, 4, p, p, p, None, None, None, None) == 1
+    assert L.sbn_quantize_mask_pack_static_ws(p, 256, 256, 6, 8, p, p, p, None, None, None, None) == 4
+    assert L.sbn_quantize_mask_pack_static_ws(p, 100, 256, 2, 4, p, p, p, None, None, None, None) == 2
+
+
+def _run_both(W_np, prev_meta_np=None):
+    N, K = W_np.shape
+    W = torch.from_numpy(W_np).cuda()
+    ref = b.alloc_packed(N, K, with_dense=True)
+    got = b.alloc_packed(N, K, with_dense=True)
+    prev_a = prev_b = flip_a = flip_b = None
+    if prev_meta_np is not None:
+        prev_a = torch.from_numpy(prev_meta_np).cuda()
+        prev_b = prev_a.clone()
+        flip_a = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+        flip_b = torch.full((1,), -2, dtype=torch.int64, device="cuda")
+    b.sbn_quantize_mask_pack(W, ref["vals"], ref["meta"], ref["w_scale"], ref["ws"], dense_q=ref["dense_q"],
+                             prev_meta=prev_a, flip_bits=flip_a)
+    b.sbn_quantize_mask_pack_static_ws(W, got["vals"], got["meta"], got["w_scale"], dense_q=got["dense_q"],
+                                       prev_meta=prev_b, flip_bits=flip_b)
+    b.sbn_check_status()
+    for key in ("vals", "meta", "w_scale", "dense_q"):
+        assert torch.equal(ref[key], got[key]), key
+    if flip_a is not None:
+        assert int(flip_a.item()) == int(flip_b.item()) >= 0
+    return ref
+
+
+@pytest.mark.gpu
+def test_static_ws_matches_workspace_entry_point_twice_in_a_row():
+    # first call: a large matrix that fills every slot of the shared scratch
+    W1 = inputs.latent_weights(2560, 2560, seed=31)
+    r1 = _run_both(W1)
+    # second call right after it: a small matrix with a different scale that uses only a few
+    # slots -- stale partial sums of the first call must not leak into its gamma
+    W2 = inputs.latent_weights(128, 256, seed=32, sigma=0.5)
+    r2 = _run_both(W2)
+    assert float(r2["w_scale"].item()) > 10 * float(r1["w_scale"].item())
+    # and once more with the flip count enabled
+    W3 = inputs.perturb_weights(W1, seed=33, sigma=1e-4)
+    _run_both(W3, prev_meta_np=r1["meta"].cpu().numpy())
