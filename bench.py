@@ -38,6 +38,12 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
 T_TOKENS = 4096
+# name -> (tokens, [(layer, K, N)], weight sigma, outlier prob, per-token lognormal sigma)
+WORKLOADS = {
+    "2b": (4096, inputs.SHAPES_2B, 0.02, 0.0, 0.0),
+    "7b": (8192, inputs.SHAPES_7B, 0.015, 0.05, 0.5),
+    "down7b": (8192, inputs.SHAPES_7B[1:], 0.015, 0.05, 0.5),      # one layer: small case for profiling
+}
 METRIC = "2:4 sparse ternary BitLinear TOPS, % sparse-INT8 peak, speedup vs dense ternary"
 
 
@@ -53,8 +59,8 @@ def load_peaks():
                 bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def step_ops(T):
-    return sum(2.0 * T * N * K for _, K, N in inputs.SHAPES_2B)
+def step_ops(T, shapes=inputs.SHAPES_2B):
+    return sum(2.0 * T * N * K for _, K, N in shapes)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -172,10 +178,10 @@ def run_reference(args):
 class Layer:
     """Device (and pinned host) buffers of one BitLinear of the workload."""
 
-    def __init__(self, name, K, N, T, seed, torch, b):
+    def __init__(self, name, K, N, T, seed, torch, b, sigma=0.02, outl=0.0, logn=0.0):
         self.name, self.K, self.N, self.T = name, K, N, T
-        W = inputs.latent_weights(N, K, seed=seed)
-        x = inputs.activations_bf16(T, K, seed=seed + 10)
+        W = inputs.latent_weights(N, K, seed=seed, sigma=sigma, outlier_prob=outl)
+        x = inputs.activations_bf16(T, K, seed=seed + 10, token_lognormal_sigma=logn)
         self.W_host = torch.from_numpy(W).pin_memory()
         self.x_host = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
         self.W = self.W_host.cuda()
@@ -211,8 +217,10 @@ def run_ours(args):
         dist.barrier()
     b.lib()
     peaks = load_peaks()
-    T = T_TOKENS
-    layers = [Layer(n, K, N, T, seed=1 + i, torch=torch, b=b) for i, (n, K, N) in enumerate(inputs.SHAPES_2B)]
+    T, shapes, sigma, outl, logn = WORKLOADS[args.workload]
+    layers = [Layer(n, K, N, T, seed=1 + i, torch=torch, b=b, sigma=sigma, outl=outl, logn=logn)
+              for i, (n, K, N) in enumerate(shapes)]
+    in_bytes = sum(L.W.numel() * 4 + L.x.numel() * 2 for L in layers)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -267,13 +275,23 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms_total = float(tt.item())
     ms_per_step = ms_total / args.steps
-    value = step_ops(T) * world / (ms_per_step * 1e-3) / 1e12
+    value = step_ops(T, shapes) * world / (ms_per_step * 1e-3) / 1e12
 
     per_kernel = {k: {} for k in KERNELS}
     for name, e in evs:
         for i, k in enumerate(KERNELS):
             per_kernel[k].setdefault(name, []).append(e[i].elapsed_time(e[i + 1]) * 1e3)   # us
     kernel_us = {k: {n: statistics.mean(v) for n, v in d.items()} for k, d in per_kernel.items()}
+
+    if args.only_step:
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": "TOPS", "ms_per_step": ms_per_step,
+                              "workload": args.workload, "gpu_launches": int(launches),
+                              "kernel_us_in_step": {k: {n: round(v, 2) for n, v in d.items()} for k, d in kernel_us.items()}}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end-to-end: host buffers, copies inside the timed region ----------------------------------
     def e2e_step():
@@ -301,7 +319,7 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_ms = float(tt.item())
     e2e_ms /= e2e_steps
-    e2e_value = step_ops(T) * world / (e2e_ms * 1e-3) / 1e12
+    e2e_value = step_ops(T, shapes) * world / (e2e_ms * 1e-3) / 1e12
     h2d = sum(L.W_host.numel() * 4 + L.x_host.numel() * 2 for L in layers)
     d2h = sum(L.y_host.numel() * 2 for L in layers)
 
@@ -376,7 +394,7 @@ def run_ours(args):
 
     # ---- CPU oracle baseline (rank 0, single GPU runs only) --------------------------------------------
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == "2b":
         import oracle
         sample = 1024
         secs = oracle_step(sample, {})
@@ -389,10 +407,10 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": {"workload": f"BitNet-2B-shaped BitLinears at T={T}: qkv 2560->3840, o 2560->2560, gate_up 2560->6912, down 6912->2560; "
-                                   "step = quantize_mask_pack + quant_act + sparse_bitlinear (bf16 out) per layer",
+            "config": {"workload": f"{args.workload}: BitLinears at T={T}: " + ", ".join(f"{n} {K}->{N}" for n, K, N in shapes) +
+                                   "; step = quantize_mask_pack + quant_act + sparse_bitlinear (bf16 out) per layer",
                        "tokens": T, "parallelism": "replicas" if world > 1 else "single",
-                       "l2": "step streams 327 MB of inputs (> 126 MB L2); isolated-kernel numbers flush L2 before every launch"},
+                       "l2": f"step streams {in_bytes / 1e6:.0f} MB of inputs (> 126 MB L2); isolated-kernel numbers flush L2 before every launch"},
             "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
@@ -416,6 +434,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS),
+                    help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling)")
+    ap.add_argument("--only-step", action="store_true", help="time the step only (used for profiler runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
