@@ -193,9 +193,11 @@ sbn_status sbn_check_status(void *stream);
 /* Static string for a status code. */
 const char *sbn_status_string(sbn_status s);
 
-/* Tuning/diagnostic knob (host state, not thread-safe): force the token-tile width of the GEMM
- * kernels to 64, 128 or 256 (0 = automatic), and the split-K factor (0 = automatic).  Results
- * do not depend on it. */
+/* Tuning/diagnostic knob (host state, not thread-safe).  token_tile: 0 = automatic; 64, 128 or
+ * 256 = force the single-CTA kernel with that token-tile width; a negative value -BN = force the
+ * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
+ * 256 dense).  split_k: split-K factor of the single-CTA kernel (0 = automatic).  Results do not
+ * depend on it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);
 
 /* Number of kernels the library has launched since it was loaded (all calls, all streams). */

@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "sbn.h"
@@ -11,6 +12,7 @@
 #include "quant_act.cuh"
 #include "quantize_mask_pack.cuh"
 #include "gemm_tcgen05.cuh"
+#include "gemm_pair_tcgen05.cuh"
 
 namespace sbn {
 
@@ -39,14 +41,15 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D row-major output tensor y [T][N] (fp32 or bf16) with a 32 x 32 element box.
-static bool encode_2d_out(CUtensorMap* map, const void* base, uint64_t N, uint64_t T, bool bf16) {
+// 2-D row-major output tensor y [T][N] (fp32 or bf16) with a 32-feature x box_tokens box.
+static bool encode_2d_out(CUtensorMap* map, const void* base, uint64_t N, uint64_t T, bool bf16,
+                          uint32_t box_tokens) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const uint64_t es = bf16 ? 2 : 4;
     cuuint64_t dims[2] = {N, T};
     cuuint64_t strides[1] = {N * es};
-    cuuint32_t box[2] = {32, 32};
+    cuuint32_t box[2] = {32, box_tokens};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -123,6 +126,98 @@ static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, 
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
+// ---- CTA-pair kernel (large T) -------------------------------------------------------------------
+// Token-tile width for the pair kernel: a small cost model of (operand ingest | MMA rate) per unit
+// of K, the accumulator drain per tile, and the number of waves over the 74 CTA pairs.
+static int pick_pair_bn(bool sparse, int T, int N, int K) {
+    if (g_force_token_tile < 0) {
+        int bn = -g_force_token_tile;
+        const int cap = sparse ? kPairMaxBnSparse : kPairMaxBnDense;
+        bn = (bn / 16) * 16;
+        if (bn < 16) bn = 16;
+        if (bn > cap) bn = cap;
+        return bn;
+    }
+    const int cap = sparse ? kPairMaxBnSparse : kPairMaxBnDense;
+    const double mac_rate = sparse ? 16384.0 : 8192.0;          // MAC / clk / SM
+    const double ingest = 64.0;                                  // B / clk / SM
+    const int full_m = N / 512, rem_m = (N % 512) ? 1 : 0;
+    int best = 128;
+    double best_cost = 1e300;
+    for (int bn = 64; bn <= cap; bn += 16) {
+        const int tt = (T + bn - 1) / bn;
+        auto tile_clk = [&](int mtiles) {
+            const double a_bytes = sparse ? 72.0 : 128.0;
+            const double bytes = mtiles * a_bytes + bn / 2.0;
+            const double macs = mtiles * 128.0 * bn;
+            const double per_k = std::max(bytes / ingest, macs / mac_rate);
+            return per_k * K + 12.0 * bn + 600.0;                // + drain and tile turnaround
+        };
+        // greedy waves: full tiles first, then the half tiles
+        const double work = static_cast<double>(full_m) * tt * tile_clk(2) + static_cast<double>(rem_m) * tt * tile_clk(1);
+        const long tiles = static_cast<long>(full_m + rem_m) * tt;
+        const long waves = (tiles + 73) / 74;
+        const double balanced = work / 74.0;
+        const double quantised = static_cast<double>(waves) * tile_clk(2);
+        const double cost = std::max(balanced, 0.5 * (balanced + quantised));
+        if (cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+template <bool SPARSE>
+static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
+                              const CUtensorMap& ty, const PairParams& pp, cudaStream_t stream) {
+    using Cfg = PairConfig<SPARSE>;
+    static bool configured = false;
+    auto kernel = bitlinear_gemm_pair_kernel<SPARSE>;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        configured = true;
+    }
+    const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
+    const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
+    kernel<<<2 * pairs, kPairThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, pp);
+    ++g_launch_count;
+    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
+static inline bool use_pair_kernel(int T) {
+    if (g_force_token_tile < 0) return true;
+    if (g_force_token_tile > 0) return false;
+    return T >= 256;
+}
+
+static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_scale, int T,
+                                const int8_t* wvals, const uint8_t* meta, const float* w_scale,
+                                int N, int K, const float* bias, void* y, sbn_out_dtype dt,
+                                int32_t* acc_out, cudaStream_t stream) {
+    const int bn = pick_pair_bn(sparse, T, N, K);
+    CUtensorMap ta, tb, te, ty;
+    bool ok;
+    if (sparse) {
+        ok = encode_2d_u8(&ta, wvals, static_cast<uint64_t>(K) / 2, N, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B) &&
+             encode_2d_u8(&te, meta, static_cast<uint64_t>(K) / 8, N, kBK / 8, kBM, CU_TENSOR_MAP_SWIZZLE_NONE);
+    } else {
+        ok = encode_2d_u8(&ta, wvals, K, N, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+        te = ta;
+    }
+    ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, 16);
+    if (!ok) return SBN_ERR_CUDA;
+    PairParams pp;
+    pp.g.T = T; pp.g.N = N; pp.g.K = K;
+    pp.g.k_blocks_total = K / kBK;
+    pp.g.k_splits = 1;
+    pp.g.a_scale = a_scale; pp.g.w_scale = w_scale; pp.g.bias = bias;
+    pp.g.y = y; pp.g.out_bf16 = (dt == SBN_OUT_BF16);
+    pp.g.acc_out = acc_out;
+    pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
+    pp.bn = bn;
+    return sparse ? launch_pair<true>(ta, tb, te, ty, pp, stream) : launch_pair<false>(ta, tb, te, ty, pp, stream);
+}
+
 static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, int T,
                            const int8_t* wvals, const uint8_t* meta, const float* w_scale,
                            int N, int K, const float* bias, void* y, sbn_out_dtype dt,
@@ -134,6 +229,9 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
         misaligned(y, 16) || misaligned(a_scale, 4) || misaligned(w_scale, 4) ||
         (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)))
         return SBN_ERR_ALIGN;
+
+    if (use_pair_kernel(T))
+        return run_gemm_pair(sparse, xq, a_scale, T, wvals, meta, w_scale, N, K, bias, y, dt, acc_out, stream);
 
     const int bn = pick_token_tile(T);
     const int splits = pick_split_k(T, N, K, bn);
@@ -154,7 +252,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
         te = ta;
     }
     ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16);
+    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, 32);
     if (!ok) return SBN_ERR_CUDA;
 
     GemmParams p;

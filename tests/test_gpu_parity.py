@@ -194,6 +194,29 @@ def test_gemm_parity_every_token_tile(sparse, tile):
     _assert_y(y_to_f32_numpy(y), y_ref)
 
 
+PAIR_CASES = [  # (T, N, K, BN): CTA-pair kernel, forced tile widths incl. ragged T and odd N/128
+    (333, 128, 256, 64), (333, 256, 128, 16), (40, 384, 512, 48), (500, 640, 384, 144),
+    (700, 1024, 1280, 240), (257, 1152, 2560, 96), (1000, 512, 6912, 240),
+]
+
+
+@pytest.mark.parametrize("sparse", [True, False])
+@pytest.mark.parametrize("T,N,K,bn", PAIR_CASES)
+def test_gemm_parity_pair_kernel(sparse, T, N, K, bn):
+    r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=bn + T)
+    b.sbn_set_gemm_tuning(-bn, 0)
+    if sparse:
+        y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    else:
+        y_ref, acc_ref = oracle.bitlinear(xq_ref, s_ref, r["dense_q"], r["scale"])
+    y, acc = gpu_gemm(sparse, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    yb, _ = gpu_gemm(sparse, xq, a_scale, g["dev"], out_dtype=torch.bfloat16, want_acc=False)
+    ref_bits = oracle.f32_to_bf16_bits(y_ref).astype(np.int32)
+    assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
+
+
 @pytest.mark.parametrize("sparse", [True, False])
 @pytest.mark.parametrize("split", [2, 5, 10])
 def test_gemm_parity_split_k(sparse, split):
