@@ -189,7 +189,7 @@ class Layer:
         self.W_stage = torch.empty_like(self.W)
         self.x_stage = torch.empty_like(self.x)
         self.packed = b.alloc_packed(N, K, with_dense=True)
-        self.xq = torch.empty((T, K), dtype=torch.int8, device="cuda")
+        self.xq = b.alloc_xq(T, K)
         self.a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
         self.y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
         self.y32 = torch.empty((T, N), dtype=torch.float32, device="cuda")

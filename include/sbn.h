@@ -33,6 +33,21 @@
  *     vals[n][2g]   = W_q[n][4g+i0],  vals[n][2g+1] = W_q[n][4g+i1]          int8  [N][K/2]
  *     nibble(g)     = i0 | (i1 << 2)
  *     meta[n][b]    = nibble(2b) | (nibble(2b+1) << 4)                       uint8 [N][K/8]
+ *
+ * Storage order of the GEMM operands ("tiled"): vals, meta, dense_q and xq are NOT stored as the
+ * plain row-major arrays above but tile by tile, each tile being the exact shared-memory image
+ * the tensor-core instruction consumes, so that a tile is one contiguous block of HBM.  Every
+ * buffer has the same number of bytes as its row-major form (xq: tokens padded to a multiple of
+ * 16) and is a pure permutation of it.  With KB = K/128, r = n % 128 (or t % 8 for xq), all
+ * offsets in bytes:
+ *     vals    element (n, c), c in [0, K/2):   ((n/128)*KB + c/64)*8192 + r*64
+ *                                              + ((((c%64)/16) ^ ((r/2)%4)) * 16) + c%16
+ *     meta    element (n, b), b in [0, K/8):   ((n/128)*KB + b/16)*2048 + r*16 + b%16
+ *     dense_q element (n, k), k in [0, K):     ((n/128)*KB + k/128)*16384 + (r/8)*1024 + (r%8)*128
+ *                                              + ((((k%128)/16) ^ (r%8)) * 16) + k%16
+ *     xq      element (t, k):                  ((k/128)*TB8 + t/8)*1024 + (t%8)*128
+ *                                              + ((((k%128)/16) ^ (t%8)) * 16) + k%16,
+ *             TB8 = 2*ceil(T/16); buffer size sbn_xq_bytes(T, K) = TB8 * KB * 1024
  */
 #ifndef SBN_H_
 #define SBN_H_
@@ -65,6 +80,9 @@ typedef enum {
     SBN_OP_BITLINEAR = 3
 } sbn_op;
 
+/* Host, pure.  Bytes of the tiled int8 activation buffer xq for T tokens of K columns. */
+size_t sbn_xq_bytes(int T, int K);
+
 /* Host, pure.  Bytes of device workspace the given call needs for these sizes (0 if none).
  * T is ignored by SBN_OP_QUANTIZE_MASK_PACK. */
 size_t sbn_workspace_bytes(int op, int T, int N, int K);
@@ -79,11 +97,12 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K);
  * Arguments
  *   W          device, fp32 [N][K], read only
  *   n_keep, m_group  the N:M pattern; only 2:4 is implemented (else SBN_ERR_UNSUPPORTED)
- *   vals       device out, int8 [N][K/2]
- *   meta       device out, uint8 [N][K/8]; may be the same buffer as prev_meta
+ *   vals       device out, int8, N*K/2 bytes, tiled order
+ *   meta       device out, uint8, N*K/8 bytes, tiled order; may be the same buffer as prev_meta
  *   w_scale    device out, one fp32: `scale`
- *   dense_q    device out or NULL, int8 [N][K]: the unmasked W_q (operand of sbn_bitlinear)
- *   prev_meta  device or NULL, uint8 [N][K/8]: metadata of the previous step's mask
+ *   dense_q    device out or NULL, int8, N*K bytes, tiled order: the unmasked W_q (operand of
+ *              sbn_bitlinear)
+ *   prev_meta  device or NULL, uint8, N*K/8 bytes, tiled order: metadata of the previous step's mask
  *   flip_bits  device out or NULL (required iff prev_meta != NULL), one uint64: number of
  *              positions whose mask bit differs from prev_meta's, i.e. the numerator of the flip
  *              rate r_t = ||m(w_t) - m(w_{t-1})||_1 / D (Sec. 4); overwritten, not accumulated
@@ -136,9 +155,8 @@ sbn_status sbn_quantize_mask_pack_static_ws(const float *W, int N, int K, int n_
  *   a = max_k |x[t][k]|, d = max(a, 1e-5), s_x = 127 / d,
  *   xq[t][k] = clamp(round_half_even(x[t][k] * s_x), -128, 127),  a_scale[t] = d / 127.
  *   x_bf16   device, bf16 [T][K]
- *   xq       device out, int8 [T][K]
+ *   xq       device out, int8, sbn_xq_bytes(T, K) bytes, tiled order (see above)
  *   a_scale  device out, fp32 [T]
- * Here K only needs K % 8 == 0.
  */
 sbn_status sbn_quant_act(const void *x_bf16, int T, int K, int8_t *xq, float *a_scale,
                          void *stream);
@@ -174,7 +192,7 @@ sbn_status sbn_bitlinear(const int8_t *xq, const float *a_scale, int T,
  * weights): copies x (bf16 [T][K], host, ideally pinned) to `x_dev`, runs sbn_quant_act and
  * sbn_sparse_bitlinear (or sbn_bitlinear when vals == NULL and dense_q != NULL), and copies
  * y ([T][N] of `dt`) back to `y_host`.  All on `stream`; returns after enqueueing.
- *   x_dev   device staging, T*K*2 bytes;  xq_dev  device, T*K bytes;  a_scale_dev device, T*4
+ *   x_dev   device staging, T*K*2 bytes;  xq_dev  device, sbn_xq_bytes(T, K);  a_scale_dev device, T*4
  *   y_dev   device staging for y
  * Weights (vals/meta or dense_q, w_scale, bias) are device pointers as above.
  */
@@ -195,7 +213,7 @@ const char *sbn_status_string(sbn_status s);
 
 /* Tuning/diagnostic knob (host state, not thread-safe).  token_tile: 0 = automatic; 64, 128 or
  * 256 = force the single-CTA kernel with that token-tile width; a negative value -BN = force the
- * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
+ * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 32, capped at 224 sparse /
  * 256 dense).  split_k: split-K factor of the single-CTA kernel (0 = automatic).  Results do not
  * depend on it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);

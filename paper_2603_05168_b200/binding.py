@@ -21,7 +21,7 @@ OUT_F32, OUT_BF16 = 0, 1
 OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
 
 EXPORTS = [
-    "sbn_workspace_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quant_act", "sbn_sparse_bitlinear",
+    "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quant_act", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -45,6 +45,8 @@ def lib() -> ctypes.CDLL:
                 "(there is no fallback path)")
         L = ctypes.CDLL(LIB_PATH)
         vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.sbn_xq_bytes.restype = sz
+        L.sbn_xq_bytes.argtypes = [i32, i32]
         L.sbn_workspace_bytes.restype = sz
         L.sbn_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sbn_quantize_mask_pack.restype = i32
@@ -92,6 +94,10 @@ def sbn_workspace_bytes(op: int, T: int, N: int, K: int) -> int:
     return int(lib().sbn_workspace_bytes(op, T, N, K))
 
 
+def sbn_xq_bytes(T: int, K: int) -> int:
+    return int(lib().sbn_xq_bytes(T, K))
+
+
 def sbn_quantize_mask_pack(W, vals, meta, w_scale, ws, dense_q=None, prev_meta=None, flip_bits=None,
                            n_keep: int = 2, m_group: int = 4):
     N, K = W.shape
@@ -124,8 +130,8 @@ def _ws_args(ws):
 
 
 def sbn_sparse_bitlinear(xq, a_scale, vals, meta, w_scale, y, bias=None, acc_out=None, ws=None):
-    T, K = xq.shape
-    N = vals.shape[0]
+    T, N = y.shape
+    K = 2 * vals.numel() // N
     dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
     wp, wb = _ws_args(ws)
     _check(lib().sbn_sparse_bitlinear(_ptr(xq), _ptr(a_scale), T, _ptr(vals), _ptr(meta), _ptr(w_scale),
@@ -134,8 +140,8 @@ def sbn_sparse_bitlinear(xq, a_scale, vals, meta, w_scale, y, bias=None, acc_out
 
 
 def sbn_bitlinear(xq, a_scale, dense_q, w_scale, y, bias=None, acc_out=None, ws=None):
-    T, K = xq.shape
-    N = dense_q.shape[0]
+    T, N = y.shape
+    K = dense_q.numel() // N
     dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
     wp, wb = _ws_args(ws)
     _check(lib().sbn_bitlinear(_ptr(xq), _ptr(a_scale), T, _ptr(dense_q), _ptr(w_scale), N, K,
@@ -180,6 +186,11 @@ def alloc_packed(N: int, K: int, device="cuda", with_dense: bool = False):
     if with_dense:
         out["dense_q"] = torch.empty((N, K), dtype=torch.int8, device=device)
     return out
+
+
+def alloc_xq(T: int, K: int, device="cuda"):
+    """Device buffer for the tiled int8 activations of T tokens x K columns."""
+    return torch.empty(sbn_xq_bytes(T, K), dtype=torch.int8, device=device)
 
 
 def alloc_gemm_ws(op: int, T: int, N: int, K: int, device="cuda"):

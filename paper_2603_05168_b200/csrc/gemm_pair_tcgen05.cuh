@@ -1,19 +1,24 @@
 // Eq. 4 on CTA pairs: the large-T kernel.
 //
-// Why pairs: an SM can take in about 64 B per clock from L2.  At the sparse int8 rate a CTA that
-// owns a 128 x 256 output tile needs ~160 B/clk of operands, so single-CTA tiles are held at a
-// third of the tensor peak by operand ingest, not by the MMA.  Here two CTAs of a cluster issue
-// one `cta_group::2` MMA (M = 256: each CTA supplies 128 weight rows and HALF of the activation
-// tile, and keeps its 128 x BN accumulator slice in its own TMEM), and every CTA runs TWO such
-// M-tiles against the same activation stage.  Per CTA and per unit of K that is
-// 2*(64+8) + BN/2 bytes (sparse) for 256 x BN MACs: ~68 B/clk at the sparse peak for BN = 240.
+// Measured facts that shape it (B200, this kernel family, one CTA pair alone on the GPU):
+//   * the time a pipeline stage costs in the TMA unit is  ~64 ns x (number of TMA instructions)
+//     + ~2.8 ns per KB, whatever the box shape -- so a stage must be fetched with as few
+//     instructions as possible;
+//   * an SM sustains roughly 100-120 GB/s of operand ingest, so the tile must reuse operands.
+// Hence: two CTAs of a cluster issue one `cta_group::2` MMA (M = 256: each CTA supplies 128
+// weight rows and HALF of the activation tile, and keeps its 128 x BN accumulator slice in its
+// own TMEM); every CTA runs TWO such M-tiles against the same activation stage; operands are
+// stored in HBM as shared-memory images (layouts.cuh) and one 3-D tensor-map box fetches, per
+// stage, both of a CTA's weight tiles (and likewise both metadata tiles, and the activation
+// atoms) for KBS consecutive 128-column blocks: three instructions per stage (sparse).
 //
-//   pair tile      512 output features x BN tokens (BN runtime, multiple of 16, <= 240 sparse /
-//                  256 dense); the last feature tile may hold only one M-tile
-//   per CTA smem   per stage: 2 x A (128 rows x 64 B sparse | 128 B dense), 2 x E (128 x 16 B),
-//                  B (BN/2 rows x 128 B); ring of STAGES stages
+//   pair tile      512 output features x BN tokens (BN runtime, multiple of 32, <= 224 sparse /
+//                  256 dense).  CTA r of the pair owns the weight row blocks 4*mt + 2r + i
+//                  (i = 0, 1 = the M-tile); a row block beyond N is skipped.
+//   per CTA smem   per stage: A[2 row blocks][KBS] (8 KB sparse | 16 KB dense each),
+//                  E[2][KBS] (2 KB each, sparse), B[KBS] (BN/2 rows x 128 B); KBS = 2 (sparse), 1
 //   TMEM           M-tile i accumulates in columns [256 i, 256 i + BN); metadata slots in columns
-//                  [256 i + 240, 256 i + 256).  Accumulators are single-buffered: the MMA of the
+//                  [256 i + 224, 256 i + 256).  Accumulators are single-buffered: the MMA of the
 //                  next tile waits until the epilogue has drained TMEM into registers.
 //   warps          0 TMA producer (both CTAs), 1 MMA issuer (leader CTA only; both allocate
 //                  TMEM), 2..9 epilogue: warps 2-5 drain M-tile 0, warps 6-9 M-tile 1
@@ -32,26 +37,34 @@ namespace sbn {
 
 constexpr int kPairThreads = 320;
 constexpr int kPairEpiWarps = 8;
-constexpr int kPairSlabBytes = 16 * 32 * 4;                       // 16 tokens x 32 features fp32
-constexpr int kPairEpiBytes = kPairEpiWarps * 2 * kPairSlabBytes; // double buffered per warp
-constexpr int kPairMaxBnSparse = 240;
+constexpr int kPairSlabBytes = 2048;                              // 32 tok x 32 feat bf16 | 16 tok fp32
+constexpr int kPairEpiBytes = kPairEpiWarps * kPairSlabBytes;     // one slab per epilogue warp
+constexpr int kPairMaxBnSparse = 224;
 constexpr int kPairMaxBnDense = 256;
 
 template <bool SPARSE>
 struct PairConfig {
-    static constexpr int A_TILE = SPARSE ? kBM * (kBK / 2) : kBM * kBK;     // one M-tile half
+    static constexpr int KBS = SPARSE ? 2 : 1;                               // 128-column blocks per stage
+    static constexpr int A_TILE = SPARSE ? kBM * (kBK / 2) : kBM * kBK;     // one row block x one k-block
     static constexpr int E_TILE = SPARSE ? kBM * (kBK / 8) : 0;
-    static constexpr int B_TILE = 128 * kBK;                                 // up to 128 token rows
-    static constexpr int STAGE_BYTES = 2 * A_TILE + 2 * E_TILE + B_TILE;
+    static constexpr int B_ROWS_MAX = SPARSE ? kPairMaxBnSparse / 2 : kPairMaxBnDense / 2;
+    static constexpr int B_TILE = B_ROWS_MAX * kBK;                          // one k-block of activations
+    static constexpr int A_BYTES = 2 * KBS * A_TILE;
+    static constexpr int E_BYTES = 2 * KBS * E_TILE;
+    static constexpr int B_BYTES = KBS * B_TILE;
+    static constexpr int STAGE_BYTES = A_BYTES + E_BYTES + B_BYTES;
     static constexpr int STAGES = (232448 - 1024 - kPairEpiBytes - kBarrierBytes) / STAGE_BYTES;
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + kPairEpiBytes + kBarrierBytes;
+    static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1 KB alignment");
     static_assert(STAGES >= 3, "not enough stages");
+    static_assert(!SPARSE || KBS == 2, "the 128x256b metadata copy covers exactly two k-blocks");
     static_assert(SMEM_BYTES <= 232448, "shared memory overflow");
 };
 
 struct PairParams {
     GemmParams g;
     int bn;                       // tokens per tile
+    int debug;                    // perf experiments only (wrong results): 4/8 = limit the grid, 16 = no MMA
 };
 
 // ---- cluster / pair PTX ------------------------------------------------------------------------
@@ -73,13 +86,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t ran
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// TMA tile load whose completion is counted on a barrier that may live in the peer CTA.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+// TMA 3-D box load whose completion is counted on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
                                                  uint32_t bar_cluster_addr) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr)
         : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols) {
@@ -97,6 +110,10 @@ __device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar) {
 }
 __device__ __forceinline__ void tcgen05_cp_128x128b_pair(uint32_t taddr, uint64_t sdesc) {
     asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// 128 lanes x 32 B: two 16 B-wide source blocks (LBO apart) land in 8 consecutive TMEM columns.
+__device__ __forceinline__ void tcgen05_cp_128x256b_pair(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.128x256b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 __device__ __forceinline__ void mma_i8_dense_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
                                                   uint32_t idesc, uint32_t accumulate) {
@@ -124,6 +141,11 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Tensor maps (all over arrays of 1 KB rows of 128 x uint64, see layouts.cuh):
+//   tmap_a  [N/128][KB * rows_per_tile][1 KB]   box {1 KB, rows_per_tile * KBS, 2}
+//   tmap_e  [N/128][KB * 2][1 KB]               box {1 KB, 2 * KBS, 2}          (sparse)
+//   tmap_b  [KB][TB8][1 KB]                     box {1 KB, BN/16, KBS}
+//   tmap_y  y [T][N]                            box {32 features, 32 (bf16) | 16 (fp32) tokens}
 template <bool SPARSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -133,13 +155,15 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                            const PairParams pp) {
     using Cfg = PairConfig<SPARSE>;
     constexpr int STAGES = Cfg::STAGES;
+    constexpr int KBS = Cfg::KBS;
+    constexpr int A_ROWS = Cfg::A_TILE / 1024;            // 1 KB rows per weight tile
     const GemmParams& p = pp.g;
     const int BN = pp.bn;
     const int half_bn = BN >> 1;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // per stage: [A0][A1][E0][E1][B]
+    // per stage: A [row block i][k-block j] | E [i][j] | B [j]
     const uint32_t smem_stage0 = smem_base;
     const uint32_t smem_epi = smem_base + STAGES * Cfg::STAGE_BYTES;
     const uint32_t bar_base = smem_epi + kPairEpiBytes;
@@ -158,10 +182,12 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int pair_id = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
 
+    const int n_blocks = p.N >> 7;
     const int tiles_m = (p.N + 511) / 512;
     const int tiles_t = (p.T + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_t;
     const int k_blocks = p.k_blocks_total;
+    const int k_stages = (k_blocks + KBS - 1) / KBS;      // pipeline stages per tile
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -190,31 +216,26 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tma_prefetch_desc(&tmap_a);
             tma_prefetch_desc(&tmap_b);
             if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);
+            const uint32_t bytes_per_cta = static_cast<uint32_t>(Cfg::A_BYTES + Cfg::E_BYTES + KBS * half_bn * kBK);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int mt = tile % tiles_m;
                 const int tt = tile / tiles_m;
-                const int m0 = mt * 512;
-                const int mt_count = (m0 + 256 < p.N) ? 2 : 1;
-                const int t_row = tt * BN + static_cast<int>(rank) * half_bn;    // this CTA's token half
-                const uint32_t bytes_per_cta = static_cast<uint32_t>(mt_count * (Cfg::A_TILE + Cfg::E_TILE) + half_bn * kBK);
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                const int nb0 = mt * 4 + static_cast<int>(rank) * 2;            // this CTA's two row blocks
+                const int t_atom = (tt * BN + static_cast<int>(rank) * half_bn) >> 3;   // this CTA's token half
+                for (int ks = 0; ks < k_stages; ++ks) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full_leader = map_to_cta(bar_full + 8 * stage, 0);
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * bytes_per_cta);
                     const uint32_t st = smem_stage0 + stage * Cfg::STAGE_BYTES;
-                    for (int i = 0; i < mt_count; ++i) {
-                        const int row = m0 + i * 256 + static_cast<int>(rank) * 128;
-                        if constexpr (SPARSE) {
-                            tma_load_2d_pair(st + i * Cfg::A_TILE, &tmap_a, kb * (kBK / 2), row, full_leader);
-                            tma_load_2d_pair(st + 2 * Cfg::A_TILE + i * Cfg::E_TILE, &tmap_e, kb * (kBK / 8), row, full_leader);
-                        } else {
-                            tma_load_2d_pair(st + i * Cfg::A_TILE, &tmap_a, kb * kBK, row, full_leader);
-                        }
-                    }
-                    tma_load_2d_pair(st + 2 * Cfg::A_TILE + 2 * Cfg::E_TILE, &tmap_b, kb * kBK, t_row, full_leader);
+                    const int kb = ks * KBS;
+                    // boxes that reach beyond the arrays (odd K/128, N % 512 != 0, last tokens) are
+                    // zero-filled by the hardware and still count their full size
+                    tma_load_3d_pair(st, &tmap_a, 0, kb * A_ROWS, nb0, full_leader);
+                    if constexpr (SPARSE) tma_load_3d_pair(st + Cfg::A_BYTES, &tmap_e, 0, kb * 2, nb0, full_leader);
+                    tma_load_3d_pair(st + Cfg::A_BYTES + Cfg::E_BYTES, &tmap_b, 0, t_atom, kb, full_leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -223,44 +244,63 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         // ------------------------------------------------------------------ MMA issuer (leader)
         if (rank == 0 && lane == 0) {
             const uint32_t idesc = make_idesc_i8(256, BN, SPARSE);
+            const uint32_t b_kb_bytes = static_cast<uint32_t>(half_bn * kBK);    // B bytes of one k-block
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_phase = 0;
+            uint32_t e_slot = 0;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int mt = tile % tiles_m;
-                const int m0 = mt * 512;
-                const int mt_count = (m0 + 256 < p.N) ? 2 : 1;
+                // M-tile i is live if at least the leader's row block 4*mt + i exists
+                const int mt_count = (mt * 4 + 1 < n_blocks) ? 2 : 1;
                 // single-buffered accumulators: wait until the epilogues of both CTAs drained them
                 if (!mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tcgen05_fence_after();
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                for (int ks = 0; ks < k_stages; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_stage0 + stage * Cfg::STAGE_BYTES;
-                    const uint32_t b_addr = st + 2 * Cfg::A_TILE + 2 * Cfg::E_TILE;
-                    const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
-                    for (int i = 0; i < mt_count; ++i) {
-                        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(i * 256);
-                        const uint32_t a_addr = st + i * Cfg::A_TILE;
+                    const int kb_live = min(KBS, k_blocks - ks * KBS);
+                    if (!(pp.debug & 16)) {
+                        uint32_t e_tmem[2] = {0u, 0u};
                         if constexpr (SPARSE) {
-                            const uint32_t e_tmem = tmem_base + static_cast<uint32_t>(i * 256 + 240 + 4 * (kb & 3));
-                            const uint64_t e_desc = make_smem_desc(st + 2 * Cfg::A_TILE + i * Cfg::E_TILE, 128, 128, kSwzNone);
-                            tcgen05_cp_128x128b_pair(e_tmem, e_desc);
-                            const uint64_t a_desc = make_smem_desc(a_addr, 16, 512, kSwz64);
-#pragma unroll
-                            for (int j = 0; j < kBK / 64; ++j) {
-                                mma_i8_sparse_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * j),
-                                                   b_desc + static_cast<uint64_t>(4 * j), e_tmem + 2 * j, idesc,
-                                                   (kb | j) != 0 ? 1u : 0u);
+                            // every tcgen05 instruction occupies the tensor pipe for ~128 clocks, copies
+                            // included: one 128x256b copy brings the metadata of BOTH k-blocks of the
+                            // stage (two 2 KB tiles, 2 KB apart) for an M-tile
+                            for (int i = 0; i < mt_count; ++i) {
+                                e_tmem[i] = tmem_base + static_cast<uint32_t>(i * 256 + 224 + 8 * (e_slot & 3u));
+                                const uint64_t e_desc = make_smem_desc(st + Cfg::A_BYTES + static_cast<uint32_t>(i * KBS * Cfg::E_TILE),
+                                                                       Cfg::E_TILE, 128, kSwzNone);
+                                tcgen05_cp_128x256b_pair(e_tmem[i], e_desc);
                             }
-                        } else {
-                            const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024, kSwz128);
+                            ++e_slot;
+                        }
+                        for (int j = 0; j < kb_live; ++j) {
+                            const uint32_t b_addr = st + Cfg::A_BYTES + Cfg::E_BYTES + static_cast<uint32_t>(j) * b_kb_bytes;
+                            const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
+                            const uint32_t first = (ks | j) == 0 ? 0u : 1u;
+                            for (int i = 0; i < mt_count; ++i) {
+                                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(i * 256);
+                                const uint32_t a_addr = st + static_cast<uint32_t>((i * KBS + j) * Cfg::A_TILE);
+                                if constexpr (SPARSE) {
+                                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 512, kSwz64);
 #pragma unroll
-                            for (int j = 0; j < kBK / 32; ++j) {
-                                mma_i8_dense_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * j),
-                                                  b_desc + static_cast<uint64_t>(2 * j), idesc,
-                                                  (kb | j) != 0 ? 1u : 0u);
+                                    for (int q = 0; q < kBK / 64; ++q) {
+                                        mma_i8_sparse_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * q),
+                                                           b_desc + static_cast<uint64_t>(4 * q),
+                                                           e_tmem[i] + static_cast<uint32_t>(4 * j + 2 * q), idesc,
+                                                           q == 0 ? first : 1u);
+                                    }
+                                } else {
+                                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024, kSwz128);
+#pragma unroll
+                                    for (int q = 0; q < kBK / 32; ++q) {
+                                        mma_i8_dense_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * q),
+                                                          b_desc + static_cast<uint64_t>(2 * q), idesc,
+                                                          q == 0 ? first : 1u);
+                                    }
+                                }
                             }
                         }
                     }
@@ -274,84 +314,128 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     } else {
         // ------------------------------------------------------------------ epilogue (8 warps)
+        // The accumulators are single-buffered, so the time from "accumulator complete" to "all
+        // warps have pulled their columns into registers" is exposed.  To keep it short: the
+        // per-token scales are fetched into registers BEFORE waiting for the accumulator, TMEM
+        // loads run one 32-column chunk ahead of the arithmetic, values are converted in
+        // registers while the previous chunk's TMA store is still reading the slab, and a chunk
+        // costs one fence + one TMA store (bf16) or two (fp32).  Every warp works on its own
+        // (private slab, private stores): sharing one slab per M-tile between four warps was
+        // measured slower because of the hand-over between warps.
         const int ew = warp - 2;                          // 0..7
         const int mtile = ew >> 2;                        // which M-tile this warp drains
         const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const float w_scale = __ldg(p.w_scale);
-        const uint32_t slab_u32 = smem_epi + static_cast<uint32_t>(ew * 2 * kPairSlabBytes);
+        const uint32_t slab_u32 = smem_epi + static_cast<uint32_t>(ew * kPairSlabBytes);
         uint8_t* const slab_ptr = smem_raw + (slab_u32 - smem_u32(smem_raw));
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
+        const int chunks = BN >> 5;                       // 32-column chunks (BN % 32 == 0)
         uint32_t acc_phase = 0;
-        int buf = 0;
         bool ok = true;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
             const int mt = tile % tiles_m;
             const int tt = tile / tiles_m;
-            const int m0 = mt * 512;
-            const int n0 = m0 + mtile * 256 + static_cast<int>(rank) * 128 + quarter * 32;
+            const int n0 = (mt * 4 + static_cast<int>(rank) * 2 + mtile) * 128 + quarter * 32;
             const int n = n0 + lane;
             const int t0 = tt * BN;
             const bool rows_valid = n0 < p.N;             // warp-uniform (N % 128 == 0)
             const float bias = (p.bias && rows_valid) ? __ldg(p.bias + n) : 0.0f;
+            // s absorbs both scales (Eq. 4): lane l keeps w_scale * a_scale of tokens t0 + 32 i + l
+            float my_scale[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int t = t0 + i * 32 + lane;
+                my_scale[i] = (i < chunks && t < p.T) ? __fmul_rn(w_scale, __ldg(p.a_scale + t)) : 0.0f;
+            }
             if (!mbar_wait(bar_acc_full, acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
-            const int chunks = BN >> 4;
-#pragma unroll 1
-            for (int c = 0; c < chunks; ++c) {
-                const int tc = t0 + c * 16;
-                const bool active = rows_valid && tc < p.T;
-                uint32_t r[16];
-                float my_scale = 0.0f;
-                if (active) {
-                    const int t = tc + (lane & 15);
-                    if (t < p.T) my_scale = __fmul_rn(w_scale, __ldg(p.a_scale + t));
-                    tmem_ld_32x32b_x16(tmem_base + lane_base + static_cast<uint32_t>(mtile * 256 + c * 16), r);
-                    tmem_ld_wait();
-                }
-                if (c == chunks - 1) {
-                    // this warp has read everything it needs from the accumulators
-                    tcgen05_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
-                }
-                if (!active) continue;
-                if (p.acc_out) {
+            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(mtile * 256);
+            // number of chunks that hold at least one real token (warp-uniform)
+            const int live = rows_valid ? (min(p.T - t0, BN) + 31) >> 5 : 0;
+            uint32_t ra[32], rb[32];
+            if (live > 0) tmem_ld_32x32b_x32(t_addr, ra);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int t = tc + j;
-                        if (t < p.T) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(r[j]);
+            for (int i = 0; i < 8; ++i) {
+                if (i < live) {
+                    uint32_t (&cur)[32] = (i & 1) ? rb : ra;
+                    uint32_t (&nxt)[32] = (i & 1) ? ra : rb;
+                    tmem_ld_wait();                                       // chunk i is in registers
+                    if (i + 1 < live) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>((i + 1) * 32), nxt);
+                    if (i + 1 == live) {
+                        // last TMEM read of this warp is complete: hand the accumulator back
+                        tcgen05_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+                    }
+                    const int tc = t0 + i * 32;
+                    if (p.acc_out) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int t = tc + j;
+                            if (t < p.T) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(cur[j]);
+                        }
+                    }
+                    if (p.out_bf16) {
+                        // convert in registers (two tokens per word), then one 32 x 32 bf16 slab
+                        uint32_t packed[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const float s0 = __shfl_sync(0xFFFFFFFFu, my_scale[i], j);
+                            const float s1 = __shfl_sync(0xFFFFFFFFu, my_scale[i], j + 1);
+                            float v0 = __fmul_rn(static_cast<float>(static_cast<int>(cur[j])), s0);
+                            float v1 = __fmul_rn(static_cast<float>(static_cast<int>(cur[j + 1])), s1);
+                            if (p.bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); }
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed[j >> 1]) : "f"(v1), "f"(v0));
+                        }
+                        // the slab's previous contents must have been read by their TMA store
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                        uint16_t* o = reinterpret_cast<uint16_t*>(slab_ptr) + lane;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            o[(2 * j) * 32] = static_cast<uint16_t>(packed[j] & 0xFFFFu);
+                            o[(2 * j + 1) * 32] = static_cast<uint16_t>(packed[j] >> 16);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(&tmap_y, n0, tc, slab_u32);
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        }
+                    } else {
+                        // two 16-token x 32-feature fp32 slabs through the same 2 KB buffer
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (tc + h * 16 < p.T) {
+                                float v[16];
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    const float sc = __shfl_sync(0xFFFFFFFFu, my_scale[i], h * 16 + j);
+                                    v[j] = __fmul_rn(static_cast<float>(static_cast<int>(cur[h * 16 + j])), sc);
+                                    if (p.bias) v[j] = __fadd_rn(v[j], bias);
+                                }
+                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                                __syncwarp();
+                                float* o = reinterpret_cast<float*>(slab_ptr) + lane;
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) o[j * 32] = v[j];
+                                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                                __syncwarp();
+                                if (lane == 0) {
+                                    tma_store_2d(&tmap_y, n0, tc + h * 16, slab_u32);
+                                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                                }
+                            }
+                        }
                     }
                 }
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            }
+            if (live == 0) {
+                // nothing to read (rows or tokens beyond the matrix): still release the accumulator
+                tcgen05_fence_before();
                 __syncwarp();
-                uint8_t* const slab = slab_ptr + buf * kPairSlabBytes;
-                if (p.out_bf16) {
-                    uint16_t* o = reinterpret_cast<uint16_t*>(slab) + lane;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float sc = __shfl_sync(0xFFFFFFFFu, my_scale, j);
-                        float v = __fmul_rn(static_cast<float>(static_cast<int>(r[j])), sc);
-                        if (p.bias) v = __fadd_rn(v, bias);
-                        o[j * 32] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-                    }
-                } else {
-                    float* o = reinterpret_cast<float*>(slab) + lane;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float sc = __shfl_sync(0xFFFFFFFFu, my_scale, j);
-                        float v = __fmul_rn(static_cast<float>(static_cast<int>(r[j])), sc);
-                        if (p.bias) v = __fadd_rn(v, bias);
-                        o[j * 32] = v;
-                    }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_2d(&tmap_y, n0, tc, slab_u32 + static_cast<uint32_t>(buf * kPairSlabBytes));
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
-                buf ^= 1;
+                if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
             }
             acc_phase ^= 1u;
         }

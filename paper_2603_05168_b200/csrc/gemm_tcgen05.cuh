@@ -16,9 +16,10 @@
 // CTA = 6 warps: warp 0 TMA producer, warp 1 MMA issuer (also owns the TMEM allocation),
 // warps 2-5 epilogue (one TMEM lane quarter each).  Persistent over output tiles
 // (128 features x BN tokens), static round-robin tile order, K-blocks of 128 logical columns:
-//   A stage   128 rows x 64 B (sparse, SWIZZLE_64B)  or 128 rows x 128 B (dense, SWIZZLE_128B)
-//   B stage   BN rows x 128 B (SWIZZLE_128B)
-//   E stage   128 rows x 16 B metadata (sparse only), plain row-major = the canonical layout
+//   A stage   128 rows x 64 B (sparse, SWIZZLE_64B image) or 128 rows x 128 B (dense, SWIZZLE_128B)
+//   B stage   BN rows x 128 B (SWIZZLE_128B image)
+//   E stage   128 rows x 16 B metadata (sparse only)
+// All three are stored in HBM as these very images (layouts.cuh) and fetched as 1 KB rows.
 // TMEM: ACC_STAGES accumulators of BN columns, then one 4-column metadata slot per smem stage.
 //
 // Every wait is bounded (wall-clock limit); a wait that runs out records SBN_ERR_TIMEOUT in the
@@ -28,6 +29,7 @@
 #include <cuda.h>
 
 #include "sbn_common.cuh"
+#include "layouts.cuh"
 
 namespace sbn {
 
@@ -46,6 +48,7 @@ struct GemmParams {
     int T, N, K;
     int k_blocks_total;          // K / 128
     int k_splits;                // split-K factor (1 = none)
+    int tb8;                     // 8-token atoms per 128-column block of the tiled xq (2*ceil(T/16))
     const float* a_scale;        // [T]
     const float* w_scale;        // [1]
     const float* bias;           // [N] or null
@@ -282,19 +285,21 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 const int split = tile % p.k_splits;
                 const int mt = (tile / p.k_splits) % tiles_m;
                 const int tt = (tile / p.k_splits) / tiles_m;
-                const int m0 = mt * kBM, t0 = tt * BN;
+                const int t0 = tt * BN;
                 const int kb0 = split * kb_per_split;
                 for (int kb = kb0; kb < kb0 + kb_per_split; ++kb) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full = bar_full + 8 * stage;
                     mbar_expect_tx(full, Cfg::TX_BYTES);
+                    // operand tiles are stored as smem images (layouts.cuh): 1 KB rows, a few per tile
+                    const int wt = mt * p.k_blocks_total + kb;            // weight tile index
                     if constexpr (SPARSE) {
-                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, kb * (kBK / 2), m0, full);
-                        tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, kb * (kBK / 8), m0, full);
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 8, full);
+                        tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, 0, wt * 2, full);
                     } else {
-                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, kb * kBK, m0, full);
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 16, full);
                     }
-                    tma_load_2d(smem_b + stage * Cfg::B_BYTES, &tmap_b, kb * kBK, t0, full);
+                    tma_load_2d(smem_b + stage * Cfg::B_BYTES, &tmap_b, 0, kb * p.tb8 + (t0 >> 3), full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }

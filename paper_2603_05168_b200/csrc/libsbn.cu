@@ -41,15 +41,29 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// 3-D view [d2][d1][1 KB] of tiled operand data (1 KB rows of 128 x uint64); box {1 KB, b1, b2}.
+static bool encode_3d_1k(CUtensorMap* map, const void* base, uint64_t d1, uint64_t d2, uint32_t b1, uint32_t b2) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || b1 == 0 || b1 > 256 || b2 == 0 || b2 > 256) return false;
+    cuuint64_t dims[3] = {128, d1, d2};
+    cuuint64_t strides[2] = {1024, 1024 * d1};
+    cuuint32_t box[3] = {128, b1, b2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 3, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // 2-D row-major output tensor y [T][N] (fp32 or bf16) with a 32-feature x box_tokens box.
 static bool encode_2d_out(CUtensorMap* map, const void* base, uint64_t N, uint64_t T, bool bf16,
-                          uint32_t box_tokens) {
+                          uint32_t box_tokens, uint32_t box_features = 32) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const uint64_t es = bf16 ? 2 : 4;
     cuuint64_t dims[2] = {N, T};
     cuuint64_t strides[1] = {N * es};
-    cuuint32_t box[2] = {32, box_tokens};
+    cuuint32_t box[2] = {box_features, box_tokens};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -58,18 +72,17 @@ static bool encode_2d_out(CUtensorMap* map, const void* base, uint64_t N, uint64
     return r == CUDA_SUCCESS;
 }
 
-// 2-D uint8 row-major tensor [rows][cols_bytes] with a [box_rows][box_cols] box.
-static bool encode_2d_u8(CUtensorMap* map, const void* base, uint64_t cols_bytes, uint64_t rows,
-                         uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle swz) {
+// Flat array of tiled operand data viewed as rows of 1 KB (128 x uint64); box = box_rows rows.
+static bool encode_flat_1k(CUtensorMap* map, const void* base, uint64_t total_bytes, uint32_t box_rows) {
     EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {cols_bytes, rows};
-    cuuint64_t strides[1] = {cols_bytes};
-    cuuint32_t box[2] = {box_cols, box_rows};
+    if (!fn || total_bytes % 1024 != 0) return false;
+    cuuint64_t dims[2] = {128, total_bytes / 1024};
+    cuuint64_t strides[1] = {1024};
+    cuuint32_t box[2] = {128, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box,
-                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -133,8 +146,8 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
     if (g_force_token_tile < 0) {
         int bn = -g_force_token_tile;
         const int cap = sparse ? kPairMaxBnSparse : kPairMaxBnDense;
-        bn = (bn / 16) * 16;
-        if (bn < 16) bn = 16;
+        bn = (bn / 32) * 32;
+        if (bn < 32) bn = 32;
         if (bn > cap) bn = cap;
         return bn;
     }
@@ -144,7 +157,7 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
     const int full_m = N / 512, rem_m = (N % 512) ? 1 : 0;
     int best = 128;
     double best_cost = 1e300;
-    for (int bn = 64; bn <= cap; bn += 16) {
+    for (int bn = 64; bn <= cap; bn += 32) {
         const int tt = (T + bn - 1) / bn;
         auto tile_clk = [&](int mtiles) {
             const double a_bytes = sparse ? 72.0 : 128.0;
@@ -177,7 +190,9 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
         configured = true;
     }
     const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
-    const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
+    int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
+    if (pp.debug & 4) pairs = 1;                 // experiment: one CTA pair only (unloaded latency)
+    if (pp.debug & 8) pairs = pairs < 8 ? pairs : 8;
     kernel<<<2 * pairs, kPairThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, pp);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
@@ -196,25 +211,29 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     const int bn = pick_pair_bn(sparse, T, N, K);
     CUtensorMap ta, tb, te, ty;
     bool ok;
+    const uint64_t KBk = static_cast<uint64_t>(K) / kBK, NB = static_cast<uint64_t>(N) / kBM;
     if (sparse) {
-        ok = encode_2d_u8(&ta, wvals, static_cast<uint64_t>(K) / 2, N, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B) &&
-             encode_2d_u8(&te, meta, static_cast<uint64_t>(K) / 8, N, kBK / 8, kBM, CU_TENSOR_MAP_SWIZZLE_NONE);
+        constexpr int kbs = PairConfig<true>::KBS;
+        ok = encode_3d_1k(&ta, wvals, KBk * 8, NB, 8 * kbs, 2) && encode_3d_1k(&te, meta, KBk * 2, NB, 2 * kbs, 2) &&
+             encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
     } else {
-        ok = encode_2d_u8(&ta, wvals, K, N, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+        constexpr int kbs = PairConfig<false>::KBS;
+        ok = encode_3d_1k(&ta, wvals, KBk * 16, NB, 16 * kbs, 2) && encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
         te = ta;
     }
-    ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn / 2, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, 16);
+    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, dt == SBN_OUT_BF16 ? 32 : 16);
     if (!ok) return SBN_ERR_CUDA;
     PairParams pp;
     pp.g.T = T; pp.g.N = N; pp.g.K = K;
     pp.g.k_blocks_total = K / kBK;
     pp.g.k_splits = 1;
+    pp.g.tb8 = static_cast<int>(xq_tb8(T));
     pp.g.a_scale = a_scale; pp.g.w_scale = w_scale; pp.g.bias = bias;
     pp.g.y = y; pp.g.out_bf16 = (dt == SBN_OUT_BF16);
     pp.g.acc_out = acc_out;
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.bn = bn;
+    pp.debug = g_force_split_k < 0 ? -g_force_split_k : 0;   // experiments: split_k < 0 carries debug bits
     return sparse ? launch_pair<true>(ta, tb, te, ty, pp, stream) : launch_pair<false>(ta, tb, te, ty, pp, stream);
 }
 
@@ -244,14 +263,14 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
 
     CUtensorMap ta, tb, te, ty;
     bool ok;
+    const uint64_t NK = static_cast<uint64_t>(N) * K;
     if (sparse) {
-        ok = encode_2d_u8(&ta, wvals, static_cast<uint64_t>(K) / 2, N, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B) &&
-             encode_2d_u8(&te, meta, static_cast<uint64_t>(K) / 8, N, kBK / 8, kBM, CU_TENSOR_MAP_SWIZZLE_NONE);
+        ok = encode_flat_1k(&ta, wvals, NK / 2, 8) && encode_flat_1k(&te, meta, NK / 8, 2);
     } else {
-        ok = encode_2d_u8(&ta, wvals, K, N, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+        ok = encode_flat_1k(&ta, wvals, NK, 16);
         te = ta;
     }
-    ok = ok && encode_2d_u8(&tb, xq, K, T, kBK, bn, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && encode_flat_1k(&tb, xq, xq_tiled_bytes(T, K), bn / 8);
     ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, 32);
     if (!ok) return SBN_ERR_CUDA;
 
@@ -259,6 +278,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     p.T = T; p.N = N; p.K = K;
     p.k_blocks_total = K / kBK;
     p.k_splits = splits;
+    p.tb8 = static_cast<int>(xq_tb8(T));
     p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias;
     p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
     p.acc_out = acc_out;
@@ -320,6 +340,11 @@ using namespace sbn;
 
 extern "C" {
 
+size_t sbn_xq_bytes(int T, int K) {
+    if (T <= 0 || K <= 0 || K % kBK != 0) return 0;
+    return xq_tiled_bytes(T, K);
+}
+
 size_t sbn_workspace_bytes(int op, int T, int N, int K) {
     switch (op) {
         case SBN_OP_QUANTIZE_MASK_PACK: return sizeof(QmpWorkspace);
@@ -378,8 +403,8 @@ sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_
 
 sbn_status sbn_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale, void* stream) {
     if (!x_bf16 || !xq || !a_scale) return SBN_ERR_NULL;
-    if (T <= 0 || K <= 0 || K % 8 != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
-    if (misaligned(x_bf16, 16) || misaligned(xq, 8) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
+    if (T <= 0 || K <= 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
     return launch_quant_act(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
 }
 

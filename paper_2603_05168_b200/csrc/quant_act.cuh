@@ -6,9 +6,12 @@
 // HBM-bound: 2 B read + 1 B written per element.  A group of G threads owns one token row and
 // keeps it in registers between the max and the rounding, so x is read from memory once.
 // Loads are 16 B (8 bf16) per lane, stores 8 B (8 int8) per lane, both fully coalesced.
+// xq is written in the tiled layout of layouts.cuh (8-token x 128 B swizzled atoms), which moves
+// 16 B chunks around inside a 128 B line but keeps every warp store a set of whole lines.
 #pragma once
 
 #include "sbn_common.cuh"
+#include "layouts.cuh"
 
 namespace sbn {
 
@@ -32,6 +35,16 @@ __device__ __forceinline__ uint32_t quant1(float x, float s_x) {
 __device__ __forceinline__ uint32_t quant_pair2(uint32_t a, uint32_t b, float s_x) {
     return quant1(bf16lo_to_f32(a), s_x) | (quant1(bf16hi_to_f32(a), s_x) << 8) |
            (quant1(bf16lo_to_f32(b), s_x) << 16) | (quant1(bf16hi_to_f32(b), s_x) << 24);
+}
+
+// Index (in 8-byte units) of the 8 int8 codes of token `t`, vector `idx` (columns 8*idx .. 8*idx+7).
+__device__ __forceinline__ size_t xq_tiled_u2_index(int t, int idx, size_t tb8) {
+    const uint32_t kb = static_cast<uint32_t>(idx) >> 4;
+    const uint32_t chunk = (static_cast<uint32_t>(idx) & 15u) >> 1;
+    const uint32_t half = static_cast<uint32_t>(idx) & 1u;
+    const uint32_t r = static_cast<uint32_t>(t) & 7u;
+    const size_t atom = static_cast<size_t>(kb) * tb8 + (static_cast<uint32_t>(t) >> 3);
+    return (atom << 7) + (r << 4) + ((chunk ^ r) << 1) + half;
 }
 
 template <int G>
@@ -79,7 +92,7 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
     const float s_x = __fdiv_rn(127.0f, d);
     if (g == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
 
-    uint2* qr = xq + static_cast<size_t>(row) * nvec;
+    const size_t tb8 = xq_tb8(T);
 #pragma unroll
     for (int i = 0; i < kActVecPerThread; ++i) {
         const int idx = g + i * G;
@@ -87,7 +100,7 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
             uint2 o;
             o.x = quant_pair2(v[i].x, v[i].y, s_x);
             o.y = quant_pair2(v[i].z, v[i].w, s_x);
-            qr[idx] = o;
+            xq[xq_tiled_u2_index(row, idx, tb8)] = o;
         }
     }
 }
@@ -112,13 +125,13 @@ quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* _
     const float d = fmaxf(m, kEps);
     const float s_x = __fdiv_rn(127.0f, d);
     if (threadIdx.x == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
-    uint2* qr = xq + static_cast<size_t>(row) * nvec;
+    const size_t tb8 = xq_tb8(T);
     for (int idx = threadIdx.x; idx < nvec; idx += kActThreads) {
         const uint4 v = __ldg(xr + idx);
         uint2 o;
         o.x = quant_pair2(v.x, v.y, s_x);
         o.y = quant_pair2(v.z, v.w, s_x);
-        qr[idx] = o;
+        xq[xq_tiled_u2_index(row, idx, tb8)] = o;
     }
 }
 

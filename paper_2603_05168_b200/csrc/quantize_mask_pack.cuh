@@ -14,8 +14,8 @@
 //                                     last -- still resident in the 126 MB L2 -- is read first.
 //
 // Both passes are HBM-bound streaming kernels: 16 B loads per lane, a warp instruction covers
-// 512 contiguous bytes; stores are 2 B (vals), 4 B (dense W_q) per lane contiguous across the
-// warp, and 1 B per even lane (metadata).
+// 512 contiguous bytes; a warp store covers one whole 64 B (vals), 128 B (dense W_q) or 16 B
+// (metadata) row of an operand tile (tiled layouts, see layouts.cuh).
 //
 // Ternarisation without a per-element division: W_q = sign(w) * [ fl(|w| / scale) > 0.5 ]
 // (round-half-even sends exactly 0.5 to 0, everything above to >= 1, the clamp caps at 1).
@@ -25,6 +25,7 @@
 #pragma once
 
 #include "sbn_common.cuh"
+#include "layouts.cuh"
 
 namespace sbn {
 
@@ -131,14 +132,13 @@ __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
 
 template <bool WRITE_DENSE, bool COUNT_FLIPS>
 __global__ void __launch_bounds__(kQmpThreads)
-mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, double inv_count_unused,
+mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, uint32_t KB,
                  double count, const double* __restrict__ partial, int num_partials,
                  uint16_t* __restrict__ vals, uint8_t* meta,
                  float* __restrict__ w_scale, uint32_t* __restrict__ dense_q,
                  const uint8_t* prev_meta, unsigned long long* __restrict__ flip_bits) {
     __shared__ double s_warp[kQmpThreads / 32];
     __shared__ float s_thr;
-    (void)inv_count_unused;
 
     // Fixed-order reduction of the pass-1 partials: thread j adds partial[j], partial[j + 256],
     // ... then the block tree; every CTA gets the same bits.
@@ -158,24 +158,38 @@ mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, double inv_cou
     const int warp = threadIdx.x >> 5;
     unsigned int flips = 0;
 
+    // One warp iteration = 32 consecutive groups = one (row, 128-column block) unit; unit index
+    // u = n * KB + kb.  Outputs go to the tiled layouts of layouts.cuh.
     for (size_t it = blockIdx.x; it < num_tiles; it += gridDim.x) {
         const size_t tile = num_tiles - 1 - it;                       // backwards: L2-warm first
         const size_t g_base = tile * (kQmpTileFloats / 4) + static_cast<size_t>(warp) * 128;
+        const uint32_t u_base = static_cast<uint32_t>(tile * 32 + static_cast<size_t>(warp) * 4);
+        uint32_t n_cur = u_base / KB;
+        uint32_t kb_cur = u_base - n_cur * KB;
         float4 w[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) w[j] = __ldg(W4 + g_base + j * 32 + lane);
+        size_t tile_idx[4];           // (n/128)*KB + kb
+        uint32_t row_in_tile[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            tile_idx[j] = static_cast<size_t>(n_cur >> 7) * KB + kb_cur;
+            row_in_tile[j] = n_cur & 127u;
+            if (++kb_cur == KB) { kb_cur = 0; ++n_cur; }
+        }
         uint32_t prev[4];
         if constexpr (COUNT_FLIPS) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                prev[j] = (lane & 1) ? 0u : prev_meta[(g_base + j * 32 + lane) >> 1];
+                prev[j] = (lane & 1) ? 0u : prev_meta[(tile_idx[j] << 11) + (row_in_tile[j] << 4) + (lane >> 1)];
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const size_t g = g_base + j * 32 + lane;                  // group index, row-major
             const GroupResult r = process_group(w[j], thr);
-            vals[g] = static_cast<uint16_t>(r.vals16);
-            if constexpr (WRITE_DENSE) dense_q[g] = r.dense32;
+            const uint32_t rr = row_in_tile[j];
+            // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
+            vals[((tile_idx[j] << 13) + vals_in_tile(rr, 2u * lane)) >> 1] = static_cast<uint16_t>(r.vals16);
+            if constexpr (WRITE_DENSE) dense_q[((tile_idx[j] << 14) + sw128_in_tile(rr, 4u * lane)) >> 2] = r.dense32;
             const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, r.nibble, 1);
             if ((lane & 1) == 0) {
                 const uint32_t byte = r.nibble | (hi << 4);
@@ -183,7 +197,7 @@ mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, double inv_cou
                     flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev[j] & 15u)) +
                              __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev[j] >> 4) & 15u));
                 }
-                meta[g >> 1] = static_cast<uint8_t>(byte);
+                meta[(tile_idx[j] << 11) + (rr << 4) + (lane >> 1)] = static_cast<uint8_t>(byte);
             }
         }
     }
@@ -231,7 +245,7 @@ inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t
     const double cnt = static_cast<double>(count);
 #define SBN_QMP_LAUNCH(D, F)                                                                   \
     mask_pack_kernel<D, F><<<static_cast<unsigned>(grid), kQmpThreads, 0, stream>>>(           \
-        W4, num_tiles, 0.0, cnt, partial, P, v16, meta, w_scale, d32, prev_meta, flip_bits)
+        W4, num_tiles, static_cast<uint32_t>(K / 128), cnt, partial, P, v16, meta, w_scale, d32, prev_meta, flip_bits)
     if (dense_q && prev_meta) SBN_QMP_LAUNCH(true, true);
     else if (dense_q) SBN_QMP_LAUNCH(true, false);
     else if (prev_meta) SBN_QMP_LAUNCH(false, true);

@@ -6,6 +6,62 @@ import torch
 from paper_2603_05168_b200 import binding as b
 
 
+# ---- the library's tiled storage orders, restated from the formulas documented in include/sbn.h --
+def _vals_offsets(N, K):
+    n = np.arange(N, dtype=np.int64)[:, None]
+    c = np.arange(K // 2, dtype=np.int64)[None, :]
+    KB, r, cc = K // 128, n & 127, c & 63
+    return ((n >> 7) * KB + (c >> 6)) * 8192 + (r << 6) + ((((cc >> 4) ^ ((r >> 1) & 3))) << 4) + (cc & 15)
+
+
+def _meta_offsets(N, K):
+    n = np.arange(N, dtype=np.int64)[:, None]
+    b = np.arange(K // 8, dtype=np.int64)[None, :]
+    KB, r = K // 128, n & 127
+    return ((n >> 7) * KB + (b >> 4)) * 2048 + (r << 4) + (b & 15)
+
+
+def _dense_offsets(N, K):
+    n = np.arange(N, dtype=np.int64)[:, None]
+    k = np.arange(K, dtype=np.int64)[None, :]
+    KB, r, c = K // 128, n & 127, k & 127
+    return ((n >> 7) * KB + (k >> 7)) * 16384 + ((r >> 3) << 10) + ((r & 7) << 7) + ((((c >> 4) ^ (r & 7))) << 4) + (c & 15)
+
+
+def _xq_offsets(T, K):
+    t = np.arange(T, dtype=np.int64)[:, None]
+    k = np.arange(K, dtype=np.int64)[None, :]
+    TB8, r, c = 2 * ((T + 15) // 16), t & 7, k & 127
+    return ((k >> 7) * TB8 + (t >> 3)) * 1024 + (r << 7) + ((((c >> 4) ^ r)) << 4) + (c & 15)
+
+
+def untile(flat: np.ndarray, offsets: np.ndarray) -> np.ndarray:
+    """tiled byte buffer -> plain row-major array."""
+    return np.ascontiguousarray(flat.reshape(-1)[offsets])
+
+
+def tile(canonical: np.ndarray, offsets: np.ndarray, nbytes: int) -> np.ndarray:
+    """plain row-major array -> tiled byte buffer (bytes no element maps to stay 0)."""
+    out = np.zeros(nbytes, canonical.dtype)
+    out[offsets] = canonical
+    return out
+
+
+def tile_vals(vals):
+    N, K2 = vals.shape
+    return tile(vals, _vals_offsets(N, 2 * K2), vals.size)
+
+
+def tile_meta(meta):
+    N, K8 = meta.shape
+    return tile(meta, _meta_offsets(N, 8 * K8), meta.size)
+
+
+def tile_xq(xq):
+    T, K = xq.shape
+    return tile(xq, _xq_offsets(T, K), b.sbn_xq_bytes(T, K))
+
+
 def dev(a: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
@@ -22,18 +78,20 @@ def gpu_quantize_mask_pack(W: np.ndarray, with_dense=True, prev_meta=None, in_pl
     pm = None
     if prev_meta is not None:
         flip = torch.full((1,), 12345, dtype=torch.int64, device="cuda")   # must be overwritten
+        prev_tiled = tile_meta(prev_meta).reshape(N, K // 8)
         if in_place:
-            bufs["meta"].copy_(dev(prev_meta))
+            bufs["meta"].copy_(dev(prev_tiled))
             pm = bufs["meta"]
         else:
-            pm = dev(prev_meta)
+            pm = dev(prev_tiled)
     b.sbn_quantize_mask_pack(Wd, bufs["vals"], bufs["meta"], bufs["w_scale"], bufs["ws"],
                              dense_q=bufs.get("dense_q"), prev_meta=pm, flip_bits=flip)
     b.sbn_check_status()
-    out = dict(vals=bufs["vals"].cpu().numpy(), meta=bufs["meta"].cpu().numpy(),
+    out = dict(vals=untile(bufs["vals"].cpu().numpy(), _vals_offsets(N, K)),
+               meta=untile(bufs["meta"].cpu().numpy(), _meta_offsets(N, K)),
                scale=np.float32(bufs["w_scale"].cpu().numpy()[0]), dev=bufs)
     if with_dense:
-        out["dense_q"] = bufs["dense_q"].cpu().numpy()
+        out["dense_q"] = untile(bufs["dense_q"].cpu().numpy(), _dense_offsets(N, K))
     if flip is not None:
         out["flips"] = int(flip.cpu().numpy()[0])
     return out
@@ -42,17 +100,22 @@ def gpu_quantize_mask_pack(W: np.ndarray, with_dense=True, prev_meta=None, in_pl
 def gpu_quant_act(x_bits: np.ndarray):
     T, K = x_bits.shape
     xd = bf16_dev(x_bits)
-    xq = torch.empty((T, K), dtype=torch.int8, device="cuda")
+    xq = b.alloc_xq(T, K)
     a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
     b.sbn_quant_act(xd, xq, a_scale)
     b.sbn_check_status()
     return xq, a_scale
 
 
+def xq_to_numpy(xq: torch.Tensor, T: int, K: int) -> np.ndarray:
+    """Tiled device activations -> plain [T][K] int8."""
+    return untile(xq.cpu().numpy(), _xq_offsets(T, K))
+
+
 def gpu_gemm(sparse: bool, xq, a_scale, packed_dev, out_dtype=torch.float32, bias=None, want_acc=True):
     """xq / a_scale: device tensors; packed_dev: dict of device tensors from alloc_packed."""
-    T, K = xq.shape
-    N = packed_dev["vals"].shape[0]
+    T = a_scale.numel()
+    N, K = packed_dev["vals"].shape[0], 2 * packed_dev["vals"].shape[1]
     y = torch.full((T, N), float("nan"), dtype=out_dtype, device="cuda")
     acc = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device="cuda") if want_acc else None
     op = b.OP_SPARSE_BITLINEAR if sparse else b.OP_BITLINEAR

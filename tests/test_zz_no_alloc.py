@@ -71,4 +71,4 @@ def test_static_ws_matches_workspace_entry_point_twice_in_a_row():
     assert float(r2["w_scale"].item()) > 10 * float(r1["w_scale"].item())
     # and once more with the flip count enabled
     W3 = inputs.perturb_weights(W1, seed=33, sigma=1e-4)
-    _run_both(W3, prev_meta_np=r1["meta"].cpu().numpy())
+    _run_both(W3, prev_meta_np=r1["meta"].cpu().numpy())      # r1's metadata is already in the library's order
