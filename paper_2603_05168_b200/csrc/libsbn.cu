@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 
 #include "sbn.h"
@@ -371,7 +372,7 @@ sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int 
         (prev_meta && misaligned(prev_meta, 16)) || (flip_bits && misaligned(flip_bits, 8)))
         return SBN_ERR_ALIGN;
     return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
-                                     static_cast<QmpWorkspace*>(ws)->partial,
+                                     static_cast<QmpWorkspace*>(ws),
                                      static_cast<cudaStream_t>(stream));
 }
 
@@ -395,9 +396,9 @@ sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_
         return SBN_ERR_ALIGN;
     void* scratch = static_scratch_for_current_device();
     if (!scratch) return SBN_ERR_CUDA;
-    // pass 1 writes every partial slot that pass 2 reads, so stale contents are harmless
+    // every slot that is read carries this call's nonce, so stale contents are harmless
     return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
-                                     static_cast<QmpWorkspace*>(scratch)->partial,
+                                     static_cast<QmpWorkspace*>(scratch),
                                      static_cast<cudaStream_t>(stream));
 }
 

@@ -16,7 +16,6 @@
 namespace sbn {
 
 constexpr int kActThreads = 256;
-constexpr int kActVecPerThread = 8;   // up to 8 x 16 B of one row per thread
 
 __device__ __forceinline__ float absmax8(const uint4& v) {
     float m = fmaxf(fabsf(bf16lo_to_f32(v.x)), fabsf(bf16hi_to_f32(v.x)));
@@ -47,61 +46,70 @@ __device__ __forceinline__ size_t xq_tiled_u2_index(int t, int idx, size_t tb8) 
     return (atom << 7) + (r << 4) + ((chunk ^ r) << 1) + half;
 }
 
-template <int G>
-__global__ void __launch_bounds__(kActThreads)
+// G threads per token row, VPT 16-byte vectors per thread (G * VPT >= K / 8).  Persistent CTAs:
+// every row group walks over rows with a grid-sized stride and loads its NEXT row while it reduces,
+// rounds and stores the current one, so each SM always has loads in flight (a non-pipelined
+// version of this kernel was latency-bound at a third of the HBM rate).
+template <int G, int VPT>
+__global__ void __launch_bounds__(kActThreads, (VPT <= 4) ? 3 : 2)
 quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
                  float* __restrict__ a_scale) {
     constexpr int ROWS = kActThreads / G;
     constexpr int WARPS_PER_ROW = (G + 31) / 32;
-    __shared__ float s_max[kActThreads / 32];
+    __shared__ float s_max[2][kActThreads / 32];
 
     const int r = threadIdx.x / G;
     const int g = threadIdx.x % G;
-    const int row = blockIdx.x * ROWS + r;
-    const bool active = row < T;
-    const uint4* xr = x + static_cast<size_t>(active ? row : 0) * nvec;
-
-    uint4 v[kActVecPerThread];
-    float amax = 0.0f;
-#pragma unroll
-    for (int i = 0; i < kActVecPerThread; ++i) {
-        const int idx = g + i * G;
-        if (active && idx < nvec) {
-            v[i] = __ldg(xr + idx);
-        } else {
-            v[i] = make_uint4(0u, 0u, 0u, 0u);
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < kActVecPerThread; ++i) amax = fmaxf(amax, absmax8(v[i]));
-
-    amax = warp_max(amax);
-    if constexpr (WARPS_PER_ROW > 1) {
-        const int warp = threadIdx.x >> 5;
-        if ((threadIdx.x & 31) == 0) s_max[warp] = amax;
-        __syncthreads();
-        const int w0 = (r * G) >> 5;
-        float m = s_max[w0];
-#pragma unroll
-        for (int w = 1; w < WARPS_PER_ROW; ++w) m = fmaxf(m, s_max[w0 + w]);
-        amax = m;
-    }
-    if (!active) return;
-
-    const float d = fmaxf(amax, kEps);
-    const float s_x = __fdiv_rn(127.0f, d);
-    if (g == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
-
+    const int row_stride = gridDim.x * ROWS;
     const size_t tb8 = xq_tb8(T);
+    const int iters = (T + row_stride - 1) / row_stride;        // same for every thread of the CTA
+
+    uint4 cur[VPT], nxt[VPT];
+    int row = blockIdx.x * ROWS + r;
 #pragma unroll
-    for (int i = 0; i < kActVecPerThread; ++i) {
+    for (int i = 0; i < VPT; ++i) {
         const int idx = g + i * G;
-        if (idx < nvec) {
-            uint2 o;
-            o.x = quant_pair2(v[i].x, v[i].y, s_x);
-            o.y = quant_pair2(v[i].z, v[i].w, s_x);
-            xq[xq_tiled_u2_index(row, idx, tb8)] = o;
+        cur[i] = (row < T && idx < nvec) ? __ldg(x + static_cast<size_t>(row) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    for (int it = 0; it < iters; ++it, row += row_stride) {
+        const int row_n = row + row_stride;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = g + i * G;
+            nxt[i] = (row_n < T && idx < nvec) ? __ldg(x + static_cast<size_t>(row_n) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
         }
+        float amax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) amax = fmaxf(amax, absmax8(cur[i]));
+        amax = warp_max(amax);
+        if constexpr (WARPS_PER_ROW > 1) {
+            const int warp = threadIdx.x >> 5;
+            float* sm = s_max[it & 1];                               // double buffered: one barrier per row
+            if ((threadIdx.x & 31) == 0) sm[warp] = amax;
+            __syncthreads();
+            const int w0 = (r * G) >> 5;
+            float m = sm[w0];
+#pragma unroll
+            for (int w = 1; w < WARPS_PER_ROW; ++w) m = fmaxf(m, sm[w0 + w]);
+            amax = m;
+        }
+        if (row < T) {
+            const float d = fmaxf(amax, kEps);
+            const float s_x = __fdiv_rn(127.0f, d);
+            if (g == 0) a_scale[row] = __fdiv_rn(d, 127.0f);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int idx = g + i * G;
+                if (idx < nvec) {
+                    uint2 o;
+                    o.x = quant_pair2(cur[i].x, cur[i].y, s_x);
+                    o.y = quant_pair2(cur[i].z, cur[i].w, s_x);
+                    xq[xq_tiled_u2_index(row, idx, tb8)] = o;
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) cur[i] = nxt[i];
     }
 }
 
@@ -135,23 +143,31 @@ quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* _
     }
 }
 
+template <int G, int VPT>
+static void launch_quant_act_cfg(const uint4* x, int T, int nvec, uint2* q, float* a_scale, cudaStream_t stream) {
+    constexpr int rows = kActThreads / G;
+    const int ctas_per_sm = (VPT <= 4) ? 3 : 2;
+    int grid = (T + rows - 1) / rows;
+    if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
+    quant_act_kernel<G, VPT><<<grid, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+}
+
 inline sbn_status launch_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale,
                                    cudaStream_t stream) {
     const int nvec = K / 8;
     const uint4* x = static_cast<const uint4*>(x_bf16);
     uint2* q = reinterpret_cast<uint2*>(xq);
-    const int per_thread_cap = kActVecPerThread;
-    if (nvec <= 32 * per_thread_cap) {
-        quant_act_kernel<32><<<(T + 7) / 8, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
-    } else if (nvec <= 64 * per_thread_cap) {
-        quant_act_kernel<64><<<(T + 3) / 4, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
-    } else if (nvec <= 128 * per_thread_cap) {
-        quant_act_kernel<128><<<(T + 1) / 2, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
-    } else if (nvec <= 256 * per_thread_cap) {
-        quant_act_kernel<256><<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
-    } else {
-        quant_act_long_row_kernel<<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
-    }
+    // smallest group that keeps <= 3 (then 4, 6, 8) vectors per thread
+    if (nvec <= 32 * 2) launch_quant_act_cfg<32, 2>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 64 * 2) launch_quant_act_cfg<64, 2>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 128 * 2) launch_quant_act_cfg<128, 2>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 128 * 3) launch_quant_act_cfg<128, 3>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 2) launch_quant_act_cfg<256, 2>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 3) launch_quant_act_cfg<256, 3>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 4) launch_quant_act_cfg<256, 4>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 6) launch_quant_act_cfg<256, 6>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 8) launch_quant_act_cfg<256, 8>(x, T, nvec, q, a_scale, stream);
+    else quant_act_long_row_kernel<<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }

@@ -1,21 +1,23 @@
 // Part 1 of the path: absmean ternary quantisation (Eq. 1), 2:4 magnitude mask from the master
 // weights (Eq. 2), W_eff = W_q (.) M (Eq. 3), compressed value + metadata layout.
 //
-// gamma needs the whole matrix before any element can be rounded, so there are two passes:
+// gamma needs the whole matrix before any element can be rounded, so W has to be looked at
+// twice.  One persistent cooperative kernel (one 1024-thread CTA per SM) does both passes:
 //
-//   pass 1  absmean_partials_kernel   sum|W| in fp64, fixed grid, one partial per CTA
-//                                     (fixed assignment of elements to threads and a fixed
-//                                     reduction tree -> the same bits on every run)
-//   pass 2  mask_pack_kernel          every CTA re-reduces the partials in the same fixed order
-//                                     (no atomics, no counter, no third launch), derives the
-//                                     scale, then streams W once more: top-2-of-4, ternarise,
-//                                     write vals / meta (/ dense W_q / flip count).
-//                                     Pass 2 walks the matrix backwards, so what pass 1 read
-//                                     last -- still resident in the 126 MB L2 -- is read first.
+//   pass 1   every CTA owns a contiguous range of (row, 128-column) units, streams it once,
+//            accumulates sum|W| in fp64 and KEEPS the first part of its range in shared memory
+//            (200 KB per SM: 148 SMs hold 29.6 MB of W on chip);
+//   exchange every CTA publishes {call nonce, partial sum} in the workspace and waits (bounded)
+//            until all slots carry this call's nonce -- no atomics, no counter, nothing to
+//            initialise, stale slots of earlier calls can never match; every CTA then adds the
+//            148 partials in the same fixed order, so all get the same bits, run after run;
+//   pass 2   top-2-of-4, ternarise, pack: the resident part comes from shared memory, the rest
+//            is read again, newest first (what pass 1 read last is still in the 126 MB L2).
 //
-// Both passes are HBM-bound streaming kernels: 16 B loads per lane, a warp instruction covers
-// 512 contiguous bytes; a warp store covers one whole 64 B (vals), 128 B (dense W_q) or 16 B
-// (metadata) row of an operand tile (tiled layouts, see layouts.cuh).
+// HBM traffic per parameter: 4 B (one read) + 0.625 B written for the resident part, one more
+// (mostly L2-served) 4 B read for the rest.  16 B loads per lane, a warp covers one 512 B unit;
+// a warp store covers one whole 64 B (vals), 128 B (dense W_q) or 16 B (metadata) row of an
+// operand tile (tiled layouts, see layouts.cuh).
 //
 // Ternarisation without a per-element division: W_q = sign(w) * [ fl(|w| / scale) > 0.5 ]
 // (round-half-even sends exactly 0.5 to 0, everything above to >= 1, the clamp caps at 1).
@@ -29,62 +31,27 @@
 
 namespace sbn {
 
-constexpr int kQmpThreads = 256;
-constexpr int kQmpMaxPartials = kNumSMs * 4;          // pass-1 grid upper bound
-constexpr int kQmpTileFloats = kQmpThreads * 16;      // 4 float4 per thread per tile
+constexpr int kQmpThreads = 1024;
+constexpr int kQmpWarps = kQmpThreads / 32;
+constexpr int kQmpMaxCtas = kNumSMs;                       // one CTA per SM, all co-resident
+constexpr int kQmpResidentUnits = 400;                     // 400 x 512 B = 200 KB of W kept in smem
+constexpr int kQmpSmemBytes = kQmpResidentUnits * 512;
+constexpr unsigned long long kQmpWaitLimitNs = 2000000000ull;
 
+struct QmpSlot {                 // one per CTA, 16 B
+    unsigned long long nonce;    // identifies the call that wrote `partial`
+    double partial;              // this CTA's sum |W|
+};
 struct QmpWorkspace {            // layout of the caller's workspace
-    double partial[kQmpMaxPartials];
+    QmpSlot slot[kQmpMaxCtas];
 };
 
-// ------------------------------------------------------------------------------------------------
-// pass 1
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ double block_sum_fixed(double v, double* s_warp) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    const int warp = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) s_warp[warp] = v;
-    __syncthreads();
-    double t = 0.0;
-#pragma unroll
-    for (int w = 0; w < kQmpThreads / 32; ++w) t += s_warp[w];
-    __syncthreads();
-    return t;       // identical in every thread
+__device__ __forceinline__ unsigned long long global_timer_ns_qmp() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
 
-__global__ void __launch_bounds__(kQmpThreads)
-absmean_partials_kernel(const float4* __restrict__ W4, size_t n4, double* __restrict__ partial,
-                        unsigned long long* __restrict__ flip_bits) {
-    __shared__ double s_warp[kQmpThreads / 32];
-    const size_t stride = static_cast<size_t>(gridDim.x) * kQmpThreads;
-    size_t i = static_cast<size_t>(blockIdx.x) * kQmpThreads + threadIdx.x;
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    // four independent 16 B loads in flight per thread
-    for (; i + 3 * stride < n4; i += 4 * stride) {
-        const float4 v0 = __ldg(W4 + i);
-        const float4 v1 = __ldg(W4 + i + stride);
-        const float4 v2 = __ldg(W4 + i + 2 * stride);
-        const float4 v3 = __ldg(W4 + i + 3 * stride);
-        a0 += (double)fabsf(v0.x); a1 += (double)fabsf(v0.y); a2 += (double)fabsf(v0.z); a3 += (double)fabsf(v0.w);
-        a0 += (double)fabsf(v1.x); a1 += (double)fabsf(v1.y); a2 += (double)fabsf(v1.z); a3 += (double)fabsf(v1.w);
-        a0 += (double)fabsf(v2.x); a1 += (double)fabsf(v2.y); a2 += (double)fabsf(v2.z); a3 += (double)fabsf(v2.w);
-        a0 += (double)fabsf(v3.x); a1 += (double)fabsf(v3.y); a2 += (double)fabsf(v3.z); a3 += (double)fabsf(v3.w);
-    }
-    for (; i < n4; i += stride) {
-        const float4 v0 = __ldg(W4 + i);
-        a0 += (double)fabsf(v0.x); a1 += (double)fabsf(v0.y); a2 += (double)fabsf(v0.z); a3 += (double)fabsf(v0.w);
-    }
-    const double t = block_sum_fixed((a0 + a1) + (a2 + a3), s_warp);
-    if (threadIdx.x == 0) {
-        partial[blockIdx.x] = t;
-        if (blockIdx.x == 0 && flip_bits != nullptr) *flip_bits = 0ull;   // pass 2 accumulates
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// pass 2
-// ------------------------------------------------------------------------------------------------
 // Smallest fp32 a with fl(a / scale) > 0.5, searched around 0.5 * scale with IEEE divisions.
 __device__ __forceinline__ float ternary_threshold(float scale) {
     float a = 0.5f * scale;
@@ -130,21 +97,97 @@ __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
     return (1u << (nib & 3u)) | (1u << ((nib >> 2) & 3u));
 }
 
-template <bool WRITE_DENSE, bool COUNT_FLIPS>
-__global__ void __launch_bounds__(kQmpThreads)
-mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, uint32_t KB,
-                 double count, const double* __restrict__ partial, int num_partials,
-                 uint16_t* __restrict__ vals, uint8_t* meta,
-                 float* __restrict__ w_scale, uint32_t* __restrict__ dense_q,
-                 const uint8_t* prev_meta, unsigned long long* __restrict__ flip_bits) {
-    __shared__ double s_warp[kQmpThreads / 32];
-    __shared__ float s_thr;
+// Sum of `v` over the CTA in a fixed order; identical in every thread.
+__device__ __forceinline__ double qmp_block_sum(double v, double* s_warp) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const int warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) s_warp[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kQmpWarps; ++w) t += s_warp[w];
+    __syncthreads();
+    return t;
+}
 
-    // Fixed-order reduction of the pass-1 partials: thread j adds partial[j], partial[j + 256],
-    // ... then the block tree; every CTA gets the same bits.
-    double v = 0.0;
-    for (int j = threadIdx.x; j < num_partials; j += kQmpThreads) v += partial[j];
-    const double S = block_sum_fixed(v, s_warp);
+__device__ __forceinline__ double abs_sum4(const float4 v) {
+    return ((double)fabsf(v.x) + (double)fabsf(v.y)) + ((double)fabsf(v.z) + (double)fabsf(v.w));
+}
+
+template <bool WRITE_DENSE, bool COUNT_FLIPS>
+__global__ void __launch_bounds__(kQmpThreads, 1)
+quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uint32_t KB, double count,
+                          QmpSlot* slots, unsigned long long nonce,
+                          uint16_t* __restrict__ vals, uint8_t* meta, float* __restrict__ w_scale,
+                          uint32_t* __restrict__ dense_q, const uint8_t* prev_meta,
+                          unsigned long long* __restrict__ flip_bits) {
+    extern __shared__ float4 s_w[];                     // resident units, 32 float4 each
+    __shared__ double s_warp[kQmpWarps];
+    __shared__ float s_thr;
+    __shared__ int s_ok;
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t per = (num_units + gridDim.x - 1) / gridDim.x;
+    const uint32_t u_begin = min(num_units, blockIdx.x * per);
+    const uint32_t u_end = min(num_units, u_begin + per);
+    const uint32_t n_res = min(u_end - u_begin, static_cast<uint32_t>(kQmpResidentUnits));
+
+    // ---- pass 1: sum |W| over this CTA's range (4 independent 16 B loads in flight per thread)
+    double acc = 0.0;
+    {
+        uint32_t u = u_begin + warp;
+        for (; u + 3 * kQmpWarps < u_end; u += 4 * kQmpWarps) {
+            const float4 v0 = __ldg(W4 + static_cast<size_t>(u) * 32 + lane);
+            const float4 v1 = __ldg(W4 + static_cast<size_t>(u + kQmpWarps) * 32 + lane);
+            const float4 v2 = __ldg(W4 + static_cast<size_t>(u + 2 * kQmpWarps) * 32 + lane);
+            const float4 v3 = __ldg(W4 + static_cast<size_t>(u + 3 * kQmpWarps) * 32 + lane);
+            acc += (abs_sum4(v0) + abs_sum4(v1)) + (abs_sum4(v2) + abs_sum4(v3));
+            const uint32_t r = u - u_begin;
+            if (r < n_res) s_w[r * 32 + lane] = v0;
+            if (r + kQmpWarps < n_res) s_w[(r + kQmpWarps) * 32 + lane] = v1;
+            if (r + 2 * kQmpWarps < n_res) s_w[(r + 2 * kQmpWarps) * 32 + lane] = v2;
+            if (r + 3 * kQmpWarps < n_res) s_w[(r + 3 * kQmpWarps) * 32 + lane] = v3;
+        }
+        for (; u < u_end; u += kQmpWarps) {
+            const float4 v0 = __ldg(W4 + static_cast<size_t>(u) * 32 + lane);
+            acc += abs_sum4(v0);
+            const uint32_t r = u - u_begin;
+            if (r < n_res) s_w[r * 32 + lane] = v0;
+        }
+    }
+    const double mine = qmp_block_sum(acc, s_warp);
+
+    // ---- exchange: publish, then wait (bounded) until every slot carries this call's nonce
+    if (threadIdx.x == 0) {
+        s_ok = 1;
+        if (blockIdx.x == 0 && flip_bits != nullptr) *flip_bits = 0ull;     // pass 2 accumulates
+        slots[blockIdx.x].partial = mine;
+        __threadfence();
+        *reinterpret_cast<volatile unsigned long long*>(&slots[blockIdx.x].nonce) = nonce;
+    }
+    __syncthreads();
+    double other = 0.0;
+    if (threadIdx.x < gridDim.x) {
+        const volatile unsigned long long* flag = &slots[threadIdx.x].nonce;
+        const unsigned long long t0 = global_timer_ns_qmp();
+        unsigned int spins = 0;
+        bool seen = (*flag == nonce);
+        while (!seen) {
+            seen = (*flag == nonce);
+            if (!seen && ((++spins & 0xFFu) == 0) && global_timer_ns_qmp() - t0 > kQmpWaitLimitNs) break;
+        }
+        if (seen) {
+            __threadfence();
+            other = *reinterpret_cast<const volatile double*>(&slots[threadIdx.x].partial);
+        } else {
+            s_ok = 0;
+            atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+        }
+    }
+    const double S = qmp_block_sum(other, s_warp);          // fixed order: the same bits in every CTA
+    if (!s_ok) return;                                       // a peer never arrived: give up cleanly
     const float gamma = static_cast<float>(S / count);
     const float scale = fmaxf(gamma, kEps);
     if (threadIdx.x == 0) {
@@ -154,50 +197,57 @@ mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, uint32_t KB,
     __syncthreads();
     const float thr = s_thr;
 
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
+    // ---- pass 2: a warp takes four units at a time (four 16 B loads in flight per lane); the
+    // re-read part newest first, then the resident part from shared memory
     unsigned int flips = 0;
-
-    // One warp iteration = 32 consecutive groups = one (row, 128-column block) unit; unit index
-    // u = n * KB + kb.  Outputs go to the tiled layouts of layouts.cuh.
-    for (size_t it = blockIdx.x; it < num_tiles; it += gridDim.x) {
-        const size_t tile = num_tiles - 1 - it;                       // backwards: L2-warm first
-        const size_t g_base = tile * (kQmpTileFloats / 4) + static_cast<size_t>(warp) * 128;
-        const uint32_t u_base = static_cast<uint32_t>(tile * 32 + static_cast<size_t>(warp) * 4);
-        uint32_t n_cur = u_base / KB;
-        uint32_t kb_cur = u_base - n_cur * KB;
+    const uint32_t n_units = u_end - u_begin;
+    // (row, k-block) of the warp's first unit by one division, then stepped down by 32 units a time
+    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+    int n_cur = 0, kb_cur = 0;
+    if (static_cast<uint32_t>(warp) < n_units) {
+        const uint32_t u_first = u_begin + (n_units - 1 - warp);
+        n_cur = static_cast<int>(u_first / KB);
+        kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
+    }
+    for (uint32_t i0 = warp; i0 < n_units; i0 += 4 * kQmpWarps) {
         float4 w[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) w[j] = __ldg(W4 + g_base + j * 32 + lane);
-        size_t tile_idx[4];           // (n/128)*KB + kb
-        uint32_t row_in_tile[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            tile_idx[j] = static_cast<size_t>(n_cur >> 7) * KB + kb_cur;
-            row_in_tile[j] = n_cur & 127u;
-            if (++kb_cur == KB) { kb_cur = 0; ++n_cur; }
-        }
         uint32_t prev[4];
-        if constexpr (COUNT_FLIPS) {
+        size_t tile_idx[4];
+        uint32_t rr[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                prev[j] = (lane & 1) ? 0u : prev_meta[(tile_idx[j] << 11) + (row_in_tile[j] << 4) + (lane >> 1)];
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t i = i0 + q * kQmpWarps;
+            // i-th unit in processing order: units n_units-1 .. n_res (from global), then n_res-1 .. 0
+            if (i < n_units) {
+                const uint32_t r = n_units - 1 - i;
+                w[q] = (r < n_res) ? s_w[r * 32 + lane] : __ldg(W4 + static_cast<size_t>(u_begin + r) * 32 + lane);
+                tile_idx[q] = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+                rr[q] = static_cast<uint32_t>(n_cur) & 127u;
+                n_cur -= step_n;
+                kb_cur -= step_kb;
+                if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
+                if constexpr (COUNT_FLIPS) {
+                    prev[q] = (lane & 1) ? 0u : prev_meta[(tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1)];
+                }
+            }
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const GroupResult r = process_group(w[j], thr);
-            const uint32_t rr = row_in_tile[j];
-            // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
-            vals[((tile_idx[j] << 13) + vals_in_tile(rr, 2u * lane)) >> 1] = static_cast<uint16_t>(r.vals16);
-            if constexpr (WRITE_DENSE) dense_q[((tile_idx[j] << 14) + sw128_in_tile(rr, 4u * lane)) >> 2] = r.dense32;
-            const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, r.nibble, 1);
-            if ((lane & 1) == 0) {
-                const uint32_t byte = r.nibble | (hi << 4);
-                if constexpr (COUNT_FLIPS) {
-                    flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev[j] & 15u)) +
-                             __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev[j] >> 4) & 15u));
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t i = i0 + q * kQmpWarps;
+            if (i < n_units) {
+                const GroupResult g = process_group(w[q], thr);
+                // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
+                vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(g.vals16);
+                if constexpr (WRITE_DENSE) dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = g.dense32;
+                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, g.nibble, 1);
+                if ((lane & 1) == 0) {
+                    const uint32_t byte = g.nibble | (hi << 4);
+                    if constexpr (COUNT_FLIPS) {
+                        flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev[q] & 15u)) +
+                                 __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev[q] >> 4) & 15u));
+                    }
+                    meta[(tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1)] = static_cast<uint8_t>(byte);
                 }
-                meta[(tile_idx[j] << 11) + (rr << 4) + (lane >> 1)] = static_cast<uint8_t>(byte);
             }
         }
     }
@@ -205,54 +255,58 @@ mask_pack_kernel(const float4* __restrict__ W4, size_t num_tiles, uint32_t KB,
     if constexpr (COUNT_FLIPS) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) flips += __shfl_xor_sync(0xFFFFFFFFu, flips, o);
-        __shared__ unsigned int s_flips[kQmpThreads / 32];
+        __shared__ unsigned int s_flips[kQmpWarps];
         if (lane == 0) s_flips[warp] = flips;
         __syncthreads();
         if (threadIdx.x == 0) {
             unsigned long long t = 0;
 #pragma unroll
-            for (int w2 = 0; w2 < kQmpThreads / 32; ++w2) t += s_flips[w2];
+            for (int w2 = 0; w2 < kQmpWarps; ++w2) t += s_flips[w2];
             if (t) atomicAdd(flip_bits, t);
         }
     }
 }
 
-inline int qmp_num_partials(size_t n4) {
-    const size_t per_cta = static_cast<size_t>(kQmpThreads) * 4;
-    size_t want = (n4 + per_cta - 1) / per_cta;
-    if (want < 1) want = 1;
-    if (want > static_cast<size_t>(kQmpMaxPartials)) want = kQmpMaxPartials;
-    return static_cast<int>(want);
+// Per-call nonce: unique within the process, never 0.
+inline unsigned long long qmp_next_nonce() {
+    static std::atomic<unsigned long long> counter{0x5B4E0000ull};
+    return counter.fetch_add(1) + 1;
 }
 
 inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t* vals,
                                             uint8_t* meta, float* w_scale, int8_t* dense_q,
                                             const uint8_t* prev_meta,
-                                            unsigned long long* flip_bits, double* partial,
+                                            unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
-    const size_t count = static_cast<size_t>(N) * K;
-    const size_t n4 = count / 4;
-    const int P = qmp_num_partials(n4);
-    absmean_partials_kernel<<<P, kQmpThreads, 0, stream>>>(
-        reinterpret_cast<const float4*>(W), n4, partial, prev_meta ? flip_bits : nullptr);
-    ++g_launch_count;
-
-    const size_t num_tiles = count / kQmpTileFloats;
-    size_t grid = num_tiles < static_cast<size_t>(kNumSMs * 8) ? num_tiles : kNumSMs * 8;
+    const size_t count_sz = static_cast<size_t>(N) * K;
+    uint32_t num_units = static_cast<uint32_t>(count_sz / 128);
+    uint32_t KB = static_cast<uint32_t>(K / 128);
+    double count = static_cast<double>(count_sz);
     const float4* W4 = reinterpret_cast<const float4*>(W);
+    QmpSlot* slots = ws->slot;
+    unsigned long long nonce = qmp_next_nonce();
     uint16_t* v16 = reinterpret_cast<uint16_t*>(vals);
     uint32_t* d32 = reinterpret_cast<uint32_t*>(dense_q);
-    const double cnt = static_cast<double>(count);
-#define SBN_QMP_LAUNCH(D, F)                                                                   \
-    mask_pack_kernel<D, F><<<static_cast<unsigned>(grid), kQmpThreads, 0, stream>>>(           \
-        W4, num_tiles, static_cast<uint32_t>(K / 128), cnt, partial, P, v16, meta, w_scale, d32, prev_meta, flip_bits)
-    if (dense_q && prev_meta) SBN_QMP_LAUNCH(true, true);
-    else if (dense_q) SBN_QMP_LAUNCH(true, false);
-    else if (prev_meta) SBN_QMP_LAUNCH(false, true);
-    else SBN_QMP_LAUNCH(false, false);
-#undef SBN_QMP_LAUNCH
+    const unsigned grid = num_units < static_cast<uint32_t>(kQmpMaxCtas) ? num_units : kQmpMaxCtas;
+    void* args[] = {&W4, &num_units, &KB, &count, &slots, &nonce, &v16, &meta, &w_scale, &d32,
+                    const_cast<uint8_t**>(&prev_meta), &flip_bits};
+    const void* fn;
+    if (dense_q && prev_meta) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<true, true>);
+    else if (dense_q) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<true, false>);
+    else if (prev_meta) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<false, true>);
+    else fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<false, false>);
+    static bool configured[4] = {false, false, false, false};
+    const int idx = (dense_q ? 2 : 0) + (prev_meta ? 1 : 0);
+    if (!configured[idx]) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kQmpSmemBytes) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        configured[idx] = true;
+    }
+    // cooperative launch: all CTAs are guaranteed to be resident together, which the exchange needs
+    if (cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kQmpThreads), args, kQmpSmemBytes, stream) != cudaSuccess)
+        return SBN_ERR_CUDA;
     ++g_launch_count;
-    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+    return SBN_OK;
 }
 
 }  // namespace sbn
