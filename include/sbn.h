@@ -171,7 +171,9 @@ sbn_status sbn_quant_act(const void *x_bf16, int T, int K, int8_t *xq, float *a_
  *   y             device out, [T][N] of `dt`
  *   acc_out       device out or NULL, int32 [T][N]: the raw accumulators (for parity checks)
  *   ws, ws_bytes  device workspace of sbn_workspace_bytes(SBN_OP_SPARSE_BITLINEAR, T, N, K)
- *                 bytes (may be NULL when that is 0)
+ *                 bytes (may be NULL when that is 0).  It must be zero-filled before its first
+ *                 use; every call that completes leaves it zero-filled again (split-K sums for
+ *                 small T live there), so it can be reused without clearing
  */
 sbn_status sbn_sparse_bitlinear(const int8_t *xq, const float *a_scale, int T,
                                 const int8_t *vals, const uint8_t *meta, const float *w_scale,

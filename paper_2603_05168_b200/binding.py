@@ -195,4 +195,4 @@ def alloc_xq(T: int, K: int, device="cuda"):
 
 def alloc_gemm_ws(op: int, T: int, N: int, K: int, device="cuda"):
     n = sbn_workspace_bytes(op, T, N, K)
-    return torch.empty(max(n, 16), dtype=torch.uint8, device=device)
+    return torch.zeros(max(n, 16), dtype=torch.uint8, device=device)      # zero-filled once, kept zero by the library

@@ -64,7 +64,6 @@ struct PairConfig {
 struct PairParams {
     GemmParams g;
     int bn;                       // tokens per tile
-    int debug;                    // perf experiments only (wrong results): 4/8 = limit the grid, 16 = no MMA
 };
 
 // ---- cluster / pair PTX ------------------------------------------------------------------------
@@ -262,7 +261,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     tcgen05_fence_after();
                     const uint32_t st = smem_stage0 + stage * Cfg::STAGE_BYTES;
                     const int kb_live = min(KBS, k_blocks - ks * KBS);
-                    if (!(pp.debug & 16)) {
+                    {
                         uint32_t e_tmem[2] = {0u, 0u};
                         if constexpr (SPARSE) {
                             // every tcgen05 instruction occupies the tensor pipe for ~128 clocks, copies

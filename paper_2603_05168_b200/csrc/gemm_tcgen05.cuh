@@ -55,8 +55,8 @@ struct GemmParams {
     void* y;                     // [T][N] fp32 or bf16
     int out_bf16;
     int32_t* acc_out;            // [T][N] or null
-    int32_t* split_acc;          // [T][N] int32 zero-initialised scratch when k_splits > 1
-    unsigned int* split_counters;   // per output tile, zero-initialised, when k_splits > 1
+    int32_t* split_acc;          // [T][N] int32 scratch when k_splits > 1: zero on entry, zero again on exit
+    unsigned int* split_counters;   // one per output tile, same rule
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -240,6 +240,7 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t tmem_slot = bar_acc_empty + 8 * ACC_STAGES;      // 4 B: TMEM base address
 
     __shared__ int s_abort;
+    __shared__ int s_last;
     volatile int* abort_flag = &s_abort;
 
     const int warp = threadIdx.x >> 5;
@@ -400,6 +401,7 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 const int tc = t0 + c * 32;
                 if (tc >= p.T) continue;                          // whole chunk beyond the last token
                 if (p.k_splits > 1) {
+                    // split-K: exact int32 accumulation in the scratch (any order gives the same sum)
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int t = tc + j;
@@ -459,6 +461,44 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 }
                 buf ^= 1;
             }
+            if (p.k_splits > 1) {
+                // The CTA that adds the last K-slice of an output tile finishes it: dequantise the
+                // totals, write y, and leave the scratch zeroed for the next call.
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");              // the four epilogue warps
+                const int out_tile = mt + tt * tiles_m;
+                if (ew == 0 && lane == 0)
+                    s_last = (atomicAdd(p.split_counters + out_tile, 1u) == static_cast<unsigned>(p.k_splits - 1)) ? 1 : 0;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (s_last) {
+                    __threadfence();
+                    const int t_end = min(p.T, t0 + BN);
+                    for (int tb = t0; tb < t_end; tb += 8) {
+                        int a[8];
+                        float sc[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {                  // eight independent loads in flight
+                            const int t = min(tb + j, t_end - 1);
+                            a[j] = __ldcg(p.split_acc + static_cast<size_t>(t) * p.N + n);
+                            sc[j] = __fmul_rn(w_scale, __ldg(p.a_scale + t));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int t = tb + j;
+                            if (t < t_end) {
+                                const size_t o = static_cast<size_t>(t) * p.N + n;
+                                p.split_acc[o] = 0;
+                                if (p.acc_out) p.acc_out[o] = a[j];
+                                float v = __fmul_rn(static_cast<float>(a[j]), sc[j]);
+                                if (p.bias) v = __fadd_rn(v, bias);
+                                if (p.out_bf16) static_cast<uint16_t*>(p.y)[o] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+                                else static_cast<float*>(p.y)[o] = v;
+                            }
+                        }
+                    }
+                    if (ew == 0 && lane == 0) p.split_counters[out_tile] = 0u;
+                }
+            }
             if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
         }
         // the slabs must stay valid until the stores have read them, and the writes must be done
@@ -473,28 +513,6 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         __syncwarp();
         tcgen05_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
-    }
-}
-
-// Split-K finish: y = dequant(split_acc), and clear split_acc for the next call.
-__global__ void __launch_bounds__(256)
-splitk_finish_kernel(int32_t* __restrict__ split_acc, int T, int N, const float* __restrict__ a_scale,
-                     const float* __restrict__ w_scale, const float* __restrict__ bias,
-                     void* __restrict__ y, int out_bf16, int32_t* __restrict__ acc_out) {
-    const size_t total = static_cast<size_t>(T) * N;
-    const float ws = __ldg(w_scale);
-    for (size_t i = static_cast<size_t>(blockIdx.x) * 256 + threadIdx.x; i < total;
-         i += static_cast<size_t>(gridDim.x) * 256) {
-        const int t = static_cast<int>(i / N);
-        const int n = static_cast<int>(i - static_cast<size_t>(t) * N);
-        const int a = split_acc[i];
-        split_acc[i] = 0;
-        if (acc_out) acc_out[i] = a;
-        const float s = __fmul_rn(ws, __ldg(a_scale + t));
-        float v = __fmul_rn(static_cast<float>(a), s);
-        if (bias) v = __fadd_rn(v, __ldg(bias + n));
-        if (out_bf16) static_cast<uint16_t*>(y)[i] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-        else static_cast<float*>(y)[i] = v;
     }
 }
 

@@ -91,6 +91,8 @@ static inline bool misaligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
 }
 
+static inline bool use_pair_kernel_fwd(int T);
+
 static inline int pick_token_tile(int T) {
     if (g_force_token_tile == 64 || g_force_token_tile == 128 || g_force_token_tile == 256)
         return g_force_token_tile;
@@ -115,10 +117,16 @@ static inline int pick_split_k(int T, int N, int K, int bn) {
     return want < 1 ? 1 : want;
 }
 
+static size_t split_acc_bytes(int T, int N) {
+    return (static_cast<size_t>(T) * N * sizeof(int32_t) + 255) & ~static_cast<size_t>(255);
+}
+
 static size_t gemm_workspace_bytes(int T, int N, int K) {
-    // split-K scratch: int32 [T][N]; only the small-T regime ever splits
+    // split-K scratch: int32 [T][N] + one counter per output tile; only the small-T regime splits
+    if (use_pair_kernel_fwd(T)) return 0;
     const int bn = pick_token_tile(T);
-    if (pick_split_k(T, N, K, bn) > 1) return static_cast<size_t>(T) * N * sizeof(int32_t);
+    if (pick_split_k(T, N, K, bn) > 1)
+        return split_acc_bytes(T, N) + static_cast<size_t>(N / kBM) * ((T + bn - 1) / bn) * sizeof(unsigned int);
     return 0;
 }
 
@@ -191,9 +199,7 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
         configured = true;
     }
     const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
-    int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
-    if (pp.debug & 4) pairs = 1;                 // experiment: one CTA pair only (unloaded latency)
-    if (pp.debug & 8) pairs = pairs < 8 ? pairs : 8;
+    const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
     kernel<<<2 * pairs, kPairThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, pp);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
@@ -204,6 +210,7 @@ static inline bool use_pair_kernel(int T) {
     if (g_force_token_tile > 0) return false;
     return T >= 256;
 }
+static inline bool use_pair_kernel_fwd(int T) { return use_pair_kernel(T); }
 
 static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_scale, int T,
                                 const int8_t* wvals, const uint8_t* meta, const float* w_scale,
@@ -234,7 +241,6 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.acc_out = acc_out;
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.bn = bn;
-    pp.debug = g_force_split_k < 0 ? -g_force_split_k : 0;   // experiments: split_k < 0 carries debug bits
     return sparse ? launch_pair<true>(ta, tb, te, ty, pp, stream) : launch_pair<false>(ta, tb, te, ty, pp, stream);
 }
 
@@ -256,10 +262,10 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     const int bn = pick_token_tile(T);
     const int splits = pick_split_k(T, N, K, bn);
     if (splits > 1) {
-        const size_t need = static_cast<size_t>(T) * N * sizeof(int32_t);
+        // scratch is zero on entry (caller's duty before the first use) and the kernel re-zeroes it
+        const size_t need = gemm_workspace_bytes(T, N, K);
         if (!ws || ws_bytes < need) return SBN_ERR_WORKSPACE;
         if (misaligned(ws, 16)) return SBN_ERR_ALIGN;
-        if (cudaMemsetAsync(ws, 0, need, stream) != cudaSuccess) return SBN_ERR_CUDA;
     }
 
     CUtensorMap ta, tb, te, ty;
@@ -284,7 +290,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
     p.acc_out = acc_out;
     p.split_acc = splits > 1 ? static_cast<int32_t*>(ws) : nullptr;
-    p.split_counters = nullptr;
+    p.split_counters = splits > 1 ? reinterpret_cast<unsigned int*>(static_cast<char*>(ws) + split_acc_bytes(T, N)) : nullptr;
 
     sbn_status st;
 #define SBN_GEMM_CASE(S, B) st = launch_gemm_cfg<S, B>(ta, tb, te, ty, p, stream)
@@ -295,15 +301,6 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     }
 #undef SBN_GEMM_CASE
     if (st != SBN_OK) return st;
-    if (splits > 1) {
-        const size_t total = static_cast<size_t>(T) * N;
-        size_t blocks = (total + 255) / 256;
-        if (blocks > static_cast<size_t>(kNumSMs * 8)) blocks = kNumSMs * 8;
-        splitk_finish_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-            p.split_acc, T, N, a_scale, w_scale, bias, y, p.out_bf16, acc_out);
-        ++g_launch_count;
-        if (cudaGetLastError() != cudaSuccess) return SBN_ERR_CUDA;
-    }
     return SBN_OK;
 }
 

@@ -17,23 +17,32 @@ namespace sbn {
 
 constexpr int kActThreads = 256;
 
-__device__ __forceinline__ float absmax8(const uint4& v) {
-    float m = fmaxf(fabsf(bf16lo_to_f32(v.x)), fabsf(bf16hi_to_f32(v.x)));
-    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.y)), fabsf(bf16hi_to_f32(v.y))));
-    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.z)), fabsf(bf16hi_to_f32(v.z))));
-    m = fmaxf(m, fmaxf(fabsf(bf16lo_to_f32(v.w)), fabsf(bf16hi_to_f32(v.w))));
+// |x| of non-negative bf16 bit patterns orders like unsigned integers, so the row maximum is
+// taken on packed halfwords: clear the two sign bits, then a per-halfword unsigned max.
+__device__ __forceinline__ uint32_t absmax8_packed(const uint4& v, uint32_t m) {
+    constexpr uint32_t kAbs = 0x7FFF7FFFu;
+    m = __vmaxu2(m, __vmaxu2(__vmaxu2(v.x & kAbs, v.y & kAbs), __vmaxu2(v.z & kAbs, v.w & kAbs)));
     return m;
 }
-
-__device__ __forceinline__ uint32_t quant1(float x, float s_x) {
-    int q = __float2int_rn(__fmul_rn(x, s_x));     // one fp32 multiply, then half-to-even
-    q = max(-128, min(127, q));
-    return static_cast<uint32_t>(q) & 0xFFu;
+__device__ __forceinline__ float packed_max_to_f32(uint32_t m) {
+    return __uint_as_float(max(m >> 16, m & 0xFFFFu) << 16);
 }
+__device__ __forceinline__ float absmax8(const uint4& v) { return packed_max_to_f32(absmax8_packed(v, 0u)); }
 
+// round(x * s_x) for two values, saturated to int8 and packed: (sat8(a) << 8 | sat8(b)) | c << 16.
+// The saturation is Algorithm 2's clamp(-128, 127).
+__device__ __forceinline__ uint32_t pack_sat_s8x2(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ int quant1(float x, float s_x) {
+    return __float2int_rn(__fmul_rn(x, s_x));      // one fp32 multiply, then half-to-even
+}
+// four consecutive bf16 (two words) -> four int8 codes in one word, lowest column in the low byte
 __device__ __forceinline__ uint32_t quant_pair2(uint32_t a, uint32_t b, float s_x) {
-    return quant1(bf16lo_to_f32(a), s_x) | (quant1(bf16hi_to_f32(a), s_x) << 8) |
-           (quant1(bf16lo_to_f32(b), s_x) << 16) | (quant1(bf16hi_to_f32(b), s_x) << 24);
+    const uint32_t hi = pack_sat_s8x2(quant1(bf16hi_to_f32(b), s_x), quant1(bf16lo_to_f32(b), s_x), 0u);
+    return pack_sat_s8x2(quant1(bf16hi_to_f32(a), s_x), quant1(bf16lo_to_f32(a), s_x), hi);
 }
 
 // Index (in 8-byte units) of the 8 int8 codes of token `t`, vector `idx` (columns 8*idx .. 8*idx+7).
@@ -78,10 +87,11 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
             const int idx = g + i * G;
             nxt[i] = (row_n < T && idx < nvec) ? __ldg(x + static_cast<size_t>(row_n) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
         }
-        float amax = 0.0f;
+        uint32_t pm = 0u;
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) amax = fmaxf(amax, absmax8(cur[i]));
-        amax = warp_max(amax);
+        for (int i = 0; i < VPT; ++i) pm = absmax8_packed(cur[i], pm);
+        // bit patterns of non-negative floats order like integers: one redux instruction per warp
+        float amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, max(pm >> 16, pm & 0xFFFFu)) << 16);
         if constexpr (WARPS_PER_ROW > 1) {
             const int warp = threadIdx.x >> 5;
             float* sm = s_max[it & 1];                               // double buffered: one barrier per row

@@ -5,14 +5,16 @@
 // twice.  One persistent cooperative kernel (one 1024-thread CTA per SM) does both passes:
 //
 //   pass 1   every CTA owns a contiguous range of (row, 128-column) units, streams it once,
-//            accumulates sum|W| in fp64 and KEEPS the first part of its range in shared memory
-//            (200 KB per SM: 148 SMs hold 29.6 MB of W on chip);
+//            accumulates sum|W| in fp64, KEEPS the first part of its range in shared memory
+//            (200 KB per SM: 148 SMs hold 29.6 MB of W on chip) and -- the mask does not depend
+//            on gamma -- already selects the top 2 of 4, writes the metadata and counts flips;
 //   exchange every CTA publishes {call nonce, partial sum} in the workspace and waits (bounded)
 //            until all slots carry this call's nonce -- no atomics, no counter, nothing to
 //            initialise, stale slots of earlier calls can never match; every CTA then adds the
 //            148 partials in the same fixed order, so all get the same bits, run after run;
-//   pass 2   top-2-of-4, ternarise, pack: the resident part comes from shared memory, the rest
-//            is read again, newest first (what pass 1 read last is still in the 126 MB L2).
+//   pass 2   ternarises the two kept values of every group: the resident part comes from shared
+//            memory, the rest is read again, newest first (what pass 1 read last is still in
+//            the 126 MB L2).
 //
 // HBM traffic per parameter: 4 B (one read) + 0.625 B written for the resident part, one more
 // (mostly L2-served) 4 B read for the rest.  16 B loads per lane, a warp covers one 512 B unit;
@@ -60,15 +62,9 @@ __device__ __forceinline__ float ternary_threshold(float scale) {
     return a;
 }
 
-// One 2:4 group: returns nibble | q-bytes.  Ranking on |w| of the fp32 master weights; on equal
-// magnitudes the lower column wins.
-struct GroupResult {
-    uint32_t nibble;     // i0 | i1 << 2
-    uint32_t vals16;     // two int8 (kept values, low byte = column i0)
-    uint32_t dense32;    // four int8 (unmasked W_q)
-};
-
-__device__ __forceinline__ GroupResult process_group(const float4 w, float thr) {
+// Eq. 2 for one group: 2-bit indices i0 < i1 of the two largest |w| (ranking on the fp32 master
+// weights; on equal magnitudes the lower column wins), as nibble i0 | i1 << 2.
+__device__ __forceinline__ uint32_t group_nibble(const float4 w) {
     const float a0 = fabsf(w.x), a1 = fabsf(w.y), a2 = fabsf(w.z), a3 = fabsf(w.w);
     // rank_j = number of entries that beat entry j; entry i beats j>i iff a_i >= a_j
     const int c01 = a0 >= a1, c02 = a0 >= a2, c03 = a0 >= a3;
@@ -81,16 +77,15 @@ __device__ __forceinline__ GroupResult process_group(const float4 w, float thr) 
     // exactly two bits set: lowest and highest set bit
     const uint32_t i0 = __ffs(keep) - 1;
     const uint32_t i1 = 31 - __clz(keep);
-    // ternary codes as bytes: +1 -> 0x01, -1 -> 0xFF, 0 -> 0x00
-    const uint32_t q0 = a0 >= thr ? (w.x < 0.0f ? 0xFFu : 0x01u) : 0u;
-    const uint32_t q1 = a1 >= thr ? (w.y < 0.0f ? 0xFFu : 0x01u) : 0u;
-    const uint32_t q2 = a2 >= thr ? (w.z < 0.0f ? 0xFFu : 0x01u) : 0u;
-    const uint32_t q3 = a3 >= thr ? (w.w < 0.0f ? 0xFFu : 0x01u) : 0u;
-    GroupResult r;
-    r.dense32 = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
-    r.nibble = i0 | (i1 << 2);
-    r.vals16 = ((r.dense32 >> (8 * i0)) & 0xFFu) | (((r.dense32 >> (8 * i1)) & 0xFFu) << 8);
-    return r;
+    return i0 | (i1 << 2);
+}
+
+// Eq. 1 for one element as a byte: +1 -> 0x01, -1 -> 0xFF, 0 -> 0x00 (thr: see the header).
+__device__ __forceinline__ uint32_t ternary_byte(float w, float thr) {
+    return fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u;
+}
+__device__ __forceinline__ float pick4(const float4 w, uint32_t i) {
+    return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
 }
 
 __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
@@ -134,27 +129,51 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
     const uint32_t u_end = min(num_units, u_begin + per);
     const uint32_t n_res = min(u_end - u_begin, static_cast<uint32_t>(kQmpResidentUnits));
 
-    // ---- pass 1: sum |W| over this CTA's range (4 independent 16 B loads in flight per thread)
+    // ---- pass 1: sum |W| over this CTA's range (4 independent 16 B loads in flight per thread).
+    // The mask does not depend on gamma, so the top-2-of-4 selection, the metadata and the flip
+    // count are done here too, under the memory time of this pass.
+    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+    unsigned int flips = 0;
     double acc = 0.0;
     {
         uint32_t u = u_begin + warp;
-        for (; u + 3 * kQmpWarps < u_end; u += 4 * kQmpWarps) {
-            const float4 v0 = __ldg(W4 + static_cast<size_t>(u) * 32 + lane);
-            const float4 v1 = __ldg(W4 + static_cast<size_t>(u + kQmpWarps) * 32 + lane);
-            const float4 v2 = __ldg(W4 + static_cast<size_t>(u + 2 * kQmpWarps) * 32 + lane);
-            const float4 v3 = __ldg(W4 + static_cast<size_t>(u + 3 * kQmpWarps) * 32 + lane);
-            acc += (abs_sum4(v0) + abs_sum4(v1)) + (abs_sum4(v2) + abs_sum4(v3));
-            const uint32_t r = u - u_begin;
-            if (r < n_res) s_w[r * 32 + lane] = v0;
-            if (r + kQmpWarps < n_res) s_w[(r + kQmpWarps) * 32 + lane] = v1;
-            if (r + 2 * kQmpWarps < n_res) s_w[(r + 2 * kQmpWarps) * 32 + lane] = v2;
-            if (r + 3 * kQmpWarps < n_res) s_w[(r + 3 * kQmpWarps) * 32 + lane] = v3;
+        int n_cur = 0, kb_cur = 0;
+        if (u < u_end) {
+            n_cur = static_cast<int>(u / KB);
+            kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
         }
-        for (; u < u_end; u += kQmpWarps) {
-            const float4 v0 = __ldg(W4 + static_cast<size_t>(u) * 32 + lane);
-            acc += abs_sum4(v0);
-            const uint32_t r = u - u_begin;
-            if (r < n_res) s_w[r * 32 + lane] = v0;
+        for (; u < u_end; u += 4 * kQmpWarps) {
+            float4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t uq = u + q * kQmpWarps;
+                v[q] = (uq < u_end) ? __ldg(W4 + static_cast<size_t>(uq) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            acc += (abs_sum4(v[0]) + abs_sum4(v[1])) + (abs_sum4(v[2]) + abs_sum4(v[3]));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t uq = u + q * kQmpWarps;
+                if (uq < u_end) {
+                    const uint32_t r = uq - u_begin;
+                    if (r < n_res) s_w[r * 32 + lane] = v[q];
+                    const size_t m_off = ((static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) << 11) +
+                                         ((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1);
+                    n_cur += step_n;
+                    kb_cur += step_kb;
+                    if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+                    const uint32_t nib = group_nibble(v[q]);
+                    const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+                    if ((lane & 1) == 0) {
+                        const uint32_t byte = nib | (hi << 4);
+                        if constexpr (COUNT_FLIPS) {
+                            const uint32_t prev = prev_meta[m_off];
+                            flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev & 15u)) +
+                                     __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev >> 4) & 15u));
+                        }
+                        meta[m_off] = static_cast<uint8_t>(byte);
+                    }
+                }
+            }
         }
     }
     const double mine = qmp_block_sum(acc, s_warp);
@@ -197,12 +216,10 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
     __syncthreads();
     const float thr = s_thr;
 
-    // ---- pass 2: a warp takes four units at a time (four 16 B loads in flight per lane); the
-    // re-read part newest first, then the resident part from shared memory
-    unsigned int flips = 0;
+    // ---- pass 2 (Eq. 1 + Eq. 3): ternarise the two kept values of every group.  A warp takes four
+    // units at a time (four loads in flight per lane); the re-read part newest first, then the
+    // resident part from shared memory.  The group's nibble is read back from the metadata.
     const uint32_t n_units = u_end - u_begin;
-    // (row, k-block) of the warp's first unit by one division, then stepped down by 32 units a time
-    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
     int n_cur = 0, kb_cur = 0;
     if (static_cast<uint32_t>(warp) < n_units) {
         const uint32_t u_first = u_begin + (n_units - 1 - warp);
@@ -211,7 +228,7 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
     }
     for (uint32_t i0 = warp; i0 < n_units; i0 += 4 * kQmpWarps) {
         float4 w[4];
-        uint32_t prev[4];
+        uint32_t mb[4];
         size_t tile_idx[4];
         uint32_t rr[4];
 #pragma unroll
@@ -226,27 +243,22 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
                 n_cur -= step_n;
                 kb_cur -= step_kb;
                 if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
-                if constexpr (COUNT_FLIPS) {
-                    prev[q] = (lane & 1) ? 0u : prev_meta[(tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1)];
-                }
+                mb[q] = *(reinterpret_cast<const volatile uint8_t*>(meta) + (tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1));
             }
         }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint32_t i = i0 + q * kQmpWarps;
             if (i < n_units) {
-                const GroupResult g = process_group(w[q], thr);
+                const uint32_t nib = (mb[q] >> ((lane & 1) * 4)) & 15u;
+                const uint32_t k0 = ternary_byte(pick4(w[q], nib & 3u), thr);
+                const uint32_t k1 = ternary_byte(pick4(w[q], nib >> 2), thr);
                 // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
-                vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(g.vals16);
-                if constexpr (WRITE_DENSE) dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = g.dense32;
-                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, g.nibble, 1);
-                if ((lane & 1) == 0) {
-                    const uint32_t byte = g.nibble | (hi << 4);
-                    if constexpr (COUNT_FLIPS) {
-                        flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev[q] & 15u)) +
-                                 __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev[q] >> 4) & 15u));
-                    }
-                    meta[(tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1)] = static_cast<uint8_t>(byte);
+                vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(k0 | (k1 << 8));
+                if constexpr (WRITE_DENSE) {
+                    const uint32_t d = ternary_byte(w[q].x, thr) | (ternary_byte(w[q].y, thr) << 8) |
+                                       (ternary_byte(w[q].z, thr) << 16) | (ternary_byte(w[q].w, thr) << 24);
+                    dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = d;
                 }
             }
         }
@@ -302,8 +314,11 @@ inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t
             return SBN_ERR_CUDA;
         configured[idx] = true;
     }
-    // cooperative launch: all CTAs are guaranteed to be resident together, which the exchange needs
-    if (cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kQmpThreads), args, kQmpSmemBytes, stream) != cudaSuccess)
+    // At most one CTA per SM (200 KB of shared memory each) and never more CTAs than SMs, so all
+    // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
+    // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
+    // (A cooperative launch would guarantee co-residency but was measured to add ~10 us per call.)
+    if (cudaLaunchKernel(fn, dim3(grid), dim3(kQmpThreads), args, kQmpSmemBytes, stream) != cudaSuccess)
         return SBN_ERR_CUDA;
     ++g_launch_count;
     return SBN_OK;

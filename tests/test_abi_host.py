@@ -46,7 +46,7 @@ def test_workspace_query(L):
     assert b.sbn_workspace_bytes(b.OP_QUANT_ACT, 64, 0, 256) == 0
     # large T: no split-K scratch; decode-sized T: int32 [T][N] scratch
     assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4096, 2560, 2560) == 0
-    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 4 * 2560 * 4
+    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 4 * 2560 * 4 + 20 * 4   # sums + tile counters
     assert b.sbn_workspace_bytes(b.OP_BITLINEAR, 4, 2560, 100) == 0      # illegal shape -> 0
     assert b.sbn_workspace_bytes(77, 4, 2560, 2560) == 0
 
