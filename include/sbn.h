@@ -215,7 +215,7 @@ const char *sbn_status_string(sbn_status s);
 
 /* Tuning/diagnostic knob (host state, not thread-safe).  token_tile: 0 = automatic; 64, 128 or
  * 256 = force the single-CTA kernel with that token-tile width; a negative value -BN = force the
- * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 32, capped at 224 sparse /
+ * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
  * 256 dense).  split_k: split-K factor of the single-CTA kernel (0 = automatic).  Results do not
  * depend on it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);

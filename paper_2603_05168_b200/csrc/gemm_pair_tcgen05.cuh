@@ -12,13 +12,13 @@
 // stage, both of a CTA's weight tiles (and likewise both metadata tiles, and the activation
 // atoms) for KBS consecutive 128-column blocks: three instructions per stage (sparse).
 //
-//   pair tile      512 output features x BN tokens (BN runtime, multiple of 32, <= 224 sparse /
+//   pair tile      512 output features x BN tokens (BN runtime, multiple of 16, <= 240 sparse /
 //                  256 dense).  CTA r of the pair owns the weight row blocks 4*mt + 2r + i
 //                  (i = 0, 1 = the M-tile); a row block beyond N is skipped.
 //   per CTA smem   per stage: A[2 row blocks][KBS] (8 KB sparse | 16 KB dense each),
 //                  E[2][KBS] (2 KB each, sparse), B[KBS] (BN/2 rows x 128 B); KBS = 2 (sparse), 1
-//   TMEM           M-tile i accumulates in columns [256 i, 256 i + BN); metadata slots in columns
-//                  [256 i + 224, 256 i + 256).  Accumulators are single-buffered: the MMA of the
+//   TMEM           M-tile i accumulates in columns [256 i, 256 i + BN); metadata slots (8 columns
+//                  each, 2 or 4 of them) at the top of the same 256-column half.  Accumulators are single-buffered: the MMA of the
 //                  next tile waits until the epilogue has drained TMEM into registers.
 //   warps          0 TMA producer (both CTAs), 1 MMA issuer (leader CTA only; both allocate
 //                  TMEM), 2..9 epilogue: warps 2-5 drain M-tile 0, warps 6-9 M-tile 1
@@ -39,7 +39,7 @@ constexpr int kPairThreads = 320;
 constexpr int kPairEpiWarps = 8;
 constexpr int kPairSlabBytes = 2048;                              // 32 tok x 32 feat bf16 | 16 tok fp32
 constexpr int kPairEpiBytes = kPairEpiWarps * kPairSlabBytes;     // one slab per epilogue warp
-constexpr int kPairMaxBnSparse = 224;
+constexpr int kPairMaxBnSparse = 240;
 constexpr int kPairMaxBnDense = 256;
 
 template <bool SPARSE>
@@ -53,8 +53,9 @@ struct PairConfig {
     static constexpr int E_BYTES = 2 * KBS * E_TILE;
     static constexpr int B_BYTES = KBS * B_TILE;
     static constexpr int STAGE_BYTES = A_BYTES + E_BYTES + B_BYTES;
-    static constexpr int STAGES = (232448 - 1024 - kPairEpiBytes - kBarrierBytes) / STAGE_BYTES;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + kPairEpiBytes + kBarrierBytes;
+    // the kernel has no static shared memory, so the dynamic part starts 1 KB-aligned (checked)
+    static constexpr int STAGES = (232448 - kPairEpiBytes - kBarrierBytes) / STAGE_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + kPairEpiBytes + kBarrierBytes;
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1 KB alignment");
     static_assert(STAGES >= 3, "not enough stages");
     static_assert(!SPARSE || KBS == 2, "the 128x256b metadata copy covers exactly two k-blocks");
@@ -161,7 +162,11 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int half_bn = BN >> 1;
 
     extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_base = smem_u32(smem_raw);
+    if (smem_base & 1023u) {          // swizzled tiles need 1 KB alignment; identical in every CTA
+        if (threadIdx.x == 0) atomicExch(&g_device_status, static_cast<int>(SBN_ERR_CUDA));
+        return;
+    }
     // per stage: A [row block i][k-block j] | E [i][j] | B [j]
     const uint32_t smem_stage0 = smem_base;
     const uint32_t smem_epi = smem_base + STAGES * Cfg::STAGE_BYTES;
@@ -171,9 +176,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t bar_acc_full = bar_empty + 8 * STAGES;
     const uint32_t bar_acc_empty = bar_acc_full + 8;
     const uint32_t tmem_slot = bar_acc_empty + 8;
-
-    __shared__ int s_abort;
-    volatile int* abort_flag = &s_abort;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (tmem_slot + 8 - smem_base));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -189,7 +192,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int k_stages = (k_blocks + KBS - 1) / KBS;      // pipeline stages per tile
 
     if (threadIdx.x == 0) {
-        s_abort = 0;
+        *abort_flag = 0;
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
@@ -248,6 +251,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             uint32_t phase = 0;
             uint32_t acc_phase = 0;
             uint32_t e_slot = 0;
+            const uint32_t e_slots = BN <= 224 ? 4u : 2u;              // 8-column metadata slots above the accumulator
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int mt = tile % tiles_m;
@@ -268,7 +272,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                             // included: one 128x256b copy brings the metadata of BOTH k-blocks of the
                             // stage (two 2 KB tiles, 2 KB apart) for an M-tile
                             for (int i = 0; i < mt_count; ++i) {
-                                e_tmem[i] = tmem_base + static_cast<uint32_t>(i * 256 + 224 + 8 * (e_slot & 3u));
+                                e_tmem[i] = tmem_base + static_cast<uint32_t>(i * 256 + 256 - 8 * e_slots + 8 * (e_slot % e_slots));
                                 const uint64_t e_desc = make_smem_desc(st + Cfg::A_BYTES + static_cast<uint32_t>(i * KBS * Cfg::E_TILE),
                                                                        Cfg::E_TILE, 128, kSwzNone);
                                 tcgen05_cp_128x256b_pair(e_tmem[i], e_desc);
@@ -329,7 +333,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const uint32_t slab_u32 = smem_epi + static_cast<uint32_t>(ew * kPairSlabBytes);
         uint8_t* const slab_ptr = smem_raw + (slab_u32 - smem_u32(smem_raw));
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
-        const int chunks = BN >> 5;                       // 32-column chunks (BN % 32 == 0)
+        const int chunks = (BN + 31) >> 5;                // 32-column chunks; the last one may be 16 wide
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
@@ -351,16 +355,26 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tcgen05_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(mtile * 256);
             // number of chunks that hold at least one real token (warp-uniform)
-            const int live = rows_valid ? (min(p.T - t0, BN) + 31) >> 5 : 0;
+            const int live = rows_valid ? (min(p.T - t0, BN) + 31) >> 5 : 0;      // <= chunks
+            // a 16-wide last chunk (BN % 32 == 16) is read with a 16-column load: the columns above
+            // it hold metadata; its 16 tokens go out with plain stores (bf16) / one 16-token slab
+            const int full32 = BN >> 5;
             uint32_t ra[32], rb[32];
-            if (live > 0) tmem_ld_32x32b_x32(t_addr, ra);
+            if (live > 0) {
+                if (full32 > 0) tmem_ld_32x32b_x32(t_addr, ra);
+                else tmem_ld_32x32b_x16(t_addr, reinterpret_cast<uint32_t (&)[16]>(ra));
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 if (i < live) {
                     uint32_t (&cur)[32] = (i & 1) ? rb : ra;
                     uint32_t (&nxt)[32] = (i & 1) ? ra : rb;
+                    const bool half_chunk = (i == full32);                 // the 16-wide tail
                     tmem_ld_wait();                                       // chunk i is in registers
-                    if (i + 1 < live) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>((i + 1) * 32), nxt);
+                    if (i + 1 < live) {
+                        if (i + 1 < full32) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>((i + 1) * 32), nxt);
+                        else tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>((i + 1) * 32), reinterpret_cast<uint32_t (&)[16]>(nxt));
+                    }
                     if (i + 1 == live) {
                         // last TMEM read of this warp is complete: hand the accumulator back
                         tcgen05_fence_before();
@@ -368,14 +382,25 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                         if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
                     }
                     const int tc = t0 + i * 32;
+                    const int t_lim = min(p.T, tc + (half_chunk ? 16 : 32));  // tokens of this chunk end here
                     if (p.acc_out) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
                             const int t = tc + j;
-                            if (t < p.T) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(cur[j]);
+                            if (t < t_lim) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(cur[j]);
                         }
                     }
-                    if (p.out_bf16) {
+                    if (p.out_bf16 && half_chunk) {
+                        // 16-token tail: plain 2-byte stores, 64 contiguous bytes per warp and token
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float sc = __shfl_sync(0xFFFFFFFFu, my_scale[i], j);
+                            float v = __fmul_rn(static_cast<float>(static_cast<int>(cur[j])), sc);
+                            if (p.bias) v = __fadd_rn(v, bias);
+                            const int t = tc + j;
+                            if (t < t_lim) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+                        }
+                    } else if (p.out_bf16) {
                         // convert in registers (two tokens per word), then one 32 x 32 bf16 slab
                         uint32_t packed[16];
 #pragma unroll
@@ -406,7 +431,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                         // two 16-token x 32-feature fp32 slabs through the same 2 KB buffer
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            if (tc + h * 16 < p.T) {
+                            if (tc + h * 16 < t_lim) {
                                 float v[16];
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) {

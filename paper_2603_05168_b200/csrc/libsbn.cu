@@ -155,7 +155,7 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
     if (g_force_token_tile < 0) {
         int bn = -g_force_token_tile;
         const int cap = sparse ? kPairMaxBnSparse : kPairMaxBnDense;
-        bn = (bn / 32) * 32;
+        bn = (bn / 16) * 16;
         if (bn < 32) bn = 32;
         if (bn > cap) bn = cap;
         return bn;
@@ -166,7 +166,7 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
     const int full_m = N / 512, rem_m = (N % 512) ? 1 : 0;
     int best = 128;
     double best_cost = 1e300;
-    for (int bn = 64; bn <= cap; bn += 32) {
+    for (int bn = 64; bn <= cap; bn += 16) {
         const int tt = (T + bn - 1) / bn;
         auto tile_clk = [&](int mtiles) {
             const double a_bytes = sparse ? 72.0 : 128.0;

@@ -196,7 +196,8 @@ def test_gemm_parity_every_token_tile(sparse, tile):
 
 PAIR_CASES = [  # (T, N, K, BN): CTA-pair kernel, forced tile widths incl. ragged T and odd N/128
     (333, 128, 256, 64), (333, 256, 128, 32), (40, 384, 512, 32), (500, 640, 384, 160),
-    (700, 1024, 1280, 224), (257, 1152, 2560, 96), (1000, 512, 6912, 224), (530, 256, 256, 256),
+    (700, 1024, 1280, 224), (257, 1152, 2560, 96), (1000, 512, 6912, 240), (530, 256, 256, 256),
+    (490, 384, 640, 240), (300, 256, 384, 48), (241, 512, 256, 240), (1000, 640, 512, 176),
 ]
 
 
