@@ -59,6 +59,22 @@ def load_peaks():
                 bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def max_over_ranks(ms_local, world, dist=None, device="cpu"):
+    """Replicas only: every rank runs the same work on its own GPU, nothing is exchanged on the data
+    path; the job's step time is the slowest rank's device time."""
+    if world <= 1:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ops_per_replica, world, ms_per_step):
+    """Units processed by all ranks divided by the (max over ranks) step time."""
+    return ops_per_replica * world / (ms_per_step * 1e-3) / 1e12
+
+
 def step_ops(T, shapes=inputs.SHAPES_2B):
     return sum(2.0 * T * N * K for _, K, N in shapes)
 
@@ -282,12 +298,9 @@ def run_ours(args):
     launches = b.sbn_launch_count() - launches0
     b.sbn_check_status()
     ms_total = sum(a_ev.elapsed_time(c_ev) for a_ev, c_ev in chunk_times)
-    if world > 1:
-        tt = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = step_ops(T, shapes) * world / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(step_ops(T, shapes), world, ms_per_step)
 
     per_kernel = {k: {} for k in KERNELS}
     for name, e in evs:
@@ -325,13 +338,8 @@ def run_ours(args):
     e2.record(stream)
     barrier()
     b.sbn_check_status()
-    e2e_ms = s2.elapsed_time(e2)
-    if world > 1:
-        tt = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_ms /= e2e_steps
-    e2e_value = step_ops(T, shapes) * world / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(s2.elapsed_time(e2), world, dist, "cuda") / e2e_steps
+    e2e_value = whole_job_tops(step_ops(T, shapes), world, e2e_ms)
     h2d = sum(L.W_host.numel() * 4 + L.x_host.numel() * 2 for L in layers)
     d2h = sum(L.y_host.numel() * 2 for L in layers)
 
