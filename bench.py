@@ -549,18 +549,28 @@ def run_dynamic_step(args):
     ys = {N: torch.empty((T, N), dtype=torch.bfloat16, device="cuda") for N in sorted({N for _, _, N in inputs.LAYER_2B})}
     params = sum(K * N for _, K, N, _, _ in mats)
 
+    # one batched launch per step; two job arrays because prev/current metadata swap every step
+    job_ws = torch.empty(b.sbn_batch_workspace_bytes(len(mats)), dtype=torch.uint8, device="cuda")
+    plain_jobs = b.make_pack_jobs([dict(W=W, vals=p["vals"], meta=p["meta"], w_scale=p["w_scale"]) for _, _, _, W, p in mats])
+    flip_jobs = [b.make_pack_jobs([dict(W=W, vals=p["vals"], meta=p["meta"] if par == 0 else p["prev"], w_scale=p["w_scale"],
+                                        prev_meta=p["prev"] if par == 0 else p["meta"], flip_bits=p["flips"])
+                                   for _, _, _, W, p in mats]) for par in (0, 1)]
+    state = {"par": 1}            # after the plain pack the current metadata is in p["meta"]
+
     def repack(with_flips):
-        for _, K, N, W, p in mats:
-            if with_flips:
-                p["prev"], p["meta"] = p["meta"], p["prev"]
-                b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"], prev_meta=p["prev"], flip_bits=p["flips"])
-            else:
-                b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"])
+        if not with_flips:
+            b.sbn_quantize_mask_pack_batched(plain_jobs, job_ws)
+            return
+        b.sbn_quantize_mask_pack_batched(flip_jobs[state["par"]], job_ws)
+        state["par"] ^= 1
+
+    def cur_meta(p):
+        return p["meta"] if state["par"] == 1 else p["prev"]
 
     def forward():
         for _, K, N, W, p in mats:
             xq, a_scale = acts[K]
-            b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], ys[N])
+            b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], cur_meta(p), p["w_scale"], ys[N])
 
     repack(False)
     forward()

@@ -116,6 +116,28 @@ sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int 
                                   void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Part 1 for many matrices in ONE launch -- the dynamic-mask training step recomputes the mask of
+ * every BitLinear at every step (Sec. 2.3, "Dynamic Mask Recomputation"; Algorithm 1).  Each job
+ * is exactly one sbn_quantize_mask_pack call (same arguments, same results, bit for bit); the
+ * kernel pipelines the jobs so that launch and exchange latencies are paid once per batch.
+ *   jobs   host array of `count` jobs (read before the call returns)
+ *   ws     device workspace of sbn_batch_workspace_bytes(count) bytes; no initialisation needed
+ */
+typedef struct {
+    const float *W;                   /* device, fp32 [N][K] */
+    int N, K;
+    int8_t *vals;                     /* device out, tiled */
+    uint8_t *meta;                    /* device out, tiled; may equal prev_meta */
+    float *w_scale;                   /* device out, one fp32 */
+    int8_t *dense_q;                  /* device out or NULL */
+    const uint8_t *prev_meta;         /* device or NULL */
+    unsigned long long *flip_bits;    /* device out; required iff prev_meta != NULL */
+} sbn_pack_job;
+size_t sbn_batch_workspace_bytes(int count);
+sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job *jobs, void *ws, size_t ws_bytes,
+                                          void *stream);
+
+/*
  * Same operation as sbn_quantize_mask_pack, for callers that have no workspace to give.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)
  *

@@ -21,7 +21,8 @@ OUT_F32, OUT_BF16 = 0, 1
 OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
 
 EXPORTS = [
-    "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quant_act", "sbn_sparse_bitlinear",
+    "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
+    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -53,6 +54,10 @@ def lib() -> ctypes.CDLL:
         L.sbn_quantize_mask_pack.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.sbn_quantize_mask_pack_static_ws.restype = i32
         L.sbn_quantize_mask_pack_static_ws.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.sbn_batch_workspace_bytes.restype = sz
+        L.sbn_batch_workspace_bytes.argtypes = [i32]
+        L.sbn_quantize_mask_pack_batched.restype = i32
+        L.sbn_quantize_mask_pack_batched.argtypes = [i32, vp, vp, sz, vp]
         L.sbn_quant_act.restype = i32
         L.sbn_quant_act.argtypes = [vp, i32, i32, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
@@ -116,6 +121,37 @@ def sbn_quantize_mask_pack_static_ws(W, vals, meta, w_scale, dense_q=None, prev_
                                                   _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta),
                                                   _ptr(flip_bits), _stream()),
            "sbn_quantize_mask_pack_static_ws")
+
+
+class PackJob(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("N", ctypes.c_int), ("K", ctypes.c_int), ("vals", ctypes.c_void_p),
+                ("meta", ctypes.c_void_p), ("w_scale", ctypes.c_void_p), ("dense_q", ctypes.c_void_p),
+                ("prev_meta", ctypes.c_void_p), ("flip_bits", ctypes.c_void_p)]
+
+
+def sbn_batch_workspace_bytes(count: int) -> int:
+    return int(lib().sbn_batch_workspace_bytes(int(count)))
+
+
+def make_pack_jobs(jobs):
+    """jobs: list of dicts with W, vals, meta, w_scale and optionally dense_q, prev_meta, flip_bits
+    (torch CUDA tensors).  Returns the ctypes array to hand to sbn_quantize_mask_pack_batched; it can
+    be reused every step as long as the tensors stay where they are."""
+    arr = (PackJob * len(jobs))()
+    for a, j in zip(arr, jobs):
+        N, K = j["W"].shape
+        a.W, a.N, a.K = j["W"].data_ptr(), N, K
+        a.vals, a.meta, a.w_scale = j["vals"].data_ptr(), j["meta"].data_ptr(), j["w_scale"].data_ptr()
+        for key in ("dense_q", "prev_meta", "flip_bits"):
+            t = j.get(key)
+            setattr(a, key, t.data_ptr() if t is not None else None)
+    return arr
+
+
+def sbn_quantize_mask_pack_batched(job_array, ws):
+    _check(lib().sbn_quantize_mask_pack_batched(len(job_array), ctypes.cast(job_array, ctypes.c_void_p), _ptr(ws),
+                                                ws.numel() * ws.element_size(), _stream()),
+           "sbn_quantize_mask_pack_batched")
 
 
 def sbn_quant_act(x_bf16, xq, a_scale):

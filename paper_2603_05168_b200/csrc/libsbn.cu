@@ -7,6 +7,7 @@
 #include <algorithm>
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 #include "sbn.h"
 #include "sbn_common.cuh"
@@ -345,7 +346,7 @@ size_t sbn_xq_bytes(int T, int K) {
 
 size_t sbn_workspace_bytes(int op, int T, int N, int K) {
     switch (op) {
-        case SBN_OP_QUANTIZE_MASK_PACK: return sizeof(QmpWorkspace);
+        case SBN_OP_QUANTIZE_MASK_PACK: return sizeof(QmpWorkspace);       // one matrix; batches: sbn_batch_workspace_bytes
         case SBN_OP_QUANT_ACT: return 0;
         case SBN_OP_SPARSE_BITLINEAR:
         case SBN_OP_BITLINEAR:
@@ -371,6 +372,46 @@ sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int 
     return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(ws),
                                      static_cast<cudaStream_t>(stream));
+}
+
+size_t sbn_batch_workspace_bytes(int count) {
+    if (count <= 0) return 0;
+    const size_t descs = (static_cast<size_t>(count) * sizeof(QmpDesc) + 255) & ~static_cast<size_t>(255);
+    return descs + static_cast<size_t>(count) * sizeof(QmpWorkspace);
+}
+
+sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, void* ws, size_t ws_bytes,
+                                          void* stream) {
+    if (count <= 0) return SBN_ERR_SHAPE;
+    if (!jobs) return SBN_ERR_NULL;
+    if (!ws || ws_bytes < sbn_batch_workspace_bytes(count)) return SBN_ERR_WORKSPACE;
+    if (misaligned(ws, 16)) return SBN_ERR_ALIGN;
+    std::vector<QmpDesc> descs(static_cast<size_t>(count));
+    uint32_t max_units = 0;
+    for (int i = 0; i < count; ++i) {
+        const sbn_pack_job& j = jobs[i];
+        if (!j.W || !j.vals || !j.meta || !j.w_scale) return SBN_ERR_NULL;
+        if (j.prev_meta && !j.flip_bits) return SBN_ERR_NULL;
+        if (j.N <= 0 || j.K <= 0 || j.N % kBM != 0 || j.K % kBK != 0 || j.K > (1 << 20)) return SBN_ERR_SHAPE;
+        if (misaligned(j.W, 16) || misaligned(j.vals, 16) || misaligned(j.meta, 16) || misaligned(j.w_scale, 4) ||
+            (j.dense_q && misaligned(j.dense_q, 16)) || (j.prev_meta && misaligned(j.prev_meta, 16)) ||
+            (j.flip_bits && misaligned(j.flip_bits, 8)))
+            return SBN_ERR_ALIGN;
+        descs[i] = qmp_make_desc(j.W, j.N, j.K, j.vals, j.meta, j.w_scale, j.dense_q, j.prev_meta, j.flip_bits);
+        max_units = std::max(max_units, descs[i].num_units);
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t desc_bytes = (static_cast<size_t>(count) * sizeof(QmpDesc) + 255) & ~static_cast<size_t>(255);
+    QmpDesc* rest_dev = static_cast<QmpDesc*>(ws);
+    if (count > 1) {
+        // jobs 1.. are read by the kernel from the workspace (job 0 travels as a kernel argument);
+        // the source vector is pageable, so the runtime stages it before this call returns
+        if (cudaMemcpyAsync(rest_dev, descs.data() + 1, static_cast<size_t>(count - 1) * sizeof(QmpDesc),
+                            cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return SBN_ERR_CUDA;
+    }
+    QmpSlot* slots = reinterpret_cast<QmpSlot*>(static_cast<char*>(ws) + desc_bytes);
+    return launch_quantize_mask_pack_batch(descs[0], rest_dev, count, max_units, slots, s);
 }
 
 sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_keep, int m_group,

@@ -2,7 +2,8 @@
 // weights (Eq. 2), W_eff = W_q (.) M (Eq. 3), compressed value + metadata layout.
 //
 // gamma needs the whole matrix before any element can be rounded, so W has to be looked at
-// twice.  One persistent cooperative kernel (one 1024-thread CTA per SM) does both passes:
+// twice.  One persistent kernel (one 1024-thread CTA per SM) does both passes, for one matrix or
+// for a whole batch of them (pipelined, see the kernel):
 //
 //   pass 1   every CTA owns a contiguous range of (row, 128-column) units, streams it once,
 //            accumulates sum|W| in fp64, KEEPS the first part of its range in shared memory
@@ -110,119 +111,96 @@ __device__ __forceinline__ double abs_sum4(const float4 v) {
     return ((double)fabsf(v.x) + (double)fabsf(v.y)) + ((double)fabsf(v.z) + (double)fabsf(v.w));
 }
 
-template <bool WRITE_DENSE, bool COUNT_FLIPS>
-__global__ void __launch_bounds__(kQmpThreads, 1)
-quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uint32_t KB, double count,
-                          QmpSlot* slots, unsigned long long nonce,
-                          uint16_t* __restrict__ vals, uint8_t* meta, float* __restrict__ w_scale,
-                          uint32_t* __restrict__ dense_q, const uint8_t* prev_meta,
-                          unsigned long long* __restrict__ flip_bits) {
-    extern __shared__ float4 s_w[];                     // resident units, 32 float4 each
-    __shared__ double s_warp[kQmpWarps];
-    __shared__ float s_thr;
-    __shared__ int s_ok;
+// One matrix of a batch (device-visible copy of the call's arguments).
+struct QmpDesc {
+    const float4* W4;
+    uint16_t* vals;
+    uint8_t* meta;
+    float* w_scale;
+    uint32_t* dense_q;                 // or null
+    const uint8_t* prev_meta;          // or null
+    unsigned long long* flip_bits;     // or null
+    uint32_t num_units;                // N * K / 128
+    uint32_t KB;                       // K / 128
+};
 
+struct QmpRange {                      // this CTA's share of one matrix
+    uint32_t u_begin, u_end, n_res;
+};
+
+__device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d, uint32_t res_cap) {
+    QmpRange r;
+    const uint32_t per = (d.num_units + gridDim.x - 1) / gridDim.x;
+    r.u_begin = min(d.num_units, blockIdx.x * per);
+    r.u_end = min(d.num_units, r.u_begin + per);
+    r.n_res = min(r.u_end - r.u_begin, res_cap);
+    return r;
+}
+
+// pass 1 of one matrix: returns this CTA's sum |W| (identical in every thread); also writes the
+// metadata, keeps the first n_res units in `s_w` and accumulates the flip count into `flips`.
+__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, float4* s_w, double* s_warp,
+                                            unsigned int& flips) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint32_t per = (num_units + gridDim.x - 1) / gridDim.x;
-    const uint32_t u_begin = min(num_units, blockIdx.x * per);
-    const uint32_t u_end = min(num_units, u_begin + per);
-    const uint32_t n_res = min(u_end - u_begin, static_cast<uint32_t>(kQmpResidentUnits));
-
-    // ---- pass 1: sum |W| over this CTA's range (4 independent 16 B loads in flight per thread).
-    // The mask does not depend on gamma, so the top-2-of-4 selection, the metadata and the flip
-    // count are done here too, under the memory time of this pass.
+    const uint32_t KB = d.KB;
     const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
-    unsigned int flips = 0;
+    const bool count_flips = d.prev_meta != nullptr;
     double acc = 0.0;
-    {
-        uint32_t u = u_begin + warp;
-        int n_cur = 0, kb_cur = 0;
-        if (u < u_end) {
-            n_cur = static_cast<int>(u / KB);
-            kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
+    uint32_t u = rg.u_begin + warp;
+    int n_cur = 0, kb_cur = 0;
+    if (u < rg.u_end) {
+        n_cur = static_cast<int>(u / KB);
+        kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
+    }
+    for (; u < rg.u_end; u += 4 * kQmpWarps) {
+        float4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {                     // four independent 16 B loads in flight
+            const uint32_t uq = u + q * kQmpWarps;
+            v[q] = (uq < rg.u_end) ? __ldg(d.W4 + static_cast<size_t>(uq) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        for (; u < u_end; u += 4 * kQmpWarps) {
-            float4 v[4];
+        acc += (abs_sum4(v[0]) + abs_sum4(v[1])) + (abs_sum4(v[2]) + abs_sum4(v[3]));
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t uq = u + q * kQmpWarps;
-                v[q] = (uq < u_end) ? __ldg(W4 + static_cast<size_t>(uq) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            acc += (abs_sum4(v[0]) + abs_sum4(v[1])) + (abs_sum4(v[2]) + abs_sum4(v[3]));
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t uq = u + q * kQmpWarps;
-                if (uq < u_end) {
-                    const uint32_t r = uq - u_begin;
-                    if (r < n_res) s_w[r * 32 + lane] = v[q];
-                    const size_t m_off = ((static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) << 11) +
-                                         ((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1);
-                    n_cur += step_n;
-                    kb_cur += step_kb;
-                    if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
-                    const uint32_t nib = group_nibble(v[q]);
-                    const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
-                    if ((lane & 1) == 0) {
-                        const uint32_t byte = nib | (hi << 4);
-                        if constexpr (COUNT_FLIPS) {
-                            const uint32_t prev = prev_meta[m_off];
-                            flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev & 15u)) +
-                                     __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev >> 4) & 15u));
-                        }
-                        meta[m_off] = static_cast<uint8_t>(byte);
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t uq = u + q * kQmpWarps;
+            if (uq < rg.u_end) {
+                const uint32_t r = uq - rg.u_begin;
+                if (r < rg.n_res) s_w[r * 32 + lane] = v[q];
+                const size_t m_off = ((static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) << 11) +
+                                     ((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1);
+                n_cur += step_n;
+                kb_cur += step_kb;
+                if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+                const uint32_t nib = group_nibble(v[q]);
+                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+                if ((lane & 1) == 0) {
+                    const uint32_t byte = nib | (hi << 4);
+                    if (count_flips) {
+                        const uint32_t prev = d.prev_meta[m_off];
+                        flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev & 15u)) +
+                                 __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev >> 4) & 15u));
                     }
+                    d.meta[m_off] = static_cast<uint8_t>(byte);
                 }
             }
         }
     }
-    const double mine = qmp_block_sum(acc, s_warp);
+    return qmp_block_sum(acc, s_warp);
+}
 
-    // ---- exchange: publish, then wait (bounded) until every slot carries this call's nonce
-    if (threadIdx.x == 0) {
-        s_ok = 1;
-        if (blockIdx.x == 0 && flip_bits != nullptr) *flip_bits = 0ull;     // pass 2 accumulates
-        slots[blockIdx.x].partial = mine;
-        __threadfence();
-        *reinterpret_cast<volatile unsigned long long*>(&slots[blockIdx.x].nonce) = nonce;
-    }
-    __syncthreads();
-    double other = 0.0;
-    if (threadIdx.x < gridDim.x) {
-        const volatile unsigned long long* flag = &slots[threadIdx.x].nonce;
-        const unsigned long long t0 = global_timer_ns_qmp();
-        unsigned int spins = 0;
-        bool seen = (*flag == nonce);
-        while (!seen) {
-            seen = (*flag == nonce);
-            if (!seen && ((++spins & 0xFFu) == 0) && global_timer_ns_qmp() - t0 > kQmpWaitLimitNs) break;
-        }
-        if (seen) {
-            __threadfence();
-            other = *reinterpret_cast<const volatile double*>(&slots[threadIdx.x].partial);
-        } else {
-            s_ok = 0;
-            atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
-        }
-    }
-    const double S = qmp_block_sum(other, s_warp);          // fixed order: the same bits in every CTA
-    if (!s_ok) return;                                       // a peer never arrived: give up cleanly
-    const float gamma = static_cast<float>(S / count);
-    const float scale = fmaxf(gamma, kEps);
-    if (threadIdx.x == 0) {
-        s_thr = ternary_threshold(scale);
-        if (blockIdx.x == 0) *w_scale = scale;
-    }
-    __syncthreads();
-    const float thr = s_thr;
-
-    // ---- pass 2 (Eq. 1 + Eq. 3): ternarise the two kept values of every group.  A warp takes four
-    // units at a time (four loads in flight per lane); the re-read part newest first, then the
-    // resident part from shared memory.  The group's nibble is read back from the metadata.
-    const uint32_t n_units = u_end - u_begin;
+// pass 2 of one matrix (Eq. 1 + Eq. 3): ternarise the two kept values of every group.  A warp takes
+// four units at a time; the re-read part newest first, then the resident part from shared memory.
+__device__ __forceinline__ void qmp_pass2(const QmpDesc& d, const QmpRange rg, const float4* s_w, float thr) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t KB = d.KB;
+    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+    const uint32_t n_units = rg.u_end - rg.u_begin;
+    const bool write_dense = d.dense_q != nullptr;
     int n_cur = 0, kb_cur = 0;
     if (static_cast<uint32_t>(warp) < n_units) {
-        const uint32_t u_first = u_begin + (n_units - 1 - warp);
+        const uint32_t u_first = rg.u_begin + (n_units - 1 - warp);
         n_cur = static_cast<int>(u_first / KB);
         kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
     }
@@ -237,13 +215,13 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
             // i-th unit in processing order: units n_units-1 .. n_res (from global), then n_res-1 .. 0
             if (i < n_units) {
                 const uint32_t r = n_units - 1 - i;
-                w[q] = (r < n_res) ? s_w[r * 32 + lane] : __ldg(W4 + static_cast<size_t>(u_begin + r) * 32 + lane);
+                w[q] = (r < rg.n_res) ? s_w[r * 32 + lane] : __ldg(d.W4 + static_cast<size_t>(rg.u_begin + r) * 32 + lane);
                 tile_idx[q] = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
                 rr[q] = static_cast<uint32_t>(n_cur) & 127u;
                 n_cur -= step_n;
                 kb_cur -= step_kb;
                 if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
-                mb[q] = *(reinterpret_cast<const volatile uint8_t*>(meta) + (tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1));
+                mb[q] = *(reinterpret_cast<const volatile uint8_t*>(d.meta) + (tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1));
             }
         }
 #pragma unroll
@@ -254,28 +232,110 @@ quantize_mask_pack_kernel(const float4* __restrict__ W4, uint32_t num_units, uin
                 const uint32_t k0 = ternary_byte(pick4(w[q], nib & 3u), thr);
                 const uint32_t k1 = ternary_byte(pick4(w[q], nib >> 2), thr);
                 // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
-                vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(k0 | (k1 << 8));
-                if constexpr (WRITE_DENSE) {
-                    const uint32_t d = ternary_byte(w[q].x, thr) | (ternary_byte(w[q].y, thr) << 8) |
-                                       (ternary_byte(w[q].z, thr) << 16) | (ternary_byte(w[q].w, thr) << 24);
-                    dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = d;
+                d.vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(k0 | (k1 << 8));
+                if (write_dense) {
+                    const uint32_t dq = ternary_byte(w[q].x, thr) | (ternary_byte(w[q].y, thr) << 8) |
+                                        (ternary_byte(w[q].z, thr) << 16) | (ternary_byte(w[q].w, thr) << 24);
+                    d.dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = dq;
                 }
             }
         }
     }
+}
 
-    if constexpr (COUNT_FLIPS) {
+// Batch of `count` matrices in one persistent launch, software-pipelined over the matrices:
+//   P1(0) | P1(1) P2(0) | P1(2) P2(1) | ... | P2(count-1)
+// so by the time a CTA needs gamma of matrix m, every CTA has long published its partial for m,
+// and the per-launch and per-exchange latencies are paid once per batch, not once per matrix.
+// Shared memory is split in two halves that alternate between consecutive matrices (a batch of
+// one uses it all).  `first` is matrix 0 (passed by value), `rest` matrices 1.. in global memory.
+__global__ void __launch_bounds__(kQmpThreads, 1)
+quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
+                          QmpSlot* slots, unsigned long long nonce) {
+    extern __shared__ float4 s_w[];                     // resident units, 32 float4 each
+    __shared__ double s_warp[kQmpWarps];
+    __shared__ float s_thr;
+    __shared__ int s_ok;
+    __shared__ unsigned int s_flips[kQmpWarps];
+    __shared__ unsigned long long s_flip_total[2];
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t res_cap = count == 1 ? kQmpResidentUnits : kQmpResidentUnits / 2;
+    if (threadIdx.x == 0) s_ok = 1;
+    __syncthreads();
+
+    QmpDesc d_prev = first;
+    QmpRange rg_prev = {0u, 0u, 0u};
+    for (int m = 0; m <= count; ++m) {
+        // ---- pass 1 of matrix m, publish its partial
+        QmpDesc d_cur = first;
+        QmpRange rg_cur = {0u, 0u, 0u};
+        if (m < count) {
+            if (m > 0) d_cur = rest[m - 1];
+            rg_cur = qmp_range(d_cur, res_cap);
+            float4* half = s_w + static_cast<size_t>(count == 1 ? 0 : (m & 1)) * (kQmpResidentUnits / 2) * 32;
+            unsigned int flips = 0;
+            const double mine = qmp_pass1(d_cur, rg_cur, half, s_warp, flips);
+            // this CTA's flip count of matrix m; it is added to the global counter one phase later,
+            // after the exchange has shown that CTA 0 zeroed that counter
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) flips += __shfl_xor_sync(0xFFFFFFFFu, flips, o);
-        __shared__ unsigned int s_flips[kQmpWarps];
-        if (lane == 0) s_flips[warp] = flips;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned long long t = 0;
+            for (int o = 16; o > 0; o >>= 1) flips += __shfl_xor_sync(0xFFFFFFFFu, flips, o);
+            if (lane == 0) s_flips[warp] = flips;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned long long t = 0;
 #pragma unroll
-            for (int w2 = 0; w2 < kQmpWarps; ++w2) t += s_flips[w2];
-            if (t) atomicAdd(flip_bits, t);
+                for (int w2 = 0; w2 < kQmpWarps; ++w2) t += s_flips[w2];
+                s_flip_total[m & 1] = t;
+                if (blockIdx.x == 0 && d_cur.flip_bits != nullptr) *d_cur.flip_bits = 0ull;
+                QmpSlot* sl = slots + static_cast<size_t>(m) * gridDim.x + blockIdx.x;
+                sl->partial = mine;
+                __threadfence();
+                *reinterpret_cast<volatile unsigned long long*>(&sl->nonce) = nonce;
+            }
+            __syncthreads();
         }
+        // ---- exchange + pass 2 of matrix m-1 (published one phase ago by every CTA)
+        if (m >= 1) {
+            const QmpSlot* base = slots + static_cast<size_t>(m - 1) * gridDim.x;
+            double other = 0.0;
+            if (threadIdx.x < gridDim.x) {
+                const volatile unsigned long long* flag = &base[threadIdx.x].nonce;
+                const unsigned long long t0 = global_timer_ns_qmp();
+                unsigned int spins = 0;
+                bool seen = (*flag == nonce);
+                while (!seen) {
+                    seen = (*flag == nonce);
+                    if (!seen && ((++spins & 0xFFu) == 0) && global_timer_ns_qmp() - t0 > kQmpWaitLimitNs) break;
+                }
+                if (seen) {
+                    __threadfence();
+                    other = *reinterpret_cast<const volatile double*>(&base[threadIdx.x].partial);
+                } else {
+                    s_ok = 0;
+                    atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+                }
+            }
+            const double S = qmp_block_sum(other, s_warp);      // fixed order: the same bits in every CTA
+            if (!s_ok) return;                                   // a peer never arrived: give up cleanly
+            if (threadIdx.x == 0 && d_prev.flip_bits != nullptr && s_flip_total[(m - 1) & 1] != 0ull)
+                atomicAdd(d_prev.flip_bits, s_flip_total[(m - 1) & 1]);
+            const double cnt = static_cast<double>(d_prev.num_units) * 128.0;
+            const float gamma = static_cast<float>(S / cnt);
+            const float scale = fmaxf(gamma, kEps);
+            if (threadIdx.x == 0) {
+                s_thr = ternary_threshold(scale);
+                if (blockIdx.x == 0) *d_prev.w_scale = scale;
+            }
+            __syncthreads();
+            const float thr = s_thr;
+            const float4* half = s_w + static_cast<size_t>(count == 1 ? 0 : ((m - 1) & 1)) * (kQmpResidentUnits / 2) * 32;
+            qmp_pass2(d_prev, rg_prev, half, thr);
+            __syncthreads();                                     // s_thr / smem half may be reused
+        }
+        d_prev = d_cur;
+        rg_prev = rg_cur;
     }
 }
 
@@ -285,43 +345,47 @@ inline unsigned long long qmp_next_nonce() {
     return counter.fetch_add(1) + 1;
 }
 
+inline QmpDesc qmp_make_desc(const float* W, int N, int K, int8_t* vals, uint8_t* meta, float* w_scale,
+                             int8_t* dense_q, const uint8_t* prev_meta, unsigned long long* flip_bits) {
+    QmpDesc d;
+    d.W4 = reinterpret_cast<const float4*>(W);
+    d.vals = reinterpret_cast<uint16_t*>(vals);
+    d.meta = meta;
+    d.w_scale = w_scale;
+    d.dense_q = reinterpret_cast<uint32_t*>(dense_q);
+    d.prev_meta = prev_meta;
+    d.flip_bits = prev_meta ? flip_bits : nullptr;
+    d.num_units = static_cast<uint32_t>(static_cast<size_t>(N) * K / 128);
+    d.KB = static_cast<uint32_t>(K / 128);
+    return d;
+}
+
+// Launch for `count` matrices: `first` by value, the others already copied to `rest_dev`.
+inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const QmpDesc* rest_dev, int count,
+                                                  uint32_t max_units, QmpSlot* slots, cudaStream_t stream) {
+    unsigned long long nonce = qmp_next_nonce();
+    const unsigned grid = max_units < static_cast<uint32_t>(kQmpMaxCtas) ? max_units : kQmpMaxCtas;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(quantize_mask_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQmpSmemBytes) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        configured = true;
+    }
+    // At most one CTA per SM (200 KB of shared memory each) and never more CTAs than SMs, so all
+    // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
+    // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
+    quantize_mask_pack_kernel<<<grid, kQmpThreads, kQmpSmemBytes, stream>>>(first, rest_dev, count, slots, nonce);
+    ++g_launch_count;
+    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
 inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t* vals,
                                             uint8_t* meta, float* w_scale, int8_t* dense_q,
                                             const uint8_t* prev_meta,
                                             unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
-    const size_t count_sz = static_cast<size_t>(N) * K;
-    uint32_t num_units = static_cast<uint32_t>(count_sz / 128);
-    uint32_t KB = static_cast<uint32_t>(K / 128);
-    double count = static_cast<double>(count_sz);
-    const float4* W4 = reinterpret_cast<const float4*>(W);
-    QmpSlot* slots = ws->slot;
-    unsigned long long nonce = qmp_next_nonce();
-    uint16_t* v16 = reinterpret_cast<uint16_t*>(vals);
-    uint32_t* d32 = reinterpret_cast<uint32_t*>(dense_q);
-    const unsigned grid = num_units < static_cast<uint32_t>(kQmpMaxCtas) ? num_units : kQmpMaxCtas;
-    void* args[] = {&W4, &num_units, &KB, &count, &slots, &nonce, &v16, &meta, &w_scale, &d32,
-                    const_cast<uint8_t**>(&prev_meta), &flip_bits};
-    const void* fn;
-    if (dense_q && prev_meta) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<true, true>);
-    else if (dense_q) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<true, false>);
-    else if (prev_meta) fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<false, true>);
-    else fn = reinterpret_cast<const void*>(&quantize_mask_pack_kernel<false, false>);
-    static bool configured[4] = {false, false, false, false};
-    const int idx = (dense_q ? 2 : 0) + (prev_meta ? 1 : 0);
-    if (!configured[idx]) {
-        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kQmpSmemBytes) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        configured[idx] = true;
-    }
-    // At most one CTA per SM (200 KB of shared memory each) and never more CTAs than SMs, so all
-    // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
-    // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
-    // (A cooperative launch would guarantee co-residency but was measured to add ~10 us per call.)
-    if (cudaLaunchKernel(fn, dim3(grid), dim3(kQmpThreads), args, kQmpSmemBytes, stream) != cudaSuccess)
-        return SBN_ERR_CUDA;
-    ++g_launch_count;
-    return SBN_OK;
+    const QmpDesc d = qmp_make_desc(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
+    return launch_quantize_mask_pack_batch(d, nullptr, 1, d.num_units, ws->slot, stream);
 }
 
 }  // namespace sbn

@@ -84,6 +84,16 @@ def test_argument_validation_on_host(L):
     assert gemm(xq=odd) == ALIGN
     assert gemm(T=4, N=2560, K=2560) == WS          # decode shape needs split-K scratch
     assert L.sbn_bitlinear(p, p, 64, None, p, 256, 256, None, p, 0, None, None, 0, None) == NULL
+    from paper_2603_05168_b200 import binding as b
+    assert L.sbn_quantize_mask_pack_batched(0, p, p, 1 << 20, None) == SHAPE
+    assert L.sbn_quantize_mask_pack_batched(2, None, p, 1 << 20, None) == NULL
+    jobs = (b.PackJob * 2)()
+    for j in jobs:
+        j.W, j.N, j.K, j.vals, j.meta, j.w_scale = 0x1000, 256, 256, 0x1000, 0x1000, 0x1000
+    assert L.sbn_quantize_mask_pack_batched(2, ctypes.cast(jobs, ctypes.c_void_p), p, 16, None) == WS
+    jobs[1].K = 100
+    assert L.sbn_quantize_mask_pack_batched(2, ctypes.cast(jobs, ctypes.c_void_p), p, 1 << 20, None) == SHAPE
+    assert b.sbn_batch_workspace_bytes(3) >= 3 * 148 * 16
 
 
 def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):

@@ -149,6 +149,44 @@ def test_flip_count_parity(in_place):
     assert same["flips"] == 0
 
 
+def test_quantize_mask_pack_batched_matches_single_calls():
+    # one launch for several matrices of different shapes (with and without dense W_q / flip count):
+    # every job must reproduce the single call -- and the oracle -- bit for bit
+    shapes = [(256, 2560), (640, 256), (128, 128), (384, 1280), (2560, 640)]
+    Ws = [inputs.latent_weights(N, K, seed=40 + i, sigma=0.02 * (i + 1)) for i, (N, K) in enumerate(shapes)]
+    refs = [_oracle_pack(W) for W in Ws]
+    prevs = [oracle.quantize_mask_pack(inputs.perturb_weights(W, seed=60 + i, sigma=2e-3))["meta"] for i, W in enumerate(Ws)]
+    jobs, singles = [], []
+    for i, W in enumerate(Ws):
+        N, K = W.shape
+        use_prev, use_dense = (i % 2 == 0), (i % 3 != 0)
+        bufs = b.alloc_packed(N, K, with_dense=use_dense)
+        job = dict(W=dev(W), vals=bufs["vals"], meta=bufs["meta"], w_scale=bufs["w_scale"], dense_q=bufs.get("dense_q"))
+        if use_prev:
+            from gpu_harness import tile_meta
+            job["prev_meta"] = dev(tile_meta(prevs[i]).reshape(N, K // 8))
+            job["flip_bits"] = torch.full((1,), 777, dtype=torch.int64, device="cuda")
+        jobs.append(job)
+        singles.append(gpu_quantize_mask_pack(W, with_dense=use_dense, prev_meta=prevs[i] if use_prev else None))
+    arr = b.make_pack_jobs(jobs)
+    ws = torch.empty(b.sbn_batch_workspace_bytes(len(jobs)), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                        # twice: the second run meets stale slots
+        b.sbn_quantize_mask_pack_batched(arr, ws)
+    b.sbn_check_status()
+    from gpu_harness import _meta_offsets, _vals_offsets, untile
+    for i, (job, one, r) in enumerate(zip(jobs, singles, refs)):
+        N, K = Ws[i].shape
+        assert np.float32(job["w_scale"].cpu().numpy()[0]) == r["scale"] == one["scale"]
+        assert np.array_equal(untile(job["vals"].cpu().numpy(), _vals_offsets(N, K)), r["vals"])
+        assert np.array_equal(untile(job["meta"].cpu().numpy(), _meta_offsets(N, K)), r["meta"])
+        assert np.array_equal(job["vals"].cpu().numpy(), one["dev"]["vals"].cpu().numpy())
+        if job.get("dense_q") is not None:
+            assert np.array_equal(job["dense_q"].cpu().numpy(), one["dev"]["dense_q"].cpu().numpy())
+        if "flip_bits" in job:
+            want = oracle.flip_count(oracle.unpack24(r["vals"], prevs[i])[1], r["mask"])
+            assert int(job["flip_bits"].item()) == want == one["flips"]
+
+
 # ------------------------------------------------------------------------------------------------
 # part 3 and the dense baseline
 # ------------------------------------------------------------------------------------------------
