@@ -6,9 +6,10 @@
 // for a whole batch of them (pipelined, see the kernel):
 //
 //   pass 1   every CTA owns a contiguous range of (row, 128-column) units, streams it once,
-//            accumulates sum|W| in fp64, KEEPS the first part of its range in shared memory
-//            (200 KB per SM: 148 SMs hold 29.6 MB of W on chip) and -- the mask does not depend
-//            on gamma -- already selects the top 2 of 4, writes the metadata and counts flips;
+//            accumulates sum|W| in fp64 and -- the mask does not depend on gamma -- already
+//            selects the top 2 of 4, writes the metadata and counts flips.  It KEEPS the two
+//            selected weights of every group of the first part of its range in shared memory
+//            (8 B per group, 200 KB per SM: 148 SMs hold the kept half of 59 MB of W on chip);
 //   exchange every CTA publishes {call nonce, partial sum} in the workspace and waits (bounded)
 //            until all slots carry this call's nonce -- no atomics, no counter, nothing to
 //            initialise, stale slots of earlier calls can never match; every CTA then adds the
@@ -19,7 +20,7 @@
 //
 // HBM traffic per parameter: 4 B (one read) + 0.625 B written for the resident part, one more
 // (mostly L2-served) 4 B read for the rest.  16 B loads per lane, a warp covers one 512 B unit;
-// a warp store covers one whole 64 B (vals), 128 B (dense W_q) or 16 B (metadata) row of an
+// a warp store covers whole 64 B (vals), 128 B (dense W_q) or 16 B (metadata) rows of an
 // operand tile (tiled layouts, see layouts.cuh).
 //
 // Ternarisation without a per-element division: W_q = sign(w) * [ fl(|w| / scale) > 0.5 ]
@@ -37,8 +38,8 @@ namespace sbn {
 constexpr int kQmpThreads = 1024;
 constexpr int kQmpWarps = kQmpThreads / 32;
 constexpr int kQmpMaxCtas = kNumSMs;                       // one CTA per SM, all co-resident
-constexpr int kQmpResidentUnits = 400;                     // 400 x 512 B = 200 KB of W kept in smem
-constexpr int kQmpSmemBytes = kQmpResidentUnits * 512;
+constexpr int kQmpResidentUnits = 800;                     // units whose kept pairs stay in shared memory
+constexpr int kQmpSmemBytes = kQmpResidentUnits * 256;    // 32 groups x 8 B per unit: 200 KB
 constexpr unsigned long long kQmpWaitLimitNs = 2000000000ull;
 
 struct QmpSlot {                 // one per CTA, 16 B
@@ -63,30 +64,45 @@ __device__ __forceinline__ float ternary_threshold(float scale) {
     return a;
 }
 
-// Eq. 2 for one group: 2-bit indices i0 < i1 of the two largest |w| (ranking on the fp32 master
-// weights; on equal magnitudes the lower column wins), as nibble i0 | i1 << 2.
-__device__ __forceinline__ uint32_t group_nibble(const float4 w) {
+// Eq. 2 for one group: the two largest |w| of four (ranking on the fp32 master weights; on equal
+// magnitudes the lower column wins).  Returns the nibble i0 | i1 << 2 (i0 < i1) and the two kept
+// weights in column order.  The winners of the pairs (0,1) and (2,3) are the answer unless the
+// loser of one pair still beats the winner of the other:
+//   min(a0,a1) >= max(a2,a3)  ->  columns 0,1   (a tie goes to the lower column, hence >=)
+//   min(a2,a3) >  max(a0,a1)  ->  columns 2,3   (and hence > here)
+__device__ __forceinline__ uint32_t select_pair(const float4 w, float& v0, float& v1) {
     const float a0 = fabsf(w.x), a1 = fabsf(w.y), a2 = fabsf(w.z), a3 = fabsf(w.w);
-    // rank_j = number of entries that beat entry j; entry i beats j>i iff a_i >= a_j
-    const int c01 = a0 >= a1, c02 = a0 >= a2, c03 = a0 >= a3;
-    const int c12 = a1 >= a2, c13 = a1 >= a3, c23 = a2 >= a3;
-    const int r0 = (1 - c01) + (1 - c02) + (1 - c03);
-    const int r1 = c01 + (1 - c12) + (1 - c13);
-    const int r2 = c02 + c12 + (1 - c23);
-    const int r3 = c03 + c13 + c23;
-    const uint32_t keep = (r0 < 2 ? 1u : 0u) | (r1 < 2 ? 2u : 0u) | (r2 < 2 ? 4u : 0u) | (r3 < 2 ? 8u : 0u);
-    // exactly two bits set: lowest and highest set bit
-    const uint32_t i0 = __ffs(keep) - 1;
-    const uint32_t i1 = 31 - __clz(keep);
-    return i0 | (i1 << 2);
+    const bool c01 = a0 >= a1, c23 = a2 >= a3;
+    const bool both01 = fminf(a0, a1) >= fmaxf(a2, a3);
+    const bool both23 = fminf(a2, a3) > fmaxf(a0, a1);
+    v0 = c01 ? w.x : w.y;
+    v1 = c23 ? w.z : w.w;
+    uint32_t nib = (c01 ? 0u : 1u) | (c23 ? 8u : 12u);
+    if (both01) { v0 = w.x; v1 = w.y; nib = 4u; }
+    if (both23) { v0 = w.z; v1 = w.w; nib = 14u; }
+    return nib;
 }
 
-// Eq. 1 for one element as a byte: +1 -> 0x01, -1 -> 0xFF, 0 -> 0x00 (thr: see the header).
-__device__ __forceinline__ uint32_t ternary_byte(float w, float thr) {
-    return fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u;
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
-__device__ __forceinline__ float pick4(const float4 w, uint32_t i) {
-    return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
+
+// Eq. 1 for four elements as four bytes (+1 -> 0x01, -1 -> 0xFF, 0 -> 0x00; thr: see the header),
+// lowest byte = first argument.  The sign bytes come from byte permutes in sign-replication mode.
+__device__ __forceinline__ uint32_t ternary_bytes4(float w0, float w1, float w2, float w3, float thr) {
+    const uint32_t s01 = prmt(__float_as_uint(w0), __float_as_uint(w1), 0x00FBu);   // bytes 0,1: 0xFF if negative
+    const uint32_t s23 = prmt(__float_as_uint(w2), __float_as_uint(w3), 0x00FBu);
+    const uint32_t sgn = prmt(s01, s23, 0x5410u);
+    const uint32_t keep = (fabsf(w0) >= thr ? 0x000000FFu : 0u) | (fabsf(w1) >= thr ? 0x0000FF00u : 0u) |
+                          (fabsf(w2) >= thr ? 0x00FF0000u : 0u) | (fabsf(w3) >= thr ? 0xFF000000u : 0u);
+    return (sgn | 0x01010101u) & keep;
+}
+__device__ __forceinline__ uint32_t ternary_bytes2(float w0, float w1, float thr) {
+    const uint32_t sgn = prmt(__float_as_uint(w0), __float_as_uint(w1), 0x00FBu);
+    const uint32_t keep = (fabsf(w0) >= thr ? 0x00FFu : 0u) | (fabsf(w1) >= thr ? 0xFF00u : 0u);
+    return (sgn | 0x0101u) & keep;
 }
 
 __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
@@ -133,13 +149,14 @@ __device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d, uint32_t res_cap
     const uint32_t per = (d.num_units + gridDim.x - 1) / gridDim.x;
     r.u_begin = min(d.num_units, blockIdx.x * per);
     r.u_end = min(d.num_units, r.u_begin + per);
-    r.n_res = min(r.u_end - r.u_begin, res_cap);
+    r.n_res = d.dense_q != nullptr ? 0u : min(r.u_end - r.u_begin, res_cap);   // dense W_q needs all four weights
     return r;
 }
 
 // pass 1 of one matrix: returns this CTA's sum |W| (identical in every thread); also writes the
-// metadata, keeps the first n_res units in `s_w` and accumulates the flip count into `flips`.
-__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, float4* s_w, double* s_warp,
+// metadata, keeps the two selected weights of every group of the first n_res units in `s_pair`
+// (8 B per group: all that pass 2 needs) and accumulates the flip count into `flips`.
+__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, float2* s_pair, double* s_warp,
                                             unsigned int& flips) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -166,79 +183,98 @@ __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg,
             const uint32_t uq = u + q * kQmpWarps;
             if (uq < rg.u_end) {
                 const uint32_t r = uq - rg.u_begin;
-                if (r < rg.n_res) s_w[r * 32 + lane] = v[q];
-                const size_t m_off = ((static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) << 11) +
-                                     ((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1);
+                float2 kept;
+                const uint32_t nib = select_pair(v[q], kept.x, kept.y);
+                if (r < rg.n_res) s_pair[r * 32 + lane] = kept;
+                const size_t m_off = static_cast<size_t>((static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) * 2048u +
+                                     (((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1));
                 n_cur += step_n;
                 kb_cur += step_kb;
                 if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
-                const uint32_t nib = group_nibble(v[q]);
-                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
-                if ((lane & 1) == 0) {
-                    const uint32_t byte = nib | (hi << 4);
-                    if (count_flips) {
-                        const uint32_t prev = d.prev_meta[m_off];
-                        flips += __popc(nibble_to_mask(byte & 15u) ^ nibble_to_mask(prev & 15u)) +
-                                 __popc(nibble_to_mask(byte >> 4) ^ nibble_to_mask((prev >> 4) & 15u));
-                    }
-                    d.meta[m_off] = static_cast<uint8_t>(byte);
+                if (count_flips) {
+                    const uint32_t prev = (static_cast<uint32_t>(d.prev_meta[m_off]) >> ((lane & 1) * 4)) & 15u;
+                    flips += __popc(nibble_to_mask(nib) ^ nibble_to_mask(prev));
                 }
+                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+                if ((lane & 1) == 0) d.meta[m_off] = static_cast<uint8_t>(nib | (hi << 4));
             }
         }
     }
     return qmp_block_sum(acc, s_warp);
 }
 
-// pass 2 of one matrix (Eq. 1 + Eq. 3): ternarise the two kept values of every group.  A warp takes
-// four units at a time; the re-read part newest first, then the resident part from shared memory.
-__device__ __forceinline__ void qmp_pass2(const QmpDesc& d, const QmpRange rg, const float4* s_w, float thr) {
+// pass 2 of one matrix (Eq. 1 + Eq. 3): ternarise the two kept values of every group.
+//  * resident units: a half-warp per unit, a lane takes two groups (one 16 B shared-memory read,
+//    one 4 B store; the 16 lanes cover the 64 B tile row of the unit);
+//  * the other units are read again, newest first (what pass 1 read last is still in L2), a warp
+//    per unit and four units at a time, and the selection is redone.  When the dense W_q is
+//    wanted all units go this way (it needs all four weights of a group).
+__device__ __forceinline__ void qmp_pass2(const QmpDesc& d, const QmpRange rg, const float2* s_pair, float thr) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const uint32_t KB = d.KB;
-    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
     const uint32_t n_units = rg.u_end - rg.u_begin;
     const bool write_dense = d.dense_q != nullptr;
-    int n_cur = 0, kb_cur = 0;
-    if (static_cast<uint32_t>(warp) < n_units) {
-        const uint32_t u_first = rg.u_begin + (n_units - 1 - warp);
-        n_cur = static_cast<int>(u_first / KB);
-        kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
-    }
-    for (uint32_t i0 = warp; i0 < n_units; i0 += 4 * kQmpWarps) {
-        float4 w[4];
-        uint32_t mb[4];
-        size_t tile_idx[4];
-        uint32_t rr[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t i = i0 + q * kQmpWarps;
-            // i-th unit in processing order: units n_units-1 .. n_res (from global), then n_res-1 .. 0
-            if (i < n_units) {
-                const uint32_t r = n_units - 1 - i;
-                w[q] = (r < rg.n_res) ? s_w[r * 32 + lane] : __ldg(d.W4 + static_cast<size_t>(rg.u_begin + r) * 32 + lane);
-                tile_idx[q] = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-                rr[q] = static_cast<uint32_t>(n_cur) & 127u;
-                n_cur -= step_n;
-                kb_cur -= step_kb;
-                if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
-                mb[q] = *(reinterpret_cast<const volatile uint8_t*>(d.meta) + (tile_idx[q] << 11) + (rr[q] << 4) + (lane >> 1));
-            }
+    {   // ---- the part pass 1 left in L2 / HBM
+        const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+        const uint32_t n_far = n_units - rg.n_res;
+        int n_cur = 0, kb_cur = 0;
+        if (static_cast<uint32_t>(warp) < n_far) {
+            const uint32_t u_first = rg.u_begin + (n_units - 1 - warp);
+            n_cur = static_cast<int>(u_first / KB);
+            kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
         }
+        for (uint32_t i0 = warp; i0 < n_far; i0 += 4 * kQmpWarps) {
+            float4 w[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t i = i0 + q * kQmpWarps;
-            if (i < n_units) {
-                const uint32_t nib = (mb[q] >> ((lane & 1) * 4)) & 15u;
-                const uint32_t k0 = ternary_byte(pick4(w[q], nib & 3u), thr);
-                const uint32_t k1 = ternary_byte(pick4(w[q], nib >> 2), thr);
-                // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
-                d.vals[((tile_idx[q] << 13) + vals_in_tile(rr[q], 2u * lane)) >> 1] = static_cast<uint16_t>(k0 | (k1 << 8));
-                if (write_dense) {
-                    const uint32_t dq = ternary_byte(w[q].x, thr) | (ternary_byte(w[q].y, thr) << 8) |
-                                        (ternary_byte(w[q].z, thr) << 16) | (ternary_byte(w[q].w, thr) << 24);
-                    d.dense_q[((tile_idx[q] << 14) + sw128_in_tile(rr[q], 4u * lane)) >> 2] = dq;
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t i = i0 + q * kQmpWarps;
+                w[q] = (i < n_far) ? __ldg(d.W4 + static_cast<size_t>(rg.u_begin + (n_units - 1 - i)) * 32 + lane)
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t i = i0 + q * kQmpWarps;
+                if (i < n_far) {
+                    const size_t tile_idx = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+                    const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+                    n_cur -= step_n;
+                    kb_cur -= step_kb;
+                    if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
+                    float k0, k1;
+                    select_pair(w[q], k0, k1);
+                    // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
+                    d.vals[((tile_idx << 13) + vals_in_tile(rr, 2u * lane)) >> 1] = static_cast<uint16_t>(ternary_bytes2(k0, k1, thr));
+                    if (write_dense)
+                        d.dense_q[((tile_idx << 14) + sw128_in_tile(rr, 4u * lane)) >> 2] =
+                            ternary_bytes4(w[q].x, w[q].y, w[q].z, w[q].w, thr);
                 }
             }
+        }
+    }
+    {   // ---- the resident part
+        const int l16 = lane & 15;
+        const uint32_t first = 2u * warp + (lane >> 4);
+        constexpr uint32_t kStep = 2u * kQmpWarps;
+        const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
+        int n_cur = 0, kb_cur = 0;
+        if (first < rg.n_res) {
+            const uint32_t u_first = rg.u_begin + first;
+            n_cur = static_cast<int>(u_first / KB);
+            kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
+        }
+        const float4* s_quad = reinterpret_cast<const float4*>(s_pair);     // two groups per 16 B
+        uint32_t* vals32 = reinterpret_cast<uint32_t*>(d.vals);
+#pragma unroll 2
+        for (uint32_t r = first; r < rg.n_res; r += kStep) {
+            const float4 p = s_quad[r * 16 + l16];
+            const size_t tile_idx = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+            n_cur += step_n;
+            kb_cur += step_kb;
+            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+            // compressed columns 4*l16 .. 4*l16+3 of this 64 B tile row
+            vals32[((tile_idx << 13) + vals_in_tile(rr, 4u * l16)) >> 2] = ternary_bytes4(p.x, p.y, p.z, p.w, thr);
         }
     }
 }
@@ -252,7 +288,7 @@ __device__ __forceinline__ void qmp_pass2(const QmpDesc& d, const QmpRange rg, c
 __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
                           QmpSlot* slots, unsigned long long nonce) {
-    extern __shared__ float4 s_w[];                     // resident units, 32 float4 each
+    extern __shared__ float2 s_w[];                     // kept pairs of the resident units, 32 float2 each
     __shared__ double s_warp[kQmpWarps];
     __shared__ float s_thr;
     __shared__ int s_ok;
@@ -274,7 +310,7 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
         if (m < count) {
             if (m > 0) d_cur = rest[m - 1];
             rg_cur = qmp_range(d_cur, res_cap);
-            float4* half = s_w + static_cast<size_t>(count == 1 ? 0 : (m & 1)) * (kQmpResidentUnits / 2) * 32;
+            float2* half = s_w + static_cast<size_t>(count == 1 ? 0 : (m & 1)) * (kQmpResidentUnits / 2) * 32;
             unsigned int flips = 0;
             const double mine = qmp_pass1(d_cur, rg_cur, half, s_warp, flips);
             // this CTA's flip count of matrix m; it is added to the global counter one phase later,
@@ -330,7 +366,7 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             __syncthreads();
             const float thr = s_thr;
-            const float4* half = s_w + static_cast<size_t>(count == 1 ? 0 : ((m - 1) & 1)) * (kQmpResidentUnits / 2) * 32;
+            const float2* half = s_w + static_cast<size_t>(count == 1 ? 0 : ((m - 1) & 1)) * (kQmpResidentUnits / 2) * 32;
             qmp_pass2(d_prev, rg_prev, half, thr);
             __syncthreads();                                     // s_thr / smem half may be reused
         }
