@@ -288,7 +288,7 @@ def run_ours(args):
         torch.cuda._sleep(int(6e6 + n_chunk * 2.5e6))
         a_ev.record(stream)
         for _ in range(n_chunk):
-            step(evs)
+            step()
         c_ev.record(stream)
         chunk_times.append((a_ev, c_ev))
         done += n_chunk
@@ -302,6 +302,12 @@ def run_ours(args):
     ms_per_step = ms_total / args.steps
     value = whole_job_tops(step_ops(T, shapes), world, ms_per_step)
 
+    # per-kernel times inside the step sequence: a separate, instrumented pass (an event between
+    # two kernels would keep the second from starting its prologue under the first one's tail)
+    torch.cuda._sleep(int(6e6))
+    for _ in range(min(args.steps, 8)):
+        step(evs)
+    torch.cuda.synchronize()
     per_kernel = {k: {} for k in KERNELS}
     for name, e in evs:
         for i, k in enumerate(KERNELS):

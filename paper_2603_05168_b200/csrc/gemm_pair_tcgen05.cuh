@@ -209,6 +209,8 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     __syncthreads();
     cluster_sync_all();                  // the peer's barriers exist before anything is signalled
     tcgen05_fence_after();
+    pdl_wait();                          // nothing above touches global memory
+    pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 

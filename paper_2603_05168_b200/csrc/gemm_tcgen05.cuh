@@ -270,6 +270,8 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     }
     __syncthreads();
     tcgen05_fence_after();
+    pdl_wait();                          // nothing above touches global memory
+    pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 

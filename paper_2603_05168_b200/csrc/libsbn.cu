@@ -144,9 +144,9 @@ static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, 
     }
     const int tiles = (p.N / kBM) * ((p.T + BN - 1) / BN) * p.k_splits;
     const int grid = tiles < kNumSMs ? tiles : kNumSMs;
-    kernel<<<grid, kGemmThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, p);
+    const cudaError_t err = launch_kernel(kernel, dim3(grid), dim3(kGemmThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, ty, p);
     ++g_launch_count;
-    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
 // ---- CTA-pair kernel (large T) -------------------------------------------------------------------
@@ -201,9 +201,9 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
     }
     const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
     const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
-    kernel<<<2 * pairs, kPairThreads, Cfg::SMEM_BYTES, stream>>>(ta, tb, te, ty, pp);
+    const cudaError_t err = launch_kernel(kernel, dim3(2 * pairs), dim3(kPairThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, ty, pp);
     ++g_launch_count;
-    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
 static inline bool use_pair_kernel(int T) {

@@ -73,6 +73,9 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
     const size_t tb8 = xq_tb8(T);
     const int iters = (T + row_stride - 1) / row_stride;        // same for every thread of the CTA
 
+    pdl_wait();
+    pdl_launch_dependents();
+
     uint4 cur[VPT], nxt[VPT];
     int row = blockIdx.x * ROWS + r;
 #pragma unroll
@@ -129,6 +132,8 @@ __global__ void __launch_bounds__(kActThreads)
 quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
                           float* __restrict__ a_scale) {
     __shared__ float s_max[kActThreads / 32];
+    pdl_wait();
+    pdl_launch_dependents();
     const int row = blockIdx.x;
     if (row >= T) return;
     const uint4* xr = x + static_cast<size_t>(row) * nvec;
@@ -159,7 +164,7 @@ static void launch_quant_act_cfg(const uint4* x, int T, int nvec, uint2* q, floa
     const int ctas_per_sm = (VPT <= 4) ? 3 : 2;
     int grid = (T + rows - 1) / rows;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
-    quant_act_kernel<G, VPT><<<grid, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    launch_kernel(quant_act_kernel<G, VPT>, dim3(grid), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
 }
 
 inline sbn_status launch_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale,
@@ -177,7 +182,7 @@ inline sbn_status launch_quant_act(const void* x_bf16, int T, int K, int8_t* xq,
     else if (nvec <= 256 * 4) launch_quant_act_cfg<256, 4>(x, T, nvec, q, a_scale, stream);
     else if (nvec <= 256 * 6) launch_quant_act_cfg<256, 6>(x, T, nvec, q, a_scale, stream);
     else if (nvec <= 256 * 8) launch_quant_act_cfg<256, 8>(x, T, nvec, q, a_scale, stream);
-    else quant_act_long_row_kernel<<<T, kActThreads, 0, stream>>>(x, T, nvec, q, a_scale);
+    else launch_kernel(quant_act_long_row_kernel, dim3(T), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }

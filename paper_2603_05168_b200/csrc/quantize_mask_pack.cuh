@@ -109,6 +109,12 @@ __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
     return (1u << (nib & 3u)) | (1u << ((nib >> 2) & 3u));
 }
 
+// Ask the L2 to fetch [p, p + bytes) (a multiple of 16 B) -- issued by one thread, no destination.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+constexpr int kQmpPrefetchAhead = 3;                       // pass 1 iterations (128 units = 64 KB each) ahead
+
 // Sum of `v` over the CTA in a fixed order; identical in every thread.
 __device__ __forceinline__ double qmp_block_sum(double v, double* s_warp) {
 #pragma unroll
@@ -170,7 +176,19 @@ __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg,
         n_cur = static_cast<int>(u / KB);
         kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
     }
+    // One thread keeps the L2 a few iterations ahead of the loads (the CTA's range is contiguous),
+    // so the 32 warps x 4 loads in flight per SM do not have to cover the whole HBM latency.
+    if (threadIdx.x == 0) {
+        for (int j = 1; j < kQmpPrefetchAhead; ++j) {
+            const uint32_t ub = rg.u_begin + j * 4 * kQmpWarps;
+            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 4u * kQmpWarps) * 512u);
+        }
+    }
     for (; u < rg.u_end; u += 4 * kQmpWarps) {
+        if (threadIdx.x == 0) {                            // here u is the first unit of this iteration
+            const uint32_t ub = u + kQmpPrefetchAhead * 4 * kQmpWarps;
+            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 4u * kQmpWarps) * 512u);
+        }
         float4 v[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {                     // four independent 16 B loads in flight
@@ -300,6 +318,8 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
     const uint32_t res_cap = count == 1 ? kQmpResidentUnits : kQmpResidentUnits / 2;
     if (threadIdx.x == 0) s_ok = 1;
     __syncthreads();
+    pdl_wait();
+    pdl_launch_dependents();
 
     QmpDesc d_prev = first;
     QmpRange rg_prev = {0u, 0u, 0u};
@@ -410,9 +430,10 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
     // At most one CTA per SM (200 KB of shared memory each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
-    quantize_mask_pack_kernel<<<grid, kQmpThreads, kQmpSmemBytes, stream>>>(first, rest_dev, count, slots, nonce);
+    const cudaError_t err = launch_kernel(quantize_mask_pack_kernel, dim3(grid), dim3(kQmpThreads), kQmpSmemBytes, stream,
+                                          first, rest_dev, count, slots, nonce);
     ++g_launch_count;
-    return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
 inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t* vals,

@@ -3,6 +3,8 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
+#include <utility>
 
 #include "sbn.h"
 
@@ -17,6 +19,43 @@ __device__ int g_device_status = 0;
 
 // Host-side count of kernel launches made by the library.
 static unsigned long long g_launch_count = 0;
+
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// programmatic-stream-serialisation attribute and starts with
+//     <set-up that touches no global memory>;  pdl_wait();  pdl_launch_dependents();
+// pdl_wait returns once the preceding kernel of the stream has completed and its writes are
+// visible, so everything after it is ordered exactly as in a plain stream; what is gained is
+// that the CTAs of the next kernel become resident (and do their set-up) on SMs the previous
+// kernel has already left, instead of after a full launch round trip.  All kernels here are
+// persistent with every CTA resident from the start, so an early dependent only ever takes
+// resources nobody else is waiting for.  SBN_DISABLE_PDL=1 in the environment turns the
+// attribute off (the two instructions are then no-ops).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+inline bool pdl_enabled() {
+    static const bool on = [] {
+        const char* e = getenv("SBN_DISABLE_PDL");
+        return !(e && e[0] == '1');
+    }();
+    return on;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
