@@ -1,27 +1,33 @@
 // Part 1 of the path: absmean ternary quantisation (Eq. 1), 2:4 magnitude mask from the master
 // weights (Eq. 2), W_eff = W_q (.) M (Eq. 3), compressed value + metadata layout.
 //
-// gamma needs the whole matrix before any element can be rounded, so W has to be looked at
-// twice.  One persistent kernel (one 1024-thread CTA per SM) does both passes, for one matrix or
-// for a whole batch of them (pipelined, see the kernel):
+// gamma needs the whole matrix before any element can be rounded, but almost every element can be
+// rounded correctly from an ESTIMATE of gamma: W_q = sign(w) [ |w| >= thr(gamma) ] and only the
+// few |w| that lie within a few percent of thr depend on its exact value.  One persistent kernel
+// (one 1024-thread CTA per SM) therefore reads W ONCE, for one matrix or a batch of them:
 //
-//   pass 1   every CTA owns a contiguous range of (row, 128-column) units, streams it once,
-//            accumulates sum|W| in fp64 and -- the mask does not depend on gamma -- already
-//            selects the top 2 of 4, writes the metadata and counts flips.  It KEEPS the two
-//            selected weights of every group of the first part of its range in shared memory
-//            (8 B per group, 200 KB per SM: 148 SMs hold the kept half of 59 MB of W on chip);
+//   sample   every CTA adds |w| over the same 256 scattered 512 B units of the matrix (128 KB,
+//            L2-served for all CTAs but the first) -> gamma_est, and brackets the threshold:
+//            thr_lo = thr(0.97 gamma_est), thr_hi = thr(1.03 gamma_est);
+//   pass 1   every CTA owns a contiguous range of (row, 128-column) units and streams it:
+//            sum|W| in fp64 (the exact gamma), top 2 of 4 per group (Eq. 2: the mask does not
+//            depend on gamma), metadata, flip count, and the two kept values ternarised
+//            PROVISIONALLY: |w| >= thr_hi -> +-1 and |w| < thr_lo -> 0 are final whatever gamma
+//            turns out to be inside the bracket; the others (~2 % for Gaussian weights) are
+//            appended as {byte position, w} to a list in shared memory;
 //   exchange every CTA publishes {call nonce, partial sum} in the workspace and waits (bounded)
 //            until all slots carry this call's nonce -- no atomics, no counter, nothing to
 //            initialise, stale slots of earlier calls can never match; every CTA then adds the
 //            148 partials in the same fixed order, so all get the same bits, run after run;
-//   pass 2   ternarises the two kept values of every group: the resident part comes from shared
-//            memory, the rest is read again, newest first (what pass 1 read last is still in
-//            the 126 MB L2).
+//   fix-up   with the exact thr: if thr_lo <= thr <= thr_hi (and the list did not overflow) only
+//            the listed bytes are rewritten -- the result is exactly Eq. 1, not an approximation.
+//            Otherwise (a sample that misrepresents the matrix, the 1e-5 clamp, a request for the
+//            dense W_q, which needs all four weights of a group) the CTA reads its range again
+//            and ternarises everything with the exact thr: slower, same result.
 //
-// HBM traffic per parameter: 4 B (one read) + 0.625 B written for the resident part, one more
-// (mostly L2-served) 4 B read for the rest.  16 B loads per lane, a warp covers one 512 B unit;
-// a warp store covers whole 64 B (vals), 128 B (dense W_q) or 16 B (metadata) rows of an
-// operand tile (tiled layouts, see layouts.cuh).
+// HBM traffic per parameter: 4 B read + 0.625 B written.  16 B loads per lane, a warp covers one
+// 512 B unit; a warp store covers whole 64 B (vals), 128 B (dense W_q) or 16 B (metadata) rows of
+// an operand tile (tiled layouts, see layouts.cuh).
 //
 // Ternarisation without a per-element division: W_q = sign(w) * [ fl(|w| / scale) > 0.5 ]
 // (round-half-even sends exactly 0.5 to 0, everything above to >= 1, the clamp caps at 1).
@@ -38,8 +44,10 @@ namespace sbn {
 constexpr int kQmpThreads = 1024;
 constexpr int kQmpWarps = kQmpThreads / 32;
 constexpr int kQmpMaxCtas = kNumSMs;                       // one CTA per SM, all co-resident
-constexpr int kQmpResidentUnits = 800;                     // units whose kept pairs stay in shared memory
-constexpr int kQmpSmemBytes = kQmpResidentUnits * 256;    // 32 groups x 8 B per unit: 200 KB
+constexpr int kQmpListCap = 8192;                          // undecided entries per CTA and matrix
+constexpr int kQmpSmemBytes = 2 * kQmpListCap * 8;         // two lists (consecutive matrices of a batch)
+constexpr int kQmpSampleUnits = 256;                       // units in the gamma_est sample
+constexpr float kQmpBracket = 0.03f;                       // gamma_est * (1 -+ this) brackets gamma
 constexpr unsigned long long kQmpWaitLimitNs = 2000000000ull;
 
 struct QmpSlot {                 // one per CTA, 16 B
@@ -147,192 +155,226 @@ struct QmpDesc {
 };
 
 struct QmpRange {                      // this CTA's share of one matrix
-    uint32_t u_begin, u_end, n_res;
+    uint32_t u_begin, u_end;
+};
+struct QmpEntry {                      // one undecided kept value
+    uint32_t byte_off;                 // its byte in vals
+    float w;
 };
 
-__device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d, uint32_t res_cap) {
+__device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d) {
     QmpRange r;
     const uint32_t per = (d.num_units + gridDim.x - 1) / gridDim.x;
     r.u_begin = min(d.num_units, blockIdx.x * per);
     r.u_end = min(d.num_units, r.u_begin + per);
-    r.n_res = d.dense_q != nullptr ? 0u : min(r.u_end - r.u_begin, res_cap);   // dense W_q needs all four weights
     return r;
 }
 
-// pass 1 of one matrix: returns this CTA's sum |W| (identical in every thread); also writes the
-// metadata, keeps the two selected weights of every group of the first n_res units in `s_pair`
-// (8 B per group: all that pass 2 needs) and accumulates the flip count into `flips`.
-__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, float2* s_pair, double* s_warp,
+// gamma_est: mean |w| over kQmpSampleUnits units scattered over the matrix (the same units in every
+// CTA; a multiplicative hash keeps them off any row / column-block period).  fp32 is plenty here.
+__device__ __forceinline__ float qmp_sample_gamma(const QmpDesc& d, double* s_warp) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t n_s = min(d.num_units, static_cast<uint32_t>(kQmpSampleUnits));
+    const uint32_t stride = d.num_units / n_s;                        // >= 1
+    float acc = 0.0f;
+    constexpr int kPerWarp = kQmpSampleUnits / kQmpWarps;
+    float4 v[kPerWarp];
+#pragma unroll
+    for (int i = 0; i < kPerWarp; ++i) {                  // all loads of the warp in flight at once
+        const uint32_t sidx = warp + i * kQmpWarps;
+        const uint32_t u = sidx * stride + ((sidx * 2654435761u) >> 8) % stride;
+        v[i] = sidx < n_s ? __ldg(d.W4 + static_cast<size_t>(u) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < kPerWarp; ++i) acc += (fabsf(v[i].x) + fabsf(v[i].y)) + (fabsf(v[i].z) + fabsf(v[i].w));
+    const double total = qmp_block_sum(static_cast<double>(acc), s_warp);
+    return static_cast<float>(total / (static_cast<double>(n_s) * 128.0));
+}
+
+// Appends the undecided ones of four consecutive kept values (bytes byte_off .. byte_off + 3 of vals).
+__device__ __forceinline__ void qmp_list_undecided(const float (&k)[4], const float thr_lo, const float thr_hi,
+                                                   const uint32_t byte_off, QmpEntry* list, unsigned int* list_count) {
+    bool und[4];
+    unsigned int cnt = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float a = fabsf(k[i]);
+        und[i] = a >= thr_lo && a < thr_hi;
+        cnt += und[i] ? 1u : 0u;
+    }
+    if (cnt != 0u) {                                       // a few percent of the lanes get here
+        unsigned int at = atomicAdd(list_count, cnt);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (und[i]) {
+                if (at < static_cast<unsigned int>(kQmpListCap)) { list[at].byte_off = byte_off + i; list[at].w = k[i]; }
+                ++at;
+            }
+        }
+    }
+}
+
+// pass 1 of one matrix: returns this CTA's sum |W| (identical in every thread); writes the metadata
+// and the provisional vals, lists the undecided kept values and accumulates the flip count.
+// A lane takes TWO adjacent groups (32 B of a row), so it owns a whole metadata byte and four
+// consecutive bytes of vals and the per-unit index arithmetic is shared by two groups; a half-warp
+// covers one 512 B unit, a warp two units per load pair and four per iteration.
+__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
+                                            QmpEntry* list, unsigned int* list_count, double* s_warp,
                                             unsigned int& flips) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    const uint32_t l16 = lane & 15;
     const uint32_t KB = d.KB;
-    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+    constexpr uint32_t kStep = 2 * kQmpWarps;                // units between a thread's consecutive units
+    const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
     const bool count_flips = d.prev_meta != nullptr;
     double acc = 0.0;
-    uint32_t u = rg.u_begin + warp;
-    int n_cur = 0, kb_cur = 0;
-    if (u < rg.u_end) {
-        n_cur = static_cast<int>(u / KB);
-        kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
-    }
+    const uint32_t u_first = rg.u_begin + 2 * warp + (lane >> 4);
+    int n_cur = static_cast<int>(u_first / KB);
+    int kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
     // One thread keeps the L2 a few iterations ahead of the loads (the CTA's range is contiguous),
-    // so the 32 warps x 4 loads in flight per SM do not have to cover the whole HBM latency.
+    // so the loads in flight per SM do not have to cover the whole HBM latency.
     if (threadIdx.x == 0) {
         for (int j = 1; j < kQmpPrefetchAhead; ++j) {
-            const uint32_t ub = rg.u_begin + j * 4 * kQmpWarps;
-            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 4u * kQmpWarps) * 512u);
+            const uint32_t ub = rg.u_begin + j * 2 * kStep;
+            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 2 * kStep) * 512u);
         }
     }
-    for (; u < rg.u_end; u += 4 * kQmpWarps) {
-        if (threadIdx.x == 0) {                            // here u is the first unit of this iteration
-            const uint32_t ub = u + kQmpPrefetchAhead * 4 * kQmpWarps;
-            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 4u * kQmpWarps) * 512u);
+    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += 2 * kStep) {
+        if (threadIdx.x == 0) {
+            const uint32_t ub = u0 + kQmpPrefetchAhead * 2 * kStep;
+            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 2 * kStep) * 512u);
         }
-        float4 v[4];
+        float4 va[2], vb[2];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {                     // four independent 16 B loads in flight
-            const uint32_t uq = u + q * kQmpWarps;
-            v[q] = (uq < rg.u_end) ? __ldg(d.W4 + static_cast<size_t>(uq) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int q = 0; q < 2; ++q) {                     // four independent 16 B loads in flight
+            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
+            const float4* src = d.W4 + static_cast<size_t>(uq) * 32 + 2 * l16;
+            va[q] = (uq < rg.u_end) ? __ldg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+            vb[q] = (uq < rg.u_end) ? __ldg(src + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        acc += (abs_sum4(v[0]) + abs_sum4(v[1])) + (abs_sum4(v[2]) + abs_sum4(v[3]));
+        acc += (abs_sum4(va[0]) + abs_sum4(vb[0])) + (abs_sum4(va[1]) + abs_sum4(vb[1]));
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t uq = u + q * kQmpWarps;
+        for (int q = 0; q < 2; ++q) {
+            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
+            const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+            n_cur += step_n;
+            kb_cur += step_kb;
+            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
             if (uq < rg.u_end) {
-                const uint32_t r = uq - rg.u_begin;
-                float2 kept;
-                const uint32_t nib = select_pair(v[q], kept.x, kept.y);
-                if (r < rg.n_res) s_pair[r * 32 + lane] = kept;
-                const size_t m_off = static_cast<size_t>((static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur)) * 2048u +
-                                     (((static_cast<uint32_t>(n_cur) & 127u) << 4) + (lane >> 1));
-                n_cur += step_n;
-                kb_cur += step_kb;
-                if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+                float k[4];
+                const uint32_t nib0 = select_pair(va[q], k[0], k[1]);
+                const uint32_t nib1 = select_pair(vb[q], k[2], k[3]);
+                const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
                 if (count_flips) {
-                    const uint32_t prev = (static_cast<uint32_t>(d.prev_meta[m_off]) >> ((lane & 1) * 4)) & 15u;
-                    flips += __popc(nibble_to_mask(nib) ^ nibble_to_mask(prev));
+                    const uint32_t prev = d.prev_meta[m_off];
+                    flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
+                                    (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
                 }
-                const uint32_t hi = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
-                if ((lane & 1) == 0) d.meta[m_off] = static_cast<uint8_t>(nib | (hi << 4));
+                d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
+                // provisional Eq. 1 + Eq. 3: compressed columns 4*l16 .. 4*l16+3 of this 64 B tile row
+                const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
+                reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
+                qmp_list_undecided(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
             }
         }
     }
     return qmp_block_sum(acc, s_warp);
 }
 
-// pass 2 of one matrix (Eq. 1 + Eq. 3): ternarise the two kept values of every group.
-//  * resident units: a half-warp per unit, a lane takes two groups (one 16 B shared-memory read,
-//    one 4 B store; the 16 lanes cover the 64 B tile row of the unit);
-//  * the other units are read again, newest first (what pass 1 read last is still in L2), a warp
-//    per unit and four units at a time, and the selection is redone.  When the dense W_q is
-//    wanted all units go this way (it needs all four weights of a group).
-__device__ __forceinline__ void qmp_pass2(const QmpDesc& d, const QmpRange rg, const float2* s_pair, float thr) {
+// Ternarise a whole range again with the exact threshold (the path taken when the bracket missed,
+// the list overflowed or the dense W_q is wanted): a warp per unit, four units at a time, newest
+// first (what pass 1 read last is still in L2).
+__device__ __forceinline__ void qmp_pass2_full(const QmpDesc& d, const QmpRange rg, float thr) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const uint32_t KB = d.KB;
     const uint32_t n_units = rg.u_end - rg.u_begin;
     const bool write_dense = d.dense_q != nullptr;
-    {   // ---- the part pass 1 left in L2 / HBM
-        const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
-        const uint32_t n_far = n_units - rg.n_res;
-        int n_cur = 0, kb_cur = 0;
-        if (static_cast<uint32_t>(warp) < n_far) {
-            const uint32_t u_first = rg.u_begin + (n_units - 1 - warp);
-            n_cur = static_cast<int>(u_first / KB);
-            kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
-        }
-        for (uint32_t i0 = warp; i0 < n_far; i0 += 4 * kQmpWarps) {
-            float4 w[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t i = i0 + q * kQmpWarps;
-                w[q] = (i < n_far) ? __ldg(d.W4 + static_cast<size_t>(rg.u_begin + (n_units - 1 - i)) * 32 + lane)
-                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t i = i0 + q * kQmpWarps;
-                if (i < n_far) {
-                    const size_t tile_idx = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-                    const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
-                    n_cur -= step_n;
-                    kb_cur -= step_kb;
-                    if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
-                    float k0, k1;
-                    select_pair(w[q], k0, k1);
-                    // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
-                    d.vals[((tile_idx << 13) + vals_in_tile(rr, 2u * lane)) >> 1] = static_cast<uint16_t>(ternary_bytes2(k0, k1, thr));
-                    if (write_dense)
-                        d.dense_q[((tile_idx << 14) + sw128_in_tile(rr, 4u * lane)) >> 2] =
-                            ternary_bytes4(w[q].x, w[q].y, w[q].z, w[q].w, thr);
-                }
-            }
-        }
+    const int step_n = static_cast<int>(kQmpWarps / KB), step_kb = static_cast<int>(kQmpWarps % KB);
+    int n_cur = 0, kb_cur = 0;
+    if (static_cast<uint32_t>(warp) < n_units) {
+        const uint32_t u_first = rg.u_begin + (n_units - 1 - warp);
+        n_cur = static_cast<int>(u_first / KB);
+        kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
     }
-    {   // ---- the resident part
-        const int l16 = lane & 15;
-        const uint32_t first = 2u * warp + (lane >> 4);
-        constexpr uint32_t kStep = 2u * kQmpWarps;
-        const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
-        int n_cur = 0, kb_cur = 0;
-        if (first < rg.n_res) {
-            const uint32_t u_first = rg.u_begin + first;
-            n_cur = static_cast<int>(u_first / KB);
-            kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
+    for (uint32_t i0 = warp; i0 < n_units; i0 += 4 * kQmpWarps) {
+        float4 w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t i = i0 + q * kQmpWarps;
+            w[q] = (i < n_units) ? __ldg(d.W4 + static_cast<size_t>(rg.u_begin + (n_units - 1 - i)) * 32 + lane)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        const float4* s_quad = reinterpret_cast<const float4*>(s_pair);     // two groups per 16 B
-        uint32_t* vals32 = reinterpret_cast<uint32_t*>(d.vals);
-#pragma unroll 2
-        for (uint32_t r = first; r < rg.n_res; r += kStep) {
-            const float4 p = s_quad[r * 16 + l16];
-            const size_t tile_idx = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
-            n_cur += step_n;
-            kb_cur += step_kb;
-            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
-            // compressed columns 4*l16 .. 4*l16+3 of this 64 B tile row
-            vals32[((tile_idx << 13) + vals_in_tile(rr, 4u * l16)) >> 2] = ternary_bytes4(p.x, p.y, p.z, p.w, thr);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t i = i0 + q * kQmpWarps;
+            if (i < n_units) {
+                const size_t tile_idx = static_cast<size_t>(static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+                const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+                n_cur -= step_n;
+                kb_cur -= step_kb;
+                if (kb_cur < 0) { kb_cur += static_cast<int>(KB); --n_cur; }
+                float k0, k1;
+                select_pair(w[q], k0, k1);
+                // compressed columns 2*lane, 2*lane+1 of this 64 B tile row
+                d.vals[((tile_idx << 13) + vals_in_tile(rr, 2u * lane)) >> 1] = static_cast<uint16_t>(ternary_bytes2(k0, k1, thr));
+                if (write_dense)
+                    d.dense_q[((tile_idx << 14) + sw128_in_tile(rr, 4u * lane)) >> 2] =
+                        ternary_bytes4(w[q].x, w[q].y, w[q].z, w[q].w, thr);
+            }
         }
     }
 }
 
 // Batch of `count` matrices in one persistent launch, software-pipelined over the matrices:
-//   P1(0) | P1(1) P2(0) | P1(2) P2(1) | ... | P2(count-1)
+//   S+P1(0) | S+P1(1) F(0) | S+P1(2) F(1) | ... | F(count-1)        (S sample, F exchange + fix-up)
 // so by the time a CTA needs gamma of matrix m, every CTA has long published its partial for m,
 // and the per-launch and per-exchange latencies are paid once per batch, not once per matrix.
-// Shared memory is split in two halves that alternate between consecutive matrices (a batch of
-// one uses it all).  `first` is matrix 0 (passed by value), `rest` matrices 1.. in global memory.
+// The two undecided lists alternate between consecutive matrices.  `first` is matrix 0 (passed by
+// value), `rest` matrices 1.. in global memory.
 __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
                           QmpSlot* slots, unsigned long long nonce) {
-    extern __shared__ float2 s_w[];                     // kept pairs of the resident units, 32 float2 each
+    extern __shared__ QmpEntry s_list[];                // [2][kQmpListCap]
     __shared__ double s_warp[kQmpWarps];
     __shared__ float s_thr;
     __shared__ int s_ok;
     __shared__ unsigned int s_flips[kQmpWarps];
     __shared__ unsigned long long s_flip_total[2];
+    __shared__ unsigned int s_list_count[2];
+    __shared__ float s_bracket[2][2];                   // [matrix parity][lo, hi]
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint32_t res_cap = count == 1 ? kQmpResidentUnits : kQmpResidentUnits / 2;
     if (threadIdx.x == 0) s_ok = 1;
     __syncthreads();
     pdl_wait();
     pdl_launch_dependents();
 
     QmpDesc d_prev = first;
-    QmpRange rg_prev = {0u, 0u, 0u};
+    QmpRange rg_prev = {0u, 0u};
     for (int m = 0; m <= count; ++m) {
-        // ---- pass 1 of matrix m, publish its partial
+        // ---- sample + pass 1 of matrix m, publish its partial
         QmpDesc d_cur = first;
-        QmpRange rg_cur = {0u, 0u, 0u};
+        QmpRange rg_cur = {0u, 0u};
         if (m < count) {
             if (m > 0) d_cur = rest[m - 1];
-            rg_cur = qmp_range(d_cur, res_cap);
-            float2* half = s_w + static_cast<size_t>(count == 1 ? 0 : (m & 1)) * (kQmpResidentUnits / 2) * 32;
+            rg_cur = qmp_range(d_cur);
+            const int par = m & 1;
+            const float gamma_est = qmp_sample_gamma(d_cur, s_warp);
+            if (threadIdx.x == 0) {
+                s_list_count[par] = 0u;
+                s_bracket[par][0] = ternary_threshold(fmaxf(gamma_est * (1.0f - kQmpBracket), kEps));
+                s_bracket[par][1] = ternary_threshold(fmaxf(gamma_est * (1.0f + kQmpBracket), kEps));
+            }
+            __syncthreads();
             unsigned int flips = 0;
-            const double mine = qmp_pass1(d_cur, rg_cur, half, s_warp, flips);
+            const double mine = qmp_pass1(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1],
+                                          s_list + par * kQmpListCap, &s_list_count[par], s_warp, flips);
             // this CTA's flip count of matrix m; it is added to the global counter one phase later,
             // after the exchange has shown that CTA 0 zeroed that counter
 #pragma unroll
@@ -343,7 +385,7 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                 unsigned long long t = 0;
 #pragma unroll
                 for (int w2 = 0; w2 < kQmpWarps; ++w2) t += s_flips[w2];
-                s_flip_total[m & 1] = t;
+                s_flip_total[par] = t;
                 if (blockIdx.x == 0 && d_cur.flip_bits != nullptr) *d_cur.flip_bits = 0ull;
                 QmpSlot* sl = slots + static_cast<size_t>(m) * gridDim.x + blockIdx.x;
                 sl->partial = mine;
@@ -352,8 +394,9 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             __syncthreads();
         }
-        // ---- exchange + pass 2 of matrix m-1 (published one phase ago by every CTA)
+        // ---- exchange + fix-up of matrix m-1 (published one phase ago by every CTA)
         if (m >= 1) {
+            const int par = (m - 1) & 1;
             const QmpSlot* base = slots + static_cast<size_t>(m - 1) * gridDim.x;
             double other = 0.0;
             if (threadIdx.x < gridDim.x) {
@@ -375,8 +418,8 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             const double S = qmp_block_sum(other, s_warp);      // fixed order: the same bits in every CTA
             if (!s_ok) return;                                   // a peer never arrived: give up cleanly
-            if (threadIdx.x == 0 && d_prev.flip_bits != nullptr && s_flip_total[(m - 1) & 1] != 0ull)
-                atomicAdd(d_prev.flip_bits, s_flip_total[(m - 1) & 1]);
+            if (threadIdx.x == 0 && d_prev.flip_bits != nullptr && s_flip_total[par] != 0ull)
+                atomicAdd(d_prev.flip_bits, s_flip_total[par]);
             const double cnt = static_cast<double>(d_prev.num_units) * 128.0;
             const float gamma = static_cast<float>(S / cnt);
             const float scale = fmaxf(gamma, kEps);
@@ -386,9 +429,22 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             __syncthreads();
             const float thr = s_thr;
-            const float2* half = s_w + static_cast<size_t>(count == 1 ? 0 : ((m - 1) & 1)) * (kQmpResidentUnits / 2) * 32;
-            qmp_pass2(d_prev, rg_prev, half, thr);
-            __syncthreads();                                     // s_thr / smem half may be reused
+            const unsigned int listed = s_list_count[par];
+            const bool bracket_ok = s_bracket[par][0] <= thr && thr <= s_bracket[par][1] &&
+                                    listed <= static_cast<unsigned int>(kQmpListCap) && d_prev.dense_q == nullptr &&
+                                    d_prev.num_units <= (1u << 26);        // listed byte offsets are 32-bit
+            if (bracket_ok) {
+                // every byte not on the list is already final; the listed ones get the exact compare
+                const QmpEntry* list = s_list + par * kQmpListCap;
+                uint8_t* vb = reinterpret_cast<uint8_t*>(d_prev.vals);
+                for (unsigned int e = threadIdx.x; e < listed; e += kQmpThreads) {
+                    const float w = list[e].w;
+                    vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
+                }
+            } else {
+                qmp_pass2_full(d_prev, rg_prev, thr);
+            }
+            __syncthreads();                                     // s_thr / this list may be reused
         }
         d_prev = d_cur;
         rg_prev = rg_cur;
