@@ -483,7 +483,7 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
             return SBN_ERR_CUDA;
         configured = true;
     }
-    // At most one CTA per SM (200 KB of shared memory each) and never more CTAs than SMs, so all
+    // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
     const cudaError_t err = launch_kernel(quantize_mask_pack_kernel, dim3(grid), dim3(kQmpThreads), kQmpSmemBytes, stream,

@@ -70,24 +70,31 @@ def test_quant_act_edge_rows():
 # ------------------------------------------------------------------------------------------------
 # part 1: quantise, mask, pack
 # ------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("N,K,seed", [(256, 256, 0), (128, 128, 1), (384, 2560, 2), (128, 6912, 3), (640, 2560, 4)])
-def test_quantize_mask_pack_parity(N, K, seed):
+# with_dense=False is the single-pass route (provisional ternarisation + fix-up list); asking for the
+# dense W_q makes the kernel ternarise everything in a second pass -- both must give the same bits.
+@pytest.mark.parametrize("with_dense", [True, False])
+@pytest.mark.parametrize("N,K,seed", [(256, 256, 0), (128, 128, 1), (384, 2560, 2), (128, 6912, 3), (640, 2560, 4),
+                                      (2048, 2560, 7)])
+def test_quantize_mask_pack_parity(N, K, seed, with_dense):
     W = inputs.latent_weights(N, K, seed=seed)
     r = _oracle_pack(W)
-    g = gpu_quantize_mask_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=with_dense)
     assert g["scale"] == r["scale"]
     assert np.array_equal(g["vals"], r["vals"])
     assert np.array_equal(g["meta"], r["meta"])
-    assert np.array_equal(g["dense_q"], r["dense_q"])
+    if with_dense:
+        assert np.array_equal(g["dense_q"], r["dense_q"])
 
 
-def test_quantize_mask_pack_heavy_tail():
+@pytest.mark.parametrize("with_dense", [True, False])
+def test_quantize_mask_pack_heavy_tail(with_dense):
     W = inputs.latent_weights(256, 4096, seed=5, sigma=0.015, outlier_prob=0.05, outlier_mult=10.0)
     r = _oracle_pack(W)
-    g = gpu_quantize_mask_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=with_dense)
     assert g["scale"] == r["scale"]
     assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
-    assert np.array_equal(g["dense_q"], r["dense_q"])
+    if with_dense:
+        assert np.array_equal(g["dense_q"], r["dense_q"])
 
 
 def test_quantize_mask_pack_adversarial():
@@ -105,24 +112,90 @@ def test_quantize_mask_pack_adversarial():
     s = r["scale"]
     W[6, :4] = [0.5 * s, -0.5 * s, 1.5 * s, np.nextafter(np.float32(0.5 * s), np.float32(1))]
     r = _oracle_pack(W)
-    g = gpu_quantize_mask_pack(W)
-    assert g["scale"] == r["scale"]
-    assert np.array_equal(g["vals"], r["vals"])
-    assert np.array_equal(g["meta"], r["meta"])
-    assert np.array_equal(g["dense_q"], r["dense_q"])
+    for with_dense in (True, False):
+        g = gpu_quantize_mask_pack(W, with_dense=with_dense)
+        assert g["scale"] == r["scale"]
+        assert np.array_equal(g["vals"], r["vals"])
+        assert np.array_equal(g["meta"], r["meta"])
+        if with_dense:
+            assert np.array_equal(g["dense_q"], r["dense_q"])
 
 
 def test_quantize_mask_pack_degenerate_scales():
     Z = np.zeros((128, 128), np.float32)
     r = oracle.quantize_mask_pack(Z)
-    g = gpu_quantize_mask_pack(Z)
-    assert g["scale"] == r["scale"] == np.float32(1e-5)
-    assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
+    for with_dense in (True, False):
+        g = gpu_quantize_mask_pack(Z, with_dense=with_dense)
+        assert g["scale"] == r["scale"] == np.float32(1e-5)
+        assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
     tiny = np.full((128, 128), 7e-6, np.float32)          # gamma below the clamp, 0.7 -> rounds to 1
     r = oracle.quantize_mask_pack(tiny)
-    g = gpu_quantize_mask_pack(tiny)
-    assert g["scale"] == r["scale"] and np.array_equal(g["vals"], r["vals"])
-    assert np.array_equal(g["dense_q"], r["dense_q"])
+    for with_dense in (True, False):
+        g = gpu_quantize_mask_pack(tiny, with_dense=with_dense)
+        assert g["scale"] == r["scale"] and np.array_equal(g["vals"], r["vals"])
+        if with_dense:
+            assert np.array_equal(g["dense_q"], r["dense_q"])
+
+
+def _sampled_units(N, K):
+    """The units the kernel's gamma estimate looks at (restated from the kernel's description:
+    256 units, unit s at s * stride + (s * 2654435761 mod 2^32 >> 8) mod stride)."""
+    num_units = N * K // 128
+    n_s = min(num_units, 256)
+    stride = num_units // n_s
+    sidx = np.arange(n_s, dtype=np.uint64)
+    return (sidx * stride + (((sidx * 2654435761) & 0xFFFFFFFF) >> 8) % stride).astype(np.int64)
+
+
+def test_quantize_mask_pack_misleading_sample():
+    # the sampled units are 1000x smaller than the rest: the bracket around the estimated threshold
+    # misses the exact one and the kernel has to take its second pass -- same bits as the oracle
+    N, K = 1024, 2560
+    W = inputs.latent_weights(N, K, seed=11)
+    KB = K // 128
+    for u in _sampled_units(N, K):
+        n, kb = divmod(int(u), KB)
+        W[n, kb * 128:(kb + 1) * 128] *= np.float32(1e-3)
+    r = _oracle_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
+    # and the other way round: sampled units 1000x larger
+    W = inputs.latent_weights(N, K, seed=12)
+    for u in _sampled_units(N, K):
+        n, kb = divmod(int(u), KB)
+        W[n, kb * 128:(kb + 1) * 128] *= np.float32(1e3)
+    r = _oracle_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
+
+
+@pytest.mark.parametrize("N,K", [(256, 512), (1024, 2560)])
+def test_quantize_mask_pack_everything_near_the_threshold(N, K):
+    # 15 of 16 groups keep two values within 1 % of half the scale (the rounding threshold), the
+    # 16th carries the mass that puts gamma there: nearly every kept value is undecided until the
+    # exact gamma is known.  The small case exercises a long fix-up list, the large one (139
+    # units = 8340 listed values per CTA) overflows the list and falls back to the second pass.
+    rng = np.random.default_rng(13)
+    a = np.float32(0.01)
+    G = N * K // 4
+    groups = np.zeros((G, 4), np.float32)
+    heavy = (np.arange(G) % 16) == 0
+    f = heavy.mean()
+    H = np.float32((3.0 + f) / f) * a
+    jitter = (1.0 + 0.01 * rng.uniform(-1, 1, size=(G, 2))).astype(np.float32)
+    sign = rng.choice(np.array([-1.0, 1.0], np.float32), size=(G, 2))
+    groups[:, 1:3] = a * jitter * sign
+    groups[heavy, 1:3] = H * sign[heavy]
+    groups[:, 0] = a * np.float32(1e-3)
+    W = groups.reshape(N, K)
+    r = _oracle_pack(W)
+    kept = r["vals"]
+    assert 0.2 < np.count_nonzero(kept) / kept.size < 0.8, "the construction should split the kept values"
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
 
 
 def test_worked_example_not_the_negative_control():
