@@ -21,24 +21,26 @@
 //                  each, 2 or 4 of them) at the top of the same 256-column half.  Accumulators are single-buffered: the MMA of the
 //                  next tile waits until the epilogue has drained TMEM into registers.
 //   warps          0 TMA producer (both CTAs), 1 MMA issuer (leader CTA only; both allocate
-//                  TMEM), 2..9 epilogue: warps 2-5 drain M-tile 0, warps 6-9 M-tile 1
+//                  TMEM), 2..17 epilogue: warp 2 + e drains M-tile (e >> 2) & 1, TMEM lane
+//                  quarter (2 + e) & 3, the even (e < 8) or odd 32-column chunks
 //   barriers       full[s]      leader's copy: 1 arrival (leader's expect_tx of BOTH CTAs' bytes),
 //                               both CTAs' TMA loads complete_tx on it
 //                  empty[s]     every CTA's own copy, arrived by tcgen05.commit multicast
 //                  acc_full     every CTA's own copy, commit multicast
-//                  acc_empty    leader's copy: 16 arrivals (8 epilogue warps x 2 CTAs)
+//                  acc_empty    leader's copy: 32 arrivals (16 epilogue warps x 2 CTAs)
 //
 // No TMA multicast is used: every CTA fetches its own boxes.  All waits are bounded.
 #pragma once
+
+#include <type_traits>
 
 #include "gemm_tcgen05.cuh"
 
 namespace sbn {
 
-constexpr int kPairThreads = 320;
-constexpr int kPairEpiWarps = 8;
-constexpr int kPairSlabBytes = 2048;                              // 32 tok x 32 feat bf16 | 16 tok fp32
-constexpr int kPairEpiBytes = kPairEpiWarps * kPairSlabBytes;     // one slab per epilogue warp
+constexpr int kPairEpiWarps = 16;
+constexpr int kPairThreads = 32 * (2 + kPairEpiWarps);           // 576 threads, at most 96 registers each
+constexpr int kPairEpiBytes = 2 * 256 * 4;                        // per-token scales of the current and the next tile
 constexpr int kPairMaxBnSparse = 240;
 constexpr int kPairMaxBnDense = 256;
 
@@ -66,6 +68,27 @@ struct PairParams {
     GemmParams g;
     int bn;                       // tokens per tile
 };
+
+// int32 accumulator -> fp32, exactly.  The conversion instruction runs at a quarter of the ALU
+// rate and the epilogue needs one per output element, so while |acc| < 2^22 (always true for
+// K < 32768: |acc| <= 128 K) the integer is added into the mantissa of 1.5 * 2^23 and the
+// constant is subtracted again -- full-rate instructions, no rounding anywhere.  Two elements at
+// a time: the subtraction and the multiplication by s (Eq. 4) use the packed fp32x2 forms.
+template <bool SMALL>
+__device__ __forceinline__ void acc2_scaled(uint32_t a0, uint32_t a1, float s0, float s1, float& v0, float& v1) {
+    if constexpr (SMALL) {
+        uint64_t m, c, sc, d;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(m) : "r"(0x4B400000u + a0), "r"(0x4B400000u + a1));
+        asm("mov.b64 %0, {%1, %1};" : "=l"(c) : "r"(0xCB400000u));                 // -12582912.0f twice
+        asm("mov.b64 %0, {%1, %2};" : "=l"(sc) : "f"(s0), "f"(s1));
+        asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(m), "l"(c));
+        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(d), "l"(sc));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(v0), "=f"(v1) : "l"(d));
+    } else {
+        v0 = __fmul_rn(static_cast<float>(static_cast<int>(a0)), s0);
+        v1 = __fmul_rn(static_cast<float>(static_cast<int>(a1)), s1);
+    }
+}
 
 // ---- cluster / pair PTX ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -146,6 +169,120 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
 //   tmap_e  [N/128][KB * 2][1 KB]               box {1 KB, 2 * KBS, 2}          (sparse)
 //   tmap_b  [KB][TB8][1 KB]                     box {1 KB, BN/16, KBS}
 //   tmap_y  y [T][N]                            box {32 features, 32 (bf16) | 16 (fp32) tokens}
+// Epilogue of one pair tile for one warp, bf16 outputs (see the kernel for the scheme): phase A
+// drains this warp's chunks chunk0 + 2 k of the accumulator into packed registers and hands the
+// accumulator back, phase B stores them.
+template <bool SMALL>
+__device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, const int t0, const int n, const float bias,
+                                                        const int live, const int full32, const uint32_t t_addr,
+                                                        const float* sc_tile, const int lane, const int chunk0,
+                                                        const uint32_t acc_empty_leader) {
+    uint32_t packed[4][16];
+    const bool has_bias = p.bias != nullptr;
+    // ---- phase A
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int i = chunk0 + 2 * k;
+        if (i < live) {
+            const bool half_chunk = (i == full32);                 // the 16-wide tail
+            // 16 columns at a time: the tile's packed outputs take most of the registers
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (h == 0 || !half_chunk) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>(i * 32 + h * 16), r);
+                    const float2* sc2 = reinterpret_cast<const float2*>(sc_tile + i * 32 + h * 16);   // uniform reads
+                    tmem_ld_wait();
+                    if (i + 2 >= live && (h == 1 || half_chunk)) {
+                        // last TMEM read of this warp is complete: hand the accumulator back
+                        tcgen05_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; j += 2) {
+                        float v0, v1;
+                        const float2 sq = sc2[j >> 1];
+                        acc2_scaled<SMALL>(r[j], r[j + 1], sq.x, sq.y, v0, v1);
+                        if (has_bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); }
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed[k][(h * 16 + j) >> 1]) : "f"(v1), "f"(v0));
+                    }
+                }
+            }
+        }
+    }
+    // ---- phase B
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int i = chunk0 + 2 * k;
+        if (i < live) {
+            const int tc = t0 + i * 32;
+            const int cnt = min(p.T - tc, (i == full32) ? 16 : 32);   // live tokens of the chunk (warp-uniform)
+            uint16_t* y = static_cast<uint16_t*>(p.y) + static_cast<size_t>(tc) * p.N + n;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                const uint32_t pk = packed[k][j >> 1];
+                if (j < cnt) y[0] = static_cast<uint16_t>(pk & 0xFFFFu);
+                if (j + 1 < cnt) y[p.N] = static_cast<uint16_t>(pk >> 16);
+                y += 2 * static_cast<size_t>(p.N);             // running pointer: no table of 32 row addresses
+            }
+        }
+    }
+}
+
+// The same for fp32 outputs and / or the raw accumulator dump: these do not fit in registers and
+// are stored while the accumulator drains.
+template <bool SMALL>
+__device__ __forceinline__ void pair_epilogue_tile_direct(const GemmParams& p, const int t0, const int n, const float bias,
+                                                          const int live, const int full32, const uint32_t t_addr,
+                                                          const float* sc_tile, const int lane, const int chunk0,
+                                                          const uint32_t acc_empty_leader) {
+#pragma unroll 1
+    for (int i = chunk0; i < live; i += 2) {
+        const bool half_chunk = (i == full32);
+        const int tc = t0 + i * 32;
+        const int cnt = min(p.T - tc, half_chunk ? 16 : 32);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (h == 0 || !half_chunk) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>(i * 32 + h * 16), r);
+                const float2* sc2 = reinterpret_cast<const float2*>(sc_tile + i * 32 + h * 16);
+                tmem_ld_wait();
+                if (i + 2 >= live && (h == 1 || half_chunk)) {
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const int jj = h * 16 + j;                    // token inside the chunk
+                    const size_t off = static_cast<size_t>(tc + jj) * p.N + n;
+                    if (p.acc_out) {
+                        if (jj < cnt) p.acc_out[off] = static_cast<int>(r[j]);
+                        if (jj + 1 < cnt) p.acc_out[off + p.N] = static_cast<int>(r[j + 1]);
+                    }
+                    float v0, v1;
+                    const float2 sq = sc2[j >> 1];
+                    acc2_scaled<SMALL>(r[j], r[j + 1], sq.x, sq.y, v0, v1);
+                    if (p.bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); }
+                    if (p.out_bf16) {
+                        uint32_t pk;
+                        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(v1), "f"(v0));
+                        uint16_t* y = static_cast<uint16_t*>(p.y) + off;
+                        if (jj < cnt) y[0] = static_cast<uint16_t>(pk & 0xFFFFu);
+                        if (jj + 1 < cnt) y[p.N] = static_cast<uint16_t>(pk >> 16);
+                    } else {
+                        float* y = static_cast<float*>(p.y) + off;
+                        if (jj < cnt) y[0] = v0;
+                        if (jj + 1 < cnt) y[p.N] = v1;
+                    }
+                }
+            }
+        }
+    }
+}
+
 template <bool SPARSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -318,24 +455,35 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (8 warps)
-        // The accumulators are single-buffered, so the time from "accumulator complete" to "all
-        // warps have pulled their columns into registers" is exposed.  To keep it short: the
-        // per-token scales are fetched into registers BEFORE waiting for the accumulator, TMEM
-        // loads run one 32-column chunk ahead of the arithmetic, values are converted in
-        // registers while the previous chunk's TMA store is still reading the slab, and a chunk
-        // costs one fence + one TMA store (bf16) or two (fp32).  Every warp works on its own
-        // (private slab, private stores): sharing one slab per M-tile between four warps was
-        // measured slower because of the hand-over between warps.
-        const int ew = warp - 2;                          // 0..7
-        const int mtile = ew >> 2;                        // which M-tile this warp drains
+        // ------------------------------------------------------------------ epilogue (16 warps)
+        // The accumulators are single-buffered, so the time from "accumulator complete" to
+        // "accumulator handed back" is exposed -- and a B200 takes writes at ~3.5 TB/s in total
+        // (a plain memset runs at that rate), 24 GB/s per SM: a CTA that stores its 120 KB of
+        // bf16 outputs while it drains needs ~5 us, whatever the instruction stream looks like,
+        // because all CTAs reach the end of their tiles together.  So the drain does not store:
+        //   phase A   TMEM -> registers, scale (Eq. 4), convert, keep the tile's outputs PACKED
+        //             IN REGISTERS (bf16: 4 chunks x 32 tokens = 64 registers per thread), hand the
+        //             accumulator back -- only arithmetic, ~1.5 us;
+        //   phase B   store them while the next tile's MMAs run.
+        // Two warps per (M-tile, TMEM lane quarter) take the even / the odd 32-column chunks.
+        // A thread owns one output feature (TMEM lane) and 32 tokens of a chunk; y is token-major,
+        // so it stores 2 B per token and the warp's 32 lanes make that a contiguous 64 B piece of
+        // the token's row -- no transposition, no shared memory.  The per-token scales of the tile
+        // are staged in shared memory once per tile and read with uniform 16 B loads.
+        // fp32 outputs (and the raw accumulator dump) do not fit in registers: they are stored
+        // from phase A directly.
+        const int ew = warp - 2;                          // 0..15
         const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
+        const int mtile = (ew >> 2) & 1;                  // which M-tile this warp drains
+        const int chunk0 = ew >> 3;                       // chunks chunk0, chunk0 + 2, chunk0 + 4, chunk0 + 6
+        static_assert(kPairEpiWarps == 16, "chunk assignment assumes two warps per lane quarter and M-tile");
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const float w_scale = __ldg(p.w_scale);
-        const uint32_t slab_u32 = smem_epi + static_cast<uint32_t>(ew * kPairSlabBytes);
-        uint8_t* const slab_ptr = smem_raw + (slab_u32 - smem_u32(smem_raw));
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
-        const int chunks = (BN + 31) >> 5;                // 32-column chunks; the last one may be 16 wide
+        const bool small_acc = k_blocks < 256;            // |acc| <= 128 K < 2^22
+        float* const s_scale = reinterpret_cast<float*>(smem_raw + (smem_epi - smem_base));   // [2][256]
+        const int et = threadIdx.x - 64;                  // 0..511 among the epilogue threads
+        uint32_t tile_par = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
@@ -346,127 +494,37 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const int t0 = tt * BN;
             const bool rows_valid = n0 < p.N;             // warp-uniform (N % 128 == 0)
             const float bias = (p.bias && rows_valid) ? __ldg(p.bias + n) : 0.0f;
-            // s absorbs both scales (Eq. 4): lane l keeps w_scale * a_scale of tokens t0 + 32 i + l
-            float my_scale[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int t = t0 + i * 32 + lane;
-                my_scale[i] = (i < chunks && t < p.T) ? __fmul_rn(w_scale, __ldg(p.a_scale + t)) : 0.0f;
-            }
+            // number of 32-column chunks that hold at least one real token (warp-uniform)
+            const int live = rows_valid ? (min(p.T - t0, BN) + 31) >> 5 : 0;
+            // a 16-wide last chunk (BN % 32 == 16) is read with a 16-column load: the columns above
+            // it hold metadata
+            const int full32 = BN >> 5;
+            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(mtile * 256);
+            // s of Eq. 4 for the tile's tokens, shared by all epilogue warps (double-buffered over
+            // tiles: one named barrier per tile orders the fill against every reader)
+            float* const sc_tile = s_scale + tile_par * 256;
+            if (et < BN) sc_tile[et] = (t0 + et < p.T) ? __fmul_rn(w_scale, __ldg(p.a_scale + t0 + et)) : 0.0f;
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kPairEpiWarps) : "memory");
+            tile_par ^= 1u;
             if (!mbar_wait(bar_acc_full, acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
-            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(mtile * 256);
-            // number of chunks that hold at least one real token (warp-uniform)
-            const int live = rows_valid ? (min(p.T - t0, BN) + 31) >> 5 : 0;      // <= chunks
-            // a 16-wide last chunk (BN % 32 == 16) is read with a 16-column load: the columns above
-            // it hold metadata; its 16 tokens go out with plain stores (bf16) / one 16-token slab
-            const int full32 = BN >> 5;
-            uint32_t ra[32], rb[32];
-            if (live > 0) {
-                if (full32 > 0) tmem_ld_32x32b_x32(t_addr, ra);
-                else tmem_ld_32x32b_x16(t_addr, reinterpret_cast<uint32_t (&)[16]>(ra));
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (i < live) {
-                    uint32_t (&cur)[32] = (i & 1) ? rb : ra;
-                    uint32_t (&nxt)[32] = (i & 1) ? ra : rb;
-                    const bool half_chunk = (i == full32);                 // the 16-wide tail
-                    tmem_ld_wait();                                       // chunk i is in registers
-                    if (i + 1 < live) {
-                        if (i + 1 < full32) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>((i + 1) * 32), nxt);
-                        else tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>((i + 1) * 32), reinterpret_cast<uint32_t (&)[16]>(nxt));
-                    }
-                    if (i + 1 == live) {
-                        // last TMEM read of this warp is complete: hand the accumulator back
-                        tcgen05_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
-                    }
-                    const int tc = t0 + i * 32;
-                    const int t_lim = min(p.T, tc + (half_chunk ? 16 : 32));  // tokens of this chunk end here
-                    if (p.acc_out) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int t = tc + j;
-                            if (t < t_lim) p.acc_out[static_cast<size_t>(t) * p.N + n] = static_cast<int>(cur[j]);
-                        }
-                    }
-                    if (p.out_bf16 && half_chunk) {
-                        // 16-token tail: plain 2-byte stores, 64 contiguous bytes per warp and token
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float sc = __shfl_sync(0xFFFFFFFFu, my_scale[i], j);
-                            float v = __fmul_rn(static_cast<float>(static_cast<int>(cur[j])), sc);
-                            if (p.bias) v = __fadd_rn(v, bias);
-                            const int t = tc + j;
-                            if (t < t_lim) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-                        }
-                    } else if (p.out_bf16) {
-                        // convert in registers (two tokens per word), then one 32 x 32 bf16 slab
-                        uint32_t packed[16];
-#pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            const float s0 = __shfl_sync(0xFFFFFFFFu, my_scale[i], j);
-                            const float s1 = __shfl_sync(0xFFFFFFFFu, my_scale[i], j + 1);
-                            float v0 = __fmul_rn(static_cast<float>(static_cast<int>(cur[j])), s0);
-                            float v1 = __fmul_rn(static_cast<float>(static_cast<int>(cur[j + 1])), s1);
-                            if (p.bias) { v0 = __fadd_rn(v0, bias); v1 = __fadd_rn(v1, bias); }
-                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed[j >> 1]) : "f"(v1), "f"(v0));
-                        }
-                        // the slab's previous contents must have been read by their TMA store
-                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                        __syncwarp();
-                        uint16_t* o = reinterpret_cast<uint16_t*>(slab_ptr) + lane;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            o[(2 * j) * 32] = static_cast<uint16_t>(packed[j] & 0xFFFFu);
-                            o[(2 * j + 1) * 32] = static_cast<uint16_t>(packed[j] >> 16);
-                        }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(&tmap_y, n0, tc, slab_u32);
-                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                        }
-                    } else {
-                        // two 16-token x 32-feature fp32 slabs through the same 2 KB buffer
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            if (tc + h * 16 < t_lim) {
-                                float v[16];
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) {
-                                    const float sc = __shfl_sync(0xFFFFFFFFu, my_scale[i], h * 16 + j);
-                                    v[j] = __fmul_rn(static_cast<float>(static_cast<int>(cur[h * 16 + j])), sc);
-                                    if (p.bias) v[j] = __fadd_rn(v[j], bias);
-                                }
-                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                                __syncwarp();
-                                float* o = reinterpret_cast<float*>(slab_ptr) + lane;
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) o[j * 32] = v[j];
-                                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                                __syncwarp();
-                                if (lane == 0) {
-                                    tma_store_2d(&tmap_y, n0, tc + h * 16, slab_u32);
-                                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-            if (live == 0) {
+
+            // bf16 outputs stay in registers until phase B (K >= 32768 takes the plain route: its
+            // int32 -> fp32 conversion needs the slow instruction and more registers)
+            const bool keep = p.out_bf16 && !p.acc_out && small_acc;
+            if (chunk0 >= live) {
                 // nothing to read (rows or tokens beyond the matrix): still release the accumulator
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+            } else if (keep) {
+                pair_epilogue_tile_bf16<true>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
+            } else {
+                if (small_acc) pair_epilogue_tile_direct<true>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
+                else pair_epilogue_tile_direct<false>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
             }
             acc_phase ^= 1u;
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        __syncwarp();
     }
 
     // teardown: nobody leaves while the peer may still touch this CTA's smem, barriers or TMEM
