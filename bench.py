@@ -34,6 +34,10 @@ from paper_2603_05168_b200 import inputs  # noqa: E402
 DATASHEET_INT8_DENSE_TOPS = 4500.0
 DATASHEET_INT8_SPARSE_TOPS = 9000.0
 NOMINAL_BF16_DENSE_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the sparse GEMM per launch, from one ncu capture of
+# this bench's step (mean over the step's GEMM launches; the outputs mostly stay in L2, so this is far
+# below the algorithmic operand + output bytes -- the kernel is tensor-bound, the figure is context).
+GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 26.0e6, "down7b": 228.4e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -417,7 +421,8 @@ def run_ours(args):
         peak = peaks["bf16_tflops"] * ratio
         achieved = sum(L.ops for L in layers) / (tot[dominant] * 1e-6) / 1e12
         roofline = {"bound": "tensor", "kernel": "bitlinear_gemm_kernel<sparse>", "achieved": round(achieved, 1),
-                    "peak": round(peak, 1), "unit": "TOP/s", "frac": round(achieved / peak, 4), "traffic": None,
+                    "peak": round(peak, 1), "unit": "TOP/s", "frac": round(achieved / peak, 4),
+                    "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(args.workload),
                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {ratio:g} (nominal sparse-int8 : bf16)",
                     "frac_of_datasheet_sparse_int8": round(achieved / DATASHEET_INT8_SPARSE_TOPS, 4)}
     else:
