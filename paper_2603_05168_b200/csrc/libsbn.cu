@@ -92,8 +92,6 @@ static inline bool misaligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
 }
 
-static inline bool use_pair_kernel_fwd(int T);
-
 static inline int pick_token_tile(int T) {
     if (g_force_token_tile == 64 || g_force_token_tile == 128 || g_force_token_tile == 256)
         return g_force_token_tile;
@@ -122,12 +120,18 @@ static size_t split_acc_bytes(int T, int N) {
     return (static_cast<size_t>(T) * N * sizeof(int32_t) + 255) & ~static_cast<size_t>(255);
 }
 
-static size_t gemm_workspace_bytes(int T, int N, int K) {
+struct GemmPlan {
+    bool pair;      // CTA-pair kernel (two M-tiles per CTA) or single-CTA tiles
+    int bn;         // token tile
+    int splits;     // split-K factor (single-CTA kernel only)
+};
+static GemmPlan plan_gemm(bool sparse, int T, int N, int K);
+
+static size_t gemm_workspace_bytes(bool sparse, int T, int N, int K) {
     // split-K scratch: int32 [T][N] + one counter per output tile; only the small-T regime splits
-    if (use_pair_kernel_fwd(T)) return 0;
-    const int bn = pick_token_tile(T);
-    if (pick_split_k(T, N, K, bn) > 1)
-        return split_acc_bytes(T, N) + static_cast<size_t>(N / kBM) * ((T + bn - 1) / bn) * sizeof(unsigned int);
+    const GemmPlan plan = plan_gemm(sparse, T, N, K);
+    if (!plan.pair && plan.splits > 1)
+        return split_acc_bytes(T, N) + static_cast<size_t>(N / kBM) * ((T + plan.bn - 1) / plan.bn) * sizeof(unsigned int);
     return 0;
 }
 
@@ -206,18 +210,57 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
-static inline bool use_pair_kernel(int T) {
-    if (g_force_token_tile < 0) return true;
-    if (g_force_token_tile > 0) return false;
-    return T >= 256;
+// Which kernel, which token tile, whether to split K: a small model of the measured times (us).
+//   single-CTA kernel   F(bn) + waves * (K/128 / splits) * c(bn)  [+ split-K: 1 + 8e-6 per atomic]
+//                       F = 3.0 + 0.02 bn (prologue + last epilogue), c = 0.23 (bn <= 128) | 0.275 (256)
+//   CTA-pair kernel     4.3 + 0.02 bn + waves * K/128 * 0.31 + (waves - 1) * 2.5 (exposed drains)
+// waves over 148 CTAs resp. 74 pairs.  Small problems are latency-bound and favour many small
+// single-CTA tiles; large ones favour the pair kernel's operand reuse.  K is split only when the
+// tiles cannot fill the machine and the int32 atomics cost less than the K-loop they save.
+static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
+    GemmPlan best = {false, 64, 1};
+    const int kb = K / kBK;
+    const int rows = N / kBM;
+    if (g_force_token_tile < 0) return GemmPlan{true, pick_pair_bn(sparse, T, N, K), 1};
+    if (g_force_token_tile > 0 || g_force_split_k > 0) {        // diagnostics: single-CTA kernel as told
+        const int bn = pick_token_tile(T);
+        return GemmPlan{false, bn, pick_split_k(T, N, K, bn)};
+    }
+    const double mm = sparse ? 1.0 : 1.3;                       // dense K-loop relative to sparse
+    double best_t = 1e300;
+    auto consider = [&](const GemmPlan& g, double t) { if (t < best_t) { best_t = t; best = g; } };
+    const int bns[3] = {64, 128, 256};
+    for (int bn : bns) {
+        if (bn > 64 && T <= bn / 2) continue;                   // a tile mostly beyond T
+        const long tiles = static_cast<long>(rows) * ((T + bn - 1) / bn);
+        const double c = (bn == 256 ? 0.275 : 0.23) * mm;
+        const double F = 3.0 + 0.02 * bn;
+        const long waves = (tiles + kNumSMs - 1) / kNumSMs;
+        consider(GemmPlan{false, bn, 1}, F + waves * kb * c);
+        if (bn == 64 && tiles * 2 <= kNumSMs) {
+            // smallest split that gives at least ~100 units of work
+            int sp = static_cast<int>((100 + tiles - 1) / tiles);
+            if (sp > kb) sp = kb;
+            while (sp > 1 && kb % sp != 0) ++sp;                // next divisor upwards (kb divides itself)
+            if (sp > 1 && sp <= kb) {
+                const double atomics = 8e-6 * static_cast<double>(T) * N * sp;
+                consider(GemmPlan{false, bn, sp}, F + (kb / sp) * c + 1.0 + atomics);
+            }
+        }
+    }
+    {
+        const int bn = pick_pair_bn(sparse, T, N, K);
+        const long tiles = static_cast<long>((N + 511) / 512) * ((T + bn - 1) / bn);
+        const long waves = (tiles + kNumSMs / 2 - 1) / (kNumSMs / 2);
+        consider(GemmPlan{true, bn, 1}, 4.3 + 0.02 * bn + waves * kb * 0.31 * (sparse ? 1.0 : 1.4) + (waves - 1) * 2.5);
+    }
+    return best;
 }
-static inline bool use_pair_kernel_fwd(int T) { return use_pair_kernel(T); }
 
 static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_scale, int T,
                                 const int8_t* wvals, const uint8_t* meta, const float* w_scale,
                                 int N, int K, const float* bias, void* y, sbn_out_dtype dt,
-                                int32_t* acc_out, cudaStream_t stream) {
-    const int bn = pick_pair_bn(sparse, T, N, K);
+                                int32_t* acc_out, int bn, cudaStream_t stream) {
     CUtensorMap ta, tb, te, ty;
     bool ok;
     const uint64_t KBk = static_cast<uint64_t>(K) / kBK, NB = static_cast<uint64_t>(N) / kBM;
@@ -257,14 +300,15 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
         (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)))
         return SBN_ERR_ALIGN;
 
-    if (use_pair_kernel(T))
-        return run_gemm_pair(sparse, xq, a_scale, T, wvals, meta, w_scale, N, K, bias, y, dt, acc_out, stream);
+    const GemmPlan plan = plan_gemm(sparse, T, N, K);
+    if (plan.pair)
+        return run_gemm_pair(sparse, xq, a_scale, T, wvals, meta, w_scale, N, K, bias, y, dt, acc_out, plan.bn, stream);
 
-    const int bn = pick_token_tile(T);
-    const int splits = pick_split_k(T, N, K, bn);
+    const int bn = plan.bn;
+    const int splits = plan.splits;
     if (splits > 1) {
         // scratch is zero on entry (caller's duty before the first use) and the kernel re-zeroes it
-        const size_t need = gemm_workspace_bytes(T, N, K);
+        const size_t need = gemm_workspace_bytes(sparse, T, N, K);
         if (!ws || ws_bytes < need) return SBN_ERR_WORKSPACE;
         if (misaligned(ws, 16)) return SBN_ERR_ALIGN;
     }
@@ -351,7 +395,7 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K) {
         case SBN_OP_SPARSE_BITLINEAR:
         case SBN_OP_BITLINEAR:
             if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return 0;
-            return gemm_workspace_bytes(T, N, K);
+            return gemm_workspace_bytes(op == SBN_OP_SPARSE_BITLINEAR, T, N, K);
         default: return 0;
     }
 }
