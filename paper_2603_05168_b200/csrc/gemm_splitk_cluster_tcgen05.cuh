@@ -1,0 +1,267 @@
+// Eq. 4 for few tokens: split-K inside a thread-block cluster.
+//
+// With T up to a few hundred there are only N/128 x ceil(T/BN) output tiles -- far fewer than SMs --
+// and a CTA that walks the whole K of its tile is bound by what ONE SM can pull out of L2
+// (~100 GB/s: 18 KB per 128 columns -> 0.23 us each).  Splitting K over CTAs puts more SMs on the
+// weight stream; the partial accumulators then have to be added.  Through global memory that is
+// one int32 atomic per output element and slice, which costs more than the K-loop it saves once
+// T reaches 64.  Here the S CTAs that share an output tile form a CLUSTER and add their partial
+// accumulators through distributed shared memory:
+//
+//   CTA r of the cluster   k-blocks [r q, min((r+1) q, K/128)),  q = ceil(K/128 / S)
+//   mainloop               as in the single-CTA kernel (TMA producer warp, MMA issuer warp,
+//                          metadata through tcgen05.cp, one accumulator in TMEM)
+//   reduce-scatter         every CTA owns BN/S tokens of the tile; each epilogue thread (one output
+//                          feature = one TMEM lane) writes its partial sums of token j straight into
+//                          the shared memory of the CTA that owns j (st.shared::cluster), slot [r]
+//   barrier.cluster        (hardware barrier: nothing spins)
+//   finish                 every CTA adds the S partials of its tokens, applies s = w_scale *
+//                          a_scale[t] (+ bias) and stores y (and the int32 dump when asked for)
+//
+// No scratch in global memory, no atomics, nothing to keep zeroed; a CTA never touches a peer's
+// shared memory after the barrier, so CTAs leave independently.  All mbarrier waits are bounded.
+#pragma once
+
+#include "gemm_pair_tcgen05.cuh"
+
+namespace sbn {
+
+constexpr int kSplitThreads = 192;        // warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue
+constexpr int kSplitMaxCluster = 8;
+
+template <bool SPARSE, int BN>
+struct SplitConfig {
+    static constexpr int A_BYTES = SPARSE ? kBM * (kBK / 2) : kBM * kBK;
+    static constexpr int B_BYTES = BN * kBK;
+    static constexpr int E_BYTES = SPARSE ? kBM * (kBK / 8) : 0;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
+    static constexpr int STAGES = SPARSE ? 6 : 4;
+    static constexpr int REDUCE_BYTES = BN * kBM * 4;          // [S][BN/S tokens][128 features] int32
+    static constexpr int META_COL0 = BN;                        // metadata columns above the accumulator
+    static constexpr uint32_t TMEM_COLS = (BN + 4 * STAGES <= 64) ? 64 : (BN + 4 * STAGES <= 128 ? 128 : 256);
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + REDUCE_BYTES + kBarrierBytes;
+    static_assert(SMEM_BYTES <= 232448, "shared memory overflow");
+    static_assert(BN % 32 == 0 && BN <= 128, "token tile");
+};
+
+__device__ __forceinline__ void st_shared_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+
+template <bool SPARSE, int BN>
+__global__ void __launch_bounds__(kSplitThreads, 1)
+bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                                     const __grid_constant__ CUtensorMap tmap_b,
+                                     const __grid_constant__ CUtensorMap tmap_e,
+                                     const GemmParams p) {
+    using Cfg = SplitConfig<SPARSE, BN>;
+    constexpr int STAGES = Cfg::STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    // 1 KB alignment: required by the 128 B swizzle atoms; the offset is the same in every CTA of
+    // the cluster (same kernel, same static shared memory), so peers' buffers sit at the same offset
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_a = smem_base;
+    const uint32_t smem_b = smem_a + STAGES * Cfg::A_BYTES;
+    const uint32_t smem_e = smem_b + STAGES * Cfg::B_BYTES;
+    const uint32_t smem_red = smem_base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t bar_base = smem_red + Cfg::REDUCE_BYTES;
+    const uint32_t bar_full = bar_base;
+    const uint32_t bar_empty = bar_full + 8 * STAGES;
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;
+    const uint32_t tmem_slot = bar_acc_full + 8;
+
+    __shared__ int s_abort;
+    volatile int* abort_flag = &s_abort;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const uint32_t S = cluster_nctarank();
+    const int tile = blockIdx.x / static_cast<int>(S);          // clusters are consecutive blocks
+    const int tiles_m = p.N / kBM;
+    const int mt = tile % tiles_m;
+    const int tt = tile / tiles_m;
+    const int t0 = tt * BN;
+    const int q = (p.k_blocks_total + static_cast<int>(S) - 1) / static_cast<int>(S);
+    const int kb0 = min(p.k_blocks_total, static_cast<int>(rank) * q);
+    const int kb1 = min(p.k_blocks_total, kb0 + q);
+    const int tok_per_cta = BN / static_cast<int>(S);           // S is 2, 4 or 8 (host's duty): a power of two
+    const int tok_shift = __ffs(tok_per_cta) - 1;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+        tcgen05_fence_before();
+    }
+    __syncthreads();
+    tcgen05_fence_after();
+    // a peer's shared memory may only be written once that CTA has started: every thread arrives
+    // here and waits just before the scatter, so the barrier costs nothing on the way in
+    cluster_arrive();
+    pdl_wait();                          // nothing above touches global memory
+    pdl_launch_dependents();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    bool ok = true;
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmap_a);
+            tma_prefetch_desc(&tmap_b);
+            if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) break;
+                const uint32_t full = bar_full + 8 * stage;
+                mbar_expect_tx(full, Cfg::STAGE_BYTES);
+                const int wt = mt * p.k_blocks_total + kb;            // weight tile index
+                if constexpr (SPARSE) {
+                    tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 8, full);
+                    tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, 0, wt * 2, full);
+                } else {
+                    tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 16, full);
+                }
+                tma_load_2d(smem_b + stage * Cfg::B_BYTES, &tmap_b, 0, kb * p.tb8 + (t0 >> 3), full);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        __syncwarp();
+        cluster_wait();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && kb1 > kb0) {
+            constexpr uint32_t idesc = make_idesc_i8(kBM, BN, SPARSE);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool good = true;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { good = false; break; }
+                tcgen05_fence_after();
+                const uint32_t a_addr = smem_a + stage * Cfg::A_BYTES;
+                const uint32_t b_addr = smem_b + stage * Cfg::B_BYTES;
+                const uint32_t first = (kb == kb0) ? 0u : 1u;
+                if constexpr (SPARSE) {
+                    const uint32_t e_tmem = tmem_base + static_cast<uint32_t>(Cfg::META_COL0 + 4 * stage);
+                    const uint64_t e_desc = make_smem_desc(smem_e + stage * Cfg::E_BYTES, 128, 128, kSwzNone);
+                    tcgen05_cp_128x128b(e_tmem, e_desc);
+                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 512, kSwz64);
+                    const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
+#pragma unroll
+                    for (int j = 0; j < kBK / 64; ++j)
+                        mma_i8_sparse(tmem_base, a_desc + static_cast<uint64_t>(2 * j), b_desc + static_cast<uint64_t>(4 * j),
+                                      e_tmem + 2 * j, idesc, j == 0 ? first : 1u);
+                } else {
+                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024, kSwz128);
+                    const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
+#pragma unroll
+                    for (int j = 0; j < kBK / 32; ++j)
+                        mma_i8_dense(tmem_base, a_desc + static_cast<uint64_t>(2 * j), b_desc + static_cast<uint64_t>(2 * j),
+                                     idesc, j == 0 ? first : 1u);
+                }
+                tcgen05_commit(bar_empty + 8 * stage);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (good) tcgen05_commit(bar_acc_full);
+        }
+        __syncwarp();
+        cluster_wait();
+    } else {
+        // ------------------------------------------------------------------ epilogue, part 1: scatter
+        const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
+        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+        const int f = quarter * 32 + lane;                // feature inside the tile
+        const bool have = kb1 > kb0;                      // an empty K slice contributes zeros
+        if (have) {
+            ok = mbar_wait(bar_acc_full, 0u, abort_flag);
+            tcgen05_fence_after();
+        }
+        cluster_wait();                                   // all peers have started
+        // slot [rank][token % tok_per_cta][feature] in the owner's buffer
+        const uint32_t my_slot = smem_red + (rank * static_cast<uint32_t>(tok_per_cta)) * (kBM * 4) + static_cast<uint32_t>(f) * 4u;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            uint32_t r[32];
+            if (have && ok) {
+                tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(c * 32), r);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int tok = c * 32 + j;
+                const uint32_t owner = static_cast<uint32_t>(tok >> tok_shift);
+                const uint32_t local = my_slot + static_cast<uint32_t>(tok & (tok_per_cta - 1)) * (kBM * 4);
+                st_shared_cluster_u32(map_to_cta(local, owner), r[j]);
+            }
+        }
+        tcgen05_fence_before();
+    }
+    // s of Eq. 4 for the tokens this CTA finishes, fetched before the barrier (lane l: tokens l and
+    // l + 32 of its share) so that the finishing loop has no global load to wait for
+    float sc_a = 0.0f, sc_b = 0.0f;
+    if (warp >= 2) {
+        const float w_scale = __ldg(p.w_scale);
+        const int ta = t0 + static_cast<int>(rank) * tok_per_cta + lane;
+        if (lane < tok_per_cta && ta < p.T) sc_a = __fmul_rn(w_scale, __ldg(p.a_scale + ta));
+        if (lane + 32 < tok_per_cta && ta + 32 < p.T) sc_b = __fmul_rn(w_scale, __ldg(p.a_scale + ta + 32));
+    }
+
+    // every CTA's partials are in place (release / acquire at cluster scope)
+    __syncthreads();
+    cluster_sync_all();
+
+    if (warp >= 2) {
+        // ------------------------------------------------------------------ epilogue, part 2: finish my tokens
+        const int quarter = warp & 3;
+        const int f = quarter * 32 + lane;
+        const int n = mt * kBM + f;
+        const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
+        const int32_t* red = reinterpret_cast<const int32_t*>(smem_raw + (smem_red - smem_u32(smem_raw)));
+        const bool fine = (*abort_flag == 0);
+        const int t_first = t0 + static_cast<int>(rank) * tok_per_cta;
+        const int n_tok = fine ? min(tok_per_cta, p.T - t_first) : 0;          // warp-uniform
+        for (int j = 0; j < n_tok; ++j) {
+            const int t = t_first + j;
+            const float sc = __shfl_sync(0xFFFFFFFFu, j < 32 ? sc_a : sc_b, j & 31);
+            int acc = 0;
+            for (uint32_t s = 0; s < S; ++s) acc += red[(s * tok_per_cta + j) * kBM + f];
+            if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
+            float v = __fmul_rn(static_cast<float>(acc), sc);
+            if (p.bias) v = __fadd_rn(v, bias);
+            if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+            else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
+        }
+    }
+
+    // teardown
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tcgen05_fence_after();
+        tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace sbn

@@ -329,6 +329,30 @@ def test_gemm_parity_pair_kernel(sparse, T, N, K, bn):
     assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
 
 
+CLUSTER_CASES = [  # (T, N, K, token tile, cluster size): split-K reduced in distributed shared memory
+    (64, 256, 2560, 64, 4), (1, 128, 256, 64, 2), (7, 256, 640, 64, 4),      # 5 k-blocks over 4 CTAs: one empty slice
+    (100, 384, 6912, 64, 8), (130, 256, 1280, 128, 8), (200, 128, 384, 128, 2), (33, 512, 128, 64, 8),   # one k-block
+    (257, 256, 2560, 128, 4),
+]
+
+
+@pytest.mark.parametrize("sparse", [True, False])
+@pytest.mark.parametrize("T,N,K,tile,cluster", CLUSTER_CASES)
+def test_gemm_parity_cluster_split_k(sparse, T, N, K, tile, cluster):
+    r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=cluster + T)
+    b.sbn_set_gemm_tuning(tile, -cluster)
+    if sparse:
+        y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    else:
+        y_ref, acc_ref = oracle.bitlinear(xq_ref, s_ref, r["dense_q"], r["scale"])
+    y, acc = gpu_gemm(sparse, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    yb, _ = gpu_gemm(sparse, xq, a_scale, g["dev"], out_dtype=torch.bfloat16, want_acc=False)
+    ref_bits = oracle.f32_to_bf16_bits(y_ref).astype(np.int32)
+    assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
+
+
 @pytest.mark.parametrize("sparse", [True, False])
 @pytest.mark.parametrize("split", [2, 5, 10])
 def test_gemm_parity_split_k(sparse, split):
