@@ -163,12 +163,6 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
         : "r"(taddr) : "memory");
 }
 
-// ---------------------------------------------------------------------------------------------
-// Tensor maps (all over arrays of 1 KB rows of 128 x uint64, see layouts.cuh):
-//   tmap_a  [N/128][KB * rows_per_tile][1 KB]   box {1 KB, rows_per_tile * KBS, 2}
-//   tmap_e  [N/128][KB * 2][1 KB]               box {1 KB, 2 * KBS, 2}          (sparse)
-//   tmap_b  [KB][TB8][1 KB]                     box {1 KB, BN/16, KBS}
-//   tmap_y  y [T][N]                            box {32 features, 32 (bf16) | 16 (fp32) tokens}
 // Epilogue of one pair tile for one warp, bf16 outputs (see the kernel for the scheme): phase A
 // drains this warp's chunks chunk0 + 2 k of the accumulator into packed registers and hands the
 // accumulator back, phase B stores them.
@@ -283,12 +277,16 @@ __device__ __forceinline__ void pair_epilogue_tile_direct(const GemmParams& p, c
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tensor maps (all over arrays of 1 KB rows of 128 x uint64, see layouts.cuh):
+//   tmap_a  [N/128][KB * rows_per_tile][1 KB]   box {1 KB, rows_per_tile * KBS, 2}
+//   tmap_e  [N/128][KB * 2][1 KB]               box {1 KB, 2 * KBS, 2}          (sparse)
+//   tmap_b  [KB][TB8][1 KB]                     box {1 KB, BN/16, KBS}
 template <bool SPARSE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                            const __grid_constant__ CUtensorMap tmap_b,
                            const __grid_constant__ CUtensorMap tmap_e,
-                           const __grid_constant__ CUtensorMap tmap_y,
                            const PairParams pp) {
     using Cfg = PairConfig<SPARSE>;
     constexpr int STAGES = Cfg::STAGES;

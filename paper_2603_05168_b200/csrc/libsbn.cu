@@ -197,7 +197,7 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
 
 template <bool SPARSE>
 static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
-                              const CUtensorMap& ty, const PairParams& pp, cudaStream_t stream) {
+                              const PairParams& pp, cudaStream_t stream) {
     using Cfg = PairConfig<SPARSE>;
     static bool configured = false;
     auto kernel = bitlinear_gemm_pair_kernel<SPARSE>;
@@ -208,7 +208,7 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
     }
     const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
     const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
-    const cudaError_t err = launch_kernel(kernel, dim3(2 * pairs), dim3(kPairThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, ty, pp);
+    const cudaError_t err = launch_kernel(kernel, dim3(2 * pairs), dim3(kPairThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, pp);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -282,7 +282,7 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
                                 const int8_t* wvals, const uint8_t* meta, const float* w_scale,
                                 int N, int K, const float* bias, void* y, sbn_out_dtype dt,
                                 int32_t* acc_out, int bn, cudaStream_t stream) {
-    CUtensorMap ta, tb, te, ty;
+    CUtensorMap ta, tb, te;
     bool ok;
     const uint64_t KBk = static_cast<uint64_t>(K) / kBK, NB = static_cast<uint64_t>(N) / kBM;
     if (sparse) {
@@ -294,7 +294,6 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
         ok = encode_3d_1k(&ta, wvals, KBk * 16, NB, 16 * kbs, 2) && encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
         te = ta;
     }
-    ok = ok && encode_2d_out(&ty, y, N, T, dt == SBN_OUT_BF16, dt == SBN_OUT_BF16 ? 32 : 16);
     if (!ok) return SBN_ERR_CUDA;
     PairParams pp;
     pp.g.T = T; pp.g.N = N; pp.g.K = K;
@@ -306,7 +305,7 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.acc_out = acc_out;
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.bn = bn;
-    return sparse ? launch_pair<true>(ta, tb, te, ty, pp, stream) : launch_pair<false>(ta, tb, te, ty, pp, stream);
+    return sparse ? launch_pair<true>(ta, tb, te, pp, stream) : launch_pair<false>(ta, tb, te, pp, stream);
 }
 
 template <bool SPARSE, int BN>
