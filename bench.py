@@ -341,13 +341,19 @@ def run_ours(args):
         return
 
     # ---- end-to-end: host buffers, copies inside the timed region ----------------------------------
+    # Layers alternate between two streams, so the device-to-host copy of one layer's y runs while
+    # the next layer's W and x come in (the link is full duplex); each layer has its own staging
+    # buffers, and a layer always uses the same stream, which orders its reuse across steps.
+    e2e_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+
     def e2e_step():
-        for L in layers:
+        for i, L in enumerate(layers):
             p = L.packed
-            L.W_stage.copy_(L.W_host, non_blocking=True)
-            b.sbn_quantize_mask_pack(L.W_stage, p["vals"], p["meta"], p["w_scale"], p["ws"])
-            b.sbn_layer_forward_host(L.x_host, L.x_stage, L.xq, L.a_scale, p["w_scale"], L.y, L.y_host,
-                                     vals=p["vals"], meta=p["meta"], ws=L.ws)
+            with torch.cuda.stream(e2e_streams[i % 2]):
+                L.W_stage.copy_(L.W_host, non_blocking=True)
+                b.sbn_quantize_mask_pack(L.W_stage, p["vals"], p["meta"], p["w_scale"], p["ws"])
+                b.sbn_layer_forward_host(L.x_host, L.x_stage, L.xq, L.a_scale, p["w_scale"], L.y, L.y_host,
+                                         vals=p["vals"], meta=p["meta"], ws=L.ws)
     e2e_steps = max(2, min(args.steps, 5))
     for _ in range(2):
         e2e_step()
@@ -355,8 +361,14 @@ def run_ours(args):
     s2 = torch.cuda.Event(enable_timing=True)
     e2 = torch.cuda.Event(enable_timing=True)
     s2.record(stream)
+    for st in e2e_streams:
+        st.wait_event(s2)
     for _ in range(e2e_steps):
         e2e_step()
+    for st in e2e_streams:
+        done_ev = torch.cuda.Event()
+        done_ev.record(st)
+        stream.wait_event(done_ev)
     e2.record(stream)
     barrier()
     b.sbn_check_status()
