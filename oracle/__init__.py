@@ -53,6 +53,7 @@ def _load():
             "sbn_oracle_unpack24": (None, [vp, vp, i64, i64, vp, vp]),
             "sbn_oracle_quantize_mask_pack": (i32, [vp, i64, i64, vp, vp, vp, vp, vp, vp]),
             "sbn_oracle_quant_act": (None, [vp, i64, i64, vp, vp]),
+            "sbn_oracle_norm_quant_act": (None, [vp, i64, i64, vp, f32, vp, vp, vp, vp]),
             "sbn_oracle_acc_dense": (None, [vp, vp, i64, i64, i64, vp]),
             "sbn_oracle_acc_packed": (None, [vp, vp, vp, i64, i64, i64, vp]),
             "sbn_oracle_acc_packed_sampled": (None, [vp, vp, vp, i64, i64, vp, vp, i64, vp]),
@@ -181,6 +182,23 @@ def quant_act(x_bf16_bits):
     a_scale = np.zeros(T, np.float32)
     _load().sbn_oracle_quant_act(_p(x), T, K, _p(xq), _p(a_scale))
     return xq, a_scale
+
+
+def norm_quant_act(x_bf16_bits, g=None, eps=1e-6, want_xn=False):
+    """Algorithm 1's x~ = Q_a(Norm(x)), Norm read as RMSNorm with gain g (None = ones).
+    Returns dict(xq int8 [T][K], a_scale fp32 [T], near_tie bool [T][, xn fp32 [T][K]])."""
+    x = _c(x_bf16_bits, np.uint16)
+    T, K = x.shape
+    gg = None if g is None else _c(g, np.float32)
+    xq = np.zeros((T, K), np.int8)
+    a_scale = np.zeros(T, np.float32)
+    near = np.zeros(T, np.uint8)
+    xn = np.zeros((T, K), np.float32) if want_xn else None
+    _load().sbn_oracle_norm_quant_act(_p(x), T, K, _p(gg), ctypes.c_float(eps), _p(xq), _p(a_scale), _p(xn), _p(near))
+    out = dict(xq=xq, a_scale=a_scale, near_tie=near.astype(bool))
+    if want_xn:
+        out["xn"] = xn
+    return out
 
 
 # -- Eq. 4 ---------------------------------------------------------------------------------------

@@ -241,6 +241,73 @@ void sbn_oracle_quant_act(const uint16_t *x_bf16, int64_t T, int64_t K,
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * Algorithm 1, forward step  x~ = Q_a(Norm(x)).  The paper does not say which norm; it is read as
+ * RMSNorm with a learned per-channel gain g (the norm BitNet-style blocks put in front of every
+ * quantised linear layer):
+ *     ms = mean_k x[k]^2            (double accumulation, one cast to float)
+ *     r  = 1 / sqrt(ms + eps)       (float)
+ *     xn[k] = (x[k] * r) * g[k]     (float, two rounded products; g == NULL means g = 1)
+ * followed by Q_a of Sec. 2.1 on the float xn (no rounding to bf16 in between: the two steps are
+ * one operation here).  near_tie[t] (optional) is set when a pairwise summation of the squares
+ * gives a different float ms for row t; xn_out (optional) receives the normalised row.
+ * ------------------------------------------------------------------------------------------- */
+static double pairwise_sq_sum(const uint16_t *x, int64_t n)
+{
+    if (n <= 64) {
+        double s = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            double v = (double)bf16_bits_to_f32(x[i]);
+            s += v * v;
+        }
+        return s;
+    }
+    int64_t h = n / 2;
+    return pairwise_sq_sum(x, h) + pairwise_sq_sum(x + h, n - h);
+}
+
+void sbn_oracle_norm_quant_act(const uint16_t *x_bf16, int64_t T, int64_t K, const float *g,
+                               float eps, int8_t *xq, float *a_scale, float *xn_out,
+                               uint8_t *near_tie)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *x = x_bf16 + t * K;
+        double S = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            double v = (double)bf16_bits_to_f32(x[k]);
+            S += v * v;
+        }
+        float ms = (float)(S / (double)K);
+        if (near_tie) near_tie[t] = ((float)(pairwise_sq_sum(x, K) / (double)K) != ms);
+        volatile float den = ms + eps;
+        volatile float root = sqrtf(den);
+        volatile float r = 1.0f / root;
+        float *xn = (float *)malloc((size_t)K * sizeof(float));
+        float a = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            volatile float p1 = bf16_bits_to_f32(x[k]) * r;
+            volatile float p2 = g ? p1 * g[k] : p1;
+            xn[k] = p2;
+            float v = fabsf(p2);
+            if (v > a) a = v;
+        }
+        float d = (a > SBN_ORACLE_EPS) ? a : SBN_ORACLE_EPS;
+        volatile float s_x = 127.0f / d;
+        for (int64_t k = 0; k < K; ++k) {
+            volatile float p = xn[k] * s_x;
+            float q = rintf(p);
+            if (q > 127.0f) q = 127.0f;
+            if (q < -128.0f) q = -128.0f;
+            xq[t * K + k] = (int8_t)q;
+            if (xn_out) xn_out[t * K + k] = xn[k];
+        }
+        volatile float as = d / 127.0f;
+        a_scale[t] = as;
+        free(xn);
+    }
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Eq. 4, integer part, route (i): acc[t][n] = sum_k x~[t][k] * Wmat[n][k] with Wmat a plain
  * dense [N][K] int8 matrix (W_eff for the sparse layer, W_q for the dense BitLinear baseline).
  * ------------------------------------------------------------------------------------------- */

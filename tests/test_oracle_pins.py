@@ -370,3 +370,87 @@ def test_flip_rate_of_the_dynamic_mask_workload():
     Wp = inputs.perturb_weights(W, seed=18, sigma=1e-4)
     r = oracle.flip_count(oracle.nm_mask(W), oracle.nm_mask(Wp)) / W.size
     assert 2.5e-3 < r < 4.5e-3
+
+
+# ------------------------------------------------------------------------------------------------
+# Algorithm 1: x~ = Q_a(Norm(x)), Norm read as RMSNorm with gain g.
+# ------------------------------------------------------------------------------------------------
+def _bf16_bits(a):
+    return inputs.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def _bits_to_f64(bits):
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def test_norm_quant_act_reduces_to_quant_act_on_unit_rms_rows():
+    # rows of +-1 have mean square exactly 1: with eps = 0 and no gain Norm is the identity, and the
+    # result must be the (separately pinned) activation quantiser's, bit for bit
+    rng = np.random.default_rng(21)
+    x = _bf16_bits(rng.choice(np.array([-1.0, 1.0], np.float32), size=(7, 384)))
+    r = oracle.norm_quant_act(x, None, 0.0)
+    xq, s = oracle.quant_act(x)
+    assert np.array_equal(r["xq"], xq) and np.array_equal(r["a_scale"], s)
+    assert set(np.unique(r["xq"]).tolist()) == {-127, 127}
+    assert np.all(r["a_scale"] == np.float32(1.0) / np.float32(127.0))
+
+
+def test_norm_quant_act_ignores_power_of_four_scaling():
+    # x -> 4x: the mean square is multiplied by 16 exactly, its root by 4 exactly, so with eps = 0 the
+    # normalised row -- hence codes and scale -- must not change at all
+    x = inputs.activations_bf16(9, 640, seed=22)
+    x4 = _bf16_bits(_bits_to_f64(x) * 4.0)
+    a = oracle.norm_quant_act(x, None, 0.0, want_xn=True)
+    c = oracle.norm_quant_act(x4, None, 0.0, want_xn=True)
+    assert np.array_equal(a["xn"], c["xn"])
+    assert np.array_equal(a["xq"], c["xq"]) and np.array_equal(a["a_scale"], c["a_scale"])
+
+
+def test_norm_quant_act_gain():
+    x = inputs.activations_bf16(6, 512, seed=23)
+    base = oracle.norm_quant_act(x, None, 1e-6)
+    half = oracle.norm_quant_act(x, np.full(512, 0.5, np.float32), 1e-6)
+    # a power-of-two gain on every channel scales the row exactly: same codes, half the scale
+    assert np.array_equal(half["xq"], base["xq"])
+    assert np.array_equal(half["a_scale"], base["a_scale"] * np.float32(0.5))
+    # a channel with gain 0 quantises to 0; a channel with a dominant gain takes the code +-127
+    g = np.ones(512, np.float32)
+    g[5] = 0.0
+    g[9] = 1000.0
+    r = oracle.norm_quant_act(x, g, 1e-6)
+    assert np.all(r["xq"][:, 5] == 0)
+    assert np.all(np.abs(r["xq"][:, 9].astype(np.int32)) == 127)
+
+
+def test_norm_quant_act_against_float64():
+    T, K = 11, 768
+    x = inputs.activations_bf16(T, K, seed=24, token_lognormal_sigma=0.5)
+    g = (1.0 + 0.1 * np.random.default_rng(25).standard_normal(K)).astype(np.float32)
+    eps = 1e-5
+    r = oracle.norm_quant_act(x, g, eps, want_xn=True)
+    xf = _bits_to_f64(x)
+    xn = xf / np.sqrt((xf ** 2).mean(axis=1, keepdims=True) + eps) * g.astype(np.float64)
+    assert np.max(np.abs(r["xn"] - xn) / np.maximum(np.abs(xn), 1e-30)) < 4e-7      # three fp32 roundings
+    d = np.maximum(np.abs(xn).max(axis=1, keepdims=True), 1e-5)
+    p = xn * (127.0 / d)
+    code = np.clip(np.rint(p), -128, 127)
+    safe = np.abs(np.abs(p - np.floor(p)) - 0.5) > 1e-3          # away from a rounding boundary
+    assert safe.mean() > 0.99
+    assert np.array_equal(r["xq"][safe], code[safe].astype(np.int8))
+    assert np.max(np.abs(r["xq"].astype(np.float64) - code)) <= 1
+    assert np.allclose(r["a_scale"], (d / 127.0).ravel(), rtol=1e-6)
+    assert not r["near_tie"].any()
+
+
+def test_norm_quant_act_degenerate_rows():
+    x = np.zeros((3, 256), np.uint16)                              # all-zero rows: eps keeps r finite
+    r = oracle.norm_quant_act(x, None, 1e-6)
+    assert not r["xq"].any()
+    assert np.all(r["a_scale"] == np.float32(1e-5) / np.float32(127.0))
+    # constant-magnitude rows: |xn| = 1 (to rounding) whatever the magnitude, so every code is +-127
+    for c in (3.0, 0.0078125, 1000.0):
+        row = _bf16_bits(np.tile(np.array([c, -c], np.float32), 128))[None, :]
+        r = oracle.norm_quant_act(row, None, 0.0, want_xn=True)
+        assert np.all(np.abs(r["xq"].astype(np.int32)) == 127)
+        assert np.all(np.sign(r["xq"][0, ::2]) == 1) and np.all(np.sign(r["xq"][0, 1::2]) == -1)
+        assert abs(float(r["a_scale"][0]) * 127.0 - 1.0) < 3e-7
