@@ -211,6 +211,7 @@ class Layer:
         self.packed = b.alloc_packed(N, K, with_dense=True)
         self.xq = b.alloc_xq(T, K)
         self.a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+        self.gain = torch.from_numpy((1.0 + 0.1 * np.random.default_rng(seed + 20).standard_normal(K)).astype(np.float32)).cuda()
         self.y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
         self.y32 = torch.empty((T, N), dtype=torch.float32, device="cuda")
         self.y_host = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
@@ -418,6 +419,11 @@ def run_ours(args):
         row["quantize_mask_pack_gbs"] = round(L.N * L.K * 4.625 / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
         row["quant_act_us"] = round(act, 2)
         row["quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act / 1e3, 1)
+        if L.K <= 16384:
+            # Algorithm 1's x~ = Q_a(Norm(x)) as one kernel (RMSNorm with gain fused into the quantiser)
+            nact = time_cold(lambda: b.sbn_norm_quant_act(L.x, L.xq, L.a_scale, gain=L.gain, eps=1e-6), iters)
+            row["norm_quant_act_us"] = round(nact, 2)
+            row["norm_quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4 + L.K * 4) / nact / 1e3, 1)
         gemm[L.name] = row
     b.sbn_check_status()
     sampler.stop()

@@ -184,6 +184,21 @@ sbn_status sbn_quant_act(const void *x_bf16, int T, int K, int8_t *xq, float *a_
                          void *stream);
 
 /*
+ * Part 2 with the preceding normalisation fused in -- Algorithm 1, forward: x~ = Q_a(Norm(x)).
+ * The paper does not name the norm; it is taken as RMSNorm with a per-channel gain:
+ *   ms = mean_k x[t][k]^2 (accumulated in fp64),  r = 1 / sqrt(ms + eps),
+ *   xn[k] = (x[t][k] * r) * gain[k]              (fp32; gain == NULL means all ones)
+ * followed by the quantiser above applied to the fp32 xn (which is never written to memory).
+ *   x_bf16   device, bf16 [T][K], K % 128 == 0, K <= 16384 (else SBN_ERR_UNSUPPORTED)
+ *   gain     device, fp32 [K], 16-byte aligned, or NULL
+ *   eps      >= 0
+ *   xq, a_scale   as for sbn_quant_act
+ * Asynchronous on `stream`; caller owns all buffers.
+ */
+sbn_status sbn_norm_quant_act(const void *x_bf16, int T, int K, const float *gain, float eps,
+                              int8_t *xq, float *a_scale, void *stream);
+
+/*
  * Part 3 -- Eq. 4: acc[t][n] = sum_k xq[t][k] * W_eff[n][k] in int32 (exact), then
  *   y[t][n] = float(acc[t][n]) * (w_scale * a_scale[t]) (+ bias[n]),
  * written as fp32 or as bf16 (round-to-nearest-even of the fp32 value).

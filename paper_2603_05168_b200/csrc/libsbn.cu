@@ -12,6 +12,7 @@
 #include "sbn.h"
 #include "sbn_common.cuh"
 #include "quant_act.cuh"
+#include "norm_quant_act.cuh"
 #include "quantize_mask_pack.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_pair_tcgen05.cuh"
@@ -535,6 +536,17 @@ sbn_status sbn_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_
     if (T <= 0 || K <= 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
     if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
     return launch_quant_act(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_norm_quant_act(const void* x_bf16, int T, int K, const float* gain, float eps, int8_t* xq,
+                              float* a_scale, void* stream) {
+    if (!x_bf16 || !xq || !a_scale) return SBN_ERR_NULL;
+    if (T <= 0 || K <= 0 || K % kBK != 0) return SBN_ERR_SHAPE;
+    if (K > 16384) return SBN_ERR_UNSUPPORTED;
+    if (!(eps >= 0.0f)) return SBN_ERR_SHAPE;
+    if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4) || (gain && misaligned(gain, 16)))
+        return SBN_ERR_ALIGN;
+    return launch_norm_quant_act(x_bf16, T, K, gain, eps, xq, a_scale, static_cast<cudaStream_t>(stream));
 }
 
 sbn_status sbn_sparse_bitlinear(const int8_t* xq, const float* a_scale, int T, const int8_t* vals,

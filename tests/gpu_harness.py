@@ -107,6 +107,17 @@ def gpu_quant_act(x_bits: np.ndarray):
     return xq, a_scale
 
 
+def gpu_norm_quant_act(x_bits: np.ndarray, gain=None, eps=1e-6):
+    T, K = x_bits.shape
+    xd = bf16_dev(x_bits)
+    xq = b.alloc_xq(T, K)
+    a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+    gd = None if gain is None else dev(np.asarray(gain, np.float32))
+    b.sbn_norm_quant_act(xd, xq, a_scale, gain=gd, eps=eps)
+    b.sbn_check_status()
+    return xq, a_scale
+
+
 def xq_to_numpy(xq: torch.Tensor, T: int, K: int) -> np.ndarray:
     """Tiled device activations -> plain [T][K] int8."""
     return untile(xq.cpu().numpy(), _xq_offsets(T, K))

@@ -12,7 +12,7 @@ from paper_2603_05168_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
-    from gpu_harness import (bf16_tensor_bits, dev, gpu_gemm, gpu_quant_act, gpu_quantize_mask_pack,
+    from gpu_harness import (gpu_norm_quant_act, bf16_tensor_bits, dev, gpu_gemm, gpu_quant_act, gpu_quantize_mask_pack,
                              xq_to_numpy, y_to_f32_numpy)
 
 
@@ -65,6 +65,42 @@ def test_quant_act_edge_rows():
     assert np.array_equal(xq_to_numpy(xq, 6, K), xq_ref)
     assert np.array_equal(s.cpu().numpy(), s_ref)
     assert xq_ref[0, :8].tolist() == [127, 0, 2, 2, 0, -2, -2, 4]
+
+
+# ------------------------------------------------------------------------------------------------
+# part 2 with the norm fused in (Algorithm 1: x~ = Q_a(Norm(x)))
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("with_gain", [True, False])
+@pytest.mark.parametrize("T,K", [(64, 256), (1, 2560), (5, 128), (67, 2560), (33, 6912), (19, 11008),
+                                  (300, 4096), (9, 16384), (130, 1024)])
+def test_norm_quant_act_parity(T, K, with_gain):
+    x = inputs.activations_bf16(T, K, seed=T + K, token_lognormal_sigma=0.5)
+    gain = (1.0 + 0.2 * np.random.default_rng(K).standard_normal(K)).astype(np.float32) if with_gain else None
+    r = oracle.norm_quant_act(x, gain, 1e-6)
+    xq, s = gpu_norm_quant_act(x, gain, 1e-6)
+    ok = ~r["near_tie"]
+    assert ok.all(), "a row's mean square sits on an fp32 rounding boundary for this seed"
+    assert np.array_equal(s.cpu().numpy(), r["a_scale"])
+    assert np.array_equal(xq_to_numpy(xq, T, K), r["xq"])
+
+
+def test_norm_quant_act_edge_rows():
+    K = 512
+    x = np.zeros((5, K), np.float32)
+    x[1, :] = 3.0                                         # constant row: every code 127
+    x[2, ::2], x[2, 1::2] = 0.0078125, -0.0078125
+    x[3, 7] = 65280.0                                     # one huge outlier
+    x[4, :] = np.linspace(-1, 1, K)
+    bits = inputs.f32_to_bf16_bits(x)
+    for eps in (0.0, 1e-6, 1e-2):
+        if eps == 0.0:
+            sel = [1, 2, 3, 4]                            # eps = 0 on an all-zero row is 0/0
+        else:
+            sel = [0, 1, 2, 3, 4]
+        r = oracle.norm_quant_act(bits[sel], None, eps)
+        xq, s = gpu_norm_quant_act(bits[sel], None, eps)
+        assert np.array_equal(s.cpu().numpy(), r["a_scale"])
+        assert np.array_equal(xq_to_numpy(xq, len(sel), K), r["xq"])
 
 
 # ------------------------------------------------------------------------------------------------
