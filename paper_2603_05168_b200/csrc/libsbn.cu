@@ -143,13 +143,8 @@ template <bool SPARSE, int BN>
 static sbn_status launch_gemm_cfg(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
                                   const CUtensorMap& ty, const GemmParams& p, cudaStream_t stream) {
     using Cfg = GemmConfig<SPARSE, BN>;
-    static bool configured = false;
     auto kernel = bitlinear_gemm_kernel<SPARSE, BN>;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem<bitlinear_gemm_kernel<SPARSE, BN>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
     const int tiles = (p.N / kBM) * ((p.T + BN - 1) / BN) * p.k_splits;
     const int grid = tiles < kNumSMs ? tiles : kNumSMs;
     const cudaError_t err = launch_kernel(kernel, dim3(grid), dim3(kGemmThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, ty, p);
@@ -200,13 +195,8 @@ template <bool SPARSE>
 static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
                               const PairParams& pp, cudaStream_t stream) {
     using Cfg = PairConfig<SPARSE>;
-    static bool configured = false;
     auto kernel = bitlinear_gemm_pair_kernel<SPARSE>;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem<bitlinear_gemm_pair_kernel<SPARSE>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
     const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
     const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
     const cudaError_t err = launch_kernel(kernel, dim3(2 * pairs), dim3(kPairThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, pp);
@@ -313,13 +303,8 @@ template <bool SPARSE, int BN>
 static sbn_status launch_splitk_cluster(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
                                         const GemmParams& p, int cluster, cudaStream_t stream) {
     using Cfg = SplitConfig<SPARSE, BN>;
-    static bool configured = false;
     auto kernel = bitlinear_gemm_splitk_cluster_kernel<SPARSE, BN>;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem<bitlinear_gemm_splitk_cluster_kernel<SPARSE, BN>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
     const int tiles = (p.N / kBM) * ((p.T + BN - 1) / BN);
     const cudaError_t err = launch_kernel_cluster(kernel, dim3(tiles * cluster), dim3(kSplitThreads), Cfg::SMEM_BYTES, stream,
                                                   static_cast<unsigned>(cluster), ta, tb, te, p);
@@ -620,6 +605,6 @@ void sbn_set_gemm_tuning(int token_tile, int split_k) {
     g_force_split_k = split_k;
 }
 
-unsigned long long sbn_launch_count(void) { return g_launch_count; }
+unsigned long long sbn_launch_count(void) { return g_launch_count.load(); }
 
 }  // extern "C"

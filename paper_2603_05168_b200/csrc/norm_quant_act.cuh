@@ -189,12 +189,7 @@ static cudaError_t launch_norm_quant_act_cfg(const uint4* x, int T, int nvec, co
     int grid = (T + rows - 1) / rows;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
     const size_t smem = gain ? static_cast<size_t>(nvec) * 32 : 0;          // K floats
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(norm_quant_act_kernel<G, VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536) != cudaSuccess)
-            return cudaErrorUnknown;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem<norm_quant_act_kernel<G, VPT>>(65536)) return cudaErrorUnknown;
     return launch_kernel(norm_quant_act_kernel<G, VPT>, dim3(grid), dim3(kActThreads), smem, stream, x, T, nvec, gain, eps, q, a_scale);
 }
 

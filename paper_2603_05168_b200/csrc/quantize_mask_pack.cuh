@@ -477,12 +477,7 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
                                                   uint32_t max_units, QmpSlot* slots, cudaStream_t stream) {
     unsigned long long nonce = qmp_next_nonce();
     const unsigned grid = max_units < static_cast<uint32_t>(kQmpMaxCtas) ? max_units : kQmpMaxCtas;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(quantize_mask_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQmpSmemBytes) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem<quantize_mask_pack_kernel>(kQmpSmemBytes)) return SBN_ERR_CUDA;
     // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
+#include <atomic>
 #include <utility>
 
 #include "sbn.h"
@@ -18,7 +19,7 @@ constexpr float kEps = 1e-5f;         // Algorithm 2's clamp for both scales
 __device__ int g_device_status = 0;
 
 // Host-side count of kernel launches made by the library.
-static unsigned long long g_launch_count = 0;
+static std::atomic<unsigned long long> g_launch_count{0ull};
 
 // Programmatic dependent launch.  Every kernel of the library is launched with the
 // programmatic-stream-serialisation attribute and starts with
@@ -39,6 +40,20 @@ inline bool pdl_enabled() {
         return !(e && e[0] == '1');
     }();
     return on;
+}
+
+// Opt-in to more than 48 KB of dynamic shared memory.  The attribute is per device, so it is set once
+// per (kernel, device); the record is a bit mask per kernel instantiation (devices beyond 63 simply
+// set it on every launch).  Safe to call from several host threads.
+template <auto Kernel>
+inline bool ensure_dynamic_smem(int bytes) {
+    static std::atomic<unsigned long long> done{0ull};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return true;
+    if (cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+    return true;
 }
 
 // `cluster` > 1 launches the grid as clusters of that many consecutive CTAs (runtime cluster size).
