@@ -198,11 +198,15 @@ def run_reference(args):
 class Layer:
     """Device (and pinned host) buffers of one BitLinear of the workload."""
 
-    def __init__(self, name, K, N, T, seed, torch, b, sigma=0.02, outl=0.0, logn=0.0):
+    def __init__(self, name, K, N, T, seed, torch, b, sigma=0.02, outl=0.0, logn=0.0, masters="fp32"):
         self.name, self.K, self.N, self.T = name, K, N, T
         W = inputs.latent_weights(N, K, seed=seed, sigma=sigma, outlier_prob=outl)
         x = inputs.activations_bf16(T, K, seed=seed + 10, token_lognormal_sigma=logn)
-        self.W_host = torch.from_numpy(W).pin_memory()
+        if masters == "bf16":     # master weights kept in bf16 (the paper's own example)
+            self.W_host = torch.from_numpy(inputs.f32_to_bf16_bits(W).view(np.int16)).view(torch.bfloat16).pin_memory()
+        else:
+            self.W_host = torch.from_numpy(W).pin_memory()
+        self.w_bytes = self.W_host.element_size()
         self.x_host = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
         self.W = self.W_host.cuda()
         self.x = self.x_host.cuda()
@@ -239,9 +243,9 @@ def run_ours(args):
     b.lib()
     peaks = load_peaks()
     T, shapes, sigma, outl, logn = WORKLOADS[args.workload]
-    layers = [Layer(n, K, N, T, seed=1 + i, torch=torch, b=b, sigma=sigma, outl=outl, logn=logn)
+    layers = [Layer(n, K, N, T, seed=1 + i, torch=torch, b=b, sigma=sigma, outl=outl, logn=logn, masters=args.masters)
               for i, (n, K, N) in enumerate(shapes)]
-    in_bytes = sum(L.W.numel() * 4 + L.x.numel() * 2 for L in layers)
+    in_bytes = sum(L.W.numel() * L.w_bytes + L.x.numel() * 2 for L in layers)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -375,7 +379,7 @@ def run_ours(args):
     b.sbn_check_status()
     e2e_ms = max_over_ranks(s2.elapsed_time(e2), world, dist, "cuda") / e2e_steps
     e2e_value = whole_job_tops(step_ops(T, shapes), world, e2e_ms)
-    h2d = sum(L.W_host.numel() * 4 + L.x_host.numel() * 2 for L in layers)
+    h2d = sum(L.W_host.numel() * L.w_bytes + L.x_host.numel() * 2 for L in layers)
     d2h = sum(L.y_host.numel() * 2 for L in layers)
 
     # ---- isolated kernels, cold L2 (a 512 MB buffer is overwritten before every launch) --------
@@ -416,7 +420,7 @@ def run_ours(args):
         qmp = time_cold(lambda: b.sbn_quantize_mask_pack(L.W, p["vals"], p["meta"], p["w_scale"], p["ws"]), iters)
         act = time_cold(lambda: b.sbn_quant_act(L.x, L.xq, L.a_scale), iters)
         row["quantize_mask_pack_us"] = round(qmp, 2)
-        row["quantize_mask_pack_gbs"] = round(L.N * L.K * 4.625 / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
+        row["quantize_mask_pack_gbs"] = round(L.N * L.K * (L.w_bytes + 0.625) / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
         row["quant_act_us"] = round(act, 2)
         row["quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act / 1e3, 1)
         if L.K <= 16384:
@@ -444,7 +448,7 @@ def run_ours(args):
                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {ratio:g} (nominal sparse-int8 : bf16)",
                     "frac_of_datasheet_sparse_int8": round(achieved / DATASHEET_INT8_SPARSE_TOPS, 4)}
     else:
-        per_param = 4.625 if dominant == "quantize_mask_pack" else None
+        per_param = (layers[0].w_bytes + 0.625) if dominant == "quantize_mask_pack" else None
         if dominant == "quantize_mask_pack":
             bytes_ = sum(L.N * L.K * per_param for L in layers)
         else:
@@ -576,6 +580,8 @@ def run_dynamic_step(args):
     for layer in range(n_layers):
         for name, K, N in inputs.LAYER_2B:
             W = torch.randn((N, K), generator=gen, device="cuda", dtype=torch.float32) * 0.02
+            if args.masters == "bf16":
+                W = W.to(torch.bfloat16)
             p = b.alloc_packed(N, K)
             p["prev"] = torch.empty_like(p["meta"])
             p["flips"] = torch.zeros(1, dtype=torch.int64, device="cuda")
@@ -621,7 +627,7 @@ def run_dynamic_step(args):
     steps = max(1, min(args.steps, 5))
     for s_i in range(steps + 1):
         for _, K, N, W, p in mats:                                # the optimiser step stand-in
-            W.add_(torch.randn(W.shape, generator=gen, device="cuda", dtype=torch.float32), alpha=1e-4)
+            W.add_(torch.randn(W.shape, generator=gen, device="cuda", dtype=torch.float32).to(W.dtype), alpha=1e-4)
         torch.cuda.synchronize()
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         torch.cuda._sleep(int(4e7))
@@ -644,8 +650,9 @@ def run_dynamic_step(args):
         "metric": "dynamic-mask training step latency (re-pack 210 matrices + 210 sparse BitLinears at T=2048)",
         "unit": "ms", "workload": "dyn", "value": rep + fwd, "higher_is_better": False,
         "repack_ms": round(rep, 3), "forward_ms": round(fwd, 3), "params": params,
-        "repack_gbs_algorithmic": round(params * 4.75 / (rep * 1e-3) / 1e9, 1),     # 4 B read + 0.625 written + 0.125 prev meta
-        "repack_frac_of_hbm": round(params * 4.75 / (rep * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "masters": args.masters,
+        "repack_gbs_algorithmic": round(params * ((2 if args.masters == "bf16" else 4) + 0.75) / (rep * 1e-3) / 1e9, 1),   # W read + 0.625 written + 0.125 prev meta
+        "repack_frac_of_hbm": round(params * ((2 if args.masters == "bf16" else 4) + 0.75) / (rep * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
         "forward_tops": round(fwd_ops / (fwd * 1e-3) / 1e12, 1),
         "forward_pct_sparse_int8_datasheet": round(100 * fwd_ops / (fwd * 1e-3) / 1e12 / DATASHEET_INT8_SPARSE_TOPS, 1),
         "flip_rate": statistics.mean(rates), "steps": steps, "data": "synthetic (torch CUDA generator, seed 1234)",
@@ -663,6 +670,8 @@ def main():
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1,4,16,64), sparse vs dense, cold L2; "
                          "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048")
+    ap.add_argument("--masters", default="fp32", choices=["fp32", "bf16"],
+                    help="precision of the master weights the pack kernel reads (default fp32, the configuration of the metric)")
     ap.add_argument("--only-step", action="store_true", help="time the step only (used for profiler runs)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -116,6 +116,16 @@ sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int 
                                   void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * The same operation on bf16 master weights (Sec. 2.2 keeps the master weight "e.g. in bf16"): W is
+ * read as bf16 [N][K] (16-byte aligned), every value is taken as the real number it represents, and
+ * everything else -- arguments, results, exactness -- is as above.  Half the weight traffic.
+ */
+sbn_status sbn_quantize_mask_pack_bf16(const void *W_bf16, int N, int K, int n_keep, int m_group,
+                                       int8_t *vals, uint8_t *meta, float *w_scale, int8_t *dense_q,
+                                       const uint8_t *prev_meta, unsigned long long *flip_bits,
+                                       void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Part 1 for many matrices in ONE launch -- the dynamic-mask training step recomputes the mask of
  * every BitLinear at every step (Sec. 2.3, "Dynamic Mask Recomputation"; Algorithm 1).  Each job
  * is exactly one sbn_quantize_mask_pack call (same arguments, same results, bit for bit); the
@@ -124,7 +134,7 @@ sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int 
  *   ws     device workspace of sbn_batch_workspace_bytes(count) bytes; no initialisation needed
  */
 typedef struct {
-    const float *W;                   /* device, fp32 [N][K] */
+    const void *W;                    /* device, [N][K], fp32 or (w_bf16 != 0) bf16 */
     int N, K;
     int8_t *vals;                     /* device out, tiled */
     uint8_t *meta;                    /* device out, tiled; may equal prev_meta */
@@ -132,6 +142,7 @@ typedef struct {
     int8_t *dense_q;                  /* device out or NULL */
     const uint8_t *prev_meta;         /* device or NULL */
     unsigned long long *flip_bits;    /* device out; required iff prev_meta != NULL */
+    int w_bf16;                       /* 0: W is fp32; 1: W is bf16 (see sbn_quantize_mask_pack_bf16) */
 } sbn_pack_job;
 size_t sbn_batch_workspace_bytes(int count);
 sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job *jobs, void *ws, size_t ws_bytes,

@@ -21,7 +21,7 @@ OUT_F32, OUT_BF16 = 0, 1
 OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
 
 EXPORTS = [
-    "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
+    "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
     "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_norm_quant_act", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sbn_quantize_mask_pack.restype = i32
         L.sbn_quantize_mask_pack.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.sbn_quantize_mask_pack_bf16.restype = i32
+        L.sbn_quantize_mask_pack_bf16.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.sbn_quantize_mask_pack_static_ws.restype = i32
         L.sbn_quantize_mask_pack_static_ws.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.sbn_batch_workspace_bytes.restype = sz
@@ -107,10 +109,12 @@ def sbn_xq_bytes(T: int, K: int) -> int:
 
 def sbn_quantize_mask_pack(W, vals, meta, w_scale, ws, dense_q=None, prev_meta=None, flip_bits=None,
                            n_keep: int = 2, m_group: int = 4):
+    """W: fp32 or bf16 CUDA tensor [N][K] (bf16 master weights go to sbn_quantize_mask_pack_bf16)."""
     N, K = W.shape
-    _check(lib().sbn_quantize_mask_pack(_ptr(W), N, K, n_keep, m_group, _ptr(vals), _ptr(meta),
-                                        _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta), _ptr(flip_bits),
-                                        _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+    fn = lib().sbn_quantize_mask_pack_bf16 if W.dtype == torch.bfloat16 else lib().sbn_quantize_mask_pack
+    _check(fn(_ptr(W), N, K, n_keep, m_group, _ptr(vals), _ptr(meta),
+              _ptr(w_scale), _ptr(dense_q), _ptr(prev_meta), _ptr(flip_bits),
+              _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "sbn_quantize_mask_pack")
 
 
@@ -128,7 +132,7 @@ def sbn_quantize_mask_pack_static_ws(W, vals, meta, w_scale, dense_q=None, prev_
 class PackJob(ctypes.Structure):
     _fields_ = [("W", ctypes.c_void_p), ("N", ctypes.c_int), ("K", ctypes.c_int), ("vals", ctypes.c_void_p),
                 ("meta", ctypes.c_void_p), ("w_scale", ctypes.c_void_p), ("dense_q", ctypes.c_void_p),
-                ("prev_meta", ctypes.c_void_p), ("flip_bits", ctypes.c_void_p)]
+                ("prev_meta", ctypes.c_void_p), ("flip_bits", ctypes.c_void_p), ("w_bf16", ctypes.c_int)]
 
 
 def sbn_batch_workspace_bytes(count: int) -> int:
@@ -143,6 +147,7 @@ def make_pack_jobs(jobs):
     for a, j in zip(arr, jobs):
         N, K = j["W"].shape
         a.W, a.N, a.K = j["W"].data_ptr(), N, K
+        a.w_bf16 = 1 if j["W"].dtype == torch.bfloat16 else 0
         a.vals, a.meta, a.w_scale = j["vals"].data_ptr(), j["meta"].data_ptr(), j["w_scale"].data_ptr()
         for key in ("dense_q", "prev_meta", "flip_bits"):
             t = j.get(key)

@@ -432,10 +432,10 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K) {
     }
 }
 
-sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int m_group,
-                                  int8_t* vals, uint8_t* meta, float* w_scale, int8_t* dense_q,
-                                  const uint8_t* prev_meta, unsigned long long* flip_bits,
-                                  void* ws, size_t ws_bytes, void* stream) {
+static sbn_status quantize_mask_pack_any(const void* W, bool w_bf16, int N, int K, int n_keep, int m_group,
+                                         int8_t* vals, uint8_t* meta, float* w_scale, int8_t* dense_q,
+                                         const uint8_t* prev_meta, unsigned long long* flip_bits,
+                                         void* ws, size_t ws_bytes, void* stream) {
     if (!W || !vals || !meta || !w_scale) return SBN_ERR_NULL;
     if (prev_meta && !flip_bits) return SBN_ERR_NULL;
     if (n_keep != 2 || m_group != 4) return SBN_ERR_UNSUPPORTED;
@@ -445,9 +445,25 @@ sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int 
         misaligned(w_scale, 4) || (dense_q && misaligned(dense_q, 16)) ||
         (prev_meta && misaligned(prev_meta, 16)) || (flip_bits && misaligned(flip_bits, 8)))
         return SBN_ERR_ALIGN;
-    return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+    return launch_quantize_mask_pack(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(ws),
                                      static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_quantize_mask_pack(const float* W, int N, int K, int n_keep, int m_group,
+                                  int8_t* vals, uint8_t* meta, float* w_scale, int8_t* dense_q,
+                                  const uint8_t* prev_meta, unsigned long long* flip_bits,
+                                  void* ws, size_t ws_bytes, void* stream) {
+    return quantize_mask_pack_any(W, false, N, K, n_keep, m_group, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+                                  ws, ws_bytes, stream);
+}
+
+sbn_status sbn_quantize_mask_pack_bf16(const void* W_bf16, int N, int K, int n_keep, int m_group,
+                                       int8_t* vals, uint8_t* meta, float* w_scale, int8_t* dense_q,
+                                       const uint8_t* prev_meta, unsigned long long* flip_bits,
+                                       void* ws, size_t ws_bytes, void* stream) {
+    return quantize_mask_pack_any(W_bf16, true, N, K, n_keep, m_group, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+                                  ws, ws_bytes, stream);
 }
 
 size_t sbn_batch_workspace_bytes(int count) {
@@ -473,7 +489,7 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
             (j.dense_q && misaligned(j.dense_q, 16)) || (j.prev_meta && misaligned(j.prev_meta, 16)) ||
             (j.flip_bits && misaligned(j.flip_bits, 8)))
             return SBN_ERR_ALIGN;
-        descs[i] = qmp_make_desc(j.W, j.N, j.K, j.vals, j.meta, j.w_scale, j.dense_q, j.prev_meta, j.flip_bits);
+        descs[i] = qmp_make_desc(j.W, j.w_bf16 != 0, j.N, j.K, j.vals, j.meta, j.w_scale, j.dense_q, j.prev_meta, j.flip_bits);
         max_units = std::max(max_units, descs[i].num_units);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -511,7 +527,7 @@ sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_
     void* scratch = static_scratch_for_current_device();
     if (!scratch) return SBN_ERR_CUDA;
     // every slot that is read carries this call's nonce, so stale contents are harmless
-    return launch_quantize_mask_pack(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
+    return launch_quantize_mask_pack(W, false, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(scratch),
                                      static_cast<cudaStream_t>(stream));
 }

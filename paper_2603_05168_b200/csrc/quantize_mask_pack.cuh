@@ -143,7 +143,7 @@ __device__ __forceinline__ double abs_sum4(const float4 v) {
 
 // One matrix of a batch (device-visible copy of the call's arguments).
 struct QmpDesc {
-    const float4* W4;
+    const void* W;                     // fp32 [N][K], or bf16 [N][K] when w_bf16
     uint16_t* vals;
     uint8_t* meta;
     float* w_scale;
@@ -152,6 +152,7 @@ struct QmpDesc {
     unsigned long long* flip_bits;     // or null
     uint32_t num_units;                // N * K / 128
     uint32_t KB;                       // K / 128
+    uint32_t w_bf16;                   // master weights are bf16 (Sec. 2.2 keeps them "e.g. in bf16")
 };
 
 struct QmpRange {                      // this CTA's share of one matrix
@@ -161,6 +162,30 @@ struct QmpEntry {                      // one undecided kept value
     uint32_t byte_off;                 // its byte in vals
     float w;
 };
+
+// One group (4 consecutive weights) of unit u for lane `lane` (a warp covers the unit's 32 groups).
+template <bool BF16>
+__device__ __forceinline__ float4 qmp_load_group(const void* W, size_t u, int lane) {
+    if constexpr (BF16) {
+        const uint2 v = __ldg(static_cast<const uint2*>(W) + u * 32 + lane);
+        return make_float4(bf16lo_to_f32(v.x), bf16hi_to_f32(v.x), bf16lo_to_f32(v.y), bf16hi_to_f32(v.y));
+    } else {
+        return __ldg(static_cast<const float4*>(W) + u * 32 + lane);
+    }
+}
+// Two adjacent groups of unit u for lane l16 of a half-warp (16 lanes cover the unit).
+template <bool BF16>
+__device__ __forceinline__ void qmp_load_group_pair(const void* W, size_t u, uint32_t l16, float4& a, float4& b) {
+    if constexpr (BF16) {
+        const uint4 v = __ldg(static_cast<const uint4*>(W) + u * 16 + l16);
+        a = make_float4(bf16lo_to_f32(v.x), bf16hi_to_f32(v.x), bf16lo_to_f32(v.y), bf16hi_to_f32(v.y));
+        b = make_float4(bf16lo_to_f32(v.z), bf16hi_to_f32(v.z), bf16lo_to_f32(v.w), bf16hi_to_f32(v.w));
+    } else {
+        const float4* src = static_cast<const float4*>(W) + u * 32 + 2 * l16;
+        a = __ldg(src);
+        b = __ldg(src + 1);
+    }
+}
 
 __device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d) {
     QmpRange r;
@@ -172,6 +197,7 @@ __device__ __forceinline__ QmpRange qmp_range(const QmpDesc& d) {
 
 // gamma_est: mean |w| over kQmpSampleUnits units scattered over the matrix (the same units in every
 // CTA; a multiplicative hash keeps them off any row / column-block period).  fp32 is plenty here.
+template <bool BF16>
 __device__ __forceinline__ float qmp_sample_gamma(const QmpDesc& d, double* s_warp) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -184,7 +210,7 @@ __device__ __forceinline__ float qmp_sample_gamma(const QmpDesc& d, double* s_wa
     for (int i = 0; i < kPerWarp; ++i) {                  // all loads of the warp in flight at once
         const uint32_t sidx = warp + i * kQmpWarps;
         const uint32_t u = sidx * stride + ((sidx * 2654435761u) >> 8) % stride;
-        v[i] = sidx < n_s ? __ldg(d.W4 + static_cast<size_t>(u) * 32 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[i] = sidx < n_s ? qmp_load_group<BF16>(d.W, u, lane) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
     for (int i = 0; i < kPerWarp; ++i) acc += (fabsf(v[i].x) + fabsf(v[i].y)) + (fabsf(v[i].z) + fabsf(v[i].w));
@@ -220,6 +246,7 @@ __device__ __forceinline__ void qmp_list_undecided(const float (&k)[4], const fl
 // A lane takes TWO adjacent groups (32 B of a row), so it owns a whole metadata byte and four
 // consecutive bytes of vals and the per-unit index arithmetic is shared by two groups; a half-warp
 // covers one 512 B unit, a warp two units per load pair and four per iteration.
+template <bool BF16>
 __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
                                             QmpEntry* list, unsigned int* list_count, double* s_warp,
                                             unsigned int& flips) {
@@ -228,6 +255,7 @@ __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg,
     const uint32_t l16 = lane & 15;
     const uint32_t KB = d.KB;
     constexpr uint32_t kStep = 2 * kQmpWarps;                // units between a thread's consecutive units
+    constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
     const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
     const bool count_flips = d.prev_meta != nullptr;
     double acc = 0.0;
@@ -239,21 +267,20 @@ __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg,
     if (threadIdx.x == 0) {
         for (int j = 1; j < kQmpPrefetchAhead; ++j) {
             const uint32_t ub = rg.u_begin + j * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 2 * kStep) * 512u);
+            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
         }
     }
     for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += 2 * kStep) {
         if (threadIdx.x == 0) {
             const uint32_t ub = u0 + kQmpPrefetchAhead * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(d.W4 + static_cast<size_t>(ub) * 32, min(rg.u_end - ub, 2 * kStep) * 512u);
+            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
         }
         float4 va[2], vb[2];
 #pragma unroll
         for (int q = 0; q < 2; ++q) {                     // four independent 16 B loads in flight
             const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
-            const float4* src = d.W4 + static_cast<size_t>(uq) * 32 + 2 * l16;
-            va[q] = (uq < rg.u_end) ? __ldg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
-            vb[q] = (uq < rg.u_end) ? __ldg(src + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            va[q] = vb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (uq < rg.u_end) qmp_load_group_pair<BF16>(d.W, uq, l16, va[q], vb[q]);
         }
         acc += (abs_sum4(va[0]) + abs_sum4(vb[0])) + (abs_sum4(va[1]) + abs_sum4(vb[1]));
 #pragma unroll
@@ -288,6 +315,7 @@ __device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg,
 // Ternarise a whole range again with the exact threshold (the path taken when the bracket missed,
 // the list overflowed or the dense W_q is wanted): a warp per unit, four units at a time, newest
 // first (what pass 1 read last is still in L2).
+template <bool BF16>
 __device__ __forceinline__ void qmp_pass2_full(const QmpDesc& d, const QmpRange rg, float thr) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -306,7 +334,7 @@ __device__ __forceinline__ void qmp_pass2_full(const QmpDesc& d, const QmpRange 
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const uint32_t i = i0 + q * kQmpWarps;
-            w[q] = (i < n_units) ? __ldg(d.W4 + static_cast<size_t>(rg.u_begin + (n_units - 1 - i)) * 32 + lane)
+            w[q] = (i < n_units) ? qmp_load_group<BF16>(d.W, rg.u_begin + (n_units - 1 - i), lane)
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
@@ -365,7 +393,7 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             if (m > 0) d_cur = rest[m - 1];
             rg_cur = qmp_range(d_cur);
             const int par = m & 1;
-            const float gamma_est = qmp_sample_gamma(d_cur, s_warp);
+            const float gamma_est = d_cur.w_bf16 ? qmp_sample_gamma<true>(d_cur, s_warp) : qmp_sample_gamma<false>(d_cur, s_warp);
             if (threadIdx.x == 0) {
                 s_list_count[par] = 0u;
                 s_bracket[par][0] = ternary_threshold(fmaxf(gamma_est * (1.0f - kQmpBracket), kEps));
@@ -373,8 +401,11 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             __syncthreads();
             unsigned int flips = 0;
-            const double mine = qmp_pass1(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1],
-                                          s_list + par * kQmpListCap, &s_list_count[par], s_warp, flips);
+            const double mine = d_cur.w_bf16
+                ? qmp_pass1<true>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                  &s_list_count[par], s_warp, flips)
+                : qmp_pass1<false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                   &s_list_count[par], s_warp, flips);
             // this CTA's flip count of matrix m; it is added to the global counter one phase later,
             // after the exchange has shown that CTA 0 zeroed that counter
 #pragma unroll
@@ -442,7 +473,8 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                     vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
                 }
             } else {
-                qmp_pass2_full(d_prev, rg_prev, thr);
+                if (d_prev.w_bf16) qmp_pass2_full<true>(d_prev, rg_prev, thr);
+                else qmp_pass2_full<false>(d_prev, rg_prev, thr);
             }
             __syncthreads();                                     // s_thr / this list may be reused
         }
@@ -457,10 +489,11 @@ inline unsigned long long qmp_next_nonce() {
     return counter.fetch_add(1) + 1;
 }
 
-inline QmpDesc qmp_make_desc(const float* W, int N, int K, int8_t* vals, uint8_t* meta, float* w_scale,
+inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* vals, uint8_t* meta, float* w_scale,
                              int8_t* dense_q, const uint8_t* prev_meta, unsigned long long* flip_bits) {
     QmpDesc d;
-    d.W4 = reinterpret_cast<const float4*>(W);
+    d.W = W;
+    d.w_bf16 = w_bf16 ? 1u : 0u;
     d.vals = reinterpret_cast<uint16_t*>(vals);
     d.meta = meta;
     d.w_scale = w_scale;
@@ -487,12 +520,12 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
-inline sbn_status launch_quantize_mask_pack(const float* W, int N, int K, int8_t* vals,
+inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, int K, int8_t* vals,
                                             uint8_t* meta, float* w_scale, int8_t* dense_q,
                                             const uint8_t* prev_meta,
                                             unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
-    const QmpDesc d = qmp_make_desc(W, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
+    const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
     return launch_quantize_mask_pack_batch(d, nullptr, 1, d.num_units, ws->slot, stream);
 }
 

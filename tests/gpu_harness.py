@@ -70,10 +70,11 @@ def bf16_dev(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def gpu_quantize_mask_pack(W: np.ndarray, with_dense=True, prev_meta=None, in_place=False):
+def gpu_quantize_mask_pack(W: np.ndarray, with_dense=True, prev_meta=None, in_place=False, w_bf16_bits=None):
+    """W fp32 [N][K]; or, with w_bf16_bits (uint16 bit patterns), bf16 master weights."""
     N, K = W.shape
     bufs = b.alloc_packed(N, K, with_dense=with_dense)
-    Wd = dev(W)
+    Wd = dev(W) if w_bf16_bits is None else bf16_dev(w_bf16_bits)
     flip = None
     pm = None
     if prev_meta is not None:

@@ -12,7 +12,7 @@ from paper_2603_05168_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
-    from gpu_harness import (gpu_norm_quant_act, bf16_tensor_bits, dev, gpu_gemm, gpu_quant_act, gpu_quantize_mask_pack,
+    from gpu_harness import (gpu_norm_quant_act, bf16_dev, bf16_tensor_bits, dev, gpu_gemm, gpu_quant_act, gpu_quantize_mask_pack,
                              xq_to_numpy, y_to_f32_numpy)
 
 
@@ -171,6 +171,48 @@ def test_quantize_mask_pack_degenerate_scales():
         assert g["scale"] == r["scale"] and np.array_equal(g["vals"], r["vals"])
         if with_dense:
             assert np.array_equal(g["dense_q"], r["dense_q"])
+
+
+@pytest.mark.parametrize("with_dense", [True, False])
+@pytest.mark.parametrize("N,K,seed", [(256, 256, 30), (384, 2560, 31), (128, 6912, 32), (2048, 2560, 33)])
+def test_quantize_mask_pack_bf16_masters(N, K, seed, with_dense):
+    # master weights kept in bf16 (Sec. 2.2): the kernel reads bf16, the oracle gets the same real
+    # numbers as fp32 -- bf16 -> fp32 is exact, so the results must agree bit for bit.  bf16 weights
+    # produce many exact magnitude ties inside a group, which exercises the tie rule as well.
+    bits = inputs.f32_to_bf16_bits(inputs.latent_weights(N, K, seed=seed))
+    W = (bits.astype(np.uint32) << 16).view(np.float32).reshape(N, K)
+    r = _oracle_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=with_dense, w_bf16_bits=bits)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(g["vals"], r["vals"])
+    assert np.array_equal(g["meta"], r["meta"])
+    if with_dense:
+        assert np.array_equal(g["dense_q"], r["dense_q"])
+
+
+def test_quantize_mask_pack_batched_mixed_master_dtypes():
+    shapes = [(256, 512), (384, 256), (128, 1280)]
+    jobs, refs = [], []
+    for i, (N, K) in enumerate(shapes):
+        W = inputs.latent_weights(N, K, seed=40 + i)
+        if i % 2 == 0:
+            bits = inputs.f32_to_bf16_bits(W)
+            W = (bits.astype(np.uint32) << 16).view(np.float32).reshape(N, K)
+            Wd = bf16_dev(bits)
+        else:
+            Wd = dev(W)
+        refs.append(_oracle_pack(W))
+        p = b.alloc_packed(N, K)
+        jobs.append(dict(W=Wd, vals=p["vals"], meta=p["meta"], w_scale=p["w_scale"]))
+    arr = b.make_pack_jobs(jobs)
+    ws = torch.empty(b.sbn_batch_workspace_bytes(len(jobs)), dtype=torch.uint8, device="cuda")
+    b.sbn_quantize_mask_pack_batched(arr, ws)
+    b.sbn_check_status()
+    from gpu_harness import _meta_offsets, _vals_offsets, untile
+    for (N, K), j, r in zip(shapes, jobs, refs):
+        assert np.float32(j["w_scale"].cpu().numpy()[0]) == r["scale"]
+        assert np.array_equal(untile(j["vals"].cpu().numpy(), _vals_offsets(N, K)), r["vals"])
+        assert np.array_equal(untile(j["meta"].cpu().numpy(), _meta_offsets(N, K)), r["meta"])
 
 
 def _sampled_units(N, K):
