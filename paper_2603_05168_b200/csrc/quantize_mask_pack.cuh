@@ -8,7 +8,7 @@
 //
 //   sample   every CTA adds |w| over the same 256 scattered 512 B units of the matrix (128 KB,
 //            L2-served for all CTAs but the first) -> gamma_est, and brackets the threshold:
-//            thr_lo = thr(0.97 gamma_est), thr_hi = thr(1.03 gamma_est);
+//            thr_lo ~ thr(0.97 gamma_est), thr_hi ~ thr(1.03 gamma_est);
 //   pass 1   every CTA owns a contiguous range of (row, 128-column) units and streams it:
 //            sum|W| in fp64 (the exact gamma), top 2 of 4 per group (Eq. 2: the mask does not
 //            depend on gamma), metadata, flip count, and the two kept values ternarised
@@ -396,8 +396,10 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             const float gamma_est = d_cur.w_bf16 ? qmp_sample_gamma<true>(d_cur, s_warp) : qmp_sample_gamma<false>(d_cur, s_warp);
             if (threadIdx.x == 0) {
                 s_list_count[par] = 0u;
-                s_bracket[par][0] = ternary_threshold(fmaxf(gamma_est * (1.0f - kQmpBracket), kEps));
-                s_bracket[par][1] = ternary_threshold(fmaxf(gamma_est * (1.0f + kQmpBracket), kEps));
+                // any lo <= hi will do (the exact threshold is checked against them later), so no
+                // divisions here: thr(scale) is 0.5 * scale to within a few ulps
+                s_bracket[par][0] = 0.5f * fmaxf(gamma_est * (1.0f - kQmpBracket), kEps) * (1.0f - 1e-6f);
+                s_bracket[par][1] = 0.5f * fmaxf(gamma_est * (1.0f + kQmpBracket), kEps) * (1.0f + 1e-6f);
             }
             __syncthreads();
             unsigned int flips = 0;
