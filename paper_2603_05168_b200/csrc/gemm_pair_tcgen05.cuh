@@ -216,8 +216,8 @@ __device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, con
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
                 const uint32_t pk = packed[k][j >> 1];
-                if (j < cnt) y[0] = static_cast<uint16_t>(pk & 0xFFFFu);
-                if (j + 1 < cnt) y[p.N] = static_cast<uint16_t>(pk >> 16);
+                if (j < cnt) __stcs(y, static_cast<uint16_t>(pk & 0xFFFFu));
+                if (j + 1 < cnt) __stcs(y + p.N, static_cast<uint16_t>(pk >> 16));
                 y += 2 * static_cast<size_t>(p.N);             // running pointer: no table of 32 row addresses
             }
         }
