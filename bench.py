@@ -37,7 +37,7 @@ NOMINAL_BF16_DENSE_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the sparse GEMM per launch, from one ncu capture of
 # this bench's step (mean over the step's GEMM launches; the outputs mostly stay in L2, so this is far
 # below the algorithmic operand + output bytes -- the kernel is tensor-bound, the figure is context).
-GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 26.0e6, "down7b": 228.4e6}
+GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 25.2e6, "down7b": 215.9e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 

@@ -161,7 +161,8 @@ norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4
                     int q[8];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        // rint(xn * s_x) for two values: multiply, then add 1.5 * 2^23 (see quant1).  The
+                        // rint(xn * s_x) for two values: multiply, then add 1.5 * 2^23 -- the adder's round-to-nearest-even
+                        // IS the rounding of the method, and the integer is left in the low mantissa bits.  The
                         // adds are scalar: a packed multiply followed by a packed add came out with ONE
                         // rounding (a fused multiply-add), which breaks exact ties such as 63.5.
                         float lo, hi;

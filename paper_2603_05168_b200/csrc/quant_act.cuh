@@ -36,14 +36,8 @@ __device__ __forceinline__ uint32_t pack_sat_s8x2(int a, int b, uint32_t c) {
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
 }
-// rint(x * s_x) as an integer: one fp32 multiply, then half-to-even.  The conversion instruction
-// runs at an eighth of the ALU rate; adding 1.5 * 2^23 rounds to the same integer (the adder's
-// round-to-nearest-even IS the rounding of Algorithm 2's .round()) and leaves it in the low mantissa
-// bits.  Exact for |x * s_x| < 2^22; here it is at most 127.5 up to rounding.  The saturating pack
-// that follows applies the clamp.
 __device__ __forceinline__ int quant1(float x, float s_x) {
-    const float p = __fmul_rn(x, s_x);
-    return static_cast<int>(__float_as_uint(__fadd_rn(p, 12582912.0f)) - 0x4B400000u);
+    return __float2int_rn(__fmul_rn(x, s_x));      // one fp32 multiply, then half-to-even
 }
 // four consecutive bf16 (two words) -> four int8 codes in one word, lowest column in the low byte
 __device__ __forceinline__ uint32_t quant_pair2(uint32_t a, uint32_t b, float s_x) {
