@@ -88,7 +88,10 @@ norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4
             float f[8];
             bf16x8_to_f32(cur[i], f);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) s4[j & 3] += static_cast<double>(__fmul_rn(f[j], f[j]));   // the product is exact
+            for (int j = 0; j < 8; ++j) {                                   // exact product, one rounding in the add
+                const double dv = static_cast<double>(f[j]);
+                s4[j & 3] = __fma_rn(dv, dv, s4[j & 3]);
+            }
         }
         double ss = (s4[0] + s4[1]) + (s4[2] + s4[3]);
 #pragma unroll
