@@ -338,6 +338,36 @@ def test_quantize_mask_pack_batched_matches_single_calls():
             assert int(job["flip_bits"].item()) == want == one["flips"]
 
 
+def test_quantize_mask_pack_full_size_in_the_bench_configuration():
+    # the four BitNet-2B-shaped matrices exactly as bench.py packs them: one batched launch, no
+    # dense output (the single-pass route); every byte against the oracle
+    from gpu_harness import _meta_offsets, _vals_offsets, untile
+    Ws = [inputs.latent_weights(N, K, seed=1 + i) for i, (_, K, N) in enumerate(inputs.SHAPES_2B)]
+    jobs = []
+    for W in Ws:
+        N, K = W.shape
+        bufs = b.alloc_packed(N, K)
+        jobs.append(dict(W=dev(W), vals=bufs["vals"], meta=bufs["meta"], w_scale=bufs["w_scale"]))
+    arr = b.make_pack_jobs(jobs)
+    ws = torch.empty(b.sbn_batch_workspace_bytes(len(jobs)), dtype=torch.uint8, device="cuda")
+    b.sbn_quantize_mask_pack_batched(arr, ws)
+    b.sbn_check_status()
+    for W, job in zip(Ws, jobs):
+        N, K = W.shape
+        r = _oracle_pack(W)
+        assert np.float32(job["w_scale"].cpu().numpy()[0]) == r["scale"]
+        assert np.array_equal(untile(job["vals"].cpu().numpy(), _vals_offsets(N, K)), r["vals"])
+        assert np.array_equal(untile(job["meta"].cpu().numpy(), _meta_offsets(N, K)), r["meta"])
+
+
+def test_quant_act_full_size():
+    x = inputs.activations_bf16(4096, 6912, seed=14, token_lognormal_sigma=0.5)
+    xq_ref, s_ref = oracle.quant_act(x)
+    xq, s = gpu_quant_act(x)
+    assert np.array_equal(s.cpu().numpy(), s_ref)
+    assert np.array_equal(xq_to_numpy(xq, 4096, 6912), xq_ref)
+
+
 # ------------------------------------------------------------------------------------------------
 # part 3 and the dense baseline
 # ------------------------------------------------------------------------------------------------
