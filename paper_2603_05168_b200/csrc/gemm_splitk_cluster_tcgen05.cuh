@@ -115,7 +115,14 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     // a peer's shared memory may only be written once that CTA has started: every thread arrives
     // here and waits just before the scatter, so the barrier costs nothing on the way in
     cluster_arrive();
-    pdl_wait();                          // nothing above touches global memory
+    // this CTA's slice of the weights goes to L2 while the previous kernel is still finishing (a
+    // prefetch into L2, the point of coherence, cannot make anything stale)
+    if (threadIdx.x == 32 && kb1 > kb0) {
+        const size_t wt0 = static_cast<size_t>(mt) * p.k_blocks_total + kb0;
+        prefetch_l2_bulk(static_cast<const char*>(p.w_vals) + wt0 * p.w_tile_bytes, static_cast<uint32_t>((kb1 - kb0) * p.w_tile_bytes));
+        if (p.w_meta) prefetch_l2_bulk(static_cast<const char*>(p.w_meta) + wt0 * 2048, static_cast<uint32_t>((kb1 - kb0) * 2048));
+    }
+    pdl_wait();                          // nothing above reads or writes global memory
     pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));

@@ -57,6 +57,9 @@ struct GemmParams {
     int32_t* acc_out;            // [T][N] or null
     int32_t* split_acc;          // [T][N] int32 scratch when k_splits > 1: zero on entry, zero again on exit
     unsigned int* split_counters;   // one per output tile, same rule
+    const void* w_vals;          // the weight operand (compressed values, or the dense W_q) and its metadata
+    const void* w_meta;          //   (null for dense): only used to warm the L2 before the dependency wait
+    int w_tile_bytes;            // bytes of one 128 x 128 weight tile (8192 sparse, 16384 dense)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -270,7 +273,16 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     }
     __syncthreads();
     tcgen05_fence_after();
-    pdl_wait();                          // nothing above touches global memory
+    // The weights of this CTA's first tile go to L2 while the previous kernel is still finishing: a
+    // prefetch into L2 (the point of coherence) cannot make anything stale, whoever wrote them.
+    if (threadIdx.x == 32 && blockIdx.x < num_tiles) {
+        const int split = blockIdx.x % p.k_splits;
+        const int mt0 = (blockIdx.x / p.k_splits) % tiles_m;
+        const size_t wt0 = static_cast<size_t>(mt0) * p.k_blocks_total + static_cast<size_t>(split) * kb_per_split;
+        prefetch_l2_bulk(static_cast<const char*>(p.w_vals) + wt0 * p.w_tile_bytes, static_cast<uint32_t>(kb_per_split * p.w_tile_bytes));
+        if (p.w_meta) prefetch_l2_bulk(static_cast<const char*>(p.w_meta) + wt0 * 2048, static_cast<uint32_t>(kb_per_split * 2048));
+    }
+    pdl_wait();                          // nothing above reads or writes global memory
     pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));

@@ -295,6 +295,7 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.y = y; pp.g.out_bf16 = (dt == SBN_OUT_BF16);
     pp.g.acc_out = acc_out;
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
+    pp.g.w_vals = wvals; pp.g.w_meta = sparse ? meta : nullptr; pp.g.w_tile_bytes = sparse ? 8192 : 16384;
     pp.bn = bn;
     return sparse ? launch_pair<true>(ta, tb, te, pp, stream) : launch_pair<false>(ta, tb, te, pp, stream);
 }
@@ -360,6 +361,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     p.acc_out = acc_out;
     p.split_acc = splits > 1 ? static_cast<int32_t*>(ws) : nullptr;
     p.split_counters = splits > 1 ? reinterpret_cast<unsigned int*>(static_cast<char*>(ws) + split_acc_bytes(T, N)) : nullptr;
+    p.w_vals = wvals; p.w_meta = sparse ? meta : nullptr; p.w_tile_bytes = sparse ? 8192 : 16384;
 
     if (plan.cluster > 1) {
         p.k_splits = 1;

@@ -117,10 +117,6 @@ __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
     return (1u << (nib & 3u)) | (1u << ((nib >> 2) & 3u));
 }
 
-// Ask the L2 to fetch [p, p + bytes) (a multiple of 16 B) -- issued by one thread, no destination.
-__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
 constexpr int kQmpPrefetchAhead = 3;                       // pass 1 iterations (128 units = 64 KB each) ahead
 
 // Sum of `v` over the CTA in a fixed order; identical in every thread.
