@@ -61,6 +61,22 @@ def test_argument_validation_on_host(L):
     assert L.sbn_quant_act(p, 0, 256, p, p, None) == SHAPE
     assert L.sbn_quant_act(p, 4, 100, p, p, None) == SHAPE
     assert L.sbn_quant_act(odd, 4, 256, p, p, None) == ALIGN
+    nq = lambda **k: L.sbn_norm_quant_act(k.get("x", p), k.get("T", 4), k.get("K", 256), k.get("g", p),
+                                          ctypes.c_float(k.get("eps", 1e-6)), p, p, None)
+    assert nq(x=None) == NULL
+    assert nq(T=0) == SHAPE
+    assert nq(K=100) == SHAPE
+    assert nq(K=16384 + 128) == UNSUP           # row no longer fits in registers
+    assert nq(eps=-1.0) == SHAPE
+    assert nq(g=odd) == ALIGN
+    assert nq(x=odd) == ALIGN
+    qmp16 = lambda **k: L.sbn_quantize_mask_pack_bf16(k.get("W", p), k.get("N", 256), k.get("K", 256), k.get("n", 2),
+                                                      k.get("m", 4), p, p, p, None, None, None, p, k.get("wsb", 1 << 20), None)
+    assert qmp16(W=None) == NULL
+    assert qmp16(n=6, m=8) == UNSUP
+    assert qmp16(K=64) == SHAPE
+    assert qmp16(wsb=8) == WS
+    assert qmp16(W=odd) == ALIGN
     qmp = lambda **k: L.sbn_quantize_mask_pack(k.get("W", p), k.get("N", 256), k.get("K", 256), k.get("n", 2),
                                                k.get("m", 4), p, p, p, None, k.get("prev"), k.get("flip"),
                                                k.get("ws", p), k.get("wsb", 1 << 20), None)
