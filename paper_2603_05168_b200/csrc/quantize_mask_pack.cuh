@@ -36,6 +36,8 @@
 // and the per-element work is a compare.
 #pragma once
 
+#include <algorithm>
+
 #include "sbn_common.cuh"
 #include "layouts.cuh"
 
@@ -507,7 +509,10 @@ inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* v
 inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const QmpDesc* rest_dev, int count,
                                                   uint32_t max_units, QmpSlot* slots, cudaStream_t stream) {
     unsigned long long nonce = qmp_next_nonce();
-    const unsigned grid = max_units < static_cast<uint32_t>(kQmpMaxCtas) ? max_units : kQmpMaxCtas;
+    // every CTA must be resident at once (they exchange partial sums): never more CTAs than this
+    // device has SMs, and never more than the workspace has slots
+    const unsigned cap = static_cast<unsigned>(std::min(device_sm_count(), kQmpMaxCtas));
+    const unsigned grid = max_units < cap ? max_units : cap;
     if (!ensure_dynamic_smem<quantize_mask_pack_kernel>(kQmpSmemBytes)) return SBN_ERR_CUDA;
     // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if

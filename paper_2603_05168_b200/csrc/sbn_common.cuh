@@ -56,6 +56,19 @@ inline bool ensure_dynamic_smem(int bytes) {
     return true;
 }
 
+// SMs of the current device (cached per device; kNumSMs if the query fails).
+inline int device_sm_count() {
+    static std::atomic<int> cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kNumSMs;
+    int n = cached[dev].load(std::memory_order_acquire);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = kNumSMs;
+        cached[dev].store(n, std::memory_order_release);
+    }
+    return n;
+}
+
 // `cluster` > 1 launches the grid as clusters of that many consecutive CTAs (runtime cluster size).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
