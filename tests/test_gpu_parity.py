@@ -437,6 +437,36 @@ def test_gemm_parity_pair_kernel(sparse, T, N, K, bn):
     assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
 
 
+def _random_gemm_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        T = int(rng.choice([1, 2, 3, 7, 15, 16, 17, 31, 33, 63, 64, 65, 100, 127, 128, 129, 200, 255, 256, 257, 300,
+                            511, 513, 700, 1023, 1100]))
+        N = 128 * int(rng.integers(1, 9))
+        K = 128 * int(rng.integers(1, 25))
+        out.append((T, N, K))
+    return out
+
+
+@pytest.mark.parametrize("sparse", [True, False])
+@pytest.mark.parametrize("T,N,K", _random_gemm_shapes(24, seed=2024))
+def test_gemm_parity_automatic_dispatch_random_shapes(sparse, T, N, K):
+    # whatever kernel, tile and split the dispatcher picks for the shape: accumulators bit-exact,
+    # outputs within tolerance
+    r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=T + N + K)
+    if sparse:
+        y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    else:
+        y_ref, acc_ref = oracle.bitlinear(xq_ref, s_ref, r["dense_q"], r["scale"])
+    y, acc = gpu_gemm(sparse, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    yb, _ = gpu_gemm(sparse, xq, a_scale, g["dev"], out_dtype=torch.bfloat16, want_acc=False)
+    ref_bits = oracle.f32_to_bf16_bits(y_ref).astype(np.int32)
+    assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
+
+
 CLUSTER_CASES = [  # (T, N, K, token tile, cluster size): split-K reduced in distributed shared memory
     (64, 256, 2560, 64, 4), (1, 128, 256, 64, 2), (7, 256, 640, 64, 4),      # 5 k-blocks over 4 CTAs: one empty slice
     (100, 384, 6912, 64, 8), (130, 256, 1280, 128, 8), (200, 128, 384, 128, 2), (33, 512, 128, 64, 8),   # one k-block
