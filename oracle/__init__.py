@@ -173,6 +173,24 @@ def quantize_mask_pack(W):
                 near_tie=bool(nt[0]))
 
 
+def quantize_mask_nm(W, n_keep, m_group):
+    """Eq. 1-3 for a general N:M pattern (Sec. 2.2; 6:8 is the pattern of the paper's main
+    results): gamma and W_q from the DENSE matrix, the mask from the pre-quantised |W|,
+    W_eff = W_q (.) M.  No packed form: the paper fixes none, so parity is on W_eff and the mask.
+    Returns a dict: scale, mask, w_eff."""
+    W = _c(W, np.float32)
+    _, scale, _ = absmean_scale(W)
+    mask = nm_mask(W, n_keep, m_group)
+    w_eff = apply_mask(ternarize(W, scale), mask)
+    return dict(scale=scale, mask=mask, w_eff=w_eff)
+
+
+def nm_bitlinear(xq, a_scale, w_eff, scale, bias=None):
+    """Eq. 4 with W_eff given element by element (any N:M pattern): (y fp32 [T][N], acc int32)."""
+    acc = acc_dense(xq, w_eff)
+    return dequant(acc, scale, a_scale, bias), acc
+
+
 # -- activations ---------------------------------------------------------------------------------
 def quant_act(x_bf16_bits):
     """x given as uint16 bf16 bit patterns [T][K]; returns (xq int8 [T][K], a_scale fp32 [T])."""

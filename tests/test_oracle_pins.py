@@ -454,3 +454,63 @@ def test_norm_quant_act_degenerate_rows():
         assert np.all(np.abs(r["xq"].astype(np.int32)) == 127)
         assert np.all(np.sign(r["xq"][0, ::2]) == 1) and np.all(np.sign(r["xq"][0, 1::2]) == -1)
         assert abs(float(r["a_scale"][0]) * 127.0 - 1.0) < 3e-7
+
+
+# ---- general N:M composition (Sec. 2.2; the 6:8 pattern of the main results) -------------------
+def test_nm_composition_at_2_of_4_equals_the_packed_route():
+    # two routes to W_eff that share no packing code: element-wise composition vs unpacking the
+    # compressed values + metadata
+    W = inputs.latent_weights(64, 256, seed=71)
+    r = oracle.quantize_mask_pack(W)
+    w_eff_packed, mask_packed = oracle.unpack24(r["vals"], r["meta"])
+    c = oracle.quantize_mask_nm(W, 2, 4)
+    assert c["scale"] == r["scale"]
+    assert np.array_equal(c["mask"], mask_packed)
+    assert np.array_equal(c["w_eff"], w_eff_packed)
+
+
+def test_nm_composition_6_of_8_hand_case():
+    # gamma = mean|W| = (1+2+3+4+5+6+0.5+0.25)/8 = 2.71875; W/gamma rounds to
+    # 0 (0.37), 1 (0.74), -1, 1, 1 (1.84 clamps), -1, 0, 0; the two smallest |w| (columns 6, 7) are dropped
+    W = np.array([[1.0, 2.0, -3.0, 4.0, 5.0, -6.0, 0.5, -0.25]], np.float32)
+    c = oracle.quantize_mask_nm(W, 6, 8)
+    assert c["scale"] == np.float32(2.71875)
+    assert c["mask"].tolist() == [[1, 1, 1, 1, 1, 1, 0, 0]]
+    assert c["w_eff"].tolist() == [[0, 1, -1, 1, 1, -1, 0, 0]]
+    # all equal magnitudes: the lower columns win the ties
+    c = oracle.quantize_mask_nm(np.full((1, 8), -1.0, np.float32), 6, 8)
+    assert c["mask"].tolist() == [[1, 1, 1, 1, 1, 1, 0, 0]]
+    assert c["w_eff"].tolist() == [[-1, -1, -1, -1, -1, -1, 0, 0]]
+
+
+def test_nm_composition_6_of_8_properties_and_negative_control():
+    W = inputs.latent_weights(32, 512, seed=72)
+    c = oracle.quantize_mask_nm(W, 6, 8)
+    grp_mask = c["mask"].reshape(32, -1, 8)
+    assert (grp_mask.sum(-1) == 6).all()
+    a = np.abs(W).reshape(32, -1, 8)
+    kept_min = np.where(grp_mask == 1, a, np.inf).min(-1)
+    drop_max = np.where(grp_mask == 0, a, -np.inf).max(-1)
+    assert (kept_min >= drop_max).all()
+    # gamma is the DENSE mean (quant-then-mask, Eq. 3): same scale as the 2:4 and the unmasked paths
+    assert c["scale"] == oracle.quantize_mask_nm(W, 2, 4)["scale"] == oracle.quantize_mask_nm(W, 8, 8)["scale"]
+    # 8:8 is the dense BitLinear weight
+    assert np.array_equal(oracle.quantize_mask_nm(W, 8, 8)["w_eff"], oracle.ternarize(W, c["scale"]))
+    # negative control: gamma from the masked subset (mask-then-quant) gives another matrix
+    Wm = W * c["mask"]
+    _, scale_m, _ = oracle.absmean_scale(Wm)
+    assert scale_m != c["scale"]
+    assert not np.array_equal(oracle.ternarize(Wm, scale_m), c["w_eff"])
+
+
+def test_nm_bitlinear_is_the_integer_matmul():
+    rng = np.random.default_rng(73)
+    W = inputs.latent_weights(16, 64, seed=73)
+    c = oracle.quantize_mask_nm(W, 6, 8)
+    xq = rng.integers(-128, 128, size=(5, 64), dtype=np.int8)
+    a_scale = rng.uniform(0.01, 0.1, size=5).astype(np.float32)
+    y, acc = oracle.nm_bitlinear(xq, a_scale, c["w_eff"], c["scale"])
+    ref = xq.astype(np.int64) @ c["w_eff"].astype(np.int64).T
+    assert np.array_equal(acc, ref)
+    s = np.float32(c["scale"]) * a_scale
+    assert np.array_equal(y, (ref.astype(np.float32).T * s).T.astype(np.float32))
