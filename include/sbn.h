@@ -96,7 +96,8 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K);
  *   mask   = the two largest |W| of every group of four; equal magnitudes -> lower column kept
  * Arguments
  *   W          device, fp32 [N][K], read only
- *   n_keep, m_group  the N:M pattern; only 2:4 is implemented (else SBN_ERR_UNSUPPORTED)
+ *   n_keep, m_group  the N:M pattern: 2:4, or 6:8 (see "The 6:8 pattern" below); anything else
+ *              SBN_ERR_UNSUPPORTED
  *   vals       device out, int8, N*K/2 bytes, tiled order
  *   meta       device out, uint8, N*K/8 bytes, tiled order; may be the same buffer as prev_meta
  *   w_scale    device out, one fp32: `scale`
@@ -114,6 +115,27 @@ sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int 
                                   int8_t *vals, uint8_t *meta, float *w_scale, int8_t *dense_q,
                                   const uint8_t *prev_meta, unsigned long long *flip_bits,
                                   void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The 6:8 pattern (Sec. 2.2 with N:M = 6:8, the pattern of the paper's main results and of its
+ * throughput table): of every 8 consecutive input weights the 6 largest |W| are kept (equal
+ * magnitudes -> lower column kept); gamma, scale and W_q as above, from the dense matrix.
+ * The paper does not say how 6:8 reaches 2:4 hardware.  Here a group of 8 columns is covered by
+ * three overlapping 4-column windows (columns 0-3, 2-5, 4-7); the 6 kept columns are dealt out so
+ * that each window holds exactly two of them, which makes the [N][K] 6:8 matrix a 2:4 matrix
+ * [N][K'] with K' = sbn_expanded_k(K, 6, 8) = 3K/2 over activations expanded the same way
+ * (K' column 12 g + 4 w + s holds column 8 g + 2 w + s; sbn_quant_act_expand68 writes them).
+ * sbn_sparse_bitlinear then runs unchanged with K' in place of K: 3/4 of the dense MMA work.
+ * With n_keep = 6, m_group = 8, sbn_quantize_mask_pack and sbn_quantize_mask_pack_bf16 take
+ *   K          a multiple of 256 (else SBN_ERR_SHAPE)
+ *   vals       N*K'/2 bytes and meta N*K'/8 bytes: the 2:4 form of the [N][K'] matrix, tiled order
+ *   prev_meta  N*K'/8 bytes, the same form; flip_bits counts differing bits of the 6:8 masks [N][K]
+ *   dense_q    must be NULL (the dense W_q does not depend on the pattern; SBN_ERR_UNSUPPORTED)
+ * Which window carries a kept column is this library's choice (window 0 takes the kept ones of
+ * columns 0,1 and fills up with the lowest kept of 2,3; window 2 takes the kept ones of 6,7 and
+ * fills up with the highest kept of 4,5; window 1 takes the rest); W_eff and the mask are unique.
+ */
+int sbn_expanded_k(int K, int n_keep, int m_group);   /* K for 2:4, 3K/2 for 6:8 (K % 256 == 0), else 0 */
 
 /*
  * The same operation on bf16 master weights (Sec. 2.2 keeps the master weight "e.g. in bf16"): W is
@@ -193,6 +215,16 @@ sbn_status sbn_quantize_mask_pack_static_ws(const float *W, int N, int K, int n_
  */
 sbn_status sbn_quant_act(const void *x_bf16, int T, int K, int8_t *xq, float *a_scale,
                          void *stream);
+
+/*
+ * The same quantiser writing the activations expanded for the 6:8 pattern (see above): the codes
+ * and a_scale are exactly those of sbn_quant_act; xq is the tiled form of the [T][K'] matrix with
+ * K' = 3K/2, xq'[t][12 g + 4 w + s] = xq[t][8 g + 2 w + s] (g < K/8, w < 3, s < 4).
+ *   K    a multiple of 256
+ *   xq   device out, sbn_xq_bytes(T, 3K/2) bytes
+ */
+sbn_status sbn_quant_act_expand68(const void *x_bf16, int T, int K, int8_t *xq, float *a_scale,
+                                  void *stream);
 
 /*
  * Part 2 with the preceding normalisation fused in -- Algorithm 1, forward: x~ = Q_a(Norm(x)).

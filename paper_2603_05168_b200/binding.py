@@ -22,7 +22,7 @@ OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2
 
 EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
-    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_norm_quant_act", "sbn_sparse_bitlinear",
+    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -62,6 +62,10 @@ def lib() -> ctypes.CDLL:
         L.sbn_quantize_mask_pack_batched.argtypes = [i32, vp, vp, sz, vp]
         L.sbn_quant_act.restype = i32
         L.sbn_quant_act.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.sbn_quant_act_expand68.restype = i32
+        L.sbn_quant_act_expand68.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.sbn_expanded_k.restype = i32
+        L.sbn_expanded_k.argtypes = [i32, i32, i32]
         L.sbn_norm_quant_act.restype = i32
         L.sbn_norm_quant_act.argtypes = [vp, i32, i32, vp, ctypes.c_float, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
@@ -166,6 +170,16 @@ def sbn_quant_act(x_bf16, xq, a_scale):
     _check(lib().sbn_quant_act(_ptr(x_bf16), T, K, _ptr(xq), _ptr(a_scale), _stream()), "sbn_quant_act")
 
 
+def sbn_quant_act_expand68(x_bf16, xq, a_scale):
+    T, K = x_bf16.shape
+    _check(lib().sbn_quant_act_expand68(_ptr(x_bf16), T, K, _ptr(xq), _ptr(a_scale), _stream()),
+           "sbn_quant_act_expand68")
+
+
+def sbn_expanded_k(K: int, n_keep: int, m_group: int) -> int:
+    return int(lib().sbn_expanded_k(K, n_keep, m_group))
+
+
 def sbn_norm_quant_act(x_bf16, xq, a_scale, gain=None, eps: float = 1e-6):
     T, K = x_bf16.shape
     _check(lib().sbn_norm_quant_act(_ptr(x_bf16), T, K, _ptr(gain), ctypes.c_float(eps), _ptr(xq), _ptr(a_scale),
@@ -224,11 +238,14 @@ def sbn_launch_count() -> int:
 
 
 # -- small conveniences for callers (allocation only) ---------------------------------------------
-def alloc_packed(N: int, K: int, device="cuda", with_dense: bool = False):
-    """Device buffers for one packed weight matrix."""
+def alloc_packed(N: int, K: int, device="cuda", with_dense: bool = False, n_keep: int = 2, m_group: int = 4):
+    """Device buffers for one packed weight matrix (for 6:8: the 2:4 form over K' = 3K/2 columns)."""
+    Kp = sbn_expanded_k(K, n_keep, m_group)
+    if Kp == 0:
+        raise ValueError(f"unsupported pattern {n_keep}:{m_group} for K = {K}")
     out = dict(
-        vals=torch.empty((N, K // 2), dtype=torch.int8, device=device),
-        meta=torch.empty((N, K // 8), dtype=torch.uint8, device=device),
+        vals=torch.empty((N, Kp // 2), dtype=torch.int8, device=device),
+        meta=torch.empty((N, Kp // 8), dtype=torch.uint8, device=device),
         w_scale=torch.empty(1, dtype=torch.float32, device=device),
         ws=torch.empty(sbn_workspace_bytes(OP_QUANTIZE_MASK_PACK, 0, N, K), dtype=torch.uint8, device=device),
     )

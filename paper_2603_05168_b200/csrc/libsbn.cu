@@ -14,6 +14,7 @@
 #include "quant_act.cuh"
 #include "norm_quant_act.cuh"
 #include "quantize_mask_pack.cuh"
+#include "quantize_mask_pack68.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_pair_tcgen05.cuh"
 #include "gemm_splitk_cluster_tcgen05.cuh"
@@ -440,13 +441,21 @@ static sbn_status quantize_mask_pack_any(const void* W, bool w_bf16, int N, int 
                                          void* ws, size_t ws_bytes, void* stream) {
     if (!W || !vals || !meta || !w_scale) return SBN_ERR_NULL;
     if (prev_meta && !flip_bits) return SBN_ERR_NULL;
-    if (n_keep != 2 || m_group != 4) return SBN_ERR_UNSUPPORTED;
+    const bool p68 = n_keep == 6 && m_group == 8;
+    if (!p68 && (n_keep != 2 || m_group != 4)) return SBN_ERR_UNSUPPORTED;
+    if (p68 && dense_q) return SBN_ERR_UNSUPPORTED;           // the dense W_q does not depend on the pattern
     if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (p68 && K % (2 * kBK) != 0) return SBN_ERR_SHAPE;     // K' = 3K/2 must be a whole number of 128-column blocks
     if (!ws || ws_bytes < sizeof(QmpWorkspace)) return SBN_ERR_WORKSPACE;
     if (misaligned(W, 16) || misaligned(vals, 16) || misaligned(meta, 16) || misaligned(ws, 16) ||
         misaligned(w_scale, 4) || (dense_q && misaligned(dense_q, 16)) ||
         (prev_meta && misaligned(prev_meta, 16)) || (flip_bits && misaligned(flip_bits, 8)))
         return SBN_ERR_ALIGN;
+    if (p68) {
+        const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, nullptr, prev_meta, flip_bits);
+        return launch_quantize_mask_pack_batch<68>(d, nullptr, 1, d.num_units, static_cast<QmpWorkspace*>(ws)->slot,
+                                                   static_cast<cudaStream_t>(stream));
+    }
     return launch_quantize_mask_pack(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(ws),
                                      static_cast<cudaStream_t>(stream));
@@ -539,6 +548,20 @@ sbn_status sbn_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_
     if (T <= 0 || K <= 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
     if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
     return launch_quant_act(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_quant_act_expand68(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale, void* stream) {
+    if (!x_bf16 || !xq || !a_scale) return SBN_ERR_NULL;
+    if (T <= 0 || K <= 0 || K % (2 * kBK) != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4)) return SBN_ERR_ALIGN;
+    return launch_quant_act<true>(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
+}
+
+int sbn_expanded_k(int K, int n_keep, int m_group) {
+    if (K <= 0) return 0;
+    if (n_keep == 2 && m_group == 4) return K;
+    if (n_keep == 6 && m_group == 8 && K % (2 * kBK) == 0 && K <= (1 << 20)) return K / 2 * 3;
+    return 0;
 }
 
 sbn_status sbn_norm_quant_act(const void* x_bf16, int T, int K, const float* gain, float eps, int8_t* xq,

@@ -55,11 +55,37 @@ __device__ __forceinline__ size_t xq_tiled_u2_index(int t, int idx, size_t tb8) 
     return (atom << 7) + (r << 4) + ((chunk ^ r) << 1) + half;
 }
 
+// The 6:8 pattern runs on the 2:4 tensor cores over activations expanded from K to K' = 3K/2
+// columns (quantize_mask_pack68.cuh): every group of 8 codes q0..q7 becomes the three windows
+// q0..q3 | q2..q5 | q4..q7, i.e. K' column 12 g + 4 w + s holds column 8 g + 2 w + s.  A lane's
+// 8 codes leave as three 4-byte words; this is the index (in 4-byte units) of window w of
+// token t, group idx in the tiled xq layout of a [T][K'] matrix.
+__device__ __forceinline__ size_t xq68_tiled_u32_index(int t, int idx, int w, size_t tb8) {
+    const uint32_t kp = 12u * static_cast<uint32_t>(idx) + 4u * static_cast<uint32_t>(w);   // K' byte column
+    const uint32_t kb = kp >> 7;
+    const uint32_t chunk = (kp & 127u) >> 4;
+    const uint32_t r = static_cast<uint32_t>(t) & 7u;
+    const size_t atom = static_cast<size_t>(kb) * tb8 + (static_cast<uint32_t>(t) >> 3);
+    return (atom << 8) + (r << 5) + ((chunk ^ r) << 2) + ((kp & 15u) >> 2);
+}
+// Stores the 8 codes (o.x = q0..q3, o.y = q4..q7) of group idx of token t: plain, or expanded.
+template <bool EXPAND68>
+__device__ __forceinline__ void store_codes8(uint2* __restrict__ xq, int t, int idx, size_t tb8, const uint2 o) {
+    if constexpr (EXPAND68) {
+        uint32_t* q = reinterpret_cast<uint32_t*>(xq);
+        q[xq68_tiled_u32_index(t, idx, 0, tb8)] = o.x;
+        q[xq68_tiled_u32_index(t, idx, 1, tb8)] = __byte_perm(o.x, o.y, 0x5432);     // q2 q3 q4 q5
+        q[xq68_tiled_u32_index(t, idx, 2, tb8)] = o.y;
+    } else {
+        xq[xq_tiled_u2_index(t, idx, tb8)] = o;
+    }
+}
+
 // G threads per token row, VPT 16-byte vectors per thread (G * VPT >= K / 8).  Persistent CTAs:
 // every row group walks over rows with a grid-sized stride and loads its NEXT row while it reduces,
 // rounds and stores the current one, so each SM always has loads in flight (a non-pipelined
 // version of this kernel was latency-bound at a third of the HBM rate).
-template <int G, int VPT>
+template <int G, int VPT, bool EXPAND68 = false>
 __global__ void __launch_bounds__(kActThreads, (VPT <= 4) ? 3 : 2)
 quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
                  float* __restrict__ a_scale) {
@@ -117,7 +143,7 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
                     uint2 o;
                     o.x = quant_pair2(cur[i].x, cur[i].y, s_x);
                     o.y = quant_pair2(cur[i].z, cur[i].w, s_x);
-                    xq[xq_tiled_u2_index(row, idx, tb8)] = o;
+                    store_codes8<EXPAND68>(xq, row, idx, tb8, o);
                 }
             }
         }
@@ -128,6 +154,7 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
 
 // Rows too long for the register-resident kernel (K > 16384): one CTA per row, two passes over
 // the row (the second one served by L1/L2).
+template <bool EXPAND68 = false>
 __global__ void __launch_bounds__(kActThreads)
 quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
                           float* __restrict__ a_scale) {
@@ -154,35 +181,36 @@ quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* _
         uint2 o;
         o.x = quant_pair2(v.x, v.y, s_x);
         o.y = quant_pair2(v.z, v.w, s_x);
-        xq[xq_tiled_u2_index(row, idx, tb8)] = o;
+        store_codes8<EXPAND68>(xq, row, idx, tb8, o);
     }
 }
 
-template <int G, int VPT>
+template <int G, int VPT, bool EXPAND68>
 static void launch_quant_act_cfg(const uint4* x, int T, int nvec, uint2* q, float* a_scale, cudaStream_t stream) {
     constexpr int rows = kActThreads / G;
     const int ctas_per_sm = (VPT <= 4) ? 3 : 2;
     int grid = (T + rows - 1) / rows;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
-    launch_kernel(quant_act_kernel<G, VPT>, dim3(grid), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
+    launch_kernel(quant_act_kernel<G, VPT, EXPAND68>, dim3(grid), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
 }
 
+template <bool EXPAND68 = false>
 inline sbn_status launch_quant_act(const void* x_bf16, int T, int K, int8_t* xq, float* a_scale,
                                    cudaStream_t stream) {
     const int nvec = K / 8;
     const uint4* x = static_cast<const uint4*>(x_bf16);
     uint2* q = reinterpret_cast<uint2*>(xq);
     // smallest group that keeps <= 3 (then 4, 6, 8) vectors per thread
-    if (nvec <= 32 * 2) launch_quant_act_cfg<32, 2>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 64 * 2) launch_quant_act_cfg<64, 2>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 128 * 2) launch_quant_act_cfg<128, 2>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 128 * 3) launch_quant_act_cfg<128, 3>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 256 * 2) launch_quant_act_cfg<256, 2>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 256 * 3) launch_quant_act_cfg<256, 3>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 256 * 4) launch_quant_act_cfg<256, 4>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 256 * 6) launch_quant_act_cfg<256, 6>(x, T, nvec, q, a_scale, stream);
-    else if (nvec <= 256 * 8) launch_quant_act_cfg<256, 8>(x, T, nvec, q, a_scale, stream);
-    else launch_kernel(quant_act_long_row_kernel, dim3(T), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
+    if (nvec <= 32 * 2) launch_quant_act_cfg<32, 2, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 64 * 2) launch_quant_act_cfg<64, 2, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 128 * 2) launch_quant_act_cfg<128, 2, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 128 * 3) launch_quant_act_cfg<128, 3, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 2) launch_quant_act_cfg<256, 2, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 3) launch_quant_act_cfg<256, 3, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 4) launch_quant_act_cfg<256, 4, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 6) launch_quant_act_cfg<256, 6, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else if (nvec <= 256 * 8) launch_quant_act_cfg<256, 8, EXPAND68>(x, T, nvec, q, a_scale, stream);
+    else launch_kernel(quant_act_long_row_kernel<EXPAND68>, dim3(T), dim3(kActThreads), 0, stream, x, T, nvec, q, a_scale);
     ++g_launch_count;
     return cudaGetLastError() == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }

@@ -356,12 +356,19 @@ __device__ __forceinline__ void qmp_pass2_full(const QmpDesc& d, const QmpRange 
     }
 }
 
+// The pass of the 6:8 pattern (quantize_mask_pack68.cuh; FINAL = values only, exact threshold).
+template <bool BF16, bool FINAL>
+__device__ __forceinline__ double qmp68_pass(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
+                                             QmpEntry* list, unsigned int* list_count, double* s_warp,
+                                             unsigned int& flips);
+
 // Batch of `count` matrices in one persistent launch, software-pipelined over the matrices:
 //   S+P1(0) | S+P1(1) F(0) | S+P1(2) F(1) | ... | F(count-1)        (S sample, F exchange + fix-up)
 // so by the time a CTA needs gamma of matrix m, every CTA has long published its partial for m,
 // and the per-launch and per-exchange latencies are paid once per batch, not once per matrix.
 // The two undecided lists alternate between consecutive matrices.  `first` is matrix 0 (passed by
-// value), `rest` matrices 1.. in global memory.
+// value), `rest` matrices 1.. in global memory.  PATTERN: 24 or 68 (all matrices of a batch alike).
+template <int PATTERN>
 __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
                           QmpSlot* slots, unsigned long long nonce) {
@@ -401,11 +408,20 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             }
             __syncthreads();
             unsigned int flips = 0;
-            const double mine = d_cur.w_bf16
-                ? qmp_pass1<true>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                  &s_list_count[par], s_warp, flips)
-                : qmp_pass1<false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                   &s_list_count[par], s_warp, flips);
+            double mine;
+            if constexpr (PATTERN == 68) {
+                mine = d_cur.w_bf16
+                    ? qmp68_pass<true, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                              &s_list_count[par], s_warp, flips)
+                    : qmp68_pass<false, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                               &s_list_count[par], s_warp, flips);
+            } else {
+                mine = d_cur.w_bf16
+                    ? qmp_pass1<true>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                      &s_list_count[par], s_warp, flips)
+                    : qmp_pass1<false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                       &s_list_count[par], s_warp, flips);
+            }
             // this CTA's flip count of matrix m; it is added to the global counter one phase later,
             // after the exchange has shown that CTA 0 zeroed that counter
 #pragma unroll
@@ -463,7 +479,7 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             const unsigned int listed = s_list_count[par];
             const bool bracket_ok = s_bracket[par][0] <= thr && thr <= s_bracket[par][1] &&
                                     listed <= static_cast<unsigned int>(kQmpListCap) && d_prev.dense_q == nullptr &&
-                                    d_prev.num_units <= (1u << 26);        // listed byte offsets are 32-bit
+                                    d_prev.num_units <= (PATTERN == 68 ? (1u << 25) : (1u << 26));   // listed byte offsets are 32-bit
             if (bracket_ok) {
                 // every byte not on the list is already final; the listed ones get the exact compare
                 const QmpEntry* list = s_list + par * kQmpListCap;
@@ -472,6 +488,10 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                     const float w = list[e].w;
                     vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
                 }
+            } else if constexpr (PATTERN == 68) {
+                unsigned int unused = 0;
+                if (d_prev.w_bf16) qmp68_pass<true, true>(d_prev, rg_prev, thr, thr, nullptr, nullptr, s_warp, unused);
+                else qmp68_pass<false, true>(d_prev, rg_prev, thr, thr, nullptr, nullptr, s_warp, unused);
             } else {
                 if (d_prev.w_bf16) qmp_pass2_full<true>(d_prev, rg_prev, thr);
                 else qmp_pass2_full<false>(d_prev, rg_prev, thr);
@@ -506,6 +526,7 @@ inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* v
 }
 
 // Launch for `count` matrices: `first` by value, the others already copied to `rest_dev`.
+template <int PATTERN = 24>
 inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const QmpDesc* rest_dev, int count,
                                                   uint32_t max_units, QmpSlot* slots, cudaStream_t stream) {
     unsigned long long nonce = qmp_next_nonce();
@@ -513,11 +534,11 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
     // device has SMs, and never more than the workspace has slots
     const unsigned cap = static_cast<unsigned>(std::min(device_sm_count(), kQmpMaxCtas));
     const unsigned grid = max_units < cap ? max_units : cap;
-    if (!ensure_dynamic_smem<quantize_mask_pack_kernel>(kQmpSmemBytes)) return SBN_ERR_CUDA;
+    if (!ensure_dynamic_smem<quantize_mask_pack_kernel<PATTERN>>(kQmpSmemBytes)) return SBN_ERR_CUDA;
     // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
-    const cudaError_t err = launch_kernel(quantize_mask_pack_kernel, dim3(grid), dim3(kQmpThreads), kQmpSmemBytes, stream,
+    const cudaError_t err = launch_kernel(quantize_mask_pack_kernel<PATTERN>, dim3(grid), dim3(kQmpThreads), kQmpSmemBytes, stream,
                                           first, rest_dev, count, slots, nonce);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;

@@ -98,6 +98,66 @@ def gpu_quantize_mask_pack(W: np.ndarray, with_dense=True, prev_meta=None, in_pl
     return out
 
 
+# ---- the 6:8 pattern: index maps between the K columns and the K' = 3K/2 expanded columns --------
+def expand68_columns(K):
+    """For every expanded column 12 g + 4 w + s the original column 8 g + 2 w + s (as documented in
+    include/sbn.h)."""
+    kp = np.arange(3 * K // 2, dtype=np.int64)
+    g, rem = kp // 12, kp % 12
+    return 8 * g + 2 * (rem // 4) + (rem % 4)
+
+
+def fold68(mat_p):
+    """[N][K'] array over the expanded columns -> [N][K]: sum of the (up to two) expanded columns that
+    carry each original column."""
+    N, Kp = mat_p.shape
+    K = Kp * 2 // 3
+    out = np.zeros((N, K), np.int64)
+    np.add.at(out, (np.arange(N)[:, None], expand68_columns(K)[None, :]), mat_p.astype(np.int64))
+    return out
+
+
+def gpu_quantize_mask_pack68(W: np.ndarray, prev_meta=None, in_place=False, w_bf16_bits=None):
+    """6:8 pack.  Returns the 2:4 form of the [N][K'] matrix in plain order (vals [N][K'/2],
+    meta [N][K'/8]), the scale, the device buffers and, with prev_meta (plain [N][K'/8]), flips."""
+    N, K = W.shape
+    Kp = 3 * K // 2
+    bufs = b.alloc_packed(N, K, n_keep=6, m_group=8)
+    Wd = dev(W) if w_bf16_bits is None else bf16_dev(w_bf16_bits)
+    flip = pm = None
+    if prev_meta is not None:
+        flip = torch.full((1,), 12345, dtype=torch.int64, device="cuda")
+        prev_tiled = tile_meta(prev_meta).reshape(N, Kp // 8)
+        if in_place:
+            bufs["meta"].copy_(dev(prev_tiled))
+            pm = bufs["meta"]
+        else:
+            pm = dev(prev_tiled)
+    bufs["vals"].fill_(77)                                   # every byte must be written
+    if not in_place:
+        bufs["meta"].fill_(0xEE)
+    b.sbn_quantize_mask_pack(Wd, bufs["vals"], bufs["meta"], bufs["w_scale"], bufs["ws"],
+                             prev_meta=pm, flip_bits=flip, n_keep=6, m_group=8)
+    b.sbn_check_status()
+    out = dict(vals=untile(bufs["vals"].cpu().numpy(), _vals_offsets(N, Kp)),
+               meta=untile(bufs["meta"].cpu().numpy(), _meta_offsets(N, Kp)),
+               scale=np.float32(bufs["w_scale"].cpu().numpy()[0]), dev=bufs)
+    if flip is not None:
+        out["flips"] = int(flip.cpu().numpy()[0])
+    return out
+
+
+def gpu_quant_act_expand68(x_bits: np.ndarray):
+    T, K = x_bits.shape
+    xd = bf16_dev(x_bits)
+    xq = b.alloc_xq(T, 3 * K // 2)
+    xq.fill_(99)
+    a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+    b.sbn_quant_act_expand68(xd, xq, a_scale)
+    b.sbn_check_status()
+    return xq, a_scale
+
+
 def gpu_quant_act(x_bits: np.ndarray):
     T, K = x_bits.shape
     xd = bf16_dev(x_bits)

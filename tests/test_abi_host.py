@@ -73,7 +73,8 @@ def test_argument_validation_on_host(L):
     qmp16 = lambda **k: L.sbn_quantize_mask_pack_bf16(k.get("W", p), k.get("N", 256), k.get("K", 256), k.get("n", 2),
                                                       k.get("m", 4), p, p, p, None, None, None, p, k.get("wsb", 1 << 20), None)
     assert qmp16(W=None) == NULL
-    assert qmp16(n=6, m=8) == UNSUP
+    assert qmp16(n=5, m=8) == UNSUP
+    assert qmp16(n=6, m=8, K=384) == SHAPE      # 6:8 needs K % 256 == 0
     assert qmp16(K=64) == SHAPE
     assert qmp16(wsb=8) == WS
     assert qmp16(W=odd) == ALIGN
@@ -81,7 +82,14 @@ def test_argument_validation_on_host(L):
                                                k.get("m", 4), p, p, p, None, k.get("prev"), k.get("flip"),
                                                k.get("ws", p), k.get("wsb", 1 << 20), None)
     assert qmp(W=None) == NULL
-    assert qmp(n=6, m=8) == UNSUP
+    assert qmp(n=4, m=8) == UNSUP
+    assert qmp(n=6, m=8, K=128) == SHAPE        # 6:8 needs K % 256 == 0
+    assert L.sbn_quantize_mask_pack(p, 256, 256, 6, 8, p, p, p, p, None, None, p, 1 << 20, None) == UNSUP   # 6:8 with dense_q
+    assert L.sbn_quant_act_expand68(None, 4, 256, p, p, None) == NULL
+    assert L.sbn_quant_act_expand68(p, 4, 384, p, p, None) == SHAPE
+    assert L.sbn_quant_act_expand68(p, 4, 256, odd, p, None) == ALIGN
+    assert L.sbn_expanded_k(2560, 6, 8) == 3840 and L.sbn_expanded_k(2560, 2, 4) == 2560
+    assert L.sbn_expanded_k(2560 + 128, 6, 8) == 0 and L.sbn_expanded_k(2560, 3, 4) == 0
     assert qmp(N=100) == SHAPE
     assert qmp(K=64) == SHAPE
     assert qmp(wsb=8) == WS

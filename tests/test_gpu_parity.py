@@ -12,7 +12,8 @@ from paper_2603_05168_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
-    from gpu_harness import (gpu_norm_quant_act, bf16_dev, bf16_tensor_bits, dev, gpu_gemm, gpu_quant_act, gpu_quantize_mask_pack,
+    from gpu_harness import (gpu_norm_quant_act, bf16_dev, bf16_tensor_bits, dev, expand68_columns, fold68, gpu_gemm,
+                             gpu_quant_act, gpu_quant_act_expand68, gpu_quantize_mask_pack, gpu_quantize_mask_pack68,
                              xq_to_numpy, y_to_f32_numpy)
 
 
@@ -274,6 +275,157 @@ def test_quantize_mask_pack_everything_near_the_threshold(N, K):
     g = gpu_quantize_mask_pack(W, with_dense=False)
     assert g["scale"] == r["scale"]
     assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
+
+
+# ---- the 6:8 pattern (Sec. 2.2): three overlapping windows turn it into 2:4 over K' = 3K/2 -------
+def _decode68(g):
+    """GPU 6:8 result -> (mask [N][K], W_eff [N][K]) after checking that it is a valid 2:4 form in
+    which no original column is carried by two windows."""
+    nib = np.stack([g["meta"] & 15, g["meta"] >> 4], axis=-1)
+    assert ((nib & 3) < (nib >> 2)).all(), "metadata indices must be ascending within a group of four"
+    w_eff_p, mask_p = oracle.unpack24(g["vals"], g["meta"])
+    assert (mask_p.reshape(mask_p.shape[0], -1, 4).sum(-1) == 2).all()
+    assert np.isin(g["vals"], (-1, 0, 1)).all()
+    mask = fold68(mask_p)
+    assert mask.max() <= 1, "a column is kept in two windows"
+    return mask.astype(np.uint8), fold68(w_eff_p).astype(np.int8)
+
+
+def _assert_pack68(W, g):
+    r = oracle.quantize_mask_nm(W, 6, 8)
+    mask, w_eff = _decode68(g)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(mask, r["mask"])
+    assert np.array_equal(w_eff, r["w_eff"])
+    return r
+
+
+@pytest.mark.parametrize("N,K,seed", [(128, 256, 50), (256, 512, 51), (384, 2560, 52), (128, 6912, 53), (2048, 2560, 54),
+                                      (640, 1280, 55)])
+def test_pack68_parity(N, K, seed):
+    W = inputs.latent_weights(N, K, seed=seed)
+    _assert_pack68(W, gpu_quantize_mask_pack68(W))
+
+
+def test_pack68_bf16_masters_and_ties():
+    bits = inputs.f32_to_bf16_bits(inputs.latent_weights(384, 2560, seed=56))
+    W = (bits.astype(np.uint32) << 16).view(np.float32).reshape(384, 2560)
+    _assert_pack68(W, gpu_quantize_mask_pack68(W, w_bf16_bits=bits))
+
+
+def test_pack68_every_kept_set():
+    # all 28 ways of dropping two columns of eight, each with distinct magnitudes and with ties at
+    # the boundary (the dropped pair equal to a kept column: the lower column must win)
+    N, K = 128, 256
+    rng = np.random.default_rng(57)
+    W = rng.uniform(1.0, 2.0, size=(N, K)).astype(np.float32) * rng.choice(np.array([-1, 1], np.float32), size=(N, K))
+    pairs = [(i, j) for i in range(8) for j in range(i + 1, 8)]
+    grp = W.reshape(N, K // 8, 8)
+    for idx, (i, j) in enumerate(pairs):
+        grp[idx, :, i] *= np.float32(0.01)
+        grp[idx, :, j] *= np.float32(0.02)
+        grp[idx + 28, :, :] = np.float32(1.0)                 # all equal but two smaller ones
+        grp[idx + 28, :, i] = np.float32(0.5)
+        grp[idx + 28, :, j] = np.float32(0.5)
+        grp[idx + 56, :, :] = np.float32(-0.5)                # ties between dropped and kept columns
+        grp[idx + 56, :, i] = np.float32(0.75)
+        grp[idx + 56, :, j] = np.float32(-0.75)
+    W[120, :] = 0.0                                           # all-zero groups: columns 0..5 kept
+    W[121, :] = 0.3
+    _assert_pack68(W, gpu_quantize_mask_pack68(W))
+
+
+def test_pack68_misleading_sample_and_list_overflow():
+    N, K = 1024, 2560
+    W = inputs.latent_weights(N, K, seed=58)
+    KB = K // 128
+    for u in _sampled_units(N, K):
+        n, kb = divmod(int(u), KB)
+        W[n, kb * 128:(kb + 1) * 128] *= np.float32(1e-3)
+    _assert_pack68(W, gpu_quantize_mask_pack68(W))
+    # nearly every kept value within 1 % of the rounding threshold: the list overflows
+    rng = np.random.default_rng(59)
+    a = np.float32(0.01)
+    G = N * K // 8
+    groups = (a * (1.0 + 0.01 * rng.uniform(-1, 1, size=(G, 8)))).astype(np.float32)
+    groups *= rng.choice(np.array([-1.0, 1.0], np.float32), size=(G, 8))
+    heavy = (np.arange(G) % 16) == 0
+    # mean |w| must come out near 2a for thr = scale / 2 to sit at a: heavy groups carry the rest
+    groups[heavy] *= np.float32(17.0)
+    W = groups.reshape(N, K)
+    r = _assert_pack68(W, gpu_quantize_mask_pack68(W))
+    frac = np.count_nonzero(r["w_eff"]) / (0.75 * r["w_eff"].size)
+    assert 0.2 < frac < 0.9, "the construction should split the kept values"
+    # a short list (small matrix): the fix-up route
+    _assert_pack68(W[:256, :512].copy(), gpu_quantize_mask_pack68(W[:256, :512].copy()))
+
+
+def test_pack68_degenerate_scales():
+    Z = np.zeros((128, 256), np.float32)
+    g = gpu_quantize_mask_pack68(Z)
+    assert g["scale"] == np.float32(1e-5)
+    _assert_pack68(Z, g)
+    tiny = np.full((128, 256), 7e-6, np.float32)
+    _assert_pack68(tiny, gpu_quantize_mask_pack68(tiny))
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+def test_pack68_flip_count(in_place):
+    W = inputs.latent_weights(256, 2560, seed=60)
+    Wp = inputs.perturb_weights(W, seed=61, sigma=1e-4)
+    g0 = gpu_quantize_mask_pack68(W)
+    r0 = _assert_pack68(W, g0)
+    g1 = gpu_quantize_mask_pack68(Wp, prev_meta=g0["meta"], in_place=in_place)
+    r1 = _assert_pack68(Wp, g1)
+    expected = oracle.flip_count(r0["mask"], r1["mask"])
+    assert expected > 0
+    assert g1["flips"] == expected
+    assert gpu_quantize_mask_pack68(W, prev_meta=g0["meta"])["flips"] == 0
+
+
+def test_pack68_rejects_what_it_cannot_do():
+    p = b.alloc_packed(128, 256, n_keep=6, m_group=8)
+    W = dev(np.zeros((128, 256), np.float32))
+    dense = torch.empty((128, 256), dtype=torch.int8, device="cuda")
+    with pytest.raises(b.SbnError):
+        b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"], dense_q=dense, n_keep=6, m_group=8)
+    W2 = dev(np.zeros((128, 384), np.float32))                    # K' = 576 is not a multiple of 128
+    with pytest.raises(b.SbnError):
+        b.sbn_quantize_mask_pack(W2, p["vals"], p["meta"], p["w_scale"], p["ws"], n_keep=6, m_group=8)
+    assert b.sbn_expanded_k(256, 6, 8) == 384 and b.sbn_expanded_k(384, 6, 8) == 0
+    assert b.sbn_expanded_k(384, 2, 4) == 384 and b.sbn_expanded_k(256, 5, 8) == 0
+
+
+@pytest.mark.parametrize("T,K", [(64, 256), (1, 2560), (5, 512), (67, 2560), (33, 6912), (19, 11008), (300, 4096),
+                                 (3, 32768)])
+def test_quant_act_expand68_parity(T, K):
+    bits = inputs.activations_bf16(T, K, seed=T + K, token_lognormal_sigma=1.0)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    xq, s = gpu_quant_act_expand68(bits)
+    assert np.array_equal(s.cpu().numpy(), s_ref)
+    assert np.array_equal(xq_to_numpy(xq, T, 3 * K // 2), xq_ref[:, expand68_columns(K)])
+
+
+SPARSE68_SHAPES = [(64, 256, 256), (1, 128, 512), (5, 128, 256), (130, 384, 512), (300, 256, 2560), (64, 128, 6912),
+                   (700, 512, 1280), (1100, 640, 2560)]
+
+
+@pytest.mark.parametrize("T,N,K", SPARSE68_SHAPES)
+def test_sparse68_layer_parity(T, N, K):
+    # whole 6:8 layer: pack -> expanded activations -> the unchanged sparse GEMM over K' columns;
+    # the accumulators must be those of the plain integer matmul with the oracle's 6:8 W_eff
+    W = inputs.latent_weights(N, K, seed=T + N + K)
+    bits = inputs.activations_bf16(T, K, seed=T + N + K + 1, token_lognormal_sigma=0.5)
+    r = oracle.quantize_mask_nm(W, 6, 8)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    y_ref, acc_ref = oracle.nm_bitlinear(xq_ref, s_ref, r["w_eff"], r["scale"])
+    g = gpu_quantize_mask_pack68(W)
+    xq, a_scale = gpu_quant_act_expand68(bits)
+    y, acc = gpu_gemm(True, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    yb, _ = gpu_gemm(True, xq, a_scale, g["dev"], out_dtype=torch.bfloat16, want_acc=False)
+    assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - oracle.f32_to_bf16_bits(y_ref).astype(np.int32)).max() <= 1
 
 
 def test_worked_example_not_the_negative_control():
