@@ -593,6 +593,94 @@ def run_decode_sweep(args):
                       "rows": rows, "gpu_launches": b.sbn_launch_count()}))
 
 
+def run_pattern68(args):
+    """The 6:8 pattern (the paper's deployed pattern) next to 2:4 and dense on the same matrices:
+    per layer the isolated kernels with a cold L2 (pack, activation quantiser, GEMM), and the
+    whole step (pack + quantise + GEMM for all layers) back to back.  Work is counted as the dense
+    2 T N K whatever the pattern, so TOPS compare directly.  6:8 runs as 2:4 over 3K/2 expanded
+    columns: 3/4 of the dense MMA work."""
+    import torch
+    from paper_2603_05168_b200 import binding as b
+    from paper_2603_05168_b200 import build as sbn_build
+    sbn_build.build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    time_cold = _cold_timer(torch, stream, flush)
+    cases = [(n, K, N, 4096) for n, K, N in inputs.SHAPES_2B] + [("down_7b", 11008, 4096, 8192)]
+    rows, layers = [], []
+    for i, (name, K, N, T) in enumerate(cases):
+        W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i)).cuda()
+        x = torch.from_numpy(inputs.activations_bf16(T, K, seed=11 + i).view(np.int16)).cuda().view(torch.bfloat16)
+        p24 = b.alloc_packed(N, K, with_dense=True)
+        p68 = b.alloc_packed(N, K, n_keep=6, m_group=8)
+        Kp = b.sbn_expanded_k(K, 6, 8)
+        xq, xq68 = b.alloc_xq(T, K), b.alloc_xq(T, Kp)
+        a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+        y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+        ws24 = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, K)
+        ws68 = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, Kp)
+        wsd = b.alloc_gemm_ws(b.OP_BITLINEAR, T, N, K)
+        f = {
+            "pack24": lambda W=W, p=p24: b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"]),
+            "pack68": lambda W=W, p=p68: b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"], n_keep=6, m_group=8),
+            "act": lambda x=x, xq=xq, a=a_scale: b.sbn_quant_act(x, xq, a),
+            "act68": lambda x=x, xq=xq68, a=a_scale: b.sbn_quant_act_expand68(x, xq, a),
+            "gemm24": lambda xq=xq, a=a_scale, p=p24, y=y, ws=ws24: b.sbn_sparse_bitlinear(xq, a, p["vals"], p["meta"], p["w_scale"], y, ws=ws),
+            "gemm68": lambda xq=xq68, a=a_scale, p=p68, y=y, ws=ws68: b.sbn_sparse_bitlinear(xq, a, p["vals"], p["meta"], p["w_scale"], y, ws=ws),
+            "dense": lambda xq=xq, a=a_scale, p=p24, y=y, ws=wsd: b.sbn_bitlinear(xq, a, p["dense_q"], p["w_scale"], y, ws=ws),
+        }
+        b.sbn_quantize_mask_pack(W, p24["vals"], p24["meta"], p24["w_scale"], p24["ws"], dense_q=p24["dense_q"])
+        for fn in f.values():
+            for _ in range(3):
+                fn()
+        us = {k: time_cold(fn, 12) for k, fn in f.items()}
+        ops = 2.0 * T * N * K
+        rows.append({"layer": name, "T": T, "K": K, "N": N, **{k + "_us": round(v, 2) for k, v in us.items()},
+                     "dense_tops": round(ops / us["dense"] / 1e6, 1), "sparse24_tops": round(ops / us["gemm24"] / 1e6, 1),
+                     "sparse68_tops": round(ops / us["gemm68"] / 1e6, 1),
+                     "speedup24_vs_dense": round(us["dense"] / us["gemm24"], 3),
+                     "speedup68_vs_dense": round(us["dense"] / us["gemm68"], 3),
+                     "pack68_gbs": round(N * K * (4 + 0.9375) / us["pack68"] / 1e3, 1),       # W once + 0.75 B vals + 0.1875 B meta
+                     "act68_gbs": round((T * K * 3.5 + T * 4) / us["act68"] / 1e3, 1)})       # 2 B read + 1.5 B written
+        if T == 4096:
+            layers.append((f, ops))
+    # whole steps over the four 2B-shaped layers, back to back
+    def step(kind):
+        for f, _ in layers:
+            if kind == "68":
+                f["pack68"](); f["act68"](); f["gemm68"]()
+            elif kind == "24":
+                f["pack24"](); f["act"](); f["gemm24"]()
+            else:
+                f["act"](); f["dense"]()
+    steps = {}
+    for kind in ("68", "24", "dense_forward_only"):
+        for _ in range(3):
+            step(kind)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(int(2e7))
+        a = torch.cuda.Event(enable_timing=True)
+        c = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.steps):
+            step(kind)
+        c.record(stream)
+        torch.cuda.synchronize()
+        steps[kind] = a.elapsed_time(c) / args.steps
+    b.sbn_check_status()
+    total_ops = sum(o for _, o in layers)
+    print(json.dumps({"metric": "6:8 sparse ternary BitLinear next to 2:4 and dense (dense-equivalent TOPS)", "unit": "TOPS",
+                      "workload": "p68", "rows": rows,
+                      "step_ms": {k: round(v, 4) for k, v in steps.items()},
+                      "step_tops": {k: round(total_ops / v / 1e9, 1) for k, v in steps.items()},
+                      "note": "steps 68 / 24: one pack launch per layer (the headline step batches the 2:4 packs into one launch); "
+                              "dense_forward_only: activation quantiser + dense GEMM, no packing",
+                      "gpu_launches": b.sbn_launch_count()}))
+
+
 def run_dynamic_step(args):
     """Dynamic-mask training step (the mask is recomputed every step): perturb all master weights
     (outside the timed region), then timed: quantise/mask/pack all 30 x 7 matrices with the flip
@@ -699,10 +787,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "dyn"],
+    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "dyn", "p68"],
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1..512), sparse vs dense, cold L2 and streamed; "
-                         "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048")
+                         "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048; "
+                         "p68 = the 6:8 pattern next to 2:4 and dense on the same matrices")
     ap.add_argument("--masters", default="fp32", choices=["fp32", "bf16"],
                     help="precision of the master weights the pack kernel reads (default fp32, the configuration of the metric)")
     ap.add_argument("--only-step", action="store_true", help="time the step only (used for profiler runs)")
@@ -713,6 +802,8 @@ def main():
         run_decode_sweep(args)
     elif args.workload == "dyn":
         run_dynamic_step(args)
+    elif args.workload == "p68":
+        run_pattern68(args)
     else:
         run_ours(args)
 

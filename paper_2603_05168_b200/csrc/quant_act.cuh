@@ -58,24 +58,35 @@ __device__ __forceinline__ size_t xq_tiled_u2_index(int t, int idx, size_t tb8) 
 // The 6:8 pattern runs on the 2:4 tensor cores over activations expanded from K to K' = 3K/2
 // columns (quantize_mask_pack68.cuh): every group of 8 codes q0..q7 becomes the three windows
 // q0..q3 | q2..q5 | q4..q7, i.e. K' column 12 g + 4 w + s holds column 8 g + 2 w + s.  A lane's
-// 8 codes leave as three 4-byte words; this is the index (in 4-byte units) of window w of
-// token t, group idx in the tiled xq layout of a [T][K'] matrix.
-__device__ __forceinline__ size_t xq68_tiled_u32_index(int t, int idx, int w, size_t tb8) {
-    const uint32_t kp = 12u * static_cast<uint32_t>(idx) + 4u * static_cast<uint32_t>(w);   // K' byte column
+// 8 codes become 12 bytes; the 48 bytes of four adjacent lanes (a quad) are three whole 16-byte
+// chunks of the tiled [T][K'] layout, which lanes 0..2 of the quad store after one exchange.
+// Index (in 16-byte units) of chunk c (0..2) of the quad that starts at group idx4 (a multiple of 4)
+// of token t.
+__device__ __forceinline__ size_t xq68_tiled_u4_index(int t, int idx4, int c, size_t tb8) {
+    const uint32_t kp = 12u * static_cast<uint32_t>(idx4) + 16u * static_cast<uint32_t>(c);   // K' byte column
     const uint32_t kb = kp >> 7;
     const uint32_t chunk = (kp & 127u) >> 4;
     const uint32_t r = static_cast<uint32_t>(t) & 7u;
     const size_t atom = static_cast<size_t>(kb) * tb8 + (static_cast<uint32_t>(t) >> 3);
-    return (atom << 8) + (r << 5) + ((chunk ^ r) << 2) + ((kp & 15u) >> 2);
+    return (atom << 6) + (r << 3) + (chunk ^ r);
 }
 // Stores the 8 codes (o.x = q0..q3, o.y = q4..q7) of group idx of token t: plain, or expanded.
+// Expanded: must be reached by all 32 lanes of a warp together (idx consecutive over the lanes).
 template <bool EXPAND68>
 __device__ __forceinline__ void store_codes8(uint2* __restrict__ xq, int t, int idx, size_t tb8, const uint2 o) {
     if constexpr (EXPAND68) {
-        uint32_t* q = reinterpret_cast<uint32_t*>(xq);
-        q[xq68_tiled_u32_index(t, idx, 0, tb8)] = o.x;
-        q[xq68_tiled_u32_index(t, idx, 1, tb8)] = __byte_perm(o.x, o.y, 0x5432);     // q2 q3 q4 q5
-        q[xq68_tiled_u32_index(t, idx, 2, tb8)] = o.y;
+        const uint32_t mid = __byte_perm(o.x, o.y, 0x5432);                          // q2 q3 q4 q5
+        const uint32_t na = __shfl_down_sync(0xFFFFFFFFu, o.x, 1);
+        const uint32_t nm = __shfl_down_sync(0xFFFFFFFFu, mid, 1);
+        const uint32_t nc = __shfl_down_sync(0xFFFFFFFFu, o.y, 1);
+        const int j = idx & 3;
+        // the quad's 12 words are a m c | a m c | a m c | a m c; lane j stores words 4j .. 4j+3
+        uint4 v;
+        v.x = j == 0 ? o.x : (j == 1 ? mid : o.y);
+        v.y = j == 0 ? mid : (j == 1 ? o.y : na);
+        v.z = j == 0 ? o.y : (j == 1 ? na : nm);
+        v.w = j == 0 ? na : (j == 1 ? nm : nc);
+        if (j < 3) reinterpret_cast<uint4*>(xq)[xq68_tiled_u4_index(t, idx & ~3, j, tb8)] = v;
     } else {
         xq[xq_tiled_u2_index(t, idx, tb8)] = o;
     }

@@ -98,13 +98,17 @@ __device__ __forceinline__ double qmp68_pass(const QmpDesc& d, const QmpRange rg
     uint8_t* vals_b = reinterpret_cast<uint8_t*>(d.vals);
     double acc = 0.0;
     const uint32_t u_first = rg.u_begin + 2 * warp + (lane >> 4);
+    const uint32_t step_n = kStep / KB, step_kb = kStep % KB;  // a thread's next unit, without a division
+    uint32_t n = u_first / KB;
+    uint32_t kb = u_first - n * KB;
     if (threadIdx.x == 0) {
         for (int j = 1; j < kQmpPrefetchAhead; ++j) {
             const uint32_t ub = rg.u_begin + j * kStep;
             if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, kStep) * kUnitBytes);
         }
     }
-    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += kStep) {
+    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += kStep, n += step_n, kb += step_kb) {
+        if (kb >= KB) { kb -= KB; ++n; }
         if (threadIdx.x == 0) {
             const uint32_t ub = u0 + kQmpPrefetchAhead * kStep;
             if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, kStep) * kUnitBytes);
@@ -114,8 +118,6 @@ __device__ __forceinline__ double qmp68_pass(const QmpDesc& d, const QmpRange rg
         float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
         if (active) qmp_load_group_pair<BF16>(d.W, uq, l16, va, vb);
         if constexpr (!FINAL) acc += abs_sum4(va) + abs_sum4(vb);
-        const uint32_t n = uq / KB;
-        const uint32_t kb = uq - n * KB;
         const uint32_t g_row = kb * 16u + l16;                 // group of 8 within the row
         const float w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
         float a[8];
