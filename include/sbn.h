@@ -241,6 +241,11 @@ sbn_status sbn_quant_act_expand68(const void *x_bf16, int T, int K, int8_t *xq, 
 sbn_status sbn_norm_quant_act(const void *x_bf16, int T, int K, const float *gain, float eps,
                               int8_t *xq, float *a_scale, void *stream);
 
+/* The same with the codes written expanded for the 6:8 pattern (as sbn_quant_act_expand68:
+ * K % 256 == 0, xq of sbn_xq_bytes(T, 3K/2) bytes). */
+sbn_status sbn_norm_quant_act_expand68(const void *x_bf16, int T, int K, const float *gain,
+                                       float eps, int8_t *xq, float *a_scale, void *stream);
+
 /*
  * Part 3 -- Eq. 4: acc[t][n] = sum_k xq[t][k] * W_eff[n][k] in int32 (exact), then
  *   y[t][n] = float(acc[t][n]) * (w_scale * a_scale[t]) (+ bias[n]),

@@ -22,7 +22,7 @@ OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2
 
 EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
-    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_sparse_bitlinear",
+    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_expanded_k.argtypes = [i32, i32, i32]
         L.sbn_norm_quant_act.restype = i32
         L.sbn_norm_quant_act.argtypes = [vp, i32, i32, vp, ctypes.c_float, vp, vp, vp]
+        L.sbn_norm_quant_act_expand68.restype = i32
+        L.sbn_norm_quant_act_expand68.argtypes = [vp, i32, i32, vp, ctypes.c_float, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
         L.sbn_sparse_bitlinear.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
         L.sbn_bitlinear.restype = i32
@@ -180,10 +182,11 @@ def sbn_expanded_k(K: int, n_keep: int, m_group: int) -> int:
     return int(lib().sbn_expanded_k(K, n_keep, m_group))
 
 
-def sbn_norm_quant_act(x_bf16, xq, a_scale, gain=None, eps: float = 1e-6):
+def sbn_norm_quant_act(x_bf16, xq, a_scale, gain=None, eps: float = 1e-6, expand68: bool = False):
     T, K = x_bf16.shape
-    _check(lib().sbn_norm_quant_act(_ptr(x_bf16), T, K, _ptr(gain), ctypes.c_float(eps), _ptr(xq), _ptr(a_scale),
-                                    _stream()), "sbn_norm_quant_act")
+    fn = lib().sbn_norm_quant_act_expand68 if expand68 else lib().sbn_norm_quant_act
+    _check(fn(_ptr(x_bf16), T, K, _ptr(gain), ctypes.c_float(eps), _ptr(xq), _ptr(a_scale), _stream()),
+           "sbn_norm_quant_act")
 
 
 def _ws_args(ws):

@@ -557,6 +557,17 @@ sbn_status sbn_quant_act_expand68(const void* x_bf16, int T, int K, int8_t* xq, 
     return launch_quant_act<true>(x_bf16, T, K, xq, a_scale, static_cast<cudaStream_t>(stream));
 }
 
+sbn_status sbn_norm_quant_act_expand68(const void* x_bf16, int T, int K, const float* gain, float eps, int8_t* xq,
+                                       float* a_scale, void* stream) {
+    if (!x_bf16 || !xq || !a_scale) return SBN_ERR_NULL;
+    if (T <= 0 || K <= 0 || K % (2 * kBK) != 0) return SBN_ERR_SHAPE;
+    if (K > 16384) return SBN_ERR_UNSUPPORTED;
+    if (!(eps >= 0.0f)) return SBN_ERR_SHAPE;
+    if (misaligned(x_bf16, 16) || misaligned(xq, 16) || misaligned(a_scale, 4) || (gain && misaligned(gain, 16)))
+        return SBN_ERR_ALIGN;
+    return launch_norm_quant_act<true>(x_bf16, T, K, gain, eps, xq, a_scale, static_cast<cudaStream_t>(stream));
+}
+
 int sbn_expanded_k(int K, int n_keep, int m_group) {
     if (K <= 0) return 0;
     if (n_keep == 2 && m_group == 4) return K;

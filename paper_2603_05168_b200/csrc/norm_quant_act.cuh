@@ -40,7 +40,7 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
 
 // G threads per token row, VPT 16-byte vectors per thread (G * VPT >= K / 8).  The gains are copied
 // to shared memory once per CTA (rows differ, channels do not).
-template <int G, int VPT>
+template <int G, int VPT, bool EXPAND68 = false>
 __global__ void __launch_bounds__(kActThreads, (VPT <= 4) ? 3 : 2)
 norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4* __restrict__ gain, float eps,
                       uint2* __restrict__ xq, float* __restrict__ a_scale) {
@@ -176,7 +176,7 @@ norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4
                     uint2 ov;                                      // lowest column in the lowest byte
                     ov.x = pack_sat_s8x2(q[1], q[0], pack_sat_s8x2(q[3], q[2], 0u));
                     ov.y = pack_sat_s8x2(q[5], q[4], pack_sat_s8x2(q[7], q[6], 0u));
-                    xq[xq_tiled_u2_index(row, idx, tb8)] = ov;
+                    store_codes8<EXPAND68>(xq, row, idx, tb8, ov);     // plain, or expanded for the 6:8 pattern
                 }
             }
         }
@@ -185,7 +185,7 @@ norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4
     }
 }
 
-template <int G, int VPT>
+template <int G, int VPT, bool EXPAND68>
 static cudaError_t launch_norm_quant_act_cfg(const uint4* x, int T, int nvec, const float4* gain, float eps, uint2* q,
                                              float* a_scale, cudaStream_t stream) {
     constexpr int rows = kActThreads / G;
@@ -193,11 +193,12 @@ static cudaError_t launch_norm_quant_act_cfg(const uint4* x, int T, int nvec, co
     int grid = (T + rows - 1) / rows;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
     const size_t smem = gain ? static_cast<size_t>(nvec) * 32 : 0;          // K floats
-    if (!ensure_dynamic_smem<norm_quant_act_kernel<G, VPT>>(65536)) return cudaErrorUnknown;
-    return launch_kernel(norm_quant_act_kernel<G, VPT>, dim3(grid), dim3(kActThreads), smem, stream, x, T, nvec, gain, eps, q, a_scale);
+    if (!ensure_dynamic_smem<norm_quant_act_kernel<G, VPT, EXPAND68>>(65536)) return cudaErrorUnknown;
+    return launch_kernel(norm_quant_act_kernel<G, VPT, EXPAND68>, dim3(grid), dim3(kActThreads), smem, stream, x, T, nvec, gain, eps, q, a_scale);
 }
 
 // K up to 16384 (the register-resident row); longer rows are refused by the caller.
+template <bool EXPAND68 = false>
 inline sbn_status launch_norm_quant_act(const void* x_bf16, int T, int K, const float* gain, float eps, int8_t* xq,
                                         float* a_scale, cudaStream_t stream) {
     const int nvec = K / 8;
@@ -205,15 +206,15 @@ inline sbn_status launch_norm_quant_act(const void* x_bf16, int T, int K, const 
     const float4* g4 = reinterpret_cast<const float4*>(gain);
     uint2* q = reinterpret_cast<uint2*>(xq);
     cudaError_t err;
-    if (nvec <= 32 * 2) err = launch_norm_quant_act_cfg<32, 2>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 64 * 2) err = launch_norm_quant_act_cfg<64, 2>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 128 * 2) err = launch_norm_quant_act_cfg<128, 2>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 128 * 3) err = launch_norm_quant_act_cfg<128, 3>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 256 * 2) err = launch_norm_quant_act_cfg<256, 2>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 256 * 3) err = launch_norm_quant_act_cfg<256, 3>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 256 * 4) err = launch_norm_quant_act_cfg<256, 4>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 256 * 6) err = launch_norm_quant_act_cfg<256, 6>(x, T, nvec, g4, eps, q, a_scale, stream);
-    else if (nvec <= 256 * 8) err = launch_norm_quant_act_cfg<256, 8>(x, T, nvec, g4, eps, q, a_scale, stream);
+    if (nvec <= 32 * 2) err = launch_norm_quant_act_cfg<32, 2, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 64 * 2) err = launch_norm_quant_act_cfg<64, 2, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 128 * 2) err = launch_norm_quant_act_cfg<128, 2, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 128 * 3) err = launch_norm_quant_act_cfg<128, 3, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 256 * 2) err = launch_norm_quant_act_cfg<256, 2, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 256 * 3) err = launch_norm_quant_act_cfg<256, 3, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 256 * 4) err = launch_norm_quant_act_cfg<256, 4, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 256 * 6) err = launch_norm_quant_act_cfg<256, 6, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
+    else if (nvec <= 256 * 8) err = launch_norm_quant_act_cfg<256, 8, EXPAND68>(x, T, nvec, g4, eps, q, a_scale, stream);
     else return SBN_ERR_UNSUPPORTED;
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;

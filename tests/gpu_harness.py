@@ -168,13 +168,14 @@ def gpu_quant_act(x_bits: np.ndarray):
     return xq, a_scale
 
 
-def gpu_norm_quant_act(x_bits: np.ndarray, gain=None, eps=1e-6):
+def gpu_norm_quant_act(x_bits: np.ndarray, gain=None, eps=1e-6, expand68=False):
     T, K = x_bits.shape
     xd = bf16_dev(x_bits)
-    xq = b.alloc_xq(T, K)
+    xq = b.alloc_xq(T, 3 * K // 2 if expand68 else K)
+    xq.fill_(55)
     a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
     gd = None if gain is None else dev(np.asarray(gain, np.float32))
-    b.sbn_norm_quant_act(xd, xq, a_scale, gain=gd, eps=eps)
+    b.sbn_norm_quant_act(xd, xq, a_scale, gain=gd, eps=eps, expand68=expand68)
     b.sbn_check_status()
     return xq, a_scale
 

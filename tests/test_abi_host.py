@@ -88,6 +88,9 @@ def test_argument_validation_on_host(L):
     assert L.sbn_quant_act_expand68(None, 4, 256, p, p, None) == NULL
     assert L.sbn_quant_act_expand68(p, 4, 384, p, p, None) == SHAPE
     assert L.sbn_quant_act_expand68(p, 4, 256, odd, p, None) == ALIGN
+    assert L.sbn_norm_quant_act_expand68(p, 4, 384, p, ctypes.c_float(1e-6), p, p, None) == SHAPE
+    assert L.sbn_norm_quant_act_expand68(p, 4, 16384 + 256, p, ctypes.c_float(1e-6), p, p, None) == UNSUP
+    assert L.sbn_norm_quant_act_expand68(p, 4, 256, odd, ctypes.c_float(1e-6), p, p, None) == ALIGN
     assert L.sbn_expanded_k(2560, 6, 8) == 3840 and L.sbn_expanded_k(2560, 2, 4) == 2560
     assert L.sbn_expanded_k(2560 + 128, 6, 8) == 0 and L.sbn_expanded_k(2560, 3, 4) == 0
     assert qmp(N=100) == SHAPE

@@ -406,6 +406,19 @@ def test_quant_act_expand68_parity(T, K):
     assert np.array_equal(xq_to_numpy(xq, T, 3 * K // 2), xq_ref[:, expand68_columns(K)])
 
 
+@pytest.mark.parametrize("T,K", [(64, 256), (1, 2560), (67, 2560), (33, 6912), (19, 11008), (300, 4096), (3, 16384)])
+def test_norm_quant_act_expand68_parity(T, K):
+    bits = inputs.activations_bf16(T, K, seed=T + K + 5, token_lognormal_sigma=1.0)
+    gain = (1.0 + 0.1 * np.random.default_rng(K).standard_normal(K)).astype(np.float32)
+    r = oracle.norm_quant_act(bits, gain, 1e-6)
+    xq, s = gpu_norm_quant_act(bits, gain, 1e-6, expand68=True)
+    got = xq_to_numpy(xq, T, 3 * K // 2)
+    ref = r["xq"][:, expand68_columns(K)]
+    assert (~r["near_tie"]).all(), "a row's mean square sits on an fp32 rounding boundary for this seed"
+    assert np.array_equal(s.cpu().numpy(), r["a_scale"])
+    assert np.array_equal(got, ref)
+
+
 SPARSE68_SHAPES = [(64, 256, 256), (1, 128, 512), (5, 128, 256), (130, 384, 512), (300, 256, 2560), (64, 128, 6912),
                    (700, 512, 1280), (1100, 640, 2560)]
 
