@@ -610,6 +610,8 @@ def run_pattern68(args):
     flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     time_cold = _cold_timer(torch, stream, flush)
     cases = [(n, K, N, 4096) for n, K, N in inputs.SHAPES_2B] + [("down_7b", 11008, 4096, 8192)]
+    if args.only_step:                      # profiler runs: the one 7B-class layer only
+        cases = cases[-1:]
     rows, layers = [], []
     for i, (name, K, N, T) in enumerate(cases):
         W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i)).cuda()
@@ -647,6 +649,12 @@ def run_pattern68(args):
                      "act68_gbs": round((T * K * 3.5 + T * 4) / us["act68"] / 1e3, 1)})       # 2 B read + 1.5 B written
         if T == 4096:
             layers.append((f, ops))
+    if not layers:
+        b.sbn_check_status()
+        print(json.dumps({"metric": "6:8 sparse ternary BitLinear next to 2:4 and dense (dense-equivalent TOPS)", "unit": "TOPS",
+                          "workload": "p68", "rows": rows, "gpu_launches": b.sbn_launch_count()}))
+        return
+
     # whole steps over the four 2B-shaped layers, back to back
     def step(kind):
         for f, _ in layers:
