@@ -751,3 +751,29 @@ def test_full_size_sampled(name, T, K, N, sigma, outl, logn):
         bound = 127 * K // 2 if sparse else 127 * K
         assert accn.min() >= -bound and accn.max() <= bound
         assert not torch.isnan(y.float()).any()
+
+
+@pytest.mark.parametrize("name,T,K,N", [("down", 4096, 6912, 2560), ("down_7b", 8192, 11008, 4096)])
+def test_full_size_sampled_68(name, T, K, N):
+    # the 6:8 layer at full size, in the configuration bench.py --workload p68 times: pack parity
+    # on the whole matrix, activations on the whole batch, accumulators and outputs on samples
+    W = inputs.latent_weights(N, K, seed=24)
+    x = inputs.activations_bf16(T, K, seed=25, token_lognormal_sigma=0.5)
+    g = gpu_quantize_mask_pack68(W)
+    r = _assert_pack68(W, g)
+    xq_ref, s_ref = oracle.quant_act(x)
+    xq, a_scale = gpu_quant_act_expand68(x)
+    assert np.array_equal(a_scale.cpu().numpy(), s_ref)
+    assert np.array_equal(xq_to_numpy(xq, T, 3 * K // 2), xq_ref[:, expand68_columns(K)])
+    t_idx, n_idx = inputs.sample_positions(T, N, 4096, seed=26)
+    t_idx[:4] = [0, T - 1, 0, T - 1]
+    n_idx[:4] = [0, 0, N - 1, N - 1]
+    y, acc = gpu_gemm(True, xq, a_scale, g["dev"], out_dtype=torch.bfloat16)
+    acc_ref = oracle.acc_dense_sampled(xq_ref, r["w_eff"], t_idx, n_idx)
+    assert np.array_equal(acc.cpu().numpy()[t_idx, n_idx], acc_ref)
+    y_ref = oracle.dequant(acc_ref.reshape(-1, 1), r["scale"], s_ref[t_idx]).ravel()
+    got_bits = bf16_tensor_bits(y)[t_idx, n_idx].astype(np.int32)
+    assert np.abs(got_bits - oracle.f32_to_bf16_bits(y_ref).astype(np.int32)).max() <= 1
+    accn = acc.cpu().numpy()
+    assert accn.min() >= -127 * 3 * K // 4 and accn.max() <= 127 * 3 * K // 4
+    assert not torch.isnan(y.float()).any()
