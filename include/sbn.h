@@ -23,6 +23,13 @@
  *   - Errors are return codes.  Argument errors are detected on the host before anything is
  *     launched.  Device-side waits are bounded; a wait that runs out records SBN_ERR_TIMEOUT in a
  *     device status word that sbn_check_status reads back.
+ *   - The kernels are launched with programmatic stream serialisation: a kernel's set-up may
+ *     overlap the end of the kernel before it on the same stream, results are those of plain
+ *     stream order.  One rule follows for callers that write vals / meta / dense_q with a kernel
+ *     of their own: that kernel must not signal programmatic launch completion early
+ *     (cudaTriggerProgrammaticLaunchCompletion / griddepcontrol.launch_dependents), because the
+ *     few-token GEMM fetches weights before its dependency wait.  Copies and ordinary kernels are
+ *     fine.  SBN_DISABLE_PDL=1 in the environment turns the overlap off.
  *   - Inputs must be finite.  NaN/Inf give unspecified results.
  *   - Shape limits of the GPU path: N % 128 == 0, K % 128 == 0, T >= 1, K <= 2^20, pointers
  *     16-byte aligned (cudaMalloc alignment is always enough).
@@ -64,7 +71,7 @@ typedef enum {
     SBN_ERR_NULL = 1,        /* a required pointer is NULL */
     SBN_ERR_SHAPE = 2,       /* a dimension is <= 0 or breaks the divisibility rules above */
     SBN_ERR_ALIGN = 3,       /* a pointer is not 16-byte aligned */
-    SBN_ERR_UNSUPPORTED = 4, /* pattern other than 2:4, unknown dtype or op */
+    SBN_ERR_UNSUPPORTED = 4, /* pattern other than 2:4 / 6:8, unknown dtype or op */
     SBN_ERR_WORKSPACE = 5,   /* workspace missing or smaller than sbn_workspace_bytes() */
     SBN_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, tensor map, ...) */
     SBN_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (see sbn_check_status) */

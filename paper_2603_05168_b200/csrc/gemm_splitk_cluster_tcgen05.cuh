@@ -11,9 +11,11 @@
 //   CTA r of the cluster   k-blocks [r q, min((r+1) q, K/128)),  q = ceil(K/128 / S)
 //   mainloop               as in the single-CTA kernel (TMA producer warp, MMA issuer warp,
 //                          metadata through tcgen05.cp, one accumulator in TMEM)
-//   reduce-scatter         every CTA owns BN/S tokens of the tile; each epilogue thread (one output
-//                          feature = one TMEM lane) writes its partial sums of token j straight into
-//                          the shared memory of the CTA that owns j (st.shared::cluster), slot [r]
+//   reduce-scatter         CTA r owns the tokens j with j % S == r (interleaved, so that a tile with
+//                          few real tokens still spreads them over all CTAs); each epilogue thread
+//                          (one output feature = one TMEM lane) writes its partial sums of every
+//                          REAL token j straight into the shared memory of the CTA that owns j
+//                          (st.shared::cluster), slot [r]; padding tokens are skipped
 //   barrier.cluster        (hardware barrier: nothing spins)
 //   finish                 every CTA adds the S partials of its tokens, applies s = w_scale *
 //                          a_scale[t] (+ bias) and stores y (and the int32 dump when asked for)
@@ -21,6 +23,8 @@
 // No scratch in global memory, no atomics, nothing to keep zeroed; a CTA never touches a peer's
 // shared memory after the barrier, so CTAs leave independently.  All mbarrier waits are bounded.
 #pragma once
+
+#include <type_traits>
 
 #include "gemm_pair_tcgen05.cuh"
 
@@ -35,12 +39,16 @@ struct SplitConfig {
     static constexpr int B_BYTES = BN * kBK;
     static constexpr int E_BYTES = SPARSE ? kBM * (kBK / 8) : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-    static constexpr int STAGES = SPARSE ? 6 : 4;
+    // BN = 64: few enough stages that TWO CTAs fit on an SM (< 113 KB each), so the CTAs of the next
+    // launch of a decode loop are resident -- and already pulling their weights -- while this one
+    // reduces and finishes; the K slice of a CTA is short, and four 18 KB stages cover the L2 latency
+    static constexpr int STAGES = (BN == 64) ? (SPARSE ? 4 : 3) : (SPARSE ? 6 : 4);
+    static constexpr int CTAS_PER_SM = (BN == 64) ? 2 : 1;
     static constexpr int REDUCE_BYTES = BN * kBM * 4;          // [S][BN/S tokens][128 features] int32
     static constexpr int META_COL0 = BN;                        // metadata columns above the accumulator
     static constexpr uint32_t TMEM_COLS = (BN + 4 * STAGES <= 64) ? 64 : (BN + 4 * STAGES <= 128 ? 128 : 256);
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + REDUCE_BYTES + kBarrierBytes;
-    static_assert(SMEM_BYTES <= 232448, "shared memory overflow");
+    static_assert(SMEM_BYTES <= 232448 / CTAS_PER_SM - 1024 * (CTAS_PER_SM - 1), "shared memory overflow");
     static_assert(BN % 32 == 0 && BN <= 128, "token tile");
 };
 
@@ -56,7 +64,7 @@ __device__ __forceinline__ uint32_t cluster_nctarank() {
 }
 
 template <bool SPARSE, int BN>
-__global__ void __launch_bounds__(kSplitThreads, 1)
+__global__ void __launch_bounds__(kSplitThreads, SplitConfig<SPARSE, BN>::CTAS_PER_SM)
 bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                      const __grid_constant__ CUtensorMap tmap_b,
                                      const __grid_constant__ CUtensorMap tmap_e,
@@ -94,7 +102,8 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int kb0 = min(p.k_blocks_total, static_cast<int>(rank) * q);
     const int kb1 = min(p.k_blocks_total, kb0 + q);
     const int tok_per_cta = BN / static_cast<int>(S);           // S is 2, 4 or 8 (host's duty): a power of two
-    const int tok_shift = __ffs(tok_per_cta) - 1;
+    const int s_shift = __ffs(static_cast<int>(S)) - 1;
+    const int tile_tokens = min(BN, p.T - t0);                  // real tokens of this tile
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -115,14 +124,34 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     // a peer's shared memory may only be written once that CTA has started: every thread arrives
     // here and waits just before the scatter, so the barrier costs nothing on the way in
     cluster_arrive();
-    // this CTA's slice of the weights goes to L2 while the previous kernel is still finishing (a
-    // prefetch into L2, the point of coherence, cannot make anything stale)
-    if (threadIdx.x == 32 && kb1 > kb0) {
-        const size_t wt0 = static_cast<size_t>(mt) * p.k_blocks_total + kb0;
-        prefetch_l2_bulk(static_cast<const char*>(p.w_vals) + wt0 * p.w_tile_bytes, static_cast<uint32_t>((kb1 - kb0) * p.w_tile_bytes));
-        if (p.w_meta) prefetch_l2_bulk(static_cast<const char*>(p.w_meta) + wt0 * 2048, static_cast<uint32_t>((kb1 - kb0) * 2048));
+    // The weights of the first stages are fetched while the previous kernel of the stream is still
+    // finishing.  This is safe because no kernel that WRITES packed weights signals its dependents
+    // early (see sbn_common.cuh): a kernel that is running implies every earlier weight producer
+    // has completed.  The activations (written by the kernel right before this one) wait.
+    const int n_pre = min(STAGES, kb1 - kb0);
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+        if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);
+        for (int i = 0; i < n_pre; ++i) {
+            const uint32_t full = bar_full + 8 * i;
+            mbar_expect_tx(full, Cfg::STAGE_BYTES);
+            const int wt = mt * p.k_blocks_total + kb0 + i;
+            if constexpr (SPARSE) {
+                tma_load_2d(smem_a + i * Cfg::A_BYTES, &tmap_a, 0, wt * 8, full);
+                tma_load_2d(smem_e + i * Cfg::E_BYTES, &tmap_e, 0, wt * 2, full);
+            } else {
+                tma_load_2d(smem_a + i * Cfg::A_BYTES, &tmap_a, 0, wt * 16, full);
+            }
+        }
+        // the rest of this CTA's slice goes to L2 (the point of coherence: nothing can go stale there)
+        if (kb1 - kb0 > n_pre) {
+            const size_t wt0 = static_cast<size_t>(mt) * p.k_blocks_total + kb0 + n_pre;
+            prefetch_l2_bulk(static_cast<const char*>(p.w_vals) + wt0 * p.w_tile_bytes, static_cast<uint32_t>((kb1 - kb0 - n_pre) * p.w_tile_bytes));
+            if (p.w_meta) prefetch_l2_bulk(static_cast<const char*>(p.w_meta) + wt0 * 2048, static_cast<uint32_t>((kb1 - kb0 - n_pre) * 2048));
+        }
     }
-    pdl_wait();                          // nothing above reads or writes global memory
+    pdl_wait();
     pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
@@ -131,21 +160,20 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            tma_prefetch_desc(&tmap_a);
-            tma_prefetch_desc(&tmap_b);
-            if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);
             int stage = 0;
             uint32_t phase = 0;
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) break;
                 const uint32_t full = bar_full + 8 * stage;
-                mbar_expect_tx(full, Cfg::STAGE_BYTES);
-                const int wt = mt * p.k_blocks_total + kb;            // weight tile index
-                if constexpr (SPARSE) {
-                    tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 8, full);
-                    tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, 0, wt * 2, full);
-                } else {
-                    tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 16, full);
+                if (kb - kb0 >= n_pre) {                                 // the first n_pre stages got their weights above
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) break;
+                    mbar_expect_tx(full, Cfg::STAGE_BYTES);
+                    const int wt = mt * p.k_blocks_total + kb;            // weight tile index
+                    if constexpr (SPARSE) {
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 8, full);
+                        tma_load_2d(smem_e + stage * Cfg::E_BYTES, &tmap_e, 0, wt * 2, full);
+                    } else {
+                        tma_load_2d(smem_a + stage * Cfg::A_BYTES, &tmap_a, 0, wt * 16, full);
+                    }
                 }
                 tma_load_2d(smem_b + stage * Cfg::B_BYTES, &tmap_b, 0, kb * p.tb8 + (t0 >> 3), full);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -202,10 +230,10 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
             tcgen05_fence_after();
         }
         cluster_wait();                                   // all peers have started
-        // slot [rank][token % tok_per_cta][feature] in the owner's buffer
+        // slot [rank][token / S][feature] in the buffer of the owner, CTA token % S
         const uint32_t my_slot = smem_red + (rank * static_cast<uint32_t>(tok_per_cta)) * (kBM * 4) + static_cast<uint32_t>(f) * 4u;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = 0; c * 32 < tile_tokens; ++c) {
             uint32_t r[32];
             if (have && ok) {
                 tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(c * 32), r);
@@ -217,21 +245,24 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const int tok = c * 32 + j;
-                const uint32_t owner = static_cast<uint32_t>(tok >> tok_shift);
-                const uint32_t local = my_slot + static_cast<uint32_t>(tok & (tok_per_cta - 1)) * (kBM * 4);
-                st_shared_cluster_u32(map_to_cta(local, owner), r[j]);
+                if (tok < tile_tokens) {                                   // warp-uniform
+                    const uint32_t owner = static_cast<uint32_t>(tok) & (S - 1u);
+                    const uint32_t local = my_slot + static_cast<uint32_t>(tok >> s_shift) * (kBM * 4);
+                    st_shared_cluster_u32(map_to_cta(local, owner), r[j]);
+                }
             }
         }
         tcgen05_fence_before();
     }
-    // s of Eq. 4 for the tokens this CTA finishes, fetched before the barrier (lane l: tokens l and
-    // l + 32 of its share) so that the finishing loop has no global load to wait for
+    // s of Eq. 4 for the tokens this CTA finishes, fetched before the barrier (lane l: its l-th and
+    // (l + 32)-th token) so that the finishing loop has no global load to wait for
     float sc_a = 0.0f, sc_b = 0.0f;
     if (warp >= 2) {
         const float w_scale = __ldg(p.w_scale);
-        const int ta = t0 + static_cast<int>(rank) * tok_per_cta + lane;
-        if (lane < tok_per_cta && ta < p.T) sc_a = __fmul_rn(w_scale, __ldg(p.a_scale + ta));
-        if (lane + 32 < tok_per_cta && ta + 32 < p.T) sc_b = __fmul_rn(w_scale, __ldg(p.a_scale + ta + 32));
+        const int ja = lane * static_cast<int>(S) + static_cast<int>(rank);          // token inside the tile
+        const int jb = (lane + 32) * static_cast<int>(S) + static_cast<int>(rank);
+        if (lane < tok_per_cta && ja < tile_tokens) sc_a = __fmul_rn(w_scale, __ldg(p.a_scale + t0 + ja));
+        if (lane + 32 < tok_per_cta && jb < tile_tokens) sc_b = __fmul_rn(w_scale, __ldg(p.a_scale + t0 + jb));
     }
 
     // every CTA's partials are in place (release / acquire at cluster scope)
@@ -246,19 +277,39 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
         const int32_t* red = reinterpret_cast<const int32_t*>(smem_raw + (smem_red - smem_u32(smem_raw)));
         const bool fine = (*abort_flag == 0);
-        const int t_first = t0 + static_cast<int>(rank) * tok_per_cta;
-        const int n_tok = fine ? min(tok_per_cta, p.T - t_first) : 0;          // warp-uniform
-        for (int j = 0; j < n_tok; ++j) {
-            const int t = t_first + j;
-            const float sc = __shfl_sync(0xFFFFFFFFu, j < 32 ? sc_a : sc_b, j & 31);
-            int acc = 0;
-            for (uint32_t s = 0; s < S; ++s) acc += red[(s * tok_per_cta + j) * kBM + f];
-            if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
-            float v = __fmul_rn(static_cast<float>(acc), sc);
-            if (p.bias) v = __fadd_rn(v, bias);
-            if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-            else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
-        }
+        // my tokens: rank, rank + S, ... below tile_tokens
+        const int n_tok = fine ? max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift) : 0;   // warp-uniform
+        auto finish = [&](auto s_const) {
+            constexpr int SS = decltype(s_const)::value;
+            auto emit = [&](int j, int acc) {
+                const int t = t0 + j * SS + static_cast<int>(rank);
+                const float sc = __shfl_sync(0xFFFFFFFFu, j < 32 ? sc_a : sc_b, j & 31);
+                if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
+                float v = __fmul_rn(static_cast<float>(acc), sc);
+                if (p.bias) v = __fadd_rn(v, bias);
+                if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+                else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
+            };
+            int j = 0;
+            for (; j + 4 <= n_tok; j += 4) {              // four tokens at a time: 4 * S independent loads in flight
+                int acc[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int s2 = 0; s2 < SS; ++s2)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) acc[u] += red[(s2 * tok_per_cta + j + u) * kBM + f];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) emit(j + u, acc[u]);
+            }
+            for (; j < n_tok; ++j) {
+                int acc = 0;
+#pragma unroll
+                for (int s2 = 0; s2 < SS; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];
+                emit(j, acc);
+            }
+        };
+        if (S == 2u) finish(std::integral_constant<int, 2>{});
+        else if (S == 4u) finish(std::integral_constant<int, 4>{});
+        else finish(std::integral_constant<int, 8>{});
     }
 
     // teardown

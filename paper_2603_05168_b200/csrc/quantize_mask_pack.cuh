@@ -385,8 +385,9 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
     const int warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) s_ok = 1;
     __syncthreads();
+    // No early signal to the next kernel of the stream: this kernel writes packed weights, and the
+    // GEMM kernels fetch weights before their own dependency wait (see sbn_common.cuh).
     pdl_wait();
-    pdl_launch_dependents();
 
     QmpDesc d_prev = first;
     QmpRange rg_prev = {0u, 0u};

@@ -31,6 +31,14 @@ static std::atomic<unsigned long long> g_launch_count{0ull};
 // persistent with every CTA resident from the start, so an early dependent only ever takes
 // resources nobody else is waiting for.  SBN_DISABLE_PDL=1 in the environment turns the
 // attribute off (the two instructions are then no-ops).
+// One exception in each direction, which belong together: the few-token GEMM kernel fetches its
+// first stages of WEIGHTS before pdl_wait (they do not depend on the kernel right before it in a
+// decode loop, and their latency is most of that kernel's time), and in return the kernels that
+// WRITE packed weights (quantize_mask_pack) never call pdl_launch_dependents.  Without that signal
+// a successor starts only after the writer has completed and flushed, so any kernel that is
+// running -- and everything it may have launched early -- comes after every weight producer.
+// Weights written by copies or by kernels of other libraries are ordered the same way (they give no
+// early signal); a caller's own kernel that writes vals / meta must not give one either.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
