@@ -15,13 +15,16 @@
 //                          few real tokens still spreads them over all CTAs); each epilogue thread
 //                          (one output feature = one TMEM lane) writes its partial sums of every
 //                          REAL token j straight into the shared memory of the CTA that owns j
-//                          (st.shared::cluster), slot [r]; padding tokens are skipped
-//   barrier.cluster        (hardware barrier: nothing spins)
+//                          with st.async, slot [r]; padding tokens are skipped.  Every such store
+//                          counts its 4 bytes on an mbarrier of the OWNER, which expects exactly
+//                          (its tokens) x S x 128 x 4 bytes: no cluster-wide barrier after the
+//                          scatter, each CTA goes on as soon as ITS partials are complete
 //   finish                 every CTA adds the S partials of its tokens, applies s = w_scale *
 //                          a_scale[t] (+ bias) and stores y (and the int32 dump when asked for)
 //
-// No scratch in global memory, no atomics, nothing to keep zeroed; a CTA never touches a peer's
-// shared memory after the barrier, so CTAs leave independently.  All mbarrier waits are bounded.
+// No scratch in global memory, no atomics, nothing to keep zeroed.  A CTA leaves only after all
+// bytes addressed to it have arrived, and nothing is addressed to a CTA that owns no real token,
+// so no store ever targets shared memory of a CTA that has exited.  All mbarrier waits are bounded.
 #pragma once
 
 #include <type_traits>
@@ -52,8 +55,10 @@ struct SplitConfig {
     static_assert(BN % 32 == 0 && BN <= 128, "token tile");
 };
 
-__device__ __forceinline__ void st_shared_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+// 4-byte store into a peer's shared memory that counts its bytes on an mbarrier of that peer.
+__device__ __forceinline__ void st_async_cluster_u32(uint32_t cluster_addr, uint32_t v, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "r"(v), "r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -84,7 +89,8 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t bar_full = bar_base;
     const uint32_t bar_empty = bar_full + 8 * STAGES;
     const uint32_t bar_acc_full = bar_empty + 8 * STAGES;
-    const uint32_t tmem_slot = bar_acc_full + 8;
+    const uint32_t bar_red = bar_acc_full + 8;               // counts the bytes of partial sums sent to this CTA
+    const uint32_t tmem_slot = bar_red + 8;
 
     __shared__ int s_abort;
     volatile int* abort_flag = &s_abort;
@@ -104,6 +110,8 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int tok_per_cta = BN / static_cast<int>(S);           // S is 2, 4 or 8 (host's duty): a power of two
     const int s_shift = __ffs(static_cast<int>(S)) - 1;
     const int tile_tokens = min(BN, p.T - t0);                  // real tokens of this tile
+    // my tokens: rank, rank + S, ... below tile_tokens
+    const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift);
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -112,7 +120,10 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
             mbar_init(bar_empty + 8 * s, 1);
         }
         mbar_init(bar_acc_full, 1);
+        mbar_init(bar_red, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // armed before any peer can send: peers scatter only after this CTA's cluster_arrive below
+        mbar_expect_tx(bar_red, static_cast<uint32_t>(my_tokens) * S * (kBM * 4));
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
@@ -248,7 +259,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 if (tok < tile_tokens) {                                   // warp-uniform
                     const uint32_t owner = static_cast<uint32_t>(tok) & (S - 1u);
                     const uint32_t local = my_slot + static_cast<uint32_t>(tok >> s_shift) * (kBM * 4);
-                    st_shared_cluster_u32(map_to_cta(local, owner), r[j]);
+                    st_async_cluster_u32(map_to_cta(local, owner), r[j], map_to_cta(bar_red, owner));
                 }
             }
         }
@@ -265,11 +276,11 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         if (lane + 32 < tok_per_cta && jb < tile_tokens) sc_b = __fmul_rn(w_scale, __ldg(p.a_scale + t0 + jb));
     }
 
-    // every CTA's partials are in place (release / acquire at cluster scope)
-    __syncthreads();
-    cluster_sync_all();
-
     if (warp >= 2) {
+        // all partial sums addressed to this CTA have landed (the barrier's phase completes with the
+        // last byte; its completion makes the asynchronous stores visible to the waiting threads)
+        if (!mbar_wait(bar_red, 0u, abort_flag)) ok = false;
+        ok = __all_sync(0xFFFFFFFFu, ok);                 // the loop below shuffles: one verdict per warp
         // ------------------------------------------------------------------ epilogue, part 2: finish my tokens
         const int quarter = warp & 3;
         const int f = quarter * 32 + lane;
@@ -277,8 +288,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const float bias = p.bias ? __ldg(p.bias + n) : 0.0f;
         const int32_t* red = reinterpret_cast<const int32_t*>(smem_raw + (smem_red - smem_u32(smem_raw)));
         const bool fine = (*abort_flag == 0);
-        // my tokens: rank, rank + S, ... below tile_tokens
-        const int n_tok = fine ? max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift) : 0;   // warp-uniform
+        const int n_tok = (fine && ok) ? my_tokens : 0;
         auto finish = [&](auto s_const) {
             constexpr int SS = decltype(s_const)::value;
             auto emit = [&](int j, int acc) {
