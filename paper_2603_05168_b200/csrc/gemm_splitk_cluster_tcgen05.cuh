@@ -42,11 +42,13 @@ struct SplitConfig {
     static constexpr int B_BYTES = BN * kBK;
     static constexpr int E_BYTES = SPARSE ? kBM * (kBK / 8) : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
-    // BN = 64: few enough stages that TWO CTAs fit on an SM (< 113 KB each), so the CTAs of the next
+    // BN <= 64: few enough stages that TWO CTAs fit on an SM (< 113 KB each), so the CTAs of the next
     // launch of a decode loop are resident -- and already pulling their weights -- while this one
-    // reduces and finishes; the K slice of a CTA is short, and four 18 KB stages cover the L2 latency
-    static constexpr int STAGES = (BN == 64) ? (SPARSE ? 4 : 3) : (SPARSE ? 6 : 4);
-    static constexpr int CTAS_PER_SM = (BN == 64) ? 2 : 1;
+    // reduces and finishes.  A stage that is filled before the dependency wait costs nothing, one
+    // that has to be refilled costs an L2 round trip on the critical path: the 32-token tile keeps
+    // six (sparse) stages, enough for the whole K slice of a CTA at the usual sizes.
+    static constexpr int STAGES = (BN == 32) ? (SPARSE ? 6 : 4) : (BN == 64) ? (SPARSE ? 4 : 3) : (SPARSE ? 6 : 4);
+    static constexpr int CTAS_PER_SM = (BN <= 64) ? 2 : 1;
     static constexpr int REDUCE_BYTES = BN * kBM * 4;          // [S][BN/S tokens][128 features] int32
     static constexpr int META_COL0 = BN;                        // metadata columns above the accumulator
     static constexpr uint32_t TMEM_COLS = (BN + 4 * STAGES <= 64) ? 64 : (BN + 4 * STAGES <= 128 ? 128 : 256);

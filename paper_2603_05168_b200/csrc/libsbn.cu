@@ -221,7 +221,7 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
         int S = -g_force_split_k;
         S = S >= 8 ? 8 : (S >= 4 ? 4 : 2);
         while (S > 1 && S > K / kBK) S /= 2;
-        const int bn = g_force_token_tile == 128 ? 128 : 64;
+        const int bn = g_force_token_tile == 128 ? 128 : (g_force_token_tile == 32 ? 32 : 64);
         if (S > 1) return GemmPlan{false, bn, 1, S};
     }
     if (g_force_token_tile > 0 || g_force_split_k > 0) {        // diagnostics: single-CTA kernel as told
@@ -231,6 +231,27 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     const double mm = sparse ? 1.0 : 1.3;                       // dense K-loop relative to sparse
     double best_t = 1e300;
     auto consider = [&](const GemmPlan& g, double t) { if (t < best_t) { best_t = t; best = g; } };
+    // split-K inside clusters of 2 or 4 CTAs: the K-loop shrinks and the reduction stays on chip.
+    // Fitted to a sweep in a decode loop (weights from HBM, launches back to back), in us:
+    //   a(bn) + q * (0.22 sparse | 0.27 dense: one metadata copy + two MMAs resp. four MMAs per
+    //   128 columns at ~65 ns each whatever the tile width) + tokens of a tile * (scatter + finish / S)
+    //   + crowding once more CTAs than SMs are resident (tiles up to 64 tokens fit two per SM).
+    // All CTAs must be resident at once: a second wave costs a whole kernel lifetime.
+    auto consider_cluster = [&](int bn) {
+        const long tiles = static_cast<long>(rows) * ((T + bn - 1) / bn);
+        const long slots = bn <= 64 ? 2L * kNumSMs : kNumSMs;
+        const double a = bn == 32 ? 3.0 : (bn == 64 ? 3.3 : 3.7);
+        const int tt = std::min(bn, T);
+        for (int S = 2; S <= 4; S *= 2) {
+            if (S > kb || tiles * S > slots) break;
+            const int q = (kb + S - 1) / S;
+            const double per_tok = (bn == 128 ? 0.018 : 0.013) + 0.042 / S;
+            const long ctas = tiles * S;
+            const double crowd = ctas > kNumSMs ? 0.3 + 1.6 * static_cast<double>(ctas - kNumSMs) / kNumSMs : 0.0;
+            consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) + per_tok * tt + crowd);
+        }
+    };
+    if (g_allow_cluster) consider_cluster(32);
     const int bns[3] = {64, 128, 256};
     for (int bn : bns) {
         if (bn > 64 && T <= bn / 2) continue;                   // a tile mostly beyond T
@@ -239,17 +260,7 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
         const double F = 3.0 + 0.02 * bn;
         const long waves = (tiles + kNumSMs - 1) / kNumSMs;
         consider(GemmPlan{false, bn, 1, 0}, F + waves * kb * c);
-        if (bn <= 128 && g_allow_cluster) {
-            // split-K inside clusters of 2 or 4 CTAs: the K-loop shrinks and the reduction stays on
-            // chip.  Measured: ~4.7 us fixed (+2 for the 128-token tile), 0.065 us per token a CTA
-            // finishes; a second wave of clusters costs a whole kernel lifetime, so one wave only.
-            for (int S = 2; S <= 4; S *= 2) {
-                if (S > kb || tiles * S > kNumSMs) break;
-                const int q = (kb + S - 1) / S;
-                const int fin = std::min(bn / S, T);
-                consider(GemmPlan{false, bn, 1, S}, 5.2 + (bn == 128 ? 2.0 : 0.0) + q * c + 0.065 * fin);
-            }
-        }
+        if (bn <= 128 && g_allow_cluster) consider_cluster(bn);
         if (bn == 64 && tiles * 2 <= kNumSMs) {
             // smallest split that gives at least ~100 units of work
             int sp = static_cast<int>((100 + tiles - 1) / tiles);
@@ -366,9 +377,11 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
 
     if (plan.cluster > 1) {
         p.k_splits = 1;
-        if (sparse) return bn == 64 ? launch_splitk_cluster<true, 64>(ta, tb, te, p, plan.cluster, stream)
+        if (sparse) return bn == 32 ? launch_splitk_cluster<true, 32>(ta, tb, te, p, plan.cluster, stream)
+                         : bn == 64 ? launch_splitk_cluster<true, 64>(ta, tb, te, p, plan.cluster, stream)
                                     : launch_splitk_cluster<true, 128>(ta, tb, te, p, plan.cluster, stream);
-        return bn == 64 ? launch_splitk_cluster<false, 64>(ta, tb, te, p, plan.cluster, stream)
+        return bn == 32 ? launch_splitk_cluster<false, 32>(ta, tb, te, p, plan.cluster, stream)
+             : bn == 64 ? launch_splitk_cluster<false, 64>(ta, tb, te, p, plan.cluster, stream)
                         : launch_splitk_cluster<false, 128>(ta, tb, te, p, plan.cluster, stream);
     }
 

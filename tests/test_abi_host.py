@@ -44,9 +44,15 @@ def test_workspace_query(L):
     from paper_2603_05168_b200 import binding as b
     assert b.sbn_workspace_bytes(b.OP_QUANTIZE_MASK_PACK, 0, 256, 256) >= 8 * 148
     assert b.sbn_workspace_bytes(b.OP_QUANT_ACT, 64, 0, 256) == 0
-    # large T: no split-K scratch; decode-sized T: int32 [T][N] scratch
+    # large T: no split-K; few tokens: split-K inside clusters, reduced on chip -- no scratch either
     assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4096, 2560, 2560) == 0
-    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 4 * 2560 * 4 + 20 * 4   # sums + tile counters
+    assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 0
+    # split-K through global memory (here forced): int32 [T][N] sums + one counter per output tile
+    b.sbn_set_gemm_tuning(64, 5)
+    try:
+        assert b.sbn_workspace_bytes(b.OP_SPARSE_BITLINEAR, 4, 2560, 2560) == 4 * 2560 * 4 + 20 * 4
+    finally:
+        b.sbn_set_gemm_tuning(0, 0)
     assert b.sbn_workspace_bytes(b.OP_BITLINEAR, 4, 2560, 100) == 0      # illegal shape -> 0
     assert b.sbn_workspace_bytes(77, 4, 2560, 2560) == 0
 

@@ -636,6 +636,8 @@ CLUSTER_CASES = [  # (T, N, K, token tile, cluster size): split-K reduced in dis
     (64, 256, 2560, 64, 4), (1, 128, 256, 64, 2), (7, 256, 640, 64, 4),      # 5 k-blocks over 4 CTAs: one empty slice
     (100, 384, 6912, 64, 8), (130, 256, 1280, 128, 8), (200, 128, 384, 128, 2), (33, 512, 128, 64, 8),   # one k-block
     (257, 256, 2560, 128, 4),
+    (16, 256, 2560, 32, 4), (1, 128, 256, 32, 2), (31, 384, 6912, 32, 8), (32, 128, 1280, 32, 4), (45, 256, 640, 32, 4),
+    (70, 128, 2560, 32, 2),
 ]
 
 
