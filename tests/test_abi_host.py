@@ -115,7 +115,11 @@ def test_argument_validation_on_host(L):
     assert gemm(K=192) == SHAPE
     assert gemm(dt=5) == UNSUP
     assert gemm(xq=odd) == ALIGN
-    assert gemm(T=4, N=2560, K=2560) == WS          # decode shape needs split-K scratch
+    L.sbn_set_gemm_tuning(64, 5)                    # split-K through global memory needs its scratch
+    try:
+        assert gemm(T=4, N=2560, K=2560) == WS
+    finally:
+        L.sbn_set_gemm_tuning(0, 0)
     assert L.sbn_bitlinear(p, p, 64, None, p, 256, 256, None, p, 0, None, None, 0, None) == NULL
     from paper_2603_05168_b200 import binding as b
     assert L.sbn_quantize_mask_pack_batched(0, p, p, 1 << 20, None) == SHAPE
