@@ -296,6 +296,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int BN = pp.bn;
     const int half_bn = BN >> 1;
 
+    pdl_launch_dependents();             // lets the kernels after this one become resident as early as possible
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = smem_u32(smem_raw);
     if (smem_base & 1023u) {          // swizzled tiles need 1 KB alignment; identical in every CTA
@@ -345,7 +346,6 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     cluster_sync_all();                  // the peer's barriers exist before anything is signalled
     tcgen05_fence_after();
     pdl_wait();                          // nothing above touches global memory
-    pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 

@@ -115,6 +115,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     // my tokens: rank, rank + S, ... below tile_tokens
     const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift);
 
+    pdl_launch_dependents();             // lets the kernels after this one become resident as early as possible
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) {
@@ -165,7 +166,6 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
     }
     pdl_wait();
-    pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 

@@ -227,6 +227,7 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     constexpr int STAGES = Cfg::STAGES;
     constexpr int ACC_STAGES = Cfg::ACC_STAGES;
 
+    pdl_launch_dependents();             // lets the kernels after this one become resident as early as possible
     extern __shared__ uint8_t smem_raw[];
     // 1 KB alignment: required by the 128 B swizzle atoms (8 rows x 128 B)
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -283,7 +284,6 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         if (p.w_meta) prefetch_l2_bulk(static_cast<const char*>(p.w_meta) + wt0 * 2048, static_cast<uint32_t>(kb_per_split * 2048));
     }
     pdl_wait();                          // nothing above reads or writes global memory
-    pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 

@@ -58,8 +58,8 @@ norm_quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, const float4
     const int iters = (T + row_stride - 1) / row_stride;        // same for every thread of the CTA
     const bool has_gain = gain != nullptr;
 
+    pdl_launch_dependents();             // the next kernel may become resident (and fetch weights) right away
     pdl_wait();
-    pdl_launch_dependents();
 
     extern __shared__ float4 s_gain[];                           // [nvec * 2] when a gain is given
     if (has_gain) {

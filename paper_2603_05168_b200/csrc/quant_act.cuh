@@ -110,8 +110,8 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
     const size_t tb8 = xq_tb8(T);
     const int iters = (T + row_stride - 1) / row_stride;        // same for every thread of the CTA
 
+    pdl_launch_dependents();             // the next kernel may become resident (and fetch weights) right away
     pdl_wait();
-    pdl_launch_dependents();
 
     uint4 cur[VPT], nxt[VPT];
     int row = blockIdx.x * ROWS + r;
@@ -170,8 +170,8 @@ __global__ void __launch_bounds__(kActThreads)
 quant_act_long_row_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict__ xq,
                           float* __restrict__ a_scale) {
     __shared__ float s_max[kActThreads / 32];
+    pdl_launch_dependents();             // the next kernel may become resident (and fetch weights) right away
     pdl_wait();
-    pdl_launch_dependents();
     const int row = blockIdx.x;
     if (row >= T) return;
     const uint4* xr = x + static_cast<size_t>(row) * nvec;

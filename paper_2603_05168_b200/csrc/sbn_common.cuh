@@ -23,11 +23,14 @@ static std::atomic<unsigned long long> g_launch_count{0ull};
 
 // Programmatic dependent launch.  Every kernel of the library is launched with the
 // programmatic-stream-serialisation attribute and starts with
-//     <set-up that touches no global memory>;  pdl_wait();  pdl_launch_dependents();
+//     pdl_launch_dependents();  <set-up that touches no global memory>;  pdl_wait();
 // pdl_wait returns once the preceding kernel of the stream has completed and its writes are
 // visible, so everything after it is ordered exactly as in a plain stream; what is gained is
 // that the CTAs of the next kernel become resident (and do their set-up) on SMs the previous
-// kernel has already left, instead of after a full launch round trip.  All kernels here are
+// kernel has already left, instead of after a full launch round trip.  The signal comes first, so
+// in a chain of short kernels (quantiser, GEMM, quantiser, GEMM, ...) a kernel is resident while
+// the one TWO places ahead still runs: its own wait keeps it correct, and a GEMM uses the time to
+// fetch weights.  All kernels here are
 // persistent with every CTA resident from the start, so an early dependent only ever takes
 // resources nobody else is waiting for.  SBN_DISABLE_PDL=1 in the environment turns the
 // attribute off (the two instructions are then no-ops).
