@@ -779,3 +779,33 @@ def test_full_size_sampled_68(name, T, K, N):
     accn = acc.cpu().numpy()
     assert accn.min() >= -127 * 3 * K // 4 and accn.max() <= 127 * 3 * K // 4
     assert not torch.isnan(y.float()).any()
+
+
+@pytest.mark.parametrize("T,N,K", [(16, 256, 2560), (64, 384, 1280), (300, 256, 2560)])
+def test_gemm_after_repack_sees_the_new_weights(T, N, K):
+    # The few-token GEMM fetches weights before its dependency wait; that is only correct because
+    # the pack kernel gives its successors no early start.  Re-pack two different matrices into
+    # the SAME buffers and run the GEMM right behind each pack, with nothing in between and no
+    # synchronisation: every output must belong to the matrix packed just before it.
+    Wa = inputs.latent_weights(N, K, seed=81)
+    Wb = inputs.latent_weights(N, K, seed=82)
+    bits = inputs.activations_bf16(T, K, seed=83)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    refs = []
+    for W in (Wa, Wb):
+        r = _oracle_pack(W)
+        refs.append(oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])[1])
+    assert not np.array_equal(refs[0], refs[1])
+    xq, a_scale = gpu_quant_act(bits)
+    Wd = [dev(Wa), dev(Wb)]
+    p = b.alloc_packed(N, K)
+    ws = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, K)
+    reps = 12
+    accs = [torch.zeros((T, N), dtype=torch.int32, device="cuda") for _ in range(reps)]
+    y = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    for i in range(reps):
+        b.sbn_quantize_mask_pack(Wd[i % 2], p["vals"], p["meta"], p["w_scale"], p["ws"])
+        b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y, acc_out=accs[i], ws=ws)
+    b.sbn_check_status()
+    for i in range(reps):
+        assert np.array_equal(accs[i].cpu().numpy(), refs[i % 2]), f"launch {i} used stale weights"
