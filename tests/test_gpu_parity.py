@@ -781,12 +781,13 @@ def test_full_size_sampled_68(name, T, K, N):
     assert not torch.isnan(y.float()).any()
 
 
-@pytest.mark.parametrize("T,N,K", [(16, 256, 2560), (64, 384, 1280), (300, 256, 2560)])
+@pytest.mark.parametrize("T,N,K", [(16, 256, 2560), (64, 384, 1280), (300, 256, 2560), (16, 3840, 2560), (1, 2560, 6912)])
 def test_gemm_after_repack_sees_the_new_weights(T, N, K):
     # The few-token GEMM fetches weights before its dependency wait; that is only correct because
     # the pack kernel gives its successors no early start.  Re-pack two different matrices into
     # the SAME buffers and run the GEMM right behind each pack, with nothing in between and no
-    # synchronisation: every output must belong to the matrix packed just before it.
+    # synchronisation: every output must belong to the matrix packed just before it.  (A build whose
+    # pack kernel signalled early did return stale results on the 3840 x 2560 case.)
     Wa = inputs.latent_weights(N, K, seed=81)
     Wb = inputs.latent_weights(N, K, seed=82)
     bits = inputs.activations_bf16(T, K, seed=83)
@@ -800,7 +801,7 @@ def test_gemm_after_repack_sees_the_new_weights(T, N, K):
     Wd = [dev(Wa), dev(Wb)]
     p = b.alloc_packed(N, K)
     ws = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, K)
-    reps = 12
+    reps = 24
     accs = [torch.zeros((T, N), dtype=torch.int32, device="cuda") for _ in range(reps)]
     y = torch.empty((T, N), dtype=torch.float32, device="cuda")
     for i in range(reps):
