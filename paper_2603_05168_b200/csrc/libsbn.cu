@@ -266,7 +266,7 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
             int sp = static_cast<int>((100 + tiles - 1) / tiles);
             if (sp > kb) sp = kb;
             while (sp > 1 && kb % sp != 0) ++sp;                // next divisor upwards (kb divides itself)
-            if (sp > 1 && sp <= kb) {
+            if (sp > 1 && sp <= kb && sp <= 10) {               // many slices: the atomics dominate (33 us measured at 43)
                 const double atomics = 8e-6 * static_cast<double>(T) * N * sp;
                 consider(GemmPlan{false, bn, sp, 0}, F + (kb / sp) * c + 1.0 + atomics);
             }
