@@ -51,6 +51,8 @@ def _load():
             "sbn_oracle_apply_mask": (None, [vp, vp, i64, i64, vp]),
             "sbn_oracle_pack24": (i32, [vp, vp, i64, i64, vp, vp]),
             "sbn_oracle_unpack24": (None, [vp, vp, i64, i64, vp, vp]),
+            "sbn_oracle_bitpack24": (i32, [vp, vp, i64, i64, vp]),
+            "sbn_oracle_bitunpack24": (i32, [vp, i64, i64, vp, vp]),
             "sbn_oracle_quantize_mask_pack": (i32, [vp, i64, i64, vp, vp, vp, vp, vp, vp]),
             "sbn_oracle_quant_act": (None, [vp, i64, i64, vp, vp]),
             "sbn_oracle_norm_quant_act": (None, [vp, i64, i64, vp, f32, vp, vp, vp, vp]),
@@ -151,6 +153,31 @@ def unpack24(vals, meta):
     mask = np.zeros((N, K), np.uint8)
     _load().sbn_oracle_unpack24(_p(vals), _p(meta), N, K, _p(weff), _p(mask))
     return weff, mask
+
+
+def bitpack24(vals, meta):
+    """Compressed 2:4 form -> 6-bit group codes, 24 bytes per row and 128-column block
+    (uint8 [N][K/128][24]); see the C source for the code."""
+    vals = _c(vals, np.int8)
+    meta = _c(meta, np.uint8)
+    N, K2 = vals.shape
+    K = 2 * K2
+    bits = np.zeros((N, K // 128, 24), np.uint8)
+    if _load().sbn_oracle_bitpack24(_p(vals), _p(meta), N, K, _p(bits)) != 0:
+        raise ValueError("not a legal compressed 2:4 form of ternary values (or K % 128 != 0)")
+    return bits
+
+
+def bitunpack24(bits):
+    bits = _c(bits, np.uint8)
+    N, KB, w = bits.shape
+    assert w == 24
+    K = KB * 128
+    vals = np.zeros((N, K // 2), np.int8)
+    meta = np.zeros((N, K // 8), np.uint8)
+    if _load().sbn_oracle_bitunpack24(_p(bits), N, K, _p(vals), _p(meta)) != 0:
+        raise ValueError("illegal group code")
+    return vals, meta
 
 
 def quantize_mask_pack(W):

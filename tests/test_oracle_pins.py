@@ -514,3 +514,52 @@ def test_nm_bitlinear_is_the_integer_matmul():
     assert np.array_equal(acc, ref)
     s = np.float32(c["scale"]) * a_scale
     assert np.array_equal(y, (ref.astype(np.float32).T * s).T.astype(np.float32))
+
+
+# ---- bit-packed storage of the compressed 2:4 form (1.5 bits per weight) -------------------------
+def test_bitpack24_is_a_bijection_on_all_54_group_states():
+    # every (pair of kept columns, two ternary values) exactly once, in one row of 54 groups
+    # (padded to 64 groups = 256 columns with the state "columns 0,1, values 0,0")
+    pairs = [(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)]
+    states = [(p, v0, v1) for p in pairs for v0 in (-1, 0, 1) for v1 in (-1, 0, 1)]
+    assert len(states) == 54
+    G = 64
+    vals = np.zeros((1, 2 * G), np.int8)
+    nib = np.full(G, 0 | (1 << 2), np.uint8)
+    for g, ((i0, i1), v0, v1) in enumerate(states):
+        vals[0, 2 * g], vals[0, 2 * g + 1] = v0, v1
+        nib[g] = i0 | (i1 << 2)
+    meta = (nib[0::2] | (nib[1::2] << 4)).reshape(1, G // 2)
+    bits = oracle.bitpack24(vals, meta)
+    assert bits.shape == (1, 2, 24)                         # 24 bytes per 128 columns: 1.5 bits per weight
+    # decode the bit string by hand: code g at bits 6g .. 6g+5, little-endian
+    codes = []
+    for kb in range(2):
+        big = int.from_bytes(bits[0, kb].tobytes(), "little")
+        codes += [(big >> (6 * g)) & 63 for g in range(32)]
+    assert sorted(codes[:54]) == list(range(54))            # all 54 codes, each once
+    assert codes[0] == 0 and codes[53] == 53                # lexicographic: pair, v0, v1
+    assert codes[4] == 4 and codes[9] == 9                  # (0,1),0,0 -> 4 ; (0,2),-1,-1 -> 9
+    v2, m2 = oracle.bitunpack24(bits)
+    assert np.array_equal(v2, vals) and np.array_equal(m2, meta)
+
+
+def test_bitpack24_round_trip_and_rejections():
+    W = inputs.latent_weights(64, 512, seed=91)
+    r = oracle.quantize_mask_pack(W)
+    bits = oracle.bitpack24(r["vals"], r["meta"])
+    assert bits.size * 8 == 1.5 * W.size
+    v2, m2 = oracle.bitunpack24(bits)
+    assert np.array_equal(v2, r["vals"]) and np.array_equal(m2, r["meta"])
+    bad = r["meta"].copy()
+    bad[0, 0] = 0x11                                        # i0 == i1
+    with pytest.raises(ValueError):
+        oracle.bitpack24(r["vals"], bad)
+    badv = r["vals"].copy()
+    badv[0, 0] = 2
+    with pytest.raises(ValueError):
+        oracle.bitpack24(badv, r["meta"])
+    badb = bits.copy()
+    badb[0, 0, 0] |= 63                                     # code 63 does not exist
+    with pytest.raises(ValueError):
+        oracle.bitunpack24(badb)
