@@ -18,6 +18,7 @@
 #include "gemm_tcgen05.cuh"
 #include "gemm_pair_tcgen05.cuh"
 #include "gemm_splitk_cluster_tcgen05.cuh"
+#include "gemm_packed_cluster_tcgen05.cuh"
 
 namespace sbn {
 
@@ -636,6 +637,46 @@ sbn_status sbn_layer_forward_host(const void* x_bf16_host, int T, int K, void* x
     const size_t y_bytes = static_cast<size_t>(T) * N * (dt == SBN_OUT_BF16 ? 2 : 4);
     if (cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SBN_ERR_CUDA;
     return SBN_OK;
+}
+
+sbn_status sbn_bitpack24(const int8_t* vals, const uint8_t* meta, int N, int K, uint8_t* packed, void* stream) {
+    if (!vals || !meta || !packed) return SBN_ERR_NULL;
+    if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(vals, 16) || misaligned(meta, 16) || misaligned(packed, 16)) return SBN_ERR_ALIGN;
+    return launch_bitpack24(vals, meta, N, K, packed, static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, int T, const uint8_t* packed,
+                                       const float* w_scale, int N, int K, const float* bias, void* y,
+                                       sbn_out_dtype dt, int32_t* acc_out, void* stream) {
+    if (!xq || !a_scale || !packed || !w_scale || !y) return SBN_ERR_NULL;
+    if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (dt != SBN_OUT_F32 && dt != SBN_OUT_BF16) return SBN_ERR_UNSUPPORTED;
+    if (T > 1024 || K < 2 * kBK) return SBN_ERR_UNSUPPORTED;          // the few-token regime only
+    if (misaligned(xq, 16) || misaligned(packed, 16) || misaligned(y, 16) || misaligned(a_scale, 4) ||
+        misaligned(w_scale, 4) || (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)))
+        return SBN_ERR_ALIGN;
+    using Cfg = PackedSplitConfig;
+    CUtensorMap tb;
+    if (!encode_flat_1k(&tb, xq, xq_tiled_bytes(T, K), Cfg::BN / 8)) return SBN_ERR_CUDA;
+    GemmParams p;
+    p.T = T; p.N = N; p.K = K;
+    p.k_blocks_total = K / kBK;
+    p.k_splits = 1;
+    p.tb8 = static_cast<int>(xq_tb8(T));
+    p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias;
+    p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
+    p.acc_out = acc_out;
+    p.split_acc = nullptr; p.split_counters = nullptr;
+    p.w_vals = packed; p.w_meta = nullptr; p.w_tile_bytes = kPackedTileBytes;
+    const int tiles = (N / kBM) * ((T + Cfg::BN - 1) / Cfg::BN);
+    // clusters of 4 while every CTA can be resident at once (two per SM), else of 2
+    const int cluster = (p.k_blocks_total >= 4 && tiles * 4 <= 2 * device_sm_count()) ? 4 : 2;
+    if (!ensure_dynamic_smem<bitlinear_gemm_packed_cluster_kernel>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
+    const cudaError_t err = launch_kernel_cluster(bitlinear_gemm_packed_cluster_kernel, dim3(tiles * cluster), dim3(kSplitThreads),
+                                                  Cfg::SMEM_BYTES, static_cast<cudaStream_t>(stream), static_cast<unsigned>(cluster), tb, p);
+    ++g_launch_count;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
 sbn_status sbn_check_status(void* stream) {
