@@ -51,8 +51,8 @@ def _load():
             "sbn_oracle_apply_mask": (None, [vp, vp, i64, i64, vp]),
             "sbn_oracle_pack24": (i32, [vp, vp, i64, i64, vp, vp]),
             "sbn_oracle_unpack24": (None, [vp, vp, i64, i64, vp, vp]),
-            "sbn_oracle_bitpack24": (i32, [vp, vp, i64, i64, vp]),
-            "sbn_oracle_bitunpack24": (i32, [vp, i64, i64, vp, vp]),
+            "sbn_oracle_pack_vals2": (i32, [vp, i64, i64, vp]),
+            "sbn_oracle_unpack_vals2": (i32, [vp, i64, i64, vp]),
             "sbn_oracle_quantize_mask_pack": (i32, [vp, i64, i64, vp, vp, vp, vp, vp, vp]),
             "sbn_oracle_quant_act": (None, [vp, i64, i64, vp, vp]),
             "sbn_oracle_norm_quant_act": (None, [vp, i64, i64, vp, f32, vp, vp, vp, vp]),
@@ -155,29 +155,26 @@ def unpack24(vals, meta):
     return weff, mask
 
 
-def bitpack24(vals, meta):
-    """Compressed 2:4 form -> 6-bit group codes, 24 bytes per row and 128-column block
-    (uint8 [N][K/128][24]); see the C source for the code."""
+def pack_vals2(vals):
+    """Kept values int8 [N][K/2] -> two bits each (t = v + 1), uint8 [N][K/8]: the two values of a
+    group in one nibble (t0 | t1 << 2), even groups in the low nibble of their byte."""
     vals = _c(vals, np.int8)
-    meta = _c(meta, np.uint8)
     N, K2 = vals.shape
     K = 2 * K2
-    bits = np.zeros((N, K // 128, 24), np.uint8)
-    if _load().sbn_oracle_bitpack24(_p(vals), _p(meta), N, K, _p(bits)) != 0:
-        raise ValueError("not a legal compressed 2:4 form of ternary values (or K % 128 != 0)")
-    return bits
+    out = np.zeros((N, K // 8), np.uint8)
+    if _load().sbn_oracle_pack_vals2(_p(vals), N, K, _p(out)) != 0:
+        raise ValueError("values are not ternary (or K % 8 != 0)")
+    return out
 
 
-def bitunpack24(bits):
-    bits = _c(bits, np.uint8)
-    N, KB, w = bits.shape
-    assert w == 24
-    K = KB * 128
+def unpack_vals2(vals2):
+    vals2 = _c(vals2, np.uint8)
+    N, K8 = vals2.shape
+    K = 8 * K8
     vals = np.zeros((N, K // 2), np.int8)
-    meta = np.zeros((N, K // 8), np.uint8)
-    if _load().sbn_oracle_bitunpack24(_p(bits), N, K, _p(vals), _p(meta)) != 0:
-        raise ValueError("illegal group code")
-    return vals, meta
+    if _load().sbn_oracle_unpack_vals2(_p(vals2), N, K, _p(vals)) != 0:
+        raise ValueError("illegal field value 3")
+    return vals
 
 
 def quantize_mask_pack(W):

@@ -180,63 +180,39 @@ void sbn_oracle_unpack24(const int8_t *vals, const uint8_t *meta, int64_t N, int
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Bit-packed storage of the compressed 2:4 form (not in the paper: a storage format of this build
- * for the weight-bound few-token regime).  A group of four keeps two positions (6 choices) with a
- * ternary value each (9 choices): 54 states, one 6-bit code
- *     code = pair * 9 + (v0 + 1) * 3 + (v1 + 1),
- *     pair = index of (i0, i1) in (0,1) (0,2) (0,3) (1,2) (1,3) (2,3).
- * The 32 codes of a row's 128-column block fill 24 bytes, code g at bits 6g .. 6g+5 of the
- * little-endian bit string: 1.5 bits per weight.  bits: [N][K/128][24].
- * Returns 0, or -1 on an illegal nibble or a non-ternary value.
+ * Packed storage of the kept values (not in the paper: a storage format of this build for the
+ * weight-bound few-token regime).  A kept value is ternary: two bits hold t = v + 1 in {0, 1, 2}.
+ * The two values of a group share a nibble, t0 | t1 << 2; group 2b sits in the low nibble of byte b
+ * of its row, group 2b+1 in the high one.  vals2: [N][K/8] bytes -- with the metadata (unchanged,
+ * [N][K/8] bytes) that is 2 bits per weight instead of 5.
+ * Returns 0, or -1 on a non-ternary value (pack) / the unused field value 3 (unpack).
  * ------------------------------------------------------------------------------------------- */
-static int pair_index(int i0, int i1)
+int sbn_oracle_pack_vals2(const int8_t *vals, int64_t N, int64_t K, uint8_t *vals2)
 {
-    static const int first[4] = {0, 3, 5, 6};       /* pairs starting with i0 come after these many */
-    if (i0 < 0 || i1 > 3 || i0 >= i1) return -1;
-    return first[i0] + (i1 - i0 - 1);
-}
-
-int sbn_oracle_bitpack24(const int8_t *vals, const uint8_t *meta, int64_t N, int64_t K, uint8_t *bits)
-{
-    if (K % 128 != 0) return -1;
-    const int64_t KB = K / 128;
-    memset(bits, 0, (size_t)(N * KB * 24));
+    if (K % 8 != 0) return -1;
+    memset(vals2, 0, (size_t)(N * (K / 8)));
     for (int64_t n = 0; n < N; ++n) {
         for (int64_t g = 0; g < K / 4; ++g) {
-            uint8_t byte = meta[n * (K / 8) + g / 2];
-            int nib = (g & 1) ? (byte >> 4) : (byte & 15);
-            int p = pair_index(nib & 3, (nib >> 2) & 3);
             int v0 = vals[n * (K / 2) + 2 * g], v1 = vals[n * (K / 2) + 2 * g + 1];
-            if (p < 0 || v0 < -1 || v0 > 1 || v1 < -1 || v1 > 1) return -1;
-            unsigned code = (unsigned)(p * 9 + (v0 + 1) * 3 + (v1 + 1));
-            uint8_t *row = bits + (n * KB + g / 32) * 24;
-            int bit = 6 * (int)(g % 32);
-            for (int b = 0; b < 6; ++b)
-                if (code & (1u << b)) row[(bit + b) / 8] |= (uint8_t)(1u << ((bit + b) % 8));
+            if (v0 < -1 || v0 > 1 || v1 < -1 || v1 > 1) return -1;
+            uint8_t nib = (uint8_t)((v0 + 1) | ((v1 + 1) << 2));
+            vals2[n * (K / 8) + g / 2] |= (uint8_t)((g & 1) ? (nib << 4) : nib);
         }
     }
     return 0;
 }
 
-int sbn_oracle_bitunpack24(const uint8_t *bits, int64_t N, int64_t K, int8_t *vals, uint8_t *meta)
+int sbn_oracle_unpack_vals2(const uint8_t *vals2, int64_t N, int64_t K, int8_t *vals)
 {
-    static const int pi0[6] = {0, 0, 0, 1, 1, 2}, pi1[6] = {1, 2, 3, 2, 3, 3};
-    if (K % 128 != 0) return -1;
-    const int64_t KB = K / 128;
-    memset(meta, 0, (size_t)(N * (K / 8)));
+    if (K % 8 != 0) return -1;
     for (int64_t n = 0; n < N; ++n) {
         for (int64_t g = 0; g < K / 4; ++g) {
-            const uint8_t *row = bits + (n * KB + g / 32) * 24;
-            int bit = 6 * (int)(g % 32);
-            unsigned code = 0;
-            for (int b = 0; b < 6; ++b)
-                if (row[(bit + b) / 8] & (1u << ((bit + b) % 8))) code |= 1u << b;
-            if (code >= 54) return -1;
-            int p = (int)(code / 9), r = (int)(code % 9);
-            vals[n * (K / 2) + 2 * g] = (int8_t)(r / 3 - 1);
-            vals[n * (K / 2) + 2 * g + 1] = (int8_t)(r % 3 - 1);
-            uint8_t nib = (uint8_t)(pi0[p] | (pi1[p] << 2));
-            meta[n * (K / 8) + g / 2] |= (uint8_t)((g & 1) ? (nib << 4) : nib);
+            uint8_t byte = vals2[n * (K / 8) + g / 2];
+            int nib = (g & 1) ? (byte >> 4) : (byte & 15);
+            int t0 = nib & 3, t1 = (nib >> 2) & 3;
+            if (t0 == 3 || t1 == 3) return -1;
+            vals[n * (K / 2) + 2 * g] = (int8_t)(t0 - 1);
+            vals[n * (K / 2) + 2 * g + 1] = (int8_t)(t1 - 1);
         }
     }
     return 0;

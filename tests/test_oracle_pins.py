@@ -516,50 +516,34 @@ def test_nm_bitlinear_is_the_integer_matmul():
     assert np.array_equal(y, (ref.astype(np.float32).T * s).T.astype(np.float32))
 
 
-# ---- bit-packed storage of the compressed 2:4 form (1.5 bits per weight) -------------------------
-def test_bitpack24_is_a_bijection_on_all_54_group_states():
-    # every (pair of kept columns, two ternary values) exactly once, in one row of 54 groups
-    # (padded to 64 groups = 256 columns with the state "columns 0,1, values 0,0")
-    pairs = [(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)]
-    states = [(p, v0, v1) for p in pairs for v0 in (-1, 0, 1) for v1 in (-1, 0, 1)]
-    assert len(states) == 54
-    G = 64
+# ---- packed storage of the kept values (2 bits each) ------------------------------------------------
+def test_pack_vals2_hand_case_and_all_states():
+    # all nine (v0, v1) states in one row, padded to a legal width with (0, 0) groups
+    states = [(v0, v1) for v0 in (-1, 0, 1) for v1 in (-1, 0, 1)]
+    G = 16
     vals = np.zeros((1, 2 * G), np.int8)
-    nib = np.full(G, 0 | (1 << 2), np.uint8)
-    for g, ((i0, i1), v0, v1) in enumerate(states):
+    for g, (v0, v1) in enumerate(states):
         vals[0, 2 * g], vals[0, 2 * g + 1] = v0, v1
-        nib[g] = i0 | (i1 << 2)
-    meta = (nib[0::2] | (nib[1::2] << 4)).reshape(1, G // 2)
-    bits = oracle.bitpack24(vals, meta)
-    assert bits.shape == (1, 2, 24)                         # 24 bytes per 128 columns: 1.5 bits per weight
-    # decode the bit string by hand: code g at bits 6g .. 6g+5, little-endian
-    codes = []
-    for kb in range(2):
-        big = int.from_bytes(bits[0, kb].tobytes(), "little")
-        codes += [(big >> (6 * g)) & 63 for g in range(32)]
-    assert sorted(codes[:54]) == list(range(54))            # all 54 codes, each once
-    assert codes[0] == 0 and codes[53] == 53                # lexicographic: pair, v0, v1
-    assert codes[4] == 4 and codes[9] == 9                  # (0,1),0,0 -> 4 ; (0,2),-1,-1 -> 9
-    v2, m2 = oracle.bitunpack24(bits)
-    assert np.array_equal(v2, vals) and np.array_equal(m2, meta)
+    out = oracle.pack_vals2(vals)
+    assert out.shape == (1, G // 2)
+    nibs = [(v0 + 1) | ((v1 + 1) << 2) for v0, v1 in states] + [5] * (G - 9)     # (0,0) -> 1 | 1 << 2 = 5
+    expect = [nibs[2 * b] | (nibs[2 * b + 1] << 4) for b in range(G // 2)]
+    assert out[0].tolist() == expect
+    assert out[0, 0] == (0 | (0 << 2)) | ((0 | (1 << 2)) << 4)       # (-1,-1) then (-1,0): 0x40
+    assert np.array_equal(oracle.unpack_vals2(out), vals)
 
 
-def test_bitpack24_round_trip_and_rejections():
+def test_pack_vals2_round_trip_and_rejections():
     W = inputs.latent_weights(64, 512, seed=91)
     r = oracle.quantize_mask_pack(W)
-    bits = oracle.bitpack24(r["vals"], r["meta"])
-    assert bits.size * 8 == 1.5 * W.size
-    v2, m2 = oracle.bitunpack24(bits)
-    assert np.array_equal(v2, r["vals"]) and np.array_equal(m2, r["meta"])
-    bad = r["meta"].copy()
-    bad[0, 0] = 0x11                                        # i0 == i1
+    v2 = oracle.pack_vals2(r["vals"])
+    assert (v2.size + r["meta"].size) * 8 == 2 * W.size              # 2 bits per weight with the metadata
+    assert np.array_equal(oracle.unpack_vals2(v2), r["vals"])
+    bad = r["vals"].copy()
+    bad[0, 0] = 2
     with pytest.raises(ValueError):
-        oracle.bitpack24(r["vals"], bad)
-    badv = r["vals"].copy()
-    badv[0, 0] = 2
+        oracle.pack_vals2(bad)
+    badb = v2.copy()
+    badb[0, 0] |= 3
     with pytest.raises(ValueError):
-        oracle.bitpack24(badv, r["meta"])
-    badb = bits.copy()
-    badb[0, 0, 0] |= 63                                     # code 63 does not exist
-    with pytest.raises(ValueError):
-        oracle.bitunpack24(badb)
+        oracle.unpack_vals2(badb)
