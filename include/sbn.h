@@ -273,28 +273,26 @@ sbn_status sbn_sparse_bitlinear(const int8_t *xq, const float *a_scale, int T,
                                 int32_t *acc_out, void *ws, size_t ws_bytes, void *stream);
 
 /*
- * Bit-packed weights for the weight-bound few-token regime (not in the paper: a storage format of
- * this library).  A group of four has 6 x 9 = 54 states (which two columns are kept, a ternary
- * value each); sbn_bitpack24 turns the compressed form into one 6-bit code per group,
- *     code = pair * 9 + (v0 + 1) * 3 + (v1 + 1),  pair = index of (i0, i1) in
- *     (0,1) (0,2) (0,3) (1,2) (1,3) (2,3),
- * i.e. 1.5 bits per weight instead of the 5 bits of vals + meta.  Layout: one 3072-byte tile per
- * (128 rows, 128 columns) block, tiles in the order of the vals tiles ((n/128) * K/128 + k/128);
- * inside a tile row r owns bytes 24 r .. 24 r + 23, the code of its group g (0..31) at bits
- * 6 g .. 6 g + 5 of that little-endian 192-bit string.
- *   vals, meta   device, outputs of sbn_quantize_mask_pack (2:4), tiled order
- *   packed       device out, N*K*3/16 bytes, 16-byte aligned
- * sbn_sparse_bitlinear_packed is sbn_sparse_bitlinear on such weights (same results, bit for
- * bit): the kernel fetches the 3 KB tiles and expands them in shared memory next to the MMAs.
- * Few tokens only: T <= 1024 and K >= 256, else SBN_ERR_UNSUPPORTED (intended for T up to ~64,
- * where the weight stream is what a call costs); no workspace.
+ * Packed weights for the weight-bound few-token regime (not in the paper: a storage format of this
+ * library).  A kept value is ternary, so two bits hold it: t = v + 1 in {0, 1, 2}.  sbn_pack_vals2
+ * turns the value bytes of the compressed form into nibbles, t0 | t1 << 2 per group, group 2b in the
+ * low nibble of byte b of its row and group 2b+1 in the high one: vals2 is [N][K/8] bytes, stored
+ * tile by tile exactly like meta (same offsets).  With the metadata, which stays as it is, a
+ * weight costs 2 bits instead of 5.
+ *   vals    device, output of sbn_quantize_mask_pack (2:4), tiled order
+ *   vals2   device out, N*K/8 bytes, 16-byte aligned
+ * sbn_sparse_bitlinear_packed is sbn_sparse_bitlinear on (vals2, meta): same results, bit for bit.
+ * The kernel fetches 4 KB per 128 x 128 block instead of 10 KB and expands the values in shared
+ * memory next to the MMAs.  Few tokens only: T <= 1024 and K >= 256, else SBN_ERR_UNSUPPORTED
+ * (intended for T <= 32 on large matrices, where the weight stream is what a call costs); no
+ * workspace.  Like every producer of weights, a caller's kernel that writes vals2 must not signal
+ * programmatic launch completion early.
  */
-sbn_status sbn_bitpack24(const int8_t *vals, const uint8_t *meta, int N, int K, uint8_t *packed,
-                         void *stream);
+sbn_status sbn_pack_vals2(const int8_t *vals, int N, int K, uint8_t *vals2, void *stream);
 sbn_status sbn_sparse_bitlinear_packed(const int8_t *xq, const float *a_scale, int T,
-                                       const uint8_t *packed, const float *w_scale, int N, int K,
-                                       const float *bias, void *y, sbn_out_dtype dt,
-                                       int32_t *acc_out, void *stream);
+                                       const uint8_t *vals2, const uint8_t *meta,
+                                       const float *w_scale, int N, int K, const float *bias,
+                                       void *y, sbn_out_dtype dt, int32_t *acc_out, void *stream);
 
 /*
  * Baseline -- dense BitLinear (Sec. 2.1): same as above with the unmasked ternary

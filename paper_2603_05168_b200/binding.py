@@ -22,7 +22,7 @@ OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2
 
 EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
-    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_bitpack24", "sbn_sparse_bitlinear_packed",
+    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_launch_count",
 ]
@@ -72,10 +72,10 @@ def lib() -> ctypes.CDLL:
         L.sbn_norm_quant_act_expand68.argtypes = [vp, i32, i32, vp, ctypes.c_float, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
         L.sbn_sparse_bitlinear.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
-        L.sbn_bitpack24.restype = i32
-        L.sbn_bitpack24.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.sbn_pack_vals2.restype = i32
+        L.sbn_pack_vals2.argtypes = [vp, i32, i32, vp, vp]
         L.sbn_sparse_bitlinear_packed.restype = i32
-        L.sbn_sparse_bitlinear_packed.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp]
+        L.sbn_sparse_bitlinear_packed.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp]
         L.sbn_bitlinear.restype = i32
         L.sbn_bitlinear.argtypes = [vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
         L.sbn_layer_forward_host.restype = i32
@@ -209,23 +209,24 @@ def sbn_sparse_bitlinear(xq, a_scale, vals, meta, w_scale, y, bias=None, acc_out
            "sbn_sparse_bitlinear")
 
 
-def sbn_bitpack24(vals, meta, packed):
+def sbn_pack_vals2(vals, vals2):
     N = vals.shape[0]
     K = 2 * vals.numel() // N
-    _check(lib().sbn_bitpack24(_ptr(vals), _ptr(meta), N, K, _ptr(packed), _stream()), "sbn_bitpack24")
+    _check(lib().sbn_pack_vals2(_ptr(vals), N, K, _ptr(vals2), _stream()), "sbn_pack_vals2")
 
 
-def sbn_sparse_bitlinear_packed(xq, a_scale, packed, w_scale, y, K, bias=None, acc_out=None):
+def sbn_sparse_bitlinear_packed(xq, a_scale, vals2, meta, w_scale, y, bias=None, acc_out=None):
     T, N = y.shape
+    K = 8 * vals2.numel() // N
     dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
-    _check(lib().sbn_sparse_bitlinear_packed(_ptr(xq), _ptr(a_scale), T, _ptr(packed), _ptr(w_scale), N, K,
+    _check(lib().sbn_sparse_bitlinear_packed(_ptr(xq), _ptr(a_scale), T, _ptr(vals2), _ptr(meta), _ptr(w_scale), N, K,
                                              _ptr(bias), _ptr(y), dt, _ptr(acc_out), _stream()),
            "sbn_sparse_bitlinear_packed")
 
 
-def alloc_bitpacked(N: int, K: int, device="cuda"):
-    """Device buffer for the bit-packed form of one weight matrix (1.5 bits per weight)."""
-    return torch.empty(N * K * 3 // 16, dtype=torch.uint8, device=device)
+def alloc_vals2(N: int, K: int, device="cuda"):
+    """Device buffer for the kept values at two bits each ([N][K/8] bytes, tiled like meta)."""
+    return torch.empty((N, K // 8), dtype=torch.uint8, device=device)
 
 
 def sbn_bitlinear(xq, a_scale, dense_q, w_scale, y, bias=None, acc_out=None, ws=None):

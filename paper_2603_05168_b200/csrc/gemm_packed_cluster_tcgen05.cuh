@@ -1,13 +1,14 @@
-// Eq. 4 for few tokens from BIT-PACKED weights (bitpack24.cuh: 6 bits per group of four, 1.5 bits
-// per weight, 3 KB per 128 x 128 block instead of 10 KB).
+// Eq. 4 for few tokens from PACKED weights (bitpack24.cuh: kept values at two bits each next to
+// the unchanged metadata, 2 bits per weight, 4 KB per 128 x 128 block instead of 10 KB).
 //
 // On matrices of 7B-class size the few-token GEMM is bound by the weight stream (28 MB per call at
-// 5 bits per weight).  Here the CTA fetches the 3 KB tiles with bulk copies (no tensor map: a tile is
-// one contiguous block), and its four epilogue warps -- idle during the K-loop otherwise -- expand
-// every tile into the shared-memory images the sparse MMA reads (64 B-swizzled values, metadata
-// rows), one weight row per thread through a 54-entry table.  Everything else is the cluster
-// split-K kernel of gemm_splitk_cluster_tcgen05.cuh: K slices over the S CTAs of a cluster,
-// partial sums reduced through distributed shared memory with st.async, two CTAs per SM.
+// 5 bits per weight).  Here the CTA fetches the 2 KB value tiles and the 2 KB metadata tiles with
+// bulk copies (no tensor map: a tile is one contiguous block), and its four epilogue warps -- idle
+// during the K-loop otherwise -- expand every value tile into the 64 B-swizzled shared-memory image
+// the sparse MMA reads: a thread takes 8 groups (one word in, 16 bytes out) at three ALU
+// instructions per group, no table, every shared-memory access conflict-free.  Everything else is
+// the cluster split-K kernel of gemm_splitk_cluster_tcgen05.cuh: K slices over the S CTAs of a
+// cluster, partial sums reduced through distributed shared memory with st.async, two CTAs per SM.
 //
 //   warp 0, lane 0   bulk copies of packed tiles (8-deep ring; the first 8 before the dependency
 //                    wait, like the weights of the int8-held kernel), TMA loads of the activations
@@ -30,13 +31,13 @@ struct PackedSplitConfig {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + E_BYTES;
     static constexpr int STAGES = 4;
     static constexpr int RAW_STAGES = 8;
-    static constexpr int RAW_BYTES = RAW_STAGES * kPackedTileBytes;
+    static constexpr int RAW_SLOT_BYTES = kVals2TileBytes + 2048;          // value tile | metadata tile
+    static constexpr int RAW_BYTES = RAW_STAGES * RAW_SLOT_BYTES;
     static constexpr int REDUCE_BYTES = BN * kBM * 4;
-    static constexpr int LUT_BYTES = 64 * 4;
     static constexpr int BAR_BYTES = 512;
     static constexpr int META_COL0 = BN;
     static constexpr uint32_t TMEM_COLS = 64;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + REDUCE_BYTES + RAW_BYTES + LUT_BYTES + BAR_BYTES;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + REDUCE_BYTES + RAW_BYTES + BAR_BYTES;
     static_assert(BN + 4 * STAGES <= 64, "tensor memory columns");
     static_assert(SMEM_BYTES <= 232448 / 2 - 1024, "two CTAs per SM");
 };
@@ -69,8 +70,7 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const uint32_t smem_e = smem_b + STAGES * Cfg::B_BYTES;
     const uint32_t smem_red = smem_base + STAGES * Cfg::STAGE_BYTES;
     const uint32_t smem_pk = smem_red + Cfg::REDUCE_BYTES;                 // ring of packed tiles
-    const uint32_t smem_lut = smem_pk + Cfg::RAW_BYTES;
-    const uint32_t bar_base = smem_lut + Cfg::LUT_BYTES;
+    const uint32_t bar_base = smem_pk + Cfg::RAW_BYTES;
     const uint32_t bar_full = bar_base;                                    // activations of a stage have landed
     const uint32_t bar_empty = bar_full + 8 * STAGES;                      // the MMAs of a stage are done
     const uint32_t bar_exp = bar_empty + 8 * STAGES;                       // a stage's weights are expanded (128 arrivals)
@@ -100,7 +100,10 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int s_shift = __ffs(static_cast<int>(S)) - 1;
     const int tile_tokens = min(BN, p.T - t0);
     const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift);
-    const uint8_t* pk_tiles = static_cast<const uint8_t*>(p.w_vals) + (static_cast<size_t>(mt) * p.k_blocks_total + kb0) * kPackedTileBytes;
+    const size_t tile0 = static_cast<size_t>(mt) * p.k_blocks_total + kb0;
+    const uint8_t* v2_tiles = static_cast<const uint8_t*>(p.w_vals) + tile0 * kVals2TileBytes;
+    const uint8_t* me_tiles = static_cast<const uint8_t*>(p.w_meta) + tile0 * 2048;
+    constexpr uint32_t kSlot = Cfg::RAW_SLOT_BYTES;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -120,20 +123,6 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
         mbar_expect_tx(bar_red, static_cast<uint32_t>(my_tokens) * S * (kBM * 4));
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (threadIdx.x >= 64 && threadIdx.x < 128) {
-        // code -> value byte 0 | value byte 1 << 8 | nibble << 16 | nibble << 28
-        const uint32_t c = threadIdx.x - 64;
-        uint32_t e = 0u;
-        if (c < 54u) {
-            const uint32_t pr = c / 9u, r9 = c % 9u;
-            const uint32_t i0 = pr < 3u ? 0u : (pr < 5u ? 1u : 2u);
-            const uint32_t i1 = pr < 3u ? pr + 1u : (pr < 5u ? pr - 1u : 3u);
-            const uint32_t nib = i0 | (i1 << 2);
-            const uint32_t v0 = (r9 / 3u + 0xFFu) & 0xFFu, v1 = (r9 % 3u + 0xFFu) & 0xFFu;     // t - 1 as a byte
-            e = v0 | (v1 << 8) | (nib << 16) | (nib << 28);
-        }
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(smem_lut + 4u * c), "r"(e) : "memory");
-    }
     if (warp == 1) {
         tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
         tcgen05_fence_before();
@@ -148,44 +137,50 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
         tma_prefetch_desc(&tmap_b);
         const int n_pre = min(RAW, nblk);
         for (int i = 0; i < n_pre; ++i) {
-            mbar_expect_tx(bar_pk_full + 8 * i, kPackedTileBytes);
-            bulk_load(smem_pk + i * kPackedTileBytes, pk_tiles + static_cast<size_t>(i) * kPackedTileBytes, kPackedTileBytes, bar_pk_full + 8 * i);
+            mbar_expect_tx(bar_pk_full + 8 * i, kSlot);
+            bulk_load(smem_pk + i * kSlot, v2_tiles + static_cast<size_t>(i) * kVals2TileBytes, kVals2TileBytes, bar_pk_full + 8 * i);
+            bulk_load(smem_pk + i * kSlot + kVals2TileBytes, me_tiles + static_cast<size_t>(i) * 2048, 2048, bar_pk_full + 8 * i);
         }
-        if (nblk > n_pre) prefetch_l2_bulk(pk_tiles + static_cast<size_t>(n_pre) * kPackedTileBytes, static_cast<uint32_t>((nblk - n_pre) * kPackedTileBytes));
+        if (nblk > n_pre) {
+            prefetch_l2_bulk(v2_tiles + static_cast<size_t>(n_pre) * kVals2TileBytes, static_cast<uint32_t>((nblk - n_pre) * kVals2TileBytes));
+            prefetch_l2_bulk(me_tiles + static_cast<size_t>(n_pre) * 2048, static_cast<uint32_t>((nblk - n_pre) * 2048));
+        }
     }
 
     bool ok = true;
-    // Expands k-block `blk` of this CTA's slice into its stage (one weight row per thread).
+    const uint8_t* pk_generic = smem_raw + (smem_pk - smem_u32(smem_raw));
+    // Expands k-block `blk` of this CTA's slice into its stage.  Thread (row, 16 B chunk): one word of
+    // packed values in, one chunk of the swizzled value image out, four rows per thread; the metadata
+    // tile is copied as it is.  A warp reads 512 contiguous bytes and writes 8 whole 64 B rows.
     auto expand_block = [&](int blk) {
         const int stage = blk % STAGES, slot = blk % RAW;
-        const uint32_t r = threadIdx.x - 64;                              // weight row inside the tile
+        const uint32_t tix = threadIdx.x - 64;
+        const uint32_t c = tix & 3u;
         if (!mbar_wait(bar_pk_full + 8 * slot, static_cast<uint32_t>(blk / RAW) & 1u, abort_flag)) { ok = false; return; }
         if (blk >= STAGES && !mbar_wait(bar_empty + 8 * stage, static_cast<uint32_t>(blk / STAGES - 1) & 1u, abort_flag)) { ok = false; return; }
-        uint32_t w[7];
-        const uint32_t src = smem_pk + slot * kPackedTileBytes + r * 24u;
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(pk_generic + slot * kSlot);
+        uint32_t x[4], m[4];
 #pragma unroll
-        for (int i = 0; i < 3; ++i)
-            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(w[2 * i]), "=r"(w[2 * i + 1]) : "r"(src + 8u * i));
-        w[6] = 0u;
-        mbar_arrive(bar_pk_empty + 8 * slot);                             // the packed tile may be overwritten
-        uint32_t vw[16], mw[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int g = 0; g < 32; g += 2) {
-            const int b0 = 6 * g, b1 = 6 * g + 6;
-            const uint32_t c0 = __funnelshift_r(w[b0 >> 5], w[(b0 >> 5) + 1], b0 & 31) & 63u;
-            const uint32_t c1 = __funnelshift_r(w[b1 >> 5], w[(b1 >> 5) + 1], b1 & 31) & 63u;
-            const uint32_t e0 = ld_shared_u32(smem_lut + 4u * c0);
-            const uint32_t e1 = ld_shared_u32(smem_lut + 4u * c1);
-            vw[g >> 1] = __byte_perm(e0, e1, 0x5410);                     // v0 v1 | v0' v1'
-            const uint32_t mbyte = ((e0 >> 16) & 0x0Fu) | ((e1 >> 24) & 0xF0u);
-            mw[g >> 3] |= mbyte << (8 * ((g >> 1) & 3));
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t r = (tix >> 2) + 32u * i;
+            x[i] = src[r * 4 + c];
+            m[i] = src[kVals2TileBytes / 4 + r * 4 + c];
         }
-        const uint32_t a_row = smem_a + stage * Cfg::A_BYTES + r * 64u;
-        const uint32_t sw = (r >> 1) & 3u;
+        mbar_arrive(bar_pk_empty + 8 * slot);                             // the packed tiles may be overwritten
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            st_shared_v4(a_row + ((static_cast<uint32_t>(c) ^ sw) << 4), vw[4 * c], vw[4 * c + 1], vw[4 * c + 2], vw[4 * c + 3]);
-        st_shared_v4(smem_e + stage * Cfg::E_BYTES + r * 16u, mw[0], mw[1], mw[2], mw[3]);
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t r = (tix >> 2) + 32u * i;
+            uint32_t o[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                // one byte = t0 t1 t0' t1' at two bits each -> four bytes, then t - 1 per byte
+                const uint32_t b = (x[i] >> (8 * k)) & 0xFFu;
+                const uint32_t u = b | (b << 6);
+                o[k] = __vsub4((u | (u << 12)) & 0x03030303u, 0x01010101u);
+            }
+            st_shared_v4(smem_a + stage * Cfg::A_BYTES + r * 64u + ((c ^ ((r >> 1) & 3u)) << 4), o[0], o[1], o[2], o[3]);
+            asm volatile("st.shared.u32 [%0], %1;" ::"r"(smem_e + stage * Cfg::E_BYTES + r * 16u + 4u * c), "r"(m[i]) : "memory");
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy writes -> tensor core reads
         mbar_arrive(bar_exp + 8 * stage);
     };
@@ -212,8 +207,9 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
                 if (nb >= RAW && nb < nblk) {
                     const int slot = nb % RAW;
                     if (!mbar_wait(bar_pk_empty + 8 * slot, static_cast<uint32_t>(nb / RAW - 1) & 1u, abort_flag)) break;
-                    mbar_expect_tx(bar_pk_full + 8 * slot, kPackedTileBytes);
-                    bulk_load(smem_pk + slot * kPackedTileBytes, pk_tiles + static_cast<size_t>(nb) * kPackedTileBytes, kPackedTileBytes, bar_pk_full + 8 * slot);
+                    mbar_expect_tx(bar_pk_full + 8 * slot, kSlot);
+                    bulk_load(smem_pk + slot * kSlot, v2_tiles + static_cast<size_t>(nb) * kVals2TileBytes, kVals2TileBytes, bar_pk_full + 8 * slot);
+                    bulk_load(smem_pk + slot * kSlot + kVals2TileBytes, me_tiles + static_cast<size_t>(nb) * 2048, 2048, bar_pk_full + 8 * slot);
                 }
             }
         }

@@ -639,21 +639,21 @@ sbn_status sbn_layer_forward_host(const void* x_bf16_host, int T, int K, void* x
     return SBN_OK;
 }
 
-sbn_status sbn_bitpack24(const int8_t* vals, const uint8_t* meta, int N, int K, uint8_t* packed, void* stream) {
-    if (!vals || !meta || !packed) return SBN_ERR_NULL;
+sbn_status sbn_pack_vals2(const int8_t* vals, int N, int K, uint8_t* vals2, void* stream) {
+    if (!vals || !vals2) return SBN_ERR_NULL;
     if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
-    if (misaligned(vals, 16) || misaligned(meta, 16) || misaligned(packed, 16)) return SBN_ERR_ALIGN;
-    return launch_bitpack24(vals, meta, N, K, packed, static_cast<cudaStream_t>(stream));
+    if (misaligned(vals, 16) || misaligned(vals2, 16)) return SBN_ERR_ALIGN;
+    return launch_pack_vals2(vals, N, K, vals2, static_cast<cudaStream_t>(stream));
 }
 
-sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, int T, const uint8_t* packed,
-                                       const float* w_scale, int N, int K, const float* bias, void* y,
-                                       sbn_out_dtype dt, int32_t* acc_out, void* stream) {
-    if (!xq || !a_scale || !packed || !w_scale || !y) return SBN_ERR_NULL;
+sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, int T, const uint8_t* vals2,
+                                       const uint8_t* meta, const float* w_scale, int N, int K, const float* bias,
+                                       void* y, sbn_out_dtype dt, int32_t* acc_out, void* stream) {
+    if (!xq || !a_scale || !vals2 || !meta || !w_scale || !y) return SBN_ERR_NULL;
     if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
     if (dt != SBN_OUT_F32 && dt != SBN_OUT_BF16) return SBN_ERR_UNSUPPORTED;
     if (T > 1024 || K < 2 * kBK) return SBN_ERR_UNSUPPORTED;          // the few-token regime only
-    if (misaligned(xq, 16) || misaligned(packed, 16) || misaligned(y, 16) || misaligned(a_scale, 4) ||
+    if (misaligned(xq, 16) || misaligned(vals2, 16) || misaligned(meta, 16) || misaligned(y, 16) || misaligned(a_scale, 4) ||
         misaligned(w_scale, 4) || (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)))
         return SBN_ERR_ALIGN;
     using Cfg = PackedSplitConfig;
@@ -668,7 +668,7 @@ sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, i
     p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
     p.acc_out = acc_out;
     p.split_acc = nullptr; p.split_counters = nullptr;
-    p.w_vals = packed; p.w_meta = nullptr; p.w_tile_bytes = kPackedTileBytes;
+    p.w_vals = vals2; p.w_meta = meta; p.w_tile_bytes = kVals2TileBytes;
     const int tiles = (N / kBM) * ((T + Cfg::BN - 1) / Cfg::BN);
     // clusters of 4 while every CTA can be resident at once (two per SM), else of 2
     const int cluster = (p.k_blocks_total >= 4 && tiles * 4 <= 2 * device_sm_count()) ? 4 : 2;

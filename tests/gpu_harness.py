@@ -203,28 +203,22 @@ def gpu_gemm(sparse: bool, xq, a_scale, packed_dev, out_dtype=torch.float32, bia
     return y, acc
 
 
-def _bitpacked_offsets(N, K):
-    n = np.arange(N, dtype=np.int64)[:, None, None]
-    kb = np.arange(K // 128, dtype=np.int64)[None, :, None]
-    byte = np.arange(24, dtype=np.int64)[None, None, :]
-    return ((n >> 7) * (K // 128) + kb) * 3072 + (n & 127) * 24 + byte
-
-
-def gpu_bitpack24(packed_dev):
-    """Device buffers of alloc_packed -> (device bit-packed buffer, plain uint8 [N][K/128][24])."""
+def gpu_pack_vals2(packed_dev):
+    """Device buffers of alloc_packed -> (device vals2 buffer, plain uint8 [N][K/8])."""
     N, K = packed_dev["vals"].shape[0], 2 * packed_dev["vals"].shape[1]
-    out = b.alloc_bitpacked(N, K)
+    out = b.alloc_vals2(N, K)
     out.fill_(0xAA)
-    b.sbn_bitpack24(packed_dev["vals"], packed_dev["meta"], out)
+    b.sbn_pack_vals2(packed_dev["vals"], out)
     b.sbn_check_status()
-    return out, untile(out.cpu().numpy(), _bitpacked_offsets(N, K))
+    return out, untile(out.cpu().numpy(), _meta_offsets(N, K))
 
 
-def gpu_gemm_packed(xq, a_scale, bitpacked, w_scale, N, K, out_dtype=torch.float32, bias=None, want_acc=True):
+def gpu_gemm_packed(xq, a_scale, vals2, packed_dev, out_dtype=torch.float32, bias=None, want_acc=True):
     T = a_scale.numel()
+    N = packed_dev["vals"].shape[0]
     y = torch.full((T, N), float("nan"), dtype=out_dtype, device="cuda")
     acc = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device="cuda") if want_acc else None
-    b.sbn_sparse_bitlinear_packed(xq, a_scale, bitpacked, w_scale, y, K, bias=bias, acc_out=acc)
+    b.sbn_sparse_bitlinear_packed(xq, a_scale, vals2, packed_dev["meta"], packed_dev["w_scale"], y, bias=bias, acc_out=acc)
     b.sbn_check_status()
     return y, acc
 

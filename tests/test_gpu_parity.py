@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
     from gpu_harness import (gpu_norm_quant_act, bf16_dev, bf16_tensor_bits, dev, expand68_columns, fold68, gpu_gemm,
-                             gpu_bitpack24, gpu_gemm_packed, gpu_quant_act, gpu_quant_act_expand68, gpu_quantize_mask_pack,
+                             gpu_gemm_packed, gpu_pack_vals2, gpu_quant_act, gpu_quant_act_expand68, gpu_quantize_mask_pack,
                              gpu_quantize_mask_pack68,
                              xq_to_numpy, y_to_f32_numpy)
 
@@ -813,14 +813,14 @@ def test_gemm_after_repack_sees_the_new_weights(T, N, K):
         assert np.array_equal(accs[i].cpu().numpy(), refs[i % 2]), f"launch {i} used stale weights"
 
 
-# ---- bit-packed weights (1.5 bits per weight) for the few-token regime -------------------------------
+# ---- packed weights (2 bits per weight with the metadata) for the few-token regime --------------------
 @pytest.mark.parametrize("N,K,seed", [(128, 128, 100), (256, 512, 101), (384, 2560, 102), (128, 6912, 103)])
-def test_bitpack24_parity(N, K, seed):
+def test_pack_vals2_parity(N, K, seed):
     W = inputs.latent_weights(N, K, seed=seed)
     r = _oracle_pack(W)
     g = gpu_quantize_mask_pack(W, with_dense=False)
-    _, bits = gpu_bitpack24(g["dev"])
-    assert np.array_equal(bits, oracle.bitpack24(r["vals"], r["meta"]))
+    _, v2 = gpu_pack_vals2(g["dev"])
+    assert np.array_equal(v2, oracle.pack_vals2(r["vals"]))
 
 
 PACKED_GEMM_SHAPES = [(16, 256, 2560), (1, 128, 256), (5, 128, 384), (31, 384, 6912), (32, 128, 1280), (45, 256, 640),
@@ -828,15 +828,15 @@ PACKED_GEMM_SHAPES = [(16, 256, 2560), (1, 128, 256), (5, 128, 384), (31, 384, 6
 
 
 @pytest.mark.parametrize("T,N,K", PACKED_GEMM_SHAPES)
-def test_gemm_parity_bitpacked_weights(T, N, K):
+def test_gemm_parity_packed_weights(T, N, K):
     r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=T + N + K + 7)
     y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
-    packed, _ = gpu_bitpack24(g["dev"])
-    y, acc = gpu_gemm_packed(xq, a_scale, packed, g["dev"]["w_scale"], N, K)
+    vals2, _ = gpu_pack_vals2(g["dev"])
+    y, acc = gpu_gemm_packed(xq, a_scale, vals2, g["dev"])
     assert np.array_equal(acc.cpu().numpy(), acc_ref)
     _assert_y(y_to_f32_numpy(y), y_ref)
     bias = np.random.default_rng(T).standard_normal(N).astype(np.float32)
-    yb, _ = gpu_gemm_packed(xq, a_scale, packed, g["dev"]["w_scale"], N, K, out_dtype=torch.bfloat16, bias=dev(bias), want_acc=False)
+    yb, _ = gpu_gemm_packed(xq, a_scale, vals2, g["dev"], out_dtype=torch.bfloat16, bias=dev(bias), want_acc=False)
     y_ref_b = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"], bias=bias)[0]
     ref_bits = oracle.f32_to_bf16_bits(y_ref_b).astype(np.int32)
     assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
