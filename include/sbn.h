@@ -331,7 +331,7 @@ const char *sbn_status_string(sbn_status s);
  * 256 = force the single-CTA kernel with that token-tile width; a negative value -BN = force the
  * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
  * 256 dense).  split_k: 0 = automatic; k > 0 = split K k ways through int32 atomics in the
- * workspace (single-CTA kernel); -2, -4, -8 = split K inside thread-block clusters of that many
+ * workspace (single-CTA kernel); -2, -3, -4, -8 = split K inside thread-block clusters of that many
  * CTAs (token tile 64, or 32 / 128 if token_tile says so; no workspace).  Results do not depend on
  * it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);

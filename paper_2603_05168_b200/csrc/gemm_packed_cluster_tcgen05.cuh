@@ -33,7 +33,7 @@ struct PackedSplitConfig {
     static constexpr int RAW_STAGES = 8;
     static constexpr int RAW_SLOT_BYTES = kVals2TileBytes + 2048;          // value tile | metadata tile
     static constexpr int RAW_BYTES = RAW_STAGES * RAW_SLOT_BYTES;
-    static constexpr int REDUCE_BYTES = BN * kBM * 4;
+    static constexpr int REDUCE_BYTES = (BN + 4) * kBM * 4;               // S * ceil(BN / S) token slots, S in {2, 3, 4, 8}
     static constexpr int BAR_BYTES = 512;
     static constexpr int META_COL0 = BN;
     static constexpr uint32_t TMEM_COLS = 64;
@@ -96,10 +96,9 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
     const int kb0 = min(p.k_blocks_total, static_cast<int>(rank) * q);
     const int kb1 = min(p.k_blocks_total, kb0 + q);
     const int nblk = kb1 - kb0;
-    const int tok_per_cta = BN / static_cast<int>(S);
-    const int s_shift = __ffs(static_cast<int>(S)) - 1;
+    const int tok_per_cta = (BN + static_cast<int>(S) - 1) / static_cast<int>(S);
     const int tile_tokens = min(BN, p.T - t0);
-    const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift);
+    const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) / static_cast<int>(S));
     const size_t tile0 = static_cast<size_t>(mt) * p.k_blocks_total + kb0;
     const uint8_t* v2_tiles = static_cast<const uint8_t*>(p.w_vals) + tile0 * kVals2TileBytes;
     const uint8_t* me_tiles = static_cast<const uint8_t*>(p.w_meta) + tile0 * 2048;
@@ -260,14 +259,23 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
 #pragma unroll
             for (int j = 0; j < 32; ++j) rr[j] = 0u;
         }
+        auto scatter = [&](auto s_const) {
+            constexpr int SS = decltype(s_const)::value;
+            uint32_t row_of[SS], bar_of[SS];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            if (j < tile_tokens) {
-                const uint32_t owner = static_cast<uint32_t>(j) & (S - 1u);
-                const uint32_t local = my_slot + static_cast<uint32_t>(j >> s_shift) * (kBM * 4);
-                st_async_cluster_u32(map_to_cta(local, owner), rr[j], map_to_cta(bar_red, owner));
+            for (int o = 0; o < SS; ++o) {
+                row_of[o] = map_to_cta(my_slot, static_cast<uint32_t>(o));
+                bar_of[o] = map_to_cta(bar_red, static_cast<uint32_t>(o));
             }
-        }
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (j < tile_tokens)                                       // token j: entry j / S of owner j % S
+                    st_async_cluster_u32(row_of[j % SS] + static_cast<uint32_t>(j / SS) * (kBM * 4), rr[j], bar_of[j % SS]);
+        };
+        if (S == 2u) scatter(std::integral_constant<int, 2>{});
+        else if (S == 3u) scatter(std::integral_constant<int, 3>{});
+        else if (S == 4u) scatter(std::integral_constant<int, 4>{});
+        else scatter(std::integral_constant<int, 8>{});
         tcgen05_fence_before();
     }
     float sc_a = 0.0f;
@@ -287,7 +295,7 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
         const bool fine = (*abort_flag == 0);
         const int n_tok = (fine && ok) ? my_tokens : 0;
         for (int j = 0; j < n_tok; ++j) {
-            const int t = t0 + (j << s_shift) + static_cast<int>(rank);
+            const int t = t0 + j * static_cast<int>(S) + static_cast<int>(rank);
             const float sc = __shfl_sync(0xFFFFFFFFu, sc_a, j);
             int acc = 0;
             for (uint32_t s2 = 0; s2 < S; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];

@@ -49,7 +49,7 @@ struct SplitConfig {
     // six (sparse) stages, enough for the whole K slice of a CTA at the usual sizes.
     static constexpr int STAGES = (BN == 32) ? (SPARSE ? 6 : 4) : (BN == 64) ? (SPARSE ? 4 : 3) : (SPARSE ? 6 : 4);
     static constexpr int CTAS_PER_SM = (BN <= 64) ? 2 : 1;
-    static constexpr int REDUCE_BYTES = BN * kBM * 4;          // [S][BN/S tokens][128 features] int32
+    static constexpr int REDUCE_BYTES = (BN + 4) * kBM * 4;    // [S][ceil(BN/S) tokens][128 features] int32, S in {2, 3, 4, 8}
     static constexpr int META_COL0 = BN;                        // metadata columns above the accumulator
     static constexpr uint32_t TMEM_COLS = (BN + 4 * STAGES <= 64) ? 64 : (BN + 4 * STAGES <= 128 ? 128 : 256);
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + REDUCE_BYTES + kBarrierBytes;
@@ -109,11 +109,10 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int q = (p.k_blocks_total + static_cast<int>(S) - 1) / static_cast<int>(S);
     const int kb0 = min(p.k_blocks_total, static_cast<int>(rank) * q);
     const int kb1 = min(p.k_blocks_total, kb0 + q);
-    const int tok_per_cta = BN / static_cast<int>(S);           // S is 2, 4 or 8 (host's duty): a power of two
-    const int s_shift = __ffs(static_cast<int>(S)) - 1;
+    const int tok_per_cta = (BN + static_cast<int>(S) - 1) / static_cast<int>(S);   // S is 2, 3, 4 or 8 (host's duty)
     const int tile_tokens = min(BN, p.T - t0);                  // real tokens of this tile
     // my tokens: rank, rank + S, ... below tile_tokens
-    const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) >> s_shift);
+    const int my_tokens = max(0, (tile_tokens - static_cast<int>(rank) + static_cast<int>(S) - 1) / static_cast<int>(S));
 
     pdl_launch_dependents();             // lets the kernels after this one become resident as early as possible
     if (threadIdx.x == 0) {
@@ -245,26 +244,48 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         cluster_wait();                                   // all peers have started
         // slot [rank][token / S][feature] in the buffer of the owner, CTA token % S
         const uint32_t my_slot = smem_red + (rank * static_cast<uint32_t>(tok_per_cta)) * (kBM * 4) + static_cast<uint32_t>(f) * 4u;
+        auto scatter = [&](auto s_const) {
+            constexpr int SS = decltype(s_const)::value;                  // compile-time: token / S and token % S cost nothing
 #pragma unroll 1
-        for (int c = 0; c * 32 < tile_tokens; ++c) {
-            uint32_t r[32];
-            if (have && ok) {
-                tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(c * 32), r);
-                tmem_ld_wait();
-            } else {
+            for (int c = 0; c * 32 < tile_tokens; ++c) {
+                uint32_t r[32];
+                if (have && ok) {
+                    tmem_ld_32x32b_x32(tmem_base + lane_base + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;
-            }
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                uint32_t row_of[SS], bar_of[SS];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int tok = c * 32 + j;
-                if (tok < tile_tokens) {                                   // warp-uniform
-                    const uint32_t owner = static_cast<uint32_t>(tok) & (S - 1u);
-                    const uint32_t local = my_slot + static_cast<uint32_t>(tok >> s_shift) * (kBM * 4);
-                    st_async_cluster_u32(map_to_cta(local, owner), r[j], map_to_cta(bar_red, owner));
+                for (int o = 0; o < SS; ++o) {
+                    row_of[o] = map_to_cta(my_slot, static_cast<uint32_t>(o));
+                    bar_of[o] = map_to_cta(bar_red, static_cast<uint32_t>(o));
+                }
+                // BN is a multiple of 32, but 32 is not a multiple of 3: token = c * 32 + j
+                const int base_owner = (c * 32) % SS, base_local = (c * 32) / SS;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int tok = c * 32 + j;
+                    if (tok < tile_tokens) {                               // warp-uniform
+                        if constexpr ((32 % SS) == 0) {
+                            st_async_cluster_u32(row_of[j % SS] + static_cast<uint32_t>(base_local + j / SS) * (kBM * 4), r[j], bar_of[j % SS]);
+                        } else {
+                            const int o = (base_owner + j) % SS, l = (c * 32 + j) / SS;
+                            uint32_t ra = row_of[0], ba = bar_of[0];
+#pragma unroll
+                            for (int k = 1; k < SS; ++k)
+                                if (o == k) { ra = row_of[k]; ba = bar_of[k]; }
+                            st_async_cluster_u32(ra + static_cast<uint32_t>(l) * (kBM * 4), r[j], ba);
+                        }
+                    }
                 }
             }
-        }
+        };
+        if (S == 2u) scatter(std::integral_constant<int, 2>{});
+        else if (S == 3u) scatter(std::integral_constant<int, 3>{});
+        else if (S == 4u) scatter(std::integral_constant<int, 4>{});
+        else scatter(std::integral_constant<int, 8>{});
         tcgen05_fence_before();
     }
     // s of Eq. 4 for the tokens this CTA finishes, fetched before the barrier (lane l: its l-th and
@@ -320,6 +341,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
         };
         if (S == 2u) finish(std::integral_constant<int, 2>{});
+        else if (S == 3u) finish(std::integral_constant<int, 3>{});
         else if (S == 4u) finish(std::integral_constant<int, 4>{});
         else finish(std::integral_constant<int, 8>{});
     }

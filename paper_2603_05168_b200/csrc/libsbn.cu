@@ -220,8 +220,9 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     if (g_force_token_tile < 0) return GemmPlan{true, pick_pair_bn(sparse, T, N, K), 1, 0};
     if (g_force_split_k < 0) {                                  // diagnostics: cluster split-K as told
         int S = -g_force_split_k;
-        S = S >= 8 ? 8 : (S >= 4 ? 4 : 2);
-        while (S > 1 && S > K / kBK) S /= 2;
+        S = S >= 8 ? 8 : (S >= 4 ? 4 : (S == 3 ? 3 : 2));
+        while (S > 1 && S > K / kBK) --S;
+        if (S > 4 && S < 8) S = 4;
         const int bn = g_force_token_tile == 128 ? 128 : (g_force_token_tile == 32 ? 32 : 64);
         if (S > 1) return GemmPlan{false, bn, 1, S};
     }
@@ -232,24 +233,28 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     const double mm = sparse ? 1.0 : 1.3;                       // dense K-loop relative to sparse
     double best_t = 1e300;
     auto consider = [&](const GemmPlan& g, double t) { if (t < best_t) { best_t = t; best = g; } };
-    // split-K inside clusters of 2 or 4 CTAs: the K-loop shrinks and the reduction stays on chip.
+    // split-K inside clusters of 2, 3 or 4 CTAs: the K-loop shrinks and the reduction stays on chip.
     // Fitted to a sweep in a decode loop (weights from HBM, launches back to back), in us:
-    //   a(bn) + q * (0.22 sparse | 0.27 dense: one metadata copy + two MMAs resp. four MMAs per
-    //   128 columns at ~65 ns each whatever the tile width) + tokens of a tile * (scatter + finish / S)
-    //   + crowding once more CTAs than SMs are resident (tiles up to 64 tokens fit two per SM).
-    // All CTAs must be resident at once: a second wave costs a whole kernel lifetime.
+    //   a(bn) + q * (0.22 sparse | 0.27 dense per 128 columns) * (1 + 0.6 per further CTA on the busiest
+    //   SM: co-resident CTAs share the one tensor pipe) + tokens of a tile * (scatter + finish / S).
+    // All CTAs must be resident at once (tiles up to 64 tokens fit two per SM): a second wave costs
+    // a whole kernel lifetime.  Clusters of 3 matter for matrices with 75..90 row tiles, where 2
+    // leaves SMs with two CTAs' long K slices and 4 does not fit; they need some slack in the slot
+    // count (288 CTAs in clusters of 3 did not all become resident on 296 slots).
     auto consider_cluster = [&](int bn) {
         const long tiles = static_cast<long>(rows) * ((T + bn - 1) / bn);
         const long slots = bn <= 64 ? 2L * kNumSMs : kNumSMs;
         const double a = bn == 32 ? 3.0 : (bn == 64 ? 3.3 : 3.7);
         const int tt = std::min(bn, T);
-        for (int S = 2; S <= 4; S *= 2) {
+        for (int S = 2; S <= 4; ++S) {
             if (S > kb || tiles * S > slots) break;
+            if (S == 3 && tiles * S * 100 > slots * 93) continue;
             const int q = (kb + S - 1) / S;
             const double per_tok = (bn == 128 ? 0.018 : 0.013) + 0.042 / S;
             const long ctas = tiles * S;
-            const double crowd = ctas > kNumSMs ? 0.3 + 1.6 * static_cast<double>(ctas - kNumSMs) / kNumSMs : 0.0;
-            consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) + per_tok * tt + crowd);
+            const long per_sm = (ctas + kNumSMs - 1) / kNumSMs;
+            consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) * (1.0 + 0.6 * (per_sm - 1)) + per_tok * tt +
+                                                    (per_sm > 1 ? 0.3 : 0.0) + (S == 3 ? 0.4 : 0.0));
         }
     };
     if (g_allow_cluster) consider_cluster(32);
@@ -670,8 +675,20 @@ sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, i
     p.split_acc = nullptr; p.split_counters = nullptr;
     p.w_vals = vals2; p.w_meta = meta; p.w_tile_bytes = kVals2TileBytes;
     const int tiles = (N / kBM) * ((T + Cfg::BN - 1) / Cfg::BN);
-    // clusters of 4 while every CTA can be resident at once (two per SM), else of 2
-    const int cluster = (p.k_blocks_total >= 4 && tiles * 4 <= 2 * device_sm_count()) ? 4 : 2;
+    // cluster size: the one with the shortest K-loop on the busiest SM among those that keep every
+    // CTA resident at once (two per SM); 2 if none does
+    int cluster = 2;
+    {
+        const int sms = device_sm_count();
+        long best = -1;
+        for (int S = 2; S <= 4; ++S) {
+            if (S > p.k_blocks_total || static_cast<long>(tiles) * S > 2L * sms) break;
+            if (S == 3 && static_cast<long>(tiles) * S * 100 > 2L * sms * 93) continue;
+            const long per_sm = (static_cast<long>(tiles) * S + sms - 1) / sms;
+            const long load = (10 + 6 * (per_sm - 1)) * ((p.k_blocks_total + S - 1) / S) + (S == 3 ? 18 : 0);   // tenths of a block
+            if (best < 0 || load < best) { best = load; cluster = S; }
+        }
+    }
     if (!ensure_dynamic_smem<bitlinear_gemm_packed_cluster_kernel>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
     const cudaError_t err = launch_kernel_cluster(bitlinear_gemm_packed_cluster_kernel, dim3(tiles * cluster), dim3(kSplitThreads),
                                                   Cfg::SMEM_BYTES, static_cast<cudaStream_t>(stream), static_cast<unsigned>(cluster), tb, p);

@@ -121,6 +121,20 @@ def test_argument_validation_on_host(L):
     finally:
         L.sbn_set_gemm_tuning(0, 0)
     assert L.sbn_bitlinear(p, p, 64, None, p, 256, 256, None, p, 0, None, None, 0, None) == NULL
+    # packed weights: conversion and the few-token GEMM on them
+    assert L.sbn_pack_vals2(None, 256, 256, p, None) == NULL
+    assert L.sbn_pack_vals2(p, 100, 256, p, None) == SHAPE
+    assert L.sbn_pack_vals2(p, 256, 256, odd, None) == ALIGN
+    pk = lambda **k: L.sbn_sparse_bitlinear_packed(k.get("xq", p), p, k.get("T", 16), k.get("v2", p), k.get("meta", p), p,
+                                                   k.get("N", 256), k.get("K", 512), None, p, k.get("dt", 0), None, None)
+    assert pk(v2=None) == NULL
+    assert pk(meta=None) == NULL
+    assert pk(T=0) == SHAPE
+    assert pk(K=192) == SHAPE
+    assert pk(T=2000) == UNSUP              # few tokens only
+    assert pk(K=128) == UNSUP               # at least two k-blocks to split
+    assert pk(dt=7) == UNSUP
+    assert pk(xq=odd) == ALIGN
     from paper_2603_05168_b200 import binding as b
     assert L.sbn_quantize_mask_pack_batched(0, p, p, 1 << 20, None) == SHAPE
     assert L.sbn_quantize_mask_pack_batched(2, None, p, 1 << 20, None) == NULL

@@ -639,6 +639,8 @@ CLUSTER_CASES = [  # (T, N, K, token tile, cluster size): split-K reduced in dis
     (257, 256, 2560, 128, 4),
     (16, 256, 2560, 32, 4), (1, 128, 256, 32, 2), (31, 384, 6912, 32, 8), (32, 128, 1280, 32, 4), (45, 256, 640, 32, 4),
     (70, 128, 2560, 32, 2),
+    (16, 256, 2560, 32, 3), (31, 128, 896, 32, 3), (64, 384, 1280, 64, 3), (50, 128, 4096, 64, 3), (130, 256, 1280, 128, 3),
+    (1, 128, 384, 32, 3),
 ]
 
 
