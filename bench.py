@@ -548,18 +548,24 @@ def run_decode_sweep(args):
         torch.cuda.synchronize()
         return a.elapsed_time(c) * 1e3 / reps
 
+    big = args.workload == "decode7b"
+    shapes = [("gate_up_7b", 4096, 11008), ("down_7b", 11008, 4096), ("qkv_7b", 4096, 12288), ("o_7b", 4096, 4096)] if big else inputs.SHAPES_2B
+    token_counts = (1, 16, 32, 64) if big else (1, 16, 64, 128, 256, 512)
     rows = []
-    for i, (name, K, N) in enumerate(inputs.SHAPES_2B):
+    for i, (name, K, N) in enumerate(shapes):
         W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i)).cuda()
-        n_copies = int(200e6 // (N * K * 0.625)) + 1                 # > L2 worth of compressed weights
+        n_copies = min(24, int(200e6 // (N * K * 0.625)) + 1)        # > L2 worth of compressed weights
         packs = []
         for c in range(n_copies):
             p = b.alloc_packed(N, K, with_dense=True)
             b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"], dense_q=p["dense_q"])
+            if big:                                                 # values at two bits each next to the metadata
+                p["vals2"] = b.alloc_vals2(N, K)
+                b.sbn_pack_vals2(p["vals"], p["vals2"])
             packs.append(p)
             W.mul_(-1.0)                                            # another matrix, same statistics
         p = packs[0]
-        for T in (1, 16, 64, 128, 256, 512):
+        for T in token_counts:
             x = torch.from_numpy(inputs.activations_bf16(T, K, seed=50 + T).view(np.int16)).cuda().view(torch.bfloat16)
             xq = b.alloc_xq(T, K)
             a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
@@ -572,14 +578,20 @@ def run_decode_sweep(args):
                 b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y, ws=ws_d)
             sp = time_cold(lambda: b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=ws_s), 15)
             de = time_cold(lambda: b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y, ws=ws_d), 15)
+            io = T * K + T * N * 2 + T * 4
             sp_st = time_stream([(lambda q=q: b.sbn_sparse_bitlinear(xq, a_scale, q["vals"], q["meta"], q["w_scale"], y, ws=ws_s))
                                  for q in packs])
             de_st = time_stream([(lambda q=q: b.sbn_bitlinear(xq, a_scale, q["dense_q"], q["w_scale"], y, ws=ws_d))
                                  for q in packs])
-            io = T * K + T * N * 2 + T * 4
             sp_bytes = N * K * 0.625 + io
             de_bytes = N * K * 1.0 + io
-            rows.append({"layer": name, "T": T, "sparse_us": round(sp, 2), "dense_us": round(de, 2),
+            extra = {}
+            if big:
+                pk_st = time_stream([(lambda q=q: b.sbn_sparse_bitlinear_packed(xq, a_scale, q["vals2"], q["meta"], q["w_scale"], y))
+                                     for q in packs])
+                extra = {"packed_stream_us": round(pk_st, 2), "packed_stream_gbs": round((N * K * 0.25 + io) / pk_st / 1e3, 1),
+                         "packed_vs_int8_held": round(sp_st / pk_st, 3)}
+            rows.append({"layer": name, "T": T, **extra, "sparse_us": round(sp, 2), "dense_us": round(de, 2),
                          "sparse_stream_us": round(sp_st, 2), "dense_stream_us": round(de_st, 2),
                          "sparse_gbs": round(sp_bytes / sp / 1e3, 1), "dense_gbs": round(de_bytes / de / 1e3, 1),
                          "sparse_stream_gbs": round(sp_bytes / sp_st / 1e3, 1),
@@ -589,7 +601,7 @@ def run_decode_sweep(args):
         del packs
     b.sbn_check_status()
     print(json.dumps({"metric": "small-T sparse vs dense ternary BitLinear, HBM GB/s (cold L2)", "unit": "GB/s",
-                      "workload": "decode", "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "workload": args.workload, "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
                       "rows": rows, "gpu_launches": b.sbn_launch_count()}))
 
 
@@ -795,9 +807,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "dyn", "p68"],
+    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68"],
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1..512), sparse vs dense, cold L2 and streamed; "
+                         "decode7b = the same on 7B-class matrices at T <= 64, with the 2-bit packed weights as a third arm; "
                          "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048; "
                          "p68 = the 6:8 pattern next to 2:4 and dense on the same matrices")
     ap.add_argument("--masters", default="fp32", choices=["fp32", "bf16"],
@@ -806,7 +819,7 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.workload == "decode":
+    elif args.workload in ("decode", "decode7b"):
         run_decode_sweep(args)
     elif args.workload == "dyn":
         run_dynamic_step(args)
