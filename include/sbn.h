@@ -336,6 +336,12 @@ const char *sbn_status_string(sbn_status s);
  * it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);
 
+/* Diagnostic: what the dispatcher would run for this shape (host only, launches nothing).
+ * out4[0] = kernel (0 single-CTA tiles, 1 cluster split-K, 2 CTA pair), out4[1] = tokens per tile,
+ * out4[2] = split-K factor through global memory (1 = none), out4[3] = cluster size (0 = none).
+ * All zero for an illegal shape. */
+void sbn_plan_gemm(int sparse, int T, int N, int K, int *out4);
+
 /* Number of kernels the library has launched since it was loaded (all calls, all streams). */
 unsigned long long sbn_launch_count(void);
 

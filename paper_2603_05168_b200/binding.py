@@ -24,7 +24,7 @@ EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
     "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
-    "sbn_set_gemm_tuning", "sbn_launch_count",
+    "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count",
 ]
 
 _lib = None
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_status_string.argtypes = [i32]
         L.sbn_set_gemm_tuning.restype = None
         L.sbn_set_gemm_tuning.argtypes = [i32, i32]
+        L.sbn_plan_gemm.restype = None
+        L.sbn_plan_gemm.argtypes = [i32, i32, i32, i32, vp]
         L.sbn_launch_count.restype = ctypes.c_ulonglong
         L.sbn_launch_count.argtypes = []
         _lib = L
@@ -258,6 +260,13 @@ def sbn_check_status():
 
 def sbn_set_gemm_tuning(token_tile: int = 0, split_k: int = 0):
     lib().sbn_set_gemm_tuning(int(token_tile), int(split_k))
+
+
+def sbn_plan_gemm(sparse: bool, T: int, N: int, K: int):
+    """(kernel, tokens per tile, split-K factor, cluster size) the dispatcher picks; launches nothing."""
+    out = (ctypes.c_int * 4)()
+    lib().sbn_plan_gemm(1 if sparse else 0, T, N, K, out)
+    return tuple(out)
 
 
 def sbn_launch_count() -> int:

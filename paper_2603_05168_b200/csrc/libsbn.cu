@@ -254,7 +254,7 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
             const long ctas = tiles * S;
             const long per_sm = (ctas + kNumSMs - 1) / kNumSMs;
             consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) * (1.0 + 0.6 * (per_sm - 1)) + per_tok * tt +
-                                                    (per_sm > 1 ? 0.3 : 0.0) + (S == 3 ? 0.4 : 0.0));
+                                                    (per_sm > 1 ? 0.3 : 0.0) + (S == 3 ? 0.4 + 0.03 * tt : 0.0));   // 3: owner by select, not by mask
         }
     };
     if (g_allow_cluster) consider_cluster(32);
@@ -721,6 +721,17 @@ const char* sbn_status_string(sbn_status s) {
         case SBN_ERR_TOO_LARGE: return "problem larger than the library's built-in scratch can serve";
         default: return "unknown status";
     }
+}
+
+void sbn_plan_gemm(int sparse, int T, int N, int K, int* out4) {
+    if (!out4) return;
+    out4[0] = out4[1] = out4[2] = out4[3] = 0;
+    if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return;
+    const GemmPlan g = plan_gemm(sparse != 0, T, N, K);
+    out4[0] = g.pair ? 2 : (g.cluster > 1 ? 1 : 0);
+    out4[1] = g.bn;
+    out4[2] = g.splits;
+    out4[3] = g.cluster;
 }
 
 void sbn_set_gemm_tuning(int token_tile, int split_k) {

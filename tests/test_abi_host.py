@@ -153,3 +153,19 @@ def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError):
         binding.lib()
+
+
+def test_dispatch_plan_is_sane(L):
+    # host-only: the dispatcher's choices for the shapes the benchmarks use (kernel, tile, split, cluster)
+    from paper_2603_05168_b200 import binding as b
+    assert b.sbn_plan_gemm(True, 4096, 3840, 2560)[0] == 2            # large T: the CTA-pair kernel
+    assert b.sbn_plan_gemm(True, 8192, 4096, 11008)[0] == 2
+    k, bn, split, cluster = b.sbn_plan_gemm(True, 16, 3840, 2560)     # few tokens: cluster split-K, 32-token tile
+    assert (k, bn, split) == (1, 32, 1) and cluster in (2, 3, 4)
+    for T in (1, 16, 32):
+        for (N, K) in ((3840, 2560), (2560, 6912), (11008, 4096), (4096, 11008)):
+            k, bn, split, cluster = b.sbn_plan_gemm(True, T, N, K)
+            assert k == 1 and split == 1 and cluster in (2, 3, 4), (T, N, K)
+            tiles = (N // 128) * ((T + bn - 1) // bn)
+            assert tiles * cluster <= (296 if bn <= 64 else 148)       # every CTA resident at once
+    assert b.sbn_plan_gemm(True, 16, 100, 2560) == (0, 0, 0, 0)        # illegal shape
