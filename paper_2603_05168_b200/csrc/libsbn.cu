@@ -235,8 +235,8 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     auto consider = [&](const GemmPlan& g, double t) { if (t < best_t) { best_t = t; best = g; } };
     // split-K inside clusters of 2, 3 or 4 CTAs: the K-loop shrinks and the reduction stays on chip.
     // Fitted to a sweep in a decode loop (weights from HBM, launches back to back), in us:
-    //   a(bn) + q * (0.22 sparse | 0.27 dense per 128 columns) * (1 + 0.6 per further CTA on the busiest
-    //   SM: co-resident CTAs share the one tensor pipe) + tokens of a tile * (scatter + finish / S).
+    //   a(bn) + q * (0.22 sparse | 0.27 dense per 128 columns) * (1 .. 1.6: co-resident CTAs share the
+    //   one tensor pipe) + tokens of a tile * (scatter + finish / S).
     // All CTAs must be resident at once (tiles up to 64 tokens fit two per SM): a second wave costs
     // a whole kernel lifetime.  Clusters of 3 matter for matrices with 75..90 row tiles, where 2
     // leaves SMs with two CTAs' long K slices and 4 does not fit; they need some slack in the slot
@@ -253,7 +253,9 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
             const double per_tok = (bn == 128 ? 0.018 : 0.013) + 0.042 / S;
             const long ctas = tiles * S;
             const long per_sm = (ctas + kNumSMs - 1) / kNumSMs;
-            consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) * (1.0 + 0.6 * (per_sm - 1)) + per_tok * tt +
+            // share of the SMs that hold two CTAs; the slowdown saturates once ~40 % of them do
+            const double crowd = per_sm > 1 ? std::min(1.0, 2.5 * static_cast<double>(ctas - kNumSMs) / kNumSMs) : 0.0;
+            consider(GemmPlan{false, bn, 1, S}, a + q * (sparse ? 0.22 : 0.27) * (1.0 + 0.6 * crowd) + per_tok * tt +
                                                     (per_sm > 1 ? 0.3 : 0.0) + (S == 3 ? 0.4 + 0.03 * tt : 0.0));   // 3: owner by select, not by mask
         }
     };
