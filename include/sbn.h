@@ -273,6 +273,26 @@ sbn_status sbn_sparse_bitlinear(const int8_t *xq, const float *a_scale, int T,
                                 int32_t *acc_out, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Parts 2 and 3 in one kernel, for few tokens -- Algorithm 2's forward as it stands: the per-token
+ * absmax quantiser (Sec. 2.1) and Eq. 4.  Results are those of sbn_quant_act followed by
+ * sbn_sparse_bitlinear (resp. sbn_bitlinear), bit for bit; what is saved is a kernel launch, which in
+ * a decode loop is a quarter of a BitLinear's time.  The quantised activations never reach memory.
+ *   x_bf16        device, bf16 [T][K], 16-byte aligned, K % 128 == 0
+ *   a_scale_out   device out or NULL, fp32 [T]: the per-token scales d / 127
+ *   the other arguments as for sbn_sparse_bitlinear / sbn_bitlinear; no workspace
+ * Few tokens only: T <= 256 and K >= 256, else SBN_ERR_UNSUPPORTED (meant for T <= 32; beyond that
+ * every 32-token tile quantises its own tokens again for each of the N / 128 row tiles).
+ */
+sbn_status sbn_quant_act_sparse_bitlinear(const void *x_bf16, int T, const int8_t *vals,
+                                          const uint8_t *meta, const float *w_scale, int N, int K,
+                                          const float *bias, void *y, sbn_out_dtype dt,
+                                          int32_t *acc_out, float *a_scale_out, void *stream);
+sbn_status sbn_quant_act_bitlinear(const void *x_bf16, int T, const int8_t *dense_q,
+                                   const float *w_scale, int N, int K, const float *bias, void *y,
+                                   sbn_out_dtype dt, int32_t *acc_out, float *a_scale_out,
+                                   void *stream);
+
+/*
  * Packed weights for the weight-bound few-token regime (not in the paper: a storage format of this
  * library).  A kept value is ternary, so two bits hold it: t = v + 1 in {0, 1, 2}.  sbn_pack_vals2
  * turns the value bytes of the compressed form into nibbles, t0 | t1 << 2 per group, group 2b in the

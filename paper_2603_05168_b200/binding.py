@@ -22,7 +22,7 @@ OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2
 
 EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
-    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed",
+    "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed", "sbn_quant_act_sparse_bitlinear", "sbn_quant_act_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count",
 ]
@@ -72,6 +72,10 @@ def lib() -> ctypes.CDLL:
         L.sbn_norm_quant_act_expand68.argtypes = [vp, i32, i32, vp, ctypes.c_float, vp, vp, vp]
         L.sbn_sparse_bitlinear.restype = i32
         L.sbn_sparse_bitlinear.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+        L.sbn_quant_act_sparse_bitlinear.restype = i32
+        L.sbn_quant_act_sparse_bitlinear.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp]
+        L.sbn_quant_act_bitlinear.restype = i32
+        L.sbn_quant_act_bitlinear.argtypes = [vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp, vp]
         L.sbn_pack_vals2.restype = i32
         L.sbn_pack_vals2.argtypes = [vp, i32, i32, vp, vp]
         L.sbn_sparse_bitlinear_packed.restype = i32
@@ -209,6 +213,25 @@ def sbn_sparse_bitlinear(xq, a_scale, vals, meta, w_scale, y, bias=None, acc_out
     _check(lib().sbn_sparse_bitlinear(_ptr(xq), _ptr(a_scale), T, _ptr(vals), _ptr(meta), _ptr(w_scale),
                                       N, K, _ptr(bias), _ptr(y), dt, _ptr(acc_out), wp, wb, _stream()),
            "sbn_sparse_bitlinear")
+
+
+def sbn_quant_act_sparse_bitlinear(x_bf16, vals, meta, w_scale, y, bias=None, acc_out=None, a_scale_out=None):
+    """Activation quantiser + sparse GEMM in one kernel (few tokens)."""
+    T, K = x_bf16.shape
+    N = y.shape[1]
+    dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
+    _check(lib().sbn_quant_act_sparse_bitlinear(_ptr(x_bf16), T, _ptr(vals), _ptr(meta), _ptr(w_scale), N, K, _ptr(bias),
+                                                _ptr(y), dt, _ptr(acc_out), _ptr(a_scale_out), _stream()),
+           "sbn_quant_act_sparse_bitlinear")
+
+
+def sbn_quant_act_bitlinear(x_bf16, dense_q, w_scale, y, bias=None, acc_out=None, a_scale_out=None):
+    T, K = x_bf16.shape
+    N = y.shape[1]
+    dt = OUT_BF16 if y.dtype == torch.bfloat16 else OUT_F32
+    _check(lib().sbn_quant_act_bitlinear(_ptr(x_bf16), T, _ptr(dense_q), _ptr(w_scale), N, K, _ptr(bias), _ptr(y), dt,
+                                         _ptr(acc_out), _ptr(a_scale_out), _stream()),
+           "sbn_quant_act_bitlinear")
 
 
 def sbn_pack_vals2(vals, vals2):

@@ -19,6 +19,7 @@
 #include "gemm_pair_tcgen05.cuh"
 #include "gemm_splitk_cluster_tcgen05.cuh"
 #include "gemm_packed_cluster_tcgen05.cuh"
+#include "gemm_fused_act_cluster_tcgen05.cuh"
 
 namespace sbn {
 
@@ -644,6 +645,93 @@ sbn_status sbn_layer_forward_host(const void* x_bf16_host, int T, int K, void* x
     const size_t y_bytes = static_cast<size_t>(T) * N * (dt == SBN_OUT_BF16 ? 2 : 4);
     if (cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SBN_ERR_CUDA;
     return SBN_OK;
+}
+
+// Cluster size for the 32-token few-token kernels: the cost model of plan_gemm restricted to that tile.
+static int pick_cluster_32(bool sparse, int T, int N, int K) {
+    const int kb = K / kBK, rows = N / kBM;
+    const long tiles = static_cast<long>(rows) * ((T + 31) / 32);
+    const long slots = 2L * kNumSMs;
+    int best_s = 2;
+    double best_t = 1e300;
+    for (int S = 2; S <= 4; ++S) {
+        if (S > kb) break;
+        if (tiles * S > slots && S > 2) break;
+        if (S == 3 && tiles * S * 100 > slots * 93) continue;
+        const int q = (kb + S - 1) / S;
+        const long ctas = tiles * S;
+        const double crowd = ctas > kNumSMs ? std::min(1.0, 2.5 * static_cast<double>(ctas - kNumSMs) / kNumSMs) : 0.0;
+        const int tt = std::min(32, T);
+        const double t = q * (sparse ? 0.22 : 0.27) * (1.0 + 0.6 * crowd) + (0.013 + 0.042 / S) * tt + (S == 3 ? 0.4 + 0.03 * tt : 0.0);
+        if (t < best_t) { best_t = t; best_s = S; }
+    }
+    return best_s;
+}
+
+static sbn_status run_fused_act(bool sparse, const void* x_bf16, int T, const int8_t* wvals, const uint8_t* meta,
+                                const float* w_scale, int N, int K, const float* bias, void* y, sbn_out_dtype dt,
+                                int32_t* acc_out, float* a_scale_out, cudaStream_t stream) {
+    if (!x_bf16 || !wvals || !w_scale || !y || (sparse && !meta)) return SBN_ERR_NULL;
+    if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (dt != SBN_OUT_F32 && dt != SBN_OUT_BF16) return SBN_ERR_UNSUPPORTED;
+    if (T > 256 || K < 2 * kBK) return SBN_ERR_UNSUPPORTED;           // the few-token regime only
+    if (misaligned(x_bf16, 16) || misaligned(wvals, 16) || (sparse && misaligned(meta, 16)) || misaligned(y, 16) ||
+        misaligned(w_scale, 4) || (acc_out && misaligned(acc_out, 4)) || (bias && misaligned(bias, 4)) ||
+        (a_scale_out && misaligned(a_scale_out, 4)))
+        return SBN_ERR_ALIGN;
+    CUtensorMap ta, te;
+    bool ok;
+    const uint64_t NK = static_cast<uint64_t>(N) * K;
+    if (sparse) {
+        ok = encode_flat_1k(&ta, wvals, NK / 2, 8) && encode_flat_1k(&te, meta, NK / 8, 2);
+    } else {
+        ok = encode_flat_1k(&ta, wvals, NK, 16);
+        te = ta;
+    }
+    if (!ok) return SBN_ERR_CUDA;
+    FusedActParams fp;
+    GemmParams& p = fp.g;
+    p.T = T; p.N = N; p.K = K;
+    p.k_blocks_total = K / kBK;
+    p.k_splits = 1;
+    p.tb8 = 0;
+    p.a_scale = nullptr; p.w_scale = w_scale; p.bias = bias;
+    p.y = y; p.out_bf16 = (dt == SBN_OUT_BF16);
+    p.acc_out = acc_out;
+    p.split_acc = nullptr; p.split_counters = nullptr;
+    p.w_vals = wvals; p.w_meta = sparse ? meta : nullptr; p.w_tile_bytes = sparse ? 8192 : 16384;
+    fp.x_bf16 = x_bf16;
+    fp.a_scale_out = a_scale_out;
+    const int tiles = (N / kBM) * ((T + 31) / 32);
+    const int cluster = pick_cluster_32(sparse, T, N, K);
+    cudaError_t err;
+    if (sparse) {
+        using Cfg = FusedActConfig<true>;
+        if (!ensure_dynamic_smem<bitlinear_gemm_fused_act_cluster_kernel<true>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
+        err = launch_kernel_cluster(bitlinear_gemm_fused_act_cluster_kernel<true>, dim3(tiles * cluster), dim3(kSplitThreads),
+                                    Cfg::SMEM_BYTES, stream, static_cast<unsigned>(cluster), ta, te, fp);
+    } else {
+        using Cfg = FusedActConfig<false>;
+        if (!ensure_dynamic_smem<bitlinear_gemm_fused_act_cluster_kernel<false>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
+        err = launch_kernel_cluster(bitlinear_gemm_fused_act_cluster_kernel<false>, dim3(tiles * cluster), dim3(kSplitThreads),
+                                    Cfg::SMEM_BYTES, stream, static_cast<unsigned>(cluster), ta, te, fp);
+    }
+    ++g_launch_count;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
+sbn_status sbn_quant_act_sparse_bitlinear(const void* x_bf16, int T, const int8_t* vals, const uint8_t* meta,
+                                          const float* w_scale, int N, int K, const float* bias, void* y,
+                                          sbn_out_dtype dt, int32_t* acc_out, float* a_scale_out, void* stream) {
+    return run_fused_act(true, x_bf16, T, vals, meta, w_scale, N, K, bias, y, dt, acc_out, a_scale_out,
+                         static_cast<cudaStream_t>(stream));
+}
+
+sbn_status sbn_quant_act_bitlinear(const void* x_bf16, int T, const int8_t* dense_q, const float* w_scale, int N, int K,
+                                   const float* bias, void* y, sbn_out_dtype dt, int32_t* acc_out, float* a_scale_out,
+                                   void* stream) {
+    return run_fused_act(false, x_bf16, T, dense_q, nullptr, w_scale, N, K, bias, y, dt, acc_out, a_scale_out,
+                         static_cast<cudaStream_t>(stream));
 }
 
 sbn_status sbn_pack_vals2(const int8_t* vals, int N, int K, uint8_t* vals2, void* stream) {

@@ -842,3 +842,40 @@ def test_gemm_parity_packed_weights(T, N, K):
     y_ref_b = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"], bias=bias)[0]
     ref_bits = oracle.f32_to_bf16_bits(y_ref_b).astype(np.int32)
     assert np.abs(bf16_tensor_bits(yb).astype(np.int32) - ref_bits).max() <= 1
+
+
+# ---- activation quantiser + GEMM in one kernel (few tokens) ---------------------------------------------
+FUSED_ACT_SHAPES = [(16, 256, 2560), (1, 128, 256), (5, 128, 384), (31, 384, 6912), (32, 128, 1280), (45, 256, 640),
+                    (64, 512, 2560), (100, 256, 4096), (7, 128, 11008), (3, 11008 // 128 * 128, 512)]
+
+
+@pytest.mark.parametrize("sparse", [True, False])
+@pytest.mark.parametrize("T,N,K", FUSED_ACT_SHAPES)
+def test_fused_quant_act_gemm_parity(sparse, T, N, K):
+    W = inputs.latent_weights(N, K, seed=T + N + K + 11)
+    bits = inputs.activations_bf16(T, K, seed=T + N + K + 12, token_lognormal_sigma=1.0)
+    bits[0, :] = 0                                            # an all-zero token: the 1e-5 clamp
+    r = _oracle_pack(W)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    if sparse:
+        y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    else:
+        y_ref, acc_ref = oracle.bitlinear(xq_ref, s_ref, r["dense_q"], r["scale"])
+    g = gpu_quantize_mask_pack(W)
+    p = g["dev"]
+    x = bf16_dev(bits)
+    y = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    acc = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device="cuda")
+    a_sc = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    if sparse:
+        b.sbn_quant_act_sparse_bitlinear(x, p["vals"], p["meta"], p["w_scale"], y, acc_out=acc, a_scale_out=a_sc)
+    else:
+        b.sbn_quant_act_bitlinear(x, p["dense_q"], p["w_scale"], y, acc_out=acc, a_scale_out=a_sc)
+    b.sbn_check_status()
+    assert np.array_equal(a_sc.cpu().numpy(), s_ref)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    # same bits as the two-kernel route of the library itself
+    xq, a_scale = gpu_quant_act(bits)
+    y2, _ = gpu_gemm(sparse, xq, a_scale, p)
+    assert torch.equal(y, y2)
