@@ -1,6 +1,9 @@
 // Algorithm 2's forward for few tokens in ONE kernel: per-token absmax quantisation of the bf16
-// activations (Sec. 2.1) and Eq. 4, for a decode loop where a separate quantiser launch is a
-// quarter of a BitLinear's time.
+// activations (Sec. 2.1) and Eq. 4.  One launch instead of two: 9.8 us against 12.8 us per BitLinear
+// at T = 8 when launches are plainly serialised.  Inside a chain of programmatic dependent launches
+// the separate quantiser costs only ~1.3 us and the two-kernel route is the faster one (6.4 us
+// against 7.6 us): here every one of the N / 128 row tiles reads and quantises the tile's tokens
+// again, and the exchange of row maxima is one more hop on the critical path.
 //
 // The cluster split-K kernel of gemm_splitk_cluster_tcgen05.cuh with the activation operand made
 // in place: the S CTAs of a cluster share an output tile (128 features x up to 32 tokens) and
@@ -213,7 +216,15 @@ bitlinear_gemm_fused_act_cluster_kernel(const __grid_constant__ CUtensorMap tmap
         // pass 1: maximum of |x| over this CTA's slice (bit patterns of non-negative bf16 order like integers)
         uint32_t pm = 0u;
         if (real) {
-            for (int blk = 0; blk < nblk; ++blk) {
+            int blk = 0;
+            for (; blk + 4 <= nblk; blk += 4) {                          // 16 independent loads in flight
+                uint4 v[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[i] = __ldg(xrow + (blk + (i >> 2)) * 16 + (i & 3));
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pm = absmax8_packed(v[i], pm);
+            }
+            for (; blk < nblk; ++blk) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) pm = absmax8_packed(__ldg(xrow + blk * 16 + i), pm);
             }
@@ -246,17 +257,28 @@ bitlinear_gemm_fused_act_cluster_kernel(const __grid_constant__ CUtensorMap tmap
         asm volatile("bar.sync 1, 128;" ::: "memory");                    // the scales are read by other threads in the finish
         // pass 2: x~ into the B image of every stage (row = token, 128 B, 16 B chunks XOR-ed with row % 8)
         const uint32_t brow = (static_cast<uint32_t>(tok) >> 3) * 1024u + (static_cast<uint32_t>(tok) & 7u) * 128u;
+        // (L1 is too small next to two CTAs' shared memory to keep pass 1's lines: this pass reads from L2
+        // again, one k-block ahead of the one being written)
+        uint4 nxt[4] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+        if (real && nblk > 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) nxt[i] = __ldg(xrow + i);
+        }
         for (int blk = 0; blk < nblk && ok; ++blk) {
             const int stage = blk % STAGES;
-            if (blk >= STAGES && !mbar_wait(bar_empty + 8 * stage, static_cast<uint32_t>(blk / STAGES - 1) & 1u, abort_flag)) { ok = false; break; }
-            uint32_t c[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-            if (real) {
+            uint4 cur[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 v = __ldg(xrow + blk * 16 + i);
-                    c[2 * i] = quant_pair2(v.x, v.y, s_x);
-                    c[2 * i + 1] = quant_pair2(v.z, v.w, s_x);
-                }
+            for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
+            if (real && blk + 1 < nblk) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) nxt[i] = __ldg(xrow + (blk + 1) * 16 + i);
+            }
+            if (blk >= STAGES && !mbar_wait(bar_empty + 8 * stage, static_cast<uint32_t>(blk / STAGES - 1) & 1u, abort_flag)) { ok = false; break; }
+            uint32_t c[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                c[2 * i] = quant_pair2(cur[i].x, cur[i].y, s_x);          // padding tokens: zeros in, zeros out
+                c[2 * i + 1] = quant_pair2(cur[i].z, cur[i].w, s_x);
             }
             const uint32_t base = smem_b + stage * Cfg::B_BYTES + brow;
             const uint32_t r7 = static_cast<uint32_t>(tok) & 7u;
@@ -313,18 +335,16 @@ bitlinear_gemm_fused_act_cluster_kernel(const __grid_constant__ CUtensorMap tmap
         const float* a_sc = reinterpret_cast<const float*>(smem_raw + (smem_amax + 8u * BN * 4u - smem_u32(smem_raw)));
         const bool fine = (*abort_flag == 0);
         const int n_tok = (fine && ok) ? my_tokens : 0;
-        for (int j = 0; j < n_tok; ++j) {
+        cluster_finish(S, red, tok_per_cta, n_tok, f, [&](int j, int acc) {
             const int tl = j * static_cast<int>(S) + static_cast<int>(rank);          // token inside the tile
             const float sc = __fmul_rn(w_scale, a_sc[tl]);
-            int acc = 0;
-            for (uint32_t s2 = 0; s2 < S; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];
             const size_t o = static_cast<size_t>(t0 + tl) * p.N + n;
             if (p.acc_out) p.acc_out[o] = acc;
             float v = __fmul_rn(static_cast<float>(acc), sc);
             if (p.bias) v = __fadd_rn(v, bias);
             if (p.out_bf16) static_cast<uint16_t*>(p.y)[o] = static_cast<uint16_t>(f32_to_bf16_rne(v));
             else static_cast<float*>(p.y)[o] = v;
-        }
+        });
     }
 
     tcgen05_fence_before();

@@ -294,17 +294,15 @@ bitlinear_gemm_packed_cluster_kernel(const __grid_constant__ CUtensorMap tmap_b,
         const int32_t* red = reinterpret_cast<const int32_t*>(smem_raw + (smem_red - smem_u32(smem_raw)));
         const bool fine = (*abort_flag == 0);
         const int n_tok = (fine && ok) ? my_tokens : 0;
-        for (int j = 0; j < n_tok; ++j) {
+        cluster_finish(S, red, tok_per_cta, n_tok, f, [&](int j, int acc) {
             const int t = t0 + j * static_cast<int>(S) + static_cast<int>(rank);
             const float sc = __shfl_sync(0xFFFFFFFFu, sc_a, j);
-            int acc = 0;
-            for (uint32_t s2 = 0; s2 < S; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];
             if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
             float v = __fmul_rn(static_cast<float>(acc), sc);
             if (p.bias) v = __fadd_rn(v, bias);
             if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
             else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
-        }
+        });
     }
 
     tcgen05_fence_before();

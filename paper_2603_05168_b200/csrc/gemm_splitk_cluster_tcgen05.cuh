@@ -70,6 +70,37 @@ __device__ __forceinline__ uint32_t cluster_nctarank() {
     return r;
 }
 
+// Adds the S partial sums of each of this CTA's n_tok tokens (buffer [S][tok_per_cta][128] int32, this
+// thread's feature f) and hands (local token index, sum) to `emit`.  Four tokens at a time with S known
+// at compile time: 4 * S independent loads in flight -- the one-token-at-a-time loop with a run-time S
+// was a chain of shared-memory latencies, 0.12 us per token.
+template <int SS, typename Emit>
+__device__ __forceinline__ void cluster_finish_tokens(const int32_t* red, int tok_per_cta, int n_tok, int f, Emit emit) {
+    int j = 0;
+    for (; j + 4 <= n_tok; j += 4) {
+        int acc[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int s2 = 0; s2 < SS; ++s2)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[u] += red[(s2 * tok_per_cta + j + u) * kBM + f];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) emit(j + u, acc[u]);
+    }
+    for (; j < n_tok; ++j) {
+        int acc = 0;
+#pragma unroll
+        for (int s2 = 0; s2 < SS; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];
+        emit(j, acc);
+    }
+}
+template <typename Emit>
+__device__ __forceinline__ void cluster_finish(uint32_t S, const int32_t* red, int tok_per_cta, int n_tok, int f, Emit emit) {
+    if (S == 2u) cluster_finish_tokens<2>(red, tok_per_cta, n_tok, f, emit);
+    else if (S == 3u) cluster_finish_tokens<3>(red, tok_per_cta, n_tok, f, emit);
+    else if (S == 4u) cluster_finish_tokens<4>(red, tok_per_cta, n_tok, f, emit);
+    else cluster_finish_tokens<8>(red, tok_per_cta, n_tok, f, emit);
+}
+
 template <bool SPARSE, int BN>
 __global__ void __launch_bounds__(kSplitThreads, SplitConfig<SPARSE, BN>::CTAS_PER_SM)
 bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
@@ -312,38 +343,15 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         const int32_t* red = reinterpret_cast<const int32_t*>(smem_raw + (smem_red - smem_u32(smem_raw)));
         const bool fine = (*abort_flag == 0);
         const int n_tok = (fine && ok) ? my_tokens : 0;
-        auto finish = [&](auto s_const) {
-            constexpr int SS = decltype(s_const)::value;
-            auto emit = [&](int j, int acc) {
-                const int t = t0 + j * SS + static_cast<int>(rank);
-                const float sc = __shfl_sync(0xFFFFFFFFu, j < 32 ? sc_a : sc_b, j & 31);
-                if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
-                float v = __fmul_rn(static_cast<float>(acc), sc);
-                if (p.bias) v = __fadd_rn(v, bias);
-                if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
-                else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
-            };
-            int j = 0;
-            for (; j + 4 <= n_tok; j += 4) {              // four tokens at a time: 4 * S independent loads in flight
-                int acc[4] = {0, 0, 0, 0};
-#pragma unroll
-                for (int s2 = 0; s2 < SS; ++s2)
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) acc[u] += red[(s2 * tok_per_cta + j + u) * kBM + f];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) emit(j + u, acc[u]);
-            }
-            for (; j < n_tok; ++j) {
-                int acc = 0;
-#pragma unroll
-                for (int s2 = 0; s2 < SS; ++s2) acc += red[(s2 * tok_per_cta + j) * kBM + f];
-                emit(j, acc);
-            }
-        };
-        if (S == 2u) finish(std::integral_constant<int, 2>{});
-        else if (S == 3u) finish(std::integral_constant<int, 3>{});
-        else if (S == 4u) finish(std::integral_constant<int, 4>{});
-        else finish(std::integral_constant<int, 8>{});
+        cluster_finish(S, red, tok_per_cta, n_tok, f, [&](int j, int acc) {
+            const int t = t0 + j * static_cast<int>(S) + static_cast<int>(rank);
+            const float sc = __shfl_sync(0xFFFFFFFFu, j < 32 ? sc_a : sc_b, j & 31);
+            if (p.acc_out) p.acc_out[static_cast<size_t>(t) * p.N + n] = acc;
+            float v = __fmul_rn(static_cast<float>(acc), sc);
+            if (p.bias) v = __fadd_rn(v, bias);
+            if (p.out_bf16) static_cast<uint16_t*>(p.y)[static_cast<size_t>(t) * p.N + n] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+            else static_cast<float*>(p.y)[static_cast<size_t>(t) * p.N + n] = v;
+        });
     }
 
     // teardown

@@ -169,3 +169,20 @@ def test_dispatch_plan_is_sane(L):
             tiles = (N // 128) * ((T + bn - 1) // bn)
             assert tiles * cluster <= (296 if bn <= 64 else 148)       # every CTA resident at once
     assert b.sbn_plan_gemm(True, 16, 100, 2560) == (0, 0, 0, 0)        # illegal shape
+
+
+def test_fused_entry_validation_on_host(L):
+    p = ctypes.c_void_p(0x1000)
+    odd = ctypes.c_void_p(0x1004)
+    NULL, SHAPE, ALIGN, UNSUP = 1, 2, 3, 4
+    fs = lambda **k: L.sbn_quant_act_sparse_bitlinear(k.get("x", p), k.get("T", 8), p, k.get("meta", p), p, k.get("N", 256),
+                                                      k.get("K", 512), None, p, k.get("dt", 0), None, None, None)
+    assert fs(x=None) == NULL
+    assert fs(meta=None) == NULL
+    assert fs(T=0) == SHAPE
+    assert fs(N=100) == SHAPE
+    assert fs(T=300) == UNSUP
+    assert fs(K=128) == UNSUP
+    assert fs(dt=9) == UNSUP
+    assert fs(x=odd) == ALIGN
+    assert L.sbn_quant_act_bitlinear(p, 8, None, p, 256, 512, None, p, 0, None, None, None) == NULL
