@@ -516,7 +516,7 @@ def _cold_timer(torch, stream, flush):
 
 
 def run_decode_sweep(args):
-    """Small-T regime (the paper's decode table is M = 64..512): T in {1, 16, 64, 128, 256, 512} over
+    """Small-T regime (the paper's decode table is M = 64..512): T in {1, 4, 16, 64, 128, 256, 512} over
     the four 2B-shaped matrices, sparse vs dense.  Two timings per point: `cold` = one launch after
     512 MB were written over L2 (includes the ~6 us an empty launch costs between two events), and
     `stream` = launches back to back over enough distinct weight copies that every launch reads its
@@ -550,7 +550,7 @@ def run_decode_sweep(args):
 
     big = args.workload == "decode7b"
     shapes = [("gate_up_7b", 4096, 11008), ("down_7b", 11008, 4096), ("qkv_7b", 4096, 12288), ("o_7b", 4096, 4096)] if big else inputs.SHAPES_2B
-    token_counts = (1, 16, 32, 64) if big else (1, 16, 64, 128, 256, 512)
+    token_counts = (1, 4, 16, 32, 64) if big else (1, 4, 16, 64, 128, 256, 512)
     rows = []
     for i, (name, K, N) in enumerate(shapes):
         W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i)).cuda()
