@@ -7,8 +7,9 @@
 // (one 1024-thread CTA per SM) therefore reads W ONCE, for one matrix or a batch of them:
 //
 //   sample   every CTA adds |w| over the same 256 scattered 512 B units of the matrix (128 KB,
-//            L2-served for all CTAs but the first) -> gamma_est, and brackets the threshold:
-//            thr_lo ~ thr(0.97 gamma_est), thr_hi ~ thr(1.03 gamma_est);
+//            L2-served for all CTAs but the first; 64 units for matrices below 33 M weights)
+//            -> gamma_est, and brackets the threshold: thr_lo ~ thr(0.97 gamma_est),
+//            thr_hi ~ thr(1.03 gamma_est) (0.96 / 1.04 with the small sample);
 //   pass 1   every CTA owns a contiguous range of (row, 128-column) units and streams it:
 //            sum|W| in fp64 (the exact gamma), top 2 of 4 per group (Eq. 2: the mask does not
 //            depend on gamma), metadata, flip count, and the two kept values ternarised
@@ -48,8 +49,19 @@ constexpr int kQmpWarps = kQmpThreads / 32;
 constexpr int kQmpMaxCtas = kNumSMs;                       // one CTA per SM, all co-resident
 constexpr int kQmpListCap = 8192;                          // undecided entries per CTA and matrix
 constexpr int kQmpSmemBytes = 2 * kQmpListCap * 8;         // two lists (consecutive matrices of a batch)
-constexpr int kQmpSampleUnits = 256;                       // units in the gamma_est sample
+constexpr int kQmpSampleUnits = 256;                       // units in the gamma_est sample of a large matrix
 constexpr float kQmpBracket = 0.03f;                       // gamma_est * (1 -+ this) brackets gamma
+// Matrices below 2^18 units (33.5 M weights) are sampled at a quarter of that with a wider bracket:
+// there the sample is a visible part of the kernel's time (2.5 us of ~25), and 8192 weights still put
+// the bracket at 4.8 standard errors of the mean for Gaussian weights.  Large matrices keep the
+// larger sample, which also holds for heavy-tailed weights.
+constexpr int kQmpSampleUnitsSmall = 64;
+constexpr float kQmpBracketSmall = 0.04f;
+constexpr uint32_t kQmpSmallMatrixUnits = 1u << 18;
+__host__ __device__ inline uint32_t qmp_sample_units(uint32_t num_units) {
+    const uint32_t want = num_units < kQmpSmallMatrixUnits ? kQmpSampleUnitsSmall : kQmpSampleUnits;
+    return num_units < want ? num_units : want;
+}
 constexpr unsigned long long kQmpWaitLimitNs = 2000000000ull;
 
 struct QmpSlot {                 // one per CTA, 16 B
@@ -199,7 +211,7 @@ template <bool BF16>
 __device__ __forceinline__ float qmp_sample_gamma(const QmpDesc& d, double* s_warp) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint32_t n_s = min(d.num_units, static_cast<uint32_t>(kQmpSampleUnits));
+    const uint32_t n_s = qmp_sample_units(d.num_units);
     const uint32_t stride = d.num_units / n_s;                        // >= 1
     float acc = 0.0f;
     constexpr int kPerWarp = kQmpSampleUnits / kQmpWarps;
@@ -404,8 +416,9 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                 s_list_count[par] = 0u;
                 // any lo <= hi will do (the exact threshold is checked against them later), so no
                 // divisions here: thr(scale) is 0.5 * scale to within a few ulps
-                s_bracket[par][0] = 0.5f * fmaxf(gamma_est * (1.0f - kQmpBracket), kEps) * (1.0f - 1e-6f);
-                s_bracket[par][1] = 0.5f * fmaxf(gamma_est * (1.0f + kQmpBracket), kEps) * (1.0f + 1e-6f);
+                const float b = d_cur.num_units < kQmpSmallMatrixUnits ? kQmpBracketSmall : kQmpBracket;
+                s_bracket[par][0] = 0.5f * fmaxf(gamma_est * (1.0f - b), kEps) * (1.0f - 1e-6f);
+                s_bracket[par][1] = 0.5f * fmaxf(gamma_est * (1.0f + b), kEps) * (1.0f + 1e-6f);
             }
             __syncthreads();
             unsigned int flips = 0;

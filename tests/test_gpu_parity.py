@@ -219,9 +219,10 @@ def test_quantize_mask_pack_batched_mixed_master_dtypes():
 
 def _sampled_units(N, K):
     """The units the kernel's gamma estimate looks at (restated from the kernel's description:
-    256 units, unit s at s * stride + (s * 2654435761 mod 2^32 >> 8) mod stride)."""
+    256 units -- 64 for matrices below 2^18 units -- unit s at s * stride + (s * 2654435761 mod 2^32 >> 8)
+    mod stride)."""
     num_units = N * K // 128
-    n_s = min(num_units, 256)
+    n_s = min(num_units, 64 if num_units < (1 << 18) else 256)
     stride = num_units // n_s
     sidx = np.arange(n_s, dtype=np.uint64)
     return (sidx * stride + (((sidx * 2654435761) & 0xFFFFFFFF) >> 8) % stride).astype(np.int64)
