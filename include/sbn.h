@@ -355,7 +355,8 @@ const char *sbn_status_string(sbn_status s);
  * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
  * 256 dense).  split_k: 0 = automatic; k > 0 = split K k ways through int32 atomics in the
  * workspace (single-CTA kernel); -2, -3, -4, -8 = split K inside thread-block clusters of that many
- * CTAs (token tile 64, or 32 / 128 if token_tile says so; no workspace).  Results do not depend on
+ * CTAs (token tile 64, or 32 / 128 if token_tile says so; no workspace; -2, -3, -4 also set the
+ * cluster size of sbn_sparse_bitlinear_packed and of the sbn_quant_act_*bitlinear kernels).  Results do not depend on
  * it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);
 

@@ -650,6 +650,12 @@ sbn_status sbn_layer_forward_host(const void* x_bf16_host, int T, int K, void* x
 // Cluster size for the 32-token few-token kernels: the cost model of plan_gemm restricted to that tile.
 static int pick_cluster_32(bool sparse, int T, int N, int K) {
     const int kb = K / kBK, rows = N / kBM;
+    if (g_force_split_k < 0) {                                  // diagnostics: cluster size as told
+        int S = -g_force_split_k;
+        S = S >= 4 ? 4 : (S == 3 ? 3 : 2);
+        while (S > 2 && S > kb) --S;
+        return S;
+    }
     const long tiles = static_cast<long>(rows) * ((T + 31) / 32);
     const long slots = 2L * kNumSMs;
     int best_s = 2;
@@ -765,20 +771,7 @@ sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, i
     p.split_acc = nullptr; p.split_counters = nullptr;
     p.w_vals = vals2; p.w_meta = meta; p.w_tile_bytes = kVals2TileBytes;
     const int tiles = (N / kBM) * ((T + Cfg::BN - 1) / Cfg::BN);
-    // cluster size: the one with the shortest K-loop on the busiest SM among those that keep every
-    // CTA resident at once (two per SM); 2 if none does
-    int cluster = 2;
-    {
-        const int sms = device_sm_count();
-        long best = -1;
-        for (int S = 2; S <= 4; ++S) {
-            if (S > p.k_blocks_total || static_cast<long>(tiles) * S > 2L * sms) break;
-            if (S == 3 && static_cast<long>(tiles) * S * 100 > 2L * sms * 93) continue;
-            const long per_sm = (static_cast<long>(tiles) * S + sms - 1) / sms;
-            const long load = (10 + 6 * (per_sm - 1)) * ((p.k_blocks_total + S - 1) / S) + (S == 3 ? 18 : 0);   // tenths of a block
-            if (best < 0 || load < best) { best = load; cluster = S; }
-        }
-    }
+    const int cluster = pick_cluster_32(true, T, N, K);
     if (!ensure_dynamic_smem<bitlinear_gemm_packed_cluster_kernel>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
     const cudaError_t err = launch_kernel_cluster(bitlinear_gemm_packed_cluster_kernel, dim3(tiles * cluster), dim3(kSplitThreads),
                                                   Cfg::SMEM_BYTES, static_cast<cudaStream_t>(stream), static_cast<unsigned>(cluster), tb, p);

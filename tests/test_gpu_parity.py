@@ -880,3 +880,28 @@ def test_fused_quant_act_gemm_parity(sparse, T, N, K):
     xq, a_scale = gpu_quant_act(bits)
     y2, _ = gpu_gemm(sparse, xq, a_scale, p)
     assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("cluster", [2, 3, 4])
+@pytest.mark.parametrize("T,N,K", [(16, 256, 2560), (31, 128, 896), (45, 256, 640), (7, 384, 4096)])
+def test_packed_and_fused_kernels_every_cluster_size(T, N, K, cluster):
+    # the 32-token kernels with the cluster size forced: 3 takes the select route of the scatter
+    W = inputs.latent_weights(N, K, seed=T + N + K + cluster)
+    bits = inputs.activations_bf16(T, K, seed=T + N + K + cluster + 1, token_lognormal_sigma=0.5)
+    r = _oracle_pack(W)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    p = g["dev"]
+    vals2, _ = gpu_pack_vals2(p)
+    xq, a_scale = gpu_quant_act(bits)
+    b.sbn_set_gemm_tuning(0, -cluster)
+    y, acc = gpu_gemm_packed(xq, a_scale, vals2, p)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    y2 = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    acc2 = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device="cuda")
+    b.sbn_quant_act_sparse_bitlinear(bf16_dev(bits), p["vals"], p["meta"], p["w_scale"], y2, acc_out=acc2)
+    b.sbn_check_status()
+    assert np.array_equal(acc2.cpu().numpy(), acc_ref)
+    assert torch.equal(y, y2)
