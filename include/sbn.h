@@ -353,7 +353,7 @@ const char *sbn_status_string(sbn_status s);
 /* Tuning/diagnostic knob (host state, not thread-safe).  token_tile: 0 = automatic; 64, 128 or
  * 256 = force the single-CTA kernel with that token-tile width; a negative value -BN = force the
  * CTA-pair kernel with BN tokens per tile (rounded to a multiple of 16, capped at 240 sparse /
- * 256 dense).  split_k: 0 = automatic; k > 0 = split K k ways through int32 atomics in the
+ * 256 dense; with split_k = 1 its variant with one M-tile per CTA).  split_k: 0 = automatic; k > 0 = split K k ways through int32 atomics in the
  * workspace (single-CTA kernel); -2, -3, -4, -8 = split K inside thread-block clusters of that many
  * CTAs (token tile 64, or 32 / 128 if token_tile says so; no workspace; -2, -3, -4 also set the
  * cluster size of sbn_sparse_bitlinear_packed and of the sbn_quant_act_*bitlinear kernels).  Results do not depend on
@@ -361,7 +361,8 @@ const char *sbn_status_string(sbn_status s);
 void sbn_set_gemm_tuning(int token_tile, int split_k);
 
 /* Diagnostic: what the dispatcher would run for this shape (host only, launches nothing).
- * out4[0] = kernel (0 single-CTA tiles, 1 cluster split-K, 2 CTA pair), out4[1] = tokens per tile,
+ * out4[0] = kernel (0 single-CTA tiles, 1 cluster split-K, 2 CTA pair with 512-feature tiles, 3 CTA
+ * pair with 256-feature tiles and double-buffered accumulators), out4[1] = tokens per tile,
  * out4[2] = split-K factor through global memory (1 = none), out4[3] = cluster size (0 = none).
  * All zero for an illegal shape. */
 void sbn_plan_gemm(int sparse, int T, int N, int K, int *out4);

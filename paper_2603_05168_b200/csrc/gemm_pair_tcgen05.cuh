@@ -44,15 +44,20 @@ constexpr int kPairEpiBytes = 2 * 256 * 4;                        // per-token s
 constexpr int kPairMaxBnSparse = 240;
 constexpr int kPairMaxBnDense = 256;
 
-template <bool SPARSE>
+// MT = M-tiles (128-row weight blocks) per CTA.  2: the pair tile is 512 features wide, both M-tiles
+// run against the same activation stage (least shared-memory traffic per MMA), accumulators
+// single-buffered.  1: 256 features per pair tile, the second half of tensor memory is a second
+// accumulator, so the drain of a tile hides under the next tile's MMAs and the tiles are half as
+// large -- for short K (few stages per tile) and for tile counts that quantise badly into waves.
+template <bool SPARSE, int MT = 2>
 struct PairConfig {
     static constexpr int KBS = SPARSE ? 2 : 1;                               // 128-column blocks per stage
     static constexpr int A_TILE = SPARSE ? kBM * (kBK / 2) : kBM * kBK;     // one row block x one k-block
     static constexpr int E_TILE = SPARSE ? kBM * (kBK / 8) : 0;
     static constexpr int B_ROWS_MAX = SPARSE ? kPairMaxBnSparse / 2 : kPairMaxBnDense / 2;
     static constexpr int B_TILE = B_ROWS_MAX * kBK;                          // one k-block of activations
-    static constexpr int A_BYTES = 2 * KBS * A_TILE;
-    static constexpr int E_BYTES = 2 * KBS * E_TILE;
+    static constexpr int A_BYTES = MT * KBS * A_TILE;
+    static constexpr int E_BYTES = MT * KBS * E_TILE;
     static constexpr int B_BYTES = KBS * B_TILE;
     static constexpr int STAGE_BYTES = A_BYTES + E_BYTES + B_BYTES;
     // the kernel has no static shared memory, so the dynamic part starts 1 KB-aligned (checked)
@@ -62,6 +67,7 @@ struct PairConfig {
     static_assert(STAGES >= 3, "not enough stages");
     static_assert(!SPARSE || KBS == 2, "the 128x256b metadata copy covers exactly two k-blocks");
     static_assert(SMEM_BYTES <= 232448, "shared memory overflow");
+    static_assert(MT == 1 || MT == 2, "M-tiles per CTA");
 };
 
 struct PairParams {
@@ -166,17 +172,18 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
 // Epilogue of one pair tile for one warp, bf16 outputs (see the kernel for the scheme): phase A
 // drains this warp's chunks chunk0 + 2 k of the accumulator into packed registers and hands the
 // accumulator back, phase B stores them.
-template <bool SMALL>
+template <bool SMALL, int STRIDE>
 __device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, const int t0, const int n, const float bias,
                                                         const int live, const int full32, const uint32_t t_addr,
                                                         const float* sc_tile, const int lane, const int chunk0,
                                                         const uint32_t acc_empty_leader) {
-    uint32_t packed[4][16];
+    constexpr int NK = 8 / STRIDE;                               // chunks per warp: chunk0, chunk0 + STRIDE, ...
+    uint32_t packed[NK][16];
     const bool has_bias = p.bias != nullptr;
     // ---- phase A
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int i = chunk0 + 2 * k;
+    for (int k = 0; k < NK; ++k) {
+        const int i = chunk0 + STRIDE * k;
         if (i < live) {
             const bool half_chunk = (i == full32);                 // the 16-wide tail
             // 16 columns at a time: the tile's packed outputs take most of the registers
@@ -187,7 +194,7 @@ __device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, con
                     tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>(i * 32 + h * 16), r);
                     const float2* sc2 = reinterpret_cast<const float2*>(sc_tile + i * 32 + h * 16);   // uniform reads
                     tmem_ld_wait();
-                    if (i + 2 >= live && (h == 1 || half_chunk)) {
+                    if (i + STRIDE >= live && (h == 1 || half_chunk)) {
                         // last TMEM read of this warp is complete: hand the accumulator back
                         tcgen05_fence_before();
                         __syncwarp();
@@ -207,8 +214,8 @@ __device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, con
     }
     // ---- phase B
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int i = chunk0 + 2 * k;
+    for (int k = 0; k < NK; ++k) {
+        const int i = chunk0 + STRIDE * k;
         if (i < live) {
             const int tc = t0 + i * 32;
             const int cnt = min(p.T - tc, (i == full32) ? 16 : 32);   // live tokens of the chunk (warp-uniform)
@@ -226,13 +233,13 @@ __device__ __forceinline__ void pair_epilogue_tile_bf16(const GemmParams& p, con
 
 // The same for fp32 outputs and / or the raw accumulator dump: these do not fit in registers and
 // are stored while the accumulator drains.
-template <bool SMALL>
+template <bool SMALL, int STRIDE>
 __device__ __forceinline__ void pair_epilogue_tile_direct(const GemmParams& p, const int t0, const int n, const float bias,
                                                           const int live, const int full32, const uint32_t t_addr,
                                                           const float* sc_tile, const int lane, const int chunk0,
                                                           const uint32_t acc_empty_leader) {
 #pragma unroll 1
-    for (int i = chunk0; i < live; i += 2) {
+    for (int i = chunk0; i < live; i += STRIDE) {
         const bool half_chunk = (i == full32);
         const int tc = t0 + i * 32;
         const int cnt = min(p.T - tc, half_chunk ? 16 : 32);
@@ -243,7 +250,7 @@ __device__ __forceinline__ void pair_epilogue_tile_direct(const GemmParams& p, c
                 tmem_ld_32x32b_x16(t_addr + static_cast<uint32_t>(i * 32 + h * 16), r);
                 const float2* sc2 = reinterpret_cast<const float2*>(sc_tile + i * 32 + h * 16);
                 tmem_ld_wait();
-                if (i + 2 >= live && (h == 1 || half_chunk)) {
+                if (i + STRIDE >= live && (h == 1 || half_chunk)) {
                     tcgen05_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
@@ -282,16 +289,17 @@ __device__ __forceinline__ void pair_epilogue_tile_direct(const GemmParams& p, c
 //   tmap_a  [N/128][KB * rows_per_tile][1 KB]   box {1 KB, rows_per_tile * KBS, 2}
 //   tmap_e  [N/128][KB * 2][1 KB]               box {1 KB, 2 * KBS, 2}          (sparse)
 //   tmap_b  [KB][TB8][1 KB]                     box {1 KB, BN/16, KBS}
-template <bool SPARSE>
+template <bool SPARSE, int MT = 2>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                            const __grid_constant__ CUtensorMap tmap_b,
                            const __grid_constant__ CUtensorMap tmap_e,
                            const PairParams pp) {
-    using Cfg = PairConfig<SPARSE>;
+    using Cfg = PairConfig<SPARSE, MT>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int KBS = Cfg::KBS;
     constexpr int A_ROWS = Cfg::A_TILE / 1024;            // 1 KB rows per weight tile
+    constexpr int ROWS_PER_TILE = 2 * MT;                  // 128-row weight blocks of a pair tile
     const GemmParams& p = pp.g;
     const int BN = pp.bn;
     const int half_bn = BN >> 1;
@@ -309,9 +317,9 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const uint32_t bar_base = smem_epi + kPairEpiBytes;
     const uint32_t bar_full = bar_base;
     const uint32_t bar_empty = bar_full + 8 * STAGES;
-    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;
-    const uint32_t bar_acc_empty = bar_acc_full + 8;
-    const uint32_t tmem_slot = bar_acc_empty + 8;
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;     // [2]: one per accumulator buffer (MT = 2 uses [0])
+    const uint32_t bar_acc_empty = bar_acc_full + 16;
+    const uint32_t tmem_slot = bar_acc_empty + 16;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + (tmem_slot + 8 - smem_base));
 
     const int warp = threadIdx.x >> 5;
@@ -321,7 +329,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
     const int num_pairs = gridDim.x >> 1;
 
     const int n_blocks = p.N >> 7;
-    const int tiles_m = (p.N + 511) / 512;
+    const int tiles_m = (p.N + 128 * ROWS_PER_TILE - 1) / (128 * ROWS_PER_TILE);
     const int tiles_t = (p.T + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_t;
     const int k_blocks = p.k_blocks_total;
@@ -333,8 +341,10 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        mbar_init(bar_acc_full, 1);
-        mbar_init(bar_acc_empty, 2 * kPairEpiWarps);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, 2 * kPairEpiWarps);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -362,7 +372,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int mt = tile % tiles_m;
                 const int tt = tile / tiles_m;
-                const int nb0 = mt * 4 + static_cast<int>(rank) * 2;            // this CTA's two row blocks
+                const int nb0 = mt * ROWS_PER_TILE + static_cast<int>(rank) * MT;   // this CTA's row blocks
                 const int t_atom = (tt * BN + static_cast<int>(rank) * half_bn) >> 3;   // this CTA's token half
                 for (int ks = 0; ks < k_stages; ++ks) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -386,16 +396,20 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             const uint32_t b_kb_bytes = static_cast<uint32_t>(half_bn * kBK);    // B bytes of one k-block
             int stage = 0;
             uint32_t phase = 0;
-            uint32_t acc_phase = 0;
+            uint32_t acc_iter = 0;                                      // tiles done by this pair
             uint32_t e_slot = 0;
             const uint32_t e_slots = BN <= 224 ? 4u : 2u;              // 8-column metadata slots above the accumulator
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int mt = tile % tiles_m;
-                // M-tile i is live if at least the leader's row block 4*mt + i exists
-                const int mt_count = (mt * 4 + 1 < n_blocks) ? 2 : 1;
-                // single-buffered accumulators: wait until the epilogues of both CTAs drained them
-                if (!mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                // M-tile i is live if at least the leader's row block exists
+                const int mt_count = (MT == 2 && mt * 4 + 1 < n_blocks) ? 2 : 1;
+                // MT = 2: one accumulator per M-tile, single-buffered.  MT = 1: the two halves of tensor
+                // memory alternate between consecutive tiles.  Either way: wait until the epilogues of
+                // both CTAs have drained the accumulator this tile writes.
+                const uint32_t buf = (MT == 1) ? (acc_iter & 1u) : 0u;
+                const uint32_t acc_phase = (MT == 1) ? ((acc_iter >> 1) & 1u) : (acc_iter & 1u);
+                if (!mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tcgen05_fence_after();
                 for (int ks = 0; ks < k_stages; ++ks) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
@@ -421,7 +435,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                             const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);
                             const uint32_t first = (ks | j) == 0 ? 0u : 1u;
                             for (int i = 0; i < mt_count; ++i) {
-                                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(i * 256);
+                                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>((MT == 1 ? buf : i) * 256);
                                 const uint32_t a_addr = st + static_cast<uint32_t>((i * KBS + j) * Cfg::A_TILE);
                                 if constexpr (SPARSE) {
                                     const uint64_t a_desc = make_smem_desc(a_addr, 16, 512, kSwz64);
@@ -448,8 +462,8 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tcgen05_commit_pair(bar_acc_full);
-                acc_phase ^= 1u;
+                tcgen05_commit_pair(bar_acc_full + 8 * buf);
+                ++acc_iter;
             }
         }
     } else {
@@ -472,22 +486,26 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
         // from phase A directly.
         const int ew = warp - 2;                          // 0..15
         const int quarter = warp & 3;                     // TMEM lane quarter this warp may read
-        const int mtile = (ew >> 2) & 1;                  // which M-tile this warp drains
-        const int chunk0 = ew >> 3;                       // chunks chunk0, chunk0 + 2, chunk0 + 4, chunk0 + 6
+        // MT = 2: M-tile (ew >> 2) & 1, chunks ew >> 3, + 2, + 4, + 6.  MT = 1: chunks ew >> 2, + 4.
+        constexpr int STRIDE = (MT == 2) ? 2 : 4;
+        const int mtile = (MT == 2) ? ((ew >> 2) & 1) : 0;
+        const int chunk0 = (MT == 2) ? (ew >> 3) : (ew >> 2);
         static_assert(kPairEpiWarps == 16, "chunk assignment assumes two warps per lane quarter and M-tile");
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const float w_scale = __ldg(p.w_scale);
-        const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
         const bool small_acc = k_blocks < 256;            // |acc| <= 128 K < 2^22
         float* const s_scale = reinterpret_cast<float*>(smem_raw + (smem_epi - smem_base));   // [2][256]
         const int et = threadIdx.x - 64;                  // 0..511 among the epilogue threads
         uint32_t tile_par = 0;
-        uint32_t acc_phase = 0;
+        uint32_t acc_iter = 0;
         bool ok = true;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
             const int mt = tile % tiles_m;
             const int tt = tile / tiles_m;
-            const int n0 = (mt * 4 + static_cast<int>(rank) * 2 + mtile) * 128 + quarter * 32;
+            const int n0 = (mt * ROWS_PER_TILE + static_cast<int>(rank) * MT + mtile) * 128 + quarter * 32;
+            const uint32_t buf = (MT == 1) ? (acc_iter & 1u) : 0u;
+            const uint32_t acc_phase = (MT == 1) ? ((acc_iter >> 1) & 1u) : (acc_iter & 1u);
+            const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty + 8 * buf, 0);
             const int n = n0 + lane;
             const int t0 = tt * BN;
             const bool rows_valid = n0 < p.N;             // warp-uniform (N % 128 == 0)
@@ -497,14 +515,14 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
             // a 16-wide last chunk (BN % 32 == 16) is read with a 16-column load: the columns above
             // it hold metadata
             const int full32 = BN >> 5;
-            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(mtile * 256);
+            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>((MT == 1 ? buf : static_cast<uint32_t>(mtile)) * 256);
             // s of Eq. 4 for the tile's tokens, shared by all epilogue warps (double-buffered over
             // tiles: one named barrier per tile orders the fill against every reader)
             float* const sc_tile = s_scale + tile_par * 256;
             if (et < BN) sc_tile[et] = (t0 + et < p.T) ? __fmul_rn(w_scale, __ldg(p.a_scale + t0 + et)) : 0.0f;
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kPairEpiWarps) : "memory");
             tile_par ^= 1u;
-            if (!mbar_wait(bar_acc_full, acc_phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
 
             // bf16 outputs stay in registers until phase B (K >= 32768 takes the plain route: its
@@ -516,12 +534,12 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
             } else if (keep) {
-                pair_epilogue_tile_bf16<true>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
+                pair_epilogue_tile_bf16<true, STRIDE>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
             } else {
-                if (small_acc) pair_epilogue_tile_direct<true>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
-                else pair_epilogue_tile_direct<false>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
+                if (small_acc) pair_epilogue_tile_direct<true, STRIDE>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
+                else pair_epilogue_tile_direct<false, STRIDE>(p, t0, n, bias, live, full32, t_addr, sc_tile, lane, chunk0, acc_empty_leader);
             }
-            acc_phase ^= 1u;
+            ++acc_iter;
         }
     }
 

@@ -131,6 +131,7 @@ struct GemmPlan {
     int bn;         // token tile
     int splits;     // split-K factor through global atomics (single-CTA kernel only)
     int cluster;    // > 1: split-K inside clusters of this many CTAs (reduction in shared memory)
+    int mt = 2;     // CTA-pair kernel: M-tiles per CTA (2: 512-feature tiles; 1: 256-feature tiles, double-buffered accumulators)
 };
 static GemmPlan plan_gemm(bool sparse, int T, int N, int K);
 
@@ -194,13 +195,13 @@ static int pick_pair_bn(bool sparse, int T, int N, int K) {
     return best;
 }
 
-template <bool SPARSE>
+template <bool SPARSE, int MT>
 static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& te,
                               const PairParams& pp, cudaStream_t stream) {
-    using Cfg = PairConfig<SPARSE>;
-    auto kernel = bitlinear_gemm_pair_kernel<SPARSE>;
-    if (!ensure_dynamic_smem<bitlinear_gemm_pair_kernel<SPARSE>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
-    const int tiles = ((pp.g.N + 511) / 512) * ((pp.g.T + pp.bn - 1) / pp.bn);
+    using Cfg = PairConfig<SPARSE, MT>;
+    auto kernel = bitlinear_gemm_pair_kernel<SPARSE, MT>;
+    if (!ensure_dynamic_smem<bitlinear_gemm_pair_kernel<SPARSE, MT>>(Cfg::SMEM_BYTES)) return SBN_ERR_CUDA;
+    const int tiles = ((pp.g.N + 256 * MT - 1) / (256 * MT)) * ((pp.g.T + pp.bn - 1) / pp.bn);
     const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
     const cudaError_t err = launch_kernel(kernel, dim3(2 * pairs), dim3(kPairThreads), Cfg::SMEM_BYTES, stream, ta, tb, te, pp);
     ++g_launch_count;
@@ -209,8 +210,9 @@ static sbn_status launch_pair(const CUtensorMap& ta, const CUtensorMap& tb, cons
 
 // Which kernel, which token tile, whether to split K: a small model of the measured times (us).
 //   single-CTA kernel   F(bn) + waves * (K/128 / splits) * c(bn)  [+ split-K: 1 + 8e-6 per atomic]
-//                       F = 3.0 + 0.02 bn (prologue + last epilogue), c = 0.23 (bn <= 128) | 0.275 (256)
-//   CTA-pair kernel     4.3 + 0.02 bn + waves * K/128 * 0.31 + (waves - 1) * 2.5 (exposed drains)
+//                       F = 3.0 + 0.02 bn (prologue + last epilogue), c = 0.23 (bn = 64) | 0.27 (128) | 0.49 (256)
+//   CTA-pair kernel     4.3 + 0.02 bn + waves * (K/128 * 0.31 + 2.5 (exposed drain)); dense K-loop x 1.65;
+//                       with one M-tile per CTA: 4.3 + 0.02 bn + waves * K/128 * 0.205 (dense 0.29)
 // waves over 148 CTAs resp. 74 pairs.  Small problems are latency-bound and favour many small
 // single-CTA tiles; large ones favour the pair kernel's operand reuse.  K is split only when the
 // tiles cannot fill the machine and the int32 atomics cost less than the K-loop they save.
@@ -218,7 +220,11 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     GemmPlan best = {false, 64, 1, 0};
     const int kb = K / kBK;
     const int rows = N / kBM;
-    if (g_force_token_tile < 0) return GemmPlan{true, pick_pair_bn(sparse, T, N, K), 1, 0};
+    if (g_force_token_tile < 0) {                               // diagnostics: the pair kernel as told (split_k 1 = one M-tile per CTA)
+        GemmPlan g{true, pick_pair_bn(sparse, T, N, K), 1, 0};
+        g.mt = g_force_split_k == 1 ? 1 : 2;
+        return g;
+    }
     if (g_force_split_k < 0) {                                  // diagnostics: cluster split-K as told
         int S = -g_force_split_k;
         S = S >= 8 ? 8 : (S >= 4 ? 4 : (S == 3 ? 3 : 2));
@@ -265,7 +271,7 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
     for (int bn : bns) {
         if (bn > 64 && T <= bn / 2) continue;                   // a tile mostly beyond T
         const long tiles = static_cast<long>(rows) * ((T + bn - 1) / bn);
-        const double c = (bn == 256 ? 0.275 : 0.23) * mm;
+        const double c = (bn == 256 ? 0.49 : (bn == 128 ? 0.27 : 0.23)) * mm;   // per 128 columns and wave
         const double F = 3.0 + 0.02 * bn;
         const long waves = (tiles + kNumSMs - 1) / kNumSMs;
         consider(GemmPlan{false, bn, 1, 0}, F + waves * kb * c);
@@ -285,7 +291,29 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
         const int bn = pick_pair_bn(sparse, T, N, K);
         const long tiles = static_cast<long>((N + 511) / 512) * ((T + bn - 1) / bn);
         const long waves = (tiles + kNumSMs / 2 - 1) / (kNumSMs / 2);
-        consider(GemmPlan{true, bn, 1, 0}, 4.3 + 0.02 * bn + waves * kb * 0.31 * (sparse ? 1.0 : 1.4) + (waves - 1) * 2.5);
+        consider(GemmPlan{true, bn, 1, 0}, 4.3 + 0.02 * bn + waves * kb * 0.31 * (sparse ? 1.0 : 1.65) + waves * 2.5);
+    }
+    {
+        // One M-tile per CTA: 256-feature tiles with double-buffered accumulators.  A tile costs the same
+        // whatever its token width (the MMAs' pace does not depend on it), so: fewest waves over the 74
+        // pairs, then least token padding, then the widest tile.  Per 128 columns 0.205 us (sparse) /
+        // 0.29 us (dense) against 0.31 / 0.43 for twice the features with two M-tiles, and no exposed
+        // drain: wins for short K and for the dense kernel, loses for the sparse one at K >= 4096.
+        const int cap = sparse ? kPairMaxBnSparse : kPairMaxBnDense;
+        const long rows1 = (N + 255) / 256;
+        int best_bn = 0;
+        long best_waves = 0, best_cover = 0;
+        for (int bn = cap; bn >= 128; bn -= 16) {
+            const long tt = (T + bn - 1) / bn;
+            const long waves = (rows1 * tt + kNumSMs / 2 - 1) / (kNumSMs / 2);
+            const long cover = tt * bn;
+            if (best_bn == 0 || waves < best_waves || (waves == best_waves && cover < best_cover)) {
+                best_bn = bn; best_waves = waves; best_cover = cover;
+            }
+        }
+        GemmPlan g{true, best_bn, 1, 0};
+        g.mt = 1;
+        consider(g, 4.3 + 0.02 * best_bn + best_waves * kb * (sparse ? 0.205 : 0.29));
     }
     return best;
 }
@@ -293,17 +321,17 @@ static GemmPlan plan_gemm(bool sparse, int T, int N, int K) {
 static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_scale, int T,
                                 const int8_t* wvals, const uint8_t* meta, const float* w_scale,
                                 int N, int K, const float* bias, void* y, sbn_out_dtype dt,
-                                int32_t* acc_out, int bn, cudaStream_t stream) {
+                                int32_t* acc_out, int bn, int mt, cudaStream_t stream) {
     CUtensorMap ta, tb, te;
     bool ok;
     const uint64_t KBk = static_cast<uint64_t>(K) / kBK, NB = static_cast<uint64_t>(N) / kBM;
     if (sparse) {
         constexpr int kbs = PairConfig<true>::KBS;
-        ok = encode_3d_1k(&ta, wvals, KBk * 8, NB, 8 * kbs, 2) && encode_3d_1k(&te, meta, KBk * 2, NB, 2 * kbs, 2) &&
+        ok = encode_3d_1k(&ta, wvals, KBk * 8, NB, 8 * kbs, mt) && encode_3d_1k(&te, meta, KBk * 2, NB, 2 * kbs, mt) &&
              encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
     } else {
         constexpr int kbs = PairConfig<false>::KBS;
-        ok = encode_3d_1k(&ta, wvals, KBk * 16, NB, 16 * kbs, 2) && encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
+        ok = encode_3d_1k(&ta, wvals, KBk * 16, NB, 16 * kbs, mt) && encode_3d_1k(&tb, xq, xq_tb8(T), KBk, bn / 16, kbs);
         te = ta;
     }
     if (!ok) return SBN_ERR_CUDA;
@@ -318,7 +346,8 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.g.w_vals = wvals; pp.g.w_meta = sparse ? meta : nullptr; pp.g.w_tile_bytes = sparse ? 8192 : 16384;
     pp.bn = bn;
-    return sparse ? launch_pair<true>(ta, tb, te, pp, stream) : launch_pair<false>(ta, tb, te, pp, stream);
+    if (mt == 1) return sparse ? launch_pair<true, 1>(ta, tb, te, pp, stream) : launch_pair<false, 1>(ta, tb, te, pp, stream);
+    return sparse ? launch_pair<true, 2>(ta, tb, te, pp, stream) : launch_pair<false, 2>(ta, tb, te, pp, stream);
 }
 
 template <bool SPARSE, int BN>
@@ -348,7 +377,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
 
     const GemmPlan plan = plan_gemm(sparse, T, N, K);
     if (plan.pair)
-        return run_gemm_pair(sparse, xq, a_scale, T, wvals, meta, w_scale, N, K, bias, y, dt, acc_out, plan.bn, stream);
+        return run_gemm_pair(sparse, xq, a_scale, T, wvals, meta, w_scale, N, K, bias, y, dt, acc_out, plan.bn, plan.mt, stream);
 
     const int bn = plan.bn;
     const int splits = plan.splits;
@@ -811,7 +840,7 @@ void sbn_plan_gemm(int sparse, int T, int N, int K, int* out4) {
     out4[0] = out4[1] = out4[2] = out4[3] = 0;
     if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return;
     const GemmPlan g = plan_gemm(sparse != 0, T, N, K);
-    out4[0] = g.pair ? 2 : (g.cluster > 1 ? 1 : 0);
+    out4[0] = g.pair ? (g.mt == 1 ? 3 : 2) : (g.cluster > 1 ? 1 : 0);
     out4[1] = g.bn;
     out4[2] = g.splits;
     out4[3] = g.cluster;

@@ -158,8 +158,8 @@ def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
 def test_dispatch_plan_is_sane(L):
     # host-only: the dispatcher's choices for the shapes the benchmarks use (kernel, tile, split, cluster)
     from paper_2603_05168_b200 import binding as b
-    assert b.sbn_plan_gemm(True, 4096, 3840, 2560)[0] == 2            # large T: the CTA-pair kernel
-    assert b.sbn_plan_gemm(True, 8192, 4096, 11008)[0] == 2
+    assert b.sbn_plan_gemm(True, 4096, 3840, 2560)[0] == 3            # large T, short K: CTA pairs, 256-feature tiles
+    assert b.sbn_plan_gemm(True, 8192, 4096, 11008)[0] == 2           # large T, long K: CTA pairs, 512-feature tiles
     k, bn, split, cluster = b.sbn_plan_gemm(True, 16, 3840, 2560)     # few tokens: cluster split-K, 32-token tile
     assert (k, bn, split) == (1, 32, 1) and cluster in (2, 3, 4)
     for T in (1, 16, 32):

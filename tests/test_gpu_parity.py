@@ -587,11 +587,12 @@ PAIR_CASES = [  # (T, N, K, BN): CTA-pair kernel, forced tile widths incl. ragge
 ]
 
 
+@pytest.mark.parametrize("mt", [2, 1])          # M-tiles per CTA: 512- or 256-feature pair tiles (the latter double-buffered)
 @pytest.mark.parametrize("sparse", [True, False])
 @pytest.mark.parametrize("T,N,K,bn", PAIR_CASES)
-def test_gemm_parity_pair_kernel(sparse, T, N, K, bn):
+def test_gemm_parity_pair_kernel(sparse, T, N, K, bn, mt):
     r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=bn + T)
-    b.sbn_set_gemm_tuning(-bn, 0)
+    b.sbn_set_gemm_tuning(-bn, 1 if mt == 1 else 0)
     if sparse:
         y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
     else:
