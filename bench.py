@@ -37,7 +37,7 @@ NOMINAL_BF16_DENSE_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the sparse GEMM per launch, from one ncu capture of
 # this bench's step (mean over the step's GEMM launches; the outputs mostly stay in L2, so this is far
 # below the algorithmic operand + output bytes -- the kernel is tensor-bound, the figure is context).
-GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 25.2e6, "down7b": 215.9e6}
+GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 24.3e6, "down7b": 215.9e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -442,7 +442,7 @@ def run_ours(args):
         ratio = DATASHEET_INT8_SPARSE_TOPS / NOMINAL_BF16_DENSE_TFLOPS
         peak = peaks["bf16_tflops"] * ratio
         achieved = sum(L.ops for L in layers) / (tot[dominant] * 1e-6) / 1e12
-        roofline = {"bound": "tensor", "kernel": "bitlinear_gemm_pair_kernel<sparse>", "achieved": round(achieved, 1),
+        roofline = {"bound": "tensor", "kernel": "bitlinear_gemm_pair_kernel<sparse, 1>" if args.workload == "2b" else "bitlinear_gemm_pair_kernel<sparse, 2>", "achieved": round(achieved, 1),
                     "peak": round(peak, 1), "unit": "TOP/s", "frac": round(achieved / peak, 4),
                     "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(args.workload),
                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {ratio:g} (nominal sparse-int8 : bf16)",

@@ -29,6 +29,13 @@
 //                  acc_full     every CTA's own copy, commit multicast
 //                  acc_empty    leader's copy: 32 arrivals (16 epilogue warps x 2 CTAs)
 //
+// The same kernel with ONE M-tile per CTA (template parameter MT = 1): the pair tile is 256 features
+// wide (CTA r owns row block 2*mt + r), the two 256-column halves of tensor memory alternate as
+// accumulators of consecutive tiles (acc_full / acc_empty exist once per half), and all 16 epilogue
+// warps drain the one M-tile (four per TMEM lane quarter, chunks c and c + 4) -- so the drain of a
+// tile runs under the MMAs of the next one.  It gives up half of the activation reuse; the
+// dispatcher uses it for short K and for the dense kernel (see PairConfig).
+//
 // No TMA multicast is used: every CTA fetches its own boxes.  All waits are bounded.
 #pragma once
 
