@@ -116,7 +116,19 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K);
  *              rate r_t = ||m(w_t) - m(w_{t-1})||_1 / D (Sec. 4); overwritten, not accumulated
  *   ws         device workspace of sbn_workspace_bytes(SBN_OP_QUANTIZE_MASK_PACK, 0, N, K)
  *              bytes; contents need no initialisation; must not be shared by calls that may run
- *              concurrently
+ *              concurrently.  It holds the per-CTA partial sums of |W| and a generation word that
+ *              the kernel advances on every execution, so a call captured in a CUDA graph may be
+ *              replayed on the same workspace (each replay tells its own partial sums from the
+ *              previous replay's)
+ * Residency rule (this call, the _bf16, _batched and _static_ws forms alike).  The kernel is one
+ * persistent grid of at most one CTA per SM (1024 threads each) whose CTAs exchange their partial
+ * sums through the workspace, so ALL of its CTAs must be resident at the same time.  On a GPU that
+ * runs nothing else that is always so.  Two such calls that may overlap on the GPU (different
+ * streams, no ordering between them) can each occupy part of the SMs and then wait for CTAs that
+ * cannot start; neither hangs -- every wait is bounded -- but both can end with SBN_ERR_TIMEOUT
+ * from sbn_check_status and unfinished outputs.  Order such calls (one stream, or events), or
+ * give all matrices to one sbn_quantize_mask_pack_batched call.  The same holds next to any other
+ * kernel that keeps SMs fully occupied for seconds.
  */
 sbn_status sbn_quantize_mask_pack(const float *W, int N, int K, int n_keep, int m_group,
                                   int8_t *vals, uint8_t *meta, float *w_scale, int8_t *dense_q,
@@ -159,8 +171,11 @@ sbn_status sbn_quantize_mask_pack_bf16(const void *W_bf16, int N, int K, int n_k
  * every BitLinear at every step (Sec. 2.3, "Dynamic Mask Recomputation"; Algorithm 1).  Each job
  * is exactly one sbn_quantize_mask_pack call (same arguments, same results, bit for bit); the
  * kernel pipelines the jobs so that launch and exchange latencies are paid once per batch.
- *   jobs   host array of `count` jobs (read before the call returns)
- *   ws     device workspace of sbn_batch_workspace_bytes(count) bytes; no initialisation needed
+ *   jobs   host array of `count` jobs; fully read before the call returns (pageable memory is
+ *          fine: the jobs travel to the device as kernel arguments, 48 per small launch, not through
+ *          a staging copy, so the call only enqueues and never blocks on the stream)
+ *   ws     device workspace of sbn_batch_workspace_bytes(count) bytes; no initialisation needed;
+ *          not to be shared by calls that may run concurrently
  */
 typedef struct {
     const void *W;                    /* device, [N][K], fp32 or (w_bf16 != 0) bf16 */
@@ -192,13 +207,17 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job *jobs, v
  * Arguments are those of sbn_quantize_mask_pack without ws/ws_bytes; inputs and outputs are
  * still the caller's buffers, and the results are bit-identical to that call's.
  * Limits and rules
+ *   - 2:4 only: n_keep = 2, m_group = 4; the 6:8 pattern returns SBN_ERR_UNSUPPORTED here.
  *   - N*K must not exceed SBN_STATIC_MAX_ELEMS, and the scratch the shape needs must fit in
  *     SBN_STATIC_SCRATCH_BYTES; otherwise SBN_ERR_TOO_LARGE is returned and nothing is launched.
  *   - The call itself never allocates or frees memory (no cudaMalloc/cudaFree, no allocating
  *     library routine).
  *   - The first call on each device looks up the device address of the built-in array (once per
- *     device, with that device current).  Make that first call before starting any stream
- *     capture on the device.
+ *     device, with that device current).  If nothing of this library has run on the device yet,
+ *     that lookup is also when the CUDA runtime loads the library's device code, which reserves
+ *     memory for the image (the built-in array included): it is the calls after the first that
+ *     are allocation-free.  Make that first call before starting any stream capture on the
+ *     device.
  *   - All calls on one device share the one array, and it keeps whatever the last call left in
  *     it (each call overwrites every slot it later reads, so nothing needs clearing).  Two such
  *     calls that may overlap on the GPU -- different streams, no ordering between them -- race
@@ -342,6 +361,27 @@ sbn_status sbn_layer_forward_host(const void *x_bf16_host, int T, int K,
                                   void *y_dev, void *y_host, sbn_out_dtype dt,
                                   void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * The compressed weights between the library's tiled storage order and the plain row-major arrays
+ * of the layout definition at the top of this file (Sec. 2.2 asks for "a well-defined N:M
+ * metadata/layout"; vals [N][K/2] and meta [N][K/8] as defined there are that layout, the tiled order
+ * is how this library keeps them in memory for its GEMM).  Pure permutations, device to device:
+ *   sbn_unpack_canonical   tiled vals / meta (outputs of sbn_quantize_mask_pack) -> plain arrays, for
+ *                          storing, inspecting or exporting packed weights
+ *   sbn_tile_canonical     plain arrays -> tiled order, for loading packed weights produced elsewhere
+ *                          (values must be -1, 0, +1 and every metadata nibble one of 4, 8, 9, 12, 13,
+ *                          14 -- not checked)
+ *   N, K       as for the pack call (for the 6:8 form pass K' = sbn_expanded_k(K, 6, 8))
+ *   vals / meta pairs: either pair may be NULL (both pointers) to convert only the other one
+ * Source and destination must be different buffers (SBN_ERR_UNSUPPORTED otherwise), 16-byte aligned.
+ * Asynchronous on `stream`.  sbn_tile_canonical writes weights: like every weight producer it gives
+ * the kernels behind it no early start.
+ */
+sbn_status sbn_unpack_canonical(const int8_t *vals, const uint8_t *meta, int N, int K,
+                                int8_t *vals_out, uint8_t *meta_out, void *stream);
+sbn_status sbn_tile_canonical(const int8_t *vals_plain, const uint8_t *meta_plain, int N, int K,
+                              int8_t *vals, uint8_t *meta, void *stream);
+
 /* Synchronises `stream`, returns SBN_ERR_TIMEOUT if any kernel since the last call gave up on a
  * bounded wait (and clears that record), SBN_ERR_CUDA if the stream reports an error, else
  * SBN_OK. */
@@ -359,6 +399,15 @@ const char *sbn_status_string(sbn_status s);
  * cluster size of sbn_sparse_bitlinear_packed and of the sbn_quant_act_*bitlinear kernels).  Results do not depend on
  * it. */
 void sbn_set_gemm_tuning(int token_tile, int split_k);
+
+/* Diagnostic for tests of the failure path (host state, not thread-safe; acts on the current device).
+ * wait_limit_us: limit of every bounded device-side wait from now on, in microseconds (0 = back to
+ * the default of 2 s).  break_waits != 0: the GEMM kernels' load producers issue no loads and the last
+ * CTA of the pack kernel does not publish its partial sum, so the waits of the other roles run out:
+ * every role then leaves through the kernel's abort path, the kernel returns (nothing traps, nothing
+ * waits without limit), outputs are unspecified and the next sbn_check_status reports
+ * SBN_ERR_TIMEOUT.  sbn_set_wait_test(0, 0) restores normal operation. */
+sbn_status sbn_set_wait_test(int break_waits, unsigned long long wait_limit_us);
 
 /* Diagnostic: what the dispatcher would run for this shape (host only, launches nothing).
  * out4[0] = kernel (0 single-CTA tiles, 1 cluster split-K, 2 CTA pair with 512-feature tiles, 3 CTA

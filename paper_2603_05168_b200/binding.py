@@ -24,7 +24,8 @@ EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
     "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed", "sbn_quant_act_sparse_bitlinear", "sbn_quant_act_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
-    "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count",
+    "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count", "sbn_unpack_canonical", "sbn_tile_canonical",
+    "sbn_set_wait_test",
 ]
 
 _lib = None
@@ -92,6 +93,12 @@ def lib() -> ctypes.CDLL:
         L.sbn_set_gemm_tuning.argtypes = [i32, i32]
         L.sbn_plan_gemm.restype = None
         L.sbn_plan_gemm.argtypes = [i32, i32, i32, i32, vp]
+        L.sbn_unpack_canonical.restype = i32
+        L.sbn_unpack_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.sbn_tile_canonical.restype = i32
+        L.sbn_tile_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.sbn_set_wait_test.restype = i32
+        L.sbn_set_wait_test.argtypes = [i32, ctypes.c_ulonglong]
         L.sbn_launch_count.restype = ctypes.c_ulonglong
         L.sbn_launch_count.argtypes = []
         _lib = L
@@ -275,6 +282,22 @@ def sbn_layer_forward_host(x_host, x_dev, xq_dev, a_scale_dev, w_scale, y_dev, y
                                         _ptr(vals), _ptr(meta), _ptr(dense_q), _ptr(w_scale), N,
                                         _ptr(bias), _ptr(y_dev), _ptr(y_host), dt, wp, wb, _stream()),
            "sbn_layer_forward_host")
+
+
+def sbn_unpack_canonical(vals, meta, N: int, K: int, vals_out, meta_out):
+    """Tiled vals / meta -> plain row-major [N][K/2] / [N][K/8] (either pair may be None)."""
+    _check(lib().sbn_unpack_canonical(_ptr(vals), _ptr(meta), N, K, _ptr(vals_out), _ptr(meta_out), _stream()),
+           "sbn_unpack_canonical")
+
+
+def sbn_tile_canonical(vals_plain, meta_plain, N: int, K: int, vals, meta):
+    """Plain row-major vals / meta -> the library's tiled order (either pair may be None)."""
+    _check(lib().sbn_tile_canonical(_ptr(vals_plain), _ptr(meta_plain), N, K, _ptr(vals), _ptr(meta), _stream()),
+           "sbn_tile_canonical")
+
+
+def sbn_set_wait_test(break_waits: bool = False, wait_limit_us: int = 0):
+    _check(lib().sbn_set_wait_test(1 if break_waits else 0, int(wait_limit_us)), "sbn_set_wait_test")
 
 
 def sbn_check_status():

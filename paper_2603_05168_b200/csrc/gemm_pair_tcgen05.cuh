@@ -368,7 +368,7 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (lane == 0 && !p.test_skip_loads) {
             tma_prefetch_desc(&tmap_a);
             tma_prefetch_desc(&tmap_b);
             if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);

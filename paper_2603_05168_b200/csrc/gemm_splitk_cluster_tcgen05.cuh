@@ -202,7 +202,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
     bool ok = true;
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (lane == 0 && !p.test_skip_loads) {
             int stage = 0;
             uint32_t phase = 0;
             for (int kb = kb0; kb < kb1; ++kb) {

@@ -42,7 +42,6 @@ constexpr int kEpiWarpBufBytes = 32 * 32 * 4;                 // one 32-token x 
 constexpr int kEpiBytes = 4 * 2 * kEpiWarpBufBytes;           // 4 epilogue warps, double buffered
 constexpr int kScaleBytes = 4 * 256 * 4;                      // per-token scales, one copy per epilogue warp
 constexpr int kBarrierBytes = 256;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
 struct GemmParams {
     int T, N, K;
@@ -60,6 +59,8 @@ struct GemmParams {
     const void* w_vals;          // the weight operand (compressed values, or the dense W_q) and its metadata
     const void* w_meta;          //   (null for dense): only used to warm the L2 before the dependency wait
     int w_tile_bytes;            // bytes of one 128 x 128 weight tile (8192 sparse, 16384 dense)
+    int test_skip_loads = 0;     // diagnostics (sbn_set_wait_test): the TMA producer issues no loads, so the
+                                 //   consumers' bounded waits run out and every role leaves through the abort flag
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -101,7 +102,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3FFu) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) {
                 *abort_flag = 1;
                 atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
                 return false;
@@ -289,7 +290,7 @@ bitlinear_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        if (lane == 0 && !p.test_skip_loads) {
             tma_prefetch_desc(&tmap_a);
             tma_prefetch_desc(&tmap_b);
             if constexpr (SPARSE) tma_prefetch_desc(&tmap_e);

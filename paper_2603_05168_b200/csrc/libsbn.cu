@@ -15,6 +15,7 @@
 #include "norm_quant_act.cuh"
 #include "quantize_mask_pack.cuh"
 #include "quantize_mask_pack68.cuh"
+#include "canonical_layout.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_pair_tcgen05.cuh"
 #include "gemm_splitk_cluster_tcgen05.cuh"
@@ -345,6 +346,7 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.acc_out = acc_out;
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.g.w_vals = wvals; pp.g.w_meta = sparse ? meta : nullptr; pp.g.w_tile_bytes = sparse ? 8192 : 16384;
+    pp.g.test_skip_loads = g_test_break_waits;
     pp.bn = bn;
     if (mt == 1) return sparse ? launch_pair<true, 1>(ta, tb, te, pp, stream) : launch_pair<false, 1>(ta, tb, te, pp, stream);
     return sparse ? launch_pair<true, 2>(ta, tb, te, pp, stream) : launch_pair<false, 2>(ta, tb, te, pp, stream);
@@ -412,6 +414,7 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     p.split_acc = splits > 1 ? static_cast<int32_t*>(ws) : nullptr;
     p.split_counters = splits > 1 ? reinterpret_cast<unsigned int*>(static_cast<char*>(ws) + split_acc_bytes(T, N)) : nullptr;
     p.w_vals = wvals; p.w_meta = sparse ? meta : nullptr; p.w_tile_bytes = sparse ? 8192 : 16384;
+    p.test_skip_loads = g_test_break_waits;
 
     if (plan.cluster > 1) {
         p.k_splits = 1;
@@ -505,7 +508,7 @@ static sbn_status quantize_mask_pack_any(const void* W, bool w_bf16, int N, int 
     if (p68) {
         const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, nullptr, prev_meta, flip_bits);
         return launch_quantize_mask_pack_batch<68>(d, nullptr, 1, d.num_units, static_cast<QmpWorkspace*>(ws)->slot,
-                                                   static_cast<cudaStream_t>(stream));
+                                                   &static_cast<QmpWorkspace*>(ws)->generation, static_cast<cudaStream_t>(stream));
     }
     return launch_quantize_mask_pack(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits,
                                      static_cast<QmpWorkspace*>(ws),
@@ -528,10 +531,13 @@ sbn_status sbn_quantize_mask_pack_bf16(const void* W_bf16, int N, int K, int n_k
                                   ws, ws_bytes, stream);
 }
 
+// Batch workspace: [generation word, 256 B][job descriptors 1.., padded to 256 B][count x 148 slots].
+static size_t batch_desc_bytes(int count) {
+    return (static_cast<size_t>(count) * sizeof(QmpDesc) + 255) & ~static_cast<size_t>(255);
+}
 size_t sbn_batch_workspace_bytes(int count) {
     if (count <= 0) return 0;
-    const size_t descs = (static_cast<size_t>(count) * sizeof(QmpDesc) + 255) & ~static_cast<size_t>(255);
-    return descs + static_cast<size_t>(count) * sizeof(QmpWorkspace);
+    return 256 + batch_desc_bytes(count) + static_cast<size_t>(count) * sizeof(QmpWorkspace);
 }
 
 sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, void* ws, size_t ws_bytes,
@@ -555,17 +561,22 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
         max_units = std::max(max_units, descs[i].num_units);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t desc_bytes = (static_cast<size_t>(count) * sizeof(QmpDesc) + 255) & ~static_cast<size_t>(255);
-    QmpDesc* rest_dev = static_cast<QmpDesc*>(ws);
-    if (count > 1) {
-        // jobs 1.. are read by the kernel from the workspace (job 0 travels as a kernel argument);
-        // the source vector is pageable, so the runtime stages it before this call returns
-        if (cudaMemcpyAsync(rest_dev, descs.data() + 1, static_cast<size_t>(count - 1) * sizeof(QmpDesc),
-                            cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return SBN_ERR_CUDA;
+    unsigned long long* generation = static_cast<unsigned long long*>(ws);
+    QmpDesc* rest_dev = reinterpret_cast<QmpDesc*>(static_cast<char*>(ws) + 256);
+    // Jobs 1.. are read by the kernel from the workspace (job 0 travels as a kernel argument).  They get
+    // there as arguments of small store kernels, a chunk at a time: nothing is staged through host
+    // memory, so the call only enqueues and the caller's array is free as soon as it returns.
+    for (int at = 1; at < count; at += kQmpDescChunk) {
+        QmpDescChunk chunk;
+        const int n = std::min(kQmpDescChunk, count - at);
+        for (int i = 0; i < n; ++i) chunk.d[i] = descs[static_cast<size_t>(at + i)];
+        for (int i = n; i < kQmpDescChunk; ++i) chunk.d[i] = descs[0];
+        const cudaError_t err = launch_kernel(qmp_store_descs_kernel, dim3(1), dim3(64), 0, s, chunk, rest_dev + (at - 1), n);
+        ++g_launch_count;
+        if (err != cudaSuccess) return SBN_ERR_CUDA;
     }
-    QmpSlot* slots = reinterpret_cast<QmpSlot*>(static_cast<char*>(ws) + desc_bytes);
-    return launch_quantize_mask_pack_batch(descs[0], rest_dev, count, max_units, slots, s);
+    QmpSlot* slots = reinterpret_cast<QmpSlot*>(static_cast<char*>(ws) + 256 + batch_desc_bytes(count));
+    return launch_quantize_mask_pack_batch(descs[0], rest_dev, count, max_units, slots, generation, s);
 }
 
 sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_keep, int m_group,
@@ -808,6 +819,28 @@ sbn_status sbn_sparse_bitlinear_packed(const int8_t* xq, const float* a_scale, i
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
 
+static sbn_status canonical_any(bool to_tiled, const void* vals_in, const void* meta_in, int N, int K, void* vals_out,
+                                void* meta_out, void* stream) {
+    if ((!vals_in) != (!vals_out) || (!meta_in) != (!meta_out) || (!vals_in && !meta_in)) return SBN_ERR_NULL;
+    if (N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    if (misaligned(vals_in, 16) || misaligned(vals_out, 16) || misaligned(meta_in, 16) || misaligned(meta_out, 16))
+        return SBN_ERR_ALIGN;
+    if ((vals_in && vals_in == vals_out) || (meta_in && meta_in == meta_out)) return SBN_ERR_UNSUPPORTED;   // not in place
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return to_tiled ? launch_canonical_layout<true>(vals_in, vals_out, meta_in, meta_out, N, K, s)
+                    : launch_canonical_layout<false>(vals_in, vals_out, meta_in, meta_out, N, K, s);
+}
+
+sbn_status sbn_unpack_canonical(const int8_t* vals, const uint8_t* meta, int N, int K, int8_t* vals_out,
+                                uint8_t* meta_out, void* stream) {
+    return canonical_any(false, vals, meta, N, K, vals_out, meta_out, stream);
+}
+
+sbn_status sbn_tile_canonical(const int8_t* vals_plain, const uint8_t* meta_plain, int N, int K, int8_t* vals,
+                              uint8_t* meta, void* stream) {
+    return canonical_any(true, vals_plain, meta_plain, N, K, vals, meta, stream);
+}
+
 sbn_status sbn_check_status(void* stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SBN_ERR_CUDA;
     int h = 0;
@@ -844,6 +877,13 @@ void sbn_plan_gemm(int sparse, int T, int N, int K, int* out4) {
     out4[1] = g.bn;
     out4[2] = g.splits;
     out4[3] = g.cluster;
+}
+
+sbn_status sbn_set_wait_test(int break_waits, unsigned long long wait_limit_us) {
+    const unsigned long long ns = wait_limit_us == 0ull ? kWaitLimitNs : wait_limit_us * 1000ull;
+    if (cudaMemcpyToSymbol(g_wait_limit_ns, &ns, sizeof(ns)) != cudaSuccess) return SBN_ERR_CUDA;
+    g_test_break_waits = break_waits ? 1 : 0;
+    return SBN_OK;
 }
 
 void sbn_set_gemm_tuning(int token_tile, int split_k) {

@@ -16,10 +16,13 @@
 //            PROVISIONALLY: |w| >= thr_hi -> +-1 and |w| < thr_lo -> 0 are final whatever gamma
 //            turns out to be inside the bracket; the others (~2 % for Gaussian weights) are
 //            appended as {byte position, w} to a list in shared memory;
-//   exchange every CTA publishes {call nonce, partial sum} in the workspace and waits (bounded)
-//            until all slots carry this call's nonce -- no atomics, no counter, nothing to
-//            initialise, stale slots of earlier calls can never match; every CTA then adds the
-//            148 partials in the same fixed order, so all get the same bits, run after run;
+//   exchange every CTA publishes {tag, partial sum} in the workspace and waits (bounded) until all
+//            slots carry this execution's tag -- no atomics, nothing to initialise; every CTA then
+//            adds the 148 partials in the same fixed order, so all get the same bits, run after
+//            run.  The tag joins the host's per-call nonce with a generation word that lives in
+//            the workspace and that CTA 0 advances at the end of every execution: stale slots of
+//            earlier calls never match, and neither do those of an earlier REPLAY of the same
+//            captured launch (whose nonce is frozen in the graph);
 //   fix-up   with the exact thr: if thr_lo <= thr <= thr_hi (and the list did not overflow) only
 //            the listed bytes are rewritten -- the result is exactly Eq. 1, not an approximation.
 //            Otherwise (a sample that misrepresents the matrix, the 1e-5 clamp, a request for the
@@ -62,15 +65,20 @@ __host__ __device__ inline uint32_t qmp_sample_units(uint32_t num_units) {
     const uint32_t want = num_units < kQmpSmallMatrixUnits ? kQmpSampleUnitsSmall : kQmpSampleUnits;
     return num_units < want ? num_units : want;
 }
-constexpr unsigned long long kQmpWaitLimitNs = 2000000000ull;
 
 struct QmpSlot {                 // one per CTA, 16 B
-    unsigned long long nonce;    // identifies the call that wrote `partial`
+    unsigned long long nonce;    // tag of the execution that wrote `partial`
     double partial;              // this CTA's sum |W|
 };
 struct QmpWorkspace {            // layout of the caller's workspace
     QmpSlot slot[kQmpMaxCtas];
+    unsigned long long generation;   // advanced by one per execution on this workspace (any start value)
+    unsigned long long pad_;
 };
+// Tag of one execution: the call's nonce (low word, never 0) under the workspace's generation.
+__device__ __forceinline__ unsigned long long qmp_tag(unsigned long long nonce, unsigned long long generation) {
+    return (generation << 32) | (nonce & 0xFFFFFFFFull);
+}
 
 __device__ __forceinline__ unsigned long long global_timer_ns_qmp() {
     unsigned long long t;
@@ -383,7 +391,8 @@ __device__ __forceinline__ double qmp68_pass(const QmpDesc& d, const QmpRange rg
 template <int PATTERN>
 __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
-                          QmpSlot* slots, unsigned long long nonce) {
+                          QmpSlot* slots, unsigned long long* generation, unsigned long long call_nonce,
+                          int test_withhold_slot) {
     extern __shared__ QmpEntry s_list[];                // [2][kQmpListCap]
     __shared__ double s_warp[kQmpWarps];
     __shared__ float s_thr;
@@ -400,6 +409,10 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
     // No early signal to the next kernel of the stream: this kernel writes packed weights, and the
     // GEMM kernels fetch weights before their own dependency wait (see sbn_common.cuh).
     pdl_wait();
+    // stable for the whole execution: CTA 0 advances it only after it has seen every CTA's last slot,
+    // and every CTA reads it here, before it publishes anything
+    const unsigned long long gen0 = *reinterpret_cast<volatile unsigned long long*>(generation);
+    const unsigned long long nonce = qmp_tag(call_nonce, gen0);
 
     QmpDesc d_prev = first;
     QmpRange rg_prev = {0u, 0u};
@@ -451,7 +464,10 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                 QmpSlot* sl = slots + static_cast<size_t>(m) * gridDim.x + blockIdx.x;
                 sl->partial = mine;
                 __threadfence();
-                *reinterpret_cast<volatile unsigned long long*>(&sl->nonce) = nonce;
+                // diagnostics (sbn_set_wait_test): the last CTA keeps its tag to itself, so every CTA's
+                // bounded wait for that slot runs out
+                if (!(test_withhold_slot && blockIdx.x == gridDim.x - 1))
+                    *reinterpret_cast<volatile unsigned long long*>(&sl->nonce) = nonce;
             }
             __syncthreads();
         }
@@ -467,7 +483,8 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                 bool seen = (*flag == nonce);
                 while (!seen) {
                     seen = (*flag == nonce);
-                    if (!seen && ((++spins & 0xFFu) == 0) && global_timer_ns_qmp() - t0 > kQmpWaitLimitNs) break;
+                    if (!seen && ((++spins & 0xFFu) == 0) &&
+                        global_timer_ns_qmp() - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) break;
                 }
                 if (seen) {
                     __threadfence();
@@ -515,12 +532,29 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
         d_prev = d_cur;
         rg_prev = rg_cur;
     }
+    // every CTA has published its last slot (CTA 0 has just read them all), hence has read the generation
+    if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<volatile unsigned long long*>(generation) = gen0 + 1ull;
 }
 
-// Per-call nonce: unique within the process, never 0.
+// Copies up to kQmpDescChunk job descriptors, passed by value, into the batch workspace: the batched
+// call hands its jobs to the device without a host-side staging copy.
+constexpr int kQmpDescChunk = 48;
+struct QmpDescChunk {
+    QmpDesc d[kQmpDescChunk];
+};
+static_assert(sizeof(QmpDescChunk) <= 4000, "descriptor chunk must fit the kernel parameter space");
+__global__ void __launch_bounds__(64)
+qmp_store_descs_kernel(const QmpDescChunk chunk, QmpDesc* __restrict__ dst, int n) {
+    pdl_wait();                        // the previous user of the workspace has finished; no early start for successors
+    if (threadIdx.x < static_cast<unsigned>(n)) dst[threadIdx.x] = chunk.d[threadIdx.x];
+}
+
+// Per-call nonce: unique within the process, low 32 bits never 0.
 inline unsigned long long qmp_next_nonce() {
     static std::atomic<unsigned long long> counter{0x5B4E0000ull};
-    return counter.fetch_add(1) + 1;
+    unsigned long long n = counter.fetch_add(1) + 1;
+    if ((n & 0xFFFFFFFFull) == 0ull) n = counter.fetch_add(1) + 1;
+    return n;
 }
 
 inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* vals, uint8_t* meta, float* w_scale,
@@ -542,18 +576,21 @@ inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* v
 // Launch for `count` matrices: `first` by value, the others already copied to `rest_dev`.
 template <int PATTERN = 24>
 inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const QmpDesc* rest_dev, int count,
-                                                  uint32_t max_units, QmpSlot* slots, cudaStream_t stream) {
+                                                  uint32_t max_units, QmpSlot* slots, unsigned long long* generation,
+                                                  cudaStream_t stream) {
+    const int test_withhold_slot = g_test_break_waits;
     unsigned long long nonce = qmp_next_nonce();
     // every CTA must be resident at once (they exchange partial sums): never more CTAs than this
     // device has SMs, and never more than the workspace has slots
     const unsigned cap = static_cast<unsigned>(std::min(device_sm_count(), kQmpMaxCtas));
     const unsigned grid = max_units < cap ? max_units : cap;
+    static_assert(kQmpThreads >= kQmpMaxCtas, "one thread per slot in the exchange");
     if (!ensure_dynamic_smem<quantize_mask_pack_kernel<PATTERN>>(kQmpSmemBytes)) return SBN_ERR_CUDA;
     // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
     const cudaError_t err = launch_kernel(quantize_mask_pack_kernel<PATTERN>, dim3(grid), dim3(kQmpThreads), kQmpSmemBytes, stream,
-                                          first, rest_dev, count, slots, nonce);
+                                          first, rest_dev, count, slots, generation, nonce, test_withhold_slot);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -564,7 +601,7 @@ inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, i
                                             unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
     const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
-    return launch_quantize_mask_pack_batch(d, nullptr, 1, d.num_units, ws->slot, stream);
+    return launch_quantize_mask_pack_batch(d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream);
 }
 
 }  // namespace sbn

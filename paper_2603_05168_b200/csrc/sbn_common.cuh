@@ -18,6 +18,16 @@ constexpr float kEps = 1e-5f;         // Algorithm 2's clamp for both scales
 // ran out.  Read and cleared by sbn_check_status.
 __device__ int g_device_status = 0;
 
+// Limit of every bounded device-side wait, in ns (default 2 s).  Only the slow path of a wait reads it
+// (after the first polls have failed); sbn_set_wait_test shortens it so that a test can make a wait
+// run out without anything hanging.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+__device__ unsigned long long g_wait_limit_ns = kWaitLimitNs;
+
+// Host state of sbn_set_wait_test: non-zero makes the producers of the GEMM kernels issue no loads and
+// the last CTA of the pack kernel withhold its partial sum -- the consumers' waits then run out.
+static int g_test_break_waits = 0;
+
 // Host-side count of kernel launches made by the library.
 static std::atomic<unsigned long long> g_launch_count{0ull};
 

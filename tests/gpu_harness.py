@@ -203,6 +203,16 @@ def gpu_gemm(sparse: bool, xq, a_scale, packed_dev, out_dtype=torch.float32, bia
     return y, acc
 
 
+def gpu_unpack_canonical(packed_dev, N, K):
+    """The library's own un-tiling call: device vals / meta (tiled) -> plain [N][K/2] int8 and [N][K/8]
+    uint8 numpy arrays.  No numpy permutation involved."""
+    vals_out = torch.full((N, K // 2), 99, dtype=torch.int8, device="cuda")
+    meta_out = torch.full((N, K // 8), 0xEE, dtype=torch.uint8, device="cuda")
+    b.sbn_unpack_canonical(packed_dev["vals"], packed_dev["meta"], N, K, vals_out, meta_out)
+    b.sbn_check_status()
+    return vals_out.cpu().numpy(), meta_out.cpu().numpy()
+
+
 def gpu_pack_vals2(packed_dev):
     """Device buffers of alloc_packed -> (device vals2 buffer, plain uint8 [N][K/8])."""
     N, K = packed_dev["vals"].shape[0], 2 * packed_dev["vals"].shape[1]

@@ -186,3 +186,16 @@ def test_fused_entry_validation_on_host(L):
     assert fs(dt=9) == UNSUP
     assert fs(x=odd) == ALIGN
     assert L.sbn_quant_act_bitlinear(p, 8, None, p, 256, 512, None, p, 0, None, None, None) == NULL
+
+
+def test_canonical_layout_calls_validate_on_host(L):
+    p, q = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x2000)
+    odd = ctypes.c_void_p(0x1008)
+    NULL, SHAPE, ALIGN, UNSUP = 1, 2, 3, 4
+    for fn in (L.sbn_unpack_canonical, L.sbn_tile_canonical):
+        assert fn(None, None, 256, 256, None, None, None) == NULL          # nothing to convert
+        assert fn(p, None, 256, 256, None, None, None) == NULL             # a source without its destination
+        assert fn(p, p, 256, 100, q, q, None) == SHAPE
+        assert fn(p, p, 0, 256, q, q, None) == SHAPE
+        assert fn(odd, p, 256, 256, q, q, None) == ALIGN
+        assert fn(p, p, 256, 256, p, q, None) == UNSUP                     # in place

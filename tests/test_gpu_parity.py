@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 if torch.cuda.is_available():
     from gpu_harness import (gpu_norm_quant_act, bf16_dev, bf16_tensor_bits, dev, expand68_columns, fold68, gpu_gemm,
                              gpu_gemm_packed, gpu_pack_vals2, gpu_quant_act, gpu_quant_act_expand68, gpu_quantize_mask_pack,
-                             gpu_quantize_mask_pack68,
+                             gpu_quantize_mask_pack68, gpu_unpack_canonical, tile_meta, tile_vals,
                              xq_to_numpy, y_to_f32_numpy)
 
 
@@ -906,3 +906,125 @@ def test_packed_and_fused_kernels_every_cluster_size(T, N, K, cluster):
     b.sbn_check_status()
     assert np.array_equal(acc2.cpu().numpy(), acc_ref)
     assert torch.equal(y, y2)
+
+
+# ---- the plain (canonical) layout through the library's own conversion calls ---------------------------
+@pytest.mark.parametrize("N,K,seed", [(256, 256, 0), (128, 128, 110), (384, 2560, 111), (640, 6912, 112)])
+def test_unpack_canonical_against_oracle(N, K, seed):
+    # pack on the GPU, un-tile on the GPU, compare with the oracle's plain arrays: no permutation is
+    # restated on the test's side
+    W = inputs.latent_weights(N, K, seed=seed)
+    r = _oracle_pack(W)
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    vals, meta = gpu_unpack_canonical(g["dev"], N, K)
+    assert np.array_equal(vals, r["vals"])
+    assert np.array_equal(meta, r["meta"])
+
+
+def test_tile_canonical_round_trip_and_gemm():
+    # weights packed by the ORACLE, brought into the library's order by sbn_tile_canonical, then used by
+    # the GEMM: accumulators must be the oracle's; and tile -> unpack is the identity
+    T, N, K = 70, 384, 1280
+    W = inputs.latent_weights(N, K, seed=120)
+    bits = inputs.activations_bf16(T, K, seed=121)
+    r = _oracle_pack(W)
+    xq_ref, s_ref = oracle.quant_act(bits)
+    _, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    p = b.alloc_packed(N, K)
+    p["vals"].fill_(55)
+    p["meta"].fill_(0x55)
+    b.sbn_tile_canonical(dev(r["vals"]), dev(r["meta"]), N, K, p["vals"], p["meta"])
+    p["w_scale"].copy_(torch.tensor([r["scale"]], dtype=torch.float32))
+    assert np.array_equal(p["vals"].cpu().numpy().reshape(-1), tile_vals(r["vals"]))
+    assert np.array_equal(p["meta"].cpu().numpy().reshape(-1), tile_meta(r["meta"]))
+    vals, meta = gpu_unpack_canonical(p, N, K)
+    assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"])
+    xq, a_scale = gpu_quant_act(bits)
+    _, acc = gpu_gemm(True, xq, a_scale, p)
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    # one pair only
+    only_meta = torch.zeros((N, K // 8), dtype=torch.uint8, device="cuda")
+    b.sbn_unpack_canonical(None, p["meta"], N, K, None, only_meta)
+    b.sbn_check_status()
+    assert np.array_equal(only_meta.cpu().numpy(), r["meta"])
+
+
+# ---- a captured pack call replayed on changed weights ---------------------------------------------------
+def test_quantize_mask_pack_graph_replay_on_changed_weights():
+    # A launch captured in a CUDA graph carries the same host-side nonce at every replay; the slots
+    # of the previous replay must still not be taken for this replay's partial sums.  Replays on
+    # weights of very different scale: a stale partial sum would give a wrong gamma.
+    N, K = 2560, 2560
+    Ws = [inputs.latent_weights(N, K, seed=130 + i, sigma=0.02 * (3 ** i)) for i in range(3)]
+    refs = [_oracle_pack(W) for W in Ws]
+    Wd = dev(Ws[0])
+    p = b.alloc_packed(N, K)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        b.sbn_quantize_mask_pack(Wd, p["vals"], p["meta"], p["w_scale"], p["ws"])       # set-up outside the capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        b.sbn_quantize_mask_pack(Wd, p["vals"], p["meta"], p["w_scale"], p["ws"])
+    for rep in range(6):
+        i = rep % 3
+        Wd.copy_(torch.from_numpy(Ws[i]))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        b.sbn_check_status()
+        assert np.float32(p["w_scale"].cpu().numpy()[0]) == refs[i]["scale"], f"replay {rep}"
+        vals, meta = gpu_unpack_canonical(p, N, K)
+        assert np.array_equal(vals, refs[i]["vals"]), f"replay {rep}"
+        assert np.array_equal(meta, refs[i]["meta"]), f"replay {rep}"
+
+
+# ---- bounded waits that run out --------------------------------------------------------------------------
+WAIT_CASES = [("single_cta", 64, 256, 512, (128, 1)), ("pair", 300, 512, 512, (-128, 0)), ("pair_one_m_tile", 300, 256, 512, (-128, 1)),
+              ("cluster", 16, 256, 1280, (32, -4))]
+
+
+@pytest.mark.parametrize("sparse", [True, False])
+@pytest.mark.parametrize("name,T,N,K,tuning", WAIT_CASES)
+def test_gemm_wait_runs_out_and_the_library_recovers(name, T, N, K, tuning, sparse):
+    # The load producer is told to issue nothing and the wait limit is 1 ms: the MMA issuer's wait for
+    # the first stage runs out, it raises the CTA's abort flag, every role leaves its loop, tensor
+    # memory is freed, the kernel returns and the status word says SBN_ERR_TIMEOUT.  Nothing traps
+    # and nothing hangs.  The very next ordinary call must be right, bit for bit.
+    r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=140 + T)
+    if sparse:
+        _, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    else:
+        _, acc_ref = oracle.bitlinear(xq_ref, s_ref, r["dense_q"], r["scale"])
+    b.sbn_set_gemm_tuning(*tuning)
+    b.sbn_check_status()
+    try:
+        b.sbn_set_wait_test(True, 1000)
+        with pytest.raises(b.SbnError) as err:
+            gpu_gemm(sparse, xq, a_scale, g["dev"])
+        assert err.value.code == 7                            # SBN_ERR_TIMEOUT
+    finally:
+        b.sbn_set_wait_test(False, 0)
+    b.sbn_check_status()                                      # the record was cleared by the read above
+    _, acc = gpu_gemm(sparse, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+
+
+def test_pack_wait_runs_out_and_the_library_recovers():
+    # one CTA of the pack kernel withholds its partial sum: every CTA's bounded wait for that slot runs
+    # out, all of them return, the status word says SBN_ERR_TIMEOUT; the next call is exact
+    N, K = 512, 2560
+    W = inputs.latent_weights(N, K, seed=150)
+    r = _oracle_pack(W)
+    b.sbn_check_status()
+    try:
+        b.sbn_set_wait_test(True, 1000)
+        with pytest.raises(b.SbnError) as err:
+            gpu_quantize_mask_pack(W, with_dense=False)
+        assert err.value.code == 7
+    finally:
+        b.sbn_set_wait_test(False, 0)
+    b.sbn_check_status()
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    assert g["scale"] == r["scale"]
+    assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])

@@ -3,9 +3,11 @@
 It serves callers that cannot allocate device memory where they call the library (a framework
 that owns the whole GPU through its own pool, a plug-in hook that must not allocate, a loop that
 cannot afford cudaMalloc's device-wide synchronisation): its scratch is a fixed array inside the
-library.  The GPU test drives it through the C ABI, twice in a row on different shapes, and
-requires the very same bits as sbn_quantize_mask_pack with a caller-provided workspace -- the
-second call also shows that whatever the first one left in the shared array does no harm.
+library.  The GPU tests drive it through the C ABI, twice in a row on different shapes, and
+require the very same bits as sbn_quantize_mask_pack with a caller-provided workspace -- the
+second call also shows that whatever the first one left in the shared array does no harm -- and,
+for the routes the ordinary use takes (no dense copy of the weights: the single-pass kernel with its
+fix-up list; metadata updated in place with the flip count), the CPU oracle's bits as well.
 
 This file is named so that pytest collects it last.
 """
@@ -18,6 +20,8 @@ import torch
 from paper_2603_05168_b200 import binding as b
 from paper_2603_05168_b200 import build as sbn_build
 from paper_2603_05168_b200 import inputs
+
+import oracle
 
 
 def test_static_ws_rejects_oversized_problem_on_host():
@@ -72,3 +76,34 @@ def test_static_ws_matches_workspace_entry_point_twice_in_a_row():
     # and once more with the flip count enabled
     W3 = inputs.perturb_weights(W1, seed=33, sigma=1e-4)
     _run_both(W3, prev_meta_np=r1["meta"].cpu().numpy())      # r1's metadata is already in the library's order
+
+
+@pytest.mark.gpu
+def test_static_ws_single_pass_route_and_in_place_metadata_against_the_oracle():
+    # without the dense output the kernel takes its single-pass route (provisional values + fix-up
+    # list) -- the default and the fast one; with prev_meta == meta the metadata is updated in place
+    from gpu_harness import gpu_unpack_canonical, tile_meta
+    N, K = 1024, 2560
+    W0 = inputs.latent_weights(N, K, seed=34)
+    W1 = inputs.perturb_weights(W0, seed=35, sigma=1e-4)
+    r0, r1 = oracle.quantize_mask_pack(W0), oracle.quantize_mask_pack(W1)
+    if r0["near_tie"] or r1["near_tie"]:
+        pytest.skip("gamma within rounding distance of an fp32 midpoint for this seed")
+    for rep in range(2):                                      # two calls in a row on the shared scratch
+        got = b.alloc_packed(N, K)
+        ref = b.alloc_packed(N, K)
+        for bufs in (got, ref):
+            bufs["meta"].copy_(torch.from_numpy(tile_meta(r0["meta"]).reshape(N, K // 8)))
+            bufs["flips"] = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+        Wd = torch.from_numpy(W1).cuda()
+        b.sbn_quantize_mask_pack_static_ws(Wd, got["vals"], got["meta"], got["w_scale"], prev_meta=got["meta"],
+                                           flip_bits=got["flips"])
+        b.sbn_quantize_mask_pack(Wd, ref["vals"], ref["meta"], ref["w_scale"], ref["ws"], prev_meta=ref["meta"],
+                                 flip_bits=ref["flips"])
+        b.sbn_check_status()
+        for key in ("vals", "meta", "w_scale", "flips"):
+            assert torch.equal(ref[key], got[key]), key
+        vals, meta = gpu_unpack_canonical(got, N, K)
+        assert np.float32(got["w_scale"].cpu().numpy()[0]) == r1["scale"]
+        assert np.array_equal(vals, r1["vals"]) and np.array_equal(meta, r1["meta"])
+        assert int(got["flips"].item()) == oracle.flip_count(r0["mask"], r1["mask"])
