@@ -34,10 +34,10 @@ from paper_2603_05168_b200 import inputs  # noqa: E402
 DATASHEET_INT8_DENSE_TOPS = 4500.0
 DATASHEET_INT8_SPARSE_TOPS = 9000.0
 NOMINAL_BF16_DENSE_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the sparse GEMM per launch, from one ncu capture of
-# this bench's step (mean over the step's GEMM launches; the outputs mostly stay in L2, so this is far
-# below the algorithmic operand + output bytes -- the kernel is tensor-bound, the figure is context).
-GEMM_DRAM_BYTES_PER_LAUNCH = {"2b": 24.3e6, "down7b": 215.9e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of the sparse GEMM per launch come from the ncu captures
+# summarised under profiles/ (the outputs mostly stay in L2, so this is far below the algorithmic operand
+# + output bytes -- the kernel is tensor-bound, the figure is context).
+GEMM_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -61,6 +61,20 @@ def load_peaks():
                     source="measured")
     return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS,
                 bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def gemm_dram_traffic(workload):
+    """Measured DRAM bytes per sparse-GEMM launch of this workload's step (None if no capture is on file)."""
+    try:
+        with open(GEMM_TRAFFIC_FILE) as f:
+            return float(json.load(f)[workload]["bytes_per_launch"])
+    except (OSError, KeyError, ValueError):
+        return None
+
+
+def workload_string(name, T, shapes):
+    return (f"{name}: BitLinears at T={T}: " + ", ".join(f"{n} {K}->{N}" for n, K, N in shapes) +
+            "; step = quantize_mask_pack of all layers (one batched launch), then quant_act + sparse_bitlinear (bf16 out) per layer")
 
 
 def max_over_ranks(ms_local, world, dist=None, device="cpu"):
@@ -139,7 +153,7 @@ class ClockSampler:
                     reasons.add(name)
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+        return {"sm_mhz": statistics.median(sm), "sm_mhz_min": min(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
                 "samples": len(sm)}
 
 
@@ -164,12 +178,13 @@ def oracle_step(sample_tokens: int, cache: dict):
 
 
 def run_reference(args):
-    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    """--impl reference: the CPU oracle, as it stands, on the host cores (rank 0 only), on the very
+    workload the GPU arm times: all T = 4096 tokens of all four layers per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
-    sample = 256
+    sample = T_TOKENS
     cache = {}
     for _ in range(args.warmup):
         oracle_step(sample, cache)
@@ -177,15 +192,16 @@ def run_reference(args):
     total = sum(times)
     value = step_ops(sample) * args.steps / total / 1e12
     cores = oracle.num_threads()
+    in_bytes = sum(N * K * 4 + sample * K * 2 for _, K, N in inputs.SHAPES_2B)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
         "data": "synthetic",
-        "config": {"workload": f"BitNet-2B-shaped BitLinears (qkv, o, gate_up, down), {sample}-token sample of the T={T_TOKENS} batch",
-                   "l2": "n/a (host)"},
+        "config": {"workload": workload_string("2b", sample, inputs.SHAPES_2B), "tokens": sample, "parallelism": "single",
+                   "l2": f"step streams {in_bytes / 1e6:.0f} MB of inputs (host arm: the CPU oracle on the host cores)"},
         "cpu_baseline": {"value": value, "unit": "TOPS", "cores": cores, "kind": "oracle",
-                         "sample": f"{sample} of {T_TOKENS} tokens per layer, all four weight matrices in full"},
+                         "sample": f"all {sample} tokens per layer, all four weight matrices in full, every step"},
         "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -221,6 +237,78 @@ class Layer:
         self.y_host = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
         self.ws = b.alloc_gemm_ws(b.OP_SPARSE_BITLINEAR, T, N, K)
         self.ops = 2.0 * T * N * K
+
+
+def large_m_and_sustained(torch, b, peaks, sampler, time_cold, iters):
+    """The large-M target on the two 7B-class shapes (T = 8192; weights N(0, 0.015) with 5 % x10 outliers,
+    activations with a per-token LogNormal(0, 0.5) scale): isolated sparse and dense GEMM, cold L2, both
+    output dtypes; then the down projection's GEMM launched back to back for >= 2 s (sparse, then dense)
+    with the SM clock sampled meanwhile -- what the kernel sustains, next to the burst figure."""
+    stream = torch.cuda.current_stream()
+    rows, sustained = {}, {}
+    ratio = DATASHEET_INT8_SPARSE_TOPS / NOMINAL_BF16_DENSE_TFLOPS
+    for i, (name, K, N) in enumerate(inputs.SHAPES_7B):
+        T = 8192
+        W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i, sigma=0.015, outlier_prob=0.05)).cuda()
+        x = torch.from_numpy(inputs.activations_bf16(T, K, seed=11 + i, token_lognormal_sigma=0.5).view(np.int16)).cuda().view(torch.bfloat16)
+        p = b.alloc_packed(N, K, with_dense=True)
+        b.sbn_quantize_mask_pack(W, p["vals"], p["meta"], p["w_scale"], p["ws"], dense_q=p["dense_q"])
+        del W
+        xq = b.alloc_xq(T, K)
+        a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
+        b.sbn_quant_act(x, xq, a_scale)
+        del x
+        ops = 2.0 * T * N * K
+        row = {"T": T, "K": K, "N": N}
+        ys = {"bf16": torch.empty((T, N), dtype=torch.bfloat16, device="cuda"), "f32": torch.empty((T, N), dtype=torch.float32, device="cuda")}
+        sp_fn = lambda y: b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y)
+        de_fn = lambda y: b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y)
+        for tag, y in ys.items():
+            for _ in range(3):
+                sp_fn(y)
+                de_fn(y)
+            sp = time_cold(lambda: sp_fn(y), iters)
+            de = time_cold(lambda: de_fn(y), iters)
+            row[tag] = {"sparse_us": round(sp, 2), "dense_us": round(de, 2),
+                        "sparse_tops": round(ops / sp / 1e6, 1), "dense_tops": round(ops / de / 1e6, 1),
+                        "pct_sparse_int8_datasheet": round(100 * ops / sp / 1e6 / DATASHEET_INT8_SPARSE_TOPS, 1),
+                        "pct_of_measured_bf16_burst_x4": round(100 * ops / sp / 1e6 / (peaks["bf16_tflops"] * ratio), 1),
+                        "speedup_vs_dense": round(de / sp, 3)}
+        rows[name] = row
+        if name == "down_7b":
+            y = ys["bf16"]
+            for tag, fn in (("sparse", sp_fn), ("dense", de_fn)):
+                fn(y)
+                torch.cuda.synchronize()
+                a = torch.cuda.Event(enable_timing=True)
+                c = torch.cuda.Event(enable_timing=True)
+                t0 = time.time()
+                a.record(stream)
+                n = 0
+                while time.time() - t0 < 2.2:                      # the queue fills, then the host enqueues at the GPU's pace
+                    for _ in range(64):
+                        fn(y)
+                    n += 64
+                c.record(stream)
+                torch.cuda.synchronize()
+                t1 = time.time()
+                ms = a.elapsed_time(c)
+                clk = sampler.summary(t0 + 0.3, t1 - 0.05)            # samples well inside the loaded interval
+                tops = ops * n / (ms * 1e-3) / 1e12
+                peak_sus = peaks["bf16_tflops_sustained"] * (ratio if tag == "sparse" else ratio / 2)
+                sm = clk["sm_mhz"]
+                sustained[tag] = {"launches": n, "seconds": round(ms * 1e-3, 3), "us_per_launch": round(ms * 1e3 / n, 2), "tops": round(tops, 1),
+                                  "pct_int8_datasheet": round(100 * tops / (DATASHEET_INT8_SPARSE_TOPS if tag == "sparse" else DATASHEET_INT8_DENSE_TOPS), 1),
+                                  "frac_of_measured_bf16_sustained_x_ratio": round(tops / peak_sus, 4),
+                                  "sm_mhz_median": sm, "sm_mhz_min": clk.get("sm_mhz_min"), "sm_max_mhz": clk["sm_max_mhz"],
+                                  "reasons": clk["reasons"], "clock_samples": clk["samples"],
+                                  "tops_scaled_to_max_clock": round(tops * clk["sm_max_mhz"] / sm, 1) if sm else None}
+            sustained["workload"] = f"down_7b {K}->{N} at T={T}, bf16 out, same launch back to back for >= 2 s (L2-warm)"
+            sustained["peak_source"] = (f"{peaks['source']} bf16 sustained {peaks['bf16_tflops_sustained']} TFLOP/s x {ratio:g} (sparse int8) "
+                                        f"or x {ratio / 2:g} (dense int8), nominal ratios")
+        del p, xq, ys
+        torch.cuda.empty_cache()
+    return rows, sustained
 
 
 def run_ours(args):
@@ -430,6 +518,11 @@ def run_ours(args):
             row["norm_quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4 + L.K * 4) / nact / 1e3, 1)
         gemm[L.name] = row
     b.sbn_check_status()
+    large_m, sustained, few_tokens = None, None, None
+    if rank == 0 and world == 1 and args.workload == "2b" and not args.no_extras:
+        large_m, sustained = large_m_and_sustained(torch, b, peaks, sampler, time_cold, iters)
+        few_tokens = decode_rows(torch, b, peaks, inputs.SHAPES_2B, (1, 4, 16, 64), cold=False)
+        b.sbn_check_status()
     sampler.stop()
     clocks = sampler.summary(t_wall0, t_wall1)
 
@@ -444,7 +537,8 @@ def run_ours(args):
         achieved = sum(L.ops for L in layers) / (tot[dominant] * 1e-6) / 1e12
         roofline = {"bound": "tensor", "kernel": "bitlinear_gemm_pair_kernel<sparse, 1>" if args.workload == "2b" else "bitlinear_gemm_pair_kernel<sparse, 2>", "achieved": round(achieved, 1),
                     "peak": round(peak, 1), "unit": "TOP/s", "frac": round(achieved / peak, 4),
-                    "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(args.workload),
+                    "traffic": gemm_dram_traffic(args.workload),
+                    "traffic_source": "profiles/gemm_dram_traffic.json (ncu capture of this step)",
                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {ratio:g} (nominal sparse-int8 : bf16)",
                     "frac_of_datasheet_sparse_int8": round(achieved / DATASHEET_INT8_SPARSE_TOPS, 4)}
     else:
@@ -474,8 +568,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: BitLinears at T={T}: " + ", ".join(f"{n} {K}->{N}" for n, K, N in shapes) +
-                                   "; step = quantize_mask_pack of all layers (one batched launch), then quant_act + sparse_bitlinear (bf16 out) per layer",
+            "config": {"workload": workload_string(args.workload, T, shapes),
                        "tokens": T, "parallelism": "replicas" if world > 1 else "single",
                        "l2": f"step streams {in_bytes / 1e6:.0f} MB of inputs (> 126 MB L2); isolated-kernel numbers flush L2 before every launch"},
             "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
@@ -486,6 +579,9 @@ def run_ours(args):
             "cpu_baseline": cpu_baseline,
             "kernel_us_in_step": {k: {n: round(v, 2) for n, v in d.items()} for k, d in kernel_us.items()},
             "isolated": gemm,
+            "isolated_large_m": large_m,
+            "sustained": sustained,
+            "few_tokens": few_tokens,
             "datasheet_int8_tops": {"dense": DATASHEET_INT8_DENSE_TOPS, "sparse": DATASHEET_INT8_SPARSE_TOPS},
             "measured_peaks": peaks,
         }
@@ -515,24 +611,17 @@ def _cold_timer(torch, stream, flush):
     return time_cold
 
 
-def run_decode_sweep(args):
-    """Small-T regime (the paper's decode table is M = 64..512): T in {1, 4, 16, 64, 128, 256, 512} over
-    the four 2B-shaped matrices, sparse vs dense.  Two timings per point: `cold` = one launch after
-    512 MB were written over L2 (includes the ~6 us an empty launch costs between two events), and
-    `stream` = launches back to back over enough distinct weight copies that every launch reads its
-    weights from HBM (what a decode loop over the layers of a model sees).  Memory-bound: GB/s of
+def decode_rows(torch, b, peaks, shapes, token_counts, big=False, cold=True):
+    """Few-token rows: for every (matrix, T) the sparse and the dense BitLinear, `stream` = launches back
+    to back over enough distinct weight copies that every launch reads its weights from HBM (what a
+    decode loop over the layers of a model sees), and optionally `cold` = one launch after 512 MB were
+    written over L2 (includes the ~6 us an empty launch costs between two events).  Memory-bound: GB/s of
     algorithmic bytes (weights + activations + outputs) against the measured HBM rate."""
-    import torch
-    from paper_2603_05168_b200 import binding as b
-    from paper_2603_05168_b200 import build as sbn_build
-    sbn_build.build()
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
-    peaks = load_peaks()
     stream = torch.cuda.current_stream()
-    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    time_cold = _cold_timer(torch, stream, flush)
+    time_cold = None
+    if cold:
+        flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+        time_cold = _cold_timer(torch, stream, flush)
 
     def time_stream(fns, reps=48):
         for f in fns:
@@ -548,9 +637,6 @@ def run_decode_sweep(args):
         torch.cuda.synchronize()
         return a.elapsed_time(c) * 1e3 / reps
 
-    big = args.workload == "decode7b"
-    shapes = [("gate_up_7b", 4096, 11008), ("down_7b", 11008, 4096), ("qkv_7b", 4096, 12288), ("o_7b", 4096, 4096)] if big else inputs.SHAPES_2B
-    token_counts = (1, 4, 16, 32, 64) if big else (1, 4, 16, 64, 128, 256, 512)
     rows = []
     for i, (name, K, N) in enumerate(shapes):
         W = torch.from_numpy(inputs.latent_weights(N, K, seed=1 + i)).cuda()
@@ -576,29 +662,51 @@ def run_decode_sweep(args):
             for _ in range(3):
                 b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=ws_s)
                 b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y, ws=ws_d)
-            sp = time_cold(lambda: b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=ws_s), 15)
-            de = time_cold(lambda: b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y, ws=ws_d), 15)
             io = T * K + T * N * 2 + T * 4
+            sp_bytes = N * K * 0.625 + io
+            de_bytes = N * K * 1.0 + io
+            row = {"layer": name, "T": T}
+            if cold:
+                sp = time_cold(lambda: b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], p["meta"], p["w_scale"], y, ws=ws_s), 15)
+                de = time_cold(lambda: b.sbn_bitlinear(xq, a_scale, p["dense_q"], p["w_scale"], y, ws=ws_d), 15)
+                row.update({"sparse_us": round(sp, 2), "dense_us": round(de, 2),
+                            "sparse_gbs": round(sp_bytes / sp / 1e3, 1), "dense_gbs": round(de_bytes / de / 1e3, 1),
+                            "speedup_vs_dense": round(de / sp, 3),
+                            "sparse_frac_of_hbm": round(sp_bytes / sp / 1e3 / peaks["hbm_gbs"], 4)})
             sp_st = time_stream([(lambda q=q: b.sbn_sparse_bitlinear(xq, a_scale, q["vals"], q["meta"], q["w_scale"], y, ws=ws_s))
                                  for q in packs])
             de_st = time_stream([(lambda q=q: b.sbn_bitlinear(xq, a_scale, q["dense_q"], q["w_scale"], y, ws=ws_d))
                                  for q in packs])
-            sp_bytes = N * K * 0.625 + io
-            de_bytes = N * K * 1.0 + io
-            extra = {}
             if big:
                 pk_st = time_stream([(lambda q=q: b.sbn_sparse_bitlinear_packed(xq, a_scale, q["vals2"], q["meta"], q["w_scale"], y))
                                      for q in packs])
-                extra = {"packed_stream_us": round(pk_st, 2), "packed_stream_gbs": round((N * K * 0.25 + io) / pk_st / 1e3, 1),
-                         "packed_vs_int8_held": round(sp_st / pk_st, 3)}
-            rows.append({"layer": name, "T": T, **extra, "sparse_us": round(sp, 2), "dense_us": round(de, 2),
-                         "sparse_stream_us": round(sp_st, 2), "dense_stream_us": round(de_st, 2),
-                         "sparse_gbs": round(sp_bytes / sp / 1e3, 1), "dense_gbs": round(de_bytes / de / 1e3, 1),
-                         "sparse_stream_gbs": round(sp_bytes / sp_st / 1e3, 1),
-                         "speedup_vs_dense": round(de / sp, 3), "stream_speedup_vs_dense": round(de_st / sp_st, 3),
-                         "sparse_frac_of_hbm": round(sp_bytes / sp / 1e3 / peaks["hbm_gbs"], 4),
-                         "sparse_stream_frac_of_hbm": round(sp_bytes / sp_st / 1e3 / peaks["hbm_gbs"], 4)})
+                row.update({"packed_stream_us": round(pk_st, 2), "packed_stream_gbs": round((N * K * 0.25 + io) / pk_st / 1e3, 1),
+                            "packed_vs_int8_held": round(sp_st / pk_st, 3)})
+            row.update({"sparse_stream_us": round(sp_st, 2), "dense_stream_us": round(de_st, 2),
+                        "sparse_stream_gbs": round(sp_bytes / sp_st / 1e3, 1), "dense_stream_gbs": round(de_bytes / de_st / 1e3, 1),
+                        "stream_speedup_vs_dense": round(de_st / sp_st, 3),
+                        "sparse_stream_frac_of_hbm": round(sp_bytes / sp_st / 1e3 / peaks["hbm_gbs"], 4)})
+            rows.append(row)
         del packs
+    return rows
+
+
+def run_decode_sweep(args):
+    """Small-T regime (the paper's decode table is M = 64..512): T in {1, 4, 16, 64, 128, 256, 512} over
+    the four 2B-shaped matrices (decode7b: T <= 64 over 7B-class matrices, with the 2-bit packed
+    weights as a third arm), sparse vs dense, cold and streamed (see decode_rows)."""
+    import torch
+    from paper_2603_05168_b200 import binding as b
+    from paper_2603_05168_b200 import build as sbn_build
+    sbn_build.build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    peaks = load_peaks()
+    big = args.workload == "decode7b"
+    shapes = [("gate_up_7b", 4096, 11008), ("down_7b", 11008, 4096), ("qkv_7b", 4096, 12288), ("o_7b", 4096, 4096)] if big else inputs.SHAPES_2B
+    token_counts = (1, 4, 16, 32, 64) if big else (1, 4, 16, 64, 128, 256, 512)
+    rows = decode_rows(torch, b, peaks, shapes, token_counts, big=big, cold=True)
     b.sbn_check_status()
     print(json.dumps({"metric": "small-T sparse vs dense ternary BitLinear, HBM GB/s (cold L2)", "unit": "GB/s",
                       "workload": args.workload, "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -701,6 +809,47 @@ def run_pattern68(args):
                       "gpu_launches": b.sbn_launch_count()}))
 
 
+def dyn_oracle_leg(torch, b, mats, host_W, host_x, acts, cur_meta, T):
+    """The dynamic-mask step against the CPU oracle on the seven matrices of layer 0 (host-seeded): after
+    the first timed step the scale, every packed byte (through the library's own un-tiling call) and the
+    flip count of each matrix, and 2048 sampled outputs of each of its BitLinears.  Raises on a mismatch."""
+    import oracle
+    worst_ulp, checked = 0, 0
+    for m_i in range(len(inputs.LAYER_2B)):
+        name, K, N, W, p = mats[m_i]
+        r_prev = oracle.quantize_mask_pack(host_W[("prev", m_i)])
+        r = oracle.quantize_mask_pack(host_W[m_i])
+        if r["near_tie"] or r_prev["near_tie"]:
+            continue
+        vals = torch.empty((N, K // 2), dtype=torch.int8, device="cuda")
+        meta = torch.empty((N, K // 8), dtype=torch.uint8, device="cuda")
+        b.sbn_unpack_canonical(p["vals"], cur_meta(p), N, K, vals, meta)
+        b.sbn_check_status()
+        if np.float32(p["w_scale"].cpu().numpy()[0]) != r["scale"]:
+            raise RuntimeError(f"dyn oracle leg: scale of {name} differs from the oracle")
+        if not (np.array_equal(vals.cpu().numpy(), r["vals"]) and np.array_equal(meta.cpu().numpy(), r["meta"])):
+            raise RuntimeError(f"dyn oracle leg: packed weights of {name} differ from the oracle")
+        want_flips = oracle.flip_count(r_prev["mask"], r["mask"])
+        if int(p["flips"].item()) != want_flips:
+            raise RuntimeError(f"dyn oracle leg: flip count of {name}: {int(p['flips'].item())} != oracle {want_flips}")
+        xq_ref, s_ref = oracle.quant_act(host_x[K])
+        xq, a_scale = acts[K]
+        y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+        b.sbn_sparse_bitlinear(xq, a_scale, p["vals"], cur_meta(p), p["w_scale"], y)
+        b.sbn_check_status()
+        t_idx, n_idx = inputs.sample_positions(T, N, 2048, seed=900 + m_i)
+        acc_ref = oracle.acc_packed_sampled(xq_ref, r["vals"], r["meta"], t_idx, n_idx)
+        y_ref = oracle.dequant(acc_ref.reshape(-1, 1), r["scale"], s_ref[t_idx]).ravel()
+        got = y.view(torch.int16).cpu().numpy().view(np.uint16)[t_idx, n_idx].astype(np.int32)
+        ulp = int(np.abs(got - oracle.f32_to_bf16_bits(y_ref).astype(np.int32)).max())
+        if ulp > 1:
+            raise RuntimeError(f"dyn oracle leg: outputs of {name} off by {ulp} bf16 ulp")
+        worst_ulp = max(worst_ulp, ulp)
+        checked += 1
+    return {"layer": 0, "matrices_checked": checked, "checked": "w_scale, vals, meta, flip count (all exact); 2048 sampled bf16 outputs per BitLinear",
+            "max_output_ulp": worst_ulp}
+
+
 def run_dynamic_step(args):
     """Dynamic-mask training step (the mask is recomputed every step): perturb all master weights
     (outside the timed region), then timed: quantise/mask/pack all 30 x 7 matrices with the flip
@@ -718,9 +867,18 @@ def run_dynamic_step(args):
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234)
     mats = []
+    # Oracle leg: the seven matrices of layer 0 are drawn (and perturbed) on the HOST with the seeded
+    # generators of inputs.py, so the CPU oracle sees the very same weights; the other 29 layers are drawn
+    # on the device (8 GB of host-generated weights would dominate the run).
+    oracle_leg = args.masters == "fp32" and not args.no_cpu_baseline
+    host_W = {}
     for layer in range(n_layers):
-        for name, K, N in inputs.LAYER_2B:
-            W = torch.randn((N, K), generator=gen, device="cuda", dtype=torch.float32) * 0.02
+        for j, (name, K, N) in enumerate(inputs.LAYER_2B):
+            if layer == 0 and oracle_leg:
+                host_W[j] = inputs.latent_weights(N, K, seed=700 + j)
+                W = torch.from_numpy(host_W[j]).cuda()
+            else:
+                W = torch.randn((N, K), generator=gen, device="cuda", dtype=torch.float32) * 0.02
             if args.masters == "bf16":
                 W = W.to(torch.bfloat16)
             p = b.alloc_packed(N, K)
@@ -728,9 +886,10 @@ def run_dynamic_step(args):
             p["flips"] = torch.zeros(1, dtype=torch.int64, device="cuda")
             mats.append((name, K, N, W, p))
     # one activation set per distinct K (shared by the layers; attention/norms are not on this path)
-    acts = {}
+    acts, host_x = {}, {}
     for K in sorted({K for _, K, _ in inputs.LAYER_2B}):
-        x = (torch.randn((T, K), generator=gen, device="cuda")).to(torch.bfloat16)
+        host_x[K] = inputs.activations_bf16(T, K, seed=750 + K)
+        x = torch.from_numpy(host_x[K].view(np.int16)).cuda().view(torch.bfloat16)
         xq = b.alloc_xq(T, K)
         a_scale = torch.empty(T, dtype=torch.float32, device="cuda")
         b.sbn_quant_act(x, xq, a_scale)
@@ -766,9 +925,18 @@ def run_dynamic_step(args):
     b.sbn_check_status()
     rep_ms, fwd_ms, rates = [], [], []
     steps = max(1, min(args.steps, 5))
+    oracle_report = None
     for s_i in range(steps + 1):
-        for _, K, N, W, p in mats:                                # the optimiser step stand-in
-            W.add_(torch.randn(W.shape, generator=gen, device="cuda", dtype=torch.float32).to(W.dtype), alpha=1e-4)
+        for m_i, (_, K, N, W, p) in enumerate(mats):              # the optimiser step stand-in
+            if m_i in host_W and s_i <= 1:
+                # layer 0 up to the checked step: the perturbation is drawn on the host, like the weights
+                host_prev = host_W[m_i]
+                host_W[m_i] = inputs.perturb_weights(host_prev, seed=800 + 10 * s_i + m_i, sigma=1e-4)
+                W.copy_(torch.from_numpy(host_W[m_i]))
+                if s_i == 1:
+                    host_W[("prev", m_i)] = host_prev
+            else:
+                W.add_(torch.randn(W.shape, generator=gen, device="cuda", dtype=torch.float32).to(W.dtype), alpha=1e-4)
         torch.cuda.synchronize()
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         torch.cuda._sleep(int(4e7))
@@ -784,6 +952,8 @@ def run_dynamic_step(args):
         fwd_ms.append(e[1].elapsed_time(e[2]))
         flips = sum(int(p["flips"].item()) for *_, p in mats)
         rates.append(flips / params)
+        if s_i == 1 and oracle_leg:
+            oracle_report = dyn_oracle_leg(torch, b, mats, host_W, host_x, acts, cur_meta, T)
     b.sbn_check_status()
     rep, fwd = statistics.median(rep_ms), statistics.median(fwd_ms)
     fwd_ops = sum(2.0 * T * N * K for _, K, N, _, _ in mats)
@@ -796,7 +966,9 @@ def run_dynamic_step(args):
         "repack_frac_of_hbm": round(params * ((2 if args.masters == "bf16" else 4) + 0.75) / (rep * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
         "forward_tops": round(fwd_ops / (fwd * 1e-3) / 1e12, 1),
         "forward_pct_sparse_int8_datasheet": round(100 * fwd_ops / (fwd * 1e-3) / 1e12 / DATASHEET_INT8_SPARSE_TOPS, 1),
-        "flip_rate": statistics.mean(rates), "steps": steps, "data": "synthetic (torch CUDA generator, seed 1234)",
+        "flip_rate": statistics.mean(rates), "steps": steps,
+        "data": "synthetic: layer 0 and all activations seeded on the host (inputs.py), layers 1-29 from torch's CUDA generator (seed 1234)",
+        "oracle_leg": oracle_report,
         "gpu_launches": b.sbn_launch_count()}))
 
 
@@ -807,6 +979,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="headline line only: skip the 7B-class isolated GEMMs, the sustained run and the few-token rows")
     ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68"],
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1..512), sparse vs dense, cold L2 and streamed; "

@@ -94,15 +94,20 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 
-// Bounded wait: false if the barrier did not flip within the limit or the CTA is aborting.
+// Bounded wait: false if the barrier did not flip within the limit or the CTA is aborting.  The clock
+// is only read every 1024 failed polls (the first such reading starts the limit), so a wait that is
+// over after a few polls -- every wait of a healthy run -- costs nothing but the polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
+    unsigned long long t0 = 0ull;
     unsigned int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3FFu) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) {
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0ull) {
+                t0 = now;
+            } else if (now - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) {
                 *abort_flag = 1;
                 atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
                 return false;
