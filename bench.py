@@ -74,7 +74,7 @@ def gemm_dram_traffic(workload):
 
 def workload_string(name, T, shapes):
     return (f"{name}: BitLinears at T={T}: " + ", ".join(f"{n} {K}->{N}" for n, K, N in shapes) +
-            "; step = quantize_mask_pack of all layers (one batched launch), then quant_act + sparse_bitlinear (bf16 out) per layer")
+            "; step = quantize_mask_pack of all layers (one batched launch, previous step's scales as hints), then quant_act + sparse_bitlinear (bf16 out) per layer")
 
 
 def max_over_ranks(ms_local, world, dist=None, device="cpu"):
@@ -347,7 +347,10 @@ def run_ours(args):
     # One launch re-quantises, masks and packs all layers' weights (the batched entry point runs
     # pass 1 of matrix m + 1 under the exchange and pass 2 of matrix m); then, per layer, the
     # activation quantiser and the sparse GEMM.
-    pack_jobs = b.make_pack_jobs([dict(W=L.W, vals=L.packed["vals"], meta=L.packed["meta"], w_scale=L.packed["w_scale"])
+    # gamma_hint = the scale the previous step left in w_scale (a dynamic-mask training step re-packs
+    # slowly drifting weights): the kernel then need not sample the matrix before it streams it.
+    pack_jobs = b.make_pack_jobs([dict(W=L.W, vals=L.packed["vals"], meta=L.packed["meta"], w_scale=L.packed["w_scale"],
+                                       gamma_hint=L.packed["w_scale"])
                                   for L in layers])
     pack_ws = torch.empty(b.sbn_batch_workspace_bytes(len(layers)), dtype=torch.uint8, device="cuda")
 
@@ -901,7 +904,8 @@ def run_dynamic_step(args):
     job_ws = torch.empty(b.sbn_batch_workspace_bytes(len(mats)), dtype=torch.uint8, device="cuda")
     plain_jobs = b.make_pack_jobs([dict(W=W, vals=p["vals"], meta=p["meta"], w_scale=p["w_scale"]) for _, _, _, W, p in mats])
     flip_jobs = [b.make_pack_jobs([dict(W=W, vals=p["vals"], meta=p["meta"] if par == 0 else p["prev"], w_scale=p["w_scale"],
-                                        prev_meta=p["prev"] if par == 0 else p["meta"], flip_bits=p["flips"])
+                                        prev_meta=p["prev"] if par == 0 else p["meta"], flip_bits=p["flips"],
+                                        gamma_hint=p["w_scale"])              # the previous step's scale
                                    for _, _, _, W, p in mats]) for par in (0, 1)]
     state = {"par": 1}            # after the plain pack the current metadata is in p["meta"]
 

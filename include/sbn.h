@@ -170,7 +170,8 @@ sbn_status sbn_quantize_mask_pack_bf16(const void *W_bf16, int N, int K, int n_k
  * Part 1 for many matrices in ONE launch -- the dynamic-mask training step recomputes the mask of
  * every BitLinear at every step (Sec. 2.3, "Dynamic Mask Recomputation"; Algorithm 1).  Each job
  * is exactly one sbn_quantize_mask_pack call (same arguments, same results, bit for bit); the
- * kernel pipelines the jobs so that launch and exchange latencies are paid once per batch.
+ * kernel streams through the matrices without a pause between them: the exchange of partial sums,
+ * the threshold and the fix-up of one matrix run under the pass over the next ones.
  *   jobs   host array of `count` jobs; fully read before the call returns (pageable memory is
  *          fine: the jobs travel to the device as kernel arguments, 48 per small launch, not through
  *          a staging copy, so the call only enqueues and never blocks on the stream)
@@ -187,6 +188,12 @@ typedef struct {
     const uint8_t *prev_meta;         /* device or NULL */
     unsigned long long *flip_bits;    /* device out; required iff prev_meta != NULL */
     int w_bf16;                       /* 0: W is fp32; 1: W is bf16 (see sbn_quantize_mask_pack_bf16) */
+    const float *gamma_hint;          /* device, one fp32, or NULL: an estimate of this matrix's gamma, e.g. the
+                                         w_scale of the previous training step (may be the very w_scale buffer
+                                         above: it is read before it is written).  A speed hint only -- results
+                                         never depend on it.  With a hint within a few percent of gamma the
+                                         kernel need not sample the matrix first; a hint that is far off (or not a
+                                         positive finite number) costs a second pass over that matrix */
 } sbn_pack_job;
 size_t sbn_batch_workspace_bytes(int count);
 sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job *jobs, void *ws, size_t ws_bytes,

@@ -155,7 +155,8 @@ def sbn_quantize_mask_pack_static_ws(W, vals, meta, w_scale, dense_q=None, prev_
 class PackJob(ctypes.Structure):
     _fields_ = [("W", ctypes.c_void_p), ("N", ctypes.c_int), ("K", ctypes.c_int), ("vals", ctypes.c_void_p),
                 ("meta", ctypes.c_void_p), ("w_scale", ctypes.c_void_p), ("dense_q", ctypes.c_void_p),
-                ("prev_meta", ctypes.c_void_p), ("flip_bits", ctypes.c_void_p), ("w_bf16", ctypes.c_int)]
+                ("prev_meta", ctypes.c_void_p), ("flip_bits", ctypes.c_void_p), ("w_bf16", ctypes.c_int),
+                ("gamma_hint", ctypes.c_void_p)]
 
 
 def sbn_batch_workspace_bytes(count: int) -> int:
@@ -163,8 +164,8 @@ def sbn_batch_workspace_bytes(count: int) -> int:
 
 
 def make_pack_jobs(jobs):
-    """jobs: list of dicts with W, vals, meta, w_scale and optionally dense_q, prev_meta, flip_bits
-    (torch CUDA tensors).  Returns the ctypes array to hand to sbn_quantize_mask_pack_batched; it can
+    """jobs: list of dicts with W, vals, meta, w_scale and optionally dense_q, prev_meta, flip_bits,
+    gamma_hint (torch CUDA tensors).  Returns the ctypes array to hand to sbn_quantize_mask_pack_batched; it can
     be reused every step as long as the tensors stay where they are."""
     arr = (PackJob * len(jobs))()
     for a, j in zip(arr, jobs):
@@ -172,7 +173,7 @@ def make_pack_jobs(jobs):
         a.W, a.N, a.K = j["W"].data_ptr(), N, K
         a.w_bf16 = 1 if j["W"].dtype == torch.bfloat16 else 0
         a.vals, a.meta, a.w_scale = j["vals"].data_ptr(), j["meta"].data_ptr(), j["w_scale"].data_ptr()
-        for key in ("dense_q", "prev_meta", "flip_bits"):
+        for key in ("dense_q", "prev_meta", "flip_bits", "gamma_hint"):
             t = j.get(key)
             setattr(a, key, t.data_ptr() if t is not None else None)
     return arr

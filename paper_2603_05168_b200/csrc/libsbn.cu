@@ -15,6 +15,7 @@
 #include "norm_quant_act.cuh"
 #include "quantize_mask_pack.cuh"
 #include "quantize_mask_pack68.cuh"
+#include "quantize_mask_pack_stream.cuh"
 #include "canonical_layout.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_pair_tcgen05.cuh"
@@ -547,7 +548,6 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
     if (!ws || ws_bytes < sbn_batch_workspace_bytes(count)) return SBN_ERR_WORKSPACE;
     if (misaligned(ws, 16)) return SBN_ERR_ALIGN;
     std::vector<QmpDesc> descs(static_cast<size_t>(count));
-    uint32_t max_units = 0;
     for (int i = 0; i < count; ++i) {
         const sbn_pack_job& j = jobs[i];
         if (!j.W || !j.vals || !j.meta || !j.w_scale) return SBN_ERR_NULL;
@@ -557,26 +557,36 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
             (j.dense_q && misaligned(j.dense_q, 16)) || (j.prev_meta && misaligned(j.prev_meta, 16)) ||
             (j.flip_bits && misaligned(j.flip_bits, 8)))
             return SBN_ERR_ALIGN;
-        descs[i] = qmp_make_desc(j.W, j.w_bf16 != 0, j.N, j.K, j.vals, j.meta, j.w_scale, j.dense_q, j.prev_meta, j.flip_bits);
-        max_units = std::max(max_units, descs[i].num_units);
+        if (j.gamma_hint && misaligned(j.gamma_hint, 4)) return SBN_ERR_ALIGN;
+        descs[i] = qmp_make_desc(j.W, j.w_bf16 != 0, j.N, j.K, j.vals, j.meta, j.w_scale, j.dense_q, j.prev_meta, j.flip_bits,
+                                 j.gamma_hint);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned long long* generation = static_cast<unsigned long long*>(ws);
-    QmpDesc* rest_dev = reinterpret_cast<QmpDesc*>(static_cast<char*>(ws) + 256);
-    // Jobs 1.. are read by the kernel from the workspace (job 0 travels as a kernel argument).  They get
-    // there as arguments of small store kernels, a chunk at a time: nothing is staged through host
-    // memory, so the call only enqueues and the caller's array is free as soon as it returns.
-    for (int at = 1; at < count; at += kQmpDescChunk) {
-        QmpDescChunk chunk;
-        const int n = std::min(kQmpDescChunk, count - at);
-        for (int i = 0; i < n; ++i) chunk.d[i] = descs[static_cast<size_t>(at + i)];
-        for (int i = n; i < kQmpDescChunk; ++i) chunk.d[i] = descs[0];
-        const cudaError_t err = launch_kernel(qmp_store_descs_kernel, dim3(1), dim3(64), 0, s, chunk, rest_dev + (at - 1), n);
-        ++g_launch_count;
-        if (err != cudaSuccess) return SBN_ERR_CUDA;
-    }
+    QmpDesc* descs_dev = reinterpret_cast<QmpDesc*>(static_cast<char*>(ws) + 256);
     QmpSlot* slots = reinterpret_cast<QmpSlot*>(static_cast<char*>(ws) + 256 + batch_desc_bytes(count));
-    return launch_quantize_mask_pack_batch(descs[0], rest_dev, count, max_units, slots, generation, s);
+    // One launch per kQmpMaxBatch matrices (the kernel keeps a little state per matrix on chip).  All jobs
+    // but the first of a launch are read by the kernel from the workspace (the first travels as a kernel
+    // argument).  They get there as arguments of small store kernels, a chunk at a time: nothing is staged
+    // through host memory, so the call only enqueues and the caller's array is free as soon as it returns.
+    for (int lo = 0; lo < count; lo += kQmpMaxBatch) {
+        const int n_here = std::min(kQmpMaxBatch, count - lo);
+        uint32_t max_units = 0;
+        for (int i = 0; i < n_here; ++i) max_units = std::max(max_units, descs[static_cast<size_t>(lo + i)].num_units);
+        for (int at = 1; at < n_here; at += kQmpDescChunk) {
+            QmpDescChunk chunk;
+            const int n = std::min(kQmpDescChunk, n_here - at);
+            for (int i = 0; i < n; ++i) chunk.d[i] = descs[static_cast<size_t>(lo + at + i)];
+            for (int i = n; i < kQmpDescChunk; ++i) chunk.d[i] = descs[0];
+            const cudaError_t err = launch_kernel(qmp_store_descs_kernel, dim3(1), dim3(64), 0, s, chunk, descs_dev + (lo + at - 1), n);
+            ++g_launch_count;
+            if (err != cudaSuccess) return SBN_ERR_CUDA;
+        }
+        const sbn_status st = launch_quantize_mask_pack_stream(descs[static_cast<size_t>(lo)], descs_dev + lo, n_here, max_units,
+                                                               slots + static_cast<size_t>(lo) * kQmpMaxCtas, generation, s);
+        if (st != SBN_OK) return st;
+    }
+    return SBN_OK;
 }
 
 sbn_status sbn_quantize_mask_pack_static_ws(const float* W, int N, int K, int n_keep, int m_group,

@@ -168,6 +168,7 @@ struct QmpDesc {
     uint32_t* dense_q;                 // or null
     const uint8_t* prev_meta;          // or null
     unsigned long long* flip_bits;     // or null
+    const float* gamma_hint;           // or null: the caller's estimate of gamma (e.g. the previous step's scale)
     uint32_t num_units;                // N * K / 128
     uint32_t KB;                       // K / 128
     uint32_t w_bf16;                   // master weights are bf16 (Sec. 2.2 keeps them "e.g. in bf16")
@@ -558,8 +559,10 @@ inline unsigned long long qmp_next_nonce() {
 }
 
 inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* vals, uint8_t* meta, float* w_scale,
-                             int8_t* dense_q, const uint8_t* prev_meta, unsigned long long* flip_bits) {
+                             int8_t* dense_q, const uint8_t* prev_meta, unsigned long long* flip_bits,
+                             const float* gamma_hint = nullptr) {
     QmpDesc d;
+    d.gamma_hint = gamma_hint;
     d.W = W;
     d.w_bf16 = w_bf16 ? 1u : 0u;
     d.vals = reinterpret_cast<uint16_t*>(vals);
@@ -593,15 +596,6 @@ inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const Qm
                                           first, rest_dev, count, slots, generation, nonce, test_withhold_slot);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
-}
-
-inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, int K, int8_t* vals,
-                                            uint8_t* meta, float* w_scale, int8_t* dense_q,
-                                            const uint8_t* prev_meta,
-                                            unsigned long long* flip_bits, QmpWorkspace* ws,
-                                            cudaStream_t stream) {
-    const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
-    return launch_quantize_mask_pack_batch(d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream);
 }
 
 }  // namespace sbn

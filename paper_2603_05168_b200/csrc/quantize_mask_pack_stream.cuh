@@ -1,0 +1,469 @@
+// Part 1 (Eq. 1-3, 2:4 pattern) for one matrix or a batch, as ONE uninterrupted stream over the weights.
+//
+// quantize_mask_pack.cuh explains the single-read scheme (bracketed threshold, provisional values,
+// fix-up list, exact fallback).  What costs time beside the stream itself is latency: the sample that
+// brackets the threshold (a round trip to HBM), the exchange of the per-CTA partial sums (two more),
+// the fix-up of the listed values, and a handful of CTA-wide barriers per matrix -- 5 to 7 us per
+// matrix, a third of a batch of 2B-shaped matrices and more for small ones.  Here none of that stops
+// the stream:
+//
+//   warps 0..30   stream pass 1 of matrix 0, 1, 2, ... back to back, each thread its fixed share of the
+//                 CTA's range (fixed order of additions: the partial sums are reproducible bit for bit);
+//                 no CTA-wide barrier between matrices.  A warp leaves its sum |W| and flip count of
+//                 matrix m in shared memory and counts itself on `arrived`.
+//   warp 31       the finisher.  For matrix m, in this order:
+//                   bracket of matrix m + 2 (from the caller's hint, or a sample of the matrix);
+//                   wait until the 31 streaming warps have arrived for m, add their sums in a fixed
+//                   order, publish {tag, partial} in the workspace;
+//                   exchange of matrix m - 1 (published by every CTA one matrix ago, so the slots are
+//                   there already), exact gamma, scale, threshold; fix-up of the listed values of
+//                   m - 1, or a note that m - 1 needs the exact second pass; its list becomes free.
+//                 All of it runs under pass 1 of the following matrices.
+//   three lists   matrix m - 1 is being fixed up while m waits and m + 1 is being written; a streaming
+//                 warp starts matrix m only once m - 3 is fixed (its list slot is free) and the bracket
+//                 of m exists -- both normally long done.
+//   tail          after the last matrix every warp joins: exchange and fix-up of the last matrix, then
+//                 the exact second passes that were put off (bracket missed, list overflow, or the
+//                 dense W_q wanted), all threads working.
+//
+// Every wait is bounded; one that runs out raises the CTA's abort flag and the device status word.
+#pragma once
+
+#include "quantize_mask_pack.cuh"
+
+namespace sbn {
+
+constexpr int kQmpStreamWarps = kQmpWarps - 1;             // 31 stream, warp 31 finishes
+constexpr int kQmpLists = 3;
+constexpr int kQmpStreamSmemBytes = kQmpLists * kQmpListCap * 8;
+constexpr int kQmpMaxBatch = 1024;                         // thresholds of put-off second passes live in shared memory
+
+struct QmpStreamShared {
+    double warp_sum[kQmpLists][kQmpWarps];
+    unsigned int warp_flips[kQmpLists][kQmpWarps];
+    unsigned long long flip_total[kQmpLists];
+    unsigned int arrived[kQmpLists];                       // streaming warps done with the matrix in this slot
+    unsigned int list_count[kQmpLists];
+    float bracket[4][2];                                   // [matrix % 4][lo, hi]
+    int bracket_upto;                                      // brackets exist for matrices < bracket_upto
+    int fixed_upto;                                        // matrices < fixed_upto are finished: their list slot is free
+    int abort;
+    float thr_tail;
+    float thr_second_pass[kQmpMaxBatch];                   // >= 0: this matrix needs the exact second pass with this threshold
+};
+
+__device__ __forceinline__ QmpDesc qmp_desc_of(const QmpDesc& first, const QmpDesc* rest, int m) {
+    return m == 0 ? first : rest[m - 1];
+}
+
+// Bounded wait for a shared-memory word (written by another warp of this CTA) to reach `want`.
+__device__ __forceinline__ bool qmp_wait_ge(volatile int* word, int want, volatile int* abort_flag) {
+    if (*word >= want) return true;
+    unsigned long long t0 = 0ull;
+    unsigned int spins = 0;
+    while (*word < want) {
+        __nanosleep(64);
+        if ((++spins & 0x3Fu) == 0u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns_qmp();
+            if (t0 == 0ull) {
+                t0 = now;
+            } else if (now - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// lo / hi of the bracket around the threshold that gamma_est predicts (see quantize_mask_pack.cuh)
+__device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_units, float& lo, float& hi) {
+    const float b = num_units < kQmpSmallMatrixUnits ? kQmpBracketSmall : kQmpBracket;
+    lo = 0.5f * fmaxf(gamma_est * (1.0f - b), kEps) * (1.0f - 1e-6f);
+    hi = 0.5f * fmaxf(gamma_est * (1.0f + b), kEps) * (1.0f + 1e-6f);
+}
+
+// The caller's estimate of gamma, if it gave a usable one.
+__device__ __forceinline__ bool qmp_hint(const QmpDesc& d, float& g) {
+    if (d.gamma_hint == nullptr) return false;
+    g = *reinterpret_cast<const volatile float*>(d.gamma_hint);
+    return g > 0.0f && g < 3.0e38f;
+}
+
+// gamma_est by ONE warp: the same scattered units as qmp_sample_gamma, eight unit loads in flight per
+// lane after the whole sample has been requested into L2.
+template <bool BF16>
+__device__ __forceinline__ float qmp_sample_gamma_warp(const QmpDesc& d, int lane) {
+    constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
+    const uint32_t n_s = qmp_sample_units(d.num_units);
+    const uint32_t stride = d.num_units / n_s;
+    auto unit_of = [&](uint32_t sidx) { return sidx * stride + ((sidx * 2654435761u) >> 8) % stride; };
+    for (uint32_t sidx = lane; sidx < n_s; sidx += 32u)
+        prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(unit_of(sidx)) * kUnitBytes, kUnitBytes);
+    float acc = 0.0f;
+    for (uint32_t base = 0; base < n_s; base += 8u) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            v[i] = base + i < n_s ? qmp_load_group<BF16>(d.W, unit_of(base + i), lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc += (fabsf(v[i].x) + fabsf(v[i].y)) + (fabsf(v[i].z) + fabsf(v[i].w));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    return acc / (static_cast<float>(n_s) * 128.0f);
+}
+
+// Pass 1 of one matrix for the streaming warps: this thread's share of the CTA's range.  Returns the
+// thread's sum |W|; metadata, provisional values, undecided list and flip count as in quantize_mask_pack.cuh.
+// A lane takes two adjacent groups (32 B of a row); a half-warp covers one 512 B unit, the 31 warps 62
+// units per step, two steps per iteration (four independent groups per thread keep the ALUs fed).
+template <bool BF16>
+__device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
+                                                   QmpEntry* list, unsigned int* list_count, unsigned int& flips) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t l16 = lane & 15;
+    const uint32_t KB = d.KB;
+    constexpr uint32_t kStep = 2 * kQmpStreamWarps;
+    constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
+    const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
+    const bool count_flips = d.prev_meta != nullptr;
+    double acc = 0.0;
+    const uint32_t u_first = rg.u_begin + 2 * warp + (lane >> 4);
+    int n_cur = static_cast<int>(u_first / KB);
+    int kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < kQmpPrefetchAhead; ++j) {
+            const uint32_t ub = rg.u_begin + j * 2 * kStep;
+            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
+        }
+    }
+    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += 2 * kStep) {
+        if (threadIdx.x == 0) {
+            const uint32_t ub = u0 + kQmpPrefetchAhead * 2 * kStep;
+            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
+        }
+        float4 va[2], vb[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
+            va[q] = vb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (uq < rg.u_end) qmp_load_group_pair<BF16>(d.W, uq, l16, va[q], vb[q]);
+        }
+        acc += (abs_sum4(va[0]) + abs_sum4(vb[0])) + (abs_sum4(va[1]) + abs_sum4(vb[1]));
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
+            const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+            n_cur += step_n;
+            kb_cur += step_kb;
+            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+            if (uq < rg.u_end) {
+                float k[4];
+                const uint32_t nib0 = select_pair(va[q], k[0], k[1]);
+                const uint32_t nib1 = select_pair(vb[q], k[2], k[3]);
+                const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
+                if (count_flips) {
+                    const uint32_t prev = d.prev_meta[m_off];
+                    flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
+                                    (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
+                }
+                d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
+                const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
+                reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
+                qmp_list_undecided(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
+            }
+        }
+    }
+    return acc;
+}
+
+// What the exact gamma decides for a matrix whose pass 1 is complete: true if the listed values were
+// all that had to be redone (and `fix` should run), false if the whole range must be ternarised again.
+__device__ __forceinline__ bool qmp_bracket_holds(const QmpDesc& d, float thr, float lo, float hi, unsigned int listed) {
+    return lo <= thr && thr <= hi && listed <= static_cast<unsigned int>(kQmpListCap) && d.dense_q == nullptr &&
+           d.num_units <= (1u << 26);                        // listed byte offsets are 32-bit
+}
+
+__global__ void __launch_bounds__(kQmpThreads, 1)
+quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
+                                 QmpSlot* slots, unsigned long long* generation, unsigned long long call_nonce,
+                                 int test_withhold_slot) {
+    extern __shared__ QmpEntry s_list[];                // [kQmpLists][kQmpListCap]
+    __shared__ QmpStreamShared sh;
+    __shared__ double s_warp[kQmpWarps];
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    volatile int* const abort_flag = &sh.abort;
+    if (threadIdx.x == 0) {
+        sh.bracket_upto = 0;
+        sh.fixed_upto = 0;
+        sh.abort = 0;
+        for (int i = 0; i < kQmpLists; ++i) { sh.arrived[i] = 0u; sh.list_count[i] = 0u; sh.flip_total[i] = 0ull; }
+    }
+    for (int i = threadIdx.x; i < kQmpMaxBatch; i += kQmpThreads) sh.thr_second_pass[i] = -1.0f;
+    __syncthreads();
+    // No early signal to the next kernel of the stream: this kernel writes packed weights, and the
+    // GEMM kernels fetch weights before their own dependency wait (see sbn_common.cuh).
+    pdl_wait();
+    const unsigned long long gen0 = *reinterpret_cast<volatile unsigned long long*>(generation);
+    const unsigned long long tag = qmp_tag(call_nonce, gen0);
+
+    // ---- brackets of the first two matrices: all threads
+    for (int m = 0; m < min(count, 2); ++m) {
+        const QmpDesc d = qmp_desc_of(first, rest, m);
+        float g;
+        if (!qmp_hint(d, g)) g = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
+        if (threadIdx.x == 0) qmp_bracket_from(g, d.num_units, sh.bracket[m & 3][0], sh.bracket[m & 3][1]);
+    }
+    if (threadIdx.x == 0) sh.bracket_upto = min(count, 2);
+    __syncthreads();
+
+    if (warp < kQmpStreamWarps) {
+        // ------------------------------------------------------------------ streaming warps
+        for (int m = 0; m < count; ++m) {
+            const int slot = m % kQmpLists;
+            if (!qmp_wait_ge(&sh.bracket_upto, m + 1, abort_flag)) break;
+            if (!qmp_wait_ge(&sh.fixed_upto, m - (kQmpLists - 1), abort_flag)) break;
+            const QmpDesc d = qmp_desc_of(first, rest, m);
+            const QmpRange rg = qmp_range(d);
+            const float lo = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][0]);
+            const float hi = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][1]);
+            unsigned int flips = 0;
+            double mine = d.w_bf16 ? qmp_stream_pass1<true>(d, rg, lo, hi, s_list + slot * kQmpListCap, &sh.list_count[slot], flips)
+                                   : qmp_stream_pass1<false>(d, rg, lo, hi, s_list + slot * kQmpListCap, &sh.list_count[slot], flips);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+                flips += __shfl_xor_sync(0xFFFFFFFFu, flips, o);
+            }
+            __syncwarp();                                    // every lane's list entries are written
+            if (lane == 0) {
+                sh.warp_sum[slot][warp] = mine;
+                sh.warp_flips[slot][warp] = flips;
+                __threadfence_block();                       // the sums, and this warp's list entries, before the count
+                atomicAdd(&sh.arrived[slot], 1u);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------------ the finisher (warp 31)
+        bool ok = true;
+        for (int m = 0; ok && m < count; ++m) {
+            const int slot = m % kQmpLists;
+            // bracket of matrix m + 2, well before the streaming warps ask for it
+            if (m + 2 < count) {
+                const QmpDesc d2 = qmp_desc_of(first, rest, m + 2);
+                float g;
+                if (!qmp_hint(d2, g)) g = d2.w_bf16 ? qmp_sample_gamma_warp<true>(d2, lane) : qmp_sample_gamma_warp<false>(d2, lane);
+                if (lane == 0) {
+                    qmp_bracket_from(g, d2.num_units, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1]);
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int*>(&sh.bracket_upto) = m + 3;
+                }
+                __syncwarp();
+            }
+            // matrix m: every streaming warp has arrived -> this CTA's partial sum, published
+            if (!qmp_wait_ge(reinterpret_cast<volatile int*>(&sh.arrived[slot]), kQmpStreamWarps, abort_flag)) { ok = false; break; }
+            __threadfence_block();
+            const QmpDesc d = qmp_desc_of(first, rest, m);
+            {
+                double v = lane < kQmpStreamWarps ? *reinterpret_cast<volatile double*>(&sh.warp_sum[slot][lane]) : 0.0;
+                unsigned int f = lane < kQmpStreamWarps ? *reinterpret_cast<volatile unsigned int*>(&sh.warp_flips[slot][lane]) : 0u;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+                    f += __shfl_xor_sync(0xFFFFFFFFu, f, o);
+                }
+                if (lane == 0) {
+                    sh.flip_total[slot] = f;
+                    if (blockIdx.x == 0 && d.flip_bits != nullptr) *d.flip_bits = 0ull;
+                    QmpSlot* sl = slots + static_cast<size_t>(m) * gridDim.x + blockIdx.x;
+                    sl->partial = v;
+                    __threadfence();
+                    if (!(test_withhold_slot && blockIdx.x == gridDim.x - 1))
+                        *reinterpret_cast<volatile unsigned long long*>(&sl->nonce) = tag;
+                }
+                __syncwarp();
+            }
+            // matrix m - 1: exchange, exact threshold, fix-up
+            if (m >= 1) {
+                const int pslot = (m - 1) % kQmpLists;
+                const QmpDesc dp = qmp_desc_of(first, rest, m - 1);
+                const QmpSlot* base = slots + static_cast<size_t>(m - 1) * gridDim.x;
+                // a lane looks after the slots lane, lane + 32, ...: all its flags are polled together, then all
+                // its partial sums are read together (two round trips in all, not two per slot)
+                constexpr int kPerLane = (kQmpMaxCtas + 31) / 32;
+                {
+                    unsigned long long t0 = 0ull;
+                    unsigned int spins = 0;
+                    bool seen = false;
+                    while (!seen) {
+                        seen = true;
+#pragma unroll
+                        for (int j = 0; j < kPerLane; ++j) {
+                            const unsigned int i = lane + 32u * j;
+                            if (i < gridDim.x) seen = seen && (*reinterpret_cast<const volatile unsigned long long*>(&base[i].nonce) == tag);
+                        }
+                        if (!seen && ((++spins & 0xFFu) == 0u)) {
+                            if (*abort_flag) break;
+                            const unsigned long long now = global_timer_ns_qmp();
+                            if (t0 == 0ull) t0 = now;
+                            else if (now - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) break;
+                        }
+                    }
+                    if (!seen) ok = false;
+                }
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) {
+                    if (lane == 0) { *abort_flag = 1; atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT)); }
+                    break;
+                }
+                __threadfence();
+                double part[kPerLane];
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j) {
+                    const unsigned int i = lane + 32u * j;
+                    part[j] = i < gridDim.x ? *reinterpret_cast<const volatile double*>(&base[i].partial) : 0.0;
+                }
+                double sum = 0.0;
+#pragma unroll
+                for (int j = 0; j < kPerLane; ++j) sum += part[j];                 // a lane's slots in increasing order
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);    // the same order in every CTA
+                const float gamma = static_cast<float>(sum / (static_cast<double>(dp.num_units) * 128.0));
+                const float scale = fmaxf(gamma, kEps);
+                float thr = 0.0f;
+                if (lane == 0) {
+                    thr = ternary_threshold(scale);
+                    if (blockIdx.x == 0) *dp.w_scale = scale;
+                    if (dp.flip_bits != nullptr && sh.flip_total[pslot] != 0ull) atomicAdd(dp.flip_bits, sh.flip_total[pslot]);
+                }
+                thr = __shfl_sync(0xFFFFFFFFu, thr, 0);
+                const unsigned int listed = *reinterpret_cast<volatile unsigned int*>(&sh.list_count[pslot]);
+                if (qmp_bracket_holds(dp, thr, sh.bracket[(m - 1) & 3][0], sh.bracket[(m - 1) & 3][1], listed)) {
+                    const QmpEntry* list = s_list + pslot * kQmpListCap;
+                    uint8_t* vb = reinterpret_cast<uint8_t*>(dp.vals);
+                    for (unsigned int e = lane; e < listed; e += 32u) {
+                        const float w = list[e].w;
+                        vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
+                    }
+                } else if (lane == 0) {
+                    sh.thr_second_pass[m - 1] = thr;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    sh.arrived[pslot] = 0u;
+                    sh.list_count[pslot] = 0u;
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int*>(&sh.fixed_upto) = m;
+                }
+                __syncwarp();
+            }
+        }
+    }
+    __syncthreads();
+    if (sh.abort) return;
+
+    // ---- tail: the last matrix, all threads
+    {
+        const int m = count - 1;
+        const int slot = m % kQmpLists;
+        const QmpDesc d = qmp_desc_of(first, rest, m);
+        const QmpRange rg = qmp_range(d);
+        const QmpSlot* base = slots + static_cast<size_t>(m) * gridDim.x;
+        double other = 0.0;
+        if (threadIdx.x < gridDim.x) {
+            const volatile unsigned long long* flag = &base[threadIdx.x].nonce;
+            unsigned long long t0 = 0ull;
+            unsigned int spins = 0;
+            bool seen = (*flag == tag);
+            while (!seen) {
+                seen = (*flag == tag);
+                if (!seen && ((++spins & 0xFFu) == 0u)) {
+                    const unsigned long long now = global_timer_ns_qmp();
+                    if (t0 == 0ull) t0 = now;
+                    else if (now - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) break;
+                }
+            }
+            if (seen) {
+                __threadfence();
+                other = *reinterpret_cast<const volatile double*>(&base[threadIdx.x].partial);
+            } else {
+                sh.abort = 1;
+                atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+            }
+        }
+        const double S = qmp_block_sum(other, s_warp);          // fixed order: the same bits in every CTA
+        if (sh.abort) return;                                    // a peer never arrived: give up cleanly
+        if (threadIdx.x == 0 && d.flip_bits != nullptr && sh.flip_total[slot] != 0ull) atomicAdd(d.flip_bits, sh.flip_total[slot]);
+        const float gamma = static_cast<float>(S / (static_cast<double>(d.num_units) * 128.0));
+        const float scale = fmaxf(gamma, kEps);
+        if (threadIdx.x == 0) {
+            sh.thr_tail = ternary_threshold(scale);
+            if (blockIdx.x == 0) *d.w_scale = scale;
+        }
+        __syncthreads();
+        const float thr = sh.thr_tail;
+        const unsigned int listed = sh.list_count[slot];
+        if (qmp_bracket_holds(d, thr, sh.bracket[m & 3][0], sh.bracket[m & 3][1], listed)) {
+            const QmpEntry* list = s_list + slot * kQmpListCap;
+            uint8_t* vb = reinterpret_cast<uint8_t*>(d.vals);
+            for (unsigned int e = threadIdx.x; e < listed; e += kQmpThreads) {
+                const float w = list[e].w;
+                vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
+            }
+        } else {
+            if (d.w_bf16) qmp_pass2_full<true>(d, rg, thr);
+            else qmp_pass2_full<false>(d, rg, thr);
+        }
+    }
+    // ---- the second passes that were put off
+    for (int m = 0; m + 1 < count; ++m) {
+        const float thr = sh.thr_second_pass[m];
+        if (thr >= 0.0f) {
+            const QmpDesc d = qmp_desc_of(first, rest, m);
+            const QmpRange rg = qmp_range(d);
+            if (d.w_bf16) qmp_pass2_full<true>(d, rg, thr);
+            else qmp_pass2_full<false>(d, rg, thr);
+        }
+    }
+    // every CTA has published its last slot (CTA 0 has just read them all), hence has read the generation
+    if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<volatile unsigned long long*>(generation) = gen0 + 1ull;
+}
+
+// Launch for `count` (<= kQmpMaxBatch) matrices: `first` by value, the others already copied to `rest_dev`.
+inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const QmpDesc* rest_dev, int count,
+                                                   uint32_t max_units, QmpSlot* slots, unsigned long long* generation,
+                                                   cudaStream_t stream) {
+    const int test_withhold_slot = g_test_break_waits;
+    const unsigned long long nonce = qmp_next_nonce();
+    // every CTA must be resident at once (they exchange partial sums): never more CTAs than this
+    // device has SMs, and never more than the workspace has slots
+    const unsigned cap = static_cast<unsigned>(std::min(device_sm_count(), kQmpMaxCtas));
+    const unsigned grid = max_units < cap ? max_units : cap;
+    if (!ensure_dynamic_smem<quantize_mask_pack_stream_kernel>(kQmpStreamSmemBytes)) return SBN_ERR_CUDA;
+    // At most one CTA per SM (1024 threads x 64 registers each) and never more CTAs than SMs, so all
+    // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
+    // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
+    const cudaError_t err = launch_kernel(quantize_mask_pack_stream_kernel, dim3(grid), dim3(kQmpThreads), kQmpStreamSmemBytes, stream,
+                                          first, rest_dev, count, slots, generation, nonce, test_withhold_slot);
+    ++g_launch_count;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
+inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, int K, int8_t* vals,
+                                            uint8_t* meta, float* w_scale, int8_t* dense_q,
+                                            const uint8_t* prev_meta,
+                                            unsigned long long* flip_bits, QmpWorkspace* ws,
+                                            cudaStream_t stream) {
+    const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
+    return launch_quantize_mask_pack_stream(d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream);
+}
+
+}  // namespace sbn
