@@ -514,6 +514,22 @@ def run_ours(args):
         row["quantize_mask_pack_gbs"] = round(L.N * L.K * (L.w_bytes + 0.625) / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
         row["quant_act_us"] = round(act, 2)
         row["quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act / 1e3, 1)
+        # the same kernel launched back to back over 8 distinct inputs (more than the L2 holds): what a
+        # launch costs inside a stream of kernels, without the ~6 us an isolated launch spends between two events
+        xs = [L.x] + [torch.empty_like(L.x).copy_(L.x) for _ in range(7)]
+        torch.cuda.synchronize()
+        torch.cuda._sleep(int(4e6))
+        ea, ec = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ea.record(stream)
+        for r_i in range(32):
+            b.sbn_quant_act(xs[r_i % 8], L.xq, L.a_scale)
+        ec.record(stream)
+        torch.cuda.synchronize()
+        act_st = ea.elapsed_time(ec) * 1e3 / 32
+        del xs
+        row["quant_act_stream_us"] = round(act_st, 2)
+        row["quant_act_stream_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act_st / 1e3, 1)
+        row["quant_act_stream_frac_of_hbm"] = round((L.T * L.K * 3 + L.T * 4) / act_st / 1e3 / peaks["hbm_gbs"], 4)
         if L.K <= 16384:
             # Algorithm 1's x~ = Q_a(Norm(x)) as one kernel (RMSNorm with gain fused into the quantiser)
             nact = time_cold(lambda: b.sbn_norm_quant_act(L.x, L.xq, L.a_scale, gain=L.gain, eps=1e-6), iters)

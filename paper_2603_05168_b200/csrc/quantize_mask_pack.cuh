@@ -4,7 +4,9 @@
 // gamma needs the whole matrix before any element can be rounded, but almost every element can be
 // rounded correctly from an ESTIMATE of gamma: W_q = sign(w) [ |w| >= thr(gamma) ] and only the
 // few |w| that lie within a few percent of thr depend on its exact value.  One persistent kernel
-// (one 1024-thread CTA per SM) therefore reads W ONCE, for one matrix or a batch of them:
+// (one 1024-thread CTA per SM) therefore reads W ONCE, for one matrix or a batch of them.  This file
+// holds the building blocks and the phase-by-phase kernel that the 6:8 pattern uses; the 2:4 pattern
+// runs the same phases as one uninterrupted stream (quantize_mask_pack_stream.cuh).  The phases:
 //
 //   sample   every CTA adds |w| over the same 256 scattered 512 B units of the matrix (128 KB,
 //            L2-served for all CTAs but the first; 64 units for matrices below 33 M weights)
@@ -260,77 +262,6 @@ __device__ __forceinline__ void qmp_list_undecided(const float (&k)[4], const fl
     }
 }
 
-// pass 1 of one matrix: returns this CTA's sum |W| (identical in every thread); writes the metadata
-// and the provisional vals, lists the undecided kept values and accumulates the flip count.
-// A lane takes TWO adjacent groups (32 B of a row), so it owns a whole metadata byte and four
-// consecutive bytes of vals and the per-unit index arithmetic is shared by two groups; a half-warp
-// covers one 512 B unit, a warp two units per load pair and four per iteration.
-template <bool BF16>
-__device__ __forceinline__ double qmp_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
-                                            QmpEntry* list, unsigned int* list_count, double* s_warp,
-                                            unsigned int& flips) {
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const uint32_t l16 = lane & 15;
-    const uint32_t KB = d.KB;
-    constexpr uint32_t kStep = 2 * kQmpWarps;                // units between a thread's consecutive units
-    constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
-    const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
-    const bool count_flips = d.prev_meta != nullptr;
-    double acc = 0.0;
-    const uint32_t u_first = rg.u_begin + 2 * warp + (lane >> 4);
-    int n_cur = static_cast<int>(u_first / KB);
-    int kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
-    // One thread keeps the L2 a few iterations ahead of the loads (the CTA's range is contiguous),
-    // so the loads in flight per SM do not have to cover the whole HBM latency.
-    if (threadIdx.x == 0) {
-        for (int j = 1; j < kQmpPrefetchAhead; ++j) {
-            const uint32_t ub = rg.u_begin + j * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
-        }
-    }
-    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += 2 * kStep) {
-        if (threadIdx.x == 0) {
-            const uint32_t ub = u0 + kQmpPrefetchAhead * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
-        }
-        float4 va[2], vb[2];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {                     // four independent 16 B loads in flight
-            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
-            va[q] = vb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (uq < rg.u_end) qmp_load_group_pair<BF16>(d.W, uq, l16, va[q], vb[q]);
-        }
-        acc += (abs_sum4(va[0]) + abs_sum4(vb[0])) + (abs_sum4(va[1]) + abs_sum4(vb[1]));
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
-            const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
-            n_cur += step_n;
-            kb_cur += step_kb;
-            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
-            if (uq < rg.u_end) {
-                float k[4];
-                const uint32_t nib0 = select_pair(va[q], k[0], k[1]);
-                const uint32_t nib1 = select_pair(vb[q], k[2], k[3]);
-                const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
-                if (count_flips) {
-                    const uint32_t prev = d.prev_meta[m_off];
-                    flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
-                                    (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
-                }
-                d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
-                // provisional Eq. 1 + Eq. 3: compressed columns 4*l16 .. 4*l16+3 of this 64 B tile row
-                const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
-                reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
-                qmp_list_undecided(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
-            }
-        }
-    }
-    return qmp_block_sum(acc, s_warp);
-}
-
 // Ternarise a whole range again with the exact threshold (the path taken when the bracket missed,
 // the list overflowed or the dense W_q is wanted): a warp per unit, four units at a time, newest
 // first (what pass 1 read last is still in L2).
@@ -388,7 +319,7 @@ __device__ __forceinline__ double qmp68_pass(const QmpDesc& d, const QmpRange rg
 // so by the time a CTA needs gamma of matrix m, every CTA has long published its partial for m,
 // and the per-launch and per-exchange latencies are paid once per batch, not once per matrix.
 // The two undecided lists alternate between consecutive matrices.  `first` is matrix 0 (passed by
-// value), `rest` matrices 1.. in global memory.  PATTERN: 24 or 68 (all matrices of a batch alike).
+// value), `rest` matrices 1.. in global memory.  PATTERN: 68 (the 2:4 pattern has its own kernel).
 template <int PATTERN>
 __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
@@ -437,19 +368,12 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
             __syncthreads();
             unsigned int flips = 0;
             double mine;
-            if constexpr (PATTERN == 68) {
-                mine = d_cur.w_bf16
-                    ? qmp68_pass<true, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                              &s_list_count[par], s_warp, flips)
-                    : qmp68_pass<false, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                               &s_list_count[par], s_warp, flips);
-            } else {
-                mine = d_cur.w_bf16
-                    ? qmp_pass1<true>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                      &s_list_count[par], s_warp, flips)
-                    : qmp_pass1<false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
-                                       &s_list_count[par], s_warp, flips);
-            }
+            static_assert(PATTERN == 68, "the 2:4 pattern runs in quantize_mask_pack_stream_kernel");
+            mine = d_cur.w_bf16
+                ? qmp68_pass<true, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                          &s_list_count[par], s_warp, flips)
+                : qmp68_pass<false, false>(d_cur, rg_cur, s_bracket[par][0], s_bracket[par][1], s_list + par * kQmpListCap,
+                                           &s_list_count[par], s_warp, flips);
             // this CTA's flip count of matrix m; it is added to the global counter one phase later,
             // after the exchange has shown that CTA 0 zeroed that counter
 #pragma unroll
@@ -520,13 +444,10 @@ quantize_mask_pack_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest,
                     const float w = list[e].w;
                     vb[list[e].byte_off] = static_cast<uint8_t>(fabsf(w) >= thr ? (w < 0.0f ? 0xFFu : 0x01u) : 0u);
                 }
-            } else if constexpr (PATTERN == 68) {
+            } else {
                 unsigned int unused = 0;
                 if (d_prev.w_bf16) qmp68_pass<true, true>(d_prev, rg_prev, thr, thr, nullptr, nullptr, s_warp, unused);
                 else qmp68_pass<false, true>(d_prev, rg_prev, thr, thr, nullptr, nullptr, s_warp, unused);
-            } else {
-                if (d_prev.w_bf16) qmp_pass2_full<true>(d_prev, rg_prev, thr);
-                else qmp_pass2_full<false>(d_prev, rg_prev, thr);
             }
             __syncthreads();                                     // s_thr / this list may be reused
         }
@@ -577,7 +498,7 @@ inline QmpDesc qmp_make_desc(const void* W, bool w_bf16, int N, int K, int8_t* v
 }
 
 // Launch for `count` matrices: `first` by value, the others already copied to `rest_dev`.
-template <int PATTERN = 24>
+template <int PATTERN>
 inline sbn_status launch_quantize_mask_pack_batch(const QmpDesc& first, const QmpDesc* rest_dev, int count,
                                                   uint32_t max_units, QmpSlot* slots, unsigned long long* generation,
                                                   cudaStream_t stream) {

@@ -1028,3 +1028,69 @@ def test_pack_wait_runs_out_and_the_library_recovers():
     g = gpu_quantize_mask_pack(W, with_dense=False)
     assert g["scale"] == r["scale"]
     assert np.array_equal(g["vals"], r["vals"]) and np.array_equal(g["meta"], r["meta"])
+
+
+# ---- the streaming pack kernel: hints and very long batches ------------------------------------------------
+@pytest.mark.parametrize("hint_factor", [1.0, 1.02, 2.0, 0.0, -1.0, float("inf")])
+def test_quantize_mask_pack_gamma_hint_never_changes_the_result(hint_factor):
+    # the hint only decides whether the kernel samples the matrix and whether the bracket holds
+    # (a hint far off sends the matrix through the exact second pass): the bytes must not change
+    shapes = [(256, 2560), (640, 256), (128, 128), (384, 1280), (2560, 640), (128, 6912)]
+    Ws = [inputs.latent_weights(N, K, seed=160 + i, sigma=0.02 * (i + 1)) for i, (N, K) in enumerate(shapes)]
+    refs = [_oracle_pack(W) for W in Ws]
+    jobs = []
+    for W, r in zip(Ws, refs):
+        N, K = W.shape
+        bufs = b.alloc_packed(N, K)
+        hint = torch.tensor([float(r["scale"]) * hint_factor], dtype=torch.float32, device="cuda")
+        jobs.append(dict(W=dev(W), vals=bufs["vals"], meta=bufs["meta"], w_scale=bufs["w_scale"], gamma_hint=hint))
+    arr = b.make_pack_jobs(jobs)
+    ws = torch.empty(b.sbn_batch_workspace_bytes(len(jobs)), dtype=torch.uint8, device="cuda")
+    b.sbn_quantize_mask_pack_batched(arr, ws)
+    b.sbn_check_status()
+    for job, W, r in zip(jobs, Ws, refs):
+        N, K = W.shape
+        vals, meta = gpu_unpack_canonical(job, N, K)
+        assert np.float32(job["w_scale"].cpu().numpy()[0]) == r["scale"]
+        assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"])
+
+
+def test_quantize_mask_pack_hint_in_the_scale_buffer_over_steps():
+    # the intended use: w_scale of the previous step is this step's hint, in place, while W drifts
+    N, K = 1024, 2560
+    W = inputs.latent_weights(N, K, seed=170)
+    bufs = b.alloc_packed(N, K)
+    bufs["w_scale"].fill_(float("nan"))                          # first step: no usable hint yet
+    Wd = dev(W)
+    arr = b.make_pack_jobs([dict(W=Wd, vals=bufs["vals"], meta=bufs["meta"], w_scale=bufs["w_scale"], gamma_hint=bufs["w_scale"])])
+    ws = torch.empty(b.sbn_batch_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    for step in range(4):
+        b.sbn_quantize_mask_pack_batched(arr, ws)
+        b.sbn_check_status()
+        r = _oracle_pack(W)
+        vals, meta = gpu_unpack_canonical(bufs, N, K)
+        assert np.float32(bufs["w_scale"].cpu().numpy()[0]) == r["scale"], step
+        assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"]), step
+        W = inputs.perturb_weights(W, seed=171 + step, sigma=1e-4 if step < 2 else 5e-3)   # the last drift breaks the bracket
+        Wd.copy_(torch.from_numpy(W))
+
+
+def test_quantize_mask_pack_batch_longer_than_one_launch_holds():
+    # more jobs than one launch of the kernel takes (its per-matrix state on chip is finite): the call
+    # splits the batch; every job must still equal the single call
+    count = 1030
+    base = inputs.latent_weights(128, 128 * count, seed=180).reshape(128, count, 128).transpose(1, 0, 2)
+    Ws = [np.ascontiguousarray(base[i]) * np.float32(1 + (i % 7)) for i in range(count)]
+    big = {k: torch.empty((count,) + shape, dtype=dt, device="cuda")
+           for k, shape, dt in (("vals", (128, 64), torch.int8), ("meta", (128, 16), torch.uint8), ("w_scale", (1,), torch.float32))}
+    Wd = torch.from_numpy(np.stack(Ws)).cuda()
+    jobs = [dict(W=Wd[i], vals=big["vals"][i], meta=big["meta"][i], w_scale=big["w_scale"][i]) for i in range(count)]
+    arr = b.make_pack_jobs(jobs)
+    ws = torch.empty(b.sbn_batch_workspace_bytes(count), dtype=torch.uint8, device="cuda")
+    b.sbn_quantize_mask_pack_batched(arr, ws)
+    b.sbn_check_status()
+    for i in list(range(0, count, 97)) + [1023, 1024, 1025, count - 1]:
+        r = _oracle_pack(Ws[i])
+        vals, meta = gpu_unpack_canonical(dict(vals=big["vals"][i], meta=big["meta"][i]), 128, 128)
+        assert np.float32(big["w_scale"][i].cpu().numpy()[0]) == r["scale"], i
+        assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"]), i
