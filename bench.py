@@ -992,6 +992,85 @@ def run_dynamic_step(args):
         "gpu_launches": b.sbn_launch_count()}))
 
 
+def run_mma_probe(args):
+    """What the K-loop of the large-T GEMM kernel costs, piece by piece (timing only: with a probe flag set
+    the kernel's results are wrong).  One tile per CTA pair (74 feature tiles x one token tile), so nothing
+    but the K-loop grows with K (two feature tiles x 37 token tiles, so operands are shared between pairs
+    through the L2 as in a real layer); the time per 128-column block is the slope between K = 2560 and K = 11008.
+    Modes: all loads | operands resident after the first fill | no loads | no loads and no metadata copies |
+    no loads, every MMA issued twice / four times (the extra MMAs re-read operands the tensor core has just
+    used: their marginal cost is the pipe's own pace)."""
+    import torch
+    from paper_2603_05168_b200 import binding as b
+    from paper_2603_05168_b200 import build as sbn_build
+    sbn_build.build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    stream = torch.cuda.current_stream()
+    K1, K2 = 2560, 11008
+    modes = [("all loads", 0), ("resident", 1), ("no loads", 6), ("no loads, no metadata copies", 14),
+             ("no loads, MMAs x2", 14 + 16), ("no loads, MMAs x4", 14 + 32)]
+    rows = []
+
+    def timed(fn, reps=6):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            c.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(c) * 1e3)
+        return statistics.median(ts)
+
+    for sparse in (True, False):
+        for mt in (1, 2):
+            N = 2 * 256 * mt
+            bufs = {}
+            for K in (K1, K2):
+                w = (torch.zeros((N, K // 2), dtype=torch.int8, device="cuda"), torch.full((N, K // 8), 0x44, dtype=torch.uint8, device="cuda")) \
+                    if sparse else (torch.zeros((N, K), dtype=torch.int8, device="cuda"), None)
+                bufs[K] = w
+            w_scale = torch.ones(1, dtype=torch.float32, device="cuda")
+            for bn in (64, 128, 240):
+                T = 37 * bn
+                b.sbn_set_gemm_tuning(-bn, 1 if mt == 1 else 0)
+                y = torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+                a_scale = torch.ones(T, dtype=torch.float32, device="cuda")
+                xq = {K: torch.zeros(b.sbn_xq_bytes(T, K), dtype=torch.int8, device="cuda") for K in (K1, K2)}
+                for name, flags in modes:
+                    if not sparse and (flags & 8) and not (flags & 48):
+                        continue                                   # the dense kernel has no metadata copies
+                    b.sbn_set_gemm_probe(flags)
+                    t = {}
+                    for K in (K1, K2):
+                        if sparse:
+                            fn = lambda K=K: b.sbn_sparse_bitlinear(xq[K], a_scale, bufs[K][0], bufs[K][1], w_scale, y)
+                        else:
+                            fn = lambda K=K: b.sbn_bitlinear(xq[K], a_scale, bufs[K][0], w_scale, y)
+                        t[K] = timed(fn)
+                    b.sbn_set_gemm_probe(0)
+                    us_kb = (t[K2] - t[K1]) / ((K2 - K1) / 128)
+                    reps = 4 if flags & 32 else (2 if flags & 16 else 1)
+                    mmas_per_kb = (2 if sparse else 4) * mt * reps
+                    rows.append({"kernel": ("sparse" if sparse else "dense") + f", {mt} M-tile(s) per CTA", "tokens_per_tile": bn, "mode": name,
+                                 "us_per_128_columns": round(us_kb, 4), "mmas_per_128_columns": mmas_per_kb,
+                                 "clocks_per_mma_at_1965mhz": round(us_kb * 1965.0 / mmas_per_kb, 1),
+                                 "us_K2560": round(t[K1], 2), "us_K11008": round(t[K2], 2)})
+                b.sbn_set_gemm_tuning(0, 0)
+            del bufs
+            torch.cuda.empty_cache()
+    b.sbn_check_status()
+    print(json.dumps({"metric": "K-loop cost of the CTA-pair GEMM kernel per 128 columns, by parts (timing experiments)", "unit": "us",
+                      "workload": "mmaprobe", "note": "one tile per CTA pair (2 feature tiles x 37 token tiles); slope between K = 2560 and K = 11008; the math of one MMA "
+                      "(M = 256 per pair, N tokens, K = 64 sparse / 32 dense) takes 128 clocks at N = 256 at the datasheet rate",
+                      "rows": rows, "gpu_launches": b.sbn_launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -1001,12 +1080,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="headline line only: skip the 7B-class isolated GEMMs, the sustained run and the few-token rows")
-    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68"],
+    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68", "mmaprobe"],
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1..512), sparse vs dense, cold L2 and streamed; "
                          "decode7b = the same on 7B-class matrices at T <= 64, with the 2-bit packed weights as a third arm; "
                          "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048; "
-                         "p68 = the 6:8 pattern next to 2:4 and dense on the same matrices")
+                         "p68 = the 6:8 pattern next to 2:4 and dense on the same matrices; "
+                         "mmaprobe = timing experiments on the large-T kernel's K-loop (loads, metadata copies, MMA issue)")
     ap.add_argument("--masters", default="fp32", choices=["fp32", "bf16"],
                     help="precision of the master weights the pack kernel reads (default fp32, the configuration of the metric)")
     ap.add_argument("--only-step", action="store_true", help="time the step only (used for profiler runs)")
@@ -1019,6 +1099,8 @@ def main():
         run_dynamic_step(args)
     elif args.workload == "p68":
         run_pattern68(args)
+    elif args.workload == "mmaprobe":
+        run_mma_probe(args)
     else:
         run_ours(args)
 

@@ -416,6 +416,14 @@ void sbn_set_gemm_tuning(int token_tile, int split_k);
  * SBN_ERR_TIMEOUT.  sbn_set_wait_test(0, 0) restores normal operation. */
 sbn_status sbn_set_wait_test(int break_waits, unsigned long long wait_limit_us);
 
+/* Diagnostic for timing experiments on the large-T (CTA-pair) GEMM kernel: what its K-loop costs without
+ * parts of itself.  RESULTS ARE WRONG while flags != 0 -- timing only; 0 restores normal operation.
+ * Host state, not thread-safe.  Bits: 1 = operands stay resident in shared memory (loads only for the
+ * first pipeline fill of a launch), 2 = never load weights and metadata, 4 = never load activations,
+ * 8 = no metadata copies into tensor memory, 16 / 32 = issue every stage's MMAs twice / four times.
+ * Used by `bench.py --workload mmaprobe`. */
+void sbn_set_gemm_probe(int flags);
+
 /* Diagnostic: what the dispatcher would run for this shape (host only, launches nothing).
  * out4[0] = kernel (0 single-CTA tiles, 1 cluster split-K, 2 CTA pair with 512-feature tiles, 3 CTA
  * pair with 256-feature tiles and double-buffered accumulators), out4[1] = tokens per tile,

@@ -25,7 +25,7 @@ EXPORTS = [
     "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed", "sbn_quant_act_sparse_bitlinear", "sbn_quant_act_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count", "sbn_unpack_canonical", "sbn_tile_canonical",
-    "sbn_set_wait_test",
+    "sbn_set_wait_test", "sbn_set_gemm_probe",
 ]
 
 _lib = None
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_unpack_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.sbn_tile_canonical.restype = i32
         L.sbn_tile_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.sbn_set_gemm_probe.restype = None
+        L.sbn_set_gemm_probe.argtypes = [i32]
         L.sbn_set_wait_test.restype = i32
         L.sbn_set_wait_test.argtypes = [i32, ctypes.c_ulonglong]
         L.sbn_launch_count.restype = ctypes.c_ulonglong
@@ -299,6 +301,11 @@ def sbn_tile_canonical(vals_plain, meta_plain, N: int, K: int, vals, meta):
 
 def sbn_set_wait_test(break_waits: bool = False, wait_limit_us: int = 0):
     _check(lib().sbn_set_wait_test(1 if break_waits else 0, int(wait_limit_us)), "sbn_set_wait_test")
+
+
+def sbn_set_gemm_probe(flags: int = 0):
+    """Timing experiments on the CTA-pair GEMM (results are wrong while flags != 0); see sbn.h."""
+    lib().sbn_set_gemm_probe(int(flags))
 
 
 def sbn_check_status():

@@ -384,6 +384,28 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                 for (int ks = 0; ks < k_stages; ++ks) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full_leader = map_to_cta(bar_full + 8 * stage, 0);
+                    if (p.probe) {                      // timing experiments (sbn_set_gemm_probe): leave loads out
+                        if ((p.probe & kProbeResident) && (tile != pair_id || ks >= STAGES)) {
+                            if (rank == 0) mbar_arrive(bar_full + 8 * stage);
+                            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                            continue;
+                        }
+                        const uint32_t skip = ((p.probe & kProbeNoWeights) ? static_cast<uint32_t>(Cfg::A_BYTES + Cfg::E_BYTES) : 0u) +
+                                              ((p.probe & kProbeNoActs) ? static_cast<uint32_t>(KBS * half_bn * kBK) : 0u);
+                        if (rank == 0) {
+                            if (bytes_per_cta > skip) mbar_expect_tx(bar_full + 8 * stage, 2 * (bytes_per_cta - skip));
+                            else mbar_arrive(bar_full + 8 * stage);
+                        }
+                        const uint32_t st_p = smem_stage0 + stage * Cfg::STAGE_BYTES;
+                        const int kb_p = ks * KBS;
+                        if (!(p.probe & kProbeNoWeights)) {
+                            tma_load_3d_pair(st_p, &tmap_a, 0, kb_p * A_ROWS, nb0, full_leader);
+                            if constexpr (SPARSE) tma_load_3d_pair(st_p + Cfg::A_BYTES, &tmap_e, 0, kb_p * 2, nb0, full_leader);
+                        }
+                        if (!(p.probe & kProbeNoActs)) tma_load_3d_pair(st_p + Cfg::A_BYTES + Cfg::E_BYTES, &tmap_b, 0, t_atom, kb_p, full_leader);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * bytes_per_cta);
                     const uint32_t st = smem_stage0 + stage * Cfg::STAGE_BYTES;
                     const int kb = ks * KBS;
@@ -433,10 +455,12 @@ bitlinear_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                 e_tmem[i] = tmem_base + static_cast<uint32_t>(i * 256 + 256 - 8 * e_slots + 8 * (e_slot % e_slots));
                                 const uint64_t e_desc = make_smem_desc(st + Cfg::A_BYTES + static_cast<uint32_t>(i * KBS * Cfg::E_TILE),
                                                                        Cfg::E_TILE, 128, kSwzNone);
-                                tcgen05_cp_128x256b_pair(e_tmem[i], e_desc);
+                                if (!(p.probe & kProbeNoMetaCopy)) tcgen05_cp_128x256b_pair(e_tmem[i], e_desc);
                             }
                             ++e_slot;
                         }
+                        const int mma_reps = (p.probe & kProbeMma4) ? 4 : ((p.probe & kProbeMma2) ? 2 : 1);     // 1 outside timing experiments
+                        for (int rp = 0; rp < mma_reps; ++rp)
                         for (int j = 0; j < kb_live; ++j) {
                             const uint32_t b_addr = st + Cfg::A_BYTES + Cfg::E_BYTES + static_cast<uint32_t>(j) * b_kb_bytes;
                             const uint64_t b_desc = make_smem_desc(b_addr, 16, 1024, kSwz128);

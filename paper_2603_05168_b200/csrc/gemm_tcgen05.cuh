@@ -61,7 +61,16 @@ struct GemmParams {
     int w_tile_bytes;            // bytes of one 128 x 128 weight tile (8192 sparse, 16384 dense)
     int test_skip_loads = 0;     // diagnostics (sbn_set_wait_test): the TMA producer issues no loads, so the
                                  //   consumers' bounded waits run out and every role leaves through the abort flag
+    int probe = 0;               // diagnostics (sbn_set_gemm_probe, CTA-pair kernel, timing only -- results are wrong):
+                                 //   kProbe* bits below
 };
+// Probe bits: what the K-loop costs without parts of itself.
+constexpr int kProbeResident = 1;     // operands stay in shared memory: loads only for the first STAGES stages of a launch
+constexpr int kProbeNoWeights = 2;    // never load weights / metadata
+constexpr int kProbeNoActs = 4;       // never load activations
+constexpr int kProbeNoMetaCopy = 8;   // no metadata copies into tensor memory
+constexpr int kProbeMma2 = 16;        // issue every stage's MMAs twice
+constexpr int kProbeMma4 = 32;        // ... four times
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers

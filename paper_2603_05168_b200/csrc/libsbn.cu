@@ -348,6 +348,7 @@ static sbn_status run_gemm_pair(bool sparse, const int8_t* xq, const float* a_sc
     pp.g.split_acc = nullptr; pp.g.split_counters = nullptr;
     pp.g.w_vals = wvals; pp.g.w_meta = sparse ? meta : nullptr; pp.g.w_tile_bytes = sparse ? 8192 : 16384;
     pp.g.test_skip_loads = g_test_break_waits;
+    pp.g.probe = g_gemm_probe;
     pp.bn = bn;
     if (mt == 1) return sparse ? launch_pair<true, 1>(ta, tb, te, pp, stream) : launch_pair<false, 1>(ta, tb, te, pp, stream);
     return sparse ? launch_pair<true, 2>(ta, tb, te, pp, stream) : launch_pair<false, 2>(ta, tb, te, pp, stream);
@@ -895,6 +896,8 @@ sbn_status sbn_set_wait_test(int break_waits, unsigned long long wait_limit_us) 
     g_test_break_waits = break_waits ? 1 : 0;
     return SBN_OK;
 }
+
+void sbn_set_gemm_probe(int flags) { g_gemm_probe = flags; }
 
 void sbn_set_gemm_tuning(int token_tile, int split_k) {
     g_force_token_tile = token_tile;

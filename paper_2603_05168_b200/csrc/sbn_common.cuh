@@ -27,6 +27,8 @@ __device__ unsigned long long g_wait_limit_ns = kWaitLimitNs;
 // Host state of sbn_set_wait_test: non-zero makes the producers of the GEMM kernels issue no loads and
 // the last CTA of the pack kernel withhold its partial sum -- the consumers' waits then run out.
 static int g_test_break_waits = 0;
+// Host state of sbn_set_gemm_probe (timing experiments on the CTA-pair kernel; 0 = normal operation).
+static int g_gemm_probe = 0;
 
 // Host-side count of kernel launches made by the library.
 static std::atomic<unsigned long long> g_launch_count{0ull};
