@@ -328,3 +328,52 @@ def bitlinear(xq, a_scale, dense_q, scale, bias=None):
     """Dense BitLinear (Sec. 2.1): returns (y, acc)."""
     acc = acc_dense(xq, dense_q)
     return dequant(acc, scale, a_scale, bias), acc
+
+
+# ------------------------------------------------------------------------------------------------
+# Backward of the layer under the dual straight-through estimator (Sec. 2.3, Eq. 5: the mask and the
+# quantiser are both transparent to the gradient; Algorithm 1, "Backward"; Algorithm 2's backward,
+# which returns g_out unchanged, so the weight gradient is the plain, DENSE gradient of F.linear).
+#
+# With y = F.linear(x_q, w_masked), x_q = x~ * a_scale[t] the fake-quantised activations and
+# w_masked = W_eff * scale, autograd of the linear map gives
+#     dW[n][k] = sum_t dY[t][n] * x_q[t][k]         -- reaches every master weight, pruned ones too
+#     dX[t][k] = sum_n dY[t][n] * w_masked[n][k]    -- through Q_a as the identity
+# Precision (the paper names none; its models are trained with bf16 tensors): dY arrives in bf16, the
+# two saved operands are rounded to bf16 as a bf16 training run holds them, x_q_b = bf16(x~ * a_scale)
+# and w_b = W_eff * bf16(scale) (exact, W_eff is ternary); the sums below are over those values, here
+# in float64 (numpy matmul), so what the kernels may differ by is their fp32 accumulation order only.
+# ------------------------------------------------------------------------------------------------
+def bf16_bits_to_f64(bits):
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def bf16_round(a):
+    """fp32 array -> the nearest bf16 values (ties to even), returned as float64."""
+    return bf16_bits_to_f64(f32_to_bf16_bits(np.ascontiguousarray(a, dtype=np.float32)))
+
+
+def fake_quant_act_bf16(xq, a_scale):
+    """x_q_b[t][k] = bf16(float(x~[t][k]) * a_scale[t]) -- one fp32 product, one rounding."""
+    xq = _c(xq, np.int8)
+    a_scale = _c(a_scale, np.float32)
+    return bf16_round(xq.astype(np.float32) * a_scale[:, None])
+
+
+def backward_dw(dy_bf16_bits, xq, a_scale):
+    """Eq. 5 / Algorithm 2's backward: dW = dY^T x_q_b, dense [N][K] (float64)."""
+    dY = bf16_bits_to_f64(dy_bf16_bits)
+    return dY.T @ fake_quant_act_bf16(xq, a_scale)
+
+
+def backward_dx(dy_bf16_bits, w_eff, scale):
+    """dX = dY w_b with w_b = W_eff * bf16(scale): [T][K] (float64)."""
+    dY = bf16_bits_to_f64(dy_bf16_bits)
+    s_b = float(bf16_round(np.array([scale], np.float32))[0])
+    return (dY @ _c(w_eff, np.int8).astype(np.float64)) * s_b
+
+
+def backward_dual_ste(dy_bf16_bits, xq, a_scale, w_eff, scale):
+    """Both gradients of one Sparse-BitLinear layer: (dX [T][K], dW [N][K]) in float64."""
+    return backward_dx(dy_bf16_bits, w_eff, scale), backward_dw(dy_bf16_bits, xq, a_scale)

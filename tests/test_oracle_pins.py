@@ -547,3 +547,103 @@ def test_pack_vals2_round_trip_and_rejections():
     badb[0, 0] |= 3
     with pytest.raises(ValueError):
         oracle.unpack_vals2(badb)
+
+
+# ------------------------------------------------------------------------------------------------
+# backward under the dual straight-through estimator (Sec. 2.3, Eq. 5; Algorithm 2's backward)
+# ------------------------------------------------------------------------------------------------
+def _tiny_backward_case(seed, T=5, N=4, K=8):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    x = inputs.f32_to_bf16_bits(rng.standard_normal((T, K)).astype(np.float32))
+    dy = inputs.f32_to_bf16_bits(rng.standard_normal((T, N)).astype(np.float32))
+    scale = oracle.absmean_scale(W)[1]
+    mask = oracle.nm_mask(W)
+    w_eff = oracle.apply_mask(oracle.ternarize(W, scale), mask)
+    xq, a_scale = oracle.quant_act(x)
+    return W, mask, w_eff, np.float32(scale), xq, a_scale, dy
+
+
+def test_backward_is_brute_force_on_tiny_inputs():
+    # pure-Python triple loops over the definition, operand roundings written out by hand
+    W, mask, w_eff, scale, xq, a_scale, dy = _tiny_backward_case(1)
+    T, K = xq.shape
+    N = w_eff.shape[0]
+    dY = inputs.bf16_bits_to_f32(dy).astype(np.float64)
+    s_b = float(inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(np.array([scale], np.float32)))[0])
+    dW = np.zeros((N, K)); dX = np.zeros((T, K))
+    for t in range(T):
+        for k in range(K):
+            xq_b = float(inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(np.array([np.float32(xq[t, k]) * a_scale[t]], np.float32)))[0])
+            for n in range(N):
+                dW[n, k] += dY[t, n] * xq_b
+                dX[t, k] += dY[t, n] * (float(w_eff[n, k]) * s_b)
+    gx, gw = oracle.backward_dual_ste(dy, xq, a_scale, w_eff, scale)
+    assert np.allclose(gw, dW, rtol=1e-13, atol=1e-15)
+    assert np.allclose(gx, dX, rtol=1e-13, atol=1e-15)
+
+
+def test_backward_matches_finite_differences_of_the_linear_map():
+    # y = x_q w_masked^T is bilinear, so central differences of L = sum(G * y) in one entry of
+    # w_masked (or of x_q) give the gradients exactly: a transposed operand or a wrong index fails
+    W, mask, w_eff, scale, xq, a_scale, dy = _tiny_backward_case(2, T=6, N=3, K=8)
+    G = inputs.bf16_bits_to_f32(dy).astype(np.float64)
+    xq_b = oracle.fake_quant_act_bf16(xq, a_scale)
+    w_b = w_eff.astype(np.float64) * float(oracle.bf16_round(np.array([scale], np.float32))[0])
+    loss = lambda xa, wa: float(np.sum(G * np.einsum("tk,nk->tn", xa, wa)))
+    gx, gw = oracle.backward_dual_ste(dy, xq, a_scale, w_eff, scale)
+    h = 0.5
+    for (n, k) in [(0, 0), (2, 7), (1, 3)]:
+        wp, wm = w_b.copy(), w_b.copy()
+        wp[n, k] += h; wm[n, k] -= h
+        assert abs((loss(xq_b, wp) - loss(xq_b, wm)) / (2 * h) - gw[n, k]) <= 1e-9 * max(1.0, abs(gw[n, k]))
+    for (t, k) in [(0, 0), (5, 7), (3, 2)]:
+        xp, xm = xq_b.copy(), xq_b.copy()
+        xp[t, k] += h; xm[t, k] -= h
+        assert abs((loss(xp, w_b) - loss(xm, w_b)) / (2 * h) - gx[t, k]) <= 1e-9 * max(1.0, abs(gx[t, k]))
+
+
+def test_backward_adjoint_identities():
+    # <dY, forward(x_q, w)> = <dX, x_q> = <dW, w>: the backward maps are the adjoints of the forward one
+    W, mask, w_eff, scale, xq, a_scale, dy = _tiny_backward_case(3, T=7, N=8, K=16)
+    G = inputs.bf16_bits_to_f32(dy).astype(np.float64)
+    xq_b = oracle.fake_quant_act_bf16(xq, a_scale)
+    w_b = w_eff.astype(np.float64) * float(oracle.bf16_round(np.array([scale], np.float32))[0])
+    gx, gw = oracle.backward_dual_ste(dy, xq, a_scale, w_eff, scale)
+    lhs = float(np.sum(G * (xq_b @ w_b.T)))
+    assert abs(lhs - float(np.sum(gx * xq_b))) <= 1e-12 * max(1.0, abs(lhs))
+    assert abs(lhs - float(np.sum(gw * w_b))) <= 1e-12 * max(1.0, abs(lhs))
+
+
+def test_backward_one_hot_gradient_reads_rows_back():
+    W, mask, w_eff, scale, xq, a_scale, dy = _tiny_backward_case(4, T=4, N=4, K=8)
+    one = np.zeros((4, 4), np.float32)
+    one[2, 1] = 1.0                                           # dL/dy[t=2][n=1] = 1
+    gx, gw = oracle.backward_dual_ste(inputs.f32_to_bf16_bits(one), xq, a_scale, w_eff, scale)
+    xq_b = oracle.fake_quant_act_bf16(xq, a_scale)
+    s_b = float(oracle.bf16_round(np.array([scale], np.float32))[0])
+    assert np.array_equal(gw[1], xq_b[2]) and not gw[[0, 2, 3]].any()
+    assert np.array_equal(gx[2], w_eff[1].astype(np.float64) * s_b) and not gx[[0, 1, 3]].any()
+
+
+def test_backward_weight_gradient_is_dense_not_gated_by_the_mask():
+    # Eq. 5: the mask is transparent, pruned weights receive their gradient; the gated alternative
+    # (M (.) dW) is the negative control and must differ
+    W, mask, w_eff, scale, xq, a_scale, dy = _tiny_backward_case(5, T=9, N=8, K=16)
+    gw = oracle.backward_dw(dy, xq, a_scale)
+    pruned = mask == 0
+    assert pruned.sum() == mask.size // 2
+    assert np.count_nonzero(gw[pruned]) > 0.9 * pruned.sum()
+    assert not np.array_equal(gw, gw * mask)
+
+
+def test_backward_operand_roundings():
+    # the saved activations are held in bf16: integer codes times a power-of-two scale are exact,
+    # a scale with a long mantissa is rounded once (ties to even)
+    xq = np.array([[127, -3, 64, 1]], np.int8)
+    assert np.array_equal(oracle.fake_quant_act_bf16(xq, np.array([0.25], np.float32)), xq.astype(np.float64) * 0.25)
+    s = np.float32(1.0 + 2.0 ** -9)                            # 127 * s needs more than 8 bits
+    got = oracle.fake_quant_act_bf16(np.array([[127, 1]], np.int8), np.array([s], np.float32))
+    assert got[0, 0] == 127.0 and got[0, 1] == 1.0             # 127.248 -> 127 (8-bit significand), 1.00195 -> 1
+    assert oracle.bf16_round(np.array([1.0 + 2.0 ** -8], np.float32))[0] == 1.0          # tie -> even
+    assert oracle.bf16_round(np.array([1.0 + 3 * 2.0 ** -8], np.float32))[0] == 1.0 + 2.0 ** -6
