@@ -239,6 +239,42 @@ class Layer:
         self.ops = 2.0 * T * N * K
 
 
+def backward_rows(torch, b, peaks, layers, time_cold, iters):
+    """The layer's backward under the dual straight-through estimator (Sec. 2.3, Eq. 5): dX = dY w_masked and
+    the dense dW = dY^T x_q on the tensor cores in bf16 (fp32 accumulation), per 2B-shaped layer at
+    T = 4096, cold L2.  Each time covers the whole call for that gradient: the operand preparation (W_eff^T,
+    or x_q^T and dY^T, in bf16) and the GEMM.  `library_matmul_*`: torch.matmul on ready-made bf16 operands of
+    the same shapes, as the pace of a library GEMM on this machine (context, not part of the path)."""
+    rows = {}
+    for L in layers:
+        T, N, K = L.T, L.N, L.K
+        p = L.packed
+        b.sbn_quantize_mask_pack(L.W, p["vals"], p["meta"], p["w_scale"], p["ws"])
+        b.sbn_quant_act(L.x, L.xq, L.a_scale)
+        dY = torch.from_numpy(inputs.activations_bf16(T, N, seed=77).view(np.int16)).cuda().view(torch.bfloat16)
+        dX = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+        dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+        ws = torch.empty(b.sbn_workspace_bytes(b.OP_BACKWARD, T, N, K), dtype=torch.uint8, device="cuda")
+        f_dx = lambda: b.sbn_bitlinear_backward(dY, L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], N, K, dX=dX, ws=ws)
+        f_dw = lambda: b.sbn_bitlinear_backward(dY, L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], N, K, dW=dW, ws=ws)
+        w_b = torch.empty((N, K), dtype=torch.bfloat16, device="cuda").normal_()
+        g_dx = lambda: torch.matmul(dY, w_b)
+        g_dw = lambda: torch.matmul(dY.t(), L.x)
+        for fn in (f_dx, f_dw, g_dx, g_dw):
+            for _ in range(2):
+                fn()
+        t = {k: time_cold(fn, iters) for k, fn in (("dx", f_dx), ("dw", f_dw), ("lib_dx", g_dx), ("lib_dw", g_dw))}
+        flops = 2.0 * T * N * K
+        rows[L.name] = {"dx_us": round(t["dx"], 2), "dw_us": round(t["dw"], 2),
+                        "dx_tflops": round(flops / t["dx"] / 1e6, 1), "dw_tflops": round(flops / t["dw"] / 1e6, 1),
+                        "dx_frac_of_measured_bf16_burst": round(flops / t["dx"] / 1e6 / peaks["bf16_tflops"], 4),
+                        "dw_frac_of_measured_bf16_burst": round(flops / t["dw"] / 1e6 / peaks["bf16_tflops"], 4),
+                        "library_matmul_dx_us": round(t["lib_dx"], 2), "library_matmul_dw_us": round(t["lib_dw"], 2)}
+        del dY, dX, dW, ws, w_b
+    b.sbn_check_status()
+    return rows
+
+
 def large_m_and_sustained(torch, b, peaks, sampler, time_cold, iters):
     """The large-M target on the two 7B-class shapes (T = 8192; weights N(0, 0.015) with 5 % x10 outliers,
     activations with a per-token LogNormal(0, 0.5) scale): isolated sparse and dense GEMM, cold L2, both
@@ -537,8 +573,9 @@ def run_ours(args):
             row["norm_quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4 + L.K * 4) / nact / 1e3, 1)
         gemm[L.name] = row
     b.sbn_check_status()
-    large_m, sustained, few_tokens = None, None, None
+    large_m, sustained, few_tokens, backward = None, None, None, None
     if rank == 0 and world == 1 and args.workload == "2b" and not args.no_extras:
+        backward = backward_rows(torch, b, peaks, layers, time_cold, iters)
         large_m, sustained = large_m_and_sustained(torch, b, peaks, sampler, time_cold, iters)
         few_tokens = decode_rows(torch, b, peaks, inputs.SHAPES_2B, (1, 4, 16, 64), cold=False)
         b.sbn_check_status()
@@ -598,6 +635,7 @@ def run_ours(args):
             "cpu_baseline": cpu_baseline,
             "kernel_us_in_step": {k: {n: round(v, 2) for n, v in d.items()} for k, d in kernel_us.items()},
             "isolated": gemm,
+            "backward": backward,
             "isolated_large_m": large_m,
             "sustained": sustained,
             "few_tokens": few_tokens,

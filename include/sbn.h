@@ -84,7 +84,8 @@ typedef enum {
     SBN_OP_QUANTIZE_MASK_PACK = 0,
     SBN_OP_QUANT_ACT = 1,
     SBN_OP_SPARSE_BITLINEAR = 2,
-    SBN_OP_BITLINEAR = 3
+    SBN_OP_BITLINEAR = 3,
+    SBN_OP_BACKWARD = 4
 } sbn_op;
 
 /* Host, pure.  Bytes of the tiled int8 activation buffer xq for T tokens of K columns. */
@@ -351,6 +352,31 @@ sbn_status sbn_bitlinear(const int8_t *xq, const float *a_scale, int T,
                          const int8_t *dense_q, const float *w_scale,
                          int N, int K, const float *bias, void *y, sbn_out_dtype dt,
                          int32_t *acc_out, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Backward of one Sparse-BitLinear layer under the dual straight-through estimator -- Sec. 2.3, Eq. 5
+ * (the mask is transparent to the gradient, like the quantiser), Algorithm 1 "Backward", Algorithm 2's
+ * backward (the weight function returns g_out unchanged).  With y = F.linear(x_q, w_masked), x_q the
+ * fake-quantised activations xq[t][k] * a_scale[t] and w_masked = W_eff * w_scale:
+ *   dW[n][k] = sum_t dY[t][n] * x_q[t][k]       DENSE: every master weight gets its gradient, pruned
+ *                                               ones included (the mask is NOT applied)
+ *   dX[t][k] = sum_n dY[t][n] * w_masked[n][k]  through the activation quantiser as the identity
+ * Precision (the paper states none; its models train with bf16 tensors): dY is bf16, the saved operands
+ * enter as a bf16 run holds them, x_q = bf16(xq * a_scale) and w_masked = W_eff * bf16(w_scale); products
+ * are exact, sums are accumulated in fp32 on the tensor cores; dW leaves as fp32, dX as bf16.
+ *   dY_bf16   device, bf16 [T][N]
+ *   xq, a_scale           device, the forward's quantised activations (tiled) and scales; needed for dW
+ *   vals, meta, w_scale   device, the forward's packed weights; needed for dX
+ *   dX_bf16   device out, bf16 [T][K], or NULL to skip
+ *   dW        device out, fp32 [N][K], or NULL to skip (overwritten, not accumulated)
+ *   ws        device workspace of sbn_workspace_bytes(SBN_OP_BACKWARD, T, N, K) bytes, 256-byte aligned
+ *             (W_eff^T, x_q^T and dY^T in bf16, the contraction index contiguous); no initialisation needed
+ * The bias gradient (a column sum of dY) is not computed here.
+ */
+sbn_status sbn_bitlinear_backward(const void *dY_bf16, int T, const int8_t *xq, const float *a_scale,
+                                  const int8_t *vals, const uint8_t *meta, const float *w_scale,
+                                  int N, int K, void *dX_bf16, float *dW, void *ws, size_t ws_bytes,
+                                  void *stream);
 
 /*
  * Whole forward of one layer from HOST activations (Algorithm 2's forward with pre-packed

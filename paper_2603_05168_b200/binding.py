@@ -18,14 +18,14 @@ LIB_PATH = os.path.join(_PKG, "libsbn.so")
 
 SBN_OK = 0
 OUT_F32, OUT_BF16 = 0, 1
-OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR = 0, 1, 2, 3
+OP_QUANTIZE_MASK_PACK, OP_QUANT_ACT, OP_SPARSE_BITLINEAR, OP_BITLINEAR, OP_BACKWARD = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "sbn_workspace_bytes", "sbn_xq_bytes", "sbn_quantize_mask_pack", "sbn_quantize_mask_pack_bf16", "sbn_quantize_mask_pack_static_ws", "sbn_quantize_mask_pack_batched",
     "sbn_batch_workspace_bytes", "sbn_quant_act", "sbn_quant_act_expand68", "sbn_expanded_k", "sbn_norm_quant_act", "sbn_norm_quant_act_expand68", "sbn_sparse_bitlinear", "sbn_pack_vals2", "sbn_sparse_bitlinear_packed", "sbn_quant_act_sparse_bitlinear", "sbn_quant_act_bitlinear",
     "sbn_bitlinear", "sbn_layer_forward_host", "sbn_check_status", "sbn_status_string",
     "sbn_set_gemm_tuning", "sbn_plan_gemm", "sbn_launch_count", "sbn_unpack_canonical", "sbn_tile_canonical",
-    "sbn_set_wait_test", "sbn_set_gemm_probe",
+    "sbn_set_wait_test", "sbn_set_gemm_probe", "sbn_bitlinear_backward",
 ]
 
 _lib = None
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.sbn_unpack_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.sbn_tile_canonical.restype = i32
         L.sbn_tile_canonical.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        L.sbn_bitlinear_backward.restype = i32
+        L.sbn_bitlinear_backward.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
         L.sbn_set_gemm_probe.restype = None
         L.sbn_set_gemm_probe.argtypes = [i32]
         L.sbn_set_wait_test.restype = i32
@@ -301,6 +303,15 @@ def sbn_tile_canonical(vals_plain, meta_plain, N: int, K: int, vals, meta):
 
 def sbn_set_wait_test(break_waits: bool = False, wait_limit_us: int = 0):
     _check(lib().sbn_set_wait_test(1 if break_waits else 0, int(wait_limit_us)), "sbn_set_wait_test")
+
+
+def sbn_bitlinear_backward(dY, xq, a_scale, vals, meta, w_scale, N: int, K: int, dX=None, dW=None, ws=None):
+    """Dual-STE backward of one layer: dX (bf16 [T][K]) and / or dW (fp32 [N][K]) from dY (bf16 [T][N])."""
+    T = dY.shape[0]
+    wp, wb = _ws_args(ws)
+    _check(lib().sbn_bitlinear_backward(_ptr(dY), T, _ptr(xq), _ptr(a_scale), _ptr(vals), _ptr(meta), _ptr(w_scale), N, K,
+                                        _ptr(dX), _ptr(dW), wp, wb, _stream()),
+           "sbn_bitlinear_backward")
 
 
 def sbn_set_gemm_probe(flags: int = 0):

@@ -22,6 +22,8 @@
 #include "gemm_splitk_cluster_tcgen05.cuh"
 #include "gemm_packed_cluster_tcgen05.cuh"
 #include "gemm_fused_act_cluster_tcgen05.cuh"
+#include "backward_prep.cuh"
+#include "gemm_bf16_pair_tcgen05.cuh"
 
 namespace sbn {
 
@@ -93,6 +95,21 @@ static bool encode_flat_1k(CUtensorMap* map, const void* base, uint64_t total_by
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box,
                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Row-major bf16 matrix [rows][ld] of which `inner` columns are valid, fetched in boxes of 64 columns x
+// box_rows rows with the 128-byte swizzle: the box lands in shared memory as the K-major operand image.
+static bool encode_2d_bf16_sw128(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || box_rows == 0 || box_rows > 256 || (ld * 2) % 16 != 0) return false;
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -440,6 +457,58 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
     return SBN_OK;
 }
 
+// ---- backward GEMMs (bf16) -------------------------------------------------------------------------
+static inline int backward_tp(int T) { return (T + 63) / 64 * 64; }      // token rows padded to whole K steps
+
+struct BackwardWs {
+    size_t wt_off, xt_off, dyt_off, total;
+};
+static BackwardWs backward_ws_layout(int T, int N, int K) {
+    const size_t tp = static_cast<size_t>(backward_tp(T));
+    BackwardWs w;
+    auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
+    w.wt_off = 0;
+    w.xt_off = up(static_cast<size_t>(K) * N * 2);
+    w.dyt_off = w.xt_off + up(static_cast<size_t>(K) * tp * 2);
+    w.total = w.dyt_off + up(static_cast<size_t>(N) * tp * 2);
+    return w;
+}
+
+// Output columns per tile: fewest waves over the 74 CTA pairs, weighted by what a tile costs (the A part of a
+// stage is fixed, the B part grows with the tile's width).
+static int pick_bf16_bn(int M, int Nn) {
+    const long tiles_m = (M + 255) / 256;
+    int best = 256;
+    double best_cost = 1e300;
+    for (int bn = 256; bn >= 128; bn -= 16) {
+        const long tiles = tiles_m * ((Nn + bn - 1) / bn);
+        const long waves = (tiles + kNumSMs / 2 - 1) / (kNumSMs / 2);
+        const double cost = static_cast<double>(waves) * (256.0 + bn);
+        if (cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+// D[M][Nn] = A[M][Kc] B[Nn][Kc]^T (bf16 in, fp32 accumulation), optionally times bf16(*scale).
+static sbn_status run_gemm_bf16(const void* A, int M, uint64_t lda, const void* B, int Nn, uint64_t ldb, int Kc, void* out,
+                                bool out_bf16, const float* scale, cudaStream_t stream) {
+    Bf16GemmParams p;
+    p.M = M; p.Nn = Nn; p.Kc = Kc;
+    p.bn = g_force_token_tile < 0 ? std::min(256, std::max(64, (-g_force_token_tile) / 16 * 16)) : pick_bf16_bn(M, Nn);
+    p.out = out; p.out_bf16 = out_bf16 ? 1 : 0;
+    p.scale = scale;
+    CUtensorMap ta, tb;
+    if (!encode_2d_bf16_sw128(&ta, A, static_cast<uint64_t>(Kc), static_cast<uint64_t>(M), lda, 128) ||
+        !encode_2d_bf16_sw128(&tb, B, static_cast<uint64_t>(Kc), static_cast<uint64_t>(Nn), ldb, static_cast<uint32_t>(p.bn / 2)))
+        return SBN_ERR_CUDA;
+    if (!ensure_dynamic_smem<gemm_bf16_pair_kernel>(kBf16SmemBytes)) return SBN_ERR_CUDA;
+    const int tiles = ((M + 255) / 256) * ((Nn + p.bn - 1) / p.bn);
+    const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
+    const cudaError_t err = launch_kernel(gemm_bf16_pair_kernel, dim3(2 * pairs), dim3(kBf16Threads), kBf16SmemBytes, stream, ta, tb, p);
+    ++g_launch_count;
+    return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Built-in scratch for sbn_quantize_mask_pack_static_ws: part of the library image, so callers
 // that cannot allocate still have somewhere to put the pass-1 partial sums.  In host code the
@@ -483,6 +552,9 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K) {
     switch (op) {
         case SBN_OP_QUANTIZE_MASK_PACK: return sizeof(QmpWorkspace);       // one matrix; batches: sbn_batch_workspace_bytes
         case SBN_OP_QUANT_ACT: return 0;
+        case SBN_OP_BACKWARD:
+            if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return 0;
+            return backward_ws_layout(T, N, K).total;
         case SBN_OP_SPARSE_BITLINEAR:
         case SBN_OP_BITLINEAR:
             if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0) return 0;
@@ -850,6 +922,47 @@ sbn_status sbn_unpack_canonical(const int8_t* vals, const uint8_t* meta, int N, 
 sbn_status sbn_tile_canonical(const int8_t* vals_plain, const uint8_t* meta_plain, int N, int K, int8_t* vals,
                               uint8_t* meta, void* stream) {
     return canonical_any(true, vals_plain, meta_plain, N, K, vals, meta, stream);
+}
+
+sbn_status sbn_bitlinear_backward(const void* dY_bf16, int T, const int8_t* xq, const float* a_scale, const int8_t* vals,
+                                  const uint8_t* meta, const float* w_scale, int N, int K, void* dX_bf16, float* dW,
+                                  void* ws, size_t ws_bytes, void* stream) {
+    if (!dY_bf16 || (!dX_bf16 && !dW)) return SBN_ERR_NULL;
+    if (dX_bf16 && (!vals || !meta || !w_scale)) return SBN_ERR_NULL;
+    if (dW && (!xq || !a_scale)) return SBN_ERR_NULL;
+    if (T <= 0 || N <= 0 || K <= 0 || N % kBM != 0 || K % kBK != 0 || K > (1 << 20)) return SBN_ERR_SHAPE;
+    const BackwardWs lay = backward_ws_layout(T, N, K);
+    if (!ws || ws_bytes < lay.total) return SBN_ERR_WORKSPACE;
+    if (misaligned(dY_bf16, 16) || misaligned(ws, 256) || (dX_bf16 && (misaligned(dX_bf16, 16) || misaligned(vals, 16) || misaligned(meta, 16) || misaligned(w_scale, 4))) ||
+        (dW && (misaligned(dW, 16) || misaligned(xq, 16) || misaligned(a_scale, 4))))
+        return SBN_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int tp = backward_tp(T);
+    char* base = static_cast<char*>(ws);
+    uint16_t* Wt = reinterpret_cast<uint16_t*>(base + lay.wt_off);
+    uint16_t* XT = reinterpret_cast<uint16_t*>(base + lay.xt_off);
+    uint16_t* dYT = reinterpret_cast<uint16_t*>(base + lay.dyt_off);
+    const int KB = K / kBK, NB = N / kBM, TB = (tp + 127) / 128;
+    if (dX_bf16) {
+        // dX[t][k] = bf16(scale) * sum_n dY[t][n] W_eff[n][k]: A = dY [T][N], B = W_eff^T [K][N]
+        if (launch_kernel(weff_t_bf16_kernel, dim3(KB * NB), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(vals), meta, N, K, Wt) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        ++g_launch_count;
+        const sbn_status st = run_gemm_bf16(dY_bf16, T, static_cast<uint64_t>(N), Wt, K, static_cast<uint64_t>(N), N, dX_bf16, true, w_scale, s);
+        if (st != SBN_OK) return st;
+    }
+    if (dW) {
+        // dW[n][k] = sum_t dY[t][n] x_q[t][k]: A = dY^T [N][Tp], B = x_q^T [K][Tp] (token rows zero-padded to Tp)
+        if (launch_kernel(xq_t_bf16_kernel, dim3(KB * TB), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(xq), a_scale, T, K, tp, XT) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        ++g_launch_count;
+        if (launch_kernel(transpose_bf16_kernel, dim3(NB * TB), dim3(kPrepThreads), 0, s, static_cast<const uint16_t*>(dY_bf16), T, N, tp, dYT) != cudaSuccess)
+            return SBN_ERR_CUDA;
+        ++g_launch_count;
+        const sbn_status st = run_gemm_bf16(dYT, N, static_cast<uint64_t>(tp), XT, K, static_cast<uint64_t>(tp), tp, dW, false, nullptr, s);
+        if (st != SBN_OK) return st;
+    }
+    return SBN_OK;
 }
 
 sbn_status sbn_check_status(void* stream) {

@@ -1,0 +1,140 @@
+"""GPU parity of the layer's backward under the dual straight-through estimator (Sec. 2.3, Eq. 5;
+Algorithm 2's backward) against the CPU oracle, through the C ABI.
+
+The two sides multiply the same bf16-held operands (every product is exact in fp32); the oracle adds
+in float64, the tensor cores in fp32 in an order of their own.  Tolerance, derived from that: with Kc
+terms per output the fp32 sum is off by at most Kc * 2^-23 * sum |terms| (every partial sum rounded or
+truncated once to 24 bits), so
+    |dW_gpu - dW_ref| <= T * 2^-23 * (|dY|^T |x_q|)                         (dW is fp32)
+    |dX_gpu - dX_ref| <= N * 2^-23 * (|dY| |w|) + 2^-8 |dX_ref|             (dX is rounded to bf16: 1 ulp)
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_05168_b200 import binding as b
+from paper_2603_05168_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from gpu_harness import bf16_dev, bf16_tensor_bits, gpu_quant_act, gpu_quantize_mask_pack
+
+
+@pytest.fixture(autouse=True)
+def _reset_tuning():
+    b.sbn_set_gemm_tuning(0, 0)
+    yield
+    b.sbn_set_gemm_tuning(0, 0)
+
+
+def _case(T, N, K, seed, dy_sigma=1.0, logn=0.5):
+    W = inputs.latent_weights(N, K, seed=seed)
+    x = inputs.activations_bf16(T, K, seed=seed + 1, token_lognormal_sigma=logn)
+    rng = np.random.default_rng(seed + 2)
+    dy = inputs.f32_to_bf16_bits((rng.standard_normal((T, N)) * dy_sigma).astype(np.float32))
+    r = oracle.quantize_mask_pack(W)
+    if r["near_tie"]:
+        pytest.skip("gamma within rounding distance of an fp32 midpoint for this seed")
+    xq_ref, s_ref = oracle.quant_act(x)
+    w_eff = (r["dense_q"].astype(np.int16) * r["mask"].astype(np.int16)).astype(np.int8)
+    g = gpu_quantize_mask_pack(W, with_dense=False)
+    xq, a_scale = gpu_quant_act(x)
+    return dict(T=T, N=N, K=K, r=r, w_eff=w_eff, xq_ref=xq_ref, s_ref=s_ref, dy=dy, g=g, xq=xq, a_scale=a_scale)
+
+
+def _gpu_backward(c, want_dx=True, want_dw=True):
+    T, N, K = c["T"], c["N"], c["K"]
+    dY = bf16_dev(c["dy"])
+    ws = torch.empty(b.sbn_workspace_bytes(b.OP_BACKWARD, T, N, K), dtype=torch.uint8, device="cuda")
+    dX = torch.full((T, K), float("nan"), dtype=torch.bfloat16, device="cuda") if want_dx else None
+    dW = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda") if want_dw else None
+    p = c["g"]["dev"]
+    b.sbn_bitlinear_backward(dY, c["xq"], c["a_scale"], p["vals"], p["meta"], p["w_scale"], N, K, dX=dX, dW=dW, ws=ws)
+    b.sbn_check_status()
+    return dX, dW
+
+
+def _assert_dw(c, dW):
+    ref = oracle.backward_dw(c["dy"], c["xq_ref"], c["s_ref"])
+    dY_abs = np.abs(oracle.bf16_bits_to_f64(c["dy"]))
+    bound = c["T"] * 2.0 ** -23 * (dY_abs.T @ np.abs(oracle.fake_quant_act_bf16(c["xq_ref"], c["s_ref"]))) + 1e-30
+    err = np.abs(dW.cpu().numpy().astype(np.float64) - ref)
+    bad = np.argwhere(err > bound)
+    assert bad.size == 0, f"dW: {bad.shape[0]} entries beyond the fp32-accumulation bound, first at (n, k) = {tuple(bad[0])}"
+    return ref
+
+
+def _assert_dx(c, dX):
+    ref = oracle.backward_dx(c["dy"], c["w_eff"], c["r"]["scale"])
+    s_b = float(oracle.bf16_round(np.array([c["r"]["scale"]], np.float32))[0])
+    dY_abs = np.abs(oracle.bf16_bits_to_f64(c["dy"]))
+    bound = c["N"] * 2.0 ** -23 * (dY_abs @ np.abs(c["w_eff"].astype(np.float64))) * s_b + 2.0 ** -8 * np.abs(ref) + 1e-30
+    got = inputs.bf16_bits_to_f32(bf16_tensor_bits(dX)).astype(np.float64)
+    err = np.abs(got - ref)
+    bad = np.argwhere(err > bound)
+    assert bad.size == 0, f"dX: {bad.shape[0]} entries beyond the bound, first at (t, k) = {tuple(bad[0])}"
+    return ref
+
+
+SHAPES = [(64, 256, 256), (5, 128, 128), (1, 128, 256), (130, 384, 512), (300, 256, 2560), (257, 640, 1280), (1000, 512, 1152),
+          (63, 128, 6912), (520, 2560, 640)]
+
+
+@pytest.mark.parametrize("T,N,K", SHAPES)
+def test_backward_parity(T, N, K):
+    c = _case(T, N, K, seed=200 + T + N + K)
+    dX, dW = _gpu_backward(c)
+    _assert_dw(c, dW)
+    _assert_dx(c, dX)
+
+
+@pytest.mark.parametrize("bn", [64, 112, 128, 176, 240, 256])
+def test_backward_parity_every_tile_width(bn):
+    c = _case(333, 384, 1280, seed=260 + bn)
+    b.sbn_set_gemm_tuning(-bn, 0)
+    dX, dW = _gpu_backward(c)
+    _assert_dw(c, dW)
+    _assert_dx(c, dX)
+
+
+def test_backward_weight_gradient_reaches_pruned_weights():
+    # Eq. 5: the mask is transparent -- a mask-gated gradient is the negative control
+    c = _case(200, 256, 512, seed=270)
+    _, dW = _gpu_backward(c, want_dx=False)
+    ref = _assert_dw(c, dW)
+    pruned = c["r"]["mask"] == 0
+    got = dW.cpu().numpy()
+    assert np.count_nonzero(got[pruned]) > 0.99 * pruned.sum()
+    gated = ref * c["r"]["mask"]
+    assert np.abs(got - gated).max() > 0.1 * np.abs(ref).max()
+
+
+def test_backward_either_output_alone_and_one_hot_rows():
+    c = _case(96, 256, 384, seed=280)
+    one = np.zeros((96, 256), np.float32)
+    one[17, 200] = 1.0
+    one[95, 3] = -2.0
+    c["dy"] = inputs.f32_to_bf16_bits(one)
+    dX, none = _gpu_backward(c, want_dw=False)
+    assert none is None
+    _, dW = _gpu_backward(c, want_dx=False)
+    xq_b = oracle.fake_quant_act_bf16(c["xq_ref"], c["s_ref"])
+    s_b = float(oracle.bf16_round(np.array([c["r"]["scale"]], np.float32))[0])
+    gw = dW.cpu().numpy().astype(np.float64)
+    assert np.array_equal(gw[200], xq_b[17]) and np.array_equal(gw[3], -2.0 * xq_b[95])
+    rest = np.ones(256, bool); rest[[200, 3]] = False
+    assert not gw[rest].any()
+    gx = inputs.bf16_bits_to_f32(bf16_tensor_bits(dX)).astype(np.float64)
+    assert np.array_equal(gx[17], oracle.bf16_round((c["w_eff"][200].astype(np.float64) * s_b).astype(np.float32)))
+    assert np.array_equal(gx[95], oracle.bf16_round((-2.0 * c["w_eff"][3].astype(np.float64) * s_b).astype(np.float32)))
+
+
+@pytest.mark.parametrize("name,T,K,N", [("qkv", 4096, 2560, 3840), ("down", 4096, 6912, 2560)])
+def test_backward_full_size(name, T, K, N):
+    # the benchmark's shapes, whole outputs
+    c = _case(T, N, K, seed=290)
+    dX, dW = _gpu_backward(c)
+    _assert_dw(c, dW)
+    _assert_dx(c, dX)
