@@ -370,7 +370,7 @@ sbn_status sbn_bitlinear(const int8_t *xq, const float *a_scale, int T,
  *   dX_bf16   device out, bf16 [T][K], or NULL to skip
  *   dW        device out, fp32 [N][K], or NULL to skip (overwritten, not accumulated)
  *   ws        device workspace of sbn_workspace_bytes(SBN_OP_BACKWARD, T, N, K) bytes, 256-byte aligned
- *             (W_eff^T, x_q^T and dY^T in bf16, the contraction index contiguous); no initialisation needed
+ *             (W_eff^T [K][N] and x_q [T][K] in bf16); no initialisation needed
  * The bias gradient (a column sum of dY) is not computed here.
  */
 sbn_status sbn_bitlinear_backward(const void *dY_bf16, int T, const int8_t *xq, const float *a_scale,

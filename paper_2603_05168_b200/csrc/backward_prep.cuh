@@ -1,17 +1,15 @@
 // Operands of the backward GEMMs (dual straight-through estimator, Sec. 2.3, Eq. 5; Algorithm 2's
-// backward) brought into the shape the bf16 tensor-core kernel consumes: K-major on both sides, i.e. the
-// contraction index contiguous.
+// backward) in bf16, as the tensor-core kernel of gemm_bf16_pair_tcgen05.cuh reads them:
 //
-//   dX[t][k] = sum_n dY[t][n] * w_masked[n][k]   contraction over n:  A = dY [T][N] as it is,
-//                                                 B = W_eff^T [K][N]            (weff_t_bf16_kernel)
-//   dW[n][k] = sum_t dY[t][n] * x_q[t][k]        contraction over t:  A = dY^T [N][T]  (transpose_bf16_kernel),
-//                                                 B = x_q^T [K][T]              (xq_t_bf16_kernel)
+//   dX[t][k] = sum_n dY[t][n] * w_masked[n][k]   contraction over n: A = dY [T][N] as it is (K-major),
+//                                                 B = W_eff^T [K][N] (weff_t_bf16_kernel: a 128 x 128 tile
+//                                                 transposed through shared memory, written as 256 B rows)
+//   dW[n][k] = sum_t dY[t][n] * x_q[t][k]        contraction over t: A = dY [T][N] and B = x_q [T][K]
+//                                                 (xq_bf16_kernel), both as they lie in memory; the MMA
+//                                                 reads them MN-major, so nothing is transposed
 //
 // x_q[t][k] = bf16(x~[t][k] * a_scale[t]) are the fake-quantised activations as a bf16 training run holds
-// them; W_eff is written as +-1.0 / 0.0 and its scale is applied once in the GEMM's epilogue.  All three
-// kernels are memory-bound tile transposes through shared memory: a CTA reads a 128 x 128 tile in the
-// source's order and writes 128 rows of 256 B.  Token rows are padded to a multiple of 64 with zeros
-// (row stride `Tp`), so the GEMM's K-loop needs no tail.
+// them; W_eff is written as +-1.0 / 0.0 and its scale is applied once in the GEMM's epilogue.
 #pragma once
 
 #include "sbn_common.cuh"
@@ -68,62 +66,34 @@ weff_t_bf16_kernel(const uint8_t* __restrict__ vals, const uint8_t* __restrict__
     prep_store_tile(s_t, Wt + (static_cast<size_t>(kb) * 128) * N + static_cast<size_t>(nb) * 128, static_cast<size_t>(N), kPrepTile, kPrepTile);
 }
 
-// x_q^T [K][Tp] in bf16 from the tiled int8 activations and their per-token scales; tokens >= T are zeros.
+// x_q [T][K] in bf16 (token-major, as the activations themselves) from the tiled int8 activations and their
+// per-token scales: the B operand of the weight-gradient GEMM when it reads MN-major operands.  A thread
+// converts 16 codes (one 16 B chunk) into 32 B of output.
 __global__ void __launch_bounds__(kPrepThreads)
-xq_t_bf16_kernel(const uint8_t* __restrict__ xq, const float* __restrict__ a_scale, int T, int K, int Tp, uint16_t* __restrict__ XT) {
-    __shared__ __align__(16) unsigned char s_t[kPrepTile * kPrepRowBytes];
+xq_bf16_kernel(const uint8_t* __restrict__ xq, const float* __restrict__ a_scale, int T, int K, uint16_t* __restrict__ X) {
     pdl_wait();
-    const int KB = K >> 7;
-    const int kb = blockIdx.x % KB, tb = blockIdx.x / KB;
     const size_t tb8 = xq_tb8(T);
-    const int tt = threadIdx.x >> 1, half = threadIdx.x & 1;   // token inside the tile, half of its 128 columns
-    const int t = tb * 128 + tt;
-    uint4 c[4];
-    float s = 0.0f;
-    if (t < T) {
-        s = __ldg(a_scale + t);
-        const uint8_t* atom = xq + (static_cast<size_t>(kb) * tb8 + (static_cast<uint32_t>(t) >> 3)) * 1024 + (t & 7) * 128;
+    const int chunks_per_row = K >> 4;
+    const size_t total = static_cast<size_t>(T) * chunks_per_row;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * kPrepThreads + threadIdx.x; i < total; i += static_cast<size_t>(gridDim.x) * kPrepThreads) {
+        const int t = static_cast<int>(i / chunks_per_row), ch = static_cast<int>(i % chunks_per_row);
+        const int kb = ch >> 3, c8 = ch & 7;
+        const float s = __ldg(a_scale + t);
+        const uint4 c = *reinterpret_cast<const uint4*>(xq + (static_cast<size_t>(kb) * tb8 + (static_cast<uint32_t>(t) >> 3)) * 1024 + (t & 7) * 128 +
+                                                        ((c8 ^ (t & 7)) << 4));
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        uint32_t o[8];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = *reinterpret_cast<const uint4*>(atom + (((4 * half + i) ^ (t & 7)) << 4));
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int q = static_cast<int8_t>((w[j >> 2] >> (8 * (j & 3))) & 0xFFu);
-            const int k = 64 * half + 16 * i + j;
-            *reinterpret_cast<uint16_t*>(s_t + k * kPrepRowBytes + tt * 2) = bf16_bits_of(__fmul_rn(static_cast<float>(q), s));
+        for (int j = 0; j < 8; ++j) {
+            const int q0 = static_cast<int8_t>((w[j >> 1] >> (16 * (j & 1))) & 0xFFu);
+            const int q1 = static_cast<int8_t>((w[j >> 1] >> (16 * (j & 1) + 8)) & 0xFFu);
+            o[j] = static_cast<uint32_t>(bf16_bits_of(__fmul_rn(static_cast<float>(q0), s))) |
+                   (static_cast<uint32_t>(bf16_bits_of(__fmul_rn(static_cast<float>(q1), s))) << 16);
         }
+        uint4* dst = reinterpret_cast<uint4*>(X + static_cast<size_t>(t) * K + static_cast<size_t>(ch) * 16);
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
     }
-    __syncthreads();
-    prep_store_tile(s_t, XT + (static_cast<size_t>(kb) * 128) * Tp + static_cast<size_t>(tb) * 128, static_cast<size_t>(Tp), kPrepTile,
-                    min(kPrepTile, Tp - tb * 128));
-}
-
-// dY^T [N][Tp] from dY [T][N] (bf16 bit patterns moved, not converted); tokens >= T are zeros.
-__global__ void __launch_bounds__(kPrepThreads)
-transpose_bf16_kernel(const uint16_t* __restrict__ dY, int T, int N, int Tp, uint16_t* __restrict__ dYT) {
-    __shared__ __align__(16) unsigned char s_t[kPrepTile * kPrepRowBytes];
-    pdl_wait();
-    const int NBk = N >> 7;
-    const int nb = blockIdx.x % NBk, tb = blockIdx.x / NBk;
-    const int chunk = threadIdx.x & 15;                        // 8 features
-    for (int tt = threadIdx.x >> 4; tt < kPrepTile; tt += kPrepThreads / 16) {
-        const int t = tb * 128 + tt;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (t < T) v = __ldg(reinterpret_cast<const uint4*>(dY + static_cast<size_t>(t) * N + static_cast<size_t>(nb) * 128 + chunk * 8));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint16_t*>(s_t + (chunk * 8 + j) * kPrepRowBytes + tt * 2) = static_cast<uint16_t>((w[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
-    }
-    __syncthreads();
-    prep_store_tile(s_t, dYT + (static_cast<size_t>(nb) * 128) * Tp + static_cast<size_t>(tb) * 128, static_cast<size_t>(Tp), kPrepTile,
-                    min(kPrepTile, Tp - tb * 128));
 }
 
 }  // namespace sbn

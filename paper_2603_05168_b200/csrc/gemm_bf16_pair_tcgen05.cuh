@@ -1,6 +1,6 @@
 // D[M][Nn] = A[M][Kc] * B[Nn][Kc]^T in bf16 with fp32 accumulation on the 5th-generation tensor cores --
-// the two contractions of the layer's backward pass (Sec. 2.3, Eq. 5: dX = dY w_masked, dW = dY^T x_q;
-// backward_prep.cuh brings the operands into this K-major form).
+// the two contractions of the layer's backward pass (Sec. 2.3, Eq. 5: dX = dY w_masked with K-major
+// operands, dW = dY^T x_q with MN-major ones; backward_prep.cuh makes the bf16 operands).
 //
 // Same skeleton as the int8 CTA-pair kernel (gemm_pair_tcgen05.cuh): two CTAs of a cluster issue one
 // `tcgen05.mma.cta_group::2.kind::f16` (M = 256: each CTA supplies 128 rows of A and half of the B tile
@@ -54,12 +54,20 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, u
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// Instruction descriptor for kind::f16: D = fp32, A = B = bf16, both K-major.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int mma_m, int mma_n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(mma_n >> 3) << 17) | (static_cast<uint32_t>(mma_m >> 4) << 24);
+// Instruction descriptor for kind::f16: D = fp32, A = B = bf16; both K-major, or both MN-major (the
+// contraction index is the SLOW index of the operands in memory: bits 15 / 16).
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int mma_m, int mma_n, bool mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major ? ((1u << 15) | (1u << 16)) : 0u) |
+           (static_cast<uint32_t>(mma_n >> 3) << 17) | (static_cast<uint32_t>(mma_m >> 4) << 24);
 }
 
-// tmap_a: [M][Kc] bf16, box {64, 128};  tmap_b: [Nn][Kc] bf16, box {64, bn / 2}
+// MN = false (K-major operands):  tmap_a: [M][Kc] bf16, box {64, 128};  tmap_b: [Nn][Kc] bf16, box {64, bn / 2}.
+// MN = true (MN-major operands: A is stored [Kc][M], B is stored [Kc][Nn], i.e. D = A^T B without a
+// transposed copy of either):  tmap_a: [Kc][M], box {64 of M, 64 of Kc};  tmap_b: [Kc][Nn], box {64, 64};
+// bn must be 128 or 256.  A box of 64 contraction rows x 128 B is the MN-major shared-memory image of a
+// block of 64 output rows (or columns): 8-row groups 1 KB apart along the contraction (the stride offset),
+// blocks 8 KB apart (the leading offset); an MMA of K = 16 starts 2 KB further per step.
+template <bool MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBf16Threads, 1)
 gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Bf16GemmParams p) {
     constexpr int STAGES = kBf16Stages;
@@ -133,8 +141,15 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2 * bytes_per_cta);
                     const uint32_t st = smem_base + stage * kBf16StageBytes;
                     // rows or columns beyond the tensors are zero-filled by the hardware and still count their full size
-                    tma_load_2d_pair(st, &tmap_a, ks * 64, m0, full_leader);
-                    tma_load_2d_pair(st + kBf16StageA, &tmap_b, ks * 64, n0, full_leader);
+                    if constexpr (MN) {
+                        tma_load_2d_pair(st, &tmap_a, m0, ks * 64, full_leader);
+                        tma_load_2d_pair(st + 8192, &tmap_a, m0 + 64, ks * 64, full_leader);
+                        for (int j = 0; j < half_bn / 64; ++j)
+                            tma_load_2d_pair(st + kBf16StageA + j * 8192, &tmap_b, n0 + 64 * j, ks * 64, full_leader);
+                    } else {
+                        tma_load_2d_pair(st, &tmap_a, ks * 64, m0, full_leader);
+                        tma_load_2d_pair(st + kBf16StageA, &tmap_b, ks * 64, n0, full_leader);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -142,7 +157,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader)
         if (rank == 0 && lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(256, BN);
+            const uint32_t idesc = make_idesc_bf16(256, BN, MN);
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_iter = 0;
@@ -157,12 +172,12 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_base + stage * kBf16StageBytes;
-                    const uint64_t a_desc = make_smem_desc(st, 16, 1024, kSwz128);
-                    const uint64_t b_desc = make_smem_desc(st + kBf16StageA, 16, 1024, kSwz128);
+                    const uint64_t a_desc = MN ? make_smem_desc(st, 8192, 1024, kSwz128) : make_smem_desc(st, 16, 1024, kSwz128);
+                    const uint64_t b_desc = MN ? make_smem_desc(st + kBf16StageA, 8192, 1024, kSwz128) : make_smem_desc(st + kBf16StageA, 16, 1024, kSwz128);
+                    constexpr uint64_t kStep = MN ? (2048 >> 4) : (32 >> 4);      // K = 16 elements per instruction: 16 rows, or 32 B along a row
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)        // K = 16 elements = 32 B per instruction
-                        mma_bf16_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * q), b_desc + static_cast<uint64_t>(2 * q), idesc,
-                                      (ks | q) != 0 ? 1u : 0u);
+                    for (int q = 0; q < 4; ++q)
+                        mma_bf16_pair(d_tmem, a_desc + kStep * q, b_desc + kStep * q, idesc, (ks | q) != 0 ? 1u : 0u);
                     tcgen05_commit_pair(bar_empty + 8 * stage);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }

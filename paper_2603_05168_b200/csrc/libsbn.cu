@@ -458,19 +458,15 @@ static sbn_status run_gemm(bool sparse, const int8_t* xq, const float* a_scale, 
 }
 
 // ---- backward GEMMs (bf16) -------------------------------------------------------------------------
-static inline int backward_tp(int T) { return (T + 63) / 64 * 64; }      // token rows padded to whole K steps
-
-struct BackwardWs {
-    size_t wt_off, xt_off, dyt_off, total;
+struct BackwardWs {                    // W_eff^T [K][N] and x_q [T][K], both bf16
+    size_t wt_off, xq_off, total;
 };
 static BackwardWs backward_ws_layout(int T, int N, int K) {
-    const size_t tp = static_cast<size_t>(backward_tp(T));
     BackwardWs w;
     auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
     w.wt_off = 0;
-    w.xt_off = up(static_cast<size_t>(K) * N * 2);
-    w.dyt_off = w.xt_off + up(static_cast<size_t>(K) * tp * 2);
-    w.total = w.dyt_off + up(static_cast<size_t>(N) * tp * 2);
+    w.xq_off = up(static_cast<size_t>(K) * N * 2);
+    w.total = w.xq_off + up(static_cast<size_t>(T) * K * 2);
     return w;
 }
 
@@ -490,21 +486,35 @@ static int pick_bf16_bn(int M, int Nn) {
 }
 
 // D[M][Nn] = A[M][Kc] B[Nn][Kc]^T (bf16 in, fp32 accumulation), optionally times bf16(*scale).
-static sbn_status run_gemm_bf16(const void* A, int M, uint64_t lda, const void* B, int Nn, uint64_t ldb, int Kc, void* out,
-                                bool out_bf16, const float* scale, cudaStream_t stream) {
+// mn_major: A is stored [Kc][M] (row stride lda) and B [Kc][Nn] (row stride ldb): D = A^T B.
+static sbn_status run_gemm_bf16(bool mn_major, const void* A, int M, uint64_t lda, const void* B, int Nn, uint64_t ldb, int Kc,
+                                void* out, bool out_bf16, const float* scale, cudaStream_t stream) {
     Bf16GemmParams p;
     p.M = M; p.Nn = Nn; p.Kc = Kc;
     p.bn = g_force_token_tile < 0 ? std::min(256, std::max(64, (-g_force_token_tile) / 16 * 16)) : pick_bf16_bn(M, Nn);
+    if (mn_major) p.bn = p.bn > 128 ? 256 : 128;                // whole 64-column blocks per CTA
     p.out = out; p.out_bf16 = out_bf16 ? 1 : 0;
     p.scale = scale;
     CUtensorMap ta, tb;
-    if (!encode_2d_bf16_sw128(&ta, A, static_cast<uint64_t>(Kc), static_cast<uint64_t>(M), lda, 128) ||
-        !encode_2d_bf16_sw128(&tb, B, static_cast<uint64_t>(Kc), static_cast<uint64_t>(Nn), ldb, static_cast<uint32_t>(p.bn / 2)))
-        return SBN_ERR_CUDA;
-    if (!ensure_dynamic_smem<gemm_bf16_pair_kernel>(kBf16SmemBytes)) return SBN_ERR_CUDA;
+    bool ok;
+    if (mn_major) {
+        ok = encode_2d_bf16_sw128(&ta, A, static_cast<uint64_t>(M), static_cast<uint64_t>(Kc), lda, 64) &&
+             encode_2d_bf16_sw128(&tb, B, static_cast<uint64_t>(Nn), static_cast<uint64_t>(Kc), ldb, 64);
+    } else {
+        ok = encode_2d_bf16_sw128(&ta, A, static_cast<uint64_t>(Kc), static_cast<uint64_t>(M), lda, 128) &&
+             encode_2d_bf16_sw128(&tb, B, static_cast<uint64_t>(Kc), static_cast<uint64_t>(Nn), ldb, static_cast<uint32_t>(p.bn / 2));
+    }
+    if (!ok) return SBN_ERR_CUDA;
     const int tiles = ((M + 255) / 256) * ((Nn + p.bn - 1) / p.bn);
     const int pairs = tiles < kNumSMs / 2 ? tiles : kNumSMs / 2;
-    const cudaError_t err = launch_kernel(gemm_bf16_pair_kernel, dim3(2 * pairs), dim3(kBf16Threads), kBf16SmemBytes, stream, ta, tb, p);
+    cudaError_t err;
+    if (mn_major) {
+        if (!ensure_dynamic_smem<gemm_bf16_pair_kernel<true>>(kBf16SmemBytes)) return SBN_ERR_CUDA;
+        err = launch_kernel(gemm_bf16_pair_kernel<true>, dim3(2 * pairs), dim3(kBf16Threads), kBf16SmemBytes, stream, ta, tb, p);
+    } else {
+        if (!ensure_dynamic_smem<gemm_bf16_pair_kernel<false>>(kBf16SmemBytes)) return SBN_ERR_CUDA;
+        err = launch_kernel(gemm_bf16_pair_kernel<false>, dim3(2 * pairs), dim3(kBf16Threads), kBf16SmemBytes, stream, ta, tb, p);
+    }
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -937,29 +947,28 @@ sbn_status sbn_bitlinear_backward(const void* dY_bf16, int T, const int8_t* xq, 
         (dW && (misaligned(dW, 16) || misaligned(xq, 16) || misaligned(a_scale, 4))))
         return SBN_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int tp = backward_tp(T);
     char* base = static_cast<char*>(ws);
     uint16_t* Wt = reinterpret_cast<uint16_t*>(base + lay.wt_off);
-    uint16_t* XT = reinterpret_cast<uint16_t*>(base + lay.xt_off);
-    uint16_t* dYT = reinterpret_cast<uint16_t*>(base + lay.dyt_off);
-    const int KB = K / kBK, NB = N / kBM, TB = (tp + 127) / 128;
+    uint16_t* XT = reinterpret_cast<uint16_t*>(base + lay.xq_off);
+    const int KB = K / kBK, NB = N / kBM;
     if (dX_bf16) {
         // dX[t][k] = bf16(scale) * sum_n dY[t][n] W_eff[n][k]: A = dY [T][N], B = W_eff^T [K][N]
         if (launch_kernel(weff_t_bf16_kernel, dim3(KB * NB), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(vals), meta, N, K, Wt) != cudaSuccess)
             return SBN_ERR_CUDA;
         ++g_launch_count;
-        const sbn_status st = run_gemm_bf16(dY_bf16, T, static_cast<uint64_t>(N), Wt, K, static_cast<uint64_t>(N), N, dX_bf16, true, w_scale, s);
+        const sbn_status st = run_gemm_bf16(false, dY_bf16, T, static_cast<uint64_t>(N), Wt, K, static_cast<uint64_t>(N), N, dX_bf16, true, w_scale, s);
         if (st != SBN_OK) return st;
     }
     if (dW) {
-        // dW[n][k] = sum_t dY[t][n] x_q[t][k]: A = dY^T [N][Tp], B = x_q^T [K][Tp] (token rows zero-padded to Tp)
-        if (launch_kernel(xq_t_bf16_kernel, dim3(KB * TB), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(xq), a_scale, T, K, tp, XT) != cudaSuccess)
+        // dW[n][k] = sum_t dY[t][n] x_q[t][k]
+        // both operands as they lie in memory, token-major: dY [T][N] and x_q [T][K] (bf16 copy of the
+        // fake-quantised activations); the MMA reads them MN-major, the contraction runs down the rows
+        const unsigned blocks = static_cast<unsigned>(std::min<size_t>((static_cast<size_t>(T) * (K / 16) + kPrepThreads - 1) / kPrepThreads,
+                                                                           static_cast<size_t>(device_sm_count()) * 8));
+        if (launch_kernel(xq_bf16_kernel, dim3(blocks), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(xq), a_scale, T, K, XT) != cudaSuccess)
             return SBN_ERR_CUDA;
         ++g_launch_count;
-        if (launch_kernel(transpose_bf16_kernel, dim3(NB * TB), dim3(kPrepThreads), 0, s, static_cast<const uint16_t*>(dY_bf16), T, N, tp, dYT) != cudaSuccess)
-            return SBN_ERR_CUDA;
-        ++g_launch_count;
-        const sbn_status st = run_gemm_bf16(dYT, N, static_cast<uint64_t>(tp), XT, K, static_cast<uint64_t>(tp), tp, dW, false, nullptr, s);
+        const sbn_status st = run_gemm_bf16(true, dY_bf16, N, static_cast<uint64_t>(N), XT, K, static_cast<uint64_t>(K), T, dW, false, nullptr, s);
         if (st != SBN_OK) return st;
     }
     return SBN_OK;
