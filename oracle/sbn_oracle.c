@@ -464,30 +464,6 @@ uint64_t sbn_oracle_flip_count(const uint8_t *mask_a, const uint8_t *mask_b, int
     return c;
 }
 
-/* ---------------------------------------------------------------------------------------------
- * The whole layer, sparse (Eq. 4 with W_eff) -- route (ii) -- and dense (Sec. 2.1's BitLinear).
- * ------------------------------------------------------------------------------------------- */
-void sbn_oracle_sparse_bitlinear(const int8_t *xq, const float *a_scale, int64_t T,
-                                 const int8_t *vals, const uint8_t *meta, float scale,
-                                 int64_t N, int64_t K, const float *bias,
-                                 float *y, int32_t *acc_out)
-{
-    int32_t *acc = acc_out ? acc_out : (int32_t *)malloc((size_t)(T * N) * sizeof(int32_t));
-    sbn_oracle_acc_packed(xq, vals, meta, T, N, K, acc);
-    if (y) sbn_oracle_dequant(acc, scale, a_scale, bias, T, N, y);
-    if (!acc_out) free(acc);
-}
-
-void sbn_oracle_bitlinear(const int8_t *xq, const float *a_scale, int64_t T,
-                          const int8_t *dense_q, float scale, int64_t N, int64_t K,
-                          const float *bias, float *y, int32_t *acc_out)
-{
-    int32_t *acc = acc_out ? acc_out : (int32_t *)malloc((size_t)(T * N) * sizeof(int32_t));
-    sbn_oracle_acc_dense(xq, dense_q, T, N, K, acc);
-    if (y) sbn_oracle_dequant(acc, scale, a_scale, bias, T, N, y);
-    if (!acc_out) free(acc);
-}
-
 int sbn_oracle_num_threads(void)
 {
 #ifdef _OPENMP
