@@ -477,13 +477,26 @@ def run_ours(args):
     # the next layer's W and x come in (the link is full duplex); each layer has its own staging
     # buffers, and a layer always uses the same stream, which orders its reuse across steps.
     e2e_streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    # The pack kernel's CTAs exchange partial sums, so two pack calls must never overlap on the GPU (see
+    # sbn.h): all of them go to one stream of their own, each behind the copy of its W, and a layer's
+    # forward waits for its pack.
+    pack_stream = torch.cuda.Stream()
 
     def e2e_step():
         for i, L in enumerate(layers):
             p = L.packed
-            with torch.cuda.stream(e2e_streams[i % 2]):
+            st = e2e_streams[i % 2]
+            with torch.cuda.stream(st):
                 L.W_stage.copy_(L.W_host, non_blocking=True)
+                w_in = torch.cuda.Event()
+                w_in.record(st)
+            with torch.cuda.stream(pack_stream):
+                pack_stream.wait_event(w_in)
                 b.sbn_quantize_mask_pack(L.W_stage, p["vals"], p["meta"], p["w_scale"], p["ws"])
+                packed = torch.cuda.Event()
+                packed.record(pack_stream)
+            with torch.cuda.stream(st):
+                st.wait_event(packed)
                 b.sbn_layer_forward_host(L.x_host, L.x_stage, L.xq, L.a_scale, p["w_scale"], L.y, L.y_host,
                                          vals=p["vals"], meta=p["meta"], ws=L.ws)
     e2e_steps = max(2, min(args.steps, 5))
@@ -493,11 +506,11 @@ def run_ours(args):
     s2 = torch.cuda.Event(enable_timing=True)
     e2 = torch.cuda.Event(enable_timing=True)
     s2.record(stream)
-    for st in e2e_streams:
+    for st in e2e_streams + [pack_stream]:
         st.wait_event(s2)
     for _ in range(e2e_steps):
         e2e_step()
-    for st in e2e_streams:
+    for st in e2e_streams + [pack_stream]:
         done_ev = torch.cuda.Event()
         done_ev.record(st)
         stream.wait_event(done_ev)
@@ -1030,6 +1043,27 @@ def run_dynamic_step(args):
         "gpu_launches": b.sbn_launch_count()}))
 
 
+def run_backward(args):
+    """The layer's backward (dual straight-through estimator) on the four 2B-shaped layers at T = 4096 (see
+    backward_rows); --only-step: the qkv shape alone, a few calls (the small case for profiler runs)."""
+    import torch
+    from paper_2603_05168_b200 import binding as b
+    from paper_2603_05168_b200 import build as sbn_build
+    sbn_build.build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    shapes = inputs.SHAPES_2B[:1] if args.only_step else inputs.SHAPES_2B
+    layers = [Layer(n, K, N, T_TOKENS, seed=1 + i, torch=torch, b=b) for i, (n, K, N) in enumerate(shapes)]
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    rows = backward_rows(torch, b, peaks, layers, _cold_timer(torch, stream, flush), 3 if args.only_step else 12)
+    print(json.dumps({"metric": "dual-STE backward of one Sparse-BitLinear layer: dX = dY w_masked, dW = dY^T x_q (bf16, fp32 accumulation)",
+                      "unit": "us", "workload": "bwd", "tokens": T_TOKENS, "rows": rows,
+                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s", "gpu_launches": b.sbn_launch_count()}))
+
+
 def run_mma_probe(args):
     """What the K-loop of the large-T GEMM kernel costs, piece by piece (timing only: with a probe flag set
     the kernel's results are wrong).  One tile per CTA pair (74 feature tiles x one token tile), so nothing
@@ -1118,13 +1152,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="headline line only: skip the 7B-class isolated GEMMs, the sustained run and the few-token rows")
-    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68", "mmaprobe"],
+    ap.add_argument("--workload", default="2b", choices=sorted(WORKLOADS) + ["decode", "decode7b", "dyn", "p68", "mmaprobe", "bwd"],
                     help="2b = the headline workload; 7b / down7b = 7B-class shapes (down7b: one layer, for profiling); "
                          "decode = small-T sweep (T in 1..512), sparse vs dense, cold L2 and streamed; "
                          "decode7b = the same on 7B-class matrices at T <= 64, with the 2-bit packed weights as a third arm; "
                          "dyn = dynamic-mask training step: re-pack 30 x 7 matrices + forward at T=2048; "
                          "p68 = the 6:8 pattern next to 2:4 and dense on the same matrices; "
-                         "mmaprobe = timing experiments on the large-T kernel's K-loop (loads, metadata copies, MMA issue)")
+                         "mmaprobe = timing experiments on the large-T kernel's K-loop (loads, metadata copies, MMA issue); "
+                         "bwd = the layer's backward (dual straight-through estimator) on the 2B shapes")
     ap.add_argument("--masters", default="fp32", choices=["fp32", "bf16"],
                     help="precision of the master weights the pack kernel reads (default fp32, the configuration of the metric)")
     ap.add_argument("--only-step", action="store_true", help="time the step only (used for profiler runs)")
@@ -1139,6 +1174,8 @@ def main():
         run_pattern68(args)
     elif args.workload == "mmaprobe":
         run_mma_probe(args)
+    elif args.workload == "bwd":
+        run_backward(args)
     else:
         run_ours(args)
 
