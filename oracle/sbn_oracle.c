@@ -47,8 +47,12 @@
 /* ---------------------------------------------------------------------------------------------
  * Eq. 1 (scale): gamma = ||W||_1 / (d_out * d_in), accumulated in double in row-major order.
  * scale = max(gamma, 1e-5) (Algorithm 2's clamp).
- * near_tie (optional) is set to 1 when a second summation order (pairwise) gives a different
- * fp32 gamma: the caller should then reseed instead of reporting a mismatch.
+ * near_tie (optional) is set to 1 when the ORDER of the double-precision additions can decide the fp32
+ * value of gamma: when a second order (pairwise) does round differently, or when S / D lies within
+ * 8 * sqrt(D) * 2^-53 (relative) of the midpoint between two fp32 values -- the typical spread of
+ * double-precision sums of D terms taken in different orders.  An implementation that adds the same
+ * doubles in an order of its own (a parallel reduction) may then round the other way without being
+ * wrong; the caller should reseed instead of reporting a mismatch.
  * ------------------------------------------------------------------------------------------- */
 static double pairwise_abs_sum(const float *w, int64_t n)
 {
@@ -71,7 +75,15 @@ void sbn_oracle_absmean_scale(const float *W, int64_t N, int64_t K,
     if (near_tie) {
         double S2 = pairwise_abs_sum(W, D);
         float g2 = (D > 0) ? (float)(S2 / (double)D) : 0.0f;
-        *near_tie = (g2 != gamma);
+        int close = 0;
+        if (D > 0 && gamma > 0.0f) {
+            const double q = S / (double)D;
+            const double tol = 8.0 * sqrt((double)D) * ldexp(1.0, -53) * q;
+            const double up = 0.5 * ((double)gamma + (double)nextafterf(gamma, INFINITY));
+            const double dn = 0.5 * ((double)gamma + (double)nextafterf(gamma, 0.0f));
+            close = (fabs(q - up) <= tol) || (fabs(q - dn) <= tol);
+        }
+        *near_tie = (g2 != gamma) || close;
     }
     if (gamma_out) *gamma_out = gamma;
     if (scale_out) *scale_out = (gamma > SBN_ORACLE_EPS) ? gamma : SBN_ORACLE_EPS;

@@ -662,7 +662,14 @@ def test_near_tie_flag_fires_when_the_summation_order_decides_gamma():
     gamma, scale, near_tie = oracle.absmean_scale(W)
     assert gamma == np.float32(2.0 ** 23) and scale == gamma
     assert near_tie
-    # an ordinary matrix is not flagged, and neither is the same matrix without the decisive half
+    # an ordinary matrix is not flagged
     assert not oracle.absmean_scale(inputs.latent_weights(128, 256, seed=3))[2]
+    # a sum that lies ON an fp32 midpoint is flagged even when the two orders the oracle tries agree
+    # (without the second half both give 2^30 + 64): a third order could still round the other way
     W[0, 64:] = 0.0
-    assert not oracle.absmean_scale(W)[2]
+    assert oracle.absmean_scale(W)[2]
+    # ... and one that is a comfortable 2^-30 (relative) away from the midpoint is not
+    V = np.zeros((1, 128), np.float32)
+    V[0, 0] = 2.0 ** 30
+    V[0, 1] = 64.0 + 2.0 ** -4
+    assert not oracle.absmean_scale(V)[2]
