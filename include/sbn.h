@@ -192,9 +192,10 @@ typedef struct {
     const float *gamma_hint;          /* device, one fp32, or NULL: an estimate of this matrix's gamma, e.g. the
                                          w_scale of the previous training step (may be the very w_scale buffer
                                          above: it is read before it is written).  A speed hint only -- results
-                                         never depend on it.  With a hint within a few percent of gamma the
-                                         kernel need not sample the matrix first; a hint that is far off (or not a
-                                         positive finite number) costs a second pass over that matrix */
+                                         never depend on it.  With a hint within 0.5 % of gamma the kernel need
+                                         not sample the matrix first and finds almost nothing to fix up afterwards; a
+                                         hint that is further off costs a second pass over that matrix, one that is
+                                         not a positive finite number is ignored */
 } sbn_pack_job;
 size_t sbn_batch_workspace_bytes(int count);
 sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job *jobs, void *ws, size_t ws_bytes,

@@ -240,6 +240,7 @@ __device__ __forceinline__ float qmp_sample_gamma(const QmpDesc& d, double* s_wa
 }
 
 // Appends the undecided ones of four consecutive kept values (bytes byte_off .. byte_off + 3 of vals).
+template <int CAP = kQmpListCap>
 __device__ __forceinline__ void qmp_list_undecided(const float (&k)[4], const float thr_lo, const float thr_hi,
                                                    const uint32_t byte_off, QmpEntry* list, unsigned int* list_count) {
     bool und[4];
@@ -255,7 +256,7 @@ __device__ __forceinline__ void qmp_list_undecided(const float (&k)[4], const fl
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (und[i]) {
-                if (at < static_cast<unsigned int>(kQmpListCap)) { list[at].byte_off = byte_off + i; list[at].w = k[i]; }
+                if (at < static_cast<unsigned int>(CAP)) { list[at].byte_off = byte_off + i; list[at].w = k[i]; }
                 ++at;
             }
         }

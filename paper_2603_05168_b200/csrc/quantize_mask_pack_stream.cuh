@@ -7,13 +7,19 @@
 // matrix, a third of a batch of 2B-shaped matrices and more for small ones.  Here none of that stops
 // the stream:
 //
-//   warps 0..30   stream pass 1 of matrix 0, 1, 2, ... back to back, each thread its fixed share of the
-//                 CTA's range (fixed order of additions: the partial sums are reproducible bit for bit);
-//                 no CTA-wide barrier between matrices.  A warp leaves its sum |W| and flip count of
-//                 matrix m in shared memory and counts itself on `arrived`.
+//   warp 30       the loader: one lane copies the CTA's range of matrix 0, 1, 2, ... into a ring of shared-
+//                 memory stages (60 units = 30 KB of fp32 weights each, four stages) with bulk copies that
+//                 count their bytes on a stage's `full` barrier; it refills a stage as soon as the 30
+//                 computing warps have released it (`empty` barrier).  Three stages are always in flight,
+//                 whatever the computing warps are busy with: the loads cost no registers and no issue slots.
+//   warps 0..29   pass 1 of matrix 0, 1, 2, ... back to back, stage by stage: a warp takes two units of a
+//                 stage (a half-warp per unit, a lane two adjacent groups), always the same ones (fixed order
+//                 of additions: the partial sums are reproducible bit for bit); no CTA-wide barrier between
+//                 matrices.  A warp leaves its sum |W| and flip count of matrix m in shared memory and
+//                 counts itself on `arrived`.
 //   warp 31       the finisher.  For matrix m, in this order:
 //                   bracket of matrix m + 2 (from the caller's hint, or a sample of the matrix);
-//                   wait until the 31 streaming warps have arrived for m, add their sums in a fixed
+//                   wait until the 30 computing warps have arrived for m, add their sums in a fixed
 //                   order, publish {tag, partial} in the workspace;
 //                   exchange of matrix m - 1 (published by every CTA one matrix ago, so the slots are
 //                   there already), exact gamma, scale, threshold; fix-up of the listed values of
@@ -33,9 +39,14 @@
 
 namespace sbn {
 
-constexpr int kQmpStreamWarps = kQmpWarps - 1;             // 31 stream, warp 31 finishes
+constexpr int kQmpStreamWarps = kQmpWarps - 2;             // 30 compute, warp 30 loads, warp 31 finishes
+constexpr int kQmpLoaderWarp = kQmpWarps - 2;
 constexpr int kQmpLists = 3;
-constexpr int kQmpStreamSmemBytes = kQmpLists * kQmpListCap * 8;
+constexpr int kQmpStreamListCap = 4096;                    // undecided entries per CTA and matrix (see qmp_bracket_from)
+constexpr int kQmpStageUnits = 2 * kQmpStreamWarps;        // a half-warp per unit
+constexpr int kQmpStages = 4;
+constexpr int kQmpStageBytes = kQmpStageUnits * 512;       // fp32 units; bf16 units fill half of a stage
+constexpr int kQmpStreamSmemBytes = kQmpStages * kQmpStageBytes + kQmpLists * kQmpStreamListCap * 8;
 constexpr int kQmpMaxBatch = 1024;                         // thresholds of put-off second passes live in shared memory
 
 struct QmpStreamShared {
@@ -50,6 +61,65 @@ struct QmpStreamShared {
     int abort;
     float thr_tail;
     float thr_second_pass[kQmpMaxBatch];                   // >= 0: this matrix needs the exact second pass with this threshold
+    unsigned long long bar_full[kQmpStages];               // a stage's bytes have landed
+    unsigned long long bar_empty[kQmpStages];              // the computing warps are done with a stage
+    uint32_t ring_issued, ring_stage, ring_phase;          // the loader's last position
+};
+
+// mbarrier and bulk-copy wrappers of the stage ring
+__device__ __forceinline__ uint32_t qmp_smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void qmp_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void qmp_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void qmp_mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool qmp_mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait for a barrier phase; gives up (false) when the CTA aborts or the limit runs out.  With
+// `drain` it ignores the abort flag: the loader uses it to see its last copies land before the CTA leaves.
+__device__ __forceinline__ bool qmp_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool drain = false) {
+    if (qmp_mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0ull;
+    unsigned int spins = 0;
+    while (!qmp_mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0u) {
+            if (!drain && *abort_flag) return false;
+            const unsigned long long now = global_timer_ns_qmp();
+            if (t0 == 0ull) {
+                t0 = now;
+            } else if (now - t0 > *reinterpret_cast<volatile unsigned long long*>(&g_wait_limit_ns)) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, static_cast<int>(SBN_ERR_TIMEOUT));
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void qmp_bulk_load(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ float4 qmp_lds128(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+// Position of the ring: stage and the parity of its current use.
+struct QmpRing {
+    uint32_t stage, phase;
+    __device__ __forceinline__ void advance() { if (++stage == kQmpStages) { stage = 0; phase ^= 1u; } }
 };
 
 __device__ __forceinline__ QmpDesc qmp_desc_of(const QmpDesc& first, const QmpDesc* rest, int m) {
@@ -78,9 +148,14 @@ __device__ __forceinline__ bool qmp_wait_ge(volatile int* word, int want, volati
     return true;
 }
 
-// lo / hi of the bracket around the threshold that gamma_est predicts (see quantize_mask_pack.cuh)
-__device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_units, float& lo, float& hi) {
-    const float b = num_units < kQmpSmallMatrixUnits ? kQmpBracketSmall : kQmpBracket;
+// lo / hi of the bracket around the threshold that gamma_est predicts (see quantize_mask_pack.cuh).  An
+// estimate from the caller (the scale of the previous training step, Sec. 2.2: the weights move by a
+// learning-rate-sized step) gets a bracket six times narrower than one from a sample: almost no warp then
+// meets an undecided value, and listing them is a tenth of pass 1's instructions otherwise.  A hint that
+// is off by more than that costs the exact second pass, never the result.
+constexpr float kQmpBracketHint = 0.005f;
+__device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_units, bool from_hint, float& lo, float& hi) {
+    const float b = from_hint ? kQmpBracketHint : (num_units < kQmpSmallMatrixUnits ? kQmpBracketSmall : kQmpBracket);
     lo = 0.5f * fmaxf(gamma_est * (1.0f - b), kEps) * (1.0f - 1e-6f);
     hi = 0.5f * fmaxf(gamma_est * (1.0f + b), kEps) * (1.0f + 1e-6f);
 }
@@ -116,67 +191,109 @@ __device__ __forceinline__ float qmp_sample_gamma_warp(const QmpDesc& d, int lan
     return acc / (static_cast<float>(n_s) * 128.0f);
 }
 
-// Pass 1 of one matrix for the streaming warps: this thread's share of the CTA's range.  Returns the
-// thread's sum |W|; metadata, provisional values, undecided list and flip count as in quantize_mask_pack.cuh.
-// A lane takes two adjacent groups (32 B of a row); a half-warp covers one 512 B unit, the 31 warps 62
-// units per step, two steps per iteration (four independent groups per thread keep the ALUs fed).
+// The loader: walks the CTA's ranges of matrix 0, 1, 2, ... stage by stage.  qmp_loader_issue starts up to
+// `max_copies` copies (each after its stage has been released) and returns false if a wait ran out.
+struct QmpLoader {
+    int m;                       // matrix being loaded
+    uint32_t u, u_end;           // next unit and end of the CTA's range of it (valid while `open`)
+    uint32_t unit_bytes;
+    const char* W;
+    bool open;
+    QmpRing ring;
+    uint32_t issued;             // copies of this launch (the drain after an abort needs it)
+};
+__device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpDesc& first, const QmpDesc* rest, int count, uint32_t max_copies,
+                                                 uint32_t ring_base, uint32_t bar_full0, uint32_t bar_empty0, volatile int* abort_flag) {
+    for (;;) {
+        while (!L.open) {
+            if (L.m >= count) return true;
+            const QmpDesc d = qmp_desc_of(first, rest, L.m);
+            const QmpRange rg = qmp_range(d);
+            L.u = rg.u_begin;
+            L.u_end = rg.u_end;
+            L.unit_bytes = d.w_bf16 ? 256u : 512u;
+            L.W = static_cast<const char*>(d.W);
+            if (L.u < L.u_end) L.open = true; else ++L.m;
+        }
+        if (max_copies == 0u) return true;
+        --max_copies;
+        if (!qmp_mbar_wait(bar_empty0 + 8u * L.ring.stage, L.ring.phase ^ 1u, abort_flag)) return false;
+        const uint32_t bytes = min(L.u_end - L.u, static_cast<uint32_t>(kQmpStageUnits)) * L.unit_bytes;
+        qmp_mbar_expect_tx(bar_full0 + 8u * L.ring.stage, bytes);
+        qmp_bulk_load(ring_base + L.ring.stage * kQmpStageBytes, L.W + static_cast<size_t>(L.u) * L.unit_bytes, bytes, bar_full0 + 8u * L.ring.stage);
+        ++L.issued;
+        L.ring.advance();
+        L.u += kQmpStageUnits;
+        if (L.u >= L.u_end) { L.open = false; ++L.m; }
+    }
+}
+
+// Pass 1 of one matrix for a computing warp: its two units of every stage of the CTA's range.  Returns
+// the thread's sum |W| (false in `ok` if a wait ran out); metadata, provisional values, undecided list
+// and flip count as in quantize_mask_pack.cuh.  A lane takes two adjacent groups (32 B of a row).
 template <bool BF16>
 __device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
-                                                   QmpEntry* list, unsigned int* list_count, unsigned int& flips) {
+                                                   QmpEntry* list, unsigned int* list_count, unsigned int& flips,
+                                                   QmpRing& ring, uint32_t ring_base, uint32_t bar_full0, uint32_t bar_empty0,
+                                                   volatile int* abort_flag, bool& ok) {
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const uint32_t l16 = lane & 15;
     const uint32_t KB = d.KB;
-    constexpr uint32_t kStep = 2 * kQmpStreamWarps;
     constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
-    const int step_n = static_cast<int>(kStep / KB), step_kb = static_cast<int>(kStep % KB);
+    const int step_n = static_cast<int>(kQmpStageUnits / KB), step_kb = static_cast<int>(kQmpStageUnits % KB);
     const bool count_flips = d.prev_meta != nullptr;
+    // |k| in [thr_lo, thr_hi) implies | |k| - mid | <= half (the subtraction is exact, thr_hi < 2 thr_lo;
+    // `half` is rounded up by far more than the rounding of `mid`): a cheap test with no false negatives
+    const float mid = 0.5f * (thr_lo + thr_hi);
+    const float half = fmaf(thr_hi - thr_lo, 0.50005f, thr_hi * 2.4e-7f);
     double acc = 0.0;
-    const uint32_t u_first = rg.u_begin + 2 * warp + (lane >> 4);
-    int n_cur = static_cast<int>(u_first / KB);
-    int kb_cur = static_cast<int>(u_first - static_cast<uint32_t>(n_cur) * KB);
-    if (threadIdx.x == 0) {
-        for (int j = 0; j < kQmpPrefetchAhead; ++j) {
-            const uint32_t ub = rg.u_begin + j * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
-        }
-    }
-    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += 2 * kStep) {
-        if (threadIdx.x == 0) {
-            const uint32_t ub = u0 + kQmpPrefetchAhead * 2 * kStep;
-            if (ub < rg.u_end) prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(ub) * kUnitBytes, min(rg.u_end - ub, 2 * kStep) * kUnitBytes);
-        }
-        float4 va[2], vb[2];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
-            va[q] = vb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (uq < rg.u_end) qmp_load_group_pair<BF16>(d.W, uq, l16, va[q], vb[q]);
-        }
-        acc += (abs_sum4(va[0]) + abs_sum4(vb[0])) + (abs_sum4(va[1]) + abs_sum4(vb[1]));
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-            const uint32_t uq = u0 + (u_first - rg.u_begin) + q * kStep;
-            const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-            const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
-            n_cur += step_n;
-            kb_cur += step_kb;
-            if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
-            if (uq < rg.u_end) {
-                float k[4];
-                const uint32_t nib0 = select_pair(va[q], k[0], k[1]);
-                const uint32_t nib1 = select_pair(vb[q], k[2], k[3]);
-                const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
-                if (count_flips) {
-                    const uint32_t prev = d.prev_meta[m_off];
-                    flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
-                                    (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
-                }
-                d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
-                const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
-                reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
-                qmp_list_undecided(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
+    const uint32_t in_stage = 2u * warp + (lane >> 4);               // this half-warp's unit of every stage
+    uint32_t u = rg.u_begin + in_stage;
+    int n_cur = static_cast<int>(u / KB);
+    int kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
+    const uint32_t src_off = in_stage * kUnitBytes + l16 * (kUnitBytes / 16u);
+    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += kQmpStageUnits, u += kQmpStageUnits) {
+        if (!qmp_mbar_wait(bar_full0 + 8u * ring.stage, ring.phase, abort_flag)) { ok = false; break; }
+        float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+        const bool mine = u < rg.u_end;
+        if (mine) {
+            const uint32_t src = ring_base + ring.stage * kQmpStageBytes + src_off;
+            if constexpr (BF16) {
+                const float4 raw = qmp_lds128(src);
+                const uint32_t r0 = __float_as_uint(raw.x), r1 = __float_as_uint(raw.y), r2 = __float_as_uint(raw.z), r3 = __float_as_uint(raw.w);
+                va = make_float4(bf16lo_to_f32(r0), bf16hi_to_f32(r0), bf16lo_to_f32(r1), bf16hi_to_f32(r1));
+                vb = make_float4(bf16lo_to_f32(r2), bf16hi_to_f32(r2), bf16lo_to_f32(r3), bf16hi_to_f32(r3));
+            } else {
+                va = qmp_lds128(src);
+                vb = qmp_lds128(src + 16u);
             }
+        }
+        __syncwarp();
+        if (lane == 0) qmp_mbar_arrive(bar_empty0 + 8u * ring.stage);      // the values are in registers: the stage may be refilled
+        ring.advance();
+        const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
+        const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+        n_cur += step_n;
+        kb_cur += step_kb;
+        if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+        if (mine) {
+            acc += abs_sum4(va) + abs_sum4(vb);
+            float k[4];
+            const uint32_t nib0 = select_pair(va, k[0], k[1]);
+            const uint32_t nib1 = select_pair(vb, k[2], k[3]);
+            const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
+            if (count_flips) {
+                const uint32_t prev = d.prev_meta[m_off];
+                flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
+                                (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
+            }
+            d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
+            const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
+            reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
+            const float far = fminf(fminf(fabsf(fabsf(k[0]) - mid), fabsf(fabsf(k[1]) - mid)),
+                                    fminf(fabsf(fabsf(k[2]) - mid), fabsf(fabsf(k[3]) - mid)));
+            if (far <= half) qmp_list_undecided<kQmpStreamListCap>(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
         }
     }
     return acc;
@@ -185,7 +302,7 @@ __device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRa
 // What the exact gamma decides for a matrix whose pass 1 is complete: true if the listed values were
 // all that had to be redone (and `fix` should run), false if the whole range must be ternarised again.
 __device__ __forceinline__ bool qmp_bracket_holds(const QmpDesc& d, float thr, float lo, float hi, unsigned int listed) {
-    return lo <= thr && thr <= hi && listed <= static_cast<unsigned int>(kQmpListCap) && d.dense_q == nullptr &&
+    return lo <= thr && thr <= hi && listed <= static_cast<unsigned int>(kQmpStreamListCap) && d.dense_q == nullptr &&
            d.num_units <= (1u << 26);                        // listed byte offsets are 32-bit
 }
 
@@ -193,18 +310,28 @@ __global__ void __launch_bounds__(kQmpThreads, 1)
 quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
                                  QmpSlot* slots, unsigned long long* generation, unsigned long long call_nonce,
                                  int test_withhold_slot) {
-    extern __shared__ QmpEntry s_list[];                // [kQmpLists][kQmpListCap]
+    extern __shared__ __align__(128) unsigned char s_dyn[];   // [kQmpStages][kQmpStageBytes] ring, then [kQmpLists][kQmpStreamListCap] entries
+    QmpEntry* const s_list = reinterpret_cast<QmpEntry*>(s_dyn + kQmpStages * kQmpStageBytes);
     __shared__ QmpStreamShared sh;
     __shared__ double s_warp[kQmpWarps];
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     volatile int* const abort_flag = &sh.abort;
+    const uint32_t ring_base = qmp_smem_u32(s_dyn);
+    const uint32_t bar_full0 = qmp_smem_u32(&sh.bar_full[0]), bar_empty0 = qmp_smem_u32(&sh.bar_empty[0]);
     if (threadIdx.x == 0) {
         sh.bracket_upto = 0;
         sh.fixed_upto = 0;
         sh.abort = 0;
+        sh.ring_issued = 0u; sh.ring_stage = 0u; sh.ring_phase = 0u;
         for (int i = 0; i < kQmpLists; ++i) { sh.arrived[i] = 0u; sh.list_count[i] = 0u; sh.flip_total[i] = 0ull; }
+        for (int i = 0; i < kQmpStages; ++i) {
+            qmp_mbar_init(bar_full0 + 8u * i, 1u);                     // the loader's expect_tx
+            qmp_mbar_init(bar_empty0 + 8u * i, kQmpStreamWarps);       // one arrival per computing warp
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int i = threadIdx.x; i < kQmpMaxBatch; i += kQmpThreads) sh.thr_second_pass[i] = -1.0f;
     __syncthreads();
@@ -214,18 +341,25 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     const unsigned long long gen0 = *reinterpret_cast<volatile unsigned long long*>(generation);
     const unsigned long long tag = qmp_tag(call_nonce, gen0);
 
+    // ---- the loader fills the ring before anything else: the first stages travel while the brackets are made
+    QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u, 0u}, 0u};
+    const bool is_loader = warp == kQmpLoaderWarp && lane == 0;
+    if (is_loader) qmp_loader_issue(loader, first, rest, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
+
     // ---- brackets of the first two matrices: all threads
     for (int m = 0; m < min(count, 2); ++m) {
         const QmpDesc d = qmp_desc_of(first, rest, m);
         float g;
-        if (!qmp_hint(d, g)) g = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
-        if (threadIdx.x == 0) qmp_bracket_from(g, d.num_units, sh.bracket[m & 3][0], sh.bracket[m & 3][1]);
+        const bool hinted = qmp_hint(d, g);
+        if (!hinted) g = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
+        if (threadIdx.x == 0) qmp_bracket_from(g, d.num_units, hinted, sh.bracket[m & 3][0], sh.bracket[m & 3][1]);
     }
     if (threadIdx.x == 0) sh.bracket_upto = min(count, 2);
     __syncthreads();
 
     if (warp < kQmpStreamWarps) {
-        // ------------------------------------------------------------------ streaming warps
+        // ------------------------------------------------------------------ computing warps
+        QmpRing ring{0u, 0u};
         for (int m = 0; m < count; ++m) {
             const int slot = m % kQmpLists;
             if (!qmp_wait_ge(&sh.bracket_upto, m + 1, abort_flag)) break;
@@ -235,8 +369,12 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             const float lo = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][0]);
             const float hi = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][1]);
             unsigned int flips = 0;
-            double mine = d.w_bf16 ? qmp_stream_pass1<true>(d, rg, lo, hi, s_list + slot * kQmpListCap, &sh.list_count[slot], flips)
-                                   : qmp_stream_pass1<false>(d, rg, lo, hi, s_list + slot * kQmpListCap, &sh.list_count[slot], flips);
+            bool ok = true;
+            double mine = d.w_bf16 ? qmp_stream_pass1<true>(d, rg, lo, hi, s_list + slot * kQmpStreamListCap, &sh.list_count[slot], flips,
+                                                            ring, ring_base, bar_full0, bar_empty0, abort_flag, ok)
+                                   : qmp_stream_pass1<false>(d, rg, lo, hi, s_list + slot * kQmpStreamListCap, &sh.list_count[slot], flips,
+                                                             ring, ring_base, bar_full0, bar_empty0, abort_flag, ok);
+            if (!ok) break;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
@@ -251,6 +389,15 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             }
             __syncwarp();
         }
+    } else if (warp == kQmpLoaderWarp) {
+        // ------------------------------------------------------------------ the loader (warp 30, one lane)
+        if (is_loader) {
+            qmp_loader_issue(loader, first, rest, count, 0xFFFFFFFFu, ring_base, bar_full0, bar_empty0, abort_flag);
+            sh.ring_issued = loader.issued;                  // for the drain, should the CTA abort
+            sh.ring_stage = loader.ring.stage;
+            sh.ring_phase = loader.ring.phase;
+        }
+        __syncwarp();
     } else {
         // ------------------------------------------------------------------ the finisher (warp 31)
         bool ok = true;
@@ -260,9 +407,10 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             if (m + 2 < count) {
                 const QmpDesc d2 = qmp_desc_of(first, rest, m + 2);
                 float g;
-                if (!qmp_hint(d2, g)) g = d2.w_bf16 ? qmp_sample_gamma_warp<true>(d2, lane) : qmp_sample_gamma_warp<false>(d2, lane);
+                const bool hinted = qmp_hint(d2, g);
+                if (!hinted) g = d2.w_bf16 ? qmp_sample_gamma_warp<true>(d2, lane) : qmp_sample_gamma_warp<false>(d2, lane);
                 if (lane == 0) {
-                    qmp_bracket_from(g, d2.num_units, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1]);
+                    qmp_bracket_from(g, d2.num_units, hinted, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1]);
                     __threadfence_block();
                     *reinterpret_cast<volatile int*>(&sh.bracket_upto) = m + 3;
                 }
@@ -347,7 +495,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
                 thr = __shfl_sync(0xFFFFFFFFu, thr, 0);
                 const unsigned int listed = *reinterpret_cast<volatile unsigned int*>(&sh.list_count[pslot]);
                 if (qmp_bracket_holds(dp, thr, sh.bracket[(m - 1) & 3][0], sh.bracket[(m - 1) & 3][1], listed)) {
-                    const QmpEntry* list = s_list + pslot * kQmpListCap;
+                    const QmpEntry* list = s_list + pslot * kQmpStreamListCap;
                     uint8_t* vb = reinterpret_cast<uint8_t*>(dp.vals);
                     for (unsigned int e = lane; e < listed; e += 32u) {
                         const float w = list[e].w;
@@ -368,7 +516,19 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
         }
     }
     __syncthreads();
-    if (sh.abort) return;
+    if (sh.abort) {
+        // No bulk copy may still be writing this CTA's shared memory when it leaves: the last
+        // min(issued, kQmpStages) copies are the ones that can be in flight; the ring position points past the newest.
+        if (threadIdx.x == 0) {
+            QmpRing ring{sh.ring_stage, sh.ring_phase};
+            const uint32_t back = min(sh.ring_issued, static_cast<uint32_t>(kQmpStages));
+            for (uint32_t j = 0; j < back; ++j) {
+                if (ring.stage == 0u) { ring.stage = kQmpStages - 1; ring.phase ^= 1u; } else { --ring.stage; }
+                qmp_mbar_wait(bar_full0 + 8u * ring.stage, ring.phase, abort_flag, true);
+            }
+        }
+        return;
+    }
 
     // ---- tail: the last matrix, all threads
     {
@@ -412,7 +572,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
         const float thr = sh.thr_tail;
         const unsigned int listed = sh.list_count[slot];
         if (qmp_bracket_holds(d, thr, sh.bracket[m & 3][0], sh.bracket[m & 3][1], listed)) {
-            const QmpEntry* list = s_list + slot * kQmpListCap;
+            const QmpEntry* list = s_list + slot * kQmpStreamListCap;
             uint8_t* vb = reinterpret_cast<uint8_t*>(d.vals);
             for (unsigned int e = threadIdx.x; e < listed; e += kQmpThreads) {
                 const float w = list[e].w;
