@@ -665,7 +665,8 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
             ++g_launch_count;
             if (err != cudaSuccess) return SBN_ERR_CUDA;
         }
-        const sbn_status st = launch_quantize_mask_pack_stream(descs[static_cast<size_t>(lo)], descs_dev + lo, n_here, max_units,
+        const sbn_status st = launch_quantize_mask_pack_stream(descs[static_cast<size_t>(lo)], descs[static_cast<size_t>(lo + (n_here > 1 ? 1 : 0))], descs_dev + lo,
+                                                               n_here, max_units,
                                                                slots + static_cast<size_t>(lo) * kQmpMaxCtas, generation, s);
         if (st != SBN_OK) return st;
     }

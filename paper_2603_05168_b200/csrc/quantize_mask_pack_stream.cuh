@@ -122,8 +122,14 @@ struct QmpRing {
     __device__ __forceinline__ void advance() { if (++stage == kQmpStages) { stage = 0; phase ^= 1u; } }
 };
 
-__device__ __forceinline__ QmpDesc qmp_desc_of(const QmpDesc& first, const QmpDesc* rest, int m) {
-    return m == 0 ? first : rest[m - 1];
+// Matrix m of the batch: 0 and 1 travel with the launch, `rest` holds 1, 2, ... in global memory.
+struct QmpBatch {
+    const QmpDesc& first;
+    const QmpDesc& second;
+    const QmpDesc* rest;
+};
+__device__ __forceinline__ QmpDesc qmp_desc_of(const QmpBatch& b, int m) {
+    return m == 0 ? b.first : (m == 1 ? b.second : b.rest[m - 1]);
 }
 
 // Bounded wait for a shared-memory word (written by another warp of this CTA) to reach `want`.
@@ -202,12 +208,12 @@ struct QmpLoader {
     QmpRing ring;
     uint32_t issued;             // copies of this launch (the drain after an abort needs it)
 };
-__device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpDesc& first, const QmpDesc* rest, int count, uint32_t max_copies,
+__device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpBatch& batch, int count, uint32_t max_copies,
                                                  uint32_t ring_base, uint32_t bar_full0, uint32_t bar_empty0, volatile int* abort_flag) {
     for (;;) {
         while (!L.open) {
             if (L.m >= count) return true;
-            const QmpDesc d = qmp_desc_of(first, rest, L.m);
+            const QmpDesc d = qmp_desc_of(batch, L.m);
             const QmpRange rg = qmp_range(d);
             L.u = rg.u_begin;
             L.u_end = rg.u_end;
@@ -307,7 +313,7 @@ __device__ __forceinline__ bool qmp_bracket_holds(const QmpDesc& d, float thr, f
 }
 
 __global__ void __launch_bounds__(kQmpThreads, 1)
-quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict__ rest, int count,
+quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, const QmpDesc* __restrict__ rest, int count,
                                  QmpSlot* slots, unsigned long long* generation, unsigned long long call_nonce,
                                  int test_withhold_slot) {
     extern __shared__ __align__(128) unsigned char s_dyn[];   // [kQmpStages][kQmpStageBytes] ring, then [kQmpLists][kQmpStreamListCap] entries
@@ -315,6 +321,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     __shared__ QmpStreamShared sh;
     __shared__ double s_warp[kQmpWarps];
 
+    const QmpBatch batch{first, second, rest};
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     volatile int* const abort_flag = &sh.abort;
@@ -341,18 +348,22 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     const unsigned long long gen0 = *reinterpret_cast<volatile unsigned long long*>(generation);
     const unsigned long long tag = qmp_tag(call_nonce, gen0);
 
-    // ---- the loader fills the ring before anything else: the first stages travel while the brackets are made
+    // ---- the hints of matrices 0 and 1 are asked for first (4-byte reads that would otherwise queue behind
+    // the ring's first megabytes), then the loader fills the ring: the first stages travel while the
+    // brackets are made
+    float g01[2] = {0.0f, 0.0f};
+    bool hinted01[2];
+    hinted01[0] = qmp_hint(first, g01[0]);
+    hinted01[1] = count > 1 && qmp_hint(second, g01[1]);
     QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u, 0u}, 0u};
     const bool is_loader = warp == kQmpLoaderWarp && lane == 0;
-    if (is_loader) qmp_loader_issue(loader, first, rest, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
+    if (is_loader) qmp_loader_issue(loader, batch, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
 
-    // ---- brackets of the first two matrices: all threads
+    // ---- brackets of the first two matrices: all threads (the finisher makes the others, two matrices ahead)
     for (int m = 0; m < min(count, 2); ++m) {
-        const QmpDesc d = qmp_desc_of(first, rest, m);
-        float g;
-        const bool hinted = qmp_hint(d, g);
-        if (!hinted) g = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
-        if (threadIdx.x == 0) qmp_bracket_from(g, d.num_units, hinted, sh.bracket[m & 3][0], sh.bracket[m & 3][1]);
+        const QmpDesc& d = m == 0 ? first : second;
+        if (!hinted01[m]) g01[m] = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
+        if (threadIdx.x == 0) qmp_bracket_from(g01[m], d.num_units, hinted01[m], sh.bracket[m][0], sh.bracket[m][1]);
     }
     if (threadIdx.x == 0) sh.bracket_upto = min(count, 2);
     __syncthreads();
@@ -364,7 +375,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             const int slot = m % kQmpLists;
             if (!qmp_wait_ge(&sh.bracket_upto, m + 1, abort_flag)) break;
             if (!qmp_wait_ge(&sh.fixed_upto, m - (kQmpLists - 1), abort_flag)) break;
-            const QmpDesc d = qmp_desc_of(first, rest, m);
+            const QmpDesc d = qmp_desc_of(batch, m);
             const QmpRange rg = qmp_range(d);
             const float lo = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][0]);
             const float hi = *reinterpret_cast<volatile float*>(&sh.bracket[m & 3][1]);
@@ -392,7 +403,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     } else if (warp == kQmpLoaderWarp) {
         // ------------------------------------------------------------------ the loader (warp 30, one lane)
         if (is_loader) {
-            qmp_loader_issue(loader, first, rest, count, 0xFFFFFFFFu, ring_base, bar_full0, bar_empty0, abort_flag);
+            qmp_loader_issue(loader, batch, count, 0xFFFFFFFFu, ring_base, bar_full0, bar_empty0, abort_flag);
             sh.ring_issued = loader.issued;                  // for the drain, should the CTA abort
             sh.ring_stage = loader.ring.stage;
             sh.ring_phase = loader.ring.phase;
@@ -403,9 +414,9 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
         bool ok = true;
         for (int m = 0; ok && m < count; ++m) {
             const int slot = m % kQmpLists;
-            // bracket of matrix m + 2, well before the streaming warps ask for it
+            // bracket of matrix m + 2, well before the computing warps ask for it
             if (m + 2 < count) {
-                const QmpDesc d2 = qmp_desc_of(first, rest, m + 2);
+                const QmpDesc d2 = qmp_desc_of(batch, m + 2);
                 float g;
                 const bool hinted = qmp_hint(d2, g);
                 if (!hinted) g = d2.w_bf16 ? qmp_sample_gamma_warp<true>(d2, lane) : qmp_sample_gamma_warp<false>(d2, lane);
@@ -419,7 +430,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             // matrix m: every streaming warp has arrived -> this CTA's partial sum, published
             if (!qmp_wait_ge(reinterpret_cast<volatile int*>(&sh.arrived[slot]), kQmpStreamWarps, abort_flag)) { ok = false; break; }
             __threadfence_block();
-            const QmpDesc d = qmp_desc_of(first, rest, m);
+            const QmpDesc d = qmp_desc_of(batch, m);
             {
                 double v = lane < kQmpStreamWarps ? *reinterpret_cast<volatile double*>(&sh.warp_sum[slot][lane]) : 0.0;
                 unsigned int f = lane < kQmpStreamWarps ? *reinterpret_cast<volatile unsigned int*>(&sh.warp_flips[slot][lane]) : 0u;
@@ -442,7 +453,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
             // matrix m - 1: exchange, exact threshold, fix-up
             if (m >= 1) {
                 const int pslot = (m - 1) % kQmpLists;
-                const QmpDesc dp = qmp_desc_of(first, rest, m - 1);
+                const QmpDesc dp = qmp_desc_of(batch, m - 1);
                 const QmpSlot* base = slots + static_cast<size_t>(m - 1) * gridDim.x;
                 // a lane looks after the slots lane, lane + 32, ...: all its flags are polled together, then all
                 // its partial sums are read together (two round trips in all, not two per slot)
@@ -534,7 +545,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     {
         const int m = count - 1;
         const int slot = m % kQmpLists;
-        const QmpDesc d = qmp_desc_of(first, rest, m);
+        const QmpDesc d = qmp_desc_of(batch, m);
         const QmpRange rg = qmp_range(d);
         const QmpSlot* base = slots + static_cast<size_t>(m) * gridDim.x;
         double other = 0.0;
@@ -587,7 +598,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     for (int m = 0; m + 1 < count; ++m) {
         const float thr = sh.thr_second_pass[m];
         if (thr >= 0.0f) {
-            const QmpDesc d = qmp_desc_of(first, rest, m);
+            const QmpDesc d = qmp_desc_of(batch, m);
             const QmpRange rg = qmp_range(d);
             if (d.w_bf16) qmp_pass2_full<true>(d, rg, thr);
             else qmp_pass2_full<false>(d, rg, thr);
@@ -597,8 +608,9 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc* __restrict_
     if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<volatile unsigned long long*>(generation) = gen0 + 1ull;
 }
 
-// Launch for `count` (<= kQmpMaxBatch) matrices: `first` by value, the others already copied to `rest_dev`.
-inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const QmpDesc* rest_dev, int count,
+// Launch for `count` (<= kQmpMaxBatch) matrices: matrices 0 and 1 by value (`second` is ignored when count is 1),
+// matrices 1, 2, ... already copied to `rest_dev`.
+inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const QmpDesc& second, const QmpDesc* rest_dev, int count,
                                                    uint32_t max_units, QmpSlot* slots, unsigned long long* generation,
                                                    cudaStream_t stream) {
     const int test_withhold_slot = g_test_break_waits;
@@ -612,7 +624,7 @@ inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const Q
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
     const cudaError_t err = launch_kernel(quantize_mask_pack_stream_kernel, dim3(grid), dim3(kQmpThreads), kQmpStreamSmemBytes, stream,
-                                          first, rest_dev, count, slots, generation, nonce, test_withhold_slot);
+                                          first, second, rest_dev, count, slots, generation, nonce, test_withhold_slot);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -623,7 +635,7 @@ inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, i
                                             unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
     const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
-    return launch_quantize_mask_pack_stream(d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream);
+    return launch_quantize_mask_pack_stream(d, d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream);
 }
 
 }  // namespace sbn
