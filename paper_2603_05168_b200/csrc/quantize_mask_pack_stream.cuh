@@ -18,12 +18,13 @@
 //                 matrices.  A warp leaves its sum |W| and flip count of matrix m in shared memory and
 //                 counts itself on `arrived`.
 //   warp 31       the finisher.  For matrix m, in this order:
-//                   bracket of matrix m + 2 (from the caller's hint, or a sample of the matrix);
 //                   wait until the 30 computing warps have arrived for m, add their sums in a fixed
 //                   order, publish {tag, partial} in the workspace;
 //                   exchange of matrix m - 1 (published by every CTA one matrix ago, so the slots are
 //                   there already), exact gamma, scale, threshold; fix-up of the listed values of
-//                   m - 1, or a note that m - 1 needs the exact second pass; its list becomes free.
+//                   m - 1, or a note that m - 1 needs the exact second pass; its list becomes free;
+//                   bracket of matrix m + 2 (from the caller's hint, or from a sample of the matrix that
+//                   bulk copies drop into the list just freed).
 //                 All of it runs under pass 1 of the following matrices.
 //   three lists   matrix m - 1 is being fixed up while m waits and m + 1 is being written; a streaming
 //                 warp starts matrix m only once m - 3 is fixed (its list slot is free) and the bracket
@@ -64,6 +65,7 @@ struct QmpStreamShared {
     unsigned long long bar_full[kQmpStages];               // a stage's bytes have landed
     unsigned long long bar_empty[kQmpStages];              // the computing warps are done with a stage
     uint32_t ring_issued, ring_stage, ring_phase;          // the loader's last position
+    unsigned long long bar_sample;                         // the finisher's sample has landed
 };
 
 // mbarrier and bulk-copy wrappers of the stage ring
@@ -160,8 +162,8 @@ __device__ __forceinline__ bool qmp_wait_ge(volatile int* word, int want, volati
 // meets an undecided value, and listing them is a tenth of pass 1's instructions otherwise.  A hint that
 // is off by more than that costs the exact second pass, never the result.
 constexpr float kQmpBracketHint = 0.005f;
-__device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_units, bool from_hint, float& lo, float& hi) {
-    const float b = from_hint ? kQmpBracketHint : (num_units < kQmpSmallMatrixUnits ? kQmpBracketSmall : kQmpBracket);
+__device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_units, bool from_hint, float& lo, float& hi, bool wide = false) {
+    const float b = from_hint ? kQmpBracketHint : ((wide || num_units < kQmpSmallMatrixUnits) ? kQmpBracketSmall : kQmpBracket);
     lo = 0.5f * fmaxf(gamma_est * (1.0f - b), kEps) * (1.0f - 1e-6f);
     hi = 0.5f * fmaxf(gamma_est * (1.0f + b), kEps) * (1.0f + 1e-6f);
 }
@@ -173,27 +175,44 @@ __device__ __forceinline__ bool qmp_hint(const QmpDesc& d, float& g) {
     return g > 0.0f && g < 3.0e38f;
 }
 
-// gamma_est by ONE warp: the same scattered units as qmp_sample_gamma, eight unit loads in flight per
-// lane after the whole sample has been requested into L2.
-template <bool BF16>
-__device__ __forceinline__ float qmp_sample_gamma_warp(const QmpDesc& d, int lane) {
-    constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
-    const uint32_t n_s = qmp_sample_units(d.num_units);
-    const uint32_t stride = d.num_units / n_s;
+// gamma_est by ONE warp (the finisher, for matrices 2, 3, ... of a batch without hints): the first
+// kQmpSampleUnitsSmall of qmp_sample_gamma's scattered units, fetched by bulk copies into `buf` (a list that
+// is free at that moment) -- all of them in flight at once, one round trip instead of one per eight units.
+// The smaller sample gets the wider bracket (qmp_bracket_from, `wide`).  Returns a negative number if the
+// copies did not land within the wait limit (the CTA is then aborting).
+constexpr int kQmpSampleUnitsWarp = kQmpSampleUnitsSmall;
+static_assert(kQmpSampleUnitsWarp * 512 <= kQmpStreamListCap * 8, "the sample fits a list");
+__device__ __forceinline__ float qmp_sample_gamma_warp(const QmpDesc& d, int lane, unsigned char* buf, uint32_t bar, uint32_t& bar_phase,
+                                                       volatile int* abort_flag) {
+    const uint32_t unit_bytes = d.w_bf16 ? 256u : 512u;
+    const uint32_t n_full = qmp_sample_units(d.num_units);
+    const uint32_t stride = d.num_units / n_full;
+    const uint32_t n_s = min(n_full, static_cast<uint32_t>(kQmpSampleUnitsWarp));
     auto unit_of = [&](uint32_t sidx) { return sidx * stride + ((sidx * 2654435761u) >> 8) % stride; };
+    const uint32_t buf_u32 = qmp_smem_u32(buf);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // the list's earlier (generic) use before the copies
+    if (lane == 0) qmp_mbar_expect_tx(bar, n_s * unit_bytes);
+    __syncwarp();
     for (uint32_t sidx = lane; sidx < n_s; sidx += 32u)
-        prefetch_l2_bulk(static_cast<const char*>(d.W) + static_cast<size_t>(unit_of(sidx)) * kUnitBytes, kUnitBytes);
+        qmp_bulk_load(buf_u32 + sidx * unit_bytes, static_cast<const char*>(d.W) + static_cast<size_t>(unit_of(sidx)) * unit_bytes, unit_bytes, bar);
+    const bool landed = qmp_mbar_wait(bar, bar_phase, abort_flag, true);  // sees its own copies land even if the CTA aborts
+    bar_phase ^= 1u;
+    if (!landed) return -1.0f;
     float acc = 0.0f;
-    for (uint32_t base = 0; base < n_s; base += 8u) {
-        float4 v[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            v[i] = base + i < n_s ? qmp_load_group<BF16>(d.W, unit_of(base + i), lane) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc += (fabsf(v[i].x) + fabsf(v[i].y)) + (fabsf(v[i].z) + fabsf(v[i].w));
+    const uint32_t chunks = n_s * unit_bytes / 16u;
+    for (uint32_t c = lane; c < chunks; c += 32u) {
+        const float4 v = qmp_lds128(buf_u32 + c * 16u);
+        if (d.w_bf16) {
+            const uint32_t r0 = __float_as_uint(v.x), r1 = __float_as_uint(v.y), r2 = __float_as_uint(v.z), r3 = __float_as_uint(v.w);
+            acc += ((fabsf(bf16lo_to_f32(r0)) + fabsf(bf16hi_to_f32(r0))) + (fabsf(bf16lo_to_f32(r1)) + fabsf(bf16hi_to_f32(r1)))) +
+                   ((fabsf(bf16lo_to_f32(r2)) + fabsf(bf16hi_to_f32(r2))) + (fabsf(bf16lo_to_f32(r3)) + fabsf(bf16hi_to_f32(r3))));
+        } else {
+            acc += (fabsf(v.x) + fabsf(v.y)) + (fabsf(v.z) + fabsf(v.w));
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    __syncwarp();
     return acc / (static_cast<float>(n_s) * 128.0f);
 }
 
@@ -337,6 +356,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
             qmp_mbar_init(bar_full0 + 8u * i, 1u);                     // the loader's expect_tx
             qmp_mbar_init(bar_empty0 + 8u * i, kQmpStreamWarps);       // one arrival per computing warp
         }
+        qmp_mbar_init(qmp_smem_u32(&sh.bar_sample), 1u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -412,20 +432,24 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
     } else {
         // ------------------------------------------------------------------ the finisher (warp 31)
         bool ok = true;
+        uint32_t sample_phase = 0u;
         for (int m = 0; ok && m < count; ++m) {
             const int slot = m % kQmpLists;
-            // bracket of matrix m + 2, well before the computing warps ask for it
+            // bracket of matrix m + 2 from the caller's hint, well before the computing warps ask for it
+            bool sample_next = false;
             if (m + 2 < count) {
                 const QmpDesc d2 = qmp_desc_of(batch, m + 2);
                 float g;
-                const bool hinted = qmp_hint(d2, g);
-                if (!hinted) g = d2.w_bf16 ? qmp_sample_gamma_warp<true>(d2, lane) : qmp_sample_gamma_warp<false>(d2, lane);
-                if (lane == 0) {
-                    qmp_bracket_from(g, d2.num_units, hinted, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1]);
-                    __threadfence_block();
-                    *reinterpret_cast<volatile int*>(&sh.bracket_upto) = m + 3;
+                if (qmp_hint(d2, g)) {
+                    if (lane == 0) {
+                        qmp_bracket_from(g, d2.num_units, true, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1]);
+                        __threadfence_block();
+                        *reinterpret_cast<volatile int*>(&sh.bracket_upto) = m + 3;
+                    }
+                    __syncwarp();
+                } else {
+                    sample_next = true;
                 }
-                __syncwarp();
             }
             // matrix m: every streaming warp has arrived -> this CTA's partial sum, published
             if (!qmp_wait_ge(reinterpret_cast<volatile int*>(&sh.arrived[slot]), kQmpStreamWarps, abort_flag)) { ok = false; break; }
@@ -521,6 +545,20 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
                     sh.list_count[pslot] = 0u;
                     __threadfence_block();
                     *reinterpret_cast<volatile int*>(&sh.fixed_upto) = m;
+                }
+                __syncwarp();
+            }
+            // bracket of matrix m + 2 from a sample, if it has no hint: a whole matrix before the computing warps
+            // ask for it.  The sample lands in the list that matrix m - 1 has just given back (the one m + 2 will use).
+            if (sample_next) {
+                const QmpDesc d2 = qmp_desc_of(batch, m + 2);
+                const float g = qmp_sample_gamma_warp(d2, lane, reinterpret_cast<unsigned char*>(s_list + ((m + 2) % kQmpLists) * kQmpStreamListCap),
+                                                      qmp_smem_u32(&sh.bar_sample), sample_phase, abort_flag);
+                if (g < 0.0f) { ok = false; break; }
+                if (lane == 0) {
+                    qmp_bracket_from(g, d2.num_units, false, sh.bracket[(m + 2) & 3][0], sh.bracket[(m + 2) & 3][1], true);
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int*>(&sh.bracket_upto) = m + 3;
                 }
                 __syncwarp();
             }
