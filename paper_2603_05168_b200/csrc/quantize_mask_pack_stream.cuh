@@ -64,7 +64,7 @@ struct QmpStreamShared {
     float thr_second_pass[kQmpMaxBatch];                   // >= 0: this matrix needs the exact second pass with this threshold
     unsigned long long bar_full[kQmpStages];               // a stage's bytes have landed
     unsigned long long bar_empty[kQmpStages];              // the computing warps are done with a stage
-    uint32_t ring_issued, ring_stage, ring_phase;          // the loader's last position
+    uint32_t ring_issued, ring_used;                       // the loader's copies of this launch, and its ring position
     unsigned long long bar_sample;                         // the finisher's sample has landed
 };
 
@@ -118,10 +118,13 @@ __device__ __forceinline__ float4 qmp_lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
-// Position of the ring: stage and the parity of its current use.
+// Position in the ring: the number of stages used so far gives the stage and the parity of its current use.
+static_assert((kQmpStages & (kQmpStages - 1)) == 0, "stage = count mod kQmpStages by masking");
 struct QmpRing {
-    uint32_t stage, phase;
-    __device__ __forceinline__ void advance() { if (++stage == kQmpStages) { stage = 0; phase ^= 1u; } }
+    uint32_t used;
+    __device__ __forceinline__ uint32_t stage() const { return used & (kQmpStages - 1); }
+    __device__ __forceinline__ uint32_t phase() const { return (used / kQmpStages) & 1u; }
+    __device__ __forceinline__ void advance() { ++used; }
 };
 
 // Matrix m of the batch: 0 and 1 travel with the launch, `rest` holds 1, 2, ... in global memory.
@@ -242,10 +245,10 @@ __device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpBatch& b
         }
         if (max_copies == 0u) return true;
         --max_copies;
-        if (!qmp_mbar_wait(bar_empty0 + 8u * L.ring.stage, L.ring.phase ^ 1u, abort_flag)) return false;
+        if (!qmp_mbar_wait(bar_empty0 + 8u * L.ring.stage(), L.ring.phase() ^ 1u, abort_flag)) return false;
         const uint32_t bytes = min(L.u_end - L.u, static_cast<uint32_t>(kQmpStageUnits)) * L.unit_bytes;
-        qmp_mbar_expect_tx(bar_full0 + 8u * L.ring.stage, bytes);
-        qmp_bulk_load(ring_base + L.ring.stage * kQmpStageBytes, L.W + static_cast<size_t>(L.u) * L.unit_bytes, bytes, bar_full0 + 8u * L.ring.stage);
+        qmp_mbar_expect_tx(bar_full0 + 8u * L.ring.stage(), bytes);
+        qmp_bulk_load(ring_base + L.ring.stage() * kQmpStageBytes, L.W + static_cast<size_t>(L.u) * L.unit_bytes, bytes, bar_full0 + 8u * L.ring.stage());
         ++L.issued;
         L.ring.advance();
         L.u += kQmpStageUnits;
@@ -253,9 +256,34 @@ __device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpBatch& b
     }
 }
 
-// Pass 1 of one matrix for a computing warp: its two units of every stage of the CTA's range.  Returns
-// the thread's sum |W| (false in `ok` if a wait ran out); metadata, provisional values, undecided list
-// and flip count as in quantize_mask_pack.cuh.  A lane takes two adjacent groups (32 B of a row).
+// One lane's two groups (32 B of a row) of pass 1: sum |W|, metadata, provisional values, undecided list,
+// flip count, as in quantize_mask_pack.cuh.  `meta_row` / `vals_row` point at this lane's byte / word of the
+// unit's row inside the metadata and value tiles; `v_off` is the word's byte offset in vals (for the list).
+struct QmpPass1Consts {
+    float thr_lo, thr_hi, mid, half;
+    QmpEntry* list;
+    unsigned int* list_count;
+};
+__device__ __forceinline__ void qmp_pass1_groups(const float4 va, const float4 vb, const QmpPass1Consts& c, uint8_t* meta_row,
+                                                 const uint8_t* prev_row, uint32_t* vals_row, uint32_t v_off, double& acc, unsigned int& flips) {
+    acc += abs_sum4(va) + abs_sum4(vb);
+    float k[4];
+    const uint32_t nib0 = select_pair(va, k[0], k[1]);
+    const uint32_t nib1 = select_pair(vb, k[2], k[3]);
+    if (prev_row != nullptr) {
+        const uint32_t prev = *prev_row;
+        flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
+                        (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
+    }
+    *meta_row = static_cast<uint8_t>(nib0 | (nib1 << 4));
+    *vals_row = ternary_bytes4(k[0], k[1], k[2], k[3], c.thr_hi);
+    const float far = fminf(fminf(fabsf(fabsf(k[0]) - c.mid), fabsf(fabsf(k[1]) - c.mid)),
+                            fminf(fabsf(fabsf(k[2]) - c.mid), fabsf(fabsf(k[3]) - c.mid)));
+    if (far <= c.half) qmp_list_undecided<kQmpStreamListCap>(k, c.thr_lo, c.thr_hi, v_off, c.list, c.list_count);
+}
+
+// Pass 1 of one matrix for a computing warp: its two units of every stage of the CTA's range (a half-warp
+// per unit, a lane two adjacent groups).  Returns the thread's sum |W|; `ok` turns false if a wait ran out.
 template <bool BF16>
 __device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRange rg, const float thr_lo, const float thr_hi,
                                                    QmpEntry* list, unsigned int* list_count, unsigned int& flips,
@@ -266,24 +294,33 @@ __device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRa
     const uint32_t l16 = lane & 15;
     const uint32_t KB = d.KB;
     constexpr uint32_t kUnitBytes = BF16 ? 256u : 512u;
-    const int step_n = static_cast<int>(kQmpStageUnits / KB), step_kb = static_cast<int>(kQmpStageUnits % KB);
-    const bool count_flips = d.prev_meta != nullptr;
+    const uint32_t step_n = kQmpStageUnits / KB, step_kb = kQmpStageUnits % KB;
     // |k| in [thr_lo, thr_hi) implies | |k| - mid | <= half (the subtraction is exact, thr_hi < 2 thr_lo;
     // `half` is rounded up by far more than the rounding of `mid`): a cheap test with no false negatives
-    const float mid = 0.5f * (thr_lo + thr_hi);
-    const float half = fmaf(thr_hi - thr_lo, 0.50005f, thr_hi * 2.4e-7f);
+    const QmpPass1Consts c{thr_lo, thr_hi, 0.5f * (thr_lo + thr_hi), fmaf(thr_hi - thr_lo, 0.50005f, thr_hi * 2.4e-7f), list, list_count};
     double acc = 0.0;
     const uint32_t in_stage = 2u * warp + (lane >> 4);               // this half-warp's unit of every stage
-    uint32_t u = rg.u_begin + in_stage;
-    int n_cur = static_cast<int>(u / KB);
-    int kb_cur = static_cast<int>(u - static_cast<uint32_t>(n_cur) * KB);
-    const uint32_t src_off = in_stage * kUnitBytes + l16 * (kUnitBytes / 16u);
-    for (uint32_t u0 = rg.u_begin; u0 < rg.u_end; u0 += kQmpStageUnits, u += kQmpStageUnits) {
-        if (!qmp_mbar_wait(bar_full0 + 8u * ring.stage, ring.phase, abort_flag)) { ok = false; break; }
-        float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
-        const bool mine = u < rg.u_end;
-        if (mine) {
-            const uint32_t src = ring_base + ring.stage * kQmpStageBytes + src_off;
+    const uint32_t u_first = rg.u_begin + in_stage;
+    uint32_t n_cur = u_first / KB;
+    uint32_t kb_cur = u_first - n_cur * KB;
+    const uint32_t src_off = ring_base + in_stage * kUnitBytes + l16 * (kUnitBytes / 16u);
+    // this lane's place in a row of a metadata tile (byte l16 of 16) and of a value tile (word l16 & 3 of the
+    // 16-byte chunk (l16 >> 2) ^ ((row >> 1) & 3), see layouts.cuh)
+    uint8_t* const meta_lane = d.meta + l16;
+    const uint8_t* const prev_lane = d.prev_meta != nullptr ? d.prev_meta + l16 : nullptr;
+    unsigned char* const vals_lane = reinterpret_cast<unsigned char*>(d.vals) + 4u * (l16 & 3u);
+    const uint32_t chunk = l16 >> 2;
+    const uint32_t range = rg.u_end - rg.u_begin;
+    const uint32_t n_stages = (range + kQmpStageUnits - 1) / kQmpStageUnits;
+    const uint32_t last_units = range - (n_stages - 1u) * kQmpStageUnits;          // units of the last stage (range > 0)
+    for (uint32_t st = 0; st < n_stages; ++st) {
+        const uint32_t stage = ring.stage();
+        if (!qmp_mbar_wait(bar_full0 + 8u * stage, ring.phase(), abort_flag)) { ok = false; break; }
+        const bool mine = st + 1u < n_stages || in_stage < last_units;
+        float4 va, vb;
+        {
+            // a lane without a unit (last stage only) reads what is there: finite or not, it is not used
+            const uint32_t src = src_off + stage * kQmpStageBytes;
             if constexpr (BF16) {
                 const float4 raw = qmp_lds128(src);
                 const uint32_t r0 = __float_as_uint(raw.x), r1 = __float_as_uint(raw.y), r2 = __float_as_uint(raw.z), r3 = __float_as_uint(raw.w);
@@ -295,30 +332,18 @@ __device__ __forceinline__ double qmp_stream_pass1(const QmpDesc& d, const QmpRa
             }
         }
         __syncwarp();
-        if (lane == 0) qmp_mbar_arrive(bar_empty0 + 8u * ring.stage);      // the values are in registers: the stage may be refilled
+        if (lane == 0) qmp_mbar_arrive(bar_empty0 + 8u * stage);           // the values are in registers: the stage may be refilled
         ring.advance();
-        const uint32_t tile_idx = (static_cast<uint32_t>(n_cur) >> 7) * KB + static_cast<uint32_t>(kb_cur);
-        const uint32_t rr = static_cast<uint32_t>(n_cur) & 127u;
+        const uint32_t tile_idx = (n_cur >> 7) * KB + kb_cur;
+        const uint32_t rr = n_cur & 127u;
         n_cur += step_n;
         kb_cur += step_kb;
-        if (kb_cur >= static_cast<int>(KB)) { kb_cur -= static_cast<int>(KB); ++n_cur; }
+        if (kb_cur >= KB) { kb_cur -= KB; ++n_cur; }
         if (mine) {
-            acc += abs_sum4(va) + abs_sum4(vb);
-            float k[4];
-            const uint32_t nib0 = select_pair(va, k[0], k[1]);
-            const uint32_t nib1 = select_pair(vb, k[2], k[3]);
-            const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + ((rr << 4) + l16);
-            if (count_flips) {
-                const uint32_t prev = d.prev_meta[m_off];
-                flips += __popc((nibble_to_mask(nib0) | (nibble_to_mask(nib1) << 4)) ^
-                                (nibble_to_mask(prev & 15u) | (nibble_to_mask(prev >> 4) << 4)));
-            }
-            d.meta[m_off] = static_cast<uint8_t>(nib0 | (nib1 << 4));
-            const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + vals_in_tile(rr, 4u * l16);
-            reinterpret_cast<uint32_t*>(d.vals)[v_off >> 2] = ternary_bytes4(k[0], k[1], k[2], k[3], thr_hi);
-            const float far = fminf(fminf(fabsf(fabsf(k[0]) - mid), fabsf(fabsf(k[1]) - mid)),
-                                    fminf(fabsf(fabsf(k[2]) - mid), fabsf(fabsf(k[3]) - mid)));
-            if (far <= half) qmp_list_undecided<kQmpStreamListCap>(k, thr_lo, thr_hi, static_cast<uint32_t>(v_off), list, list_count);
+            const size_t m_off = static_cast<size_t>(tile_idx) * 2048u + (rr << 4);
+            const size_t v_off = static_cast<size_t>(tile_idx) * 8192u + ((rr << 6) + ((chunk ^ ((rr >> 1) & 3u)) << 4));
+            qmp_pass1_groups(va, vb, c, meta_lane + m_off, prev_lane != nullptr ? prev_lane + m_off : nullptr,
+                             reinterpret_cast<uint32_t*>(vals_lane + v_off), static_cast<uint32_t>(v_off) + 4u * (l16 & 3u), acc, flips);
         }
     }
     return acc;
@@ -350,7 +375,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
         sh.bracket_upto = 0;
         sh.fixed_upto = 0;
         sh.abort = 0;
-        sh.ring_issued = 0u; sh.ring_stage = 0u; sh.ring_phase = 0u;
+        sh.ring_issued = 0u; sh.ring_used = 0u;
         for (int i = 0; i < kQmpLists; ++i) { sh.arrived[i] = 0u; sh.list_count[i] = 0u; sh.flip_total[i] = 0ull; }
         for (int i = 0; i < kQmpStages; ++i) {
             qmp_mbar_init(bar_full0 + 8u * i, 1u);                     // the loader's expect_tx
@@ -375,7 +400,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
     bool hinted01[2];
     hinted01[0] = qmp_hint(first, g01[0]);
     hinted01[1] = count > 1 && qmp_hint(second, g01[1]);
-    QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u, 0u}, 0u};
+    QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u}, 0u};
     const bool is_loader = warp == kQmpLoaderWarp && lane == 0;
     if (is_loader) qmp_loader_issue(loader, batch, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
 
@@ -390,7 +415,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
 
     if (warp < kQmpStreamWarps) {
         // ------------------------------------------------------------------ computing warps
-        QmpRing ring{0u, 0u};
+        QmpRing ring{0u};
         for (int m = 0; m < count; ++m) {
             const int slot = m % kQmpLists;
             if (!qmp_wait_ge(&sh.bracket_upto, m + 1, abort_flag)) break;
@@ -425,8 +450,7 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
         if (is_loader) {
             qmp_loader_issue(loader, batch, count, 0xFFFFFFFFu, ring_base, bar_full0, bar_empty0, abort_flag);
             sh.ring_issued = loader.issued;                  // for the drain, should the CTA abort
-            sh.ring_stage = loader.ring.stage;
-            sh.ring_phase = loader.ring.phase;
+            sh.ring_used = loader.ring.used;
         }
         __syncwarp();
     } else {
@@ -569,11 +593,11 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
         // No bulk copy may still be writing this CTA's shared memory when it leaves: the last
         // min(issued, kQmpStages) copies are the ones that can be in flight; the ring position points past the newest.
         if (threadIdx.x == 0) {
-            QmpRing ring{sh.ring_stage, sh.ring_phase};
+            QmpRing ring{sh.ring_used};
             const uint32_t back = min(sh.ring_issued, static_cast<uint32_t>(kQmpStages));
             for (uint32_t j = 0; j < back; ++j) {
-                if (ring.stage == 0u) { ring.stage = kQmpStages - 1; ring.phase ^= 1u; } else { --ring.stage; }
-                qmp_mbar_wait(bar_full0 + 8u * ring.stage, ring.phase, abort_flag, true);
+                --ring.used;
+                qmp_mbar_wait(bar_full0 + 8u * ring.stage(), ring.phase(), abort_flag, true);
             }
         }
         return;
