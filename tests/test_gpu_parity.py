@@ -1031,10 +1031,11 @@ def test_pack_wait_runs_out_and_the_library_recovers():
 
 
 # ---- the streaming pack kernel: hints and very long batches ------------------------------------------------
-@pytest.mark.parametrize("hint_factor", [1.0, 1.02, 2.0, 0.0, -1.0, float("inf")])
+@pytest.mark.parametrize("hint_factor", [1.0, 1.003, 0.996, 1.02, 2.0, 0.0, -1.0, float("inf")])
 def test_quantize_mask_pack_gamma_hint_never_changes_the_result(hint_factor):
     # the hint only decides whether the kernel samples the matrix and whether the bracket holds
-    # (a hint far off sends the matrix through the exact second pass): the bytes must not change
+    # (within 0.5 % of gamma: the listed values are fixed up; further off: the exact second pass):
+    # the bytes must not change
     shapes = [(256, 2560), (640, 256), (128, 128), (384, 1280), (2560, 640), (128, 6912)]
     Ws = [inputs.latent_weights(N, K, seed=160 + i, sigma=0.02 * (i + 1)) for i, (N, K) in enumerate(shapes)]
     refs = [_oracle_pack(W) for W in Ws]
