@@ -505,6 +505,58 @@ def test_quantize_mask_pack_batched_matches_single_calls():
             assert int(job["flip_bits"].item()) == want == one["flips"]
 
 
+def test_quantize_mask_pack_random_batches_against_the_oracle_and_single_calls():
+    # seeded random batches: 1..7 matrices of mixed shapes (fewer units than CTAs, ragged last stages, ranges
+    # of several stages), fp32 and bf16 masters, Gaussian and heavy-tailed, no hints / exact hints / hints
+    # inside and outside the bracket / hints on some jobs only, each batch launched twice on one workspace.
+    # Every job must carry the oracle's bits (matrices the oracle flags as near-ties excepted) and the
+    # single call's bits.
+    import random
+    rng = random.Random(20260305)
+    Ns, Ks = [128, 256, 384, 640, 2560], [128, 256, 1280, 2560, 6912]
+    checked = 0
+    for it in range(24):
+        count = rng.randint(1, 7)
+        jobs, refs, singles, shapes = [], [], [], []
+        mode = rng.choice(["none", "good", "off", "mixed"])
+        for i in range(count):
+            N, K = rng.choice(Ns), rng.choice(Ks)
+            W = inputs.latent_weights(N, K, seed=7000 + 16 * it + i, sigma=rng.choice([0.02, 0.5, 1e-3]))
+            if rng.random() < 0.2:
+                W = inputs.latent_weights(N, K, seed=7500 + 16 * it + i, sigma=0.015, outlier_prob=0.05, outlier_mult=10.0)
+            as_bf16 = rng.random() < 0.3
+            if as_bf16:
+                bits = inputs.f32_to_bf16_bits(W)
+                W = (bits.astype(np.uint32) << 16).view(np.float32).reshape(N, K)
+                Wd = bf16_dev(bits)
+            else:
+                Wd = dev(W)
+            r = oracle.quantize_mask_pack(W)
+            one = b.alloc_packed(N, K)
+            b.sbn_quantize_mask_pack(Wd, one["vals"], one["meta"], one["w_scale"], one["ws"])
+            bufs = b.alloc_packed(N, K)
+            job = dict(W=Wd, vals=bufs["vals"], meta=bufs["meta"], w_scale=bufs["w_scale"])
+            if mode in ("good", "off") or (mode == "mixed" and rng.random() < 0.5):
+                f = 1.0 if mode != "off" else rng.choice([1.004, 0.99, 1.5, 0.0])
+                job["gamma_hint"] = torch.tensor([float(r["scale"]) * f], dtype=torch.float32, device="cuda")
+            jobs.append(job); refs.append(r); singles.append(one); shapes.append((N, K))
+        arr = b.make_pack_jobs(jobs)
+        ws = torch.empty(b.sbn_batch_workspace_bytes(count), dtype=torch.uint8, device="cuda")
+        for _ in range(2):
+            b.sbn_quantize_mask_pack_batched(arr, ws)
+        b.sbn_check_status()
+        for job, r, one, (N, K) in zip(jobs, refs, singles, shapes):
+            for key in ("vals", "meta", "w_scale"):
+                assert torch.equal(job[key], one[key]), (it, N, K, mode, key)
+            if r["near_tie"]:
+                continue
+            vals, meta = gpu_unpack_canonical(job, N, K)
+            assert np.float32(job["w_scale"].cpu().numpy()[0]) == r["scale"]
+            assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"])
+            checked += 1
+    assert checked > 60
+
+
 def test_quantize_mask_pack_full_size_in_the_bench_configuration():
     # the four BitNet-2B-shaped matrices exactly as bench.py packs them: one batched launch, no
     # dense output (the single-pass route); every byte against the oracle
