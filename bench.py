@@ -243,7 +243,8 @@ def backward_rows(torch, b, peaks, layers, time_cold, iters):
     """The layer's backward under the dual straight-through estimator (Sec. 2.3, Eq. 5): dX = dY w_masked and
     the dense dW = dY^T x_q on the tensor cores in bf16 (fp32 accumulation), per 2B-shaped layer at
     T = 4096, cold L2.  Each time covers the whole call for that gradient: the operand preparation (W_eff^T,
-    or x_q^T and dY^T, in bf16) and the GEMM.  `library_matmul_*`: torch.matmul on ready-made bf16 operands of
+    or x_q, in bf16) and the GEMM; `both_us` is one call for both gradients (the two GEMMs share the machine
+    where the first one's last wave leaves pairs idle).  `library_matmul_*`: torch.matmul on ready-made bf16 operands of
     the same shapes, as the pace of a library GEMM on this machine (context, not part of the path)."""
     rows = {}
     for L in layers:
@@ -257,15 +258,17 @@ def backward_rows(torch, b, peaks, layers, time_cold, iters):
         ws = torch.empty(b.sbn_workspace_bytes(b.OP_BACKWARD, T, N, K), dtype=torch.uint8, device="cuda")
         f_dx = lambda: b.sbn_bitlinear_backward(dY, L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], N, K, dX=dX, ws=ws)
         f_dw = lambda: b.sbn_bitlinear_backward(dY, L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], N, K, dW=dW, ws=ws)
+        f_both = lambda: b.sbn_bitlinear_backward(dY, L.xq, L.a_scale, p["vals"], p["meta"], p["w_scale"], N, K, dX=dX, dW=dW, ws=ws)
         w_b = torch.empty((N, K), dtype=torch.bfloat16, device="cuda").normal_()
         g_dx = lambda: torch.matmul(dY, w_b)
         g_dw = lambda: torch.matmul(dY.t(), L.x)
-        for fn in (f_dx, f_dw, g_dx, g_dw):
+        for fn in (f_dx, f_dw, f_both, g_dx, g_dw):
             for _ in range(2):
                 fn()
-        t = {k: time_cold(fn, iters) for k, fn in (("dx", f_dx), ("dw", f_dw), ("lib_dx", g_dx), ("lib_dw", g_dw))}
+        t = {k: time_cold(fn, iters) for k, fn in (("dx", f_dx), ("dw", f_dw), ("both", f_both), ("lib_dx", g_dx), ("lib_dw", g_dw))}
         flops = 2.0 * T * N * K
         rows[L.name] = {"dx_us": round(t["dx"], 2), "dw_us": round(t["dw"], 2),
+                        "both_us": round(t["both"], 2), "both_tflops": round(2.0 * flops / t["both"] / 1e6, 1),
                         "dx_tflops": round(flops / t["dx"] / 1e6, 1), "dw_tflops": round(flops / t["dw"] / 1e6, 1),
                         "dx_frac_of_measured_bf16_burst": round(flops / t["dx"] / 1e6 / peaks["bf16_tflops"], 4),
                         "dw_frac_of_measured_bf16_burst": round(flops / t["dw"] / 1e6 / peaks["bf16_tflops"], 4),

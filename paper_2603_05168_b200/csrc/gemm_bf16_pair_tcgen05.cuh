@@ -38,6 +38,16 @@ struct Bf16GemmParams {
     void* out;                   // [M][Nn] row-major, fp32 or bf16
     int out_bf16;
     const float* scale;          // device, one fp32, or null: the result is multiplied by bf16(scale)
+    // Two launches of this kernel that do not depend on each other (dW and dX of one backward call) share
+    // the machine at the seam: the first one's last wave leaves pairs idle, the second one's CTAs move in as
+    // soon as pairs are free instead of waiting for the whole grid.
+    //   first launch:  signal_after_wait -- it lets its dependents go only after its own dependency wait, so
+    //                  that whatever it waited for is complete for them too;
+    //   second launch: wait_at_end -- no dependency wait before its work (its inputs are complete by the rule
+    //                  above), but one before it exits: it is not complete before the first launch is, and the
+    //                  kernels after it in the stream see both results.
+    int signal_after_wait = 0;
+    int wait_at_end = 0;
 };
 
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster_addr) {
@@ -74,7 +84,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int BN = p.bn;
     const int half_bn = BN >> 1;
 
-    pdl_launch_dependents();
+    if (!p.signal_after_wait) pdl_launch_dependents();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = smem_u32(smem_raw);
     if (smem_base & 1023u) {          // swizzled tiles need 1 KB alignment; identical in every CTA
@@ -119,7 +129,8 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     __syncthreads();
     cluster_sync_all();
     tcgen05_fence_after();
-    pdl_wait();                          // nothing above touches global memory
+    if (!p.wait_at_end) pdl_wait();      // nothing above touches global memory
+    if (p.signal_after_wait) pdl_launch_dependents();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
@@ -262,6 +273,7 @@ gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         tcgen05_fence_after();
         tmem_dealloc_pair(tmem_base, kTmemCols);
     }
+    if (p.wait_at_end) pdl_wait();
 }
 
 }  // namespace sbn

@@ -488,8 +488,11 @@ static int pick_bf16_bn(int M, int Nn) {
 // D[M][Nn] = A[M][Kc] B[Nn][Kc]^T (bf16 in, fp32 accumulation), optionally times bf16(*scale).
 // mn_major: A is stored [Kc][M] (row stride lda) and B [Kc][Nn] (row stride ldb): D = A^T B.
 static sbn_status run_gemm_bf16(bool mn_major, const void* A, int M, uint64_t lda, const void* B, int Nn, uint64_t ldb, int Kc,
-                                void* out, bool out_bf16, const float* scale, cudaStream_t stream) {
+                                void* out, bool out_bf16, const float* scale, cudaStream_t stream,
+                                bool signal_after_wait = false, bool wait_at_end = false) {
     Bf16GemmParams p;
+    p.signal_after_wait = signal_after_wait ? 1 : 0;
+    p.wait_at_end = wait_at_end ? 1 : 0;
     p.M = M; p.Nn = Nn; p.Kc = Kc;
     p.bn = g_force_token_tile < 0 ? std::min(256, std::max(64, (-g_force_token_tile) / 16 * 16)) : pick_bf16_bn(M, Nn);
     if (mn_major) p.bn = p.bn > 128 ? 256 : 128;                // whole 64-column blocks per CTA
@@ -952,24 +955,32 @@ sbn_status sbn_bitlinear_backward(const void* dY_bf16, int T, const int8_t* xq, 
     uint16_t* Wt = reinterpret_cast<uint16_t*>(base + lay.wt_off);
     uint16_t* XT = reinterpret_cast<uint16_t*>(base + lay.xq_off);
     const int KB = K / kBK, NB = N / kBM;
+    // Operands first (two small memory-bound kernels), then the GEMMs.  With both gradients wanted the
+    // weight-gradient GEMM goes first and the input-gradient GEMM moves into the pairs its last wave
+    // leaves idle (Bf16GemmParams: signal_after_wait / wait_at_end): the two do not depend on each other.
+    const bool both = dX_bf16 != nullptr && dW != nullptr;
     if (dX_bf16) {
-        // dX[t][k] = bf16(scale) * sum_n dY[t][n] W_eff[n][k]: A = dY [T][N], B = W_eff^T [K][N]
         if (launch_kernel(weff_t_bf16_kernel, dim3(KB * NB), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(vals), meta, N, K, Wt) != cudaSuccess)
             return SBN_ERR_CUDA;
         ++g_launch_count;
-        const sbn_status st = run_gemm_bf16(false, dY_bf16, T, static_cast<uint64_t>(N), Wt, K, static_cast<uint64_t>(N), N, dX_bf16, true, w_scale, s);
-        if (st != SBN_OK) return st;
     }
     if (dW) {
-        // dW[n][k] = sum_t dY[t][n] x_q[t][k]
-        // both operands as they lie in memory, token-major: dY [T][N] and x_q [T][K] (bf16 copy of the
-        // fake-quantised activations); the MMA reads them MN-major, the contraction runs down the rows
         const unsigned blocks = static_cast<unsigned>(std::min<size_t>((static_cast<size_t>(T) * (K / 16) + kPrepThreads - 1) / kPrepThreads,
                                                                            static_cast<size_t>(device_sm_count()) * 8));
         if (launch_kernel(xq_bf16_kernel, dim3(blocks), dim3(kPrepThreads), 0, s, reinterpret_cast<const uint8_t*>(xq), a_scale, T, K, XT) != cudaSuccess)
             return SBN_ERR_CUDA;
         ++g_launch_count;
-        const sbn_status st = run_gemm_bf16(true, dY_bf16, N, static_cast<uint64_t>(N), XT, K, static_cast<uint64_t>(K), T, dW, false, nullptr, s);
+        // dW[n][k] = sum_t dY[t][n] x_q[t][k]
+        // both operands as they lie in memory, token-major: dY [T][N] and x_q [T][K] (bf16 copy of the
+        // fake-quantised activations); the MMA reads them MN-major, the contraction runs down the rows
+        const sbn_status st = run_gemm_bf16(true, dY_bf16, N, static_cast<uint64_t>(N), XT, K, static_cast<uint64_t>(K), T, dW, false, nullptr, s,
+                                            both, false);
+        if (st != SBN_OK) return st;
+    }
+    if (dX_bf16) {
+        // dX[t][k] = bf16(scale) * sum_n dY[t][n] W_eff[n][k]: A = dY [T][N], B = W_eff^T [K][N]
+        const sbn_status st = run_gemm_bf16(false, dY_bf16, T, static_cast<uint64_t>(N), Wt, K, static_cast<uint64_t>(N), N, dX_bf16, true, w_scale, s,
+                                            false, both);
         if (st != SBN_OK) return st;
     }
     return SBN_OK;
