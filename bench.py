@@ -564,6 +564,14 @@ def run_ours(args):
         act = time_cold(lambda: b.sbn_quant_act(L.x, L.xq, L.a_scale), iters)
         row["quantize_mask_pack_us"] = round(qmp, 2)
         row["quantize_mask_pack_gbs"] = round(L.N * L.K * (L.w_bytes + 0.625) / qmp / 1e3, 1)     # algorithmic bytes: W once + vals + meta
+        # the same matrix as a batch of one whose job carries the previous scale as its estimate of gamma (what a
+        # training loop does: no sample, a narrow bracket)
+        hint_jobs = b.make_pack_jobs([dict(W=L.W, vals=p["vals"], meta=p["meta"], w_scale=p["w_scale"], gamma_hint=p["w_scale"])])
+        hint_ws = torch.empty(b.sbn_batch_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+        b.sbn_quantize_mask_pack_batched(hint_jobs, hint_ws)
+        qmp_h = time_cold(lambda: b.sbn_quantize_mask_pack_batched(hint_jobs, hint_ws), iters)
+        row["quantize_mask_pack_hint_us"] = round(qmp_h, 2)
+        row["quantize_mask_pack_hint_gbs"] = round(L.N * L.K * (L.w_bytes + 0.625) / qmp_h / 1e3, 1)
         row["quant_act_us"] = round(act, 2)
         row["quant_act_gbs"] = round((L.T * L.K * 3 + L.T * 4) / act / 1e3, 1)
         # the same kernel launched back to back over 8 distinct inputs (more than the L2 holds): what a
