@@ -172,13 +172,38 @@ __device__ __forceinline__ void qmp_bracket_from(float gamma_est, uint32_t num_u
 }
 
 // The caller's estimate of gamma, if it gave a usable one.
+__device__ __forceinline__ bool qmp_hint_usable(float g) { return g > 0.0f && g < 3.0e38f; }
 __device__ __forceinline__ bool qmp_hint(const QmpDesc& d, float& g) {
     if (d.gamma_hint == nullptr) return false;
     g = *reinterpret_cast<const volatile float*>(d.gamma_hint);
-    return g > 0.0f && g < 3.0e38f;
+    return qmp_hint_usable(g);
 }
 
-// gamma_est by ONE warp (the finisher, for matrices 2, 3, ... of a batch without hints): the first
+// qmp_sample_gamma in two halves, so that something can be started between asking for the sample and using
+// it: all of a thread's sample loads are issued (into v), later they are added up over the CTA.
+constexpr int kQmpSamplePerWarp = kQmpSampleUnits / kQmpWarps;
+__device__ __forceinline__ void qmp_sample_issue(const QmpDesc& d, float4 (&v)[kQmpSamplePerWarp]) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t n_s = qmp_sample_units(d.num_units);
+    const uint32_t stride = d.num_units / n_s;
+#pragma unroll
+    for (int i = 0; i < kQmpSamplePerWarp; ++i) {
+        const uint32_t sidx = warp + i * kQmpWarps;
+        const uint32_t u = sidx * stride + ((sidx * 2654435761u) >> 8) % stride;
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (sidx < n_s) v[i] = d.w_bf16 ? qmp_load_group<true>(d.W, u, lane) : qmp_load_group<false>(d.W, u, lane);
+    }
+}
+__device__ __forceinline__ float qmp_sample_finish(const QmpDesc& d, const float4 (&v)[kQmpSamplePerWarp], double* s_warp) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kQmpSamplePerWarp; ++i) acc += (fabsf(v[i].x) + fabsf(v[i].y)) + (fabsf(v[i].z) + fabsf(v[i].w));
+    const double total = qmp_block_sum(static_cast<double>(acc), s_warp);
+    return static_cast<float>(total / (static_cast<double>(qmp_sample_units(d.num_units)) * 128.0));
+}
+
+// gamma_est by ONE warp (the finisher, for matrices 1, 2, ... of a batch without hints): the first
 // kQmpSampleUnitsSmall of qmp_sample_gamma's scattered units, fetched by bulk copies into `buf` (a list that
 // is free at that moment) -- all of them in flight at once, one round trip instead of one per eight units.
 // The smaller sample gets the wider bracket (qmp_bracket_from, `wide`).  Returns a negative number if the
@@ -393,24 +418,27 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
     const unsigned long long gen0 = *reinterpret_cast<volatile unsigned long long*>(generation);
     const unsigned long long tag = qmp_tag(call_nonce, gen0);
 
-    // ---- the hints of matrices 0 and 1 are asked for first (4-byte reads that would otherwise queue behind
-    // the ring's first megabytes), then the loader fills the ring: the first stages travel while the
-    // brackets are made
-    float g01[2] = {0.0f, 0.0f};
-    bool hinted01[2];
-    hinted01[0] = qmp_hint(first, g01[0]);
-    hinted01[1] = count > 1 && qmp_hint(second, g01[1]);
+    // ---- What the first bracket needs is asked for BEFORE the loader fills the ring: the hints of matrices
+    // 0 and 1 (4-byte reads) or, without a usable hint, the sample of matrix 0 (all threads, one round
+    // trip).  Issued together with the ring's first copies they queue behind the 17 MB that the loaders of
+    // all CTAs ask for at the same moment (up to 3.5 us measured, and the CTA that is served last finishes
+    // last); so the loader waits for the hints to be there, or for the sample loads to be on their way.
+    float g01[2];                                            // both reads in flight before either is looked at
+    g01[0] = first.gamma_hint != nullptr ? *reinterpret_cast<const volatile float*>(first.gamma_hint) : 0.0f;
+    g01[1] = (count > 1 && second.gamma_hint != nullptr) ? *reinterpret_cast<const volatile float*>(second.gamma_hint) : 0.0f;
+    const bool hinted01[2] = {qmp_hint_usable(g01[0]), qmp_hint_usable(g01[1])};
+    float4 sample0[kQmpSamplePerWarp];
+    if (!hinted01[0]) qmp_sample_issue(first, sample0);
     QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u}, 0u};
     const bool is_loader = warp == kQmpLoaderWarp && lane == 0;
     if (is_loader) qmp_loader_issue(loader, batch, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
-
-    // ---- brackets of the first two matrices: all threads (the finisher makes the others, two matrices ahead)
-    for (int m = 0; m < min(count, 2); ++m) {
-        const QmpDesc& d = m == 0 ? first : second;
-        if (!hinted01[m]) g01[m] = d.w_bf16 ? qmp_sample_gamma<true>(d, s_warp) : qmp_sample_gamma<false>(d, s_warp);
-        if (threadIdx.x == 0) qmp_bracket_from(g01[m], d.num_units, hinted01[m], sh.bracket[m][0], sh.bracket[m][1]);
+    if (!hinted01[0]) g01[0] = qmp_sample_finish(first, sample0, s_warp);
+    if (threadIdx.x == 0) {
+        qmp_bracket_from(g01[0], first.num_units, hinted01[0], sh.bracket[0][0], sh.bracket[0][1]);
+        // matrix 1: from its hint here; without one the finisher samples it while matrix 0 streams
+        if (hinted01[1]) qmp_bracket_from(g01[1], second.num_units, true, sh.bracket[1][0], sh.bracket[1][1]);
+        sh.bracket_upto = hinted01[1] ? 2 : 1;
     }
-    if (threadIdx.x == 0) sh.bracket_upto = min(count, 2);
     __syncthreads();
 
     if (warp < kQmpStreamWarps) {
@@ -457,6 +485,21 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
         // ------------------------------------------------------------------ the finisher (warp 31)
         bool ok = true;
         uint32_t sample_phase = 0u;
+        if (count > 1 && !hinted01[1]) {
+            // bracket of matrix 1 from a sample into its own (still unused) list, while matrix 0 streams
+            const float g = qmp_sample_gamma_warp(second, lane, reinterpret_cast<unsigned char*>(s_list + 1 * kQmpStreamListCap),
+                                                  qmp_smem_u32(&sh.bar_sample), sample_phase, abort_flag);
+            if (g < 0.0f) {
+                ok = false;
+            } else {
+                if (lane == 0) {
+                    qmp_bracket_from(g, second.num_units, false, sh.bracket[1][0], sh.bracket[1][1], true);
+                    __threadfence_block();
+                    *reinterpret_cast<volatile int*>(&sh.bracket_upto) = 2;
+                }
+                __syncwarp();
+            }
+        }
         for (int m = 0; ok && m < count; ++m) {
             const int slot = m % kQmpLists;
             // bracket of matrix m + 2 from the caller's hint, well before the computing warps ask for it
