@@ -138,3 +138,28 @@ def test_backward_full_size(name, T, K, N):
     dX, dW = _gpu_backward(c)
     _assert_dw(c, dW)
     _assert_dx(c, dX)
+
+
+def test_backward_calls_back_to_back_on_one_workspace():
+    # With both gradients wanted the input-gradient GEMM starts before the weight-gradient GEMM has
+    # finished and only waits for it at its end.  Three calls in a row on one stream and one workspace, each
+    # followed at once (no synchronisation) by copies of its results and by the next call, which overwrites
+    # the operand copies in the workspace: every copy must hold that call's gradients.
+    T, N, K = 1100, 2560, 1280                      # several waves of tiles in both GEMMs
+    c = _case(T, N, K, seed=290)
+    rng = np.random.default_rng(291)
+    dys = [c["dy"]] + [inputs.f32_to_bf16_bits((rng.standard_normal((T, N)) * s).astype(np.float32)) for s in (0.5, 2.0)]
+    dY_dev = [bf16_dev(d) for d in dys]
+    ws = torch.empty(b.sbn_workspace_bytes(b.OP_BACKWARD, T, N, K), dtype=torch.uint8, device="cuda")
+    dX = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    p = c["g"]["dev"]
+    copies = []
+    for dY in dY_dev:
+        b.sbn_bitlinear_backward(dY, c["xq"], c["a_scale"], p["vals"], p["meta"], p["w_scale"], N, K, dX=dX, dW=dW, ws=ws)
+        copies.append((dX.clone(), dW.clone()))
+    b.sbn_check_status()
+    for dy, (dXc, dWc) in zip(dys, copies):
+        ci = dict(c, dy=dy)
+        _assert_dw(ci, dWc)
+        _assert_dx(ci, dXc)
