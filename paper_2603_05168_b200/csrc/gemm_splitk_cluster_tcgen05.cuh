@@ -334,7 +334,7 @@ bitlinear_gemm_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a,
         // all partial sums addressed to this CTA have landed (the barrier's phase completes with the
         // last byte; its completion makes the asynchronous stores visible to the waiting threads)
         if (!mbar_wait(bar_red, 0u, abort_flag)) ok = false;
-        ok = __all_sync(0xFFFFFFFFu, ok);                 // the loop below shuffles: one verdict per warp
+        ok = __all_sync(0xFFFFFFFFu, ok);                 // the loop below shuffles: one decision per warp
         // ------------------------------------------------------------------ epilogue, part 2: finish my tokens
         const int quarter = warp & 3;
         const int f = quarter * 32 + lane;
