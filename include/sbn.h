@@ -120,7 +120,11 @@ size_t sbn_workspace_bytes(int op, int T, int N, int K);
  *              concurrently.  It holds the per-CTA partial sums of |W| and a generation word that
  *              the kernel advances on every execution, so a call captured in a CUDA graph may be
  *              replayed on the same workspace (each replay tells its own partial sums from the
- *              previous replay's)
+ *              previous replay's).  The 2:4 kernel also leaves the scale it found there, tagged with
+ *              W and the shape: the next call for the same matrix on the same workspace starts from it
+ *              (as if it were a job's gamma_hint: no sample of the matrix, almost nothing to fix up) --
+ *              a speed-up for loops that re-pack the same buffers every step, never a change of the
+ *              result; bytes that do not carry the tag are ignored
  * Residency rule (this call, the _bf16, _batched and _static_ws forms alike).  The kernel is one
  * persistent grid of at most one CTA per SM (1024 threads each) whose CTAs exchange their partial
  * sums through the workspace, so ALL of its CTAs must be resident at the same time.  On a GPU that

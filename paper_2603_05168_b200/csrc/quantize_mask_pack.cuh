@@ -72,10 +72,24 @@ struct QmpSlot {                 // one per CTA, 16 B
     unsigned long long nonce;    // tag of the execution that wrote `partial`
     double partial;              // this CTA's sum |W|
 };
+// What a single-matrix call leaves behind for the next call on the same workspace: the scale it found,
+// tagged with the matrix it belongs to.  The next call on the same matrix (a training loop re-packs the
+// same buffers every step) takes it as its estimate of gamma -- no sample, a narrow bracket -- exactly as
+// if the caller had passed it as a hint; anything else in these bytes (an uninitialised workspace, another
+// matrix) fails the tag and is ignored.
+struct __align__(16) QmpMemo {
+    unsigned long long magic;
+    const void* W;
+    uint32_t num_units;
+    float scale;
+};
+constexpr unsigned long long kQmpMemoMagic = 0x71A93C5E2D84B6F1ull;
 struct QmpWorkspace {            // layout of the caller's workspace
     QmpSlot slot[kQmpMaxCtas];
     unsigned long long generation;   // advanced by one per execution on this workspace (any start value)
     unsigned long long pad_;
+    QmpMemo memo;
+    unsigned long long pad2_;
 };
 // Tag of one execution: the call's nonce (low word, never 0) under the workspace's generation.
 __device__ __forceinline__ unsigned long long qmp_tag(unsigned long long nonce, unsigned long long generation) {

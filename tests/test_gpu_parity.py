@@ -1147,3 +1147,35 @@ def test_quantize_mask_pack_batch_longer_than_one_launch_holds():
         vals, meta = gpu_unpack_canonical(dict(vals=big["vals"][i], meta=big["meta"][i]), 128, 128)
         assert np.float32(big["w_scale"][i].cpu().numpy()[0]) == r["scale"], i
         assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"]), i
+
+
+def test_quantize_mask_pack_scale_left_in_the_workspace_never_changes_the_result():
+    # A single-matrix call leaves its scale in the workspace, tagged with W and the shape, and the next call
+    # for the same buffer on the same workspace starts from it.  Same buffer with weights of another scale,
+    # another buffer of the same shape, the same call again, a workspace full of noise: always the oracle's bits.
+    N, K = 640, 2560
+    Wa = inputs.latent_weights(N, K, seed=410)
+    Wb = inputs.latent_weights(N, K, seed=411, sigma=0.31)          # 15 x the scale: the estimate is useless
+    Wc = inputs.perturb_weights(Wa, seed=412, sigma=1e-4)           # a training step later: the estimate is good
+    refs = {k: _oracle_pack(w) for k, w in (("a", Wa), ("b", Wb), ("c", Wc))}
+    buf = dev(Wa)
+    other = dev(Wb)
+    bufs = b.alloc_packed(N, K)
+
+    def run_and_check(W_dev, r):
+        b.sbn_quantize_mask_pack(W_dev, bufs["vals"], bufs["meta"], bufs["w_scale"], bufs["ws"])
+        b.sbn_check_status()
+        vals, meta = gpu_unpack_canonical(bufs, N, K)
+        assert np.float32(bufs["w_scale"].cpu().numpy()[0]) == r["scale"]
+        assert np.array_equal(vals, r["vals"]) and np.array_equal(meta, r["meta"])
+
+    bufs["ws"].copy_(torch.randint(0, 256, bufs["ws"].shape, dtype=torch.uint8, device="cuda"))    # noise: no tag
+    run_and_check(buf, refs["a"])
+    run_and_check(buf, refs["a"])                   # the same matrix again: starts from its own scale
+    buf.copy_(torch.from_numpy(Wc).cuda())
+    run_and_check(buf, refs["c"])                   # a step later: a good estimate
+    buf.copy_(torch.from_numpy(Wb).cuda())
+    run_and_check(buf, refs["b"])                   # same buffer, another scale: the estimate misses
+    run_and_check(other, refs["b"])                 # another buffer: the tag does not match
+    buf.copy_(torch.from_numpy(Wa).cuda())
+    run_and_check(buf, refs["a"])
