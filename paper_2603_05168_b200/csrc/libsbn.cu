@@ -659,7 +659,8 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
         const int n_here = std::min(kQmpMaxBatch, count - lo);
         uint32_t max_units = 0;
         for (int i = 0; i < n_here; ++i) max_units = std::max(max_units, descs[static_cast<size_t>(lo + i)].num_units);
-        for (int at = 1; at < n_here; at += kQmpDescChunk) {
+        // batches of up to kQmpInlineDescs matrices travel in the kernel's parameters: nothing to store first
+        for (int at = 1; n_here > kQmpInlineDescs && at < n_here; at += kQmpDescChunk) {
             QmpDescChunk chunk;
             const int n = std::min(kQmpDescChunk, n_here - at);
             for (int i = 0; i < n; ++i) chunk.d[i] = descs[static_cast<size_t>(lo + at + i)];
@@ -668,8 +669,7 @@ sbn_status sbn_quantize_mask_pack_batched(int count, const sbn_pack_job* jobs, v
             ++g_launch_count;
             if (err != cudaSuccess) return SBN_ERR_CUDA;
         }
-        const sbn_status st = launch_quantize_mask_pack_stream(descs[static_cast<size_t>(lo)], descs[static_cast<size_t>(lo + (n_here > 1 ? 1 : 0))], descs_dev + lo,
-                                                               n_here, max_units,
+        const sbn_status st = launch_quantize_mask_pack_stream(descs.data() + lo, descs_dev + lo, n_here, max_units,
                                                                slots + static_cast<size_t>(lo) * kQmpMaxCtas, generation, s);
         if (st != SBN_OK) return st;
     }

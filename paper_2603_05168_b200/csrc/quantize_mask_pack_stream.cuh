@@ -127,14 +127,18 @@ struct QmpRing {
     __device__ __forceinline__ void advance() { ++used; }
 };
 
-// Matrix m of the batch: 0 and 1 travel with the launch, `rest` holds 1, 2, ... in global memory.
+// Matrix m of the batch: the first kQmpInlineDescs travel with the launch (kernel parameters: a batch
+// that small needs no kernel that stores its descriptors first), `rest` holds 1, 2, ... in global memory.
+constexpr int kQmpInlineDescs = 8;
+struct QmpInlineDescs {
+    QmpDesc d[kQmpInlineDescs];
+};
 struct QmpBatch {
-    const QmpDesc& first;
-    const QmpDesc& second;
+    const QmpInlineDescs& inl;
     const QmpDesc* rest;
 };
 __device__ __forceinline__ QmpDesc qmp_desc_of(const QmpBatch& b, int m) {
-    return m == 0 ? b.first : (m == 1 ? b.second : b.rest[m - 1]);
+    return m < kQmpInlineDescs ? b.inl.d[m] : b.rest[m - 1];
 }
 
 // Bounded wait for a shared-memory word (written by another warp of this CTA) to reach `want`.
@@ -382,7 +386,7 @@ __device__ __forceinline__ bool qmp_bracket_holds(const QmpDesc& d, float thr, f
 }
 
 __global__ void __launch_bounds__(kQmpThreads, 1)
-quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, const QmpDesc* __restrict__ rest, int count,
+quantize_mask_pack_stream_kernel(const __grid_constant__ QmpInlineDescs inl, const QmpDesc* __restrict__ rest, int count,
                                  QmpSlot* slots, unsigned long long* generation, unsigned long long call_nonce,
                                  int test_withhold_slot, QmpMemo* memo) {
     extern __shared__ __align__(128) unsigned char s_dyn[];   // [kQmpStages][kQmpStageBytes] ring, then [kQmpLists][kQmpStreamListCap] entries
@@ -390,7 +394,9 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
     __shared__ QmpStreamShared sh;
     __shared__ double s_warp[kQmpWarps];
 
-    const QmpBatch batch{first, second, rest};
+    const QmpBatch batch{inl, rest};
+    const QmpDesc& first = inl.d[0];
+    const QmpDesc& second = inl.d[1];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     volatile int* const abort_flag = &sh.abort;
@@ -733,11 +739,13 @@ quantize_mask_pack_stream_kernel(const QmpDesc first, const QmpDesc second, cons
     }
 }
 
-// Launch for `count` (<= kQmpMaxBatch) matrices: matrices 0 and 1 by value (`second` is ignored when count is 1),
-// matrices 1, 2, ... already copied to `rest_dev`.
-inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const QmpDesc& second, const QmpDesc* rest_dev, int count,
+// Launch for `count` (<= kQmpMaxBatch) matrices: the first kQmpInlineDescs of `descs_host` by value, matrices
+// 1, 2, ... already copied to `rest_dev` if there are more than that.
+inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc* descs_host, const QmpDesc* rest_dev, int count,
                                                    uint32_t max_units, QmpSlot* slots, unsigned long long* generation,
                                                    cudaStream_t stream, QmpMemo* memo = nullptr) {
+    QmpInlineDescs inl;
+    for (int i = 0; i < kQmpInlineDescs; ++i) inl.d[i] = descs_host[i < count ? i : 0];
     const int test_withhold_slot = g_test_break_waits;
     const unsigned long long nonce = qmp_next_nonce();
     // every CTA must be resident at once (they exchange partial sums): never more CTAs than this
@@ -749,7 +757,7 @@ inline sbn_status launch_quantize_mask_pack_stream(const QmpDesc& first, const Q
     // of them become resident as soon as the SMs are free and the exchange cannot deadlock; if
     // another kernel kept SMs busy for seconds, the bounded wait reports SBN_ERR_TIMEOUT instead.
     const cudaError_t err = launch_kernel(quantize_mask_pack_stream_kernel, dim3(grid), dim3(kQmpThreads), kQmpStreamSmemBytes, stream,
-                                          first, second, rest_dev, count, slots, generation, nonce, test_withhold_slot, count == 1 ? memo : nullptr);
+                                          inl, rest_dev, count, slots, generation, nonce, test_withhold_slot, count == 1 ? memo : nullptr);
     ++g_launch_count;
     return err == cudaSuccess ? SBN_OK : SBN_ERR_CUDA;
 }
@@ -760,7 +768,7 @@ inline sbn_status launch_quantize_mask_pack(const void* W, bool w_bf16, int N, i
                                             unsigned long long* flip_bits, QmpWorkspace* ws,
                                             cudaStream_t stream) {
     const QmpDesc d = qmp_make_desc(W, w_bf16, N, K, vals, meta, w_scale, dense_q, prev_meta, flip_bits);
-    return launch_quantize_mask_pack_stream(d, d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream, &ws->memo);
+    return launch_quantize_mask_pack_stream(&d, nullptr, 1, d.num_units, ws->slot, &ws->generation, stream, &ws->memo);
 }
 
 }  // namespace sbn
