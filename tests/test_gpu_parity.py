@@ -617,6 +617,38 @@ def test_gemm_parity(sparse, T, N, K):
     _assert_y(y_to_f32_numpy(y), y_ref)
 
 
+def _random_gemm_shapes(count, seed):
+    """Seeded shapes across the dispatcher's regimes (few tokens: single-CTA tiles, split K in clusters;
+    hundreds to thousands of tokens: CTA pairs with one or two M-tiles), sized for the CPU oracle."""
+    import random
+    rng = random.Random(seed)
+    Ts = [1, 3, 8, 17, 31, 64, 100, 200, 255, 300, 511, 777, 1024, 1500, 2048]
+    Ns = [128, 256, 384, 640, 1024, 2560]
+    Ks = [128, 256, 384, 1280, 2560, 6912]
+    out = []
+    while len(out) < count:
+        T, N, K = rng.choice(Ts), rng.choice(Ns), rng.choice(Ks)
+        if T * N * K <= 6e8 and (T, N, K) not in out:
+            out.append((T, N, K))
+    return out
+
+
+@pytest.mark.parametrize("T,N,K", _random_gemm_shapes(16, seed=20260306))
+def test_gemm_parity_random_shapes_with_the_plan_the_library_picks(T, N, K):
+    # whatever kernel and tile the dispatcher chooses for the shape: accumulators exact, outputs within tolerance
+    # (fp32 out with the accumulator dump, then bf16 out alone: the register-packed epilogue of the pair kernel)
+    r, xq_ref, s_ref, g, xq, a_scale = _layer_case(T, N, K, seed=3 * T + 5 * N + 7 * K)
+    y_ref, acc_ref = oracle.sparse_bitlinear(xq_ref, s_ref, r["vals"], r["meta"], r["scale"])
+    y, acc = gpu_gemm(True, xq, a_scale, g["dev"])
+    assert np.array_equal(acc.cpu().numpy(), acc_ref)
+    _assert_y(y_to_f32_numpy(y), y_ref)
+    yb, _ = gpu_gemm(True, xq, a_scale, g["dev"], out_dtype=torch.bfloat16, want_acc=False)
+    ref_bits = oracle.f32_to_bf16_bits(y_ref).astype(np.int32)
+    got_bits = bf16_tensor_bits(yb).astype(np.int32)
+    # same sign assumed (values are not within one ulp of zero); 1 ulp = 1 step of the pattern
+    assert np.abs(got_bits - ref_bits).max() <= 1
+
+
 @pytest.mark.parametrize("sparse", [True, False])
 @pytest.mark.parametrize("tile", [64, 128, 256])
 def test_gemm_parity_every_token_tile(sparse, tile):
