@@ -113,6 +113,18 @@ __device__ __forceinline__ void qmp_bulk_load(uint32_t smem_dst, const void* gme
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
 }
+// The same for data that is read once (the master weights of pass 1): the lines are the first to leave the
+// L2 again, so the stream does not push out what the kernels after this one will read (the packed weights
+// this kernel writes, the activations).
+__device__ __forceinline__ unsigned long long qmp_policy_evict_first() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void qmp_bulk_load_once(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t bar, unsigned long long policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ float4 qmp_lds128(uint32_t addr) {
     float4 v;
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -258,6 +270,7 @@ struct QmpLoader {
     bool open;
     QmpRing ring;
     uint32_t issued;             // copies of this launch (the drain after an abort needs it)
+    unsigned long long policy;   // L2 policy of the copies: read once
 };
 __device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpBatch& batch, int count, uint32_t max_copies,
                                                  uint32_t ring_base, uint32_t bar_full0, uint32_t bar_empty0, volatile int* abort_flag) {
@@ -277,7 +290,8 @@ __device__ __forceinline__ bool qmp_loader_issue(QmpLoader& L, const QmpBatch& b
         if (!qmp_mbar_wait(bar_empty0 + 8u * L.ring.stage(), L.ring.phase() ^ 1u, abort_flag)) return false;
         const uint32_t bytes = min(L.u_end - L.u, static_cast<uint32_t>(kQmpStageUnits)) * L.unit_bytes;
         qmp_mbar_expect_tx(bar_full0 + 8u * L.ring.stage(), bytes);
-        qmp_bulk_load(ring_base + L.ring.stage() * kQmpStageBytes, L.W + static_cast<size_t>(L.u) * L.unit_bytes, bytes, bar_full0 + 8u * L.ring.stage());
+        qmp_bulk_load_once(ring_base + L.ring.stage() * kQmpStageBytes, L.W + static_cast<size_t>(L.u) * L.unit_bytes, bytes, bar_full0 + 8u * L.ring.stage(),
+                           L.policy);
         ++L.issued;
         L.ring.advance();
         L.u += kQmpStageUnits;
@@ -445,7 +459,7 @@ quantize_mask_pack_stream_kernel(const __grid_constant__ QmpInlineDescs inl, con
     const bool hinted01[2] = {qmp_hint_usable(g01[0]), qmp_hint_usable(g01[1])};
     float4 sample0[kQmpSamplePerWarp];
     if (!hinted01[0]) qmp_sample_issue(first, sample0);
-    QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u}, 0u};
+    QmpLoader loader{0, 0u, 0u, 0u, nullptr, false, QmpRing{0u}, 0u, qmp_policy_evict_first()};
     const bool is_loader = warp == kQmpLoaderWarp && lane == 0;
     if (is_loader) qmp_loader_issue(loader, batch, count, kQmpStages, ring_base, bar_full0, bar_empty0, abort_flag);
     if (!hinted01[0]) g01[0] = qmp_sample_finish(first, sample0, s_warp);
