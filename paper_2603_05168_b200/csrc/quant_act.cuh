@@ -118,14 +118,14 @@ quant_act_kernel(const uint4* __restrict__ x, int T, int nvec, uint2* __restrict
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int idx = g + i * G;
-        cur[i] = (row < T && idx < nvec) ? __ldg(x + static_cast<size_t>(row) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
+        cur[i] = (row < T && idx < nvec) ? __ldcs(x + static_cast<size_t>(row) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
     }
     for (int it = 0; it < iters; ++it, row += row_stride) {
         const int row_n = row + row_stride;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = g + i * G;
-            nxt[i] = (row_n < T && idx < nvec) ? __ldg(x + static_cast<size_t>(row_n) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
+            nxt[i] = (row_n < T && idx < nvec) ? __ldcs(x + static_cast<size_t>(row_n) * nvec + idx) : make_uint4(0u, 0u, 0u, 0u);
         }
         uint32_t pm = 0u;
 #pragma unroll
